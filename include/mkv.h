@@ -1,0 +1,215 @@
+/*
+ * mkv.h -- C ABI of libmkv: mixed-format (FP8 + TQ3) paged KV cache and decode attention for
+ * NVIDIA B200 (sm_100a), after the Minima-KV paper.
+ *
+ * One pool holds the KV pages of ONE attention layer in two physical stores (Section 4.1,
+ * "Physical stores and decode dispatch"): an FP8 arena for Recent and Anchor pages and a TQ3
+ * arena for Stale pages.  A request's logical cache is a row of a block table; every entry
+ * carries a tier tag that selects the arena and a physical page id inside it (Section 3.1:
+ * z_p in {R, A, S}).  Decode attention walks that single table in one pass and merges the FP8
+ * and TQ3 tokens under one softmax (Section 3.3, Eq. softmax-merge); no dequantised copy of the
+ * cache is ever built.
+ *
+ * Conventions
+ *   - page = 16 tokens; head_dim d in {128, 256}; query head h reads KV head h / (n_q/n_kv);
+ *     at most 8 query heads per KV head.
+ *   - "device" pointers are CUDA device memory owned by the caller, 16-byte aligned (arenas and
+ *     workspace 256-byte aligned); "host" pointers are ordinary host memory.  The library
+ *     allocates no device memory: the caller hands it arenas and workspace.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = legacy default stream).  Calls that take
+ *     a stream only enqueue work and never synchronise with the host unless stated.
+ *   - every function returns 0 (MKV_OK) or a negative mkv_status; no exceptions cross the ABI.
+ *     Host-detectable misuse (bad sizes, null pointers, unaligned pointers, unsupported shapes)
+ *     returns MKV_E_INVALID without launching anything.  Out-of-range page ids or tags met ON
+ *     THE DEVICE never fault: the kernel skips the access and records the event in the pool's
+ *     status word, read with mkv_pool_status().
+ *   - bf16 / fp16 / e4m3 data are passed as raw 16- / 8-bit words.
+ *
+ * Record formats (per page and KV head), little endian:
+ *   FP8 record, 32*d bytes:   K e4m3 [16 tokens][d], then V e4m3 [d channels][16 tokens].
+ *     stored = e4m3(x / scale) rounded to nearest even, saturating at +-448.
+ *   TQ3 record, 16*d + 32 bytes (Section 4.1: three-bit rotated key codes, FP16 key-norm
+ *     correction, three-bit value codes, FP16 scale/zero):
+ *       [0, 6d)   key codes,   [6d, 12d) value codes,   [12d, 12d+32) norm correction g[16],
+ *       [12d+32, 16d+32) value scale/zero.  Bit positions are those of the tensor-core
+ *     fragment that consumes them; mkv_page_read_raw() returns the bytes as stored.
+ */
+#ifndef MKV_H_
+#define MKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mkv_pool mkv_pool;
+typedef struct mkv_seq mkv_seq;
+
+typedef enum {
+    MKV_OK = 0,
+    MKV_E_INVALID = -1,  /* bad argument (null, size, alignment, unsupported geometry)          */
+    MKV_E_OOM_FP8 = -2,  /* FP8 arena has no free page                                          */
+    MKV_E_OOM_TQ3 = -3,  /* TQ3 arena has no free page                                          */
+    MKV_E_STATE = -4,    /* transition not allowed from the page's current tier / double free   */
+    MKV_E_BOUNDS = -5,   /* page id, slot or logical page out of range                          */
+    MKV_E_CUDA = -6,     /* a CUDA runtime call failed (see mkv_last_cuda_error)                */
+    MKV_E_TIMEOUT = -7   /* a bounded device-side wait gave up                                  */
+} mkv_status;
+
+enum { MKV_TAG_RECENT = 0, MKV_TAG_ANCHOR = 1, MKV_TAG_STALE = 2 };
+enum { MKV_FMT_FP8 = 0, MKV_FMT_TQ3 = 1 };
+/* decode kernels: the tensor-core kernel is the product; the CUDA-core kernel computes the same
+ * thing with scalar FMAs and exists so that the choice of tensor cores can be measured */
+enum { MKV_DECODE_TENSOR = 0, MKV_DECODE_SCALAR = 1 };
+
+typedef struct {
+    int32_t page_size;          /* must be 16                                                   */
+    int32_t head_dim;           /* 128 or 256                                                   */
+    int32_t n_kv_heads;
+    int32_t n_q_heads;          /* multiple of n_kv_heads, at most 8 per KV head                */
+    int32_t fp8_pages;          /* capacity of the FP8 arena (Recent + Anchor), in pages        */
+    int32_t tq3_pages;          /* capacity of the TQ3 arena (Stale), in pages                  */
+    float k_scale;              /* FP8 key scale   (dequantised = stored * scale); 1.0 typical  */
+    float v_scale;              /* FP8 value scale                                              */
+    const int8_t* k_rot_signs;  /* host, head_dim entries of +1/-1: diagonal of the randomised  */
+                                /* Hadamard rotation applied to keys before 3-bit quantisation  */
+} mkv_pool_config;
+
+typedef struct {
+    int64_t fp8_pages_total, fp8_pages_used, tq3_pages_total, tq3_pages_used;
+    int64_t fp8_bytes_used, tq3_bytes_used;   /* physical bytes of used pages (all KV heads)     */
+    int64_t bf16_bytes_equivalent;            /* the same pages held as BF16                     */
+} mkv_stats;
+
+/* ---- pool -------------------------------------------------------------------------------- */
+
+/* Bytes the caller must allocate for the two arenas (Section 4.1: FP8 store and TQ3 side store).
+ * fp8_bytes includes a 256-byte tail that holds the pool's device status word. */
+int32_t mkv_pool_query(const mkv_pool_config* cfg, size_t* fp8_arena_bytes, size_t* tq3_arena_bytes);
+
+/* Workspace for mkv_decode_attention with up to max_batch requests: split partials (m, l, O)
+ * (Section 3.3) plus merge tickets.  Independent of sequence lengths. */
+int32_t mkv_decode_workspace_bytes(const mkv_pool_config* cfg, int32_t max_batch, size_t* bytes);
+
+/* Zero the ticket header of a workspace.  Must be enqueued once before the first decode call that
+ * uses the buffer; decode leaves the header zero again when it completes. */
+int32_t mkv_workspace_init(void* workspace_dev, size_t bytes, void* stream);
+
+/* Create a pool over caller-owned arenas.  Zero-fills both arenas (so that never-written slots
+ * decode to zeros, not NaN) and synchronises `stream` before returning.  The pool owns host
+ * bookkeeping only; the arenas stay the caller's and must outlive the pool. */
+int32_t mkv_pool_create(const mkv_pool_config* cfg, void* fp8_arena_dev, void* tq3_arena_dev,
+                        void* stream, mkv_pool** out);
+/* Bookkeeping-only pool (no arenas, no device): free lists, sequence rows and statistics work;
+ * every call that would touch the device returns MKV_E_INVALID.  For schedulers that plan page
+ * transitions in a process without a GPU. */
+int32_t mkv_pool_create_host_only(const mkv_pool_config* cfg, mkv_pool** out);
+int32_t mkv_pool_destroy(mkv_pool* pool);
+
+/* Per-format free lists (Section 4.4: "per-kind free list").  ids is a host array of n entries.
+ * alloc: all-or-nothing; MKV_E_OOM_* leaves the lists untouched.  A fresh list hands out
+ * 0, 1, 2, ...; a freed id is reused first.  free: MKV_E_BOUNDS for a bad id, MKV_E_STATE for a
+ * page that is not allocated; nothing is freed in either case. */
+int32_t mkv_page_alloc(mkv_pool* pool, int32_t fmt, int32_t* ids_host, int32_t n);
+int32_t mkv_page_free(mkv_pool* pool, int32_t fmt, const int32_t* ids_host, int32_t n);
+
+/* Physical-byte counter of the pool (Section 6.3 "active-cache counter"). */
+int32_t mkv_pool_stats(const mkv_pool* pool, mkv_stats* out);
+
+/* Read and clear the device status word; synchronises `stream`.  Returns MKV_OK, or
+ * MKV_E_BOUNDS / MKV_E_STATE / MKV_E_TIMEOUT if a kernel since the last call met an out-of-range
+ * id or tag, a forbidden tier transition, or a wait that ran out. */
+int32_t mkv_pool_status(mkv_pool* pool, void* stream);
+
+/* Select the decode kernel (MKV_DECODE_TENSOR by default). */
+int32_t mkv_pool_set_decode_variant(mkv_pool* pool, int32_t variant);
+
+/* Test hooks: copy one page (all KV heads; n_kv_heads * record bytes) between the arena and a
+ * host buffer, synchronously.  Lets a test compare packed bytes with a reference encoder, or
+ * install pages encoded elsewhere. */
+int32_t mkv_page_read_raw(mkv_pool* pool, int32_t fmt, int32_t id, void* host_buf, void* stream);
+int32_t mkv_page_write_raw(mkv_pool* pool, int32_t fmt, int32_t id, const void* host_buf, void* stream);
+
+const char* mkv_last_cuda_error(void);
+
+/* ---- hot path ---------------------------------------------------------------------------- */
+
+/* Append (Algorithm 1 step 1, Section 3.1 "Recent"): write the K and V of n_tokens new tokens
+ * into FP8 pages as e4m3.
+ *   k, v          device, bf16 [n_tokens][n_kv_heads][d]
+ *   slot_mapping  device, int32 [n_tokens]: page_id * 16 + slot in the FP8 arena; negative =
+ *                 skip the token.  An id beyond the arena is skipped and flagged (MKV_E_BOUNDS).
+ * The caller publishes the page in the block table (tag MKV_TAG_RECENT) when it opens it. */
+int32_t mkv_append(mkv_pool* pool, const void* k_dev, const void* v_dev, const int32_t* slot_mapping_dev,
+                   int32_t n_tokens, void* stream);
+
+/* Demote / Retier(p, TQ3) (Algorithm 1 step 2; Section 4, "normalize-rotate-pack"): encode
+ * n_pages full FP8 pages (all KV heads) into TQ3 pages, then publish.
+ *   src_fp8_ids, dst_tq3_ids   device, int32 [n_pages]
+ *   block_table, tier_tag      device tables to publish into, or NULL
+ *   entry_index                device, int64 [n_pages]: flat index of each page's entry in the two
+ *                              tables (negative = do not publish), or NULL
+ * For every page the TQ3 record is complete and fenced before its id and MKV_TAG_STALE are
+ * written (copy-before-publish).  The FP8 source is not modified; return it to its free list with
+ * mkv_page_free() once every reader enqueued before this call has been ordered before the next
+ * writer (same-stream order suffices).  Key encoder: sign flip, Walsh-Hadamard, 3-bit Lloyd-Max
+ * codes of the normalised coordinates, fp16 norm correction |x|/|c|.  Value encoder: per channel
+ * over the page's 16 tokens, asymmetric 3-bit codes with fp16 scale and zero. */
+int32_t mkv_demote(mkv_pool* pool, const int32_t* src_fp8_ids_dev, const int32_t* dst_tq3_ids_dev,
+                   int32_t n_pages, int32_t* block_table_dev, uint8_t* tier_tag_dev,
+                   const int64_t* entry_index_dev, void* stream);
+
+/* Protect / unprotect (Fig. lifecycle: Recent -> Anchor): set the tag of one table entry to
+ * MKV_TAG_ANCHOR (flag != 0) or MKV_TAG_RECENT (flag == 0).  No data moves.  If the entry is
+ * Stale the tag is left alone and MKV_E_STATE is recorded in the status word (a Stale page must
+ * be promoted into a new FP8 page first). */
+int32_t mkv_set_anchor(mkv_pool* pool, uint8_t* tier_tag_dev, int64_t entry_index, int32_t flag, void* stream);
+
+/* Decode attention (Section 3.3; Section 4.1 "fused decode path"): for every request b and query
+ * head h, softmax(scale * q K^T) V over the seq_lens[b] tokens of row b, where each page is read
+ * in its own physical format and all tokens share one softmax normalisation.
+ *   q            device, bf16 [B][n_q_heads][d]
+ *   block_table  device, int32 [B][max_pages]; unused entries are ignored
+ *   tier_tag     device, uint8 [B][max_pages]; 0/1 = FP8 arena, 2 = TQ3 arena
+ *   seq_lens     device, int32 [B]; pages beyond ceil(len/16) are not read; the last page may be
+ *                partial (FP8 only); len == 0 gives out = 0 and lse = -inf
+ *   out          device, fp32 [B][n_q_heads][d]
+ *   lse          device, fp32 [B][n_q_heads] natural-log-sum-exp of the scaled scores, or NULL
+ *   workspace    device, at least mkv_decode_workspace_bytes(cfg, B) bytes, initialised once with
+ *                mkv_workspace_init(); two decode calls that overlap on the GPU need two buffers
+ * One launch: a split-KV kernel whose last-arriving block per (request, KV head) merges the split
+ * partials with Eq. (softmax-merge).  No host synchronisation. */
+int32_t mkv_decode_attention(mkv_pool* pool, const void* q_dev, const int32_t* block_table_dev,
+                             const uint8_t* tier_tag_dev, const int32_t* seq_lens_dev, int32_t B,
+                             int32_t max_pages, float scale, float* out_dev, float* lse_dev,
+                             void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/* ---- host-side sequence bookkeeping (Algorithm 1; no device work) ------------------------- */
+
+/* A sequence owns a row of logical pages -> (tag, physical id).  These calls only plan: they
+ * move ids between the free lists and the row and tell the caller which device call to issue. */
+int32_t mkv_seq_create(mkv_pool* pool, mkv_seq** out);
+/* Finish(q): release every page of the sequence to its free list and destroy the handle. */
+int32_t mkv_seq_finish(mkv_seq* seq);
+/* Append: slot for the next token; opens a Recent page every 16 tokens (MKV_E_OOM_FP8 if none). */
+int32_t mkv_seq_append(mkv_seq* seq, int32_t* page_id, int32_t* slot, int32_t* opened_page);
+/* Recent <-> Anchor tag of a logical page (MKV_E_STATE if it is Stale). */
+int32_t mkv_seq_protect(mkv_seq* seq, int32_t logical_page, int32_t flag);
+/* Retier to TQ3: allocates the destination, updates the row, releases the source id.  Only full,
+ * non-Stale pages qualify (MKV_E_STATE otherwise).  The caller then enqueues mkv_demote(). */
+int32_t mkv_seq_demote(mkv_seq* seq, int32_t logical_page, int32_t* src_fp8_id, int32_t* dst_tq3_id);
+/* Age: plan the demotion of every full Recent page wholly before the last `recent_tokens`
+ * tokens.  Writes up to `cap` triples and returns their number in *n (MKV_E_INVALID if more
+ * would be needed; nothing changes then). */
+int32_t mkv_seq_age(mkv_seq* seq, int32_t recent_tokens, int32_t* logical_pages, int32_t* src_fp8_ids,
+                    int32_t* dst_tq3_ids, int32_t cap, int32_t* n);
+int32_t mkv_seq_len(const mkv_seq* seq, int32_t* len, int32_t* n_pages);
+/* Copy the row (n_pages entries) to host arrays. */
+int32_t mkv_seq_row(const mkv_seq* seq, int32_t* ids_host, uint8_t* tags_host, int32_t cap);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MKV_H_ */

@@ -1,0 +1,422 @@
+// Host side of libmkv: pool bookkeeping, per-format free lists, sequence rows (Algorithm 1),
+// argument validation and the C ABI entry points.  No arithmetic of the method lives here.
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+
+#include "mkv_internal.cuh"
+
+namespace mkv {
+
+static thread_local std::string g_last_error;
+
+int32_t cuda_fail(cudaError_t e, const char* what)
+{
+    g_last_error = std::string(what) + ": " + cudaGetErrorString(e);
+    return MKV_E_CUDA;
+}
+
+static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+static int32_t check_cfg(const mkv_pool_config* c)
+{
+    if (!c) return MKV_E_INVALID;
+    if (c->page_size != kPage) return MKV_E_INVALID;
+    if (c->head_dim != 128 && c->head_dim != 256) return MKV_E_INVALID;
+    if (c->n_kv_heads < 1 || c->n_q_heads < c->n_kv_heads) return MKV_E_INVALID;
+    if (c->n_q_heads % c->n_kv_heads) return MKV_E_INVALID;
+    if (c->n_q_heads / c->n_kv_heads > kMaxGroup) return MKV_E_INVALID;
+    if (c->fp8_pages < 0 || c->tq3_pages < 0) return MKV_E_INVALID;
+    if (!(c->k_scale > 0.f) || !(c->v_scale > 0.f)) return MKV_E_INVALID;
+    return MKV_OK;
+}
+
+size_t decode_ws_header_bytes(int B, int hkv)
+{
+    size_t b = 256 + sizeof(uint32_t) * (size_t)B * hkv;
+    return (b + 255) / 256 * 256;
+}
+
+}  // namespace mkv
+
+using namespace mkv;
+
+extern "C" {
+
+const char* mkv_last_cuda_error(void) { return g_last_error.c_str(); }
+
+int32_t mkv_pool_query(const mkv_pool_config* cfg, size_t* fp8_bytes, size_t* tq3_bytes)
+{
+    int32_t rc = check_cfg(cfg);
+    if (rc) return rc;
+    if (!fp8_bytes || !tq3_bytes) return MKV_E_INVALID;
+    *fp8_bytes = (size_t)cfg->fp8_pages * cfg->n_kv_heads * fp8_record_bytes(cfg->head_dim) + kStatusTail;
+    *tq3_bytes = (size_t)cfg->tq3_pages * cfg->n_kv_heads * tq3_record_bytes(cfg->head_dim);
+    if (*tq3_bytes == 0) *tq3_bytes = 256;
+    return MKV_OK;
+}
+
+int32_t mkv_decode_workspace_bytes(const mkv_pool_config* cfg, int32_t max_batch, size_t* bytes)
+{
+    int32_t rc = check_cfg(cfg);
+    if (rc) return rc;
+    if (!bytes || max_batch < 1) return MKV_E_INVALID;
+    int group = cfg->n_q_heads / cfg->n_kv_heads;
+    size_t a = decode_ws_scalar_bytes(max_batch, cfg->n_kv_heads, group, cfg->head_dim);
+    size_t b = decode_ws_tensor_bytes(max_batch, cfg->n_kv_heads, group, cfg->head_dim);
+    *bytes = decode_ws_header_bytes(max_batch, cfg->n_kv_heads) + (a > b ? a : b);
+    return MKV_OK;
+}
+
+int32_t mkv_workspace_init(void* ws, size_t bytes, void* stream)
+{
+    if (!ws || bytes < 256 || !aligned(ws, 256)) return MKV_E_INVALID;
+    // tickets live in the header; partial slots need no initialisation
+    MKV_CUDA(cudaMemsetAsync(ws, 0, bytes, (cudaStream_t)stream));
+    return MKV_OK;
+}
+
+static mkv_pool* new_pool(const mkv_pool_config* cfg, void* fp8_arena, void* tq3_arena);
+
+int32_t mkv_pool_create_host_only(const mkv_pool_config* cfg, mkv_pool** out)
+{
+    int32_t rc = check_cfg(cfg);
+    if (rc) return rc;
+    if (!out) return MKV_E_INVALID;
+    mkv_pool* p = new_pool(cfg, nullptr, nullptr);
+    if (!p) return MKV_E_INVALID;
+    *out = p;
+    return MKV_OK;
+}
+
+static mkv_pool* new_pool(const mkv_pool_config* cfg, void* fp8_arena, void* tq3_arena)
+{
+    mkv_pool* p = new (std::nothrow) mkv_pool();
+    if (!p) return nullptr;
+    p->cfg = *cfg;
+    p->cfg.k_rot_signs = nullptr;
+    p->d = cfg->head_dim;
+    p->hkv = cfg->n_kv_heads;
+    p->hq = cfg->n_q_heads;
+    p->group = cfg->n_q_heads / cfg->n_kv_heads;
+    p->fp8 = static_cast<uint8_t*>(fp8_arena);
+    p->tq3 = static_cast<uint8_t*>(tq3_arena);
+    p->variant = MKV_DECODE_TENSOR;
+    std::memset(&p->sigma, 0, sizeof p->sigma);
+    for (int i = 0; cfg->k_rot_signs && i < cfg->head_dim; ++i)
+        if (cfg->k_rot_signs[i] < 0) p->sigma.w[i >> 5] |= 1u << (i & 31);
+    for (int f = 0; f < 2; ++f) {
+        int n = f == MKV_FMT_FP8 ? cfg->fp8_pages : cfg->tq3_pages;
+        p->free_list[f].reserve(n);
+        for (int i = n - 1; i >= 0; --i) p->free_list[f].push_back(i);   // pops 0, 1, 2, ...
+        p->allocated[f].assign(n, 0);
+    }
+    p->status_dev = nullptr;
+    p->device = -1;
+    return p;
+}
+
+int32_t mkv_pool_create(const mkv_pool_config* cfg, void* fp8_arena, void* tq3_arena, void* stream,
+                        mkv_pool** out)
+{
+    int32_t rc = check_cfg(cfg);
+    if (rc) return rc;
+    if (!out || !fp8_arena || !tq3_arena || !cfg->k_rot_signs) return MKV_E_INVALID;
+    if (!aligned(fp8_arena, 256) || !aligned(tq3_arena, 256)) return MKV_E_INVALID;
+    for (int i = 0; i < cfg->head_dim; ++i)
+        if (cfg->k_rot_signs[i] != 1 && cfg->k_rot_signs[i] != -1) return MKV_E_INVALID;
+    mkv_pool* p = new_pool(cfg, fp8_arena, tq3_arena);
+    if (!p) return MKV_E_INVALID;
+    size_t fp8_bytes, tq3_bytes;
+    mkv_pool_query(cfg, &fp8_bytes, &tq3_bytes);
+    p->status_dev = reinterpret_cast<uint32_t*>(p->fp8 + fp8_bytes - kStatusTail);
+
+    cudaError_t e = cudaGetDevice(&p->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&p->dev.sm_count, cudaDevAttrMultiProcessorCount, p->device);
+    if (e == cudaSuccess)
+        e = cudaDeviceGetAttribute(&p->dev.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, p->device);
+    cudaStream_t s = (cudaStream_t)stream;
+    if (e == cudaSuccess) e = cudaMemsetAsync(p->fp8, 0, fp8_bytes, s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(p->tq3, 0, tq3_bytes, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) {
+        delete p;
+        return cuda_fail(e, "mkv_pool_create");
+    }
+    *out = p;
+    return MKV_OK;
+}
+
+int32_t mkv_pool_destroy(mkv_pool* pool)
+{
+    if (!pool) return MKV_E_INVALID;
+    delete pool;
+    return MKV_OK;
+}
+
+int32_t mkv_page_alloc(mkv_pool* pool, int32_t fmt, int32_t* ids, int32_t n)
+{
+    if (!pool || (fmt != MKV_FMT_FP8 && fmt != MKV_FMT_TQ3) || n < 0 || (n > 0 && !ids)) return MKV_E_INVALID;
+    std::lock_guard<std::mutex> lk(pool->mu);
+    auto& fl = pool->free_list[fmt];
+    if ((size_t)n > fl.size()) return fmt == MKV_FMT_FP8 ? MKV_E_OOM_FP8 : MKV_E_OOM_TQ3;
+    for (int i = 0; i < n; ++i) {
+        ids[i] = fl.back();
+        fl.pop_back();
+        pool->allocated[fmt][ids[i]] = 1;
+    }
+    return MKV_OK;
+}
+
+int32_t mkv_page_free(mkv_pool* pool, int32_t fmt, const int32_t* ids, int32_t n)
+{
+    if (!pool || (fmt != MKV_FMT_FP8 && fmt != MKV_FMT_TQ3) || n < 0 || (n > 0 && !ids)) return MKV_E_INVALID;
+    std::lock_guard<std::mutex> lk(pool->mu);
+    auto& al = pool->allocated[fmt];
+    for (int i = 0; i < n; ++i) {
+        if (ids[i] < 0 || (size_t)ids[i] >= al.size()) return MKV_E_BOUNDS;
+        if (!al[ids[i]]) return MKV_E_STATE;
+        for (int j = 0; j < i; ++j)
+            if (ids[j] == ids[i]) return MKV_E_STATE;
+    }
+    for (int i = 0; i < n; ++i) {
+        al[ids[i]] = 0;
+        pool->free_list[fmt].push_back(ids[i]);
+    }
+    return MKV_OK;
+}
+
+int32_t mkv_pool_stats(const mkv_pool* pool, mkv_stats* out)
+{
+    if (!pool || !out) return MKV_E_INVALID;
+    mkv_pool* p = const_cast<mkv_pool*>(pool);
+    std::lock_guard<std::mutex> lk(p->mu);
+    out->fp8_pages_total = p->cfg.fp8_pages;
+    out->tq3_pages_total = p->cfg.tq3_pages;
+    out->fp8_pages_used = p->cfg.fp8_pages - (int64_t)p->free_list[0].size();
+    out->tq3_pages_used = p->cfg.tq3_pages - (int64_t)p->free_list[1].size();
+    out->fp8_bytes_used = out->fp8_pages_used * p->hkv * (int64_t)fp8_record_bytes(p->d);
+    out->tq3_bytes_used = out->tq3_pages_used * p->hkv * (int64_t)tq3_record_bytes(p->d);
+    out->bf16_bytes_equivalent = (out->fp8_pages_used + out->tq3_pages_used) * p->hkv * (int64_t)kPage * p->d * 4;
+    return MKV_OK;
+}
+
+int32_t mkv_pool_status(mkv_pool* pool, void* stream)
+{
+    if (!pool || !pool->fp8) return MKV_E_INVALID;
+    uint32_t st = 0;
+    cudaStream_t s = (cudaStream_t)stream;
+    MKV_CUDA(cudaMemcpyAsync(&st, pool->status_dev, sizeof st, cudaMemcpyDeviceToHost, s));
+    MKV_CUDA(cudaStreamSynchronize(s));
+    if (st) {
+        MKV_CUDA(cudaMemsetAsync(pool->status_dev, 0, sizeof st, s));
+        MKV_CUDA(cudaStreamSynchronize(s));
+    }
+    if (st & kStTimeout) return MKV_E_TIMEOUT;
+    if (st & kStBounds) return MKV_E_BOUNDS;
+    if (st & kStState) return MKV_E_STATE;
+    return MKV_OK;
+}
+
+int32_t mkv_pool_set_decode_variant(mkv_pool* pool, int32_t variant)
+{
+    if (!pool || (variant != MKV_DECODE_TENSOR && variant != MKV_DECODE_SCALAR)) return MKV_E_INVALID;
+    pool->variant = variant;
+    return MKV_OK;
+}
+
+static int32_t raw_span(mkv_pool* pool, int32_t fmt, int32_t id, uint8_t** ptr, size_t* bytes)
+{
+    if (!pool || !pool->fp8 || (fmt != MKV_FMT_FP8 && fmt != MKV_FMT_TQ3)) return MKV_E_INVALID;
+    int cap = fmt == MKV_FMT_FP8 ? pool->cfg.fp8_pages : pool->cfg.tq3_pages;
+    if (id < 0 || id >= cap) return MKV_E_BOUNDS;
+    size_t rec = fmt == MKV_FMT_FP8 ? fp8_record_bytes(pool->d) : tq3_record_bytes(pool->d);
+    *bytes = rec * pool->hkv;
+    *ptr = (fmt == MKV_FMT_FP8 ? pool->fp8 : pool->tq3) + (size_t)id * *bytes;
+    return MKV_OK;
+}
+
+int32_t mkv_page_read_raw(mkv_pool* pool, int32_t fmt, int32_t id, void* host_buf, void* stream)
+{
+    uint8_t* ptr;
+    size_t bytes;
+    int32_t rc = raw_span(pool, fmt, id, &ptr, &bytes);
+    if (rc) return rc;
+    if (!host_buf) return MKV_E_INVALID;
+    MKV_CUDA(cudaMemcpyAsync(host_buf, ptr, bytes, cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    MKV_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+    return MKV_OK;
+}
+
+int32_t mkv_page_write_raw(mkv_pool* pool, int32_t fmt, int32_t id, const void* host_buf, void* stream)
+{
+    uint8_t* ptr;
+    size_t bytes;
+    int32_t rc = raw_span(pool, fmt, id, &ptr, &bytes);
+    if (rc) return rc;
+    if (!host_buf) return MKV_E_INVALID;
+    MKV_CUDA(cudaMemcpyAsync(ptr, host_buf, bytes, cudaMemcpyHostToDevice, (cudaStream_t)stream));
+    MKV_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+    return MKV_OK;
+}
+
+// ---- hot-path entry points: validate on the host, then enqueue ---------------------------------
+
+int32_t mkv_append(mkv_pool* pool, const void* k, const void* v, const int32_t* slots, int32_t n, void* stream)
+{
+    if (!pool || !pool->fp8 || n < 0) return MKV_E_INVALID;
+    if (n == 0) return MKV_OK;
+    if (!k || !v || !slots || !aligned(k, 16) || !aligned(v, 16) || !aligned(slots, 4)) return MKV_E_INVALID;
+    return launch_append(pool, k, v, slots, n, (cudaStream_t)stream);
+}
+
+int32_t mkv_demote(mkv_pool* pool, const int32_t* src, const int32_t* dst, int32_t n, int32_t* bt,
+                   uint8_t* tags, const int64_t* entry, void* stream)
+{
+    if (!pool || !pool->fp8 || n < 0) return MKV_E_INVALID;
+    if (n == 0) return MKV_OK;
+    if (!src || !dst) return MKV_E_INVALID;
+    if (entry && (!bt || !tags)) return MKV_E_INVALID;
+    return launch_demote(pool, src, dst, n, bt, tags, entry, (cudaStream_t)stream);
+}
+
+int32_t mkv_set_anchor(mkv_pool* pool, uint8_t* tags, int64_t entry, int32_t flag, void* stream)
+{
+    if (!pool || !pool->fp8 || !tags || entry < 0) return MKV_E_INVALID;
+    return launch_set_anchor(pool, tags, entry, flag, (cudaStream_t)stream);
+}
+
+int32_t mkv_decode_attention(mkv_pool* pool, const void* q, const int32_t* bt, const uint8_t* tags,
+                             const int32_t* lens, int32_t B, int32_t max_pages, float scale, float* out,
+                             float* lse, void* ws, size_t ws_bytes, void* stream)
+{
+    if (!pool || !pool->fp8 || B < 0 || max_pages < 0) return MKV_E_INVALID;
+    if (B == 0) return MKV_OK;
+    if (!q || !bt || !tags || !lens || !out || !ws) return MKV_E_INVALID;
+    if (!aligned(q, 16) || !aligned(out, 16) || !aligned(ws, 256) || !aligned(bt, 4) || !aligned(lens, 4))
+        return MKV_E_INVALID;
+    size_t need;
+    if (mkv_decode_workspace_bytes(&pool->cfg, B, &need) != MKV_OK || ws_bytes < need) return MKV_E_INVALID;
+    if (!(scale == scale)) return MKV_E_INVALID;
+    if (pool->variant == MKV_DECODE_SCALAR)
+        return launch_decode_scalar(pool, q, bt, tags, lens, B, max_pages, scale, out, lse, ws, ws_bytes,
+                                    (cudaStream_t)stream);
+    return launch_decode_tensor(pool, q, bt, tags, lens, B, max_pages, scale, out, lse, ws, ws_bytes,
+                                (cudaStream_t)stream);
+}
+
+// ---- sequence rows (Algorithm 1, host bookkeeping only) ----------------------------------------
+
+int32_t mkv_seq_create(mkv_pool* pool, mkv_seq** out)
+{
+    if (!pool || !out) return MKV_E_INVALID;
+    mkv_seq* s = new (std::nothrow) mkv_seq();
+    if (!s) return MKV_E_INVALID;
+    s->pool = pool;
+    s->len = 0;
+    *out = s;
+    return MKV_OK;
+}
+
+int32_t mkv_seq_finish(mkv_seq* seq)
+{
+    if (!seq) return MKV_E_INVALID;
+    int32_t rc = MKV_OK;
+    for (size_t i = 0; i < seq->ids.size(); ++i) {
+        int fmt = seq->tags[i] == MKV_TAG_STALE ? MKV_FMT_TQ3 : MKV_FMT_FP8;
+        int32_t r = mkv_page_free(seq->pool, fmt, &seq->ids[i], 1);
+        if (r != MKV_OK) rc = r;
+    }
+    delete seq;
+    return rc;
+}
+
+int32_t mkv_seq_append(mkv_seq* seq, int32_t* page_id, int32_t* slot, int32_t* opened)
+{
+    if (!seq || !page_id || !slot) return MKV_E_INVALID;
+    bool open = seq->len % kPage == 0;
+    if (open) {
+        int32_t id;
+        int32_t rc = mkv_page_alloc(seq->pool, MKV_FMT_FP8, &id, 1);
+        if (rc) return rc;
+        seq->ids.push_back(id);
+        seq->tags.push_back(MKV_TAG_RECENT);
+    }
+    *page_id = seq->ids.back();
+    *slot = seq->len % kPage;
+    if (opened) *opened = open ? 1 : 0;
+    seq->len += 1;
+    return MKV_OK;
+}
+
+int32_t mkv_seq_protect(mkv_seq* seq, int32_t lp, int32_t flag)
+{
+    if (!seq) return MKV_E_INVALID;
+    if (lp < 0 || (size_t)lp >= seq->ids.size()) return MKV_E_BOUNDS;
+    if (seq->tags[lp] == MKV_TAG_STALE) return MKV_E_STATE;
+    if (!flag && seq->tags[lp] != MKV_TAG_ANCHOR) return MKV_E_STATE;
+    seq->tags[lp] = flag ? MKV_TAG_ANCHOR : MKV_TAG_RECENT;
+    return MKV_OK;
+}
+
+int32_t mkv_seq_demote(mkv_seq* seq, int32_t lp, int32_t* src, int32_t* dst)
+{
+    if (!seq || !src || !dst) return MKV_E_INVALID;
+    if (lp < 0 || (size_t)lp >= seq->ids.size()) return MKV_E_BOUNDS;
+    if (seq->tags[lp] == MKV_TAG_STALE) return MKV_E_STATE;
+    if ((lp + 1) * kPage > seq->len) return MKV_E_STATE;   // only full pages may become TQ3
+    int32_t id;
+    int32_t rc = mkv_page_alloc(seq->pool, MKV_FMT_TQ3, &id, 1);
+    if (rc) return rc;
+    *src = seq->ids[lp];
+    *dst = id;
+    seq->ids[lp] = id;
+    seq->tags[lp] = MKV_TAG_STALE;
+    return mkv_page_free(seq->pool, MKV_FMT_FP8, src, 1);
+}
+
+int32_t mkv_seq_age(mkv_seq* seq, int32_t recent_tokens, int32_t* lps, int32_t* srcs, int32_t* dsts,
+                    int32_t cap, int32_t* n)
+{
+    if (!seq || !n || recent_tokens < 0 || cap < 0) return MKV_E_INVALID;
+    int first_recent = (seq->len - recent_tokens > 0 ? seq->len - recent_tokens : 0) / kPage;
+    if ((size_t)first_recent > seq->ids.size()) first_recent = (int)seq->ids.size();
+    int need = 0;
+    for (int lp = 0; lp < first_recent; ++lp)
+        if (seq->tags[lp] == MKV_TAG_RECENT && (lp + 1) * kPage <= seq->len) ++need;
+    if (need > cap || (need > 0 && (!lps || !srcs || !dsts))) return MKV_E_INVALID;
+    {
+        std::lock_guard<std::mutex> lk(seq->pool->mu);
+        if ((size_t)need > seq->pool->free_list[MKV_FMT_TQ3].size()) return MKV_E_OOM_TQ3;
+    }
+    int k = 0;
+    for (int lp = 0; lp < first_recent; ++lp)
+        if (seq->tags[lp] == MKV_TAG_RECENT && (lp + 1) * kPage <= seq->len) {
+            int32_t rc = mkv_seq_demote(seq, lp, &srcs[k], &dsts[k]);
+            if (rc) return rc;
+            lps[k++] = lp;
+        }
+    *n = k;
+    return MKV_OK;
+}
+
+int32_t mkv_seq_len(const mkv_seq* seq, int32_t* len, int32_t* n_pages)
+{
+    if (!seq) return MKV_E_INVALID;
+    if (len) *len = seq->len;
+    if (n_pages) *n_pages = (int32_t)seq->ids.size();
+    return MKV_OK;
+}
+
+int32_t mkv_seq_row(const mkv_seq* seq, int32_t* ids, uint8_t* tags, int32_t cap)
+{
+    if (!seq || cap < (int32_t)seq->ids.size()) return MKV_E_INVALID;
+    for (size_t i = 0; i < seq->ids.size(); ++i) {
+        if (ids) ids[i] = seq->ids[i];
+        if (tags) tags[i] = seq->tags[i];
+    }
+    return MKV_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,129 @@
+"""Bit-exact parity of the packing kernels with the oracle: Append (bf16 -> e4m3 records) and
+Demote (FP8 record -> TQ3 record), through the C ABI, compared by raw page read-back."""
+import numpy as np
+import pytest
+import torch
+
+import mkv_workloads as W
+import oracle
+import paper_2608_23834_b200 as M
+from _gpu_util import bf16_tensor
+
+pytestmark = pytest.mark.gpu
+
+
+def special_bf16(rng, shape):
+    """N(0,1) with outliers plus values that exercise rounding ties, saturation, subnormals and zeros."""
+    x = rng.standard_normal(shape).astype(np.float32)
+    flat = x.reshape(-1)
+    specials = np.float32([0.0, -0.0, 448.0, 449.0, 464.0, 480.0, 1e4, -1e4, 2.0 ** -10, 3 * 2.0 ** -10, 2.0 ** -9,
+                           -2.0 ** -9, 17.0, 19.0, 0.0009765625, 1e-8, -1e-8, 0.28125, 0.296875, 240.0, 232.0])
+    idx = rng.choice(flat.size, size=4 * len(specials), replace=False)
+    flat[idx] = np.tile(specials, 4)
+    return W.f32_to_bf16_bits(x)
+
+
+@pytest.mark.parametrize("d,hkv,k_scale,v_scale", [(128, 2, 1.0, 1.0), (256, 4, 1.0, 1.0), (128, 1, 0.5, 2.0)])
+def test_append_is_bit_exact(d, hkv, k_scale, v_scale):
+    rng = np.random.default_rng(d + hkv)
+    n_pages = 7
+    pool = M.Pool(d, hkv, hkv * 4, n_pages, 1, np.ones(d, np.int8), k_scale, v_scale)
+    n_tok = 16 * 5 + 3
+    k_bits, v_bits = special_bf16(rng, (n_tok, hkv, d)), special_bf16(rng, (n_tok, hkv, d))
+    # tokens land on shuffled pages, in order inside each page; two tokens are skipped (-1)
+    page_of = rng.permutation(n_pages)[:6]
+    slots = np.array([page_of[t // 16] * 16 + t % 16 for t in range(n_tok)], np.int32)
+    skipped = [5, 40]
+    slots[skipped] = -1
+    # append in two calls to cover repeated launches
+    for lo, hi in ((0, 30), (30, n_tok)):
+        pool.append(bf16_tensor(k_bits[lo:hi]), bf16_tensor(v_bits[lo:hi]), torch.from_numpy(slots[lo:hi]).cuda())
+    torch.cuda.synchronize()
+    assert pool.status() == M.OK
+    kf, vf = oracle.bf16_bits_to_f32(k_bits), oracle.bf16_bits_to_f32(v_bits)
+    for lp in range(6):
+        got = pool.page_read_raw(M.FMT_FP8, int(page_of[lp])).reshape(hkv, 32 * d)
+        for h in range(hkv):
+            kk = np.zeros((16, d), np.float32)
+            vv = np.zeros((16, d), np.float32)
+            n = min(16, n_tok - 16 * lp)
+            kk[:n], vv[:n] = kf[16 * lp:16 * lp + n, h], vf[16 * lp:16 * lp + n, h]
+            ref = oracle.fp8_pack_record(kk, vv, n, k_scale, v_scale).copy()
+            for t in skipped:                       # skipped tokens leave the zero-filled slot untouched
+                if t // 16 == lp:
+                    ref[:16 * d].reshape(16, d)[t % 16] = 0
+                    ref[16 * d:].reshape(d, 16)[:, t % 16] = 0
+            assert np.array_equal(got[h], ref), (lp, h)
+    # the untouched page is still zero
+    assert not pool.page_read_raw(M.FMT_FP8, int(np.setdiff1d(np.arange(n_pages), page_of)[0])).any()
+
+
+@pytest.mark.parametrize("d,hkv,k_scale,v_scale", [(128, 2, 1.0, 1.0), (256, 4, 1.0, 1.0), (256, 1, 0.25, 4.0)])
+def test_demote_is_bit_exact_and_publishes_after_the_copy(d, hkv, k_scale, v_scale):
+    rng = np.random.default_rng(100 + d + hkv)
+    n = 9
+    sigma = (rng.integers(0, 2, d) * 2 - 1).astype(np.int8)
+    pool = M.Pool(d, hkv, hkv, n, n + 2, sigma, k_scale, v_scale)
+    recs = np.zeros((n, hkv, 32 * d), np.uint8)
+    for p in range(n):
+        for h in range(hkv):
+            k = rng.standard_normal((16, d)).astype(np.float32)
+            v = rng.standard_normal((16, d)).astype(np.float32)
+            k[:, rng.integers(0, d, 3)] *= 8
+            v[:, rng.integers(0, d, 3)] *= 8
+            if p == 1:
+                k[3] = 0.0                   # zero key vector -> codes 0, g = 0
+                v[:, 5] = 1.5                # constant channel -> scale 0
+                v[:, 6] = 0.0
+            if p == 2:
+                v[:, 7] = np.float32([0, 7, 0.5, 1.5, 2.5, 3.5, 4.5, 5.5, 6.5, 1, 2, 3, 4, 5, 6, 7])   # rounding ties
+                v[::2, 9], v[1::2, 9] = 0.0, -0.0
+            recs[p, h] = oracle.fp8_pack_record(k, v, 16, k_scale, v_scale)
+        pool.page_write_raw(M.FMT_FP8, p, recs[p])
+    src = torch.from_numpy(rng.permutation(n).astype(np.int32)).cuda()
+    dst = torch.from_numpy((rng.permutation(n + 2)[:n]).astype(np.int32)).cuda()
+    bt = torch.full((3, 8), -1, dtype=torch.int32, device="cuda:0")
+    tags = torch.zeros((3, 8), dtype=torch.uint8, device="cuda:0")
+    entry = torch.arange(n, dtype=torch.int64, device="cuda:0") * 2
+    entry[4] = -1                                       # one page is encoded but not published
+    pool.demote(src, dst, bt, tags, entry)
+    torch.cuda.synchronize()
+    assert pool.status() == M.OK
+    s, t = src.cpu().numpy(), dst.cpu().numpy()
+    for i in range(n):
+        got = pool.page_read_raw(M.FMT_TQ3, int(t[i])).reshape(hkv, 16 * d + 32)
+        for h in range(hkv):
+            ref = oracle.demote_record(recs[s[i], h], d, sigma, k_scale, v_scale)
+            assert np.array_equal(got[h], ref), (i, h, np.nonzero(got[h] != ref)[0][:8])
+        # the source page is untouched
+        assert np.array_equal(pool.page_read_raw(M.FMT_FP8, int(s[i])).reshape(hkv, 32 * d), recs[s[i]])
+    btc, tc = bt.cpu().numpy().reshape(-1), tags.cpu().numpy().reshape(-1)
+    for i in range(n):
+        if i == 4:
+            continue
+        assert btc[2 * i] == t[i] and tc[2 * i] == M.TAG_STALE
+    assert (btc[1::2] == -1).all() and (tc[1::2] == 0).all() and btc[8] == -1 and tc[8] == 0
+
+
+def test_out_of_range_ids_are_flagged_not_dereferenced():
+    d, hkv = 128, 1
+    pool = M.Pool(d, hkv, 4, 4, 4, np.ones(d, np.int8))
+    k = torch.zeros((2, hkv, d), dtype=torch.bfloat16, device="cuda:0")
+    pool.append(k, k, torch.tensor([4 * 16, 16], dtype=torch.int32, device="cuda:0"))     # page 4 does not exist
+    assert pool.status() == M.E_BOUNDS and pool.status() == M.OK
+    pool.demote(torch.tensor([0, 9], dtype=torch.int32, device="cuda:0"), torch.tensor([0, 1], dtype=torch.int32, device="cuda:0"))
+    assert pool.status() == M.E_BOUNDS
+    pool.demote(torch.tensor([0], dtype=torch.int32, device="cuda:0"), torch.tensor([-3], dtype=torch.int32, device="cuda:0"))
+    assert pool.status() == M.E_BOUNDS
+
+
+def test_set_anchor_flips_fp8_tags_and_refuses_stale():
+    pool = M.Pool(128, 1, 4, 4, 4, np.ones(128, np.int8))
+    tags = torch.tensor([[0, 0, 2, 1]], dtype=torch.uint8, device="cuda:0")
+    pool.set_anchor(tags, 1, True)
+    pool.set_anchor(tags, 3, False)
+    assert pool.status() == M.OK
+    assert tags.cpu().numpy().tolist() == [[0, 1, 2, 0]]
+    pool.set_anchor(tags, 2, True)            # Stale must be promoted first
+    assert pool.status() == M.E_STATE
+    assert tags.cpu().numpy().tolist() == [[0, 1, 2, 0]]
