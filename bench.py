@@ -1,0 +1,512 @@
+#!/usr/bin/env python
+"""Benchmark of the mixed-format (FP8 + TQ3) paged decode path on B200.
+
+One step = one decode step of the whole hot path over the batch, for every layer of the workload:
+Append of the new token's K/V into the Recent FP8 page, Demote (FP8 -> TQ3, publish) of the page
+that leaves the Recent window when one does, an Anchor tag flip at each such retier point, and
+mkv_decode_attention (table walk, query rotation, FP8 and TQ3 page scans, split partials, merge).
+Default workload: 2 requests x 59,008 tokens, 16 layers each with its own pool, d = 256,
+4 KV x 6 query heads, first 256 tokens Anchor, last 2,048 Recent, the rest TQ3.
+
+Prints ONE JSON line (rank 0).  `value` is decode tokens/s with everything resident in HBM;
+`e2e` is the same metric with the step's inputs copied from pinned host memory and its outputs read
+back inside the timed region; `roofline` is achieved KV GB/s of the decode kernel against the
+measured HBM copy bandwidth; `cpu_baseline` is the fp64 CPU oracle timed on a bounded sample.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 0..4]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import mkv_workloads as W  # noqa: E402
+
+METRIC = "decode attention tokens/s and achieved KV HBM GB/s (% of B200 peak) at 1 GPU"
+UNIT = "tokens/s"
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode_tensor_kernel launch on the default
+# workload, from the ncu capture summarised under profiles/; None until captured.
+TRAFFIC_BYTES_PER_LAUNCH = None
+FALLBACK_HBM_GBS = 6650.0
+STAGE_PAGES = 512
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": FALLBACK_HBM_GBS}, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def __exit__(self, *exc):
+        if self.proc is not None:
+            time.sleep(0.15)
+            self.proc.terminate()          # the exact child started above
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+
+    def summary(self):
+        sm, smax, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                smax.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, val in zip(names, r[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------------- ours
+class LayerState:
+    pass
+
+
+def build_layers(spec, steps_total, device, M, torch):
+    """Pools of every layer filled through the library's own Append and Demote kernels from seeded
+    synthetic bf16 K/V, plus the tables, slots and retier plan of every timed step."""
+    B, d, hkv, hq = spec.batch, spec.head_dim, spec.n_kv_heads, spec.n_q_heads
+    final_lens = [n + steps_total for n in spec.seq_lens]
+    max_pages = max((n + 15) // 16 for n in final_lens) + 1
+    tab0 = W.tables(spec)
+    n_fp8_0, n_tq3_0 = tab0.fp8_pages, tab0.tq3_pages
+    extra_pages = sum((fl + 15) // 16 - (n + 15) // 16 for fl, n in zip(final_lens, spec.seq_lens))
+    demotes_per_req = steps_total // 16 + 2
+    fp8_cap = n_fp8_0 + extra_pages + STAGE_PAGES + 8
+    tq3_cap = n_tq3_0 + B * demotes_per_req + 8
+
+    # host plan shared by all layers: table, tags, per-step slots and retier events
+    bt = np.full((B, max_pages), -1, np.int32)
+    tg = np.zeros((B, max_pages), np.uint8)
+    bt[:, :tab0.block_table.shape[1]] = tab0.block_table
+    tg[:, :tab0.tier_tag.shape[1]] = tab0.tier_tag
+    next_fp8, next_tq3 = n_fp8_0, n_tq3_0
+    lens = np.array(spec.seq_lens, np.int64)
+    n_pages = (lens + 15) // 16
+    slots = np.zeros((steps_total, B), np.int32)
+    lens_steps = np.zeros((steps_total, B), np.int32)
+    events = []              # per step: list of (b, logical page, src fp8 id, dst tq3 id)
+    recent = spec.recent_tokens if spec.stale_fraction is None else int(round((1 - spec.stale_fraction) * lens[0]))
+    for st in range(steps_total):
+        ev = []
+        for b in range(B):
+            if lens[b] % 16 == 0:                       # Append opens a Recent page
+                bt[b, n_pages[b]] = next_fp8
+                tg[b, n_pages[b]] = W.TAG_RECENT
+                next_fp8 += 1
+                n_pages[b] += 1
+            slots[st, b] = bt[b, lens[b] // 16] * 16 + lens[b] % 16
+            lens[b] += 1
+            lens_steps[st, b] = lens[b]
+            # age: a full Recent page wholly before the window is demoted (tags tracked on the host too)
+            first_recent = max(0, lens[b] - recent) // 16
+            for lp in range(max(0, first_recent - 2), first_recent):
+                if tg[b, lp] == W.TAG_RECENT:
+                    ev.append((b, lp, int(bt[b, lp]), next_tq3))
+                    tg[b, lp] = W.TAG_STALE
+                    bt[b, lp] = next_tq3
+                    next_tq3 += 1
+        events.append(ev)
+    assert next_fp8 <= fp8_cap - STAGE_PAGES and next_tq3 <= tq3_cap
+
+    layers = []
+    gen = torch.Generator(device=device)
+    for layer in range(spec.n_layers):
+        L = LayerState()
+        sigma = W.rotation_signs(spec, layer)
+        L.pool = M.Pool(d, hkv, hq, fp8_cap, tq3_cap, sigma, max_batch=B, device=device)
+        gen.manual_seed(1000 * spec.seed + layer)
+        k_out = torch.from_numpy(W.outlier_channels(spec, layer, 0)).to(device)
+        v_out = torch.from_numpy(W.outlier_channels(spec, layer, 1)).to(device)
+
+        def synth(n_tok):
+            k = torch.randn((n_tok, hkv, d), generator=gen, device=device, dtype=torch.float32)
+            v = torch.randn((n_tok, hkv, d), generator=gen, device=device, dtype=torch.float32)
+            k[:, :, k_out] *= 8.0
+            v[:, :, v_out] *= 8.0
+            return k.to(torch.bfloat16).contiguous(), v.to(torch.bfloat16).contiguous()
+
+        stage0 = fp8_cap - STAGE_PAGES
+        for b in range(B):
+            npg = (spec.seq_lens[b] + 15) // 16
+            tags_b, ids_b = tab0.tier_tag[b, :npg], tab0.block_table[b, :npg]
+            fp8_lp = np.nonzero(tags_b != W.TAG_STALE)[0]
+            # Recent/Anchor pages: append straight into their pages
+            tok = np.concatenate([np.arange(lp * 16, min(lp * 16 + 16, spec.seq_lens[b])) for lp in fp8_lp]) \
+                if len(fp8_lp) else np.zeros(0, np.int64)
+            if len(tok):
+                sm = (ids_b[tok // 16].astype(np.int64) * 16 + tok % 16).astype(np.int32)
+                k, v = synth(len(tok))
+                L.pool.append(k, v, torch.from_numpy(sm).to(device))
+            # Stale pages: append into staging FP8 pages, demote into their TQ3 pages, reuse the staging pages
+            st_lp = np.nonzero(tags_b == W.TAG_STALE)[0]
+            for c0 in range(0, len(st_lp), STAGE_PAGES):
+                chunk = st_lp[c0:c0 + STAGE_PAGES]
+                n = len(chunk)
+                sm = ((stage0 + np.arange(n))[:, None] * 16 + np.arange(16)[None, :]).reshape(-1).astype(np.int32)
+                k, v = synth(16 * n)
+                L.pool.append(k, v, torch.from_numpy(sm).to(device))
+                src = torch.arange(stage0, stage0 + n, dtype=torch.int32, device=device)
+                dst = torch.from_numpy(ids_b[chunk].astype(np.int32)).to(device)
+                L.pool.demote(src, dst)
+        torch.cuda.synchronize(device)
+        if L.pool.status() != M.OK:
+            raise RuntimeError("pool status after fill")
+        # future Recent pages are already named in the table (decode reads only ceil(len/16) entries)
+        L.bt = torch.from_numpy(initial_table(tab0, bt)).to(device)
+        L.tags = torch.from_numpy(initial_tags(tab0, tg)).to(device)
+        L.q = torch.randn((B, hq, d), generator=gen, device=device, dtype=torch.float32).to(torch.bfloat16)
+        L.k_new, L.v_new = synth(B)
+        L.out = torch.empty((B, hq, d), dtype=torch.float32, device=device)
+        layers.append(L)
+    plan = {
+        "slots": torch.from_numpy(slots).to(device), "lens": torch.from_numpy(lens_steps).to(device),
+        "events": events, "max_pages": max_pages, "lens_host": lens_steps, "slots_host": slots,
+    }
+    # device-side arguments of every retier event
+    plan["ev_dev"] = []
+    for ev in events:
+        if not ev:
+            plan["ev_dev"].append(None)
+            continue
+        src = torch.tensor([e[2] for e in ev], dtype=torch.int32, device=device)
+        dst = torch.tensor([e[3] for e in ev], dtype=torch.int32, device=device)
+        ent = torch.tensor([e[0] * max_pages + e[1] for e in ev], dtype=torch.int64, device=device)
+        plan["ev_dev"].append((src, dst, ent, [e[0] * max_pages + e[1] + 1 for e in ev]))
+    return layers, plan, tab0
+
+
+def initial_table(tab0, bt_final):
+    """Table at time zero: the initial mapping, plus the ids of pages that Append will open later;
+    entries that Demote will rewrite keep their initial FP8 ids."""
+    out = bt_final.copy()
+    w = tab0.block_table.shape[1]
+    used = tab0.block_table >= 0
+    out[:, :w][used] = tab0.block_table[used]
+    return out
+
+
+def initial_tags(tab0, tg_final):
+    out = tg_final.copy()
+    w = tab0.tier_tag.shape[1]
+    used = tab0.block_table >= 0
+    out[:, :w][used] = tab0.tier_tag[used]
+    return out
+
+
+def kv_bytes_at(spec, tags_host_rows, lens_row):
+    """Algorithmic KV bytes of one decode launch: 2d per valid FP8 token + (16d + 32) per Stale page, per KV head."""
+    d, total = spec.head_dim, 0
+    for b, ln in enumerate(lens_row):
+        npg = (int(ln) + 15) // 16
+        stale = int((tags_host_rows[b, :npg] == W.TAG_STALE).sum())
+        total += spec.n_kv_heads * ((int(ln) - 16 * stale) * 2 * d + stale * (16 * d + 32))
+    return total
+
+
+def run_ours(args):
+    import torch
+    import paper_2608_23834_b200 as M
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    device = torch.device(f"cuda:{local}")
+    torch.cuda.set_device(device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+    M.lib()
+    spec = workload_spec(args)
+    K, Wm = args.steps, args.warmup
+    total = 2 * (K + Wm)                       # device-resident run, then the end-to-end run
+    layers, plan, tab0 = build_layers(spec, total, device, M, torch)
+    B, d, hq, hkv = spec.batch, spec.head_dim, spec.n_q_heads, spec.n_kv_heads
+    stream = torch.cuda.current_stream()
+    launches = [0]
+    # host mirror of the tags, advanced with the retier events, for the byte count of each step
+    tags_host = initial_tags(tab0, np.zeros((B, plan["max_pages"]), np.uint8))
+    ev_pairs = []
+
+    def step(i, timed_events=None):
+        ev = plan["ev_dev"][i]
+        for L in layers:
+            L.pool.append(L.k_new, L.v_new, plan["slots"][i])
+            launches[0] += 1
+            if ev is not None:
+                src, dst, ent, nxt = ev
+                L.pool.demote(src, dst, L.bt, L.tags, ent)
+                for e in nxt:                     # retier checkpoint: protect / unprotect the page that follows
+                    L.pool.set_anchor(L.tags, e, True)
+                    L.pool.set_anchor(L.tags, e, False)
+                launches[0] += 1 + 2 * len(nxt)
+            if timed_events is not None:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+            L.pool.decode_attention(L.q, L.bt, L.tags, plan["lens"][i], spec.scale, out=L.out)
+            launches[0] += 1
+            if timed_events is not None:
+                e1.record(stream)
+                timed_events.append((e0, e1))
+        if ev is not None:
+            for (b, lp, _, _) in plan["events"][i]:
+                tags_host[b, lp] = W.TAG_STALE
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize(device)
+
+    # ---- device-resident run ------------------------------------------------------------------
+    for i in range(Wm):
+        step(i)
+    barrier()
+    launches[0] = 0
+    bytes_per_launch = []
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        t0.record(stream)
+        for i in range(Wm, Wm + K):
+            bytes_per_launch.append(kv_bytes_at(spec, tags_host, plan["lens_host"][i]))
+            step(i, ev_pairs)
+        t1.record(stream)
+        barrier()
+    ms = t0.elapsed_time(t1)
+    n_launch = launches[0]
+    kern_ms = [a.elapsed_time(b) for a, b in ev_pairs]
+    for L in layers:
+        if L.pool.status() != M.OK:
+            raise RuntimeError("device status word set during the timed region")
+
+    # ---- end-to-end run: host buffers in, host buffers out, through the same calls --------------
+    pin = lambda t: t.cpu().pin_memory()
+    h_q = [pin(L.q) for L in layers]
+    h_k = [pin(L.k_new) for L in layers]
+    h_v = [pin(L.v_new) for L in layers]
+    h_out = [torch.empty((B, hq, d), dtype=torch.float32).pin_memory() for _ in layers]
+    h_slots = torch.from_numpy(plan["slots_host"]).pin_memory()
+    h_lens = torch.from_numpy(plan["lens_host"]).pin_memory()
+    d_slots = torch.empty(B, dtype=torch.int32, device=device)
+    d_lens = torch.empty(B, dtype=torch.int32, device=device)
+    h2d = sum(t.numel() * t.element_size() for t in (h_q[0], h_k[0], h_v[0])) * len(layers) + 8 * B
+    d2h = h_out[0].numel() * 4 * len(layers)
+
+    def step_e2e(i):
+        ev = plan["ev_dev"][i]
+        d_slots.copy_(h_slots[i], non_blocking=True)
+        d_lens.copy_(h_lens[i], non_blocking=True)
+        for li, L in enumerate(layers):
+            L.q.copy_(h_q[li], non_blocking=True)
+            L.k_new.copy_(h_k[li], non_blocking=True)
+            L.v_new.copy_(h_v[li], non_blocking=True)
+            L.pool.append(L.k_new, L.v_new, d_slots)
+            if ev is not None:
+                src, dst, ent, nxt = ev
+                L.pool.demote(src, dst, L.bt, L.tags, ent)
+            L.pool.decode_attention(L.q, L.bt, L.tags, d_lens, spec.scale, out=L.out)
+            h_out[li].copy_(L.out, non_blocking=True)
+        torch.cuda.synchronize(device)          # the step's result is on the host
+
+    base = Wm + K
+    for i in range(Wm):
+        step_e2e(base + i)
+    barrier()
+    w0 = time.perf_counter()
+    t0.record(stream)
+    for i in range(K):
+        step_e2e(base + Wm + i)
+    t1.record(stream)
+    barrier()
+    e2e_ms = max(t0.elapsed_time(t1), (time.perf_counter() - w0) * 1e3)
+
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms, e2e_ms], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, e2e_ms = float(t[0]), float(t[1])
+
+    peaks, peak_kind = measured_peaks()
+    peak = float(peaks["hbm_gbs"])
+    avg_kernel_ms = sum(kern_ms) / len(kern_ms)
+    avg_bytes = sum(bytes_per_launch) / len(bytes_per_launch)
+    achieved = avg_bytes / (avg_kernel_ms * 1e-3) / 1e9
+    step_bytes = avg_bytes * spec.n_layers
+    result = {
+        "metric": METRIC, "value": world * B * K / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+        "warmup": Wm, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u8 codes (e4m3 / 3-bit TQ3) -> f16 tensor-core operands, f32 accumulate", "data": "synthetic",
+        "config": {"workload": workload_name(spec), "batch": B, "context_tokens": list(spec.seq_lens)[:4],
+                   "layers": spec.n_layers, "head_dim": d, "kv_heads": hkv, "q_heads": hq, "page_tokens": 16,
+                   "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "l2": "inputs larger than L2 (%.0f MB of KV per step)" % (step_bytes / 1e6),
+                   "step": "append + demote at its natural cadence + decode attention, every layer"},
+        "kv_gbs_whole_step": step_bytes / (ms / K * 1e-3) / 1e9,
+        "roofline": {"bound": "hbm", "kernel": "decode_tensor_kernel", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_kind + " copy bandwidth",
+                     "frac_of_nominal_8000": achieved / 8000.0, "traffic": TRAFFIC_BYTES_PER_LAUNCH,
+                     "algorithmic_bytes_per_launch": avg_bytes, "avg_launch_ms": avg_kernel_ms},
+        "e2e": {"value": world * B * K / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / K},
+        "gpu_launches": n_launch,
+        "clocks": clocks.summary(),
+    }
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            result["cpu_baseline"] = cpu_baseline(spec)
+        print(json.dumps(result))
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+# ---------------------------------------------------------------------------------------- oracle arm
+def workload_spec(args):
+    over = {"n_layers": args.layers} if args.layers > 0 else {}
+    if args.ctx > 0 and args.config != 4:
+        over["seq_lens"] = (args.ctx,) * W.config(args.config).batch
+    if args.config == 4:
+        return W.config(4, batch=8, ctx=32768, stale_fraction=0.5, **over)
+    return W.config(args.config, **over)
+
+
+def workload_name(spec):
+    return {"cfg2_canary_59k": "configs[2]: 2 x 59,008 tokens, 16 layers, d=256, 4 KV x 6 q heads, ~96% TQ3 pages"}.get(
+        spec.name, spec.name)
+
+
+def oracle_sample(spec, seconds_hint=20.0):
+    """One layer of the workload prepared for the oracle (bounded: at most 4 requests)."""
+    import oracle
+    from oracle.harness import build_layer
+    reqs = list(range(min(spec.batch, 4)))
+    sub = W.config(0, seq_lens=[spec.seq_lens[b] for b in reqs], head_dim=spec.head_dim, n_kv_heads=spec.n_kv_heads,
+                   group=spec.group, anchor_prefix=spec.anchor_prefix, anchor_spans=max(spec.anchor_spans, 0),
+                   anchor_span_tokens=spec.anchor_span_tokens, recent_tokens=spec.recent_tokens,
+                   n_outlier=spec.n_outlier, seed=spec.seed, stale_fraction=spec.stale_fraction)
+    tab = W.tables(sub)
+    L = build_layer(sub, tab)
+    return oracle, sub, tab, L
+
+
+def time_oracle(spec, reps=1):
+    oracle, sub, tab, L = oracle_sample(spec)
+    times = []
+    for _ in range(reps):
+        t0 = time.perf_counter()
+        oracle.decode_attention(L.fp8_arena, L.tq3_arena, sub.head_dim, sub.n_kv_heads, sub.group, L.sigma, L.q_bits,
+                                tab.block_table, tab.tier_tag, tab.seq_lens, sub.scale)
+        times.append(time.perf_counter() - t0)
+    layer_s = min(times)
+    # one decode step = all layers over the whole batch; the sample covers one layer of `sub.batch` requests
+    step_s = layer_s * spec.n_layers * spec.batch / sub.batch
+    cores = min(os.cpu_count() or 1, sub.batch * sub.n_kv_heads)
+    return {"value": spec.batch / step_s, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "fp64 dequantise-then-attend of 1 of %d layers, %d of %d requests (%.2f s, scaled to a whole step)"
+                      % (spec.n_layers, sub.batch, spec.batch, layer_s),
+            "kv_gbs": W.kv_bytes(sub, tab) / layer_s / 1e9}
+
+
+def cpu_baseline(spec):
+    return time_oracle(spec)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    spec = workload_spec(args)
+    oracle, sub, tab, L = oracle_sample(spec)
+    K, Wm = args.steps, args.warmup
+    K = min(K, 5)
+    Wm = min(Wm, 1)
+
+    def one():
+        t0 = time.perf_counter()
+        oracle.decode_attention(L.fp8_arena, L.tq3_arena, sub.head_dim, sub.n_kv_heads, sub.group, L.sigma, L.q_bits,
+                                tab.block_table, tab.tier_tag, tab.seq_lens, sub.scale)
+        return time.perf_counter() - t0
+    for _ in range(Wm):
+        one()
+    layer_s = sum(one() for _ in range(K)) / K
+    step_s = layer_s * spec.n_layers * spec.batch / sub.batch
+    cores = min(os.cpu_count() or 1, sub.batch * sub.n_kv_heads)
+    val = spec.batch / step_s
+    sample = ("each step = fp64 dequantise-then-attend of 1 of %d layers, %d of %d requests, scaled to a whole step"
+              % (spec.n_layers, sub.batch, spec.batch))
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": K, "warmup": Wm,
+        "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": workload_name(spec)},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2)
+    ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling on a small case)")
+    ap.add_argument("--ctx", type=int, default=0, help="override the context length of every request (profiling)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -27,6 +27,8 @@
 #include <cuda_fp16.h>
 #include <math_constants.h>
 
+#include <cstdlib>
+
 #include "mkv_internal.cuh"
 
 namespace mkv {
@@ -238,11 +240,30 @@ struct Geo {
     static_assert(NSTAGE >= 2, "an FP8 page takes two slots");
     static_assert(NSTAGE * SLOT >= 8 * D * 4, "ring doubles as the cross-warp reduction buffer");
     static_assert(FP8_HALF <= SLOT, "half an FP8 record fits a slot");
+    static_assert(RING >= kMaxCtas * 4 + 2 * kMaxCtas * 8 * 4, "ring doubles as the final-merge scratch");
 };
 
-template <int D, int NW, int NSTAGE>
-__global__ void __launch_bounds__(NW * 32) decode_tensor_kernel(const DecodeParams P)
+#ifdef MKV_TIMELINE
+__device__ unsigned long long g_timeline[kMaxCtas * 16];
+#define MKV_STAMP(k)                                                                     \
+    do {                                                                                 \
+        if (threadIdx.x == 0 && tl_seg == 0) {                                            \
+            unsigned long long t__;                                                      \
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t__));                       \
+            g_timeline[blockIdx.x * 16 + (k)] = t__;                                      \
+        }                                                                                \
+    } while (0)
+#else
+#define MKV_STAMP(k)
+#endif
+
+template <int D, int NW, int NSTAGE, int MINB>
+__global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const DecodeParams P)
 {
+#ifdef MKV_TIMELINE
+    int tl_seg = 0;
+#endif
+    MKV_STAMP(0);
     using G = Geo<D, NW, NSTAGE>;
     constexpr int NB = G::NB;
     constexpr uint32_t FULL = 0xffffffffu;
@@ -310,6 +331,7 @@ __global__ void __launch_bounds__(NW * 32) decode_tensor_kernel(const DecodePara
 
     int pos = my_start;
     int b = 0;
+    MKV_STAMP(1);
     while (pos < my_end) {
         // ---- locate the segment: request b, KV head h, pages [pg0, pg0 + n_seg) ---------------
         while (cum[b + 1] <= pos) ++b;
@@ -369,6 +391,7 @@ __global__ void __launch_bounds__(NW * 32) decode_tensor_kernel(const DecodePara
             }
         }
         __syncthreads();
+        MKV_STAMP(2);
 
         // ---- this warp's pages of the segment --------------------------------------------------
         const int n_my = warp < n_seg ? (n_seg - warp + NW - 1) / NW : 0;
@@ -661,7 +684,9 @@ __global__ void __launch_bounds__(NW * 32) decode_tensor_kernel(const DecodePara
         }
 
         // ---- combine the warps of the block (ring memory is idle now) ---------------------------
+        MKV_STAMP(3);
         __syncthreads();
+        MKV_STAMP(4);
         if (g == 0) {
             sm_m[warp * 8 + 2 * tq] = m_run[0];
             sm_m[warp * 8 + 2 * tq + 1] = m_run[1];
@@ -690,6 +715,7 @@ __global__ void __launch_bounds__(NW * 32) decode_tensor_kernel(const DecodePara
         }
         __syncthreads();
 
+        MKV_STAMP(5);
         const bool whole_row = (pos == row_start) && (pos + n_seg == row_end);
         const int pair = b * hkv + h;
         if (whole_row) {
@@ -732,43 +758,71 @@ __global__ void __launch_bounds__(NW * 32) decode_tensor_kernel(const DecodePara
             }
             __threadfence();
             __syncthreads();
+            MKV_STAMP(6);
             const int c0 = block_of(row_start), c1 = block_of(row_end - 1);
             if (tid == 0) {
                 const uint32_t t = atomicAdd(&P.tickets[pair], 1u);
                 *sm_flag = (t == (uint32_t)(c1 - c0)) ? 1 : 0;
             }
             __syncthreads();
+            MKV_STAMP(7);
             if (*sm_flag) {
                 // last block of the row: Eq. (softmax-merge) over the row's partials
                 __threadfence();
-                float* wts = red;                          // [n_parts][8]
                 const int n_parts = c1 - c0 + 1;
-                auto part_slot = [&](int c) -> const float* {
-                    return P.partials + (size_t)(2 * c + (row_start > range_start(c) ? 1 : 0)) * (8 * D + 16);
-                };
+                int* pslot = reinterpret_cast<int*>(red);                 // [n_parts] slot index of each part
+                float* pm = red + kMaxCtas;                               // [n_parts][8] partial maxima
+                float* wts = pm + kMaxCtas * 8;                           // [n_parts][8] weights, then l
+                for (int c = tid; c < n_parts; c += NW * 32)
+                    pslot[c] = 2 * (c0 + c) + (row_start > range_start(c0 + c) ? 1 : 0);
+                __syncthreads();
+                for (int i = tid; i < n_parts * 8; i += NW * 32) {
+                    const float* ps = P.partials + (size_t)pslot[i >> 3] * (8 * D + 16) + 8 * D;
+                    const float lj = __ldcg(ps + 8 + (i & 7));
+                    pm[i] = lj > 0.f ? __ldcg(ps + (i & 7)) : -CUDART_INF_F;
+                    wts[i] = lj;
+                }
                 __syncthreads();
                 if (tid < 8) {
                     float M = -CUDART_INF_F;
-                    for (int c = c0; c <= c1; ++c) M = fmaxf(M, __ldcg(part_slot(c) + 8 * D + tid));
-                    float L = 0.f;
-                    for (int c = c0; c <= c1; ++c) {
-                        const float* ps = part_slot(c);
-                        const float mj = __ldcg(ps + 8 * D + tid), lj = __ldcg(ps + 8 * D + 8 + tid);
-                        const float w = (lj > 0.f) ? fast_exp2(mj - M) : 0.f;
-                        wts[(c - c0) * 8 + tid] = w;
-                        L += w * lj;
-                    }
+                    for (int c = 0; c < n_parts; ++c) M = fmaxf(M, pm[c * 8 + tid]);
                     sm_m[tid] = M;
+                }
+                __syncthreads();
+                for (int i = tid; i < n_parts * 8; i += NW * 32) {
+                    const float mj = pm[i];
+                    wts[i] = mj == -CUDART_INF_F ? 0.f : fast_exp2(mj - sm_m[i & 7]) * wts[i];   // w_j * l_j
+                    pm[i] = mj == -CUDART_INF_F ? 0.f : fast_exp2(mj - sm_m[i & 7]);              // w_j
+                }
+                __syncthreads();
+                if (tid < 8) {
+                    float L = 0.f;
+                    for (int c = 0; c < n_parts; ++c) L += wts[c * 8 + tid];
                     sm_l[tid] = L;
                 }
                 __syncthreads();
-                for (int e = tid; e < 8 * D; e += NW * 32) {
-                    const int head = e & 7, ch = e >> 3;
-                    if (head >= GQ) continue;
-                    float acc = 0.f;
-                    for (int c = 0; c < n_parts; ++c) acc += wts[c * 8 + head] * __ldcg(part_slot(c0 + c) + e);
-                    const float L = sm_l[head];
-                    P.out[((size_t)b * hq + h * GQ + head) * D + ch] = L > 0.f ? acc / L : 0.f;
+                // four consecutive heads of one channel per thread; many independent loads in flight
+                for (int e4 = tid; e4 < 2 * D; e4 += NW * 32) {
+                    const int head0 = (e4 & 1) * 4, ch = e4 >> 1;
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 8
+                    for (int c = 0; c < n_parts; ++c) {
+                        const float4 v = __ldcg(reinterpret_cast<const float4*>(P.partials + (size_t)pslot[c] * (8 * D + 16)) + e4);
+                        const float4 w = *reinterpret_cast<const float4*>(pm + c * 8 + head0);
+                        acc.x = fmaf(w.x, v.x, acc.x);
+                        acc.y = fmaf(w.y, v.y, acc.y);
+                        acc.z = fmaf(w.z, v.z, acc.z);
+                        acc.w = fmaf(w.w, v.w, acc.w);
+                    }
+                    const float av[4] = {acc.x, acc.y, acc.z, acc.w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const int head = head0 + k;
+                        if (head < GQ) {
+                            const float L = sm_l[head];
+                            P.out[((size_t)b * hq + h * GQ + head) * D + ch] = L > 0.f ? av[k] / L : 0.f;
+                        }
+                    }
                 }
                 if (P.lse && tid < GQ)
                     P.lse[(size_t)b * hq + h * GQ + tid] = sm_l[tid] > 0.f ? (sm_m[tid] + log2f(sm_l[tid])) * kLn2 : -CUDART_INF_F;
@@ -776,15 +830,19 @@ __global__ void __launch_bounds__(NW * 32) decode_tensor_kernel(const DecodePara
             }
         }
         __syncthreads();
+        MKV_STAMP(8);
+#ifdef MKV_TIMELINE
+        ++tl_seg;
+#endif
         pos += n_seg;
     }
 }
 
-template <int D, int NW, int NSTAGE>
+template <int D, int NW, int NSTAGE, int MINB>
 static int32_t run_tensor(mkv_pool* p, DecodeParams& prm, cudaStream_t s)
 {
     using G = Geo<D, NW, NSTAGE>;
-    auto kern = decode_tensor_kernel<D, NW, NSTAGE>;
+    auto kern = decode_tensor_kernel<D, NW, NSTAGE, MINB>;
     static int grid_cache[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     int dev = p->device & 7;
     if (grid_cache[dev] == 0) {
@@ -799,6 +857,24 @@ static int32_t run_tensor(mkv_pool* p, DecodeParams& prm, cudaStream_t s)
     MKV_CUDA(cudaGetLastError());
     return MKV_OK;
 }
+
+// launch shape: warps per block, ring slots per warp, blocks per SM the register budget is sized for
+static int tensor_shape()
+{
+    static int shape = -1;
+    if (shape < 0) {
+        const char* e = getenv("MKV_DECODE_SHAPE");
+        shape = e ? atoi(e) : 0;
+    }
+    return shape;
+}
+
+#ifdef MKV_TIMELINE
+extern "C" int mkv_debug_timeline(unsigned long long* host, int n)
+{
+    return (int)cudaMemcpyFromSymbol(host, g_timeline, sizeof(unsigned long long) * n);
+}
+#endif
 
 int32_t launch_decode_tensor(mkv_pool* p, const void* q, const int32_t* bt, const uint8_t* tags,
                              const int32_t* lens, int B, int max_pages, float scale, float* out, float* lse,
@@ -818,8 +894,23 @@ int32_t launch_decode_tensor(mkv_pool* p, const void* q, const int32_t* bt, cons
     prm.tickets = reinterpret_cast<uint32_t*>(static_cast<uint8_t*>(ws) + 256);
     prm.partials = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + decode_ws_header_bytes(B, p->hkv));
     prm.status = p->status_dev;
-    if (p->d == 128) return run_tensor<128, 8, 3>(p, prm, s);
-    return run_tensor<256, 8, 3>(p, prm, s);
+    const int shape = tensor_shape();
+    if (p->d == 128) {
+        switch (shape) {
+        case 1: return run_tensor<128, 8, 2, 2>(p, prm, s);
+        case 2: return run_tensor<128, 12, 3, 1>(p, prm, s);
+        case 3: return run_tensor<128, 16, 2, 1>(p, prm, s);
+        case 4: return run_tensor<128, 8, 3, 3>(p, prm, s);
+        default: return run_tensor<128, 8, 3, 1>(p, prm, s);
+        }
+    }
+    switch (shape) {
+    case 1: return run_tensor<256, 8, 2, 2>(p, prm, s);
+    case 2: return run_tensor<256, 12, 3, 1>(p, prm, s);
+    case 3: return run_tensor<256, 16, 2, 1>(p, prm, s);
+    case 4: return run_tensor<256, 4, 3, 3>(p, prm, s);
+    default: return run_tensor<256, 8, 3, 1>(p, prm, s);
+    }
 }
 
 }  // namespace mkv
