@@ -89,12 +89,12 @@ typedef struct {
  * fp8_bytes includes a 256-byte tail that holds the pool's device status word. */
 int32_t mkv_pool_query(const mkv_pool_config* cfg, size_t* fp8_arena_bytes, size_t* tq3_arena_bytes);
 
-/* Workspace for mkv_decode_attention with up to max_batch requests: split partials (m, l, O)
- * (Section 3.3) plus merge tickets.  Independent of sequence lengths. */
+/* Workspace for mkv_decode_attention with up to max_batch requests: the split partials (m, l, O)
+ * of Section 3.3.  Independent of sequence lengths. */
 int32_t mkv_decode_workspace_bytes(const mkv_pool_config* cfg, int32_t max_batch, size_t* bytes);
 
-/* Zero the ticket header of a workspace.  Must be enqueued once before the first decode call that
- * uses the buffer; decode leaves the header zero again when it completes. */
+/* Clear a workspace buffer.  The decode kernels write every workspace word before they read it, so
+ * this is optional; it exists so that a caller can hand over memory with defined contents. */
 int32_t mkv_workspace_init(void* workspace_dev, size_t bytes, void* stream);
 
 /* Create a pool over caller-owned arenas.  Zero-fills both arenas (so that never-written slots
@@ -177,10 +177,10 @@ int32_t mkv_set_anchor(mkv_pool* pool, uint8_t* tier_tag_dev, int64_t entry_inde
  *                partial (FP8 only); len == 0 gives out = 0 and lse = -inf
  *   out          device, fp32 [B][n_q_heads][d]
  *   lse          device, fp32 [B][n_q_heads] natural-log-sum-exp of the scaled scores, or NULL
- *   workspace    device, at least mkv_decode_workspace_bytes(cfg, B) bytes, initialised once with
- *                mkv_workspace_init(); two decode calls that overlap on the GPU need two buffers
- * One launch: a split-KV kernel whose last-arriving block per (request, KV head) merges the split
- * partials with Eq. (softmax-merge).  No host synchronisation. */
+ *   workspace    device, at least mkv_decode_workspace_bytes(cfg, B) bytes; two decode calls that
+ *                overlap on the GPU need two buffers
+ * Two launches: a persistent split-KV scan, and a small kernel that merges the partials of rows
+ * that were split over several blocks with Eq. (softmax-merge).  No host synchronisation. */
 int32_t mkv_decode_attention(mkv_pool* pool, const void* q_dev, const int32_t* block_table_dev,
                              const uint8_t* tier_tag_dev, const int32_t* seq_lens_dev, int32_t B,
                              int32_t max_pages, float scale, float* out_dev, float* lse_dev,

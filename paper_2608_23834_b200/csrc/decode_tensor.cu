@@ -21,8 +21,8 @@
 //     MMA against a matrix of ones.  TQ3 values enter that MMA as their integer codes; the
 //     per-channel fp16 scale and zero of the page are applied to the 16x8 result in fp32.
 //   * partial results of a block that covers only part of a (request, KV head) row go to the
-//     workspace; the last block to arrive for that row (atomic ticket) merges them.  Nothing spins
-//     on another block.
+//     workspace; a small merge kernel launched right behind the scan combines them.  No block ever
+//     waits for another.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <math_constants.h>
@@ -58,7 +58,6 @@ struct DecodeParams {
     float scale;
     float* out;
     float* lse;
-    uint32_t* tickets;     // [B * hkv], zero on entry, zero on exit
     float* partials;       // [2 * grid][8*D + 16]
     uint32_t* status;
 };
@@ -227,38 +226,32 @@ __device__ __forceinline__ void affine_accumulate(float (&acc)[4], const float (
 // ------------------------------------------------------------------------------------------------
 // kernel
 // ------------------------------------------------------------------------------------------------
-// NW warps form NU = NW / HALVES units.  A unit owns a ring and processes one page at a time; with
-// HALVES == 2 the two warps of a unit split the head dimension (key blocks for the scores, channel
-// blocks for the output), exchange their partial scores through shared memory and each keep half of
-// the accumulators, which halves the registers per thread.
-template <int D, int NW, int NSTAGE, int HALVES>
+constexpr int kRound = 128;          // pages of one warp whose table entries are compacted at a time
+
+template <int D, int NW, int NSTAGE>
 struct Geo {
-    static constexpr int NU = NW / HALVES;
     static constexpr int NB = D / 16;                       // 16-wide blocks along d
     static constexpr int LW = 3 * NB / 4;                   // packed words per lane and code section
     static constexpr int TQ3_REC = 16 * D + 32;
     static constexpr int FP8_HALF = 16 * D;
     static constexpr int SLOT = (TQ3_REC + 127) / 128 * 128;
-    static constexpr int RING = NU * NSTAGE * SLOT;
-    static constexpr int QFRAG = NB * 32 * 8;               // one set of query B fragments
+    static constexpr int RING = NW * NSTAGE * SLOT;
+    static constexpr int QROT = NB * 32 * 16;               // rotated query B fragments, hi and lo interleaved
+    static constexpr int QPLAIN = NB * 32 * 8;              // plain query B fragments (FP8 pages)
     static constexpr int OFF_QT = RING;
-    static constexpr int OFF_QL = OFF_QT + QFRAG;            // low-order halves of the rotated query
-    static constexpr int OFF_QF = OFF_QL + QFRAG;
-    static constexpr int OFF_BAR = OFF_QF + QFRAG;
-    static constexpr int OFF_XCH = OFF_BAR + NU * NSTAGE * 8;   // [unit][parity][half][lane] float4
-    static constexpr int OFF_CUM = OFF_XCH + NU * 2 * 2 * 512;
+    static constexpr int OFF_QF = OFF_QT + QROT;
+    static constexpr int OFF_BAR = OFF_QF + QPLAIN;
+    static constexpr int OFF_LIST = OFF_BAR + NW * NSTAGE * 8;   // [warp][2 formats][kRound] page ids
+    static constexpr int OFF_CUM = OFF_LIST + NW * 2 * kRound * 4;
     static constexpr int OFF_STRIDE = OFF_CUM + (kMaxBatch + 1) * 4;
     static constexpr int OFF_M = OFF_STRIDE + kMaxBatch * 4;
     static constexpr int OFF_L = OFF_M + NW * 8 * 4;
     static constexpr int OFF_FLAG = OFF_L + NW * 8 * 4;
     static constexpr int SMEM = OFF_FLAG + 16;
-    static_assert(HALVES == 1 || (HALVES == 2 && D == 256), "the head dimension is split only for d = 256");
-    static_assert(HALVES == 1 || NSTAGE == 4, "a two-warp unit returns slots one page late: an FP8 page needs 2 + 2 slots");
     static_assert(NW >= 8, "one warp per column of the 8-wide head group builds the query fragments");
     static_assert(NSTAGE == 2 || NSTAGE == 4, "ring positions are taken modulo a power of two; an FP8 page takes two slots");
     static_assert(NSTAGE * SLOT >= 8 * D * 4, "ring doubles as the cross-warp reduction buffer");
     static_assert(FP8_HALF <= SLOT, "half an FP8 record fits a slot");
-    static_assert(RING >= kMaxCtas * 4 + 2 * kMaxCtas * 8 * 4, "ring doubles as the final-merge scratch");
 };
 
 #ifdef MKV_TIMELINE
@@ -298,9 +291,13 @@ struct WarpAcc {
 // Updates the running maximum (only when it is exceeded by more than 2^kRescaleSlack, so that
 // accumulators are rarely rescaled), and returns P^T as MMA B fragments split into an fp16 pair
 // hi (pb) + lo (pc), plus the page's row sums ps[0..1].
+struct PFrag {
+    uint32_t b0, b1, c0, c1;
+    float ps0, ps1;
+};
+
 template <int NB>
-__device__ __forceinline__ void softmax_page(WarpAcc<NB>& acc, const float (&s)[4], uint32_t& pb0, uint32_t& pb1,
-                                             uint32_t& pc0, uint32_t& pc1, float (&ps)[4])
+__device__ __forceinline__ void softmax_page(WarpAcc<NB>& acc, const float (&s)[4], PFrag& pf)
 {
     constexpr uint32_t FULL = 0xffffffffu;
     float mx0 = fmaxf(s[0], s[2]), mx1 = fmaxf(s[1], s[3]);
@@ -326,175 +323,146 @@ __device__ __forceinline__ void softmax_page(WarpAcc<NB>& acc, const float (&s)[
     const float p2 = fast_exp2(s[2] - acc.m[0]), p3 = fast_exp2(s[3] - acc.m[1]);
     const uint32_t ph01 = pack_f16x2(p0, p1), ph23 = pack_f16x2(p2, p3);
     const float2 h01 = half2_to_float2(ph01), h23 = half2_to_float2(ph23);
-    pb0 = movmatrix_trans(ph01);
-    pb1 = movmatrix_trans(ph23);
-    pc0 = movmatrix_trans(pack_f16x2(p0 - h01.x, p1 - h01.y));
-    pc1 = movmatrix_trans(pack_f16x2(p2 - h23.x, p3 - h23.y));
+    pf.b0 = movmatrix_trans(ph01);
+    pf.b1 = movmatrix_trans(ph23);
+    pf.c0 = movmatrix_trans(pack_f16x2(p0 - h01.x, p1 - h01.y));
+    pf.c1 = movmatrix_trans(pack_f16x2(p2 - h23.x, p3 - h23.y));
     // row sums through the tensor core: the same P that multiplies V
     const uint32_t ones[4] = {0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u};
-    mma16816_zero(ps, ones, pb0, pb1);
-    mma16816(ps, ones, pc0, pc1);
+    float ps[4];
+    mma16816_zero(ps, ones, pf.b0, pf.b1);
+    mma16816(ps, ones, pf.c0, pf.c1);
+    pf.ps0 = ps[0];
+    pf.ps1 = ps[1];
     acc.l[0] += ps[0];
     acc.l[1] += ps[1];
 }
 
-// The packed words of one lane for one code section: all of them (HALVES == 1) or the half that
-// belongs to warp half hf (d = 256: words 0..5 or 6..11 of the lane's 12).
-template <int D, int HALVES>
-__device__ __forceinline__ void load_lane_words(uint32_t sec, int lane, int hf, uint32_t (&w)[3 * (D / 16) / 4 / HALVES])
+// All packed words of one lane for one code section.
+template <int D>
+__device__ __forceinline__ void load_lane_words(uint32_t sec, int lane, uint32_t (&w)[3 * (D / 16) / 4])
 {
     constexpr int LW = 3 * (D / 16) / 4;
-    if constexpr (HALVES == 1) {
 #pragma unroll
-        for (int c = 0; c < LW / 4; ++c) {
-            const uint4 v = lds128(sec + c * 512 + lane * 16);
-            w[4 * c] = v.x; w[4 * c + 1] = v.y; w[4 * c + 2] = v.z; w[4 * c + 3] = v.w;
-        }
-        if constexpr (LW % 4 != 0) {
-            const uint2 v = lds64(sec + (LW / 4) * 512 + lane * 8);
-            w[LW - 2] = v.x; w[LW - 1] = v.y;
-        }
-    } else {
-        if (hf == 0) {
-            const uint4 v = lds128(sec + lane * 16);
-            const uint2 u = lds64(sec + 512 + lane * 16);
-            w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w; w[4] = u.x; w[5] = u.y;
-        } else {
-            const uint2 u = lds64(sec + 512 + lane * 16 + 8);
-            const uint4 v = lds128(sec + 1024 + lane * 16);
-            w[0] = u.x; w[1] = u.y; w[2] = v.x; w[3] = v.y; w[4] = v.z; w[5] = v.w;
-        }
+    for (int c = 0; c < LW / 4; ++c) {
+        const uint4 v = lds128(sec + c * 512 + lane * 16);
+        w[4 * c] = v.x; w[4 * c + 1] = v.y; w[4 * c + 2] = v.z; w[4 * c + 3] = v.w;
+    }
+    if constexpr (LW % 4 != 0) {
+        const uint2 v = lds64(sec + (LW / 4) * 512 + lane * 8);
+        w[LW - 2] = v.x; w[LW - 1] = v.y;
     }
 }
 
-// Pair exchange of partial scores (HALVES == 2): each warp stores its four partial sums, the two
-// warps meet at their named barrier, and both form the same total.
-struct PairCtx {
-    uint32_t xch;       // shared address of this unit's exchange area [parity][half][lane] float4
-    int bar_id;         // named barrier of the unit
-    int hf;             // which half this warp is
-    uint32_t parity;    // toggles every page
-};
-
-template <int HALVES>
-__device__ __forceinline__ void pair_sum(float (&S)[4], PairCtx& px, int lane)
+// Scores of the four key blocks 4j..4j+3 of a Stale page: 12 byte-table lookups per block pair and two
+// MMAs per block (query hi and lo).
+__device__ __forceinline__ void tq3_key_quad(float (&S0)[4], float (&S1)[4], uint32_t A, uint32_t Bw, uint32_t Cw,
+                                             uint32_t q_quad)
 {
-    if constexpr (HALVES == 2) {
-        const uint32_t mine = px.xch + ((px.parity * 2 + px.hf) * 32 + lane) * 16;
-        const uint32_t other = px.xch + ((px.parity * 2 + (px.hf ^ 1)) * 32 + lane) * 16;
-        asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(mine), "f"(S[0]), "f"(S[1]), "f"(S[2]), "f"(S[3]) : "memory");
-        asm volatile("bar.sync %0, 64;" ::"r"(px.bar_id) : "memory");
-        float o0, o1, o2, o3;
-        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(o0), "=f"(o1), "=f"(o2), "=f"(o3) : "r"(other));
-        S[0] += o0; S[1] += o1; S[2] += o2; S[3] += o3;
-        px.parity ^= 1u;
-    }
-}
-
-// One Stale page: record at shared address rec (key codes, value codes, g, scale/zero).
-template <int D, int HALVES>
-__device__ __forceinline__ void tq3_page(WarpAcc<D / 16 / HALVES>& acc, uint32_t rec, uint32_t qt_lane, float sc2, int lane,
-                                         PairCtx& px)
-{
-    constexpr int NB = D / 16, NBH = NB / HALVES, LWH = 3 * NB / 4 / HALVES, NT = NB / 4 / HALVES, QFRAG = NB * 32 * 8;
-    const int g = lane >> 2;
-    const int j0 = HALVES == 2 ? px.hf * NT : 0;     // first word triple / block quad of this warp
-    // ---- S = K q'^T
-    float S0[4] = {0.f, 0.f, 0.f, 0.f}, S1[4] = {0.f, 0.f, 0.f, 0.f};
-    {
-        uint32_t kw[LWH];
-        load_lane_words<D, HALVES>(rec, lane, px.hf, kw);
-        const uint32_t qt_half = qt_lane + j0 * 4 * 256;
+    uint32_t sel[4];
+    sel[0] = A & 0x77777777u;
+    sel[1] = Bw & 0x77777777u;
+    sel[2] = lop3_and_or(A >> 1, 0x44444444u, Cw & 0x33333333u);
+    sel[3] = lop3_and_or(Bw >> 1, 0x44444444u, (Cw >> 2) & 0x33333333u);
 #pragma unroll
-        for (int j = 0; j < NT; ++j) {
-            const uint32_t A = kw[3 * j], Bw = kw[3 * j + 1], Cw = kw[3 * j + 2];
-            uint32_t sel[4];
-            sel[0] = A & 0x77777777u;
-            sel[1] = Bw & 0x77777777u;
-            sel[2] = lop3_and_or(A >> 1, 0x44444444u, Cw & 0x33333333u);
-            sel[3] = lop3_and_or(Bw >> 1, 0x44444444u, (Cw >> 2) & 0x33333333u);
-#pragma unroll
-            for (int w = 0; w < 4; ++w) {
-                uint32_t a[4];
-                key_lut4(sel[w], a[0], a[1]);
-                key_lut4(sel[w] >> 16, a[2], a[3]);
-                const uint2 qv = lds64(qt_half + (4 * j + w) * 256);
-                const uint2 qw = lds64(qt_half + QFRAG + (4 * j + w) * 256);
-                if (w & 1) { mma16816(S1, a, qv.x, qv.y); mma16816(S1, a, qw.x, qw.y); }
-                else       { mma16816(S0, a, qv.x, qv.y); mma16816(S0, a, qw.x, qw.y); }
-            }
-        }
-    }
-    float St[4] = {S0[0] + S1[0], S0[1] + S1[1], S0[2] + S1[2], S0[3] + S1[3]};
-    pair_sum<HALVES>(St, px, lane);
-    const uint32_t gaddr = rec + 12 * D;
-    const float r0 = __half2float(__ushort_as_half(lds16(gaddr + 2 * g))) * sc2;
-    const float r1 = __half2float(__ushort_as_half(lds16(gaddr + 2 * g + 16))) * sc2;
-    const float s[4] = {St[0] * r0, St[1] * r0, St[2] * r1, St[3] * r1};
-    uint32_t pb0, pb1, pc0, pc1;
-    float ps[4];
-    softmax_page<NBH>(acc, s, pb0, pb1, pc0, pc1, ps);
-
-    // ---- O^T += V^T P with integer codes; scale and zero applied to the 16x8 result in fp32
-    uint32_t vw[LWH];
-    load_lane_words<D, HALVES>(rec + 6 * D, lane, px.hf, vw);
-    const uint32_t meta = rec + 12 * D + 32 + g * 16 + j0 * 2 * 128;
-#pragma unroll
-    for (int j = 0; j < NT; ++j) {
-        const uint32_t W0 = vw[3 * j], W1 = vw[3 * j + 1], W2 = vw[3 * j + 2];
-        float t[4];
+    for (int w = 0; w < 4; ++w) {
         uint32_t a[4];
-        {   // blocks 4j, 4j+1
-            const uint4 mt = lds128(meta + (2 * j) * 128);
-            const uint32_t X1 = prmt(W0, W1, 0x6341u);
-            a[0] = value_code<0>(W0);
-            a[1] = value_code<3>(W0);
-            a[2] = value_code<6>(W0);
-            a[3] = value_code<1>(X1);
-            mma16816_zero(t, a, pb0, pb1);
-            mma16816(t, a, pc0, pc1);
-            affine_accumulate(acc.o[4 * j], t, mt.x, mt.y, ps[0], ps[1]);
-            a[0] = value_code<4>(X1);
-            a[1] = value_code<7>(X1);
-            a[2] = value_code<2>(W1);
-            a[3] = value_code<5>(W1);
-            mma16816_zero(t, a, pb0, pb1);
-            mma16816(t, a, pc0, pc1);
-            affine_accumulate(acc.o[4 * j + 1], t, mt.z, mt.w, ps[0], ps[1]);
-        }
-        {   // blocks 4j+2, 4j+3
-            const uint4 mt = lds128(meta + (2 * j + 1) * 128);
-            const uint32_t X0 = prmt(W1, W2, 0x6341u), X2 = W2 >> 8;
-            a[0] = value_code<0>(X0);
-            a[1] = value_code<3>(X0);
-            a[2] = value_code<6>(X0);
-            a[3] = value_code<1>(W2);
-            mma16816_zero(t, a, pb0, pb1);
-            mma16816(t, a, pc0, pc1);
-            affine_accumulate(acc.o[4 * j + 2], t, mt.x, mt.y, ps[0], ps[1]);
-            a[0] = value_code<4>(W2);
-            a[1] = value_code<7>(W2);
-            a[2] = value_code<2>(X2);
-            a[3] = value_code<5>(X2);
-            mma16816_zero(t, a, pb0, pb1);
-            mma16816(t, a, pc0, pc1);
-            affine_accumulate(acc.o[4 * j + 3], t, mt.z, mt.w, ps[0], ps[1]);
-        }
+        key_lut4(sel[w], a[0], a[1]);
+        key_lut4(sel[w] >> 16, a[2], a[3]);
+        const uint4 q = lds128(q_quad + w * 512);          // {hi b0, hi b1, lo b0, lo b1}
+        if (w & 1) { mma16816(S1, a, q.x, q.y); mma16816(S1, a, q.z, q.w); }
+        else       { mma16816(S0, a, q.x, q.y); mma16816(S0, a, q.z, q.w); }
+    }
+}
+
+// Output update of the four channel blocks 4j..4j+3 of a Stale page: integer codes through the tensor
+// core, then the fp16 scale and zero of every channel applied to the 16x8 result in fp32.
+__device__ __forceinline__ void tq3_value_quad(float (&o0)[4], float (&o1)[4], float (&o2)[4], float (&o3)[4],
+                                               uint32_t W0, uint32_t W1, uint32_t W2, uint32_t meta_quad, const PFrag& pf)
+{
+    float t[4];
+    uint32_t a[4];
+    {   // blocks 4j, 4j+1
+        const uint4 mt = lds128(meta_quad);
+        const uint32_t X1 = prmt(W0, W1, 0x6341u);
+        a[0] = value_code<0>(W0);
+        a[1] = value_code<3>(W0);
+        a[2] = value_code<6>(W0);
+        a[3] = value_code<1>(X1);
+        mma16816_zero(t, a, pf.b0, pf.b1);
+        mma16816(t, a, pf.c0, pf.c1);
+        affine_accumulate(o0, t, mt.x, mt.y, pf.ps0, pf.ps1);
+        a[0] = value_code<4>(X1);
+        a[1] = value_code<7>(X1);
+        a[2] = value_code<2>(W1);
+        a[3] = value_code<5>(W1);
+        mma16816_zero(t, a, pf.b0, pf.b1);
+        mma16816(t, a, pf.c0, pf.c1);
+        affine_accumulate(o1, t, mt.z, mt.w, pf.ps0, pf.ps1);
+    }
+    {   // blocks 4j+2, 4j+3
+        const uint4 mt = lds128(meta_quad + 128);
+        const uint32_t X0 = prmt(W1, W2, 0x6341u), X2 = W2 >> 8;
+        a[0] = value_code<0>(X0);
+        a[1] = value_code<3>(X0);
+        a[2] = value_code<6>(X0);
+        a[3] = value_code<1>(W2);
+        mma16816_zero(t, a, pf.b0, pf.b1);
+        mma16816(t, a, pf.c0, pf.c1);
+        affine_accumulate(o2, t, mt.x, mt.y, pf.ps0, pf.ps1);
+        a[0] = value_code<4>(W2);
+        a[1] = value_code<7>(W2);
+        a[2] = value_code<2>(X2);
+        a[3] = value_code<5>(X2);
+        mma16816_zero(t, a, pf.b0, pf.b1);
+        mma16816(t, a, pf.c0, pf.c1);
+        affine_accumulate(o3, t, mt.z, mt.w, pf.ps0, pf.ps1);
+    }
+}
+
+// Software-pipelined step over Stale pages: the value phase of the current page (record rec_v, its
+// probabilities pf) and the score phase of the next page (record rec_k) are issued quad by quad in
+// one instruction stream, so that table lookups, half-precision FMAs, fp32 FMAs and MMAs of the two
+// phases overlap.  DO_V / DO_K switch the halves off for the first and the last page.
+template <int D, bool DO_V, bool DO_K>
+__device__ __forceinline__ void tq3_step(WarpAcc<D / 16>& acc, uint32_t rec_v, const PFrag& pf, uint32_t rec_k,
+                                         uint32_t qt_lane, float sc2, int lane, float (&s_next)[4])
+{
+    constexpr int NB = D / 16, LW = 3 * NB / 4;
+    const int g = lane >> 2;
+    uint32_t kw[LW], vw[LW];
+    float S0[4] = {0.f, 0.f, 0.f, 0.f}, S1[4] = {0.f, 0.f, 0.f, 0.f};
+    if constexpr (DO_K) load_lane_words<D>(rec_k, lane, kw);
+    if constexpr (DO_V) load_lane_words<D>(rec_v + 6 * D, lane, vw);
+    const uint32_t meta = rec_v + 12 * D + 32 + g * 16;
+#pragma unroll
+    for (int j = 0; j < NB / 4; ++j) {
+        if constexpr (DO_K) tq3_key_quad(S0, S1, kw[3 * j], kw[3 * j + 1], kw[3 * j + 2], qt_lane + j * 2048);
+        if constexpr (DO_V)
+            tq3_value_quad(acc.o[4 * j], acc.o[4 * j + 1], acc.o[4 * j + 2], acc.o[4 * j + 3], vw[3 * j], vw[3 * j + 1],
+                           vw[3 * j + 2], meta + j * 256, pf);
+    }
+    if constexpr (DO_K) {
+        const uint32_t gaddr = rec_k + 12 * D;
+        const float r0 = __half2float(__ushort_as_half(lds16(gaddr + 2 * g))) * sc2;
+        const float r1 = __half2float(__ushort_as_half(lds16(gaddr + 2 * g + 16))) * sc2;
+        s_next[0] = (S0[0] + S1[0]) * r0;
+        s_next[1] = (S0[1] + S1[1]) * r0;
+        s_next[2] = (S0[2] + S1[2]) * r1;
+        s_next[3] = (S0[3] + S1[3]) * r1;
     }
 }
 
 // One Recent/Anchor page: keys [16 tokens][d] e4m3 at kaddr, values [d channels][16 tokens] at vaddr.
-template <int D, int HALVES>
-__device__ __forceinline__ void fp8_page(WarpAcc<D / 16 / HALVES>& acc, uint32_t kaddr, uint32_t vaddr, uint32_t qf_lane,
-                                         float score_scale, float v_scale, int valid, int lane, PairCtx& px)
+template <int D>
+__device__ __forceinline__ void fp8_page(WarpAcc<D / 16>& acc, uint32_t kaddr, uint32_t vaddr, uint32_t qf_lane,
+                                         float score_scale, float v_scale, int valid, int lane)
 {
-    constexpr int NB = D / 16, NBH = NB / HALVES, NJ = D / 64 / HALVES;
+    constexpr int NB = D / 16;
     const int g = lane >> 2, tq = lane & 3;
-    const int jj0 = HALVES == 2 ? px.hf * NJ : 0, cb0 = HALVES == 2 ? px.hf * NBH : 0;
     float S0[4] = {0.f, 0.f, 0.f, 0.f}, S1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-    for (int jl = 0; jl < NJ; ++jl) {
-        const int j = jj0 + jl;
+    for (int j = 0; j < D / 64; ++j) {
         const uint4 r0 = lds128(kaddr + g * D + 64 * j + 16 * tq);
         const uint4 r1 = lds128(kaddr + (g + 8) * D + 64 * j + 16 * tq);
         const uint32_t w0[4] = {r0.x, r0.y, r0.z, r0.w}, w1[4] = {r1.x, r1.y, r1.z, r1.w};
@@ -510,9 +478,8 @@ __device__ __forceinline__ void fp8_page(WarpAcc<D / 16 / HALVES>& acc, uint32_t
             else       mma16816(S0, a, qv.x, qv.y);
         }
     }
-    float St[4] = {S0[0] + S1[0], S0[1] + S1[1], S0[2] + S1[2], S0[3] + S1[3]};
-    pair_sum<HALVES>(St, px, lane);
-    float s[4] = {St[0] * score_scale, St[1] * score_scale, St[2] * score_scale, St[3] * score_scale};
+    float s[4] = {(S0[0] + S1[0]) * score_scale, (S0[1] + S1[1]) * score_scale, (S0[2] + S1[2]) * score_scale,
+                  (S0[3] + S1[3]) * score_scale};
     // bytes of tokens beyond the sequence end are cleared so that stale NaN patterns cannot leak
     uint32_t keep_lo = 0xFFFFu, keep_hi = 0xFFFFu;   // byte masks for tokens (2tq,2tq+1), (2tq+8,2tq+9)
     if (valid < kPage) {
@@ -521,13 +488,12 @@ __device__ __forceinline__ void fp8_page(WarpAcc<D / 16 / HALVES>& acc, uint32_t
         keep_lo = (2 * tq < valid ? 0x00FFu : 0u) | (2 * tq + 1 < valid ? 0xFF00u : 0u);
         keep_hi = (2 * tq + 8 < valid ? 0x00FFu : 0u) | (2 * tq + 9 < valid ? 0xFF00u : 0u);
     }
-    uint32_t pb0, pb1, pc0, pc1;
-    float ps[4];
-    softmax_page<NBH>(acc, s, pb0, pb1, pc0, pc1, ps);
+    PFrag pf;
+    softmax_page<NB>(acc, s, pf);
     const bool scale_v = v_scale != 1.0f;
 #pragma unroll
-    for (int cb = 0; cb < NBH; ++cb) {
-        const uint32_t r0 = vaddr + (16 * (cb0 + cb) + g) * 16 + 2 * tq, r1 = r0 + 8 * 16;
+    for (int cb = 0; cb < NB; ++cb) {
+        const uint32_t r0 = vaddr + (16 * cb + g) * 16 + 2 * tq, r1 = r0 + 8 * 16;
         uint32_t a[4];
         a[0] = e4m3x2_to_f16x2((uint16_t)(lds16(r0) & keep_lo));
         a[1] = e4m3x2_to_f16x2((uint16_t)(lds16(r1) & keep_lo));
@@ -535,26 +501,27 @@ __device__ __forceinline__ void fp8_page(WarpAcc<D / 16 / HALVES>& acc, uint32_t
         a[3] = e4m3x2_to_f16x2((uint16_t)(lds16(r1 + 8) & keep_hi));
         if (scale_v) {
             float t[4];
-            mma16816_zero(t, a, pb0, pb1);
-            mma16816(t, a, pc0, pc1);
+            mma16816_zero(t, a, pf.b0, pf.b1);
+            mma16816(t, a, pf.c0, pf.c1);
 #pragma unroll
             for (int e = 0; e < 4; ++e) acc.o[cb][e] = fmaf(v_scale, t[e], acc.o[cb][e]);
         } else {
-            mma16816(acc.o[cb], a, pb0, pb1);
-            mma16816(acc.o[cb], a, pc0, pc1);
+            mma16816(acc.o[cb], a, pf.b0, pf.b1);
+            mma16816(acc.o[cb], a, pf.c0, pf.c1);
         }
     }
 }
 
-template <int D, int NW, int NSTAGE, int MINB, int HALVES>
+template <int D, int NW, int NSTAGE, int MINB>
 __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const DecodeParams P)
 {
 #ifdef MKV_TIMELINE
     unsigned long long tl_last = 0;
 #endif
     MKV_STAMP(0);
-    using G = Geo<D, NW, NSTAGE, HALVES>;
-    constexpr int NB = G::NB, NBH = NB / HALVES, NU = G::NU;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    using G = Geo<D, NW, NSTAGE>;
+    constexpr int NB = G::NB, NBH = NB, NU = NW;
     constexpr uint32_t FULL = 0xffffffffu;
     extern __shared__ __align__(128) uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
@@ -563,15 +530,15 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
     float* sm_m = reinterpret_cast<float*>(smem + G::OFF_M);
     float* sm_l = reinterpret_cast<float*>(smem + G::OFF_L);
     int* sm_flag = reinterpret_cast<int*>(smem + G::OFF_FLAG);
-    float* red = reinterpret_cast<float*>(smem);            // [NU][D][8] over the ring, between segments
+    float* red = reinterpret_cast<float*>(smem);            // [NW][D][8] over the ring, between segments
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tq = lane & 3;
-    const int unit = warp / HALVES, hf = warp % HALVES;
+    const int unit = warp, hf = 0;
     const int hkv = P.hkv, GQ = P.group, hq = hkv * GQ;
 
-    // ---- prologue: barriers, zero rows of empty requests, prefix of pages -----------------------
+    // ---- prologue: barriers, zero rows of empty requests, prefix of pages, page strides ---------
     if (tid == 0) {
-        for (int i = 0; i < NU * NSTAGE; ++i) mbar_init(sbase + G::OFF_BAR + 8 * i, 1);
+        for (int i = 0; i < NW * NSTAGE; ++i) mbar_init(sbase + G::OFF_BAR + 8 * i, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     for (int b = blockIdx.x; b < P.B; b += gridDim.x)
@@ -628,24 +595,14 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
     };
     const int my_start = range_start(blockIdx.x), my_end = range_start(blockIdx.x + 1);
 
-    // per-unit ring of NSTAGE slots: fill and drain positions, slots in flight, and one bit per slot with
-    // the mbarrier phase the next wait on it must see (flipped every time the slot is consumed); with two
-    // warps per unit both keep the same state and the first one issues the copies
-    uint32_t head = 0, tail = 0, in_flight = 0, phase = 0;
+    // per-warp ring of NSTAGE slots; one bit per slot holds the mbarrier phase the next wait must see
+    uint32_t phase = 0;
     bool failed = false;
-    const uint32_t ring = sbase + unit * NSTAGE * G::SLOT;
-    const uint32_t bars = sbase + G::OFF_BAR + unit * NSTAGE * 8;
-    PairCtx px;
-    px.xch = sbase + G::OFF_XCH + unit * 2048;
-    px.bar_id = 1 + unit;
-    px.hf = hf;
-    px.parity = 0;
-    const bool issuer = (hf == 0) && (lane == 0);
-    auto unit_sync = [&]() {
-        if constexpr (HALVES == 2) asm volatile("bar.sync %0, 64;" ::"r"(px.bar_id) : "memory");
-        else __syncwarp();
-    };
-    const uint32_t qt_lane = sbase + G::OFF_QT + lane * 8, qf_lane = sbase + G::OFF_QF + lane * 8;
+    const uint32_t ring = sbase + warp * NSTAGE * G::SLOT;
+    const uint32_t bars = sbase + G::OFF_BAR + warp * NSTAGE * 8;
+    const uint32_t qt_lane = sbase + G::OFF_QT + lane * 16, qf_lane = sbase + G::OFF_QF + lane * 8;
+    int* list3 = reinterpret_cast<int*>(smem + G::OFF_LIST) + warp * 2 * kRound;   // Stale page ids of the round
+    int* list8 = list3 + kRound;                                                   // FP8 page ids | valid << 27
     const float sc2 = P.scale * kLog2e;      // scores are kept in log2 units
     // bounded wait for ring slot s, then flip its expected phase
     auto wait_slot = [&](uint32_t s) {
@@ -674,7 +631,7 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
     int b = 0;
     MKV_STAMP(1);
     while (pos < my_end) {
-        // ---- locate the segment: request b, KV head h, pages [pg0, pg0 + n_seg) ---------------
+        // ---- locate the segment: request b, KV head h, positions [pg0, pg0 + n_seg) of the row ------
         while (cum[b + 1] <= pos) ++b;
         const int len = P.lens[b], n_pages = (len + kPage - 1) / kPage;
         const int h = (pos - cum[b]) / n_pages, pg0 = (pos - cum[b]) % n_pages;
@@ -682,85 +639,77 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
         const int n_seg = min(my_end, row_end) - pos;
         const int32_t* bt_row = P.bt + (size_t)b * P.max_pages;
         const uint8_t* tag_row = P.tags + (size_t)b * P.max_pages;
-        const int n_my = unit < n_seg ? (n_seg - unit + NU - 1) / NU : 0;   // this unit's pages, round-robin
+        const int n_my = warp < n_seg ? (n_seg - warp + NW - 1) / NW : 0;   // this warp's pages, round-robin
         const int stride = strides[b];
         constexpr int EPL = D / 32;
         float qx[EPL];            // this warp's query head (warps 0..7), loaded before anything else waits
 #pragma unroll
         for (int r = 0; r < EPL; ++r)
             qx[r] = (warp < GQ) ? __bfloat162float(P.q[((size_t)b * hq + h * GQ + warp) * D + lane * EPL + r]) : 0.f;
-        auto page_at = [&](int i) -> int { return (int)(((unsigned)(pg0 + i) * (unsigned)stride) % (unsigned)n_pages); };
+        const uint8_t* tq3_base = P.tq3 + (size_t)h * G::TQ3_REC;
+        const uint8_t* fp8_base = P.fp8 + (size_t)h * (2 * G::FP8_HALF);
 
-        // A walker enumerates, in order, the warp's pages of one format: 32 table entries at a time are
-        // loaded (entry i in lane i) and the matching ones are visited through a ballot mask.
-        struct Walker {
-            int chunk;
-            uint32_t mask;
-            int id;
-        };
-        auto walker_load = [&](Walker& w, int want_tq3) {
-            const int i = w.chunk * 32 + lane;
-            int kind = 0;
-            w.id = 0;
-            if (i < n_my) {
-                const int pg = page_at(unit + NU * i);
-                const int id = bt_row[pg], tag = tag_row[pg];
-                const int valid = min(kPage, len - pg * kPage);
-                if (tag == MKV_TAG_STALE)
-                    kind = (id >= 0 && id < P.tq3_pages && valid == kPage) ? 1 : 0;
-                else
-                    kind = (tag <= MKV_TAG_ANCHOR && id >= 0 && id < P.fp8_pages) ? 2 : 0;
-                if (kind == 0 && want_tq3 && hf == 0) atomicOr(P.status, kStBounds);    // flagged once (first pass)
-                w.id = id;
+        // Table entries of up to kRound of the warp's pages are compacted into two id lists, one per
+        // format (entry i of a 32-page chunk is read by lane i; ballots give the positions).
+        int n3 = 0, n8 = 0;
+        auto build_lists = [&](int round) {
+            n3 = n8 = 0;
+#pragma unroll 1
+            for (int c = 0; c < kRound / 32; ++c) {
+                const int i = round * kRound + c * 32 + lane;
+                int kind = 0, id = 0, valid = kPage;
+                if (i < n_my) {
+                    const int pg = (int)(((unsigned)(pg0 + warp + NW * i) * (unsigned)stride) % (unsigned)n_pages);
+                    id = bt_row[pg];
+                    const int tag = tag_row[pg];
+                    valid = min(kPage, len - pg * kPage);
+                    if (tag == MKV_TAG_STALE)
+                        kind = (id >= 0 && id < P.tq3_pages && valid == kPage) ? 1 : 0;
+                    else
+                        kind = (tag <= MKV_TAG_ANCHOR && id >= 0 && id < P.fp8_pages) ? 2 : 0;
+                    if (kind == 0) atomicOr(P.status, kStBounds);     // never dereferenced
+                }
+                const uint32_t m3 = __ballot_sync(FULL, kind == 1), m8 = __ballot_sync(FULL, kind == 2);
+                const uint32_t lt = (1u << lane) - 1u;
+                if (kind == 1) list3[n3 + __popc(m3 & lt)] = id;
+                if (kind == 2) list8[n8 + __popc(m8 & lt)] = id | ((valid & 15) << 27);
+                n3 += __popc(m3);
+                n8 += __popc(m8);
             }
-            w.mask = __ballot_sync(FULL, kind == (want_tq3 ? 1 : 2));
+            __syncwarp();
         };
-        // next matching page: returns false at the end; j = index inside the chunk
-        auto walker_next = [&](Walker& w, int want_tq3, int& id, int& index) -> bool {
-            while (w.mask == 0) {
-                if ((w.chunk + 1) * 32 >= n_my) return false;
-                ++w.chunk;
-                walker_load(w, want_tq3);
+        auto issue_tq3 = [&](int i) {      // copy Stale page i of the round into ring slot i % NSTAGE
+            if (lane == 0) {
+                const uint32_t s = i & (NSTAGE - 1);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                mbar_expect_tx(bars + 8 * s, G::TQ3_REC);
+                bulk_load(ring + s * G::SLOT, tq3_base + (size_t)list3[i] * hkv * G::TQ3_REC, G::TQ3_REC, bars + 8 * s);
             }
-            const int j = __ffs(w.mask) - 1;
-            w.mask &= w.mask - 1;
-            id = __shfl_sync(FULL, w.id, j);
-            index = w.chunk * 32 + j;
-            return true;
+        };
+        auto issue_fp8 = [&](int i) {      // copy FP8 page i of the round into the slot pair 2 (i % (NSTAGE/2))
+            if (lane == 0) {
+                const uint32_t s = (2 * i) & (NSTAGE - 1);
+                const uint8_t* rec = fp8_base + (size_t)(list8[i] & 0x7FFFFFF) * hkv * (2 * G::FP8_HALF);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                mbar_expect_tx(bars + 8 * s, G::FP8_HALF);
+                bulk_load(ring + s * G::SLOT, rec, G::FP8_HALF, bars + 8 * s);
+                mbar_expect_tx(bars + 8 * (s + 1), G::FP8_HALF);
+                bulk_load(ring + (s + 1) * G::SLOT, rec + G::FP8_HALF, G::FP8_HALF, bars + 8 * (s + 1));
+            }
         };
 
-        WarpAcc<NBH> acc;
+        WarpAcc<NB> acc;
 #pragma unroll
-        for (int i = 0; i < NBH; ++i) acc.o[i][0] = acc.o[i][1] = acc.o[i][2] = acc.o[i][3] = 0.f;
+        for (int i = 0; i < NB; ++i) acc.o[i][0] = acc.o[i][1] = acc.o[i][2] = acc.o[i][3] = 0.f;
         acc.l[0] = acc.l[1] = 0.f;
         acc.m[0] = acc.m[1] = -CUDART_INF_F;
 
-        // ---- pass over the Stale (TQ3) pages: start the copies, then build the query fragments -----
-        head = tail = 0;
-        Walker prod, cons;
-        prod.chunk = cons.chunk = 0;
-        prod.mask = cons.mask = 0;
-        prod.id = cons.id = 0;
-        bool prod_more = n_my > 0;
-        if (n_my > 0) {
-            walker_load(prod, 1);
-            cons = prod;
+        // first round: start the copies, then build the query fragments while they fly
+        const int n_rounds = (n_my + kRound - 1) / kRound;
+        if (n_rounds > 0) {
+            build_lists(0);
+            for (int i = 0; i < min(n3, NSTAGE); ++i) issue_tq3(i);
         }
-        auto produce_tq3 = [&]() {
-            while (prod_more && !failed && in_flight < NSTAGE) {
-                int id, index;
-                prod_more = walker_next(prod, 1, id, index);
-                if (!prod_more) break;
-                if (issuer) {
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    mbar_expect_tx(bars + 8 * head, G::TQ3_REC);
-                    bulk_load(ring + head * G::SLOT, P.tq3 + ((size_t)id * hkv + h) * G::TQ3_REC, G::TQ3_REC, bars + 8 * head);
-                }
-                head = (head + 1) & (NSTAGE - 1);
-                ++in_flight;
-            }
-        };
-        produce_tq3();
 
         // query fragments: warp hd < 8 rotates head hd (loads were issued before the copies started)
         if (warp < 8) {
@@ -789,19 +738,18 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                 }
             const float rs = rsqrtf((float)D);
             __half* qt = reinterpret_cast<__half*>(smem + G::OFF_QT);
-            __half* ql = reinterpret_cast<__half*>(smem + G::OFF_QL);
             __half* qf = reinterpret_cast<__half*>(smem + G::OFF_QF);
 #pragma unroll
             for (int r = 0; r < EPL; ++r) {
                 const int i = lane * EPL + r;
-                {   // rotated query, natural slot order: block i/16, slot s = i%16
+                {   // rotated query, natural slot order: block i/16, slot s = i%16; per lane {hi b0, hi b1, lo b0, lo b1}
                     const int kb = i >> 4, s = i & 15;
-                    const int at = (kb * 32 + 4 * hd + ((s & 7) >> 1)) * 4 + (s >> 3) * 2 + (s & 1);
+                    const int at = (kb * 32 + 4 * hd + ((s & 7) >> 1)) * 8 + (s >> 3) * 2 + (s & 1);
                     // fp16 pair hi + lo carries the rotated query to ~2^-22
                     const float v = a[r] * rs;
                     const __half vh = __float2half_rn(v);
                     qt[at] = vh;
-                    ql[at] = __float2half_rn(v - __half2float(vh));
+                    qt[at + 4] = __float2half_rn(v - __half2float(vh));
                 }
                 {   // plain query in the slot order of the FP8 key loads: 16 consecutive dims per lane
                     const int j = i >> 6, t4 = (i & 63) >> 4, wv = (i & 15) >> 2, e = i & 3;
@@ -812,83 +760,49 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
         __syncthreads();
         MKV_STAMP(2);
 
-        {
-            // With two warps per unit a slot is handed back one page late: the exchange barrier inside page
-            // n+1 is what proves that both warps have finished reading page n.
-            int id, index;
-            bool pending = false;
-            while (!failed && walker_next(cons, 1, id, index)) {
-                wait_slot(tail);
-                if (failed) break;
-#ifdef MKV_EXP_NOCOMPUTE
-                acc.l[0] += __uint_as_float(lds64(ring + tail * G::SLOT + lane * 8).x & 1u);
-                if constexpr (HALVES == 2) unit_sync();
-#else
-                tq3_page<D, HALVES>(acc, ring + tail * G::SLOT, qt_lane, sc2, lane, px);
-#endif
-                tail = (tail + 1) & (NSTAGE - 1);
-                if constexpr (HALVES == 2) {
-                    if (pending) --in_flight;
-                    pending = true;
-                } else {
-                    --in_flight;
+        for (int round = 0; round < n_rounds && !failed; ++round) {
+            if (round > 0) {
+                build_lists(round);
+                for (int i = 0; i < min(n3, NSTAGE); ++i) issue_tq3(i);
+            }
+            // ---- Stale pages: scores of page i+1 are computed together with the output update of page i
+            if (n3 > 0) {
+                float s_cur[4], s_next[4];
+                PFrag pf;
+                wait_slot(0);
+                if (!failed) tq3_step<D, false, true>(acc, 0, pf, ring, qt_lane, sc2, lane, s_cur);
+                for (int i = 0; i + 1 < n3 && !failed; ++i) {
+                    const uint32_t cur = i & (NSTAGE - 1), nxt = (i + 1) & (NSTAGE - 1);
+                    wait_slot(nxt);
+                    if (failed) break;
+                    softmax_page<NB>(acc, s_cur, pf);
+                    tq3_step<D, true, true>(acc, ring + cur * G::SLOT, pf, ring + nxt * G::SLOT, qt_lane, sc2, lane, s_next);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) s_cur[e] = s_next[e];
                     __syncwarp();
+                    if (i + NSTAGE < n3) issue_tq3(i + NSTAGE);
                 }
-                produce_tq3();
-            }
-            if constexpr (HALVES == 2) {
-                unit_sync();                  // both warps are done with the last page
-                if (pending) --in_flight;
-            }
-        }
-
-        // ---- pass over the Recent/Anchor (FP8) pages: two slots per page (keys, values) -------------
-        if (n_my > 0 && !failed) {
-            prod.chunk = 0;
-            walker_load(prod, 0);
-            cons = prod;
-            prod_more = true;
-            head = tail = 0;          // the ring is empty here; pairs sit at even positions
-            auto produce_fp8 = [&]() {
-                while (prod_more && !failed && in_flight + 2 <= NSTAGE) {
-                    int id, index;
-                    prod_more = walker_next(prod, 0, id, index);
-                    if (!prod_more) break;
-                    if (issuer) {
-                        const uint8_t* rec = P.fp8 + ((size_t)id * hkv + h) * (2 * G::FP8_HALF);
-                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                        mbar_expect_tx(bars + 8 * head, G::FP8_HALF);
-                        bulk_load(ring + head * G::SLOT, rec, G::FP8_HALF, bars + 8 * head);
-                        mbar_expect_tx(bars + 8 * (head + 1), G::FP8_HALF);
-                        bulk_load(ring + (head + 1) * G::SLOT, rec + G::FP8_HALF, G::FP8_HALF, bars + 8 * (head + 1));
-                    }
-                    head = (head + 2) & (NSTAGE - 1);
-                    in_flight += 2;
+                if (!failed) {
+                    softmax_page<NB>(acc, s_cur, pf);
+                    tq3_step<D, true, false>(acc, ring + ((n3 - 1) & (NSTAGE - 1)) * G::SLOT, pf, 0, qt_lane, sc2, lane, s_next);
                 }
-            };
-            produce_fp8();
-            int id, index;
-            bool pending = false;
-            while (!failed && walker_next(cons, 0, id, index)) {
-                wait_slot(tail);
-                wait_slot(tail + 1);
-                if (failed) break;
-                const int pg = page_at(unit + NU * index);
-                fp8_page<D, HALVES>(acc, ring + tail * G::SLOT, ring + (tail + 1) * G::SLOT, qf_lane, sc2 * P.k_scale,
-                                    P.v_scale, min(kPage, len - pg * kPage), lane, px);
-                tail = (tail + 2) & (NSTAGE - 1);
-                if constexpr (HALVES == 2) {
-                    if (pending) in_flight -= 2;
-                    pending = true;
-                } else {
-                    in_flight -= 2;
+                __syncwarp();
+            }
+            // ---- Recent/Anchor pages: two slots per page (keys, values)
+            if (n8 > 0 && !failed) {
+                for (int i = 0; i < min(n8, NSTAGE / 2); ++i) issue_fp8(i);
+                for (int i = 0; i < n8 && !failed; ++i) {
+                    const uint32_t s = (2 * i) & (NSTAGE - 1);
+                    wait_slot(s);
+                    wait_slot(s + 1);
+                    if (failed) break;
+                    const int e = list8[i];
+                    const int valid = (e >> 27) & 15;
+                    fp8_page<D>(acc, ring + s * G::SLOT, ring + (s + 1) * G::SLOT, qf_lane, sc2 * P.k_scale, P.v_scale,
+                                valid ? valid : kPage, lane);
                     __syncwarp();
+                    if (i + NSTAGE / 2 < n8) issue_fp8(i + NSTAGE / 2);
                 }
-                produce_fp8();
-            }
-            if constexpr (HALVES == 2) {
-                unit_sync();
-                if (pending) in_flight -= 2;
             }
         }
         float (&oacc)[NBH][4] = acc.o;
@@ -929,7 +843,6 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
 
         MKV_STAMP(5);
         const bool whole_row = (pos == row_start) && (pos + n_seg == row_end);
-        const int pair = b * hkv + h;
         if (whole_row) {
             for (int e = tid; e < 8 * D; e += NW * 32) {
                 const int head = e & 7, ch = e >> 3;
@@ -951,7 +864,8 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                 P.lse[(size_t)b * hq + h * GQ + tid] = l > 0.f ? (M + log2f(l)) * kLn2 : -CUDART_INF_F;
             }
         } else {
-            // partial (m, l, O) of this block for the row; slot 2c if the segment opens the block's range
+            // partial (m, l, O) of this block for the row, merged by the merge kernel that follows;
+            // slot 2c if the segment opens the block's range, 2c + 1 otherwise
             float* slot = P.partials + (size_t)(2 * blockIdx.x + (pos != my_start ? 1 : 0)) * (8 * D + 16);
             for (int e = tid; e < 8 * D; e += NW * 32) {
                 float acc = 0.f;
@@ -968,88 +882,6 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                 slot[8 * D + tid] = M;
                 slot[8 * D + 8 + tid] = l;
             }
-            __threadfence();
-            __syncthreads();
-            MKV_STAMP(6);
-            const int c0 = block_of(row_start), c1 = block_of(row_end - 1);
-            if (tid == 0) {
-                const uint32_t t = atomicAdd(&P.tickets[pair], 1u);
-                *sm_flag = (t == (uint32_t)(c1 - c0)) ? 1 : 0;
-            }
-            __syncthreads();
-            MKV_STAMP(7);
-            if (*sm_flag) {
-                // last block of the row: Eq. (softmax-merge) over the row's partials
-                __threadfence();
-                const int n_parts = c1 - c0 + 1;
-                int* pslot = reinterpret_cast<int*>(red);                 // [n_parts] slot index of each part
-                float* pm = red + kMaxCtas;                               // [n_parts][8] partial maxima
-                float* wts = pm + kMaxCtas * 8;                           // [n_parts][8] weights, then l
-                for (int c = tid; c < n_parts; c += NW * 32)
-                    pslot[c] = 2 * (c0 + c) + (row_start > range_start(c0 + c) ? 1 : 0);
-                __syncthreads();
-                for (int i = tid; i < n_parts * 8; i += NW * 32) {
-                    const float* ps = P.partials + (size_t)pslot[i >> 3] * (8 * D + 16) + 8 * D;
-                    const float lj = __ldcg(ps + 8 + (i & 7));
-                    pm[i] = lj > 0.f ? __ldcg(ps + (i & 7)) : -CUDART_INF_F;
-                    wts[i] = lj;
-                }
-                __syncthreads();
-                if (tid < 8) {
-                    float M = -CUDART_INF_F;
-                    for (int c = 0; c < n_parts; ++c) M = fmaxf(M, pm[c * 8 + tid]);
-                    sm_m[tid] = M;
-                }
-                __syncthreads();
-                for (int i = tid; i < n_parts * 8; i += NW * 32) {
-                    const float mj = pm[i];
-                    wts[i] = mj == -CUDART_INF_F ? 0.f : fast_exp2(mj - sm_m[i & 7]) * wts[i];   // w_j * l_j
-                    pm[i] = mj == -CUDART_INF_F ? 0.f : fast_exp2(mj - sm_m[i & 7]);              // w_j
-                }
-                __syncthreads();
-                if (tid < 8) {
-                    float L = 0.f;
-                    for (int c = 0; c < n_parts; ++c) L += wts[c * 8 + tid];
-                    sm_l[tid] = L;
-                }
-                __syncthreads();
-                // four consecutive heads of one channel per thread; the loads of 16 partials are issued
-                // together before any of them is used
-                for (int e4 = tid; e4 < 2 * D; e4 += NW * 32) {
-                    const int head0 = (e4 & 1) * 4, ch = e4 >> 1;
-                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                    for (int c0b = 0; c0b < n_parts; c0b += 16) {
-                        float4 v[16];
-#pragma unroll
-                        for (int k = 0; k < 16; ++k) {
-                            const int c = min(c0b + k, n_parts - 1);
-                            v[k] = __ldcg(reinterpret_cast<const float4*>(P.partials + (size_t)pslot[c] * (8 * D + 16)) + e4);
-                        }
-#pragma unroll
-                        for (int k = 0; k < 16; ++k) {
-                            if (c0b + k < n_parts) {
-                                const float4 w = *reinterpret_cast<const float4*>(pm + (c0b + k) * 8 + head0);
-                                acc.x = fmaf(w.x, v[k].x, acc.x);
-                                acc.y = fmaf(w.y, v[k].y, acc.y);
-                                acc.z = fmaf(w.z, v[k].z, acc.z);
-                                acc.w = fmaf(w.w, v[k].w, acc.w);
-                            }
-                        }
-                    }
-                    const float av[4] = {acc.x, acc.y, acc.z, acc.w};
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const int head = head0 + k;
-                        if (head < GQ) {
-                            const float L = sm_l[head];
-                            P.out[((size_t)b * hq + h * GQ + head) * D + ch] = L > 0.f ? av[k] / L : 0.f;
-                        }
-                    }
-                }
-                if (P.lse && tid < GQ)
-                    P.lse[(size_t)b * hq + h * GQ + tid] = sm_l[tid] > 0.f ? (sm_m[tid] + log2f(sm_l[tid])) * kLn2 : -CUDART_INF_F;
-                if (tid == 0) P.tickets[pair] = 0;         // leave the header clean for the next call
-            }
         }
         __syncthreads();
         MKV_STAMP(8);
@@ -1057,11 +889,132 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
     }
 }
 
-template <int D, int NW, int NSTAGE, int MINB, int HALVES>
+// Eq. (softmax-merge) for every (request, KV head) row that was split over several blocks of the scan
+// kernel: one block per row and half of the channels; a thread owns one channel and four heads, and
+// issues the loads of all partials before it uses any.  Rows that a single block covered were written
+// by that block and are skipped here.
+template <int D>
+__global__ void __launch_bounds__(D) decode_merge_kernel(const DecodeParams P, int scan_grid)
+{
+    constexpr uint32_t FULL = 0xffffffffu;
+    constexpr int kMaxParts = 40;          // loads in flight per thread; longer rows take several rounds
+    __shared__ int cum[kMaxBatch + 1];
+    __shared__ __align__(16) float w_s[kMaxCtas * 8];    // weight of every partial and head (read as float4)
+    __shared__ float l_s[kMaxCtas * 8];                  // row sums of every partial and head
+    __shared__ int slot_s[kMaxCtas];                     // workspace slot of every partial
+    __shared__ float ml_s[16];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int hkv = P.hkv, GQ = P.group, hq = hkv * GQ;
+    if (warp == 0) {
+        int run = 0;
+        for (int b0 = 0; b0 < P.B; b0 += 32) {
+            const int b = b0 + lane;
+            int n = 0;
+            if (b < P.B) {
+                const int len = P.lens[b];
+                n = len > 0 ? ((len + kPage - 1) / kPage) * hkv : 0;
+            }
+            int inc = n;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(FULL, inc, o);
+                if (lane >= o) inc += v;
+            }
+            if (b < P.B) cum[b] = run + inc - n;
+            run += __shfl_sync(FULL, inc, 31);
+        }
+        if (lane == 0) cum[P.B] = run;
+    }
+    __syncthreads();
+    const long long W = cum[P.B];
+    // everything above read only the call's inputs; the partials below are the scan kernel's output
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (W == 0) return;
+    const int C = (int)(W < (long long)scan_grid ? W : (long long)scan_grid);
+    auto range_start = [&](int c) -> int { return (int)((W * c) / C); };
+    auto block_of = [&](int x) -> int {
+        int c = (int)(((long long)x * C) / W);
+        while (c + 1 < C && range_start(c + 1) <= x) ++c;
+        while (c > 0 && range_start(c) > x) --c;
+        return c;
+    };
+    for (int row = blockIdx.x; row < P.B * hkv; row += gridDim.x) {
+        const int b = row / hkv, h = row % hkv;
+        const int len = P.lens[b];
+        if (len <= 0) continue;
+        const int n_pages = (len + kPage - 1) / kPage;
+        const int row_start = cum[b] + h * n_pages, row_end = row_start + n_pages;
+        const int c0 = block_of(row_start), c1 = block_of(row_end - 1);
+        if (c0 == c1) continue;                                   // written by its only block
+        const int n_parts = c1 - c0 + 1;
+        __syncthreads();
+        for (int j = tid; j < n_parts; j += D) slot_s[j] = 2 * (c0 + j) + (row_start > range_start(c0 + j) ? 1 : 0);
+        __syncthreads();
+        auto slot_of = [&](int j) -> const float* { return P.partials + (size_t)slot_s[j] * (8 * D + 16); };
+        // maxima and row sums of all parts -> weights e^{m_j - m} and the total l
+        for (int i = tid; i < n_parts * 8; i += D) {
+            const float* ps = slot_of(i >> 3) + 8 * D;
+            const float lj = __ldcg(ps + 8 + (i & 7));
+            l_s[i] = lj;
+            w_s[i] = lj > 0.f ? __ldcg(ps + (i & 7)) : -CUDART_INF_F;
+        }
+        __syncthreads();
+        if (tid < 8) {
+            float M = -CUDART_INF_F;
+            for (int j = 0; j < n_parts; ++j) M = fmaxf(M, w_s[j * 8 + tid]);
+            ml_s[tid] = M;
+        }
+        __syncthreads();
+        for (int i = tid; i < n_parts * 8; i += D) {
+            const float mj = w_s[i];
+            w_s[i] = mj == -CUDART_INF_F ? 0.f : fast_exp2(mj - ml_s[i & 7]);
+        }
+        __syncthreads();
+        if (tid < 8) {
+            float L = 0.f;
+            for (int j = 0; j < n_parts; ++j) L += w_s[j * 8 + tid] * l_s[j * 8 + tid];
+            ml_s[8 + tid] = L;
+        }
+        __syncthreads();
+        // thread = (channel, half of the heads): this block covers the channels blockIdx.y*D/2 ...
+        const int ch = blockIdx.y * (D / 2) + (tid >> 1), head0 = (tid & 1) * 4;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int j0 = 0; j0 < n_parts; j0 += kMaxParts) {
+            float4 v[kMaxParts];
+#pragma unroll
+            for (int k = 0; k < kMaxParts; ++k) {
+                const int j = min(j0 + k, n_parts - 1);
+                v[k] = __ldcg(reinterpret_cast<const float4*>(slot_of(j) + ch * 8 + head0));
+            }
+#pragma unroll
+            for (int k = 0; k < kMaxParts; ++k)
+                if (j0 + k < n_parts) {
+                    const float4 w = *reinterpret_cast<const float4*>(w_s + (j0 + k) * 8 + head0);
+                    acc.x = fmaf(w.x, v[k].x, acc.x);
+                    acc.y = fmaf(w.y, v[k].y, acc.y);
+                    acc.z = fmaf(w.z, v[k].z, acc.z);
+                    acc.w = fmaf(w.w, v[k].w, acc.w);
+                }
+        }
+        const float av[4] = {acc.x, acc.y, acc.z, acc.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int head = head0 + k;
+            if (head < GQ) {
+                const float L = ml_s[8 + head];
+                P.out[((size_t)b * hq + h * GQ + head) * D + ch] = L > 0.f ? av[k] / L : 0.f;
+            }
+        }
+        if (P.lse && blockIdx.y == 0 && tid < GQ)
+            P.lse[(size_t)b * hq + h * GQ + tid] = ml_s[8 + tid] > 0.f ? (ml_s[tid] + log2f(ml_s[8 + tid])) * kLn2 : -CUDART_INF_F;
+    }
+}
+
+template <int D, int NW, int NSTAGE, int MINB>
 static int32_t run_tensor(mkv_pool* p, DecodeParams& prm, cudaStream_t s)
 {
-    using G = Geo<D, NW, NSTAGE, HALVES>;
-    auto kern = decode_tensor_kernel<D, NW, NSTAGE, MINB, HALVES>;
+    using G = Geo<D, NW, NSTAGE>;
+    auto kern = decode_tensor_kernel<D, NW, NSTAGE, MINB>;
     static int grid_cache[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     int dev = p->device & 7;
     if (grid_cache[dev] == 0) {
@@ -1074,6 +1027,22 @@ static int32_t run_tensor(mkv_pool* p, DecodeParams& prm, cudaStream_t s)
     }
     kern<<<grid_cache[dev], NW * 32, G::SMEM, s>>>(prm);
     MKV_CUDA(cudaGetLastError());
+    // rows split over several blocks: at most one per block boundary, never more than the rows there are
+    int rows = prm.B * prm.hkv;
+    if (rows > grid_cache[dev]) rows = grid_cache[dev];
+    // programmatic dependent launch: the merge blocks become resident while the scan drains and wait
+    // (griddepcontrol.wait) for its completion before they read the partials
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(rows, 2);
+    cfg.blockDim = dim3(D);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    MKV_CUDA(cudaLaunchKernelEx(&cfg, decode_merge_kernel<D>, prm, grid_cache[dev]));
     return MKV_OK;
 }
 
@@ -1110,25 +1079,24 @@ int32_t launch_decode_tensor(mkv_pool* p, const void* q, const int32_t* bt, cons
     prm.bt = bt; prm.tags = tags; prm.lens = lens;
     prm.B = B; prm.max_pages = max_pages; prm.scale = scale;
     prm.out = out; prm.lse = lse;
-    prm.tickets = reinterpret_cast<uint32_t*>(static_cast<uint8_t*>(ws) + 256);
     prm.partials = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + decode_ws_header_bytes(B, p->hkv));
     prm.status = p->status_dev;
-    // Launch shapes, measured on B200 (2 x 59,008 tokens, d = 256): 8 warps with 255 registers and whole-page
-    // warps stream as fast as 16 warps in pairs; MKV_DECODE_SHAPE selects the alternatives for profiling.
+    // Launch shapes (warps per block, ring slots per warp, blocks per SM); MKV_DECODE_SHAPE selects the
+    // alternatives for profiling.
     const int shape = tensor_shape();
     if (p->d == 128) {
         switch (shape) {
-        case 1: return run_tensor<128, 8, 4, 1, 1>(p, prm, s);
-        case 2: return run_tensor<128, 12, 4, 1, 1>(p, prm, s);
-        case 3: return run_tensor<128, 8, 2, 2, 1>(p, prm, s);
-        default: return run_tensor<128, 16, 4, 1, 1>(p, prm, s);
+        case 1: return run_tensor<128, 8, 4, 1>(p, prm, s);
+        case 2: return run_tensor<128, 12, 4, 1>(p, prm, s);
+        case 3: return run_tensor<128, 8, 4, 2>(p, prm, s);
+        default: return run_tensor<128, 16, 4, 1>(p, prm, s);
         }
     }
     switch (shape) {
-    case 1: return run_tensor<256, 16, 4, 1, 2>(p, prm, s);
-    case 2: return run_tensor<256, 12, 4, 1, 1>(p, prm, s);
-    case 3: return run_tensor<256, 8, 4, 2, 2>(p, prm, s);
-    default: return run_tensor<256, 8, 4, 1, 1>(p, prm, s);
+    case 1: return run_tensor<256, 16, 2, 1>(p, prm, s);
+    case 2: return run_tensor<256, 12, 2, 1>(p, prm, s);
+    case 3: return run_tensor<256, 10, 4, 1>(p, prm, s);
+    default: return run_tensor<256, 8, 4, 1>(p, prm, s);
     }
 }
 
