@@ -186,6 +186,30 @@ int32_t mkv_decode_attention(mkv_pool* pool, const void* q_dev, const int32_t* b
                              int32_t max_pages, float scale, float* out_dev, float* lse_dev,
                              void* workspace_dev, size_t workspace_bytes, void* stream);
 
+/* The same decode attention for callers that cannot give the library a workspace because they are
+ * not allowed to allocate device memory once they are running (a server that handed its whole
+ * memory budget to the KV pool at start-up, code living inside another component's memory manager,
+ * a process whose allocator is frozen while it serves).  (The paper has no counterpart: this is a
+ * property of the library, not of the method.)  The split partials go to a fixed array inside the
+ * library image, MKV_STATIC_SCRATCH_BYTES per GPU that loads the library, held until the process
+ * exits.  Arguments, results and kernels are those of mkv_decode_attention (tensor-core kernel).
+ *   - allocates nothing: no cudaMalloc / cudaFree, no allocating library call, on any call.
+ *   - limits: B <= MKV_STATIC_MAX_BATCH, and the scan must not launch more than MKV_STATIC_MAX_BLOCKS
+ *     blocks on this GPU (it launches one per SM on B200); beyond either the call launches nothing and
+ *     returns MKV_E_INVALID, with the reason in mkv_last_cuda_error().
+ *   - the pool's device must be the current device.  The first call on a device looks up the array's
+ *     device address; make that first call before any stream capture begins.
+ *   - all calls on a device share the one array, which keeps whatever the previous call left in it
+ *     (every word is rewritten before it is read, so nothing needs clearing).  Two calls that overlap
+ *     on the GPU, e.g. on different streams, race on it: serialise them or use mkv_decode_attention
+ *     with separate workspaces. */
+#define MKV_STATIC_MAX_BLOCKS 160
+#define MKV_STATIC_MAX_BATCH 1024
+#define MKV_STATIC_SCRATCH_BYTES (2u * MKV_STATIC_MAX_BLOCKS * (8u * 256u + 16u) * 4u) /* 2,641,920 bytes */
+int32_t mkv_decode_attention_static(mkv_pool* pool, const void* q_dev, const int32_t* block_table_dev,
+                                    const uint8_t* tier_tag_dev, const int32_t* seq_lens_dev, int32_t B,
+                                    int32_t max_pages, float scale, float* out_dev, float* lse_dev, void* stream);
+
 /* ---- host-side sequence bookkeeping (Algorithm 1; no device work) ------------------------- */
 
 /* A sequence owns a row of logical pages -> (tag, physical id).  These calls only plan: they

@@ -32,6 +32,7 @@ EXPORTS = [
     "mkv_page_read_raw", "mkv_page_write_raw", "mkv_last_cuda_error", "mkv_append", "mkv_demote",
     "mkv_set_anchor", "mkv_decode_attention", "mkv_seq_create", "mkv_seq_finish", "mkv_seq_append",
     "mkv_seq_protect", "mkv_seq_demote", "mkv_seq_age", "mkv_seq_len", "mkv_seq_row",
+    "mkv_decode_attention_static",
 ]
 
 
@@ -84,6 +85,7 @@ def lib():
             "mkv_set_anchor": [vp, vp, C.c_int64, C.c_int32, vp],
             "mkv_decode_attention": [vp, vp, vp, vp, vp, C.c_int32, C.c_int32, C.c_float, f32p, f32p, vp,
                                      C.c_size_t, vp],
+            "mkv_decode_attention_static": [vp, vp, vp, vp, vp, C.c_int32, C.c_int32, C.c_float, f32p, f32p, vp],
             "mkv_seq_create": [vp, C.POINTER(vp)],
             "mkv_seq_finish": [vp],
             "mkv_seq_append": [vp, i32p, i32p, i32p],
@@ -99,9 +101,6 @@ def lib():
             fn.restype = C.c_int32
         L.mkv_last_cuda_error.restype = C.c_char_p
         L.mkv_last_cuda_error.argtypes = []
-        for name in ("mkv_decode_attention_static", "mkv_decode_static_limits"):
-            if hasattr(L, name):
-                getattr(L, name).restype = C.c_int32
         _lib = L
     return _lib
 
@@ -248,6 +247,22 @@ class Pool:
                                           block_table.shape[1], float(scale), _ptr(out), _ptr(lse), _ptr(ws),
                                           ws.numel(), _stream(stream)), "mkv_decode_attention")
         return out
+
+
+def decode_attention_static(pool: "Pool", q, block_table, tier_tag, seq_lens, scale, out=None, lse=None, stream=None):
+    """mkv_decode_attention_static: decode attention whose scratch is a fixed array inside the library,
+    for callers that must not allocate device memory (the output tensor is the caller's, as always)."""
+    B = q.shape[0]
+    assert q.dtype == torch.bfloat16 and q.is_contiguous() and q.shape == (B, pool.hq, pool.d)
+    assert block_table.dtype == torch.int32 and block_table.is_contiguous() and block_table.shape[0] == B
+    assert tier_tag.dtype == torch.uint8 and tier_tag.shape == block_table.shape and tier_tag.is_contiguous()
+    assert seq_lens.dtype == torch.int32 and seq_lens.numel() == B
+    if out is None:
+        out = torch.empty((B, pool.hq, pool.d), dtype=torch.float32, device=q.device)
+    _check(lib().mkv_decode_attention_static(pool.handle, _ptr(q), _ptr(block_table), _ptr(tier_tag), _ptr(seq_lens),
+                                             B, block_table.shape[1], float(scale), _ptr(out), _ptr(lse),
+                                             _stream(stream)), "mkv_decode_attention_static")
+    return out
 
 
 class HostPool:

@@ -59,6 +59,7 @@ struct DecodeParams {
     float* out;
     float* lse;
     float* partials;       // [2 * grid][8*D + 16]
+    int max_blocks;        // the partial area holds 2 * max_blocks slots
     uint32_t* status;
 };
 
@@ -1025,6 +1026,7 @@ static int32_t run_tensor(mkv_pool* p, DecodeParams& prm, cudaStream_t s)
         int grid = p->dev.sm_count * per_sm;
         grid_cache[dev] = grid > kMaxCtas ? kMaxCtas : grid;
     }
+    if (grid_cache[dev] > prm.max_blocks) return MKV_E_INVALID;
     kern<<<grid_cache[dev], NW * 32, G::SMEM, s>>>(prm);
     MKV_CUDA(cudaGetLastError());
     // rows split over several blocks: at most one per block boundary, never more than the rows there are
@@ -1068,6 +1070,16 @@ int32_t launch_decode_tensor(mkv_pool* p, const void* q, const int32_t* bt, cons
                              const int32_t* lens, int B, int max_pages, float scale, float* out, float* lse,
                              void* ws, size_t, cudaStream_t s)
 {
+    float* partials = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + decode_ws_header_bytes(B, p->hkv));
+    return launch_decode_tensor_at(p, q, bt, tags, lens, B, max_pages, scale, out, lse, partials, kMaxCtas, s);
+}
+
+int decode_tensor_partial_floats(int d) { return 8 * d + 16; }
+
+int32_t launch_decode_tensor_at(mkv_pool* p, const void* q, const int32_t* bt, const uint8_t* tags,
+                                const int32_t* lens, int B, int max_pages, float scale, float* out, float* lse,
+                                float* partials, int max_blocks, cudaStream_t s)
+{
     if (B > kMaxBatch) return MKV_E_INVALID;
     DecodeParams prm;
     prm.fp8 = p->fp8; prm.tq3 = p->tq3;
@@ -1079,7 +1091,8 @@ int32_t launch_decode_tensor(mkv_pool* p, const void* q, const int32_t* bt, cons
     prm.bt = bt; prm.tags = tags; prm.lens = lens;
     prm.B = B; prm.max_pages = max_pages; prm.scale = scale;
     prm.out = out; prm.lse = lse;
-    prm.partials = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + decode_ws_header_bytes(B, p->hkv));
+    prm.partials = partials;
+    prm.max_blocks = max_blocks;
     prm.status = p->status_dev;
     // Launch shapes (warps per block, ring slots per warp, blocks per SM); MKV_DECODE_SHAPE selects the
     // alternatives for profiling.

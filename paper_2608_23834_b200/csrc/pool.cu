@@ -17,6 +17,8 @@ int32_t cuda_fail(cudaError_t e, const char* what)
     return MKV_E_CUDA;
 }
 
+void set_last_error(const char* msg) { g_last_error = msg; }
+
 static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 static int32_t check_cfg(const mkv_pool_config* c)
