@@ -37,7 +37,7 @@ METRIC = "decode attention tokens/s and achieved KV HBM GB/s (% of B200 peak) at
 UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode_tensor_kernel launch on the default
 # workload, from the ncu capture summarised under profiles/; None until captured.
-TRAFFIC_BYTES_PER_LAUNCH = None
+TRAFFIC_BYTES_PER_LAUNCH = 126808064 + 4094464   # profiles/decode_tensor_cfg2.md (scan kernel, one launch)
 FALLBACK_HBM_GBS = 6650.0
 STAGE_PAGES = 512
 
@@ -265,6 +265,8 @@ def run_ours(args):
     K, Wm = args.steps, args.warmup
     total = 2 * (K + Wm)                       # device-resident run, then the end-to-end run
     layers, plan, tab0 = build_layers(spec, total, device, M, torch)
+    for L in layers:
+        L.pool.set_decode_variant(M.DECODE_SCALAR if args.variant == "scalar" else M.DECODE_TENSOR)
     B, d, hq, hkv = spec.batch, spec.head_dim, spec.n_q_heads, spec.n_kv_heads
     stream = torch.cuda.current_stream()
     launches = [0]
@@ -288,7 +290,7 @@ def run_ours(args):
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record(stream)
             L.pool.decode_attention(L.q, L.bt, L.tags, plan["lens"][i], spec.scale, out=L.out)
-            launches[0] += 1
+            launches[0] += 2                      # scan kernel + merge kernel
             if timed_events is not None:
                 e1.record(stream)
                 timed_events.append((e0, e1))
@@ -386,9 +388,9 @@ def run_ours(args):
                    "l2": "inputs larger than L2 (%.0f MB of KV per step)" % (step_bytes / 1e6),
                    "step": "append + demote at its natural cadence + decode attention, every layer"},
         "kv_gbs_whole_step": step_bytes / (ms / K * 1e-3) / 1e9,
-        "roofline": {"bound": "hbm", "kernel": "decode_tensor_kernel", "achieved": achieved, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": "decode_%s_kernel + merge" % args.variant, "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_kind + " copy bandwidth",
-                     "frac_of_nominal_8000": achieved / 8000.0, "traffic": TRAFFIC_BYTES_PER_LAUNCH,
+                     "frac_of_nominal_8000": achieved / 8000.0, "traffic": TRAFFIC_BYTES_PER_LAUNCH if (args.config == 2 and args.ctx == 0 and args.variant == "tensor") else None,
                      "algorithmic_bytes_per_launch": avg_bytes, "avg_launch_ms": avg_kernel_ms},
         "e2e": {"value": world * B * K / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / K},
@@ -497,6 +499,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2)
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling on a small case)")
+    ap.add_argument("--variant", default="tensor", choices=["tensor", "scalar"],
+                    help="decode kernel: the tensor-core product kernel, or the CUDA-core comparison kernel")
     ap.add_argument("--ctx", type=int, default=0, help="override the context length of every request (profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
