@@ -99,6 +99,22 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def max_over_ranks(values, device=None):
+    """MAX over the ranks of every entry (the step time of a multi-replica run is the slowest replica's)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def aggregate_value(batch_per_replica, steps, ms, world):
+    """Whole-job tokens/s of `world` independent replicas that each decode `batch_per_replica` tokens per step."""
+    return world * batch_per_replica * steps / (ms * 1e-3)
+
+
 # --------------------------------------------------------------------------------------------- ours
 class LayerState:
     pass
@@ -366,11 +382,7 @@ def run_ours(args):
     barrier()
     e2e_ms = max(t0.elapsed_time(t1), (time.perf_counter() - w0) * 1e3)
 
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([ms, e2e_ms], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, e2e_ms = float(t[0]), float(t[1])
+    ms, e2e_ms = max_over_ranks([ms, e2e_ms], device)
 
     peaks, peak_kind = measured_peaks()
     peak = float(peaks["hbm_gbs"])
@@ -379,7 +391,7 @@ def run_ours(args):
     achieved = avg_bytes / (avg_kernel_ms * 1e-3) / 1e9
     step_bytes = avg_bytes * spec.n_layers
     result = {
-        "metric": METRIC, "value": world * B * K / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+        "metric": METRIC, "value": aggregate_value(B, K, ms, world), "unit": UNIT, "n_gpus": world, "steps": K,
         "warmup": Wm, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "u8 codes (e4m3 / 3-bit TQ3) -> f16 tensor-core operands, f32 accumulate", "data": "synthetic",
         "config": {"workload": workload_name(spec), "batch": B, "context_tokens": list(spec.seq_lens)[:4],
@@ -392,7 +404,7 @@ def run_ours(args):
                      "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_kind + " copy bandwidth",
                      "frac_of_nominal_8000": achieved / 8000.0, "traffic": TRAFFIC_BYTES_PER_LAUNCH if (args.config == 2 and args.ctx == 0 and args.variant == "tensor") else None,
                      "algorithmic_bytes_per_launch": avg_bytes, "avg_launch_ms": avg_kernel_ms},
-        "e2e": {"value": world * B * K / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        "e2e": {"value": aggregate_value(B, K, e2e_ms, world), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / K},
         "gpu_launches": n_launch,
         "clocks": clocks.summary(),

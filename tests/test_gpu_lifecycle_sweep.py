@@ -1,0 +1,129 @@
+"""Lifecycle sweep cell (config 4 shape, scaled): every transition goes through the library --
+mkv_seq_* plans, mkv_append / mkv_demote / mkv_set_anchor kernels, mkv_decode_attention -- and is
+mirrored by the oracle (lifecycle model + codecs + fp64 attention).  Packed pages and tables must
+agree bit for bit, attention within the tolerance."""
+import numpy as np
+import pytest
+import torch
+
+import mkv_workloads as W
+import oracle
+import paper_2608_23834_b200 as M
+from _gpu_util import bf16_tensor, check_close
+from oracle.lifecycle import PoolModel, STALE
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("frac,ctx,batch", [(0.5, 512, 2), (0.95, 320, 3), (0.0, 256, 2)])
+def test_append_demote_decode_cell(frac, ctx, batch):
+    spec = W.config(4, batch=batch, ctx=ctx, stale_fraction=frac, n_kv_heads=2)
+    d, hkv, hq = spec.head_dim, spec.n_kv_heads, spec.n_q_heads
+    n_pages = ctx // 16
+    cap = batch * (n_pages + 2)
+    sigma = W.rotation_signs(spec)
+    pool = M.Pool(d, hkv, hq, cap, cap, sigma, max_batch=batch)
+    model = PoolModel(cap, cap)
+    fp8 = np.zeros((cap, hkv, 32 * d), np.uint8)          # the oracle's own arenas
+    tq3 = np.zeros((cap, hkv, 16 * d + 32), np.uint8)
+    seqs = [M.Seq(pool) for _ in range(batch)]
+    mods = [model.new_seq() for _ in range(batch)]
+    max_pages = n_pages + 2
+    bt = torch.full((batch, max_pages), -1, dtype=torch.int32, device="cuda:0")
+    tags = torch.zeros((batch, max_pages), dtype=torch.uint8, device="cuda:0")
+
+    def append_tokens(k_bits, v_bits):
+        """k_bits, v_bits: [n][batch][hkv][d]; request-major interleaving of one token each per call."""
+        slots = []
+        for t in range(k_bits.shape[0]):
+            for b in range(batch):
+                pid, sl, opened = seqs[b].append()
+                assert (pid, sl, opened) == mods[b].append()
+                if opened:
+                    bt[b, len(mods[b].pages) - 1] = pid       # publish the new Recent page
+                slots.append(pid * 16 + sl)
+                kf, vf = oracle.bf16_bits_to_f32(k_bits[t, b]), oracle.bf16_bits_to_f32(v_bits[t, b])
+                for h in range(hkv):
+                    rec = fp8[pid, h]
+                    rec[sl * d:(sl + 1) * d] = [oracle.e4m3_encode(x) for x in kf[h]]
+                    rec[16 * d + sl:32 * d:16] = [oracle.e4m3_encode(x) for x in vf[h]]
+        kk = bf16_tensor(k_bits.reshape(-1, hkv, d))
+        vv = bf16_tensor(v_bits.reshape(-1, hkv, d))
+        pool.append(kk, vv, torch.tensor(slots, dtype=torch.int32, device="cuda:0"))
+
+    def demote(pairs):
+        """pairs: list of (b, logical page, src, dst) already planned on both sides."""
+        if not pairs:
+            return
+        for b, lp, s, t in pairs:
+            for h in range(hkv):
+                tq3[t, h] = oracle.demote_record(fp8[s, h], d, sigma)
+        src = torch.tensor([p[2] for p in pairs], dtype=torch.int32, device="cuda:0")
+        dst = torch.tensor([p[3] for p in pairs], dtype=torch.int32, device="cuda:0")
+        ent = torch.tensor([p[0] * max_pages + p[1] for p in pairs], dtype=torch.int64, device="cuda:0")
+        pool.demote(src, dst, bt, tags, ent)
+
+    # ---- bring the cell to its starting state: ctx tokens, oldest floor(f*P) pages Stale ----
+    rng = np.random.default_rng(4)
+    k0 = W.f32_to_bf16_bits(rng.standard_normal((ctx, batch, hkv, d)).astype(np.float32))
+    v0 = W.f32_to_bf16_bits(rng.standard_normal((ctx, batch, hkv, d)).astype(np.float32))
+    append_tokens(k0, v0)
+    pairs = []
+    for b in range(batch):
+        for lp in range(int(np.floor(frac * n_pages))):
+            s, t = seqs[b].demote(lp)
+            assert (s, t) == mods[b].demote(lp)
+            pairs.append((b, lp, s, t))
+    demote(pairs)
+
+    # ---- the cell: append one token, demote the page leaving the Recent window, protect one, decode ----
+    k1, v1 = W.new_token_kv(spec, 0)
+    append_tokens(k1[None], v1[None])
+    recent = max(16, ctx - int(np.floor(frac * n_pages)) * 16 - 16)   # the window shrinks by one page
+    pairs = []
+    for b in range(batch):
+        moved = seqs[b].age(recent)
+        assert moved == mods[b].age(recent)
+        pairs += [(b,) + m for m in moved]
+    demote(pairs)
+    if frac == 0.5:
+        assert len(pairs) == batch
+    for b in range(batch):                                          # protect the newest full page
+        lp = n_pages - 1
+        seqs[b].protect(lp, True)
+        mods[b].protect(lp)
+        pool.set_anchor(tags, b * max_pages + lp, True)
+    torch.cuda.synchronize()
+    assert pool.status() == M.OK
+    model.check_invariants()
+
+    # tables on the device equal the host rows of both sides
+    bt_h, tg_h = bt.cpu().numpy(), tags.cpu().numpy()
+    for b in range(batch):
+        ids, tg = seqs[b].row()
+        n = len(ids)
+        assert [(int(t), int(p)) for t, p in zip(tg, ids)] == mods[b].pages
+        assert np.array_equal(bt_h[b, :n], ids) and np.array_equal(tg_h[b, :n], tg)
+    # every live page is bit-identical to the oracle's
+    for b in range(batch):
+        for tag, pid in mods[b].pages:
+            if tag == STALE:
+                assert np.array_equal(pool.page_read_raw(M.FMT_TQ3, pid).reshape(hkv, -1), tq3[pid])
+            else:
+                assert np.array_equal(pool.page_read_raw(M.FMT_FP8, pid).reshape(hkv, -1), fp8[pid])
+    st = pool.stats()
+    used, _ = model.stats()
+    assert (st.fp8_pages_used, st.tq3_pages_used) == (used[0], used[1])
+
+    lens = np.array([m.len for m in mods], np.int32)
+    q_bits = W.query(spec)
+    ref, ref_lse = oracle.decode_attention(fp8, tq3, d, hkv, spec.group, sigma, q_bits, bt_h, tg_h, lens, spec.scale)
+    for variant in (M.DECODE_TENSOR, M.DECODE_SCALAR):
+        pool.set_decode_variant(variant)
+        out = pool.decode_attention(bf16_tensor(q_bits), bt, tags, torch.from_numpy(lens).cuda(), spec.scale)
+        torch.cuda.synchronize()
+        assert pool.status() == M.OK
+        check_close(out.cpu().numpy(), ref, f"cell f={frac} variant={variant}")
+    for s in seqs:
+        s.finish()
+    assert pool.stats().fp8_pages_used == 0 and pool.stats().tq3_pages_used == 0
