@@ -225,6 +225,111 @@ __device__ __forceinline__ void affine_accumulate(float (&acc)[4], const float (
 }
 
 // ------------------------------------------------------------------------------------------------
+// Work partition, shared by the scan and the merge kernel
+// ------------------------------------------------------------------------------------------------
+// Work = (request, KV head, page) triples in row-major order; cum[b] = index of the first triple of
+// request b.  Two ways to cut it into one contiguous range per block:
+//   row-aligned (few rows: B * hkv <= grid / 4): every row gets a whole number of blocks in proportion
+//     to its pages (cumulative rounding), so that no block straddles two rows and pays the per-row set-up
+//     and reduction twice;
+//   linear (many rows): grid equal ranges that may cross row boundaries.
+constexpr int kMaxAlignedRows = kMaxCtas / 4;
+
+struct Partition {
+    int aligned;                        // 1: row-aligned, 0: linear
+    int blocks;                         // blocks that get work
+    int base[kMaxAlignedRows + 1];      // row-aligned: first block of every row
+};
+
+// Called by warp 0 (all 32 lanes) after cum[] is complete; other warps wait at the next barrier.
+__device__ __forceinline__ void build_partition(Partition* pt, const int* cum, const int32_t* lens, int B, int hkv,
+                                                int grid, int lane)
+{
+    constexpr uint32_t FULL = 0xffffffffu;
+    const long long W = cum[B];
+    const int rows = B * hkv;
+    int blocks = (int)(W < (long long)grid ? W : (long long)grid);
+    int aligned = (rows <= grid / 4 && rows <= kMaxAlignedRows && W >= grid) ? 1 : 0;
+    if (aligned) {
+        // block boundaries at the rounded cumulative share of the rows: base[r] = round(grid * first_page(r) / W);
+        // every row must end up with at least one block, otherwise the linear cut is used
+        int bad = 0;
+        const float scale = (float)grid / (float)W;
+        for (int r = lane; r <= rows; r += 32) {
+            int first = (int)W;                                 // r == rows: one past the last row
+            if (r < rows) {
+                const int b = r / hkv, h = r - b * hkv;
+                first = cum[b] + h * ((cum[b + 1] - cum[b]) / hkv);
+            }
+            pt->base[r] = r == rows ? grid : (int)((float)first * scale + 0.5f);
+        }
+        __syncwarp();
+        for (int r = lane; r < rows; r += 32) {
+            const int b = r / hkv;
+            if (cum[b + 1] > cum[b] && pt->base[r + 1] <= pt->base[r]) bad = 1;
+        }
+        if (__any_sync(FULL, bad)) aligned = 0;
+        else blocks = grid;
+    }
+    if (lane == 0) {
+        pt->aligned = aligned;
+        pt->blocks = blocks;
+    }
+}
+
+// linear range [start, end) of block c
+__device__ __forceinline__ void partition_range(const Partition* pt, const int* cum, int hkv, int B, int c, int& start,
+                                                int& end)
+{
+    const long long W = cum[B];
+    if (!pt->aligned) {
+        start = (int)((W * c) / pt->blocks);
+        end = (int)((W * (c + 1)) / pt->blocks);
+        return;
+    }
+    const int rows = B * hkv;
+    int lo = 0;                                     // row of block c: base[r] <= c < base[r + 1]
+    for (int hi = rows - 1; lo < hi;) {
+        const int mid = (lo + hi) >> 1;
+        if (pt->base[mid + 1] <= c) lo = mid + 1; else hi = mid;
+    }
+    const int r = lo, b = r / hkv, h = r - b * hkv, n = (cum[b + 1] - cum[b]) / hkv;
+    const unsigned k = pt->base[r + 1] - pt->base[r], j = c - pt->base[r];
+    const int row_start = cum[b] + h * n;
+    start = row_start + (int)(((unsigned)n * j) / k);
+    end = row_start + (int)(((unsigned)n * (j + 1)) / k);
+}
+
+__device__ __forceinline__ int partition_start(const Partition* pt, const int* cum, int hkv, int B, int c)
+{
+    int s, e;
+    partition_range(pt, cum, hkv, B, c, s, e);
+    return s;
+}
+
+// blocks c0..c1 that hold a part of the row [row_start, row_end) (row index r)
+__device__ __forceinline__ void partition_blocks_of_row(const Partition* pt, const int* cum, int B, int r, int row_start,
+                                                        int row_end, int& c0, int& c1)
+{
+    if (pt->aligned) {
+        c0 = pt->base[r];
+        c1 = pt->base[r + 1] - 1;
+        return;
+    }
+    const long long W = cum[B];
+    const int C = pt->blocks;
+    auto start = [&](int c) -> int { return (int)((W * c) / C); };
+    auto block_of = [&](int x) -> int {
+        int c = (int)(((long long)x * C) / W);
+        while (c + 1 < C && start(c + 1) <= x) ++c;
+        while (c > 0 && start(c) > x) --c;
+        return c;
+    };
+    c0 = block_of(row_start);
+    c1 = block_of(row_end - 1);
+}
+
+// ------------------------------------------------------------------------------------------------
 // kernel
 // ------------------------------------------------------------------------------------------------
 constexpr int kRound = 128;          // pages of one warp whose table entries are compacted at a time
@@ -247,8 +352,8 @@ struct Geo {
     static constexpr int OFF_STRIDE = OFF_CUM + (kMaxBatch + 1) * 4;
     static constexpr int OFF_M = OFF_STRIDE + kMaxBatch * 4;
     static constexpr int OFF_L = OFF_M + NW * 8 * 4;
-    static constexpr int OFF_FLAG = OFF_L + NW * 8 * 4;
-    static constexpr int SMEM = OFF_FLAG + 16;
+    static constexpr int OFF_PART = OFF_L + NW * 8 * 4;
+    static constexpr int SMEM = OFF_PART + (int)sizeof(Partition) + 16;
     static_assert(NW >= 8, "one warp per column of the 8-wide head group builds the query fragments");
     static_assert(NSTAGE == 2 || NSTAGE == 4, "ring positions are taken modulo a power of two; an FP8 page takes two slots");
     static_assert(NSTAGE * SLOT >= 8 * D * 4, "ring doubles as the cross-warp reduction buffer");
@@ -530,7 +635,7 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
     int* strides = reinterpret_cast<int*>(smem + G::OFF_STRIDE);
     float* sm_m = reinterpret_cast<float*>(smem + G::OFF_M);
     float* sm_l = reinterpret_cast<float*>(smem + G::OFF_L);
-    int* sm_flag = reinterpret_cast<int*>(smem + G::OFF_FLAG);
+    Partition* pt = reinterpret_cast<Partition*>(smem + G::OFF_PART);
     float* red = reinterpret_cast<float*>(smem);            // [NW][D][8] over the ring, between segments
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tq = lane & 3;
@@ -567,6 +672,10 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
             run += __shfl_sync(FULL, inc, 31);
         }
         if (lane == 0) cum[P.B] = run;
+        __syncwarp();
+        MKV_STAMP(9);
+        build_partition(pt, cum, P.lens, P.B, hkv, gridDim.x, lane);
+        MKV_STAMP(10);
     } else {
         // Pages of a row are visited in a strided order, page(i) = i * stride mod n_pages, the stride
         // coprime to n_pages and near 0.618 n_pages: every contiguous range of positions then holds the
@@ -584,17 +693,10 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
         }
     }
     __syncthreads();
-    const long long W = cum[P.B];
-    const int C = (int)(W < (long long)gridDim.x ? W : (long long)gridDim.x);   // blocks that get work
-    if ((int)blockIdx.x >= C) return;
-    auto range_start = [&](int c) -> int { return (int)((W * c) / C); };
-    auto block_of = [&](int x) -> int {      // the block whose range holds linear index x
-        int c = (int)(((long long)x * C) / W);
-        while (c + 1 < C && range_start(c + 1) <= x) ++c;
-        while (c > 0 && range_start(c) > x) --c;
-        return c;
-    };
-    const int my_start = range_start(blockIdx.x), my_end = range_start(blockIdx.x + 1);
+    MKV_STAMP(11);
+    if ((int)blockIdx.x >= pt->blocks) return;             // more blocks than work
+    int my_start, my_end;
+    partition_range(pt, cum, hkv, P.B, blockIdx.x, my_start, my_end);
 
     // per-warp ring of NSTAGE slots; one bit per slot holds the mbarrier phase the next wait must see
     uint32_t phase = 0;
@@ -903,6 +1005,7 @@ __global__ void __launch_bounds__(D) decode_merge_kernel(const DecodeParams P, i
     __shared__ __align__(16) float w_s[kMaxCtas * 8];    // weight of every partial and head (read as float4)
     __shared__ float l_s[kMaxCtas * 8];                  // row sums of every partial and head
     __shared__ int slot_s[kMaxCtas];                     // workspace slot of every partial
+    __shared__ Partition pt_s;
     __shared__ float ml_s[16];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int hkv = P.hkv, GQ = P.group, hq = hkv * GQ;
@@ -928,28 +1031,26 @@ __global__ void __launch_bounds__(D) decode_merge_kernel(const DecodeParams P, i
     }
     __syncthreads();
     const long long W = cum[P.B];
+    if (warp == 0 && W > 0) build_partition(&pt_s, cum, P.lens, P.B, hkv, scan_grid, lane);
+    __syncthreads();
+    const Partition* pt = &pt_s;
     // everything above read only the call's inputs; the partials below are the scan kernel's output
     asm volatile("griddepcontrol.wait;" ::: "memory");
     if (W == 0) return;
-    const int C = (int)(W < (long long)scan_grid ? W : (long long)scan_grid);
-    auto range_start = [&](int c) -> int { return (int)((W * c) / C); };
-    auto block_of = [&](int x) -> int {
-        int c = (int)(((long long)x * C) / W);
-        while (c + 1 < C && range_start(c + 1) <= x) ++c;
-        while (c > 0 && range_start(c) > x) --c;
-        return c;
-    };
     for (int row = blockIdx.x; row < P.B * hkv; row += gridDim.x) {
         const int b = row / hkv, h = row % hkv;
         const int len = P.lens[b];
         if (len <= 0) continue;
         const int n_pages = (len + kPage - 1) / kPage;
         const int row_start = cum[b] + h * n_pages, row_end = row_start + n_pages;
-        const int c0 = block_of(row_start), c1 = block_of(row_end - 1);
+        int c0, c1;
+        partition_blocks_of_row(pt, cum, P.B, row, row_start, row_end, c0, c1);
         if (c0 == c1) continue;                                   // written by its only block
         const int n_parts = c1 - c0 + 1;
         __syncthreads();
-        for (int j = tid; j < n_parts; j += D) slot_s[j] = 2 * (c0 + j) + (row_start > range_start(c0 + j) ? 1 : 0);
+        // a block's slot for this row: 2c if the row's part opens the block's range, 2c + 1 otherwise
+        for (int j = tid; j < n_parts; j += D)
+            slot_s[j] = 2 * (c0 + j) + (row_start > partition_start(pt, cum, hkv, P.B, c0 + j) ? 1 : 0);
         __syncthreads();
         auto slot_of = [&](int j) -> const float* { return P.partials + (size_t)slot_s[j] * (8 * D + 16); };
         // maxima and row sums of all parts -> weights e^{m_j - m} and the total l
