@@ -403,7 +403,8 @@ def run_ours(args):
         "roofline": {"bound": "hbm", "kernel": "decode_%s_kernel + merge" % args.variant, "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_kind + " copy bandwidth",
                      "frac_of_nominal_8000": achieved / 8000.0, "traffic": TRAFFIC_BYTES_PER_LAUNCH if (args.config == 2 and args.ctx == 0 and args.variant == "tensor") else None,
-                     "algorithmic_bytes_per_launch": avg_bytes, "avg_launch_ms": avg_kernel_ms},
+                     "algorithmic_bytes_per_launch": avg_bytes, "avg_launch_ms": avg_kernel_ms,
+                     "median_launch_ms": statistics.median(kern_ms), "min_launch_ms": min(kern_ms)},
         "e2e": {"value": aggregate_value(B, K, e2e_ms, world), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / K},
         "gpu_launches": n_launch,
