@@ -78,6 +78,8 @@ def lib():
         L.orc_fp8_unpack_record_f32.argtypes = [C.c_int, u8p, C.c_float, C.c_float, f32p, f32p]
         L.orc_demote_record.restype = None
         L.orc_demote_record.argtypes = [C.c_int, u8p, C.c_float, C.c_float, i8p, u8p]
+        L.orc_promote_record.restype = None
+        L.orc_promote_record.argtypes = [C.c_int, u8p, C.c_float, C.c_float, i8p, u8p]
         L.orc_tq3_record_from_f32.restype = None
         L.orc_tq3_record_from_f32.argtypes = [C.c_int, f32p, f32p, i8p, u8p]
         L.orc_decode_attention.restype = C.c_int
@@ -236,6 +238,15 @@ def demote_record(fp8_rec: np.ndarray, d: int, sigma: np.ndarray, k_scale=1.0, v
     out = np.zeros(tq3_record_bytes(d), np.uint8)
     lib().orc_demote_record(d, _p(fp8_rec, C.c_uint8), k_scale, v_scale, _p(sigma, C.c_int8),
                             _p(out, C.c_uint8))
+    return out
+
+
+def promote_record(tq3_rec: np.ndarray, d: int, sigma: np.ndarray, k_scale=1.0, v_scale=1.0) -> np.ndarray:
+    """TQ3 record -> FP8 record (Promote of Algorithm 1, data part: reconstruct, then round to e4m3)."""
+    tq3_rec = _c(tq3_rec, np.uint8)
+    sigma = _c(sigma, np.int8)
+    out = np.zeros(fp8_record_bytes(d), np.uint8)
+    lib().orc_promote_record(d, _p(tq3_rec, C.c_uint8), k_scale, v_scale, _p(sigma, C.c_int8), _p(out, C.c_uint8))
     return out
 
 

@@ -681,3 +681,51 @@ int orc_encode_request(int d, int hkv, int len, const uint16_t* k_bits, const ui
     }
     return rc;
 }
+
+/* ------------------------------------------------------------------------------------------
+ * Promote(p) of Algorithm 1, data part: reconstruct a TQ3 record into an FP8 record.
+ * The reconstruction is specified in fp32 with a fixed operation order (so that it can be
+ * reproduced bit for bit), then rounded to e4m3 like Append:
+ *   key   : y = H c (butterflies, strides ascending, c = signed fp16 levels as fp32);
+ *           k = sigma .* ((g * rs) * y), rs = fp32(1/sqrt(d));   stored = e4m3(k * (1/k_scale))
+ *   value : v = sc * code + zp as one multiplication and one addition; stored = e4m3(v * (1/v_scale))
+ * ---------------------------------------------------------------------------------------- */
+void orc_promote_record(int d, const uint8_t* tq3_rec, float k_scale, float v_scale, const int8_t* sigma,
+                        uint8_t* fp8_rec)
+{
+    uint8_t* kc = (uint8_t*)malloc(ORC_T * (size_t)d);
+    uint8_t* vc = (uint8_t*)malloc(ORC_T * (size_t)d);
+    uint16_t g[ORC_T], sc[ORC_MAXD], zp[ORC_MAXD];
+    float ik = 1.0f / k_scale, iv = 1.0f / v_scale, rs = (float)(1.0 / sqrt((double)d));
+    int t, i, h;
+    orc_tq3_unpack_record(d, tq3_rec, kc, g, vc, sc, zp);
+    memset(fp8_rec, 0, (size_t)orc_fp8_record_bytes(d));
+    for (t = 0; t < ORC_T; ++t) {
+        float y[ORC_MAXD], gr = orc_f16_to_f32(g[t]) * rs;
+        for (i = 0; i < d; ++i) {
+            float c = ORC_C[kc[t * d + i] & 3];
+            y[i] = (kc[t * d + i] & 4) ? -c : c;
+        }
+        for (h = 1; h < d; h <<= 1)
+            for (i = 0; i < d; ++i)
+                if ((i & h) == 0) {
+                    float u = y[i], w = y[i + h];
+                    y[i] = u + w;
+                    y[i + h] = u - w;
+                }
+        for (i = 0; i < d; ++i) {
+            float k = gr * y[i];
+            if (sigma[i] < 0) k = -k;
+            fp8_rec[t * d + i] = orc_e4m3_encode(k * ik);
+        }
+    }
+    for (i = 0; i < d; ++i) {
+        float s = orc_f16_to_f32(sc[i]), z = orc_f16_to_f32(zp[i]);
+        for (t = 0; t < ORC_T; ++t) {
+            float p = s * (float)vc[t * d + i];
+            float v = p + z;
+            fp8_rec[16 * d + i * ORC_T + t] = orc_e4m3_encode(v * iv);
+        }
+    }
+    free(kc); free(vc);
+}

@@ -246,3 +246,31 @@ def test_demote_equals_encoding_the_dequantised_fp8_page():
     rec8s = oracle.fp8_pack_record(k, v, 16, 0.5, 2.0)
     ks, vs = oracle.fp8_unpack_record_f32(rec8s, d, 0.5, 2.0)
     assert np.abs(ks - k).max() <= np.abs(k).max() * 2.0 ** -4 and np.abs(vs - v).max() <= np.abs(v).max() * 2.0 ** -4
+
+
+@pytest.mark.parametrize("d", [128, 256])
+def test_promote_reconstructs_the_decoded_page_up_to_fp8_rounding(d):
+    """Promote (Algorithm 1 step 3): the FP8 page written from a TQ3 record dequantises to the fp64
+    decode of that record within half an e4m3 step, and values that are e4m3-exact come back exactly."""
+    rng = np.random.default_rng(31 + d)
+    sigma = (rng.integers(0, 2, d) * 2 - 1).astype(np.int8)
+    k = rng.standard_normal((16, d)).astype(np.float32)
+    v = rng.standard_normal((16, d)).astype(np.float32)
+    v[:, 3] = 2.5                                         # constant channel: zero = 2.5, scale = 0
+    v[:, 4] = np.float32([0, 7] * 8) * 0.5                # codes 0 / 7 with scale 0.5: values 0 and 3.5
+    rec3 = oracle.tq3_record_from_f32(k, v, sigma)
+    rec8 = oracle.promote_record(rec3, d, sigma)
+    kq, vq = oracle.fp8_unpack_record_f32(rec8, d)
+    kc, g, vc, sc, zp = oracle.tq3_unpack_record(rec3, d)
+    for t in range(16):
+        ref = oracle.tq3_decode_key(kc[t], int(g[t]), sigma)
+        # e4m3 keeps 4 significant bits: relative half-step 2^-4, absolute 2^-10 in the subnormal range
+        assert np.all(np.abs(kq[t] - ref) <= np.maximum(np.abs(ref) * 2.0 ** -4, 2.0 ** -10) + 1e-6)
+    for c in range(d):
+        ref = np.array([oracle.tq3_decode_value(int(vc[t, c]), int(sc[c]), int(zp[c])) for t in range(16)])
+        assert np.all(np.abs(vq[:, c] - ref) <= np.maximum(np.abs(ref) * 2.0 ** -4, 2.0 ** -10) + 1e-6)
+    assert np.all(vq[:, 3] == 2.5) and np.array_equal(vq[:, 4], np.float32([0, 3.5] * 8))
+    # scales move the stored bytes, not the dequantised values
+    rec8s = oracle.promote_record(rec3, d, sigma, 0.5, 2.0)
+    ks, vs = oracle.fp8_unpack_record_f32(rec8s, d, 0.5, 2.0)
+    assert np.abs(ks - kq).max() <= np.abs(kq).max() * 2.0 ** -3 and np.all(vs[:, 3] == 2.5)
