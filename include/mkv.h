@@ -161,10 +161,20 @@ int32_t mkv_demote(mkv_pool* pool, const int32_t* src_fp8_ids_dev, const int32_t
                    int32_t n_pages, int32_t* block_table_dev, uint8_t* tier_tag_dev,
                    const int64_t* entry_index_dev, void* stream);
 
+/* Promote (Algorithm 1 step 3; Section 3.1 "A Stale page is materialized and promoted when it
+ * re-enters the protected budget"): reconstruct n_pages TQ3 pages (all KV heads) into newly
+ * allocated FP8 pages, then publish id and MKV_TAG_ANCHOR; arguments as for mkv_demote with the
+ * arenas swapped.  Keys: inverse Walsh-Hadamard of the signed levels times the norm correction and
+ * d^-1/2, rotation signs undone; values: scale * code + zero; both rounded to e4m3 like Append.  The
+ * TQ3 source is not modified; free it once earlier readers are ordered before its next writer. */
+int32_t mkv_promote(mkv_pool* pool, const int32_t* src_tq3_ids_dev, const int32_t* dst_fp8_ids_dev,
+                    int32_t n_pages, int32_t* block_table_dev, uint8_t* tier_tag_dev,
+                    const int64_t* entry_index_dev, void* stream);
+
 /* Protect / unprotect (Fig. lifecycle: Recent -> Anchor): set the tag of one table entry to
  * MKV_TAG_ANCHOR (flag != 0) or MKV_TAG_RECENT (flag == 0).  No data moves.  If the entry is
- * Stale the tag is left alone and MKV_E_STATE is recorded in the status word (a Stale page must
- * be promoted into a new FP8 page first). */
+ * Stale the tag is left alone and MKV_E_STATE is recorded in the status word (a Stale page is
+ * promoted into a new FP8 page with mkv_promote instead). */
 int32_t mkv_set_anchor(mkv_pool* pool, uint8_t* tier_tag_dev, int64_t entry_index, int32_t flag, void* stream);
 
 /* Decode attention (Section 3.3; Section 4.1 "fused decode path"): for every request b and query
@@ -224,6 +234,9 @@ int32_t mkv_seq_protect(mkv_seq* seq, int32_t logical_page, int32_t flag);
 /* Retier to TQ3: allocates the destination, updates the row, releases the source id.  Only full,
  * non-Stale pages qualify (MKV_E_STATE otherwise).  The caller then enqueues mkv_demote(). */
 int32_t mkv_seq_demote(mkv_seq* seq, int32_t logical_page, int32_t* src_fp8_id, int32_t* dst_tq3_id);
+/* Promote: Stale -> Anchor through a newly allocated FP8 page (MKV_E_STATE if the page is not Stale,
+ * MKV_E_OOM_FP8 if none is free).  The caller then enqueues mkv_promote(). */
+int32_t mkv_seq_promote(mkv_seq* seq, int32_t logical_page, int32_t* src_tq3_id, int32_t* dst_fp8_id);
 /* Age: plan the demotion of every full Recent page wholly before the last `recent_tokens`
  * tokens.  Writes up to `cap` triples and returns their number in *n (MKV_E_INVALID if more
  * would be needed; nothing changes then). */

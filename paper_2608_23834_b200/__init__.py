@@ -32,7 +32,7 @@ EXPORTS = [
     "mkv_page_read_raw", "mkv_page_write_raw", "mkv_last_cuda_error", "mkv_append", "mkv_demote",
     "mkv_set_anchor", "mkv_decode_attention", "mkv_seq_create", "mkv_seq_finish", "mkv_seq_append",
     "mkv_seq_protect", "mkv_seq_demote", "mkv_seq_age", "mkv_seq_len", "mkv_seq_row",
-    "mkv_decode_attention_static",
+    "mkv_decode_attention_static", "mkv_promote", "mkv_seq_promote",
 ]
 
 
@@ -82,6 +82,8 @@ def lib():
             "mkv_page_write_raw": [vp, C.c_int32, C.c_int32, vp, vp],
             "mkv_append": [vp, vp, vp, vp, C.c_int32, vp],
             "mkv_demote": [vp, vp, vp, C.c_int32, vp, vp, vp, vp],
+            "mkv_promote": [vp, vp, vp, C.c_int32, vp, vp, vp, vp],
+            "mkv_seq_promote": [vp, C.c_int32, i32p, i32p],
             "mkv_set_anchor": [vp, vp, C.c_int64, C.c_int32, vp],
             "mkv_decode_attention": [vp, vp, vp, vp, vp, C.c_int32, C.c_int32, C.c_float, f32p, f32p, vp,
                                      C.c_size_t, vp],
@@ -230,6 +232,14 @@ class Pool:
         _check(lib().mkv_demote(self.handle, _ptr(src_ids), _ptr(dst_ids), src_ids.numel(), _ptr(block_table),
                                 _ptr(tier_tag), _ptr(entry_index), _stream(stream)), "mkv_demote")
 
+    def promote(self, src_ids: torch.Tensor, dst_ids: torch.Tensor, block_table=None, tier_tag=None, entry_index=None,
+                stream=None) -> None:
+        assert src_ids.dtype == torch.int32 and dst_ids.dtype == torch.int32 and src_ids.numel() == dst_ids.numel()
+        if entry_index is not None:
+            assert entry_index.dtype == torch.int64 and block_table.dtype == torch.int32 and tier_tag.dtype == torch.uint8
+        _check(lib().mkv_promote(self.handle, _ptr(src_ids), _ptr(dst_ids), src_ids.numel(), _ptr(block_table),
+                                 _ptr(tier_tag), _ptr(entry_index), _stream(stream)), "mkv_promote")
+
     def set_anchor(self, tier_tag: torch.Tensor, entry_index: int, flag: bool, stream=None) -> None:
         _check(lib().mkv_set_anchor(self.handle, _ptr(tier_tag), int(entry_index), int(bool(flag)), _stream(stream)),
                "mkv_set_anchor")
@@ -305,6 +315,11 @@ class Seq:
     def demote(self, lp: int):
         a, b = C.c_int32(), C.c_int32()
         _check(lib().mkv_seq_demote(self.handle, lp, C.byref(a), C.byref(b)), "mkv_seq_demote")
+        return a.value, b.value
+
+    def promote(self, lp: int):
+        a, b = C.c_int32(), C.c_int32()
+        _check(lib().mkv_seq_promote(self.handle, lp, C.byref(a), C.byref(b)), "mkv_seq_promote")
         return a.value, b.value
 
     def age(self, recent_tokens: int):

@@ -8,6 +8,8 @@
 #include <cuda_fp16.h>
 #include <cuda_fp8.h>
 
+#include <cmath>
+
 #include "mkv_internal.cuh"
 
 namespace mkv {
@@ -278,6 +280,148 @@ int32_t launch_demote(mkv_pool* p, const int32_t* src, const int32_t* dst, int n
         demote_kernel<256><<<n, 256, 0, s>>>(p->fp8, p->tq3, p->cfg.fp8_pages, p->cfg.tq3_pages, p->hkv,
                                              p->cfg.k_scale, p->cfg.v_scale, p->sigma, src, dst, bt, tags, entry,
                                              p->status_dev);
+    MKV_CUDA(cudaGetLastError());
+    return MKV_OK;
+}
+
+// ------------------------------------------------------------------------------------------ promote
+// Promote (Algorithm 1 step 3): reconstruct a Stale page into a newly allocated FP8 page, then publish
+// it as Anchor.  One block per page, loops over the KV heads.  Warps rebuild key vectors (signed
+// levels, shuffle Walsh-Hadamard, norm correction, sign), threads rebuild value channels; the fp32
+// operation order is fixed so that the written bytes are reproducible.
+template <int D>
+__device__ __forceinline__ uint32_t tq3_lane_word(const uint8_t* section, int lane, int w)
+{
+    return *reinterpret_cast<const uint32_t*>(section + lane_word_offset(D, lane, w));
+}
+
+template <int D>
+__device__ int tq3_key_code_at(const uint8_t* rec, int t, int i)
+{
+    const int kb = i >> 4, s = i & 15;
+    const int lane = 4 * (t & 7) + ((s & 7) >> 1), r = (t >> 3) + 2 * (s >> 3), n = 2 * r + (s & 1), j = kb >> 2;
+    const uint32_t A = tq3_lane_word<D>(rec, lane, 3 * j), Bw = tq3_lane_word<D>(rec, lane, 3 * j + 1),
+                   Cw = tq3_lane_word<D>(rec, lane, 3 * j + 2);
+    switch (kb & 3) {
+    case 0: return (A >> (4 * n)) & 7;
+    case 1: return (Bw >> (4 * n)) & 7;
+    case 2: return ((Cw >> (4 * n)) & 3) | (((A >> (4 * n + 3)) & 1) << 2);
+    default: return ((Cw >> (4 * n + 2)) & 3) | (((Bw >> (4 * n + 3)) & 1) << 2);
+    }
+}
+
+template <int D>
+__device__ int tq3_value_code_at(const uint8_t* rec, int t, int c)
+{
+    const int cb = c >> 4, row = c & 15;
+    const int lane = 4 * (row & 7) + ((t & 7) >> 1), r = (row >> 3) + 2 * (t >> 3), half = t & 1;
+    const int j = cb >> 2, grp = (cb & 3) >> 1, k = 4 * (cb & 1) + r;
+    const uint8_t* sec = rec + 6 * D;
+    const uint32_t W0 = tq3_lane_word<D>(sec, lane, 3 * j), W1 = tq3_lane_word<D>(sec, lane, 3 * j + 1),
+                   W2 = tq3_lane_word<D>(sec, lane, 3 * j + 2);
+    auto by = [](uint32_t w, int b) { return (w >> (8 * b)) & 0xFFu; };
+    uint32_t st;
+    if (grp == 0)
+        st = half == 0 ? (by(W0, 0) | by(W0, 1) << 8 | by(W1, 0) << 16) : (by(W0, 2) | by(W0, 3) << 8 | by(W1, 2) << 16);
+    else
+        st = half == 0 ? (by(W1, 1) | by(W2, 0) << 8 | by(W2, 1) << 16) : (by(W1, 3) | by(W2, 2) << 8 | by(W2, 3) << 16);
+    return (st >> (3 * k)) & 7;
+}
+
+template <int D>
+__global__ void __launch_bounds__(256) promote_kernel(const uint8_t* __restrict__ tq3, uint8_t* __restrict__ fp8,
+                                                       int tq3_pages, int fp8_pages, int hkv, float inv_k_scale,
+                                                       float inv_v_scale, float rs, SigmaBits sigma,
+                                                       const int32_t* __restrict__ src_ids,
+                                                       const int32_t* __restrict__ dst_ids, int32_t* block_table,
+                                                       uint8_t* tier_tag, const int64_t* entry_index,
+                                                       uint32_t* __restrict__ status)
+{
+    constexpr int EPL = D / 32;
+    const int page = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int src = src_ids[page], dst = dst_ids[page];
+    if (src < 0 || src >= tq3_pages || dst < 0 || dst >= fp8_pages) {
+        if (tid == 0) atomicOr(status, kStBounds);
+        return;
+    }
+    const float C[4] = {MKV_C0, MKV_C1, MKV_C2, MKV_C3};
+    for (int h = 0; h < hkv; ++h) {
+        const uint8_t* rec3 = tq3 + ((size_t)src * hkv + h) * tq3_record_bytes(D);
+        uint8_t* rec8 = fp8 + ((size_t)dst * hkv + h) * fp8_record_bytes(D);
+        // ---- keys: warp w rebuilds tokens w and w + 8
+        for (int tok = warp; tok < kPage; tok += 8) {
+            float y[EPL];
+#pragma unroll
+            for (int r = 0; r < EPL; ++r) {
+                const int kc = tq3_key_code_at<D>(rec3, tok, lane * EPL + r);
+                y[r] = (kc & 4) ? -C[kc & 3] : C[kc & 3];
+            }
+#pragma unroll
+            for (int hh = 1; hh < EPL; hh <<= 1)
+#pragma unroll
+                for (int r = 0; r < EPL; ++r)
+                    if ((r & hh) == 0) {
+                        const float u = y[r], w = y[r + hh];
+                        y[r] = __fadd_rn(u, w);
+                        y[r + hh] = __fsub_rn(u, w);
+                    }
+#pragma unroll
+            for (int m = 1; m < 32; m <<= 1)
+#pragma unroll
+                for (int r = 0; r < EPL; ++r) {
+                    const float o = __shfl_xor_sync(0xffffffffu, y[r], m);
+                    y[r] = (lane & m) ? __fsub_rn(o, y[r]) : __fadd_rn(y[r], o);
+                }
+            const float g = __half2float(reinterpret_cast<const __half*>(rec3 + 12 * D)[tok]);
+            const float gr = __fmul_rn(g, rs);
+#pragma unroll
+            for (int r = 0; r < EPL; ++r) {
+                const int i = lane * EPL + r;
+                float k = __fmul_rn(gr, y[r]);
+                if ((sigma.w[i >> 5] >> (i & 31)) & 1u) k = -k;
+                rec8[tok * D + i] = (uint8_t)__nv_cvt_float_to_fp8(__fmul_rn(k, inv_k_scale), __NV_SATFINITE, __NV_E4M3);
+            }
+        }
+        // ---- values: one thread per channel
+        for (int c = tid; c < D; c += 256) {
+            const int cb = c >> 4, row = c & 15;
+            const __half* meta = reinterpret_cast<const __half*>(rec3 + 12 * D + 32);
+            const int mi = (cb >> 1) * 64 + (row & 7) * 8 + 4 * (cb & 1) + (row >> 3);
+            const float sc = __half2float(meta[mi]), zp = __half2float(meta[mi + 2]);
+            uint32_t out[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+            for (int t = 0; t < kPage; ++t) {
+                const float v = __fadd_rn(__fmul_rn(sc, (float)tq3_value_code_at<D>(rec3, t, c)), zp);
+                const uint32_t b = (uint32_t)__nv_cvt_float_to_fp8(__fmul_rn(v, inv_v_scale), __NV_SATFINITE, __NV_E4M3);
+                out[t >> 2] |= b << (8 * (t & 3));
+            }
+            *reinterpret_cast<uint4*>(rec8 + 16 * D + c * kPage) = make_uint4(out[0], out[1], out[2], out[3]);
+        }
+    }
+    // copy-before-publish
+    __threadfence();
+    __syncthreads();
+    if (tid == 0 && entry_index != nullptr) {
+        const int64_t e = entry_index[page];
+        if (e >= 0) {
+            block_table[e] = dst;
+            __threadfence();
+            tier_tag[e] = (uint8_t)MKV_TAG_ANCHOR;
+        }
+    }
+}
+
+int32_t launch_promote(mkv_pool* p, const int32_t* src, const int32_t* dst, int n, int32_t* bt, uint8_t* tags,
+                       const int64_t* entry, cudaStream_t s)
+{
+    const float ik = 1.0f / p->cfg.k_scale, iv = 1.0f / p->cfg.v_scale;
+    const float rs = (float)(1.0 / sqrt((double)p->d));
+    if (p->d == 128)
+        promote_kernel<128><<<n, 256, 0, s>>>(p->tq3, p->fp8, p->cfg.tq3_pages, p->cfg.fp8_pages, p->hkv, ik, iv, rs,
+                                              p->sigma, src, dst, bt, tags, entry, p->status_dev);
+    else
+        promote_kernel<256><<<n, 256, 0, s>>>(p->tq3, p->fp8, p->cfg.tq3_pages, p->cfg.fp8_pages, p->hkv, ik, iv, rs,
+                                              p->sigma, src, dst, bt, tags, entry, p->status_dev);
     MKV_CUDA(cudaGetLastError());
     return MKV_OK;
 }

@@ -283,6 +283,16 @@ int32_t mkv_demote(mkv_pool* pool, const int32_t* src, const int32_t* dst, int32
     return launch_demote(pool, src, dst, n, bt, tags, entry, (cudaStream_t)stream);
 }
 
+int32_t mkv_promote(mkv_pool* pool, const int32_t* src, const int32_t* dst, int32_t n, int32_t* bt, uint8_t* tags,
+                    const int64_t* entry, void* stream)
+{
+    if (!pool || !pool->fp8 || n < 0) return MKV_E_INVALID;
+    if (n == 0) return MKV_OK;
+    if (!src || !dst) return MKV_E_INVALID;
+    if (entry && (!bt || !tags)) return MKV_E_INVALID;
+    return launch_promote(pool, src, dst, n, bt, tags, entry, (cudaStream_t)stream);
+}
+
 int32_t mkv_set_anchor(mkv_pool* pool, uint8_t* tags, int64_t entry, int32_t flag, void* stream)
 {
     if (!pool || !pool->fp8 || !tags || entry < 0) return MKV_E_INVALID;
@@ -376,6 +386,21 @@ int32_t mkv_seq_demote(mkv_seq* seq, int32_t lp, int32_t* src, int32_t* dst)
     seq->ids[lp] = id;
     seq->tags[lp] = MKV_TAG_STALE;
     return mkv_page_free(seq->pool, MKV_FMT_FP8, src, 1);
+}
+
+int32_t mkv_seq_promote(mkv_seq* seq, int32_t lp, int32_t* src, int32_t* dst)
+{
+    if (!seq || !src || !dst) return MKV_E_INVALID;
+    if (lp < 0 || (size_t)lp >= seq->ids.size()) return MKV_E_BOUNDS;
+    if (seq->tags[lp] != MKV_TAG_STALE) return MKV_E_STATE;
+    int32_t id;
+    int32_t rc = mkv_page_alloc(seq->pool, MKV_FMT_FP8, &id, 1);
+    if (rc) return rc;
+    *src = seq->ids[lp];
+    *dst = id;
+    seq->ids[lp] = id;
+    seq->tags[lp] = MKV_TAG_ANCHOR;
+    return mkv_page_free(seq->pool, MKV_FMT_TQ3, src, 1);
 }
 
 int32_t mkv_seq_age(mkv_seq* seq, int32_t recent_tokens, int32_t* lps, int32_t* srcs, int32_t* dsts,

@@ -103,6 +103,8 @@ def test_sequence_bookkeeping_agrees_with_the_lifecycle_model_on_a_random_walk()
             op = ("append",)
         elif r < 0.82:
             op = ("demote", lp)
+        elif r < 0.86:
+            op = ("promote", lp)
         elif r < 0.90:
             op = ("protect", lp, rnd.random() < 0.7)
         elif r < 0.96:
@@ -115,6 +117,8 @@ def test_sequence_bookkeeping_agrees_with_the_lifecycle_model_on_a_random_walk()
                 want = m.append()
             elif op[0] == "demote":
                 want = m.demote(op[1])
+            elif op[0] == "promote":
+                want = m.promote(op[1])
             elif op[0] == "protect":
                 want = m.protect(op[1]) if op[2] else m.unprotect(op[1])
             elif op[0] == "age":
@@ -128,6 +132,8 @@ def test_sequence_bookkeeping_agrees_with_the_lifecycle_model_on_a_random_walk()
                 got = s.append()
             elif op[0] == "demote":
                 got = s.demote(op[1])
+            elif op[0] == "promote":
+                got = s.promote(op[1])
             elif op[0] == "protect":
                 got = s.protect(op[1], op[2])
             elif op[0] == "age":

@@ -127,3 +127,44 @@ def test_set_anchor_flips_fp8_tags_and_refuses_stale():
     pool.set_anchor(tags, 2, True)            # Stale must be promoted first
     assert pool.status() == M.E_STATE
     assert tags.cpu().numpy().tolist() == [[0, 1, 2, 0]]
+
+
+@pytest.mark.parametrize("d,hkv,k_scale,v_scale", [(128, 2, 1.0, 1.0), (256, 4, 1.0, 1.0), (128, 1, 0.5, 2.0)])
+def test_promote_is_bit_exact_and_publishes_anchor(d, hkv, k_scale, v_scale):
+    rng = np.random.default_rng(200 + d + hkv)
+    n = 6
+    sigma = (rng.integers(0, 2, d) * 2 - 1).astype(np.int8)
+    pool = M.Pool(d, hkv, hkv, n + 2, n, sigma, k_scale, v_scale)
+    recs = np.zeros((n, hkv, 16 * d + 32), np.uint8)
+    for p in range(n):
+        for h in range(hkv):
+            k = rng.standard_normal((16, d)).astype(np.float32)
+            v = rng.standard_normal((16, d)).astype(np.float32)
+            k[:, rng.integers(0, d, 3)] *= 8
+            v[:, rng.integers(0, d, 3)] *= 8
+            if p == 0:
+                k[2] = 0.0
+                v[:, 1] = -0.75
+            recs[p, h] = oracle.tq3_record_from_f32(k, v, sigma)
+        pool.page_write_raw(M.FMT_TQ3, p, recs[p])
+    src = torch.from_numpy(rng.permutation(n).astype(np.int32)).cuda()
+    dst = torch.from_numpy(rng.permutation(n + 2)[:n].astype(np.int32)).cuda()
+    bt = torch.full((2, 8), -1, dtype=torch.int32, device="cuda:0")
+    tags = torch.full((2, 8), 2, dtype=torch.uint8, device="cuda:0")
+    entry = torch.arange(n, dtype=torch.int64, device="cuda:0") * 2 + 1
+    pool.promote(src, dst, bt, tags, entry)
+    torch.cuda.synchronize()
+    assert pool.status() == M.OK
+    s, t = src.cpu().numpy(), dst.cpu().numpy()
+    for i in range(n):
+        got = pool.page_read_raw(M.FMT_FP8, int(t[i])).reshape(hkv, 32 * d)
+        for h in range(hkv):
+            ref = oracle.promote_record(recs[s[i], h], d, sigma, k_scale, v_scale)
+            assert np.array_equal(got[h], ref), (i, h, np.nonzero(got[h] != ref)[0][:8])
+        assert np.array_equal(pool.page_read_raw(M.FMT_TQ3, int(s[i])).reshape(hkv, -1), recs[s[i]])   # source untouched
+    btc, tc = bt.cpu().numpy().reshape(-1), tags.cpu().numpy().reshape(-1)
+    for i in range(n):
+        assert btc[2 * i + 1] == t[i] and tc[2 * i + 1] == M.TAG_ANCHOR
+    assert (btc[0::2] == -1).all() and (tc[0::2] == 2).all()
+    pool.promote(torch.tensor([99], dtype=torch.int32, device="cuda:0"), torch.tensor([0], dtype=torch.int32, device="cuda:0"))
+    assert pool.status() == M.E_BOUNDS

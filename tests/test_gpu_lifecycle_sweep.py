@@ -124,6 +124,33 @@ def test_append_demote_decode_cell(frac, ctx, batch):
         torch.cuda.synchronize()
         assert pool.status() == M.OK
         check_close(out.cpu().numpy(), ref, f"cell f={frac} variant={variant}")
+    # ---- Promote (Stale -> Anchor through a new FP8 page) the oldest Stale page of every request, decode again
+    pairs = []
+    for b in range(batch):
+        stale = [lp for lp, (tag, _) in enumerate(mods[b].pages) if tag == STALE]
+        if stale:
+            s_id, t_id = seqs[b].promote(stale[0])
+            assert (s_id, t_id) == mods[b].promote(stale[0])
+            pairs.append((b, stale[0], s_id, t_id))
+    if pairs:
+        for b, lp, s_id, t_id in pairs:
+            for h in range(hkv):
+                fp8[t_id, h] = oracle.promote_record(tq3[s_id, h], d, sigma)
+        src = torch.tensor([p[2] for p in pairs], dtype=torch.int32, device="cuda:0")
+        dst = torch.tensor([p[3] for p in pairs], dtype=torch.int32, device="cuda:0")
+        ent = torch.tensor([p[0] * max_pages + p[1] for p in pairs], dtype=torch.int64, device="cuda:0")
+        pool.promote(src, dst, bt, tags, ent)
+        torch.cuda.synchronize()
+        assert pool.status() == M.OK
+        bt_h, tg_h = bt.cpu().numpy(), tags.cpu().numpy()
+        for b, lp, s_id, t_id in pairs:
+            assert bt_h[b, lp] == t_id and tg_h[b, lp] == M.TAG_ANCHOR
+            assert np.array_equal(pool.page_read_raw(M.FMT_FP8, t_id).reshape(hkv, -1), fp8[t_id])
+        ref, _ = oracle.decode_attention(fp8, tq3, d, hkv, spec.group, sigma, q_bits, bt_h, tg_h, lens, spec.scale)
+        pool.set_decode_variant(M.DECODE_TENSOR)
+        out = pool.decode_attention(bf16_tensor(q_bits), bt, tags, torch.from_numpy(lens).cuda(), spec.scale)
+        check_close(out.cpu().numpy(), ref, f"cell f={frac} after promote")
+        model.check_invariants()
     for s in seqs:
         s.finish()
     assert pool.stats().fp8_pages_used == 0 and pool.stats().tq3_pages_used == 0
