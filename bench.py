@@ -306,7 +306,7 @@ def run_ours(args):
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record(stream)
             L.pool.decode_attention(L.q, L.bt, L.tags, plan["lens"][i], spec.scale, out=L.out)
-            launches[0] += 2                      # scan kernel + merge kernel
+            launches[0] += 1 if args.variant == "tensor" else 2    # tensor: one scan launch; scalar: scan + merge
             if timed_events is not None:
                 e1.record(stream)
                 timed_events.append((e0, e1))
@@ -400,7 +400,7 @@ def run_ours(args):
                    "l2": "inputs larger than L2 (%.0f MB of KV per step)" % (step_bytes / 1e6),
                    "step": "append + demote at its natural cadence + decode attention, every layer"},
         "kv_gbs_whole_step": step_bytes / (ms / K * 1e-3) / 1e9,
-        "roofline": {"bound": "hbm", "kernel": "decode_%s_kernel + merge" % args.variant, "achieved": achieved, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": "decode_tensor_kernel" if args.variant == "tensor" else "decode_scalar_kernel + merge", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_kind + " copy bandwidth",
                      "frac_of_nominal_8000": achieved / 8000.0, "traffic": TRAFFIC_BYTES_PER_LAUNCH if (args.config == 2 and args.ctx == 0 and args.variant == "tensor") else None,
                      "algorithmic_bytes_per_launch": avg_bytes, "avg_launch_ms": avg_kernel_ms,

@@ -93,8 +93,10 @@ int32_t mkv_pool_query(const mkv_pool_config* cfg, size_t* fp8_arena_bytes, size
  * of Section 3.3.  Independent of sequence lengths. */
 int32_t mkv_decode_workspace_bytes(const mkv_pool_config* cfg, int32_t max_batch, size_t* bytes);
 
-/* Clear a workspace buffer.  The decode kernels write every workspace word before they read it, so
- * this is optional; it exists so that a caller can hand over memory with defined contents. */
+/* Clear a workspace buffer.  Call it once on every newly allocated workspace before the first
+ * mkv_decode_attention that uses it: the row tickets at its start (by which the last block of a
+ * split row knows that it has to merge, Eq. softmax-merge) must start at zero.  Every decode call
+ * leaves them at zero again, so one call per allocation is enough. */
 int32_t mkv_workspace_init(void* workspace_dev, size_t bytes, void* stream);
 
 /* Create a pool over caller-owned arenas.  Zero-fills both arenas (so that never-written slots
@@ -187,10 +189,10 @@ int32_t mkv_set_anchor(mkv_pool* pool, uint8_t* tier_tag_dev, int64_t entry_inde
  *                partial (FP8 only); len == 0 gives out = 0 and lse = -inf
  *   out          device, fp32 [B][n_q_heads][d]
  *   lse          device, fp32 [B][n_q_heads] natural-log-sum-exp of the scaled scores, or NULL
- *   workspace    device, at least mkv_decode_workspace_bytes(cfg, B) bytes; two decode calls that
- *                overlap on the GPU need two buffers
- * Two launches: a persistent split-KV scan, and a small kernel that merges the partials of rows
- * that were split over several blocks with Eq. (softmax-merge).  No host synchronisation. */
+ *   workspace    device, at least mkv_decode_workspace_bytes(cfg, B) bytes, cleared once with
+ *                mkv_workspace_init; two decode calls that overlap on the GPU need two buffers
+ * One launch (tensor-core variant): a persistent split-KV scan; the block that finishes a split
+ * row last merges its partials with Eq. (softmax-merge).  No host synchronisation. */
 int32_t mkv_decode_attention(mkv_pool* pool, const void* q_dev, const int32_t* block_table_dev,
                              const uint8_t* tier_tag_dev, const int32_t* seq_lens_dev, int32_t B,
                              int32_t max_pages, float scale, float* out_dev, float* lse_dev,
@@ -210,12 +212,13 @@ int32_t mkv_decode_attention(mkv_pool* pool, const void* q_dev, const int32_t* b
  *   - the pool's device must be the current device.  The first call on a device looks up the array's
  *     device address; make that first call before any stream capture begins.
  *   - all calls on a device share the one array, which keeps whatever the previous call left in it
- *     (every word is rewritten before it is read, so nothing needs clearing).  Two calls that overlap
+ *     (partials are rewritten before they are read; the ticket words start at zero when the library is
+ *     loaded and every call returns them to zero, so nothing needs clearing).  Two calls that overlap
  *     on the GPU, e.g. on different streams, race on it: serialise them or use mkv_decode_attention
  *     with separate workspaces. */
 #define MKV_STATIC_MAX_BLOCKS 160
 #define MKV_STATIC_MAX_BATCH 1024
-#define MKV_STATIC_SCRATCH_BYTES (2u * MKV_STATIC_MAX_BLOCKS * (8u * 256u + 16u) * 4u) /* 2,641,920 bytes */
+#define MKV_STATIC_SCRATCH_BYTES (2u * MKV_STATIC_MAX_BLOCKS * (8u * 256u + 16u) * 4u + 1024u) /* 2,642,944 bytes */
 int32_t mkv_decode_attention_static(mkv_pool* pool, const void* q_dev, const int32_t* block_table_dev,
                                     const uint8_t* tier_tag_dev, const int32_t* seq_lens_dev, int32_t B,
                                     int32_t max_pages, float scale, float* out_dev, float* lse_dev, void* stream);

@@ -15,7 +15,8 @@ namespace {
 
 constexpr int kStaticMaxBlocks = MKV_STATIC_MAX_BLOCKS;
 constexpr size_t kStaticBytes = MKV_STATIC_SCRATCH_BYTES;
-static_assert(kStaticBytes >= (size_t)2 * kStaticMaxBlocks * (8 * 256 + 16) * sizeof(float), "scratch sized for d = 256");
+constexpr size_t kPartialBytes = (size_t)2 * kStaticMaxBlocks * (8 * 256 + 16) * sizeof(float);   // d = 256
+static_assert(kStaticBytes >= kPartialBytes + kStaticMaxBlocks * sizeof(uint32_t), "partials plus one ticket word per block");
 
 // The scratch itself.  In host code this name is only a handle for the runtime, not an address a
 // kernel could use; the device address is asked for once per device (below) and handed to the kernels.
@@ -57,9 +58,12 @@ extern "C" int32_t mkv_decode_attention_static(mkv_pool* pool, const void* q, co
         }
         scratch = g_scratch_addr[dev];
     }
-    // The scan writes every partial slot before the merge reads it, so nothing has to start at zero.
+    // Partial slots are written before they are read.  The ticket words behind them start at zero
+    // (the array is zero-initialised when the module is loaded) and every call leaves them at zero.
+    uint32_t* tickets = reinterpret_cast<uint32_t*>(static_cast<unsigned char*>(scratch) + kPartialBytes);
     const int32_t rc = mkv::launch_decode_tensor_at(pool, q, bt, tags, lens, B, max_pages, scale, out, lse,
-                                                    static_cast<float*>(scratch), kStaticMaxBlocks, (cudaStream_t)stream);
+                                                    static_cast<float*>(scratch), tickets, kStaticMaxBlocks,
+                                                    (cudaStream_t)stream);
     if (rc == MKV_E_INVALID)
         mkv::set_last_error("mkv_decode_attention_static: this GPU launches more blocks than MKV_STATIC_MAX_BLOCKS allows");
     return rc;

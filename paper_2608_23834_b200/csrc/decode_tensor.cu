@@ -21,8 +21,9 @@
 //     MMA against a matrix of ones.  TQ3 values enter that MMA as their integer codes; the
 //     per-channel fp16 scale and zero of the page are applied to the 16x8 result in fp32.
 //   * partial results of a block that covers only part of a (request, KV head) row go to the
-//     workspace; a small merge kernel launched right behind the scan combines them.  No block ever
-//     waits for another.
+//     workspace; every such block then takes a ticket of its row, and the block that draws the last
+//     ticket combines the row's partials (Eq. softmax-merge) and writes the output.  No block ever
+//     waits for another, and there is no second launch.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <math_constants.h>
@@ -33,7 +34,6 @@
 
 namespace mkv {
 
-constexpr int kMaxCtas = 512;        // upper bound of the persistent grid (sizes the workspace)
 constexpr int kMaxBatch = 1024;      // requests per call
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
@@ -59,6 +59,7 @@ struct DecodeParams {
     float* out;
     float* lse;
     float* partials;       // [2 * grid][8*D + 16]
+    uint32_t* tickets;     // [max_blocks] arrival counters of split rows, indexed by the row's first block; zero between calls
     int max_blocks;        // the partial area holds 2 * max_blocks slots
     uint32_t* status;
 };
@@ -332,7 +333,6 @@ __device__ __forceinline__ void partition_blocks_of_row(const Partition* pt, con
 // ------------------------------------------------------------------------------------------------
 // kernel
 // ------------------------------------------------------------------------------------------------
-constexpr int kRound = 128;          // pages of one warp whose table entries are compacted at a time
 
 template <int D, int NW, int NSTAGE>
 struct Geo {
@@ -341,21 +341,24 @@ struct Geo {
     static constexpr int TQ3_REC = 16 * D + 32;
     static constexpr int FP8_HALF = 16 * D;
     static constexpr int SLOT = (TQ3_REC + 127) / 128 * 128;
+    // pages of one warp whose table entries are compacted at a time (fewer where the ring leaves little room)
+    static constexpr int ROUND = NW * NSTAGE * SLOT > 190000 ? 64 : 128;
     static constexpr int RING = NW * NSTAGE * SLOT;
     static constexpr int QROT = NB * 32 * 16;               // rotated query B fragments, hi and lo interleaved
     static constexpr int QPLAIN = NB * 32 * 8;              // plain query B fragments (FP8 pages)
     static constexpr int OFF_QT = RING;
     static constexpr int OFF_QF = OFF_QT + QROT;
     static constexpr int OFF_BAR = OFF_QF + QPLAIN;
-    static constexpr int OFF_LIST = OFF_BAR + NW * NSTAGE * 8;   // [warp][2 formats][kRound] page ids
-    static constexpr int OFF_CUM = OFF_LIST + NW * 2 * kRound * 4;
+    static constexpr int OFF_LIST = OFF_BAR + NW * NSTAGE * 8;   // [warp][2 formats][ROUND] page ids
+    static constexpr int OFF_CUM = OFF_LIST + NW * 2 * ROUND * 4;
     static constexpr int OFF_STRIDE = OFF_CUM + (kMaxBatch + 1) * 4;
     static constexpr int OFF_M = OFF_STRIDE + kMaxBatch * 4;
     static constexpr int OFF_L = OFF_M + NW * 8 * 4;
     static constexpr int OFF_PART = OFF_L + NW * 8 * 4;
-    static constexpr int SMEM = OFF_PART + (int)sizeof(Partition) + 16;
+    static constexpr int OFF_LAST = OFF_PART + ((int)sizeof(Partition) + 15) / 16 * 16;
+    static constexpr int SMEM = OFF_LAST + 16;
     static_assert(NW >= 8, "one warp per column of the 8-wide head group builds the query fragments");
-    static_assert(NSTAGE == 2 || NSTAGE == 4, "ring positions are taken modulo a power of two; an FP8 page takes two slots");
+    static_assert(NSTAGE >= 2 && NSTAGE % 2 == 0 && NSTAGE <= 16, "an FP8 page takes a pair of slots; one phase bit per slot");
     static_assert(NSTAGE * SLOT >= 8 * D * 4, "ring doubles as the cross-warp reduction buffer");
     static_assert(FP8_HALF <= SLOT, "half an FP8 record fits a slot");
 };
@@ -618,6 +621,98 @@ __device__ __forceinline__ void fp8_page(WarpAcc<D / 16>& acc, uint32_t kaddr, u
     }
 }
 
+// Eq. (softmax-merge) of one (request, KV head) row that was split over n_parts blocks.  Part 0 sits
+// in slot first_slot, part j > 0 in slot even_base + 2j.  Called by all NT threads of the block that
+// drew the row's last ticket; `buf` is idle shared memory (n_parts * 16 + 16 floats).  Warp hd < 8
+// reduces the maxima and row sums of head hd (one trip to L2: both are loaded together and kept in
+// shared memory); a thread then owns float4 groups (one channel, four heads) of the [channel][8 heads]
+// tile and has the loads of sixteen parts in flight at a time.
+template <int D, int NT>
+__device__ __forceinline__ void merge_row(const DecodeParams& P, int first_slot, int even_base, int n_parts,
+                                          float* buf, int b, int h)
+{
+    constexpr uint32_t FULL = 0xffffffffu;
+    constexpr int STRIDE = 8 * D + 16, GPT = (2 * D + NT - 1) / NT, KP = 16;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int GQ = P.group, hq = P.hkv * GQ;
+    float* w_s = buf;                        // [n_parts][8] maxima, then weights e^{m_j - m}
+    float* l_s = buf + n_parts * 8;          // [n_parts][8] row sums
+    float* ml_s = buf + n_parts * 16;        // [8] m, [8] l of the row
+    auto slot_of = [&](int j) -> const float* {
+        return P.partials + (size_t)(j == 0 ? first_slot : even_base + 2 * j) * STRIDE;
+    };
+    __syncthreads();
+    if (warp < 8) {
+        const int hd = warp;
+        float M = -CUDART_INF_F;
+        for (int j = lane; j < n_parts; j += 32) {
+            const float* ps = slot_of(j) + 8 * D;
+            const float lj = __ldcg(ps + 8 + hd), mj = __ldcg(ps + hd);
+            l_s[j * 8 + hd] = lj;
+            w_s[j * 8 + hd] = mj;
+            if (lj > 0.f) M = fmaxf(M, mj);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(FULL, M, o));
+        float L = 0.f;
+        for (int j = lane; j < n_parts; j += 32) {      // re-reads this lane's own entries
+            const float lj = l_s[j * 8 + hd];
+            const float w = lj > 0.f ? fast_exp2(w_s[j * 8 + hd] - M) : 0.f;
+            w_s[j * 8 + hd] = w;
+            L = fmaf(w, lj, L);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) L += __shfl_xor_sync(FULL, L, o);
+        if (lane == 0) {
+            ml_s[hd] = M;
+            ml_s[8 + hd] = L;
+        }
+    }
+    float4 acc[GPT];
+#pragma unroll
+    for (int k = 0; k < GPT; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int head0 = (tid & 1) * 4;         // NT is even: every group of this thread covers the same four heads
+    for (int j0 = 0; j0 < n_parts; j0 += KP) {
+        float4 v[KP][GPT];
+#pragma unroll
+        for (int p = 0; p < KP; ++p) {
+            const float* ps = slot_of(min(j0 + p, n_parts - 1));
+#pragma unroll
+            for (int k = 0; k < GPT; ++k)
+                v[p][k] = __ldcg(reinterpret_cast<const float4*>(ps) + min(tid + k * NT, 2 * D - 1));
+        }
+        if (j0 == 0) __syncthreads();        // weights are ready (the loads above did not need them)
+#pragma unroll
+        for (int p = 0; p < KP; ++p)
+            if (j0 + p < n_parts) {
+                const float4 w = *reinterpret_cast<const float4*>(w_s + (j0 + p) * 8 + head0);
+#pragma unroll
+                for (int k = 0; k < GPT; ++k) {
+                    acc[k].x = fmaf(w.x, v[p][k].x, acc[k].x);
+                    acc[k].y = fmaf(w.y, v[p][k].y, acc[k].y);
+                    acc[k].z = fmaf(w.z, v[p][k].z, acc[k].z);
+                    acc[k].w = fmaf(w.w, v[p][k].w, acc[k].w);
+                }
+            }
+    }
+#pragma unroll
+    for (int k = 0; k < GPT; ++k) {
+        const int grp = tid + k * NT, ch = grp >> 1;
+        if (grp >= 2 * D) continue;
+        const float av[4] = {acc[k].x, acc[k].y, acc[k].z, acc[k].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int head = head0 + e;
+            if (head < GQ) {
+                const float L = ml_s[8 + head];
+                P.out[((size_t)b * hq + h * GQ + head) * D + ch] = L > 0.f ? av[e] / L : 0.f;
+            }
+        }
+    }
+    if (P.lse && tid < GQ)
+        P.lse[(size_t)b * hq + h * GQ + tid] = ml_s[8 + tid] > 0.f ? (ml_s[tid] + log2f(ml_s[8 + tid])) * kLn2 : -CUDART_INF_F;
+}
+
 template <int D, int NW, int NSTAGE, int MINB>
 __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const DecodeParams P)
 {
@@ -625,7 +720,6 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
     unsigned long long tl_last = 0;
 #endif
     MKV_STAMP(0);
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     using G = Geo<D, NW, NSTAGE>;
     constexpr int NB = G::NB, NBH = NB, NU = NW;
     constexpr uint32_t FULL = 0xffffffffu;
@@ -636,6 +730,7 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
     float* sm_m = reinterpret_cast<float*>(smem + G::OFF_M);
     float* sm_l = reinterpret_cast<float*>(smem + G::OFF_L);
     Partition* pt = reinterpret_cast<Partition*>(smem + G::OFF_PART);
+    int* last_s = reinterpret_cast<int*>(smem + G::OFF_LAST);
     float* red = reinterpret_cast<float*>(smem);            // [NW][D][8] over the ring, between segments
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tq = lane & 3;
@@ -704,8 +799,8 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
     const uint32_t ring = sbase + warp * NSTAGE * G::SLOT;
     const uint32_t bars = sbase + G::OFF_BAR + warp * NSTAGE * 8;
     const uint32_t qt_lane = sbase + G::OFF_QT + lane * 16, qf_lane = sbase + G::OFF_QF + lane * 8;
-    int* list3 = reinterpret_cast<int*>(smem + G::OFF_LIST) + warp * 2 * kRound;   // Stale page ids of the round
-    int* list8 = list3 + kRound;                                                   // FP8 page ids | valid << 27
+    int* list3 = reinterpret_cast<int*>(smem + G::OFF_LIST) + warp * 2 * G::ROUND;   // Stale page ids of the round
+    int* list8 = list3 + G::ROUND;                                                   // FP8 page ids | valid << 27
     const float sc2 = P.scale * kLog2e;      // scores are kept in log2 units
     // bounded wait for ring slot s, then flip its expected phase
     auto wait_slot = [&](uint32_t s) {
@@ -752,14 +847,14 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
         const uint8_t* tq3_base = P.tq3 + (size_t)h * G::TQ3_REC;
         const uint8_t* fp8_base = P.fp8 + (size_t)h * (2 * G::FP8_HALF);
 
-        // Table entries of up to kRound of the warp's pages are compacted into two id lists, one per
+        // Table entries of up to G::ROUND of the warp's pages are compacted into two id lists, one per
         // format (entry i of a 32-page chunk is read by lane i; ballots give the positions).
         int n3 = 0, n8 = 0;
         auto build_lists = [&](int round) {
             n3 = n8 = 0;
 #pragma unroll 1
-            for (int c = 0; c < kRound / 32; ++c) {
-                const int i = round * kRound + c * 32 + lane;
+            for (int c = 0; c < G::ROUND / 32; ++c) {
+                const int i = round * G::ROUND + c * 32 + lane;
                 int kind = 0, id = 0, valid = kPage;
                 if (i < n_my) {
                     const int pg = (int)(((unsigned)(pg0 + warp + NW * i) * (unsigned)stride) % (unsigned)n_pages);
@@ -783,7 +878,7 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
         };
         auto issue_tq3 = [&](int i) {      // copy Stale page i of the round into ring slot i % NSTAGE
             if (lane == 0) {
-                const uint32_t s = i & (NSTAGE - 1);
+                const uint32_t s = (uint32_t)i % NSTAGE;
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 mbar_expect_tx(bars + 8 * s, G::TQ3_REC);
                 bulk_load(ring + s * G::SLOT, tq3_base + (size_t)list3[i] * hkv * G::TQ3_REC, G::TQ3_REC, bars + 8 * s);
@@ -791,7 +886,7 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
         };
         auto issue_fp8 = [&](int i) {      // copy FP8 page i of the round into the slot pair 2 (i % (NSTAGE/2))
             if (lane == 0) {
-                const uint32_t s = (2 * i) & (NSTAGE - 1);
+                const uint32_t s = (uint32_t)(2 * i) % NSTAGE;
                 const uint8_t* rec = fp8_base + (size_t)(list8[i] & 0x7FFFFFF) * hkv * (2 * G::FP8_HALF);
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 mbar_expect_tx(bars + 8 * s, G::FP8_HALF);
@@ -808,7 +903,7 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
         acc.m[0] = acc.m[1] = -CUDART_INF_F;
 
         // first round: start the copies, then build the query fragments while they fly
-        const int n_rounds = (n_my + kRound - 1) / kRound;
+        const int n_rounds = (n_my + G::ROUND - 1) / G::ROUND;
         if (n_rounds > 0) {
             build_lists(0);
             for (int i = 0; i < min(n3, NSTAGE); ++i) issue_tq3(i);
@@ -875,7 +970,7 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                 wait_slot(0);
                 if (!failed) tq3_step<D, false, true>(acc, 0, pf, ring, qt_lane, sc2, lane, s_cur);
                 for (int i = 0; i + 1 < n3 && !failed; ++i) {
-                    const uint32_t cur = i & (NSTAGE - 1), nxt = (i + 1) & (NSTAGE - 1);
+                    const uint32_t cur = (uint32_t)i % NSTAGE, nxt = (uint32_t)(i + 1) % NSTAGE;
                     wait_slot(nxt);
                     if (failed) break;
                     softmax_page<NB>(acc, s_cur, pf);
@@ -887,7 +982,7 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                 }
                 if (!failed) {
                     softmax_page<NB>(acc, s_cur, pf);
-                    tq3_step<D, true, false>(acc, ring + ((n3 - 1) & (NSTAGE - 1)) * G::SLOT, pf, 0, qt_lane, sc2, lane, s_next);
+                    tq3_step<D, true, false>(acc, ring + ((uint32_t)(n3 - 1) % NSTAGE) * G::SLOT, pf, 0, qt_lane, sc2, lane, s_next);
                 }
                 __syncwarp();
             }
@@ -895,7 +990,7 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
             if (n8 > 0 && !failed) {
                 for (int i = 0; i < min(n8, NSTAGE / 2); ++i) issue_fp8(i);
                 for (int i = 0; i < n8 && !failed; ++i) {
-                    const uint32_t s = (2 * i) & (NSTAGE - 1);
+                    const uint32_t s = (uint32_t)(2 * i) % NSTAGE;
                     wait_slot(s);
                     wait_slot(s + 1);
                     if (failed) break;
@@ -967,8 +1062,8 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                 P.lse[(size_t)b * hq + h * GQ + tid] = l > 0.f ? (M + log2f(l)) * kLn2 : -CUDART_INF_F;
             }
         } else {
-            // partial (m, l, O) of this block for the row, merged by the merge kernel that follows;
-            // slot 2c if the segment opens the block's range, 2c + 1 otherwise
+            // partial (m, l, O) of this block for the row; slot 2c if the segment opens the block's range,
+            // 2c + 1 otherwise
             float* slot = P.partials + (size_t)(2 * blockIdx.x + (pos != my_start ? 1 : 0)) * (8 * D + 16);
             for (int e = tid; e < 8 * D; e += NW * 32) {
                 float acc = 0.f;
@@ -985,130 +1080,31 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                 slot[8 * D + tid] = M;
                 slot[8 * D + 8 + tid] = l;
             }
+            // ticket of the row: the block that draws the last one merges (its loads then see every
+            // other block's partial: store -> fence -> ticket on their side, ticket -> fence -> load here)
+            int c0, c1;
+            partition_blocks_of_row(pt, cum, P.B, b * hkv + h, row_start, row_end, c0, c1);
+            const int n_parts = c1 - c0 + 1;
+            __syncthreads();
+            if (tid == 0) {
+                __threadfence();
+                const uint32_t prev = atomicAdd(P.tickets + c0, 1u);
+                const int last = prev == (uint32_t)(n_parts - 1);
+                if (last) P.tickets[c0] = 0;           // leave the counter cleared for the next call
+                *last_s = last;
+            }
+            __syncthreads();
+            if (*last_s) {
+                __threadfence();
+                MKV_STAMP(6);
+                const int first_slot = 2 * c0 + (row_start > partition_start(pt, cum, hkv, P.B, c0) ? 1 : 0);
+                merge_row<D, NW * 32>(P, first_slot, 2 * c0, n_parts, red, b, h);
+                MKV_STAMP(7);
+            }
         }
         __syncthreads();
         MKV_STAMP(8);
         pos += n_seg;
-    }
-}
-
-// Eq. (softmax-merge) for every (request, KV head) row that was split over several blocks of the scan
-// kernel: one block per row and half of the channels; a thread owns one channel and four heads, and
-// issues the loads of all partials before it uses any.  Rows that a single block covered were written
-// by that block and are skipped here.
-template <int D>
-__global__ void __launch_bounds__(D) decode_merge_kernel(const DecodeParams P, int scan_grid)
-{
-    constexpr uint32_t FULL = 0xffffffffu;
-    constexpr int kMaxParts = 40;          // loads in flight per thread; longer rows take several rounds
-    __shared__ int cum[kMaxBatch + 1];
-    __shared__ __align__(16) float w_s[kMaxCtas * 8];    // weight of every partial and head (read as float4)
-    __shared__ float l_s[kMaxCtas * 8];                  // row sums of every partial and head
-    __shared__ int slot_s[kMaxCtas];                     // workspace slot of every partial
-    __shared__ Partition pt_s;
-    __shared__ float ml_s[16];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int hkv = P.hkv, GQ = P.group, hq = hkv * GQ;
-    if (warp == 0) {
-        int run = 0;
-        for (int b0 = 0; b0 < P.B; b0 += 32) {
-            const int b = b0 + lane;
-            int n = 0;
-            if (b < P.B) {
-                const int len = P.lens[b];
-                n = len > 0 ? ((len + kPage - 1) / kPage) * hkv : 0;
-            }
-            int inc = n;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int v = __shfl_up_sync(FULL, inc, o);
-                if (lane >= o) inc += v;
-            }
-            if (b < P.B) cum[b] = run + inc - n;
-            run += __shfl_sync(FULL, inc, 31);
-        }
-        if (lane == 0) cum[P.B] = run;
-    }
-    __syncthreads();
-    const long long W = cum[P.B];
-    if (warp == 0 && W > 0) build_partition(&pt_s, cum, P.lens, P.B, hkv, scan_grid, lane);
-    __syncthreads();
-    const Partition* pt = &pt_s;
-    // everything above read only the call's inputs; the partials below are the scan kernel's output
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    if (W == 0) return;
-    for (int row = blockIdx.x; row < P.B * hkv; row += gridDim.x) {
-        const int b = row / hkv, h = row % hkv;
-        const int len = P.lens[b];
-        if (len <= 0) continue;
-        const int n_pages = (len + kPage - 1) / kPage;
-        const int row_start = cum[b] + h * n_pages, row_end = row_start + n_pages;
-        int c0, c1;
-        partition_blocks_of_row(pt, cum, P.B, row, row_start, row_end, c0, c1);
-        if (c0 == c1) continue;                                   // written by its only block
-        const int n_parts = c1 - c0 + 1;
-        __syncthreads();
-        // a block's slot for this row: 2c if the row's part opens the block's range, 2c + 1 otherwise
-        for (int j = tid; j < n_parts; j += D)
-            slot_s[j] = 2 * (c0 + j) + (row_start > partition_start(pt, cum, hkv, P.B, c0 + j) ? 1 : 0);
-        __syncthreads();
-        auto slot_of = [&](int j) -> const float* { return P.partials + (size_t)slot_s[j] * (8 * D + 16); };
-        // maxima and row sums of all parts -> weights e^{m_j - m} and the total l
-        for (int i = tid; i < n_parts * 8; i += D) {
-            const float* ps = slot_of(i >> 3) + 8 * D;
-            const float lj = __ldcg(ps + 8 + (i & 7));
-            l_s[i] = lj;
-            w_s[i] = lj > 0.f ? __ldcg(ps + (i & 7)) : -CUDART_INF_F;
-        }
-        __syncthreads();
-        if (tid < 8) {
-            float M = -CUDART_INF_F;
-            for (int j = 0; j < n_parts; ++j) M = fmaxf(M, w_s[j * 8 + tid]);
-            ml_s[tid] = M;
-        }
-        __syncthreads();
-        for (int i = tid; i < n_parts * 8; i += D) {
-            const float mj = w_s[i];
-            w_s[i] = mj == -CUDART_INF_F ? 0.f : fast_exp2(mj - ml_s[i & 7]);
-        }
-        __syncthreads();
-        if (tid < 8) {
-            float L = 0.f;
-            for (int j = 0; j < n_parts; ++j) L += w_s[j * 8 + tid] * l_s[j * 8 + tid];
-            ml_s[8 + tid] = L;
-        }
-        __syncthreads();
-        // thread = (channel, half of the heads): this block covers the channels blockIdx.y*D/2 ...
-        const int ch = blockIdx.y * (D / 2) + (tid >> 1), head0 = (tid & 1) * 4;
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int j0 = 0; j0 < n_parts; j0 += kMaxParts) {
-            float4 v[kMaxParts];
-#pragma unroll
-            for (int k = 0; k < kMaxParts; ++k) {
-                const int j = min(j0 + k, n_parts - 1);
-                v[k] = __ldcg(reinterpret_cast<const float4*>(slot_of(j) + ch * 8 + head0));
-            }
-#pragma unroll
-            for (int k = 0; k < kMaxParts; ++k)
-                if (j0 + k < n_parts) {
-                    const float4 w = *reinterpret_cast<const float4*>(w_s + (j0 + k) * 8 + head0);
-                    acc.x = fmaf(w.x, v[k].x, acc.x);
-                    acc.y = fmaf(w.y, v[k].y, acc.y);
-                    acc.z = fmaf(w.z, v[k].z, acc.z);
-                    acc.w = fmaf(w.w, v[k].w, acc.w);
-                }
-        }
-        const float av[4] = {acc.x, acc.y, acc.z, acc.w};
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const int head = head0 + k;
-            if (head < GQ) {
-                const float L = ml_s[8 + head];
-                P.out[((size_t)b * hq + h * GQ + head) * D + ch] = L > 0.f ? av[k] / L : 0.f;
-            }
-        }
-        if (P.lse && blockIdx.y == 0 && tid < GQ)
-            P.lse[(size_t)b * hq + h * GQ + tid] = ml_s[8 + tid] > 0.f ? (ml_s[tid] + log2f(ml_s[8 + tid])) * kLn2 : -CUDART_INF_F;
     }
 }
 
@@ -1130,22 +1126,6 @@ static int32_t run_tensor(mkv_pool* p, DecodeParams& prm, cudaStream_t s)
     if (grid_cache[dev] > prm.max_blocks) return MKV_E_INVALID;
     kern<<<grid_cache[dev], NW * 32, G::SMEM, s>>>(prm);
     MKV_CUDA(cudaGetLastError());
-    // rows split over several blocks: at most one per block boundary, never more than the rows there are
-    int rows = prm.B * prm.hkv;
-    if (rows > grid_cache[dev]) rows = grid_cache[dev];
-    // programmatic dependent launch: the merge blocks become resident while the scan drains and wait
-    // (griddepcontrol.wait) for its completion before they read the partials
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(rows, 2);
-    cfg.blockDim = dim3(D);
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    MKV_CUDA(cudaLaunchKernelEx(&cfg, decode_merge_kernel<D>, prm, grid_cache[dev]));
     return MKV_OK;
 }
 
@@ -1171,15 +1151,17 @@ int32_t launch_decode_tensor(mkv_pool* p, const void* q, const int32_t* bt, cons
                              const int32_t* lens, int B, int max_pages, float scale, float* out, float* lse,
                              void* ws, size_t, cudaStream_t s)
 {
+    // header: 256 reserved bytes, then kMaxCtas ticket words (cleared by mkv_workspace_init, left clear by every call)
+    uint32_t* tickets = reinterpret_cast<uint32_t*>(static_cast<uint8_t*>(ws) + 256);
     float* partials = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + decode_ws_header_bytes(B, p->hkv));
-    return launch_decode_tensor_at(p, q, bt, tags, lens, B, max_pages, scale, out, lse, partials, kMaxCtas, s);
+    return launch_decode_tensor_at(p, q, bt, tags, lens, B, max_pages, scale, out, lse, partials, tickets, kMaxCtas, s);
 }
 
 int decode_tensor_partial_floats(int d) { return 8 * d + 16; }
 
 int32_t launch_decode_tensor_at(mkv_pool* p, const void* q, const int32_t* bt, const uint8_t* tags,
                                 const int32_t* lens, int B, int max_pages, float scale, float* out, float* lse,
-                                float* partials, int max_blocks, cudaStream_t s)
+                                float* partials, uint32_t* tickets, int max_blocks, cudaStream_t s)
 {
     if (B > kMaxBatch) return MKV_E_INVALID;
     DecodeParams prm;
@@ -1193,6 +1175,7 @@ int32_t launch_decode_tensor_at(mkv_pool* p, const void* q, const int32_t* bt, c
     prm.B = B; prm.max_pages = max_pages; prm.scale = scale;
     prm.out = out; prm.lse = lse;
     prm.partials = partials;
+    prm.tickets = tickets;
     prm.max_blocks = max_blocks;
     prm.status = p->status_dev;
     // Launch shapes (warps per block, ring slots per warp, blocks per SM); MKV_DECODE_SHAPE selects the
@@ -1207,8 +1190,8 @@ int32_t launch_decode_tensor_at(mkv_pool* p, const void* q, const int32_t* bt, c
         }
     }
     switch (shape) {
-    case 1: return run_tensor<256, 16, 2, 1>(p, prm, s);
-    case 2: return run_tensor<256, 12, 2, 1>(p, prm, s);
+    case 1: return run_tensor<256, 8, 6, 1>(p, prm, s);
+    case 2: return run_tensor<256, 12, 4, 1>(p, prm, s);
     case 3: return run_tensor<256, 10, 4, 1>(p, prm, s);
     default: return run_tensor<256, 8, 4, 1>(p, prm, s);
     }

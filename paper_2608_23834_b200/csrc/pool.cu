@@ -36,7 +36,9 @@ static int32_t check_cfg(const mkv_pool_config* c)
 
 size_t decode_ws_header_bytes(int B, int hkv)
 {
-    size_t b = 256 + sizeof(uint32_t) * (size_t)B * hkv;
+    // 256 reserved bytes, then the row tickets of the tensor-core scan (one word per possible block)
+    (void)B; (void)hkv;
+    size_t b = 256 + sizeof(uint32_t) * (size_t)kMaxCtas;
     return (b + 255) / 256 * 256;
 }
 
@@ -74,7 +76,7 @@ int32_t mkv_decode_workspace_bytes(const mkv_pool_config* cfg, int32_t max_batch
 int32_t mkv_workspace_init(void* ws, size_t bytes, void* stream)
 {
     if (!ws || bytes < 256 || !aligned(ws, 256)) return MKV_E_INVALID;
-    // tickets live in the header; partial slots need no initialisation
+    // the ticket words in the header must start at zero; partial slots need no initialisation
     MKV_CUDA(cudaMemsetAsync(ws, 0, bytes, (cudaStream_t)stream));
     return MKV_OK;
 }
