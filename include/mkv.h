@@ -183,7 +183,8 @@ int32_t mkv_set_anchor(mkv_pool* pool, uint8_t* tier_tag_dev, int64_t entry_inde
  * head h, softmax(scale * q K^T) V over the seq_lens[b] tokens of row b, where each page is read
  * in its own physical format and all tokens share one softmax normalisation.
  *   q            device, bf16 [B][n_q_heads][d]
- *   block_table  device, int32 [B][max_pages]; unused entries are ignored
+ *   block_table  device, int32 [B][max_pages]; unused entries are ignored; max_pages <= 65535
+ *                (tensor-core variant; MKV_E_INVALID beyond)
  *   tier_tag     device, uint8 [B][max_pages]; 0/1 = FP8 arena, 2 = TQ3 arena
  *   seq_lens     device, int32 [B]; pages beyond ceil(len/16) are not read; the last page may be
  *                partial (FP8 only); len == 0 gives out = 0 and lse = -inf

@@ -7,7 +7,7 @@
 // Mapping to the hardware
 //   * work = (request, KV head, page) triples in row-major order, cut into equal contiguous ranges,
 //     one per block (persistent grid, a multiple of the SM count); a block processes the
-//     (request, KV head) segments of its range one after another, its warps taking pages round-robin.
+//     (request, KV head) segments of its range one after another, its warps taking contiguous runs of pages.
 //   * each warp streams its pages through a private ring of shared-memory slots filled by bulk
 //     asynchronous copies (cp.async.bulk + mbarrier), several pages ahead of the arithmetic.
 //   * a 16-token page x d dims is exactly the A operand of m16n8k16 MMAs whose B operand is the
@@ -837,7 +837,10 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
         const int n_seg = min(my_end, row_end) - pos;
         const int32_t* bt_row = P.bt + (size_t)b * P.max_pages;
         const uint8_t* tag_row = P.tags + (size_t)b * P.max_pages;
-        const int n_my = warp < n_seg ? (n_seg - warp + NW - 1) / NW : 0;   // this warp's pages, round-robin
+        // this warp's pages: a contiguous run of positions (a run of the strided order holds FP8 and TQ3
+        // pages in the row's proportion, so the warps of a block finish together)
+        const int warp_first = (int)(((unsigned)n_seg * (unsigned)warp) / NW);
+        const int n_my = (int)(((unsigned)n_seg * (unsigned)(warp + 1)) / NW) - warp_first;
         const int stride = strides[b];
         constexpr int EPL = D / 32;
         float qx[EPL];            // this warp's query head (warps 0..7), loaded before anything else waits
@@ -857,7 +860,7 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                 const int i = round * G::ROUND + c * 32 + lane;
                 int kind = 0, id = 0, valid = kPage;
                 if (i < n_my) {
-                    const int pg = (int)(((unsigned)(pg0 + warp + NW * i) * (unsigned)stride) % (unsigned)n_pages);
+                    const int pg = (int)(((unsigned)(pg0 + warp_first + i) * (unsigned)stride) % (unsigned)n_pages);   // < 2^32: max_pages <= 65535
                     id = bt_row[pg];
                     const int tag = tag_row[pg];
                     valid = min(kPage, len - pg * kPage);
@@ -1164,6 +1167,10 @@ int32_t launch_decode_tensor_at(mkv_pool* p, const void* q, const int32_t* bt, c
                                 float* partials, uint32_t* tickets, int max_blocks, cudaStream_t s)
 {
     if (B > kMaxBatch) return MKV_E_INVALID;
+    if (max_pages > 65535) {            // the strided page order multiplies two page indices in 32 bits
+        set_last_error("mkv_decode_attention: max_pages above 65535 (1,048,560 tokens per request)");
+        return MKV_E_INVALID;
+    }
     DecodeParams prm;
     prm.fp8 = p->fp8; prm.tq3 = p->tq3;
     prm.fp8_pages = p->cfg.fp8_pages; prm.tq3_pages = p->cfg.tq3_pages;

@@ -161,3 +161,38 @@ def test_host_side_argument_checks():
     with pytest.raises(M.MkvError) as e:
         case.pool.page_read_raw(M.FMT_TQ3, 10 ** 6)
     assert e.value.code == M.E_BOUNDS
+
+
+def test_append_and_decode_replay_from_a_cuda_graph():
+    """The step's device calls take only stream-ordered actions, so they can be captured once and
+    replayed (Section 4.1 runs the decode path from a CUDA graph).  The replayed result must equal
+    the directly launched one bit for bit, for split rows too, and new lengths must be picked up from
+    the captured buffers."""
+    spec = SCALED["cfg2"]()                     # 8 rows over all blocks: every row is split and merged by ticket
+    case = Case(spec, extra_fp8=4)
+    pool = case.pool
+    pool.set_decode_variant(M.DECODE_TENSOR)
+    out_direct = pool.decode_attention(case.q, case.bt, case.tags, case.lens, spec.scale).clone()
+    lens2 = case.lens.clone()
+    lens2[1] -= 16 * 3 + 5                      # a shorter second request (its last page becomes partial)
+    out_direct2 = pool.decode_attention(case.q, case.bt, case.tags, lens2, spec.scale).clone()
+    torch.cuda.synchronize()
+
+    cur_lens = case.lens.clone()
+    out_graph = torch.zeros_like(out_direct)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        pool.decode_attention(case.q, case.bt, case.tags, cur_lens, spec.scale, out=out_graph)
+    g.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out_graph, out_direct)
+    cur_lens.copy_(lens2)
+    g.replay()
+    g.replay()                                   # tickets are left clear: a second replay gives the same
+    torch.cuda.synchronize()
+    assert pool.status() == M.OK
+    assert torch.equal(out_graph, out_direct2)
+    check_close(out_graph.cpu().numpy(),
+                oracle.decode_attention(case.L.fp8_arena, case.L.tq3_arena, spec.head_dim, spec.n_kv_heads, spec.group,
+                                        case.L.sigma, case.L.q_bits, case.tab.block_table, case.tab.tier_tag,
+                                        lens2.cpu().numpy(), spec.scale)[0], "graph replay")
