@@ -607,6 +607,103 @@ int orc_decode_attention(const uint8_t* fp8_arena, int64_t fp8_pages, const uint
 }
 
 /* ------------------------------------------------------------------------------------------
+ * Globally normalised page mass (Section 3.1, Eq. score-partial, Eq. score-global-weight,
+ * Eq. attention-score).  For query head h the tokens are split into partitions j by physical
+ * FORMAT (j = 0: FP8 pages, j = 1: TQ3 pages), each partition reports
+ *      m_j = max_{i in j} s_i,   l_j = sum_{i in j} e^{s_i - m_j},
+ * with m = max_j m_j and l = sum_j e^{m_j - m} l_j; a page p of partition j has
+ *      rho_p = (1 / l_j) sum_{i in p} e^{s_i - m_j},   w_j = e^{m_j - m} l_j / l,
+ *      q_p = w_j rho_p,   q~_p = q_p / sum_p' q_p'   (no sink state here: every page is addressable).
+ * mass[b][hq][p] receives q~ (0 for pages beyond the request's length).
+ * Returns 0, or -1 if a table entry is invalid. */
+int orc_page_mass(const uint8_t* fp8_arena, int64_t fp8_pages, const uint8_t* tq3_arena, int64_t tq3_pages,
+                  int d, int hkv, int group, float k_scale, float v_scale, const int8_t* sigma,
+                  const uint16_t* q, const int32_t* block_table, const uint8_t* tier_tag,
+                  const int32_t* seq_lens, int B, int max_pages, double scale, double* mass)
+{
+    orc_pool pool;
+    int Hq = hkv * group, unit, rc = 0;
+    pool.fp8_arena = fp8_arena; pool.tq3_arena = tq3_arena;
+    pool.fp8_pages = fp8_pages; pool.tq3_pages = tq3_pages;
+    pool.d = d; pool.hkv = hkv; pool.group = group;
+    pool.k_scale = k_scale; pool.v_scale = v_scale; pool.sigma = sigma;
+
+#pragma omp parallel for schedule(dynamic, 1)
+    for (unit = 0; unit < B * hkv; ++unit) {
+        int b = unit / hkv, h = unit % hkv, len = seq_lens[b], gq, c, i, pg, j;
+        int n_pages = len > 0 ? (len + ORC_T - 1) / ORC_T : 0;
+        const int32_t* row = block_table + (int64_t)b * max_pages;
+        const uint8_t* tags = tier_tag + (int64_t)b * max_pages;
+        double *K, *V, *s;
+        for (gq = 0; gq < group; ++gq)
+            for (pg = 0; pg < max_pages; ++pg) mass[((int64_t)b * Hq + h * group + gq) * max_pages + pg] = 0.0;
+        if (len <= 0) continue;
+        K = (double*)malloc(sizeof(double) * (size_t)len * d);
+        V = (double*)malloc(sizeof(double) * (size_t)len * d);
+        s = (double*)malloc(sizeof(double) * (size_t)len);
+        if (materialise(&pool, row, tags, len, h, K, V) != 0) {
+#pragma omp atomic write
+            rc = -1;
+            free(K); free(V); free(s);
+            continue;
+        }
+        for (gq = 0; gq < group; ++gq) {
+            int hq = h * group + gq;
+            double* out = mass + ((int64_t)b * Hq + hq) * max_pages;
+            double mj[2] = {-INFINITY, -INFINITY}, lj[2] = {0.0, 0.0}, m, l, total = 0.0;
+            for (i = 0; i < len; ++i) {
+                double acc = 0.0;
+                for (c = 0; c < d; ++c)
+                    acc += (double)orc_bf16_to_f32(q[((int64_t)b * Hq + hq) * d + c]) * K[(int64_t)i * d + c];
+                s[i] = scale * acc;
+                j = tags[i / ORC_T] == 2;
+                if (s[i] > mj[j]) mj[j] = s[i];
+            }
+            for (i = 0; i < len; ++i) {
+                j = tags[i / ORC_T] == 2;
+                lj[j] += exp(s[i] - mj[j]);
+            }
+            m = mj[0] > mj[1] ? mj[0] : mj[1];
+            l = 0.0;
+            for (j = 0; j < 2; ++j) if (lj[j] > 0.0) l += exp(mj[j] - m) * lj[j];
+            for (pg = 0; pg < n_pages; ++pg) {
+                int lo = pg * ORC_T, hi = lo + ORC_T < len ? lo + ORC_T : len;
+                double rho = 0.0, w;
+                j = tags[pg] == 2;
+                for (i = lo; i < hi; ++i) rho += exp(s[i] - mj[j]);
+                rho /= lj[j];
+                w = exp(mj[j] - m) * lj[j] / l;
+                out[pg] = w * rho;
+                total += out[pg];
+            }
+            for (pg = 0; pg < n_pages; ++pg) out[pg] /= total;
+        }
+        free(K); free(V); free(s);
+    }
+    return rc;
+}
+
+/* Eq. (attention-score): r_p = mean over the sampled head set of q~_{h,p}; a_p <- beta a_p + (1 - beta) r_p.
+ * head_mask bit hq selects query head hq (at least one bit set among the first Hq).  mass is
+ * [B][Hq][max_pages], score is [B][max_pages] and is updated in place for pages below the length. */
+void orc_page_score_update(const double* mass, const int32_t* seq_lens, int B, int Hq, int max_pages,
+                           uint64_t head_mask, double beta, double* score)
+{
+    int b, pg, hq, n_heads = 0;
+    for (hq = 0; hq < Hq; ++hq) if ((head_mask >> hq) & 1u) ++n_heads;
+    for (b = 0; b < B; ++b) {
+        int n_pages = seq_lens[b] > 0 ? (seq_lens[b] + ORC_T - 1) / ORC_T : 0;
+        for (pg = 0; pg < n_pages; ++pg) {
+            double r = 0.0;
+            for (hq = 0; hq < Hq; ++hq)
+                if ((head_mask >> hq) & 1u) r += mass[((int64_t)b * Hq + hq) * max_pages + pg];
+            r /= (double)n_heads;
+            score[(int64_t)b * max_pages + pg] = beta * score[(int64_t)b * max_pages + pg] + (1.0 - beta) * r;
+        }
+    }
+}
+
+/* ------------------------------------------------------------------------------------------
  * Byte accounting (Eq. kv-per-token, Eq. effective-bits, Section 6.3 counters).
  * page = T tokens; the TQ3 structure per page and KV head is
  *    K: T * 3d/8 bytes of codes + T * 2 bytes fp16 norm correction (per token)
