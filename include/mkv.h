@@ -224,6 +224,31 @@ int32_t mkv_decode_attention_static(mkv_pool* pool, const void* q_dev, const int
                                     const uint8_t* tier_tag_dev, const int32_t* seq_lens_dev, int32_t B,
                                     int32_t max_pages, float scale, float* out_dev, float* lse_dev, void* stream);
 
+/* Section 3.1 (Eq. score-partial, Eq. score-global-weight): mkv_decode_attention that also reports
+ * the globally normalised attention mass of every page, taken from the same scores, the same softmax
+ * and the same one pass over the mixed-format pages as the output (no dense view of the cache).
+ *   page_mass    device, fp32 [B][n_q_heads][max_pages]: q~_{h,p} = sum over the tokens of page p of
+ *                softmax weight of head h, divided by the sum over all pages (1 up to rounding, since
+ *                every page is addressable); pages beyond ceil(len/16) are set to 0
+ *   lse          required here (the second launch needs it)
+ * Other arguments, workspace and errors as mkv_decode_attention; always the tensor-core kernel.
+ * Two launches: the scan (which stores log2 of every page's exponential sum) and a small kernel
+ * that refers them to the row's log-sum-exp and normalises. */
+int32_t mkv_decode_attention_scored(mkv_pool* pool, const void* q_dev, const int32_t* block_table_dev,
+                                    const uint8_t* tier_tag_dev, const int32_t* seq_lens_dev, int32_t B,
+                                    int32_t max_pages, float scale, float* out_dev, float* lse_dev,
+                                    float* page_mass_dev, void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/* Eq. (attention-score): r_p = mean over the sampled head set of q~_{h,p}, a_p <- beta a_p + (1-beta) r_p
+ * for every page below each request's length (others untouched).
+ *   page_mass    device, fp32 [B][n_q_heads][max_pages] from mkv_decode_attention_scored
+ *   head_mask    bit h selects query head h (n_q_heads <= 64); no selected head: MKV_E_INVALID
+ *   beta         in [0, 1]
+ *   score        device, fp32 [B][max_pages], updated in place */
+int32_t mkv_page_score_update(const float* page_mass_dev, const int32_t* seq_lens_dev, int32_t B,
+                              int32_t n_q_heads, int32_t max_pages, uint64_t head_mask, float beta,
+                              float* score_dev, void* stream);
+
 /* ---- host-side sequence bookkeeping (Algorithm 1; no device work) ------------------------- */
 
 /* A sequence owns a row of logical pages -> (tag, physical id).  These calls only plan: they

@@ -33,6 +33,7 @@ EXPORTS = [
     "mkv_set_anchor", "mkv_decode_attention", "mkv_seq_create", "mkv_seq_finish", "mkv_seq_append",
     "mkv_seq_protect", "mkv_seq_demote", "mkv_seq_age", "mkv_seq_len", "mkv_seq_row",
     "mkv_decode_attention_static", "mkv_promote", "mkv_seq_promote",
+    "mkv_decode_attention_scored", "mkv_page_score_update",
 ]
 
 
@@ -88,6 +89,9 @@ def lib():
             "mkv_decode_attention": [vp, vp, vp, vp, vp, C.c_int32, C.c_int32, C.c_float, f32p, f32p, vp,
                                      C.c_size_t, vp],
             "mkv_decode_attention_static": [vp, vp, vp, vp, vp, C.c_int32, C.c_int32, C.c_float, f32p, f32p, vp],
+            "mkv_decode_attention_scored": [vp, vp, vp, vp, vp, C.c_int32, C.c_int32, C.c_float, f32p, f32p, f32p, vp,
+                                            C.c_size_t, vp],
+            "mkv_page_score_update": [f32p, vp, C.c_int32, C.c_int32, C.c_int32, C.c_uint64, C.c_float, f32p, vp],
             "mkv_seq_create": [vp, C.POINTER(vp)],
             "mkv_seq_finish": [vp],
             "mkv_seq_append": [vp, i32p, i32p, i32p],
@@ -257,6 +261,39 @@ class Pool:
                                           block_table.shape[1], float(scale), _ptr(out), _ptr(lse), _ptr(ws),
                                           ws.numel(), _stream(stream)), "mkv_decode_attention")
         return out
+
+    def decode_attention_scored(self, q, block_table, tier_tag, seq_lens, scale, out=None, lse=None, page_mass=None,
+                                workspace=None, stream=None):
+        """mkv_decode_attention_scored: returns (out, lse, page_mass [B][hq][max_pages])."""
+        B = q.shape[0]
+        assert q.dtype == torch.bfloat16 and q.is_contiguous() and q.shape == (B, self.hq, self.d)
+        assert block_table.dtype == torch.int32 and block_table.is_contiguous() and block_table.shape[0] == B
+        assert tier_tag.dtype == torch.uint8 and tier_tag.shape == block_table.shape and tier_tag.is_contiguous()
+        assert seq_lens.dtype == torch.int32 and seq_lens.numel() == B
+        if out is None:
+            out = torch.empty((B, self.hq, self.d), dtype=torch.float32, device=q.device)
+        if lse is None:
+            lse = torch.empty((B, self.hq), dtype=torch.float32, device=q.device)
+        if page_mass is None:
+            page_mass = torch.empty((B, self.hq, block_table.shape[1]), dtype=torch.float32, device=q.device)
+        ws = self.workspace if workspace is None else workspace
+        _check(lib().mkv_decode_attention_scored(self.handle, _ptr(q), _ptr(block_table), _ptr(tier_tag), _ptr(seq_lens),
+                                                 B, block_table.shape[1], float(scale), _ptr(out), _ptr(lse),
+                                                 _ptr(page_mass), _ptr(ws), ws.numel(), _stream(stream)),
+               "mkv_decode_attention_scored")
+        return out, lse, page_mass
+
+
+def page_score_update(page_mass, seq_lens, head_mask, beta, score, stream=None):
+    """mkv_page_score_update (Eq. attention-score): score <- beta * score + (1 - beta) * mean over the heads in
+    head_mask of page_mass, in place, for the pages below each request's length."""
+    B, hq, max_pages = page_mass.shape
+    assert page_mass.dtype == torch.float32 and page_mass.is_contiguous()
+    assert score.dtype == torch.float32 and score.is_contiguous() and score.shape == (B, max_pages)
+    assert seq_lens.dtype == torch.int32 and seq_lens.numel() == B
+    _check(lib().mkv_page_score_update(_ptr(page_mass), _ptr(seq_lens), B, hq, max_pages, C.c_uint64(int(head_mask)),
+                                       float(beta), _ptr(score), _stream(stream)), "mkv_page_score_update")
+    return score
 
 
 def decode_attention_static(pool: "Pool", q, block_table, tier_tag, seq_lens, scale, out=None, lse=None, stream=None):

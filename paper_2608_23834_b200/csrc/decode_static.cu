@@ -63,7 +63,7 @@ extern "C" int32_t mkv_decode_attention_static(mkv_pool* pool, const void* q, co
     uint32_t* tickets = reinterpret_cast<uint32_t*>(static_cast<unsigned char*>(scratch) + kPartialBytes);
     const int32_t rc = mkv::launch_decode_tensor_at(pool, q, bt, tags, lens, B, max_pages, scale, out, lse,
                                                     static_cast<float*>(scratch), tickets, kStaticMaxBlocks,
-                                                    (cudaStream_t)stream);
+                                                    nullptr, (cudaStream_t)stream);
     if (rc == MKV_E_INVALID)
         mkv::set_last_error("mkv_decode_attention_static: this GPU launches more blocks than MKV_STATIC_MAX_BLOCKS allows");
     return rc;

@@ -61,6 +61,7 @@ struct DecodeParams {
     float* partials;       // [2 * grid][8*D + 16]
     uint32_t* tickets;     // [max_blocks] arrival counters of split rows, indexed by the row's first block; zero between calls
     int max_blocks;        // the partial area holds 2 * max_blocks slots
+    float* mass;           // scored variant: [B][hq][max_pages], log2-domain page sums from the scan (else unused)
     uint32_t* status;
 };
 
@@ -349,8 +350,8 @@ struct Geo {
     static constexpr int OFF_QT = RING;
     static constexpr int OFF_QF = OFF_QT + QROT;
     static constexpr int OFF_BAR = OFF_QF + QPLAIN;
-    static constexpr int OFF_LIST = OFF_BAR + NW * NSTAGE * 8;   // [warp][2 formats][ROUND] page ids
-    static constexpr int OFF_CUM = OFF_LIST + NW * 2 * ROUND * 4;
+    static constexpr int OFF_LIST = OFF_BAR + NW * NSTAGE * 8;   // [warp][2 formats][ROUND] page ids, then [warp][2][ROUND] logical pages
+    static constexpr int OFF_CUM = OFF_LIST + NW * 4 * ROUND * 4;
     static constexpr int OFF_STRIDE = OFF_CUM + (kMaxBatch + 1) * 4;
     static constexpr int OFF_M = OFF_STRIDE + kMaxBatch * 4;
     static constexpr int OFF_L = OFF_M + NW * 8 * 4;
@@ -445,6 +446,21 @@ __device__ __forceinline__ void softmax_page(WarpAcc<NB>& acc, const float (&s)[
     pf.ps1 = ps[1];
     acc.l[0] += ps[0];
     acc.l[1] += ps[1];
+}
+
+// Scored variant (Section 3.1): log2 of the page's exponential sum, referred to an absolute origin
+// (row sum relative to the running maximum, plus that maximum), for the two heads this lane owns.
+// mass_pg points at (request, first head of the group, this page); heads are mass_stride apart.
+// The finishing kernel turns it into the globally normalised mass with the row's log-sum-exp.
+template <int NB>
+__device__ __forceinline__ void store_page_mass(const WarpAcc<NB>& acc, const PFrag& pf, float* mass_pg, int mass_stride,
+                                                int GQ, int lane)
+{
+    if (lane < 4) {                  // g == 0: one lane per head pair
+        const int h0 = 2 * lane;
+        if (h0 < GQ) mass_pg[(size_t)h0 * mass_stride] = __log2f(pf.ps0) + acc.m[0];
+        if (h0 + 1 < GQ) mass_pg[(size_t)(h0 + 1) * mass_stride] = __log2f(pf.ps1) + acc.m[1];
+    }
 }
 
 // All packed words of one lane for one code section.
@@ -563,9 +579,10 @@ __device__ __forceinline__ void tq3_step(WarpAcc<D / 16>& acc, uint32_t rec_v, c
 }
 
 // One Recent/Anchor page: keys [16 tokens][d] e4m3 at kaddr, values [d channels][16 tokens] at vaddr.
-template <int D>
+template <int D, bool SCORED>
 __device__ __forceinline__ void fp8_page(WarpAcc<D / 16>& acc, uint32_t kaddr, uint32_t vaddr, uint32_t qf_lane,
-                                         float score_scale, float v_scale, int valid, int lane)
+                                         float score_scale, float v_scale, int valid, int lane, float* mass_pg,
+                                         int mass_stride, int GQ)
 {
     constexpr int NB = D / 16;
     const int g = lane >> 2, tq = lane & 3;
@@ -599,6 +616,7 @@ __device__ __forceinline__ void fp8_page(WarpAcc<D / 16>& acc, uint32_t kaddr, u
     }
     PFrag pf;
     softmax_page<NB>(acc, s, pf);
+    if constexpr (SCORED) store_page_mass<NB>(acc, pf, mass_pg, mass_stride, GQ, lane);
     const bool scale_v = v_scale != 1.0f;
 #pragma unroll
     for (int cb = 0; cb < NB; ++cb) {
@@ -713,7 +731,7 @@ __device__ __forceinline__ void merge_row(const DecodeParams& P, int first_slot,
         P.lse[(size_t)b * hq + h * GQ + tid] = ml_s[8 + tid] > 0.f ? (ml_s[tid] + log2f(ml_s[8 + tid])) * kLn2 : -CUDART_INF_F;
 }
 
-template <int D, int NW, int NSTAGE, int MINB>
+template <int D, int NW, int NSTAGE, int MINB, bool SCORED>
 __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const DecodeParams P)
 {
 #ifdef MKV_TIMELINE
@@ -801,6 +819,8 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
     const uint32_t qt_lane = sbase + G::OFF_QT + lane * 16, qf_lane = sbase + G::OFF_QF + lane * 8;
     int* list3 = reinterpret_cast<int*>(smem + G::OFF_LIST) + warp * 2 * G::ROUND;   // Stale page ids of the round
     int* list8 = list3 + G::ROUND;                                                   // FP8 page ids | valid << 27
+    int* lpg3 = reinterpret_cast<int*>(smem + G::OFF_LIST) + (NW + warp) * 2 * G::ROUND;   // their logical pages (scored variant)
+    int* lpg8 = lpg3 + G::ROUND;
     const float sc2 = P.scale * kLog2e;      // scores are kept in log2 units
     // bounded wait for ring slot s, then flip its expected phase
     auto wait_slot = [&](uint32_t s) {
@@ -847,6 +867,7 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
 #pragma unroll
         for (int r = 0; r < EPL; ++r)
             qx[r] = (warp < GQ) ? __bfloat162float(P.q[((size_t)b * hq + h * GQ + warp) * D + lane * EPL + r]) : 0.f;
+        float* mass_row = SCORED ? P.mass + ((size_t)b * hq + (size_t)h * GQ) * P.max_pages : nullptr;
         const uint8_t* tq3_base = P.tq3 + (size_t)h * G::TQ3_REC;
         const uint8_t* fp8_base = P.fp8 + (size_t)h * (2 * G::FP8_HALF);
 
@@ -858,9 +879,9 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
 #pragma unroll 1
             for (int c = 0; c < G::ROUND / 32; ++c) {
                 const int i = round * G::ROUND + c * 32 + lane;
-                int kind = 0, id = 0, valid = kPage;
+                int kind = 0, id = 0, valid = kPage, pg = 0;
                 if (i < n_my) {
-                    const int pg = (int)(((unsigned)(pg0 + warp_first + i) * (unsigned)stride) % (unsigned)n_pages);   // < 2^32: max_pages <= 65535
+                    pg = (int)(((unsigned)(pg0 + warp_first + i) * (unsigned)stride) % (unsigned)n_pages);   // < 2^32: max_pages <= 65535
                     id = bt_row[pg];
                     const int tag = tag_row[pg];
                     valid = min(kPage, len - pg * kPage);
@@ -874,6 +895,10 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                 const uint32_t lt = (1u << lane) - 1u;
                 if (kind == 1) list3[n3 + __popc(m3 & lt)] = id;
                 if (kind == 2) list8[n8 + __popc(m8 & lt)] = id | ((valid & 15) << 27);
+                if constexpr (SCORED) {
+                    if (kind == 1) lpg3[n3 + __popc(m3 & lt)] = pg;
+                    if (kind == 2) lpg8[n8 + __popc(m8 & lt)] = pg;
+                }
                 n3 += __popc(m3);
                 n8 += __popc(m8);
             }
@@ -977,6 +1002,7 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                     wait_slot(nxt);
                     if (failed) break;
                     softmax_page<NB>(acc, s_cur, pf);
+                    if constexpr (SCORED) store_page_mass<NB>(acc, pf, mass_row + lpg3[i], P.max_pages, GQ, lane);
                     tq3_step<D, true, true>(acc, ring + cur * G::SLOT, pf, ring + nxt * G::SLOT, qt_lane, sc2, lane, s_next);
 #pragma unroll
                     for (int e = 0; e < 4; ++e) s_cur[e] = s_next[e];
@@ -985,6 +1011,7 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                 }
                 if (!failed) {
                     softmax_page<NB>(acc, s_cur, pf);
+                    if constexpr (SCORED) store_page_mass<NB>(acc, pf, mass_row + lpg3[n3 - 1], P.max_pages, GQ, lane);
                     tq3_step<D, true, false>(acc, ring + ((uint32_t)(n3 - 1) % NSTAGE) * G::SLOT, pf, 0, qt_lane, sc2, lane, s_next);
                 }
                 __syncwarp();
@@ -999,8 +1026,8 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                     if (failed) break;
                     const int e = list8[i];
                     const int valid = (e >> 27) & 15;
-                    fp8_page<D>(acc, ring + s * G::SLOT, ring + (s + 1) * G::SLOT, qf_lane, sc2 * P.k_scale, P.v_scale,
-                                valid ? valid : kPage, lane);
+                    fp8_page<D, SCORED>(acc, ring + s * G::SLOT, ring + (s + 1) * G::SLOT, qf_lane, sc2 * P.k_scale, P.v_scale,
+                                        valid ? valid : kPage, lane, SCORED ? mass_row + lpg8[i] : nullptr, P.max_pages, GQ);
                     __syncwarp();
                     if (i + NSTAGE / 2 < n8) issue_fp8(i + NSTAGE / 2);
                 }
@@ -1111,11 +1138,11 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
     }
 }
 
-template <int D, int NW, int NSTAGE, int MINB>
+template <int D, int NW, int NSTAGE, int MINB, bool SCORED = false>
 static int32_t run_tensor(mkv_pool* p, DecodeParams& prm, cudaStream_t s)
 {
     using G = Geo<D, NW, NSTAGE>;
-    auto kern = decode_tensor_kernel<D, NW, NSTAGE, MINB>;
+    auto kern = decode_tensor_kernel<D, NW, NSTAGE, MINB, SCORED>;
     static int grid_cache[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     int dev = p->device & 7;
     if (grid_cache[dev] == 0) {
@@ -1157,14 +1184,79 @@ int32_t launch_decode_tensor(mkv_pool* p, const void* q, const int32_t* bt, cons
     // header: 256 reserved bytes, then kMaxCtas ticket words (cleared by mkv_workspace_init, left clear by every call)
     uint32_t* tickets = reinterpret_cast<uint32_t*>(static_cast<uint8_t*>(ws) + 256);
     float* partials = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + decode_ws_header_bytes(B, p->hkv));
-    return launch_decode_tensor_at(p, q, bt, tags, lens, B, max_pages, scale, out, lse, partials, tickets, kMaxCtas, s);
+    return launch_decode_tensor_at(p, q, bt, tags, lens, B, max_pages, scale, out, lse, partials, tickets, kMaxCtas,
+                                   nullptr, s);
 }
 
 int decode_tensor_partial_floats(int d) { return 8 * d + 16; }
 
+// Second step of the scored variant: mass[b][hq][p] holds log2 of page p's exponential sum on an
+// absolute origin; with the row's log-sum-exp it becomes q_p = 2^(that - lse2), and q~_p = q_p / sum q_p
+// (Eq. score-global-weight and the normalisation over page-addressable mass that follows it).
+// One block per (query head, request); entries beyond the request's pages are set to zero.
+__global__ void __launch_bounds__(256) page_mass_finish_kernel(float* mass, const float* lse, const int32_t* lens,
+                                                              int hq, int max_pages)
+{
+    __shared__ float red[8];
+    const int b = blockIdx.y, h = blockIdx.x, tid = threadIdx.x;
+    const int len = lens[b], n_pages = len > 0 ? (len + kPage - 1) / kPage : 0;
+    float* row = mass + ((size_t)b * hq + h) * max_pages;
+    const float lse2 = n_pages > 0 ? lse[(size_t)b * hq + h] * kLog2e : 0.f;
+    float sum = 0.f;
+    for (int p = tid; p < n_pages; p += 256) {
+        const float qv = fast_exp2(row[p] - lse2);
+        row[p] = qv;
+        sum += qv;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    if ((tid & 31) == 0) red[tid >> 5] = sum;
+    __syncthreads();
+    float total = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) total += red[w];
+    const float inv = total > 0.f ? 1.f / total : 0.f;
+    for (int p = tid; p < max_pages; p += 256) row[p] = p < n_pages ? row[p] * inv : 0.f;
+}
+
+// Eq. (attention-score): r_p = mean over the sampled heads of q~_{h,p}; a_p <- beta a_p + (1 - beta) r_p.
+__global__ void __launch_bounds__(256) page_score_kernel(const float* mass, const int32_t* lens, int hq, int max_pages,
+                                                         unsigned long long head_mask, float beta, float inv_heads,
+                                                         float* score)
+{
+    const int b = blockIdx.y, p = blockIdx.x * 256 + threadIdx.x;
+    const int len = lens[b], n_pages = len > 0 ? (len + kPage - 1) / kPage : 0;
+    if (p >= n_pages) return;
+    float r = 0.f;
+    for (int h = 0; h < hq; ++h)
+        if ((head_mask >> h) & 1ull) r += mass[((size_t)b * hq + h) * max_pages + p];
+    float* a = score + (size_t)b * max_pages + p;
+    *a = beta * *a + (1.f - beta) * (r * inv_heads);
+}
+
+int32_t launch_page_mass_finish(float* mass, const float* lse, const int32_t* lens, int B, int hq, int max_pages,
+                                cudaStream_t s)
+{
+    page_mass_finish_kernel<<<dim3(hq, B), 256, 0, s>>>(mass, lse, lens, hq, max_pages);
+    MKV_CUDA(cudaGetLastError());
+    return MKV_OK;
+}
+
+int32_t launch_page_score(const float* mass, const int32_t* lens, int B, int hq, int max_pages, uint64_t head_mask,
+                          float beta, float* score, cudaStream_t s)
+{
+    int n = 0;
+    for (int h = 0; h < hq; ++h) n += (int)((head_mask >> h) & 1ull);
+    if (n == 0) return MKV_E_INVALID;
+    page_score_kernel<<<dim3((max_pages + 255) / 256, B), 256, 0, s>>>(mass, lens, hq, max_pages, head_mask, beta,
+                                                                         1.f / (float)n, score);
+    MKV_CUDA(cudaGetLastError());
+    return MKV_OK;
+}
+
 int32_t launch_decode_tensor_at(mkv_pool* p, const void* q, const int32_t* bt, const uint8_t* tags,
                                 const int32_t* lens, int B, int max_pages, float scale, float* out, float* lse,
-                                float* partials, uint32_t* tickets, int max_blocks, cudaStream_t s)
+                                float* partials, uint32_t* tickets, int max_blocks, float* mass, cudaStream_t s)
 {
     if (B > kMaxBatch) return MKV_E_INVALID;
     if (max_pages > 65535) {            // the strided page order multiplies two page indices in 32 bits
@@ -1184,7 +1276,13 @@ int32_t launch_decode_tensor_at(mkv_pool* p, const void* q, const int32_t* bt, c
     prm.partials = partials;
     prm.tickets = tickets;
     prm.max_blocks = max_blocks;
+    prm.mass = mass;
     prm.status = p->status_dev;
+    if (mass) {                          // scored variant: the default launch shapes only
+        const int32_t rc = p->d == 128 ? run_tensor<128, 16, 4, 1, true>(p, prm, s) : run_tensor<256, 8, 4, 1, true>(p, prm, s);
+        if (rc != MKV_OK) return rc;
+        return launch_page_mass_finish(mass, lse, lens, B, p->hkv * p->group, max_pages, s);
+    }
     // Launch shapes (warps per block, ring slots per warp, blocks per SM); MKV_DECODE_SHAPE selects the
     // alternatives for profiling.
     const int shape = tensor_shape();
@@ -1192,14 +1290,12 @@ int32_t launch_decode_tensor_at(mkv_pool* p, const void* q, const int32_t* bt, c
         switch (shape) {
         case 1: return run_tensor<128, 8, 4, 1>(p, prm, s);
         case 2: return run_tensor<128, 12, 4, 1>(p, prm, s);
-        case 3: return run_tensor<128, 8, 4, 2>(p, prm, s);
         default: return run_tensor<128, 16, 4, 1>(p, prm, s);
         }
     }
     switch (shape) {
     case 1: return run_tensor<256, 8, 6, 1>(p, prm, s);
-    case 2: return run_tensor<256, 12, 4, 1>(p, prm, s);
-    case 3: return run_tensor<256, 10, 4, 1>(p, prm, s);
+    case 2: return run_tensor<256, 10, 4, 1>(p, prm, s);
     default: return run_tensor<256, 8, 4, 1>(p, prm, s);
     }
 }

@@ -96,7 +96,9 @@ int32_t launch_decode_tensor(mkv_pool* p, const void* q, const int32_t* bt, cons
                              void* ws, size_t ws_bytes, cudaStream_t s);
 int32_t launch_decode_tensor_at(mkv_pool* p, const void* q, const int32_t* bt, const uint8_t* tags,
                                 const int32_t* lens, int B, int max_pages, float scale, float* out, float* lse,
-                                float* partials, uint32_t* tickets, int max_blocks, cudaStream_t s);
+                                float* partials, uint32_t* tickets, int max_blocks, float* mass, cudaStream_t s);
+int32_t launch_page_score(const float* mass, const int32_t* lens, int B, int hq, int max_pages, uint64_t head_mask,
+                          float beta, float* score, cudaStream_t s);
 constexpr int kMaxCtas = 512;        // upper bound of the decode scan's persistent grid (sizes workspace and tickets)
 int decode_tensor_partial_floats(int d);
 void set_last_error(const char* msg);

@@ -320,6 +320,35 @@ int32_t mkv_decode_attention(mkv_pool* pool, const void* q, const int32_t* bt, c
                                 (cudaStream_t)stream);
 }
 
+int32_t mkv_decode_attention_scored(mkv_pool* pool, const void* q, const int32_t* bt, const uint8_t* tags,
+                                    const int32_t* lens, int32_t B, int32_t max_pages, float scale, float* out,
+                                    float* lse, float* page_mass, void* ws, size_t ws_bytes, void* stream)
+{
+    if (!pool || !pool->fp8 || B < 0 || max_pages < 0) return MKV_E_INVALID;
+    if (B == 0) return MKV_OK;
+    if (!q || !bt || !tags || !lens || !out || !ws || !lse || !page_mass) return MKV_E_INVALID;
+    if (!aligned(q, 16) || !aligned(out, 16) || !aligned(ws, 256) || !aligned(bt, 4) || !aligned(lens, 4) ||
+        !aligned(page_mass, 4) || !aligned(lse, 4))
+        return MKV_E_INVALID;
+    size_t need;
+    if (mkv_decode_workspace_bytes(&pool->cfg, B, &need) != MKV_OK || ws_bytes < need) return MKV_E_INVALID;
+    if (!(scale == scale)) return MKV_E_INVALID;
+    uint32_t* tickets = reinterpret_cast<uint32_t*>(static_cast<uint8_t*>(ws) + 256);
+    float* partials = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + decode_ws_header_bytes(B, pool->hkv));
+    return launch_decode_tensor_at(pool, q, bt, tags, lens, B, max_pages, scale, out, lse, partials, tickets, kMaxCtas,
+                                   page_mass, (cudaStream_t)stream);
+}
+
+int32_t mkv_page_score_update(const float* page_mass, const int32_t* lens, int32_t B, int32_t n_q_heads,
+                              int32_t max_pages, uint64_t head_mask, float beta, float* score, void* stream)
+{
+    if (B < 0 || max_pages < 0 || n_q_heads < 1 || n_q_heads > 64) return MKV_E_INVALID;
+    if (B == 0 || max_pages == 0) return MKV_OK;
+    if (!page_mass || !lens || !score || !(beta >= 0.f && beta <= 1.f)) return MKV_E_INVALID;
+    if (n_q_heads < 64) head_mask &= (1ull << n_q_heads) - 1ull;
+    return launch_page_score(page_mass, lens, B, n_q_heads, max_pages, head_mask, beta, score, (cudaStream_t)stream);
+}
+
 // ---- sequence rows (Algorithm 1, host bookkeeping only) ----------------------------------------
 
 int32_t mkv_seq_create(mkv_pool* pool, mkv_seq** out)
