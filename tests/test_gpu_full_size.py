@@ -21,6 +21,14 @@ def test_config2_one_full_layer_every_output():
     out, lse = case.run(M.DECODE_TENSOR)
     ref, ref_lse = case.reference()
     check_case(case, out, lse, ref, ref_lse)
+    # the scored call on the same layer: same output bit for bit, page mass against the oracle
+    out_s, _, mass = case.pool.decode_attention_scored(case.q, case.bt, case.tags, case.lens, spec.scale)
+    torch.cuda.synchronize()
+    assert np.array_equal(out_s.cpu().numpy(), out)
+    ref_mass = oracle.page_mass(case.L.fp8_arena, case.L.tq3_arena, spec.head_dim, spec.n_kv_heads, spec.group, case.L.sigma,
+                                case.L.q_bits, case.tab.block_table, case.tab.tier_tag, case.tab.seq_lens, spec.scale)
+    got = mass.cpu().numpy().astype(np.float64)
+    assert (np.abs(got - ref_mass) <= 1e-6 + 1e-4 * ref_mass).all(), np.abs(got - ref_mass).max()
 
 
 def test_config1_as_specified():
