@@ -503,7 +503,7 @@ def workload_spec(args):
     if args.ctx > 0 and args.config != 4:
         over["seq_lens"] = (args.ctx,) * W.config(args.config).batch
     if args.config == 4:
-        return W.config(4, batch=8, ctx=32768, stale_fraction=0.5, **over)
+        return W.config(4, batch=args.batch or 8, ctx=args.ctx or 32768, stale_fraction=args.stale, **over)
     return W.config(args.config, **over)
 
 
@@ -592,6 +592,8 @@ def main():
     ap.add_argument("--variant", default="tensor", choices=["tensor", "scalar"],
                     help="decode kernel: the tensor-core product kernel, or the CUDA-core comparison kernel")
     ap.add_argument("--ctx", type=int, default=0, help="override the context length of every request (profiling)")
+    ap.add_argument("--batch", type=int, default=0, help="config 4 only: requests of the lifecycle cell (default 8)")
+    ap.add_argument("--stale", type=float, default=0.5, help="config 4 only: Stale fraction of the lifecycle cell")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":

@@ -231,7 +231,7 @@ __device__ __forceinline__ void affine_accumulate(float (&acc)[4], const float (
 // ------------------------------------------------------------------------------------------------
 // Work = (request, KV head, page) triples in row-major order; cum[b] = index of the first triple of
 // request b.  Two ways to cut it into one contiguous range per block:
-//   row-aligned (few rows: B * hkv <= grid / 4): every row gets a whole number of blocks in proportion
+//   row-aligned (few rows: B * hkv <= grid / 12): every row gets a whole number of blocks in proportion
 //     to its pages (cumulative rounding), so that no block straddles two rows and pays the per-row set-up
 //     and reduction twice;
 //   linear (many rows): grid equal ranges that may cross row boundaries.
@@ -251,7 +251,8 @@ __device__ __forceinline__ void build_partition(Partition* pt, const int* cum, c
     const long long W = cum[B];
     const int rows = B * hkv;
     int blocks = (int)(W < (long long)grid ? W : (long long)grid);
-    int aligned = (rows <= grid / 4 && rows <= kMaxAlignedRows && W >= grid) ? 1 : 0;
+    // with k blocks per row the rows that get one block fewer run 1/k longer: worth it from about twelve
+    int aligned = (rows * 12 <= grid && rows <= kMaxAlignedRows && W >= grid) ? 1 : 0;
     if (aligned) {
         // block boundaries at the rounded cumulative share of the rows: base[r] = round(grid * first_page(r) / W);
         // every row must end up with at least one block, otherwise the linear cut is used
@@ -367,6 +368,7 @@ struct Geo {
 #ifdef MKV_TIMELINE
 // profiling build only: thread 0 of every block accumulates the time spent in each phase
 __device__ unsigned long long g_timeline[kMaxCtas * 16];
+__device__ unsigned long long g_warp_end[kMaxCtas * 32];   // per warp: time its page loops ended, pages it had (TQ3 << 32 | FP8)
 __device__ __forceinline__ unsigned long long tl_now()
 {
     unsigned long long t;
@@ -644,13 +646,13 @@ __device__ __forceinline__ void fp8_page(WarpAcc<D / 16>& acc, uint32_t kaddr, u
 // drew the row's last ticket; `buf` is idle shared memory (n_parts * 16 + 16 floats).  Warp hd < 8
 // reduces the maxima and row sums of head hd (one trip to L2: both are loaded together and kept in
 // shared memory); a thread then owns float4 groups (one channel, four heads) of the [channel][8 heads]
-// tile and has the loads of sixteen parts in flight at a time.
+// tile and has 40 loads in flight, issued before the weights are worked out.
 template <int D, int NT>
 __device__ __forceinline__ void merge_row(const DecodeParams& P, int first_slot, int even_base, int n_parts,
                                           float* buf, int b, int h)
 {
     constexpr uint32_t FULL = 0xffffffffu;
-    constexpr int STRIDE = 8 * D + 16, GPT = (2 * D + NT - 1) / NT, KP = 16;
+    constexpr int STRIDE = 8 * D + 16, GPT = (2 * D + NT - 1) / NT, KP = 40 / GPT;   // 40 float4 loads in flight per thread
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int GQ = P.group, hq = P.hkv * GQ;
     float* w_s = buf;                        // [n_parts][8] maxima, then weights e^{m_j - m}
@@ -660,6 +662,34 @@ __device__ __forceinline__ void merge_row(const DecodeParams& P, int first_slot,
         return P.partials + (size_t)(j == 0 ? first_slot : even_base + 2 * j) * STRIDE;
     };
     __syncthreads();
+    float4 acc[GPT], v[KP][GPT];
+#pragma unroll
+    for (int k = 0; k < GPT; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int head0 = (tid & 1) * 4;         // NT is even: every group of this thread covers the same four heads
+    auto load_round = [&](int j0) {
+#pragma unroll
+        for (int p = 0; p < KP; ++p) {
+            const float* ps = slot_of(min(j0 + p, n_parts - 1));
+#pragma unroll
+            for (int k = 0; k < GPT; ++k)
+                v[p][k] = __ldcg(reinterpret_cast<const float4*>(ps) + min(tid + k * NT, 2 * D - 1));
+        }
+    };
+    auto use_round = [&](int j0) {
+#pragma unroll
+        for (int p = 0; p < KP; ++p)
+            if (j0 + p < n_parts) {
+                const float4 w = *reinterpret_cast<const float4*>(w_s + (j0 + p) * 8 + head0);
+#pragma unroll
+                for (int k = 0; k < GPT; ++k) {
+                    acc[k].x = fmaf(w.x, v[p][k].x, acc[k].x);
+                    acc[k].y = fmaf(w.y, v[p][k].y, acc[k].y);
+                    acc[k].z = fmaf(w.z, v[p][k].z, acc[k].z);
+                    acc[k].w = fmaf(w.w, v[p][k].w, acc[k].w);
+                }
+            }
+    };
+    load_round(0);                           // in flight while the weights are worked out
     if (warp < 8) {
         const int hd = warp;
         float M = -CUDART_INF_F;
@@ -686,32 +716,11 @@ __device__ __forceinline__ void merge_row(const DecodeParams& P, int first_slot,
             ml_s[8 + hd] = L;
         }
     }
-    float4 acc[GPT];
-#pragma unroll
-    for (int k = 0; k < GPT; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-    const int head0 = (tid & 1) * 4;         // NT is even: every group of this thread covers the same four heads
-    for (int j0 = 0; j0 < n_parts; j0 += KP) {
-        float4 v[KP][GPT];
-#pragma unroll
-        for (int p = 0; p < KP; ++p) {
-            const float* ps = slot_of(min(j0 + p, n_parts - 1));
-#pragma unroll
-            for (int k = 0; k < GPT; ++k)
-                v[p][k] = __ldcg(reinterpret_cast<const float4*>(ps) + min(tid + k * NT, 2 * D - 1));
-        }
-        if (j0 == 0) __syncthreads();        // weights are ready (the loads above did not need them)
-#pragma unroll
-        for (int p = 0; p < KP; ++p)
-            if (j0 + p < n_parts) {
-                const float4 w = *reinterpret_cast<const float4*>(w_s + (j0 + p) * 8 + head0);
-#pragma unroll
-                for (int k = 0; k < GPT; ++k) {
-                    acc[k].x = fmaf(w.x, v[p][k].x, acc[k].x);
-                    acc[k].y = fmaf(w.y, v[p][k].y, acc[k].y);
-                    acc[k].z = fmaf(w.z, v[p][k].z, acc[k].z);
-                    acc[k].w = fmaf(w.w, v[p][k].w, acc[k].w);
-                }
-            }
+    __syncthreads();
+    use_round(0);
+    for (int j0 = KP; j0 < n_parts; j0 += KP) {
+        load_round(j0);
+        use_round(j0);
     }
 #pragma unroll
     for (int k = 0; k < GPT; ++k) {
@@ -924,6 +933,9 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
             }
         };
 
+#ifdef MKV_TIMELINE
+        int tl_n3 = 0, tl_n8 = 0;
+#endif
         WarpAcc<NB> acc;
 #pragma unroll
         for (int i = 0; i < NB; ++i) acc.o[i][0] = acc.o[i][1] = acc.o[i][2] = acc.o[i][3] = 0.f;
@@ -991,6 +1003,9 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                 build_lists(round);
                 for (int i = 0; i < min(n3, NSTAGE); ++i) issue_tq3(i);
             }
+#ifdef MKV_TIMELINE
+            tl_n3 += n3; tl_n8 += n8;
+#endif
             // ---- Stale pages: scores of page i+1 are computed together with the output update of page i
             if (n3 > 0) {
                 float s_cur[4], s_next[4];
@@ -1038,6 +1053,13 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
         float (&m_run)[2] = acc.m;
 
         // ---- combine the warps of the block (ring memory is idle now) ---------------------------
+#ifdef MKV_TIMELINE
+        if (lane == 0 && warp < 16) {
+            g_warp_end[blockIdx.x * 32 + warp] = tl_now();
+            g_warp_end[blockIdx.x * 32 + 16 + warp] = ((unsigned long long)tl_n3 << 32) | (unsigned)tl_n8;
+            if (warp == 0) { unsigned sm__; asm volatile("mov.u32 %0, %%smid;" : "=r"(sm__)); g_warp_end[blockIdx.x * 32 + 15] = sm__; }
+        }
+#endif
         MKV_STAMP(3);
         __syncthreads();
         MKV_STAMP(4);
@@ -1174,6 +1196,10 @@ static int tensor_shape()
 extern "C" int mkv_debug_timeline(unsigned long long* host, int n)
 {
     return (int)cudaMemcpyFromSymbol(host, g_timeline, sizeof(unsigned long long) * n);
+}
+extern "C" int mkv_debug_warp_end(unsigned long long* host, int n)
+{
+    return (int)cudaMemcpyFromSymbol(host, g_warp_end, sizeof(unsigned long long) * n);
 }
 #endif
 
