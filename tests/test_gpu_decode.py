@@ -196,3 +196,42 @@ def test_append_and_decode_replay_from_a_cuda_graph():
                 oracle.decode_attention(case.L.fp8_arena, case.L.tq3_arena, spec.head_dim, spec.n_kv_heads, spec.group,
                                         case.L.sigma, case.L.q_bits, case.tab.block_table, case.tab.tier_tag,
                                         lens2.cpu().numpy(), spec.scale)[0], "graph replay")
+
+
+def test_decode_maximum_batch_of_short_requests():
+    """1,024 requests (the largest batch a call accepts) of 0 to 70 tokens: every block walks many
+    (request, KV head) rows, most of them whole, some split at a block boundary."""
+    rng = np.random.default_rng(17)
+    lens = [int(x) for x in rng.integers(0, 71, size=1024)]
+    lens[0], lens[1], lens[-1] = 0, 70, 1
+    spec = W.config(0, seq_lens=lens, head_dim=128, n_kv_heads=2, group=3, anchor_prefix=16, recent_tokens=20, n_outlier=2)
+    case = Case(spec)
+    out, lse = case.run(M.DECODE_TENSOR)
+    ref, ref_lse = case.reference()
+    check_case(case, out, lse, ref, ref_lse)
+    # one request more than the maximum is refused before anything is launched
+    q2 = torch.zeros((1025, spec.n_q_heads, 128), dtype=torch.bfloat16, device="cuda:0")
+    bt2 = torch.zeros((1025, case.bt.shape[1]), dtype=torch.int32, device="cuda:0")
+    tg2 = torch.zeros((1025, case.bt.shape[1]), dtype=torch.uint8, device="cuda:0")
+    ln2 = torch.zeros(1025, dtype=torch.int32, device="cuda:0")
+    big = M.Pool(128, 2, 6, 4, 4, case.L.sigma, max_batch=1025)
+    with pytest.raises(M.MkvError) as e:
+        big.decode_attention(q2, bt2, tg2, ln2, spec.scale)
+    assert e.value.code == M.E_INVALID
+
+
+def test_decode_one_long_row_and_the_page_limit():
+    """One request of 12,000 pages on a single KV head: 148 blocks share one row (the longest split the
+    tests see), with Anchor spans in the middle.  A table wider than 65,535 pages is refused."""
+    spec = W.config(0, seq_lens=(16 * 12000 - 5,), head_dim=128, n_kv_heads=1, group=2, anchor_prefix=64, anchor_spans=3,
+                    anchor_span_tokens=160, recent_tokens=1000, n_outlier=2)
+    case = Case(spec)
+    out, lse = case.run(M.DECODE_TENSOR)
+    ref, ref_lse = case.reference()
+    check_case(case, out, lse, ref, ref_lse)
+    wide_bt = torch.zeros((1, 65536), dtype=torch.int32, device="cuda:0")
+    wide_tg = torch.zeros((1, 65536), dtype=torch.uint8, device="cuda:0")
+    with pytest.raises(M.MkvError) as e:
+        case.pool.decode_attention(case.q, wide_bt, wide_tg, case.lens, spec.scale)
+    assert e.value.code == M.E_INVALID
+    assert b"65535" in M.lib().mkv_last_cuda_error()
