@@ -652,7 +652,7 @@ __device__ __forceinline__ void merge_row(const DecodeParams& P, int first_slot,
                                           float* buf, int b, int h)
 {
     constexpr uint32_t FULL = 0xffffffffu;
-    constexpr int STRIDE = 8 * D + 16, GPT = (2 * D + NT - 1) / NT, KP = 40 / GPT;   // 40 float4 loads in flight per thread
+    constexpr int STRIDE = 8 * D + 16, GPT = (2 * D + NT - 1) / NT, KP = 40 / GPT;   // float4 loads in flight per thread: 40, or 16 where registers are scarce
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int GQ = P.group, hq = P.hkv * GQ;
     float* w_s = buf;                        // [n_parts][8] maxima, then weights e^{m_j - m}
@@ -1305,7 +1305,7 @@ int32_t launch_decode_tensor_at(mkv_pool* p, const void* q, const int32_t* bt, c
     prm.mass = mass;
     prm.status = p->status_dev;
     if (mass) {                          // scored variant: the default launch shapes only
-        const int32_t rc = p->d == 128 ? run_tensor<128, 16, 4, 1, true>(p, prm, s) : run_tensor<256, 8, 4, 1, true>(p, prm, s);
+        const int32_t rc = p->d == 128 ? run_tensor<128, 12, 4, 1, true>(p, prm, s) : run_tensor<256, 8, 4, 1, true>(p, prm, s);
         if (rc != MKV_OK) return rc;
         return launch_page_mass_finish(mass, lse, lens, B, p->hkv * p->group, max_pages, s);
     }
@@ -1314,9 +1314,9 @@ int32_t launch_decode_tensor_at(mkv_pool* p, const void* q, const int32_t* bt, c
     const int shape = tensor_shape();
     if (p->d == 128) {
         switch (shape) {
-        case 1: return run_tensor<128, 8, 4, 1>(p, prm, s);
-        case 2: return run_tensor<128, 12, 4, 1>(p, prm, s);
-        default: return run_tensor<128, 16, 4, 1>(p, prm, s);
+        case 1: return run_tensor<128, 16, 4, 1>(p, prm, s);
+        case 2: return run_tensor<128, 8, 4, 1>(p, prm, s);
+        default: return run_tensor<128, 12, 4, 1>(p, prm, s);     // 168 registers: 7 % faster than 16 warps at 128; 10, 11, 13, 14 warps are slower
         }
     }
     switch (shape) {
