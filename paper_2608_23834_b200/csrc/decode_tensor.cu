@@ -580,7 +580,20 @@ __device__ __forceinline__ void tq3_step(WarpAcc<D / 16>& acc, uint32_t rec_v, c
     }
 }
 
+// Four 8x8 matrices of 16-bit elements from shared memory in the MMA fragment layout: lane l supplies the
+// address of row l % 8 of matrix l / 8; every lane receives, per matrix, the 32 bits at (row lane / 4,
+// 16-bit columns 2 (lane % 4), 2 (lane % 4) + 1).
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+
 // One Recent/Anchor page: keys [16 tokens][d] e4m3 at kaddr, values [d channels][16 tokens] at vaddr.
+// MMA row r of the score tile holds token pi(r) = 4 (r % 8 / 2) + r % 2 + 2 (r / 8), so that the value
+// fragments can be fetched with ldmatrix: a lane then holds the four consecutive tokens 4tq .. 4tq+3 of
+// its two channel rows, which is the order P^T has after the transposition of a score tile whose rows
+// are permuted this way.
 template <int D, bool SCORED>
 __device__ __forceinline__ void fp8_page(WarpAcc<D / 16>& acc, uint32_t kaddr, uint32_t vaddr, uint32_t qf_lane,
                                          float score_scale, float v_scale, int valid, int lane, float* mass_pg,
@@ -588,11 +601,12 @@ __device__ __forceinline__ void fp8_page(WarpAcc<D / 16>& acc, uint32_t kaddr, u
 {
     constexpr int NB = D / 16;
     const int g = lane >> 2, tq = lane & 3;
+    const int tok0 = 4 * (g >> 1) + (g & 1), tok1 = tok0 + 2;       // tokens of the lane's two score rows
     float S0[4] = {0.f, 0.f, 0.f, 0.f}, S1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int j = 0; j < D / 64; ++j) {
-        const uint4 r0 = lds128(kaddr + g * D + 64 * j + 16 * tq);
-        const uint4 r1 = lds128(kaddr + (g + 8) * D + 64 * j + 16 * tq);
+        const uint4 r0 = lds128(kaddr + tok0 * D + 64 * j + 16 * tq);
+        const uint4 r1 = lds128(kaddr + tok1 * D + 64 * j + 16 * tq);
         const uint32_t w0[4] = {r0.x, r0.y, r0.z, r0.w}, w1[4] = {r1.x, r1.y, r1.z, r1.w};
 #pragma unroll
         for (int w = 0; w < 4; ++w) {
@@ -609,34 +623,40 @@ __device__ __forceinline__ void fp8_page(WarpAcc<D / 16>& acc, uint32_t kaddr, u
     float s[4] = {(S0[0] + S1[0]) * score_scale, (S0[1] + S1[1]) * score_scale, (S0[2] + S1[2]) * score_scale,
                   (S0[3] + S1[3]) * score_scale};
     // bytes of tokens beyond the sequence end are cleared so that stale NaN patterns cannot leak
-    uint32_t keep_lo = 0xFFFFu, keep_hi = 0xFFFFu;   // byte masks for tokens (2tq,2tq+1), (2tq+8,2tq+9)
+    uint32_t keep = 0xFFFFFFFFu;                     // byte mask for the tokens 4tq .. 4tq+3 of a value word
     if (valid < kPage) {
-        if (g >= valid) s[0] = s[1] = -CUDART_INF_F;
-        if (g + 8 >= valid) s[2] = s[3] = -CUDART_INF_F;
-        keep_lo = (2 * tq < valid ? 0x00FFu : 0u) | (2 * tq + 1 < valid ? 0xFF00u : 0u);
-        keep_hi = (2 * tq + 8 < valid ? 0x00FFu : 0u) | (2 * tq + 9 < valid ? 0xFF00u : 0u);
+        if (tok0 >= valid) s[0] = s[1] = -CUDART_INF_F;
+        if (tok1 >= valid) s[2] = s[3] = -CUDART_INF_F;
+        keep = (4 * tq < valid ? 0x000000FFu : 0u) | (4 * tq + 1 < valid ? 0x0000FF00u : 0u) |
+               (4 * tq + 2 < valid ? 0x00FF0000u : 0u) | (4 * tq + 3 < valid ? 0xFF000000u : 0u);
     }
     PFrag pf;
     softmax_page<NB>(acc, s, pf);
     if constexpr (SCORED) store_page_mass<NB>(acc, pf, mass_pg, mass_stride, GQ, lane);
     const bool scale_v = v_scale != 1.0f;
 #pragma unroll
-    for (int cb = 0; cb < NB; ++cb) {
-        const uint32_t r0 = vaddr + (16 * cb + g) * 16 + 2 * tq, r1 = r0 + 8 * 16;
-        uint32_t a[4];
-        a[0] = e4m3x2_to_f16x2((uint16_t)(lds16(r0) & keep_lo));
-        a[1] = e4m3x2_to_f16x2((uint16_t)(lds16(r1) & keep_lo));
-        a[2] = e4m3x2_to_f16x2((uint16_t)(lds16(r0 + 8) & keep_hi));
-        a[3] = e4m3x2_to_f16x2((uint16_t)(lds16(r1 + 8) & keep_hi));
-        if (scale_v) {
-            float t[4];
-            mma16816_zero(t, a, pf.b0, pf.b1);
-            mma16816(t, a, pf.c0, pf.c1);
+    for (int cb = 0; cb < NB; cb += 2) {
+        // channels 16cb .. 16cb+31: rows of 16 bytes, lane l addresses row l
+        uint32_t v[4];
+        ldmatrix_x4(vaddr + cb * 256 + lane * 16, v[0], v[1], v[2], v[3]);
 #pragma unroll
-            for (int e = 0; e < 4; ++e) acc.o[cb][e] = fmaf(v_scale, t[e], acc.o[cb][e]);
-        } else {
-            mma16816(acc.o[cb], a, pf.b0, pf.b1);
-            mma16816(acc.o[cb], a, pf.c0, pf.c1);
+        for (int e = 0; e < 2; ++e) {
+            const uint32_t lo = v[2 * e] & keep, hi = v[2 * e + 1] & keep;      // channel rows g and g + 8 of block cb + e
+            uint32_t a[4];
+            a[0] = e4m3x2_to_f16x2((uint16_t)(lo & 0xFFFFu));
+            a[1] = e4m3x2_to_f16x2((uint16_t)(hi & 0xFFFFu));
+            a[2] = e4m3x2_to_f16x2((uint16_t)(lo >> 16));
+            a[3] = e4m3x2_to_f16x2((uint16_t)(hi >> 16));
+            if (scale_v) {
+                float t[4];
+                mma16816_zero(t, a, pf.b0, pf.b1);
+                mma16816(t, a, pf.c0, pf.c1);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc.o[cb + e][i] = fmaf(v_scale, t[i], acc.o[cb + e][i]);
+            } else {
+                mma16816(acc.o[cb + e], a, pf.b0, pf.b1);
+                mma16816(acc.o[cb + e], a, pf.c0, pf.c1);
+            }
         }
     }
 }
@@ -652,7 +672,7 @@ __device__ __forceinline__ void merge_row(const DecodeParams& P, int first_slot,
                                           float* buf, int b, int h)
 {
     constexpr uint32_t FULL = 0xffffffffu;
-    constexpr int STRIDE = 8 * D + 16, GPT = (2 * D + NT - 1) / NT, KP = 40 / GPT;   // float4 loads in flight per thread: 40, or 16 where registers are scarce
+    constexpr int STRIDE = 8 * D + 16, GPT = (2 * D + NT - 1) / NT, KP = 40 / GPT;   // 40 float4 loads in flight per thread
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int GQ = P.group, hq = P.hkv * GQ;
     float* w_s = buf;                        // [n_parts][8] maxima, then weights e^{m_j - m}
