@@ -282,11 +282,11 @@ def run_ours(args):
     total = 3 * (K + Wm)                       # eager run (per-launch events), graph run (timed), end-to-end run
     layers, plan, tab0 = build_layers(spec, total, device, M, torch)
     for L in layers:
-        L.pool.set_decode_variant(M.DECODE_SCALAR if args.variant == "scalar" else M.DECODE_TENSOR)
+        L.pool.set_decode_variant({"scalar": M.DECODE_SCALAR, "tmem": M.DECODE_TMEM}.get(args.variant, M.DECODE_TENSOR))
     B, d, hq, hkv = spec.batch, spec.head_dim, spec.n_q_heads, spec.n_kv_heads
     stream = torch.cuda.current_stream()
     launches = [0]
-    decode_launches = 1 if args.variant == "tensor" else 2    # tensor: one scan launch; scalar: scan + merge
+    decode_launches = 2 if args.variant == "scalar" else 1    # tensor: one scan launch; scalar: scan + merge
     # host mirror of the tags, advanced with the retier events, for the byte count of each step
     tags_host = initial_tags(tab0, np.zeros((B, plan["max_pages"]), np.uint8))
     ev_pairs = []
@@ -477,7 +477,7 @@ def run_ours(args):
                    "launch": "one CUDA graph per step (append + decode of every layer); retier calls issued directly"},
         "eager_ms_per_step": eager_ms / K,
         "kv_gbs_whole_step": step_bytes / (ms / K * 1e-3) / 1e9,
-        "roofline": {"bound": "hbm", "kernel": "decode_tensor_kernel" if args.variant == "tensor" else "decode_scalar_kernel + merge", "achieved": achieved, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": {"tensor": "decode_tensor_kernel", "tmem": "decode_tmem_kernel"}.get(args.variant, "decode_scalar_kernel + merge"), "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_kind + " copy bandwidth",
                      "frac_of_nominal_8000": achieved / 8000.0, "traffic": TRAFFIC_BYTES_PER_LAUNCH if (args.config == 2 and args.ctx == 0 and args.variant == "tensor") else None,
                      "algorithmic_bytes_per_launch": avg_bytes, "avg_launch_ms": avg_kernel_ms,
@@ -589,7 +589,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2)
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling on a small case)")
-    ap.add_argument("--variant", default="tensor", choices=["tensor", "scalar"],
+    ap.add_argument("--variant", default="tensor", choices=["tensor", "scalar", "tmem"],
                     help="decode kernel: the tensor-core product kernel, or the CUDA-core comparison kernel")
     ap.add_argument("--ctx", type=int, default=0, help="override the context length of every request (profiling)")
     ap.add_argument("--batch", type=int, default=0, help="config 4 only: requests of the lifecycle cell (default 8)")

@@ -62,7 +62,7 @@ enum { MKV_TAG_RECENT = 0, MKV_TAG_ANCHOR = 1, MKV_TAG_STALE = 2 };
 enum { MKV_FMT_FP8 = 0, MKV_FMT_TQ3 = 1 };
 /* decode kernels: the tensor-core kernel is the product; the CUDA-core kernel computes the same
  * thing with scalar FMAs and exists so that the choice of tensor cores can be measured */
-enum { MKV_DECODE_TENSOR = 0, MKV_DECODE_SCALAR = 1 };
+enum { MKV_DECODE_TENSOR = 0, MKV_DECODE_SCALAR = 1, MKV_DECODE_TMEM = 2 };
 
 typedef struct {
     int32_t page_size;          /* must be 16                                                   */

@@ -21,7 +21,7 @@ _lib = None
 OK, E_INVALID, E_OOM_FP8, E_OOM_TQ3, E_STATE, E_BOUNDS, E_CUDA, E_TIMEOUT = 0, -1, -2, -3, -4, -5, -6, -7
 TAG_RECENT, TAG_ANCHOR, TAG_STALE = 0, 1, 2
 FMT_FP8, FMT_TQ3 = 0, 1
-DECODE_TENSOR, DECODE_SCALAR = 0, 1
+DECODE_TENSOR, DECODE_SCALAR, DECODE_TMEM = 0, 1, 2
 _NAMES = {0: "MKV_OK", -1: "MKV_E_INVALID", -2: "MKV_E_OOM_FP8", -3: "MKV_E_OOM_TQ3", -4: "MKV_E_STATE",
           -5: "MKV_E_BOUNDS", -6: "MKV_E_CUDA", -7: "MKV_E_TIMEOUT"}
 

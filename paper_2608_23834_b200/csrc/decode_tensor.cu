@@ -1180,6 +1180,26 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
     }
 }
 
+#include "decode_tmem.cuh"
+
+template <int D>
+static int32_t run_tmem(mkv_pool* p, DecodeParams& prm, cudaStream_t s)
+{
+    using G = tm::TG<D>;
+    auto kern = decode_tmem_kernel<D>;
+    static bool attr_done[8] = {false, false, false, false, false, false, false, false};
+    const int dev = p->device & 7;
+    if (!attr_done[dev]) {
+        MKV_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM));
+        attr_done[dev] = true;
+    }
+    const int grid = p->dev.sm_count > kMaxCtas ? kMaxCtas : p->dev.sm_count;     // one block per SM: it takes all 512 tensor-memory columns
+    if (grid > prm.max_blocks) return MKV_E_INVALID;
+    kern<<<grid, tm::kThreads, G::SMEM, s>>>(prm);
+    MKV_CUDA(cudaGetLastError());
+    return MKV_OK;
+}
+
 template <int D, int NW, int NSTAGE, int MINB, bool SCORED = false>
 static int32_t run_tensor(mkv_pool* p, DecodeParams& prm, cudaStream_t s)
 {
@@ -1329,6 +1349,7 @@ int32_t launch_decode_tensor_at(mkv_pool* p, const void* q, const int32_t* bt, c
         if (rc != MKV_OK) return rc;
         return launch_page_mass_finish(mass, lse, lens, B, p->hkv * p->group, max_pages, s);
     }
+    if (p->variant == MKV_DECODE_TMEM && p->d == 256) return run_tmem<256>(p, prm, s);
     // Launch shapes (warps per block, ring slots per warp, blocks per SM); MKV_DECODE_SHAPE selects the
     // alternatives for profiling.
     const int shape = tensor_shape();

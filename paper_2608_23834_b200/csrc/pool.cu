@@ -225,7 +225,7 @@ int32_t mkv_pool_status(mkv_pool* pool, void* stream)
 
 int32_t mkv_pool_set_decode_variant(mkv_pool* pool, int32_t variant)
 {
-    if (!pool || (variant != MKV_DECODE_TENSOR && variant != MKV_DECODE_SCALAR)) return MKV_E_INVALID;
+    if (!pool || (variant != MKV_DECODE_TENSOR && variant != MKV_DECODE_SCALAR && variant != MKV_DECODE_TMEM)) return MKV_E_INVALID;
     pool->variant = variant;
     return MKV_OK;
 }

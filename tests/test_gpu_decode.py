@@ -11,7 +11,8 @@ from _gpu_util import Case, check_case, check_close
 
 pytestmark = pytest.mark.gpu
 
-VARIANTS = [pytest.param(M.DECODE_TENSOR, id="tensor"), pytest.param(M.DECODE_SCALAR, id="scalar")]
+VARIANTS = [pytest.param(M.DECODE_TENSOR, id="tensor"), pytest.param(M.DECODE_SCALAR, id="scalar"),
+            pytest.param(M.DECODE_TMEM, id="tmem")]     # tmem: tcgen05 kernel at d = 256, the tensor kernel at d = 128
 
 SCALED = {
     "cfg0": lambda: W.config(0),                                                        # 4,096 tokens as specified

@@ -21,6 +21,9 @@ def test_config2_one_full_layer_every_output():
     out, lse = case.run(M.DECODE_TENSOR)
     ref, ref_lse = case.reference()
     check_case(case, out, lse, ref, ref_lse)
+    out_tm, lse_tm = case.run(M.DECODE_TMEM)                 # the tcgen05 kernel on the same layer
+    check_case(case, out_tm, lse_tm, ref, ref_lse)
+    case.pool.set_decode_variant(M.DECODE_TENSOR)
     # the scored call on the same layer: same output bit for bit, page mass against the oracle
     out_s, _, mass = case.pool.decode_attention_scored(case.q, case.bt, case.tags, case.lens, spec.scale)
     torch.cuda.synchronize()
