@@ -34,8 +34,9 @@ constexpr int kTeamCols = 256;                      // tensor-memory columns of 
 // columns inside a team's range
 constexpr int kColK = 0;                            // key tile: d/2 columns (two fp16 per column)
 constexpr int kColS = 128;                          // scores: 16 columns
-constexpr int kColV = 144;                          // value tiles: 2 buffers x 2 halves x 8 columns
-constexpr int kColT = 176;                          // value products: 2 buffers x 2 halves x 16 columns
+constexpr int kColV = 144;                          // value tiles: 2 buffers x 2 pages x 2 halves x 8 columns
+constexpr int kColT = 0;                            // value products: 2 buffers x 2 pages x 2 halves x 16 columns, over the key
+                                                    // tile (dead once the scores are complete; every warp touches its own lanes only)
 
 template <int D>
 struct TG {
@@ -47,8 +48,8 @@ struct TG {
     static constexpr int QTILES = NB * 512;                            // query B tiles: 16 rows x 16 k x 2 bytes per block
     static constexpr int OFF_QT = RING;                                // rotated query (rows 0-7 high, 8-15 low halves)
     static constexpr int OFF_QF = OFF_QT + QTILES;                     // plain query (rows 0-7; rows 8-15 zero)
-    static constexpr int OFF_P = OFF_QF + QTILES;                      // per team: kTile x {high, low} x 512 bytes
-    static constexpr int OFF_PS = OFF_P + kTeams * kTile * 1024;       // per team: page sums [kTile][8] floats
+    static constexpr int OFF_P = OFF_QF + QTILES;                      // per team: kTile P tiles of 512 bytes (rows 0-7 high, 8-15 low halves)
+    static constexpr int OFF_PS = OFF_P + kTeams * kTile * 512;        // per team: page sums [kTile][8] floats
     static constexpr int OFF_BAR = OFF_PS + kTeams * kTile * 32;       // per team: 16 slot barriers, S, T0, T1 (32 x 8 bytes)
     static constexpr int OFF_LIST = OFF_BAR + kTeams * 256;            // per team: Stale ids, FP8 ids | valid << 27
     static constexpr int OFF_CNT = OFF_LIST + kTeams * 2 * kRoundT * 4;    // per team: n3, n8, 4 flags, 4 x 8 maxima
@@ -159,7 +160,7 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
     const int ttid = (warp & 3) * 32 + lane;                 // worker: thread index inside the team
     const int hkv = P.hkv, GQ = P.group, hq = hkv * GQ;
     // named barriers of the team: workers only; key tile ready; value tile ready (two, alternating); round hand-over
-    const int idW = 1 + 4 * team, idK = 2 + 4 * team, idV0 = 3 + 4 * team, idR = 9 + team;
+    const int idW = 1 + 5 * team, idK = 2 + 5 * team, idK2 = 3 + 5 * team, idV0 = 4 + 5 * team, idR = 11 + team;
 
     // ---- prologue -------------------------------------------------------------------------------
     if (tid == 0) {
@@ -172,8 +173,8 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
             if (P.lse)
                 for (int i = tid; i < hq; i += NT) P.lse[(size_t)b * hq + i] = -CUDART_INF_F;
         }
-    // rows 8-15 of the plain query tiles and of the P tiles stay zero for the whole launch
-    for (int i = tid; i < (G::QTILES + kTeams * kTile * 1024) / 4; i += NT) reinterpret_cast<uint32_t*>(smem + G::OFF_QF)[i] = 0;
+    // rows 8-15 of the plain query tiles stay zero for the whole launch
+    for (int i = tid; i < G::QTILES / 4; i += NT) reinterpret_cast<uint32_t*>(smem + G::OFF_QF)[i] = 0;
     if (warp == 0) {
         int run = 0;
         for (int b0 = 0; b0 < P.B; b0 += 32) {
@@ -224,7 +225,7 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
     bool failed = false;
     const uint32_t bars = sbase + G::OFF_BAR + team * 256;  // slot barriers 0..15, S = 16, T0 = 17, T1 = 18
     const uint32_t ring = sbase + team * 2 * kTile * G::SLOT;
-    const uint32_t ptiles = sbase + G::OFF_P + team * kTile * 1024;
+    const uint32_t ptiles = sbase + G::OFF_P + team * kTile * 512;
     float* ps_s = reinterpret_cast<float*>(smem + G::OFF_PS) + team * kTile * 8;
     int* list3 = reinterpret_cast<int*>(smem + G::OFF_LIST) + team * 2 * kRoundT;
     int* list8 = list3 + kRoundT;
@@ -249,6 +250,12 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
         }
     };
 
+#ifdef MKV_TIMELINE
+    unsigned long long tl_acc[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}, tl_last = tl_now(), tl_begin = tl_last;
+#define TM_STAMP(k) do { if (tid == 0) { const unsigned long long t__ = tl_now(); tl_acc[k] += t__ - tl_last; tl_last = t__; } } while (0)
+#else
+#define TM_STAMP(k)
+#endif
     int pos = my_start;
     int b = 0;
     while (pos < my_end) {
@@ -323,6 +330,7 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
         __syncthreads();
+        TM_STAMP(1);
 
         for (int round = 0; round < n_rounds; ++round) {
             // ---- table entries of the round -> two id lists of the team ---------------------------------
@@ -381,28 +389,39 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
                 for (int ti = 0; ti < n_tiles; ++ti) {
                     const bool stale = ti < tiles3;
                     const int np = stale ? min(kTile, n3 - ti * kTile) : min(kTile / 2, n8 - (ti - tiles3) * (kTile / 2));
-                    bar_sync(idK, 160);                      // key tile stored
+                    const uint32_t qtile = sbase + (stale ? G::OFF_QT : G::OFF_QF);
+                    bar_sync(idK, 160);                      // first half of the key tile stored
                     tc_fence_after();
                     if (lane == 0) {
-                        const uint32_t qtile = sbase + (stale ? G::OFF_QT : G::OFF_QF);
 #pragma unroll 1
-                        for (int kb = 0; kb < NB; ++kb)
+                        for (int kb = 0; kb < NB / 2; ++kb)
                             mma_ts(tb + kColS, tb + kColK + 8 * kb, b_tile_desc(qtile + kb * 512), kIdesc, kb > 0);
+                    }
+                    __syncwarp();
+                    bar_sync(idK2, 160);                     // second half
+                    tc_fence_after();
+                    if (lane == 0) {
+#pragma unroll 1
+                        for (int kb = NB / 2; kb < NB; ++kb)
+                            mma_ts(tb + kColS, tb + kColK + 8 * kb, b_tile_desc(qtile + kb * 512), kIdesc, 1);
                         mma_commit(bars + 8 * 16);
                     }
                     __syncwarp();
+                    const int nb = (np + 1) / 2;
 #pragma unroll 1
-                    for (int p = 0; p < np; ++p) {
-                        const uint32_t vb = p & 1;
-                        bar_sync(idV0 + vb, 160);            // value tile of page p stored (and, for p = 0, all P tiles)
+                    for (int bi = 0; bi < nb; ++bi) {
+                        const uint32_t vb = bi & 1;
+                        bar_sync(idV0 + vb, 160);            // value tiles of the batch stored (and, for the first, all P tiles)
                         tc_fence_after();
                         if (lane == 0) {
-                            const uint64_t dhi = b_tile_desc(ptiles + p * 1024), dlo = b_tile_desc(ptiles + p * 1024 + 512);
+#pragma unroll 1
+                            for (int e = 0; e < 2; ++e) {
+                                const int p = 2 * bi + e;
+                                if (p >= np) break;
+                                const uint64_t dp = b_tile_desc(ptiles + p * 512);
 #pragma unroll
-                            for (int m = 0; m < 2; ++m) {
-                                const uint32_t dT = tb + kColT + vb * 32 + m * 16, aV = tb + kColV + vb * 16 + m * 8;
-                                mma_ts(dT, aV, dhi, kIdesc, 0);
-                                mma_ts(dT, aV, dlo, kIdesc, 1);
+                                for (int m = 0; m < 2; ++m)
+                                    mma_ts(tb + kColT + vb * 64 + e * 32 + m * 16, tb + kColV + vb * 32 + e * 16 + m * 8, dp, kIdesc, 0);
                             }
                             mma_commit(bars + 8 * (17 + vb));
                         }
@@ -419,58 +438,70 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
                     const uint32_t buf = tcount & 1, par = (tcount >> 1) & 1;
                     ++tcount;
                     const uint32_t tile = ring + buf * kTile * G::SLOT;
+                    // every worker of the team has finished the tile before: the other buffer can be refilled now
+                    bar_sync(idW, 128);
+                    if (ti + 1 < n_tiles) issue_tile(ti + 1, tcount & 1);
 #pragma unroll 1
                     for (int s = 0; s < kTile; ++s) wait_bar(bars + 8 * (buf * kTile + s), par);
                     failed = __any_sync(FULL, failed);
+                    TM_STAMP(2);
 
-                    // ---- keys of this warp's two pages -> tensor memory ------------------------------------
+                    // ---- keys of this warp's two pages -> tensor memory, in two halves of d ---------------------
 #pragma unroll 1
-                    for (int e = 0; e < 2; ++e) {
-                        const int p = 2 * wq + e;
-                        if (p >= np) continue;
-                        const uint32_t dst = tb + kColK + my_lanes + ((uint32_t)(16 * e) << 16);
-                        if (stale) {
-                            uint32_t kw[LW];
-                            load_lane_words<D>(tile + p * G::SLOT, lane, kw);
+                    for (int half = 0; half < 2; ++half) {
+#pragma unroll 1
+                        for (int e = 0; e < 2; ++e) {
+                            const int p = 2 * wq + e;
+                            if (p >= np) continue;
+                            const uint32_t dst = tb + kColK + my_lanes + ((uint32_t)(16 * e) << 16) + 64 * half;
+                            if (stale) {
+                                // words 6 half .. 6 half + 5 of the lane: two 16-byte chunks (the second half starts mid-chunk)
+                                const uint32_t sec = tile + p * G::SLOT + lane * 16;
+                                const uint4 c0 = lds128(sec + (half ? 512 : 0)), c1 = lds128(sec + (half ? 1024 : 512));
+                                const uint32_t kw[6] = {half ? c0.z : c0.x, half ? c0.w : c0.y, half ? c1.x : c0.z,
+                                                        half ? c1.y : c0.w, half ? c1.z : c1.x, half ? c1.w : c1.y};
 #pragma unroll
-                            for (int j = 0; j < NB / 4; ++j) {
-                                const uint32_t A = kw[3 * j], Bw = kw[3 * j + 1], Cw = kw[3 * j + 2];
-                                uint32_t sel[4], r[16];
-                                sel[0] = A & 0x77777777u;
-                                sel[1] = Bw & 0x77777777u;
-                                sel[2] = lop3_and_or(A >> 1, 0x44444444u, Cw & 0x33333333u);
-                                sel[3] = lop3_and_or(Bw >> 1, 0x44444444u, (Cw >> 2) & 0x33333333u);
+                                for (int j = 0; j < 2; ++j) {
+                                    const uint32_t A = kw[3 * j], Bw = kw[3 * j + 1], Cw = kw[3 * j + 2];
+                                    uint32_t sel[4], r[16];
+                                    sel[0] = A & 0x77777777u;
+                                    sel[1] = Bw & 0x77777777u;
+                                    sel[2] = lop3_and_or(A >> 1, 0x44444444u, Cw & 0x33333333u);
+                                    sel[3] = lop3_and_or(Bw >> 1, 0x44444444u, (Cw >> 2) & 0x33333333u);
 #pragma unroll
-                                for (int w = 0; w < 4; ++w) {
-                                    uint32_t a0, a1, a2, a3;
-                                    key_lut4(sel[w], a0, a1);
-                                    key_lut4(sel[w] >> 16, a2, a3);
-                                    r[4 * w] = a0; r[4 * w + 1] = a2; r[4 * w + 2] = a1; r[4 * w + 3] = a3;
+                                    for (int w = 0; w < 4; ++w) {
+                                        uint32_t a0, a1, a2, a3;
+                                        key_lut4(sel[w], a0, a1);
+                                        key_lut4(sel[w] >> 16, a2, a3);
+                                        r[4 * w] = a0; r[4 * w + 1] = a2; r[4 * w + 2] = a1; r[4 * w + 3] = a3;
+                                    }
+                                    tmem_st_frag4(dst + 32 * j, r);
                                 }
-                                tmem_st_frag4(dst + 32 * j, r);
-                            }
-                        } else {
-                            const uint32_t kaddr = tile + 2 * p * G::SLOT;
+                            } else {
+                                const uint32_t kaddr = tile + 2 * p * G::SLOT;
 #pragma unroll
-                            for (int j = 0; j < D / 64; ++j) {
-                                const uint4 r0 = lds128(kaddr + g * D + 64 * j + 16 * tq);
-                                const uint4 r1 = lds128(kaddr + (g + 8) * D + 64 * j + 16 * tq);
-                                const uint32_t w0[4] = {r0.x, r0.y, r0.z, r0.w}, w1[4] = {r1.x, r1.y, r1.z, r1.w};
-                                uint32_t r[16];
+                                for (int jj = 0; jj < 2; ++jj) {
+                                    const int j = 2 * half + jj;
+                                    const uint4 r0 = lds128(kaddr + g * D + 64 * j + 16 * tq);
+                                    const uint4 r1 = lds128(kaddr + (g + 8) * D + 64 * j + 16 * tq);
+                                    const uint32_t w0[4] = {r0.x, r0.y, r0.z, r0.w}, w1[4] = {r1.x, r1.y, r1.z, r1.w};
+                                    uint32_t r[16];
 #pragma unroll
-                                for (int w = 0; w < 4; ++w) {
-                                    r[4 * w] = e4m3x2_to_f16x2((uint16_t)(w0[w] & 0xFFFFu));
-                                    r[4 * w + 1] = e4m3x2_to_f16x2((uint16_t)(w0[w] >> 16));
-                                    r[4 * w + 2] = e4m3x2_to_f16x2((uint16_t)(w1[w] & 0xFFFFu));
-                                    r[4 * w + 3] = e4m3x2_to_f16x2((uint16_t)(w1[w] >> 16));
+                                    for (int w = 0; w < 4; ++w) {
+                                        r[4 * w] = e4m3x2_to_f16x2((uint16_t)(w0[w] & 0xFFFFu));
+                                        r[4 * w + 1] = e4m3x2_to_f16x2((uint16_t)(w0[w] >> 16));
+                                        r[4 * w + 2] = e4m3x2_to_f16x2((uint16_t)(w1[w] & 0xFFFFu));
+                                        r[4 * w + 3] = e4m3x2_to_f16x2((uint16_t)(w1[w] >> 16));
+                                    }
+                                    tmem_st_frag4(dst + 32 * jj, r);
                                 }
-                                tmem_st_frag4(dst + 32 * j, r);
                             }
                         }
+                        tmem_wait_st();
+                        tc_fence_before();
+                        bar_arrive(half ? idK2 : idK, 160);
                     }
-                    tmem_wait_st();
-                    tc_fence_before();
-                    bar_arrive(idK, 160);
+                    TM_STAMP(3);
 
                     // ---- scores of this thread's token -------------------------------------------------------
                     const int p_me = 2 * wq + (lane >> 4), tok = lane & 15;
@@ -480,6 +511,7 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
                     wait_bar(bars + 8 * 16, scount & 1);
                     ++scount;
                     failed = __any_sync(FULL, failed);
+                    TM_STAMP(4);
                     tc_fence_after();
                     float s[8];
                     {
@@ -501,7 +533,6 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
                     ex = __any_sync(FULL, ex);
                     if (lane == 0) cnt[4 + wq] = ex ? 1 : 0;
                     bar_sync(idW, 128);
-                    if (ti + 1 < n_tiles) issue_tile(ti + 1, tcount & 1);     // every worker is done with that buffer's last tile
                     if (cnt[4] | cnt[5] | cnt[6] | cnt[7]) {
                         float mx[8];
 #pragma unroll
@@ -532,10 +563,10 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
                         }
                         bar_sync(idW, 128);                  // the maxima are read before the next tile overwrites them
                     }
-                    // probabilities of this token -> B tiles of its page (high and low fp16 halves), page sums
+                    // probabilities of this token -> B tile of its page (rows 0-7 high, 8-15 low fp16 halves), page sums
                     {
                         const int kk = stale ? k_of_token_tq3(tok) : tok;
-                        const uint32_t thi = ptiles + (p_me & (kTile - 1)) * 1024, tlo = thi + 512;
+                        const uint32_t tp = ptiles + (p_me & (kTile - 1)) * 512;
                         float pv[8];
 #pragma unroll
                         for (int i = 0; i < 8; ++i) {
@@ -543,8 +574,8 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
                             const __half ph = __float2half_rn(pr);
                             const __half pl = __float2half_rn(pr - __half2float(ph));
                             if (p_me < np) {
-                                asm volatile("st.shared.u16 [%0], %1;" ::"r"(thi + b_tile_offset(i, kk)), "h"(__half_as_ushort(ph)) : "memory");
-                                asm volatile("st.shared.u16 [%0], %1;" ::"r"(tlo + b_tile_offset(i, kk)), "h"(__half_as_ushort(pl)) : "memory");
+                                asm volatile("st.shared.u16 [%0], %1;" ::"r"(tp + b_tile_offset(i, kk)), "h"(__half_as_ushort(ph)) : "memory");
+                                asm volatile("st.shared.u16 [%0], %1;" ::"r"(tp + b_tile_offset(8 + i, kk)), "h"(__half_as_ushort(pl)) : "memory");
                             }
                             pv[i] = __half2float(ph) + __half2float(pl);
                         }
@@ -553,85 +584,100 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
 #pragma unroll
                             for (int o = 8; o > 0; o >>= 1) pv[i] += __shfl_xor_sync(FULL, pv[i], o);
                         }
-                        if (tok == 0 && p_me < kTile) {
+                        if (tok == 0) {
                             *reinterpret_cast<float4*>(ps_s + p_me * 8) = make_float4(pv[0], pv[1], pv[2], pv[3]);
                             *reinterpret_cast<float4*>(ps_s + p_me * 8 + 4) = make_float4(pv[4], pv[5], pv[6], pv[7]);
                         }
                         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     }
                     bar_sync(idW, 128);                      // page sums and P tiles of all four warps are in place
+                    TM_STAMP(5);
 
-                    // ---- values: page by page; the products of page p run while page p + 1 is unpacked ----------
-                    auto scale_page = [&](int p) {
-                        const uint32_t vb = p & 1;
+                    // ---- values: two pages at a time; the products of a batch run while the next one is unpacked -----
+                    auto scale_batch = [&](int bi) {
+                        const uint32_t vb = bi & 1;
+                        TM_STAMP(6);
                         if (vb) { wait_bar(bars + 8 * 18, tcnt1 & 1); ++tcnt1; } else { wait_bar(bars + 8 * 17, tcnt0 & 1); ++tcnt0; }
+                        TM_STAMP(7);
                         tc_fence_after();
-                        float t0[8], t1[8];
-                        tmem_ld8(tb + kColT + vb * 32 + my_lanes, t0);
-                        tmem_ld8(tb + kColT + vb * 32 + 16 + my_lanes, t1);
-                        tmem_wait_ld();
-                        const float4 pa = *reinterpret_cast<const float4*>(ps_s + p * 8), pb = *reinterpret_cast<const float4*>(ps_s + p * 8 + 4);
-                        const float ps[8] = {pa.x, pa.y, pa.z, pa.w, pb.x, pb.y, pb.z, pb.w};
-                        float sc0 = P.v_scale, zp0 = 0.f, sc1 = P.v_scale, zp1 = 0.f;
-                        if (stale) {
-                            // channel 16 cb + row: halves (scale, zero) at ((cb/2) 64 + (row%8) 8 + 4 (cb%2) + row/8) and + 2
-                            const uint32_t meta = tile + p * G::SLOT + 12 * D + 32;
-                            const int row = lane & 15, cb0 = 4 * wq + (lane >> 4), cb1 = cb0 + 2;
-                            const uint32_t i0 = (cb0 >> 1) * 64 + (row & 7) * 8 + 4 * (cb0 & 1) + (row >> 3);
-                            const uint32_t i1 = (cb1 >> 1) * 64 + (row & 7) * 8 + 4 * (cb1 & 1) + (row >> 3);
-                            sc0 = __half2float(__ushort_as_half(lds16(meta + 2 * i0)));
-                            zp0 = __half2float(__ushort_as_half(lds16(meta + 2 * i0 + 4)));
-                            sc1 = __half2float(__ushort_as_half(lds16(meta + 2 * i1)));
-                            zp1 = __half2float(__ushort_as_half(lds16(meta + 2 * i1 + 4)));
-                        }
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            acc0[i] = fmaf(sc0, t0[i], fmaf(zp0, ps[i], acc0[i]));
-                            acc1[i] = fmaf(sc1, t1[i], fmaf(zp1, ps[i], acc1[i]));
-                            l_run[i] += ps[i];
-                        }
-                    };
 #pragma unroll 1
-                    for (int p = 0; p < np; ++p) {
-                        const uint32_t vb = p & 1;
-                        const uint32_t dV = tb + kColV + vb * 16 + my_lanes;     // half m at + 8 m, rows 16..31 at + (16 << 16)
-                        if (stale) {
-                            const uint32_t sec = tile + p * G::SLOT + 6 * D;
-                            uint32_t W[3];
-#pragma unroll
-                            for (int e = 0; e < 3; ++e) {
-                                const int i = 3 * wq + e;
-                                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(W[e]) : "r"(sec + (i >> 2) * 512 + lane * 16 + (i & 3) * 4));
+                        for (int e = 0; e < 2; ++e) {
+                            const int p = 2 * bi + e;
+                            if (p >= np) break;
+                            float t0[16], t1[16];
+                            tmem_ld16(tb + kColT + vb * 64 + e * 32 + my_lanes, t0);
+                            tmem_ld16(tb + kColT + vb * 64 + e * 32 + 16 + my_lanes, t1);
+                            tmem_wait_ld();
+                            const float4 pa = *reinterpret_cast<const float4*>(ps_s + p * 8), pb = *reinterpret_cast<const float4*>(ps_s + p * 8 + 4);
+                            const float ps[8] = {pa.x, pa.y, pa.z, pa.w, pb.x, pb.y, pb.z, pb.w};
+                            float sc0 = P.v_scale, zp0 = 0.f, sc1 = P.v_scale, zp1 = 0.f;
+                            if (stale) {
+                                // channel 16 cb + row: halves (scale, zero) at ((cb/2) 64 + (row%8) 8 + 4 (cb%2) + row/8) and + 2
+                                const uint32_t meta = tile + p * G::SLOT + 12 * D + 32;
+                                const int row = lane & 15, cb0 = 4 * wq + (lane >> 4), cb1 = cb0 + 2;
+                                const uint32_t i0 = (cb0 >> 1) * 64 + (row & 7) * 8 + 4 * (cb0 & 1) + (row >> 3);
+                                const uint32_t i1 = (cb1 >> 1) * 64 + (row & 7) * 8 + 4 * (cb1 & 1) + (row >> 3);
+                                sc0 = __half2float(__ushort_as_half(lds16(meta + 2 * i0)));
+                                zp0 = __half2float(__ushort_as_half(lds16(meta + 2 * i0 + 4)));
+                                sc1 = __half2float(__ushort_as_half(lds16(meta + 2 * i1)));
+                                zp1 = __half2float(__ushort_as_half(lds16(meta + 2 * i1 + 4)));
                             }
-                            const uint32_t X1 = prmt(W[0], W[1], 0x6341u), X0 = prmt(W[1], W[2], 0x6341u), X2 = W[2] >> 8;
-                            tmem_st_frag(dV, value_code<0>(W[0]), value_code<3>(W[0]), value_code<6>(W[0]), value_code<1>(X1));
-                            tmem_st_frag(dV + (16u << 16), value_code<4>(X1), value_code<7>(X1), value_code<2>(W[1]), value_code<5>(W[1]));
-                            tmem_st_frag(dV + 8, value_code<0>(X0), value_code<3>(X0), value_code<6>(X0), value_code<1>(W[2]));
-                            tmem_st_frag(dV + 8 + (16u << 16), value_code<4>(W[2]), value_code<7>(W[2]), value_code<2>(X2), value_code<5>(X2));
-                        } else {
-                            const uint32_t vaddr = tile + (2 * p + 1) * G::SLOT;
-                            const int v = (list8[first + p] >> 27) & 15, nv = v ? v : kPage;
-                            const uint32_t keep = (4 * tq < nv ? 0x000000FFu : 0u) | (4 * tq + 1 < nv ? 0x0000FF00u : 0u) |
-                                                  (4 * tq + 2 < nv ? 0x00FF0000u : 0u) | (4 * tq + 3 < nv ? 0xFF000000u : 0u);
 #pragma unroll
-                            for (int m = 0; m < 2; ++m) {
-                                uint32_t v4[4];
-                                ldmatrix_x4(vaddr + (4 * wq + 2 * m) * 256 + lane * 16, v4[0], v4[1], v4[2], v4[3]);
+                            for (int i = 0; i < 8; ++i) {
+                                acc0[i] = fmaf(sc0, t0[i] + t0[8 + i], fmaf(zp0, ps[i], acc0[i]));
+                                acc1[i] = fmaf(sc1, t1[i] + t1[8 + i], fmaf(zp1, ps[i], acc1[i]));
+                                l_run[i] += ps[i];
+                            }
+                        }
+                        TM_STAMP(8);
+                    };
+                    const int nb = (np + 1) / 2;
+#pragma unroll 1
+                    for (int bi = 0; bi < nb; ++bi) {
+                        const uint32_t vb = bi & 1;
+#pragma unroll 1
+                        for (int e = 0; e < 2; ++e) {
+                            const int p = 2 * bi + e;
+                            if (p >= np) break;
+                            const uint32_t dV = tb + kColV + vb * 32 + e * 16 + my_lanes;   // half m at + 8 m, rows 16..31 at + (16 << 16)
+                            if (stale) {
+                                const uint32_t sec = tile + p * G::SLOT + 6 * D;
+                                uint32_t W[3];
 #pragma unroll
-                                for (int e = 0; e < 2; ++e) {
-                                    const uint32_t lo = v4[2 * e] & keep, hi = v4[2 * e + 1] & keep;
-                                    tmem_st_frag(dV + 8 * m + ((uint32_t)(16 * e) << 16), e4m3x2_to_f16x2((uint16_t)(lo & 0xFFFFu)),
-                                                 e4m3x2_to_f16x2((uint16_t)(hi & 0xFFFFu)), e4m3x2_to_f16x2((uint16_t)(lo >> 16)),
-                                                 e4m3x2_to_f16x2((uint16_t)(hi >> 16)));
+                                for (int k = 0; k < 3; ++k) {
+                                    const int i = 3 * wq + k;
+                                    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(W[k]) : "r"(sec + (i >> 2) * 512 + lane * 16 + (i & 3) * 4));
+                                }
+                                const uint32_t X1 = prmt(W[0], W[1], 0x6341u), X0 = prmt(W[1], W[2], 0x6341u), X2 = W[2] >> 8;
+                                tmem_st_frag(dV, value_code<0>(W[0]), value_code<3>(W[0]), value_code<6>(W[0]), value_code<1>(X1));
+                                tmem_st_frag(dV + (16u << 16), value_code<4>(X1), value_code<7>(X1), value_code<2>(W[1]), value_code<5>(W[1]));
+                                tmem_st_frag(dV + 8, value_code<0>(X0), value_code<3>(X0), value_code<6>(X0), value_code<1>(W[2]));
+                                tmem_st_frag(dV + 8 + (16u << 16), value_code<4>(W[2]), value_code<7>(W[2]), value_code<2>(X2), value_code<5>(X2));
+                            } else {
+                                const uint32_t vaddr = tile + (2 * p + 1) * G::SLOT;
+                                const int v = (list8[first + p] >> 27) & 15, nv = v ? v : kPage;
+                                const uint32_t keep = (4 * tq < nv ? 0x000000FFu : 0u) | (4 * tq + 1 < nv ? 0x0000FF00u : 0u) |
+                                                      (4 * tq + 2 < nv ? 0x00FF0000u : 0u) | (4 * tq + 3 < nv ? 0xFF000000u : 0u);
+#pragma unroll
+                                for (int m = 0; m < 2; ++m) {
+                                    uint32_t v4[4];
+                                    ldmatrix_x4(vaddr + (4 * wq + 2 * m) * 256 + lane * 16, v4[0], v4[1], v4[2], v4[3]);
+#pragma unroll
+                                    for (int k = 0; k < 2; ++k) {
+                                        const uint32_t lo = v4[2 * k] & keep, hi = v4[2 * k + 1] & keep;
+                                        tmem_st_frag(dV + 8 * m + ((uint32_t)(16 * k) << 16), e4m3x2_to_f16x2((uint16_t)(lo & 0xFFFFu)),
+                                                     e4m3x2_to_f16x2((uint16_t)(hi & 0xFFFFu)), e4m3x2_to_f16x2((uint16_t)(lo >> 16)),
+                                                     e4m3x2_to_f16x2((uint16_t)(hi >> 16)));
+                                    }
                                 }
                             }
                         }
                         tmem_wait_st();
                         tc_fence_before();
                         bar_arrive(idV0 + vb, 160);
-                        if (p > 0) scale_page(p - 1);
+                        if (bi > 0) scale_batch(bi - 1);
                     }
-                    if (np > 0) scale_page(np - 1);
+                    if (nb > 0) scale_batch(nb - 1);
                     failed = __any_sync(FULL, failed);
                 }
             }
@@ -639,8 +685,10 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
         }
 
         // ---- combine the teams of the block (ring memory is idle now) -------------------------------------
+        TM_STAMP(9);
         tc_fence_before();
         __syncthreads();
+        TM_STAMP(10);
         if (worker && ttid == 0) {
 #pragma unroll
             for (int i = 0; i < 8; ++i) sm_m[team * 8 + i] = m_run[i];
@@ -725,9 +773,18 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
             }
         }
         __syncthreads();
+        TM_STAMP(11);
         pos += n_seg;
     }
+#ifdef MKV_TIMELINE
+    if (tid == 0) {
+        for (int k = 0; k < 12; ++k) g_timeline[blockIdx.x * 16 + k] = tl_acc[k];
+        g_timeline[blockIdx.x * 16 + 15] = tl_begin;
+        g_timeline[blockIdx.x * 16 + 14] = tl_now();
+    }
+#endif
     tc_fence_before();
     __syncthreads();
     if (warp == kWorkerWarps) tmem_dealloc(tmem_all, 512);
 }
+#undef TM_STAMP
