@@ -60,8 +60,11 @@ typedef enum {
 
 enum { MKV_TAG_RECENT = 0, MKV_TAG_ANCHOR = 1, MKV_TAG_STALE = 2 };
 enum { MKV_FMT_FP8 = 0, MKV_FMT_TQ3 = 1 };
-/* decode kernels: the tensor-core kernel is the product; the CUDA-core kernel computes the same
- * thing with scalar FMAs and exists so that the choice of tensor cores can be measured */
+/* decode kernels: the tensor-core kernel (mma.sync, accumulators in registers) is the product; the
+ * CUDA-core kernel computes the same thing with scalar FMAs and exists so that the choice of tensor
+ * cores can be measured; MKV_DECODE_TMEM runs the products as tcgen05.mma with operands and
+ * accumulators in tensor memory and the stages of a page in specialised warps (head_dim 256; other
+ * sizes and the scored call use the tensor-core kernel) -- same results, at present slower */
 enum { MKV_DECODE_TENSOR = 0, MKV_DECODE_SCALAR = 1, MKV_DECODE_TMEM = 2 };
 
 typedef struct {

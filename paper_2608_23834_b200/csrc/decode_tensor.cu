@@ -667,12 +667,12 @@ __device__ __forceinline__ void fp8_page(WarpAcc<D / 16>& acc, uint32_t kaddr, u
 // reduces the maxima and row sums of head hd (one trip to L2: both are loaded together and kept in
 // shared memory); a thread then owns float4 groups (one channel, four heads) of the [channel][8 heads]
 // tile and has 40 loads in flight, issued before the weights are worked out.
-template <int D, int NT>
+template <int D, int NT, int KPMAX = 40>
 __device__ __forceinline__ void merge_row(const DecodeParams& P, int first_slot, int even_base, int n_parts,
                                           float* buf, int b, int h)
 {
     constexpr uint32_t FULL = 0xffffffffu;
-    constexpr int STRIDE = 8 * D + 16, GPT = (2 * D + NT - 1) / NT, KP = 40 / GPT;   // 40 float4 loads in flight per thread
+    constexpr int STRIDE = 8 * D + 16, GPT = (2 * D + NT - 1) / NT, KP = KPMAX / GPT;   // KPMAX (40) float4 loads in flight per thread
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int GQ = P.group, hq = P.hkv * GQ;
     float* w_s = buf;                        // [n_parts][8] maxima, then weights e^{m_j - m}
@@ -1193,7 +1193,7 @@ static int32_t run_tmem(mkv_pool* p, DecodeParams& prm, cudaStream_t s)
         MKV_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM));
         attr_done[dev] = true;
     }
-    const int grid = p->dev.sm_count > kMaxCtas ? kMaxCtas : p->dev.sm_count;     // one block per SM: it takes all 512 tensor-memory columns
+    const int grid = p->dev.sm_count > kMaxCtas ? kMaxCtas : p->dev.sm_count;     // one block per SM: it takes all the tensor memory
     if (grid > prm.max_blocks) return MKV_E_INVALID;
     kern<<<grid, tm::kThreads, G::SMEM, s>>>(prm);
     MKV_CUDA(cudaGetLastError());

@@ -2,41 +2,55 @@
 // Included by decode_tensor.cu (it shares that file's partition, unpack and merge code).
 //
 // Same one-pass mixed-format scan and the same split/merge as the mma.sync kernel; what changes is where
-// the products run and who owns what:
-//   * a block holds two teams of four worker warps plus one issuing warp per team.  A team works on a
-//     tile of eight Stale pages (or four Recent/Anchor pages) of its share of the row at a time.
-//   * keys: every worker warp unpacks two pages into MMA A fragments exactly as the mma.sync kernel
-//     does, but stores them to tensor memory (tcgen05.st.16x256b puts a fragment's registers at
-//     (row g | g+8, 32-bit columns 2tq, 2tq+1), i.e. a 16 x 16 tile with its K order permuted; the
-//     query tile in shared memory is written in the same permuted order).  One thread of the issuing
-//     warp then runs S[128 tokens x 16] = K q'^T as d/16 tcgen05.mma (M 128, N 16: eight heads of the
-//     high half of the rotated query and eight of the low half), accumulating in tensor memory.
-//   * softmax: a worker thread owns one token (tensor-memory lane = token): it reads its 16 scores,
-//     forms P for the eight heads and writes P (fp16 high and low halves) into the B tiles of the
-//     value product; page sums come from shuffles over the 16 lanes of a page.
-//   * values: for every page the four worker warps unpack one quad of 16-channel blocks each into
-//     tensor memory; T[256 channels x 8 heads] = codes^T P runs as four tcgen05.mma (two 128-row
-//     halves x {P high, P low}).  A worker thread owns two channels (its lane of the two halves): it
-//     reads their 2 x 8 results and applies the page's scale and zero in fp32 to 16 accumulators in
-//     registers -- two conversions per page and thread instead of the sixteen the fragment layout
-//     of mma.sync forces, and no accumulator fragments in registers.
-//   * hand-over between workers and the issuing warp is by named barriers (workers arrive, the
-//     issuing warp waits) and by mbarriers signalled with tcgen05.commit (workers wait, bounded by wall
-//     time like every other wait here); worker warps never wait for each other inside a page.
+// the products run, who owns what, and that the stages of a page run in different warps at the same time.
+// A block works on tiles of eight Stale pages (or four Recent/Anchor pages) = 128 tokens = the 128
+// lanes of tensor memory.  Its 19 warps are seven groups, each a loop "wait for the inputs of my stage,
+// do it, signal the outputs", coupled only by mbarriers (every wait bounded by wall time):
+//   producer (1 warp)   bulk copies of a tile's records into one of four shared-memory tile buffers
+//   key unpack (4)      each warp unpacks two pages into MMA A fragments exactly as the mma.sync kernel does
+//                       and stores them to tensor memory (tcgen05.st.16x256b puts a fragment at rows g, g+8,
+//                       32-bit columns 2tq, 2tq+1: a 16 x 16 tile with its K order permuted; the query tile
+//                       in shared memory is written in the same permuted order)
+//   score issue (1)     S[128 tokens x 16] = K q'^T: d/16 tcgen05.mma (M 128, N 16: the eight heads of the high
+//                       half of the rotated query and of its low half), accumulating in tensor memory
+//   softmax (4)         a thread owns one token (its tensor-memory lane): reads 16 scores, keeps the running
+//                       maxima of the block, writes P (fp16 high | low halves) into the B tile of its page,
+//                       page sums by shuffles over the 16 lanes of a page, rescale factors for the accumulators
+//   value unpack (4)    per page each warp unpacks one quad of 16-channel blocks to tensor memory
+//   value issue (1)     T[256 channels x 16] = codes^T P for two pages at a time (two 128-row halves each)
+//   scale (4)           a thread owns two channels (its lane of the two halves): reads their results and applies
+//                       the page's scale and zero in fp32 to 16 accumulators in registers -- two conversions per
+//                       page and thread instead of the sixteen the fragment layout of mma.sync forces
+// Key tiles, scores, value tiles and value products are double-buffered in tensor memory (480 of 512
+// columns), so that all stages of consecutive tiles overlap.
 namespace tm {
 
-constexpr int kTeams = 2;                           // teams per block
 constexpr int kTile = 8;                            // Stale pages per tile (Recent/Anchor pages: half as many)
-constexpr int kRoundT = 256;                        // positions of a team whose table entries are listed at a time
-constexpr int kWorkerWarps = kTeams * 4;            // warps 0 .. 7; warps 8, 9 issue the MMAs of team 0, 1
-constexpr int kThreads = (kWorkerWarps + kTeams) * 32;
-constexpr int kTeamCols = 256;                      // tensor-memory columns of a team
-// columns inside a team's range
+constexpr int kRing = 4;                            // tile buffers in shared memory
+constexpr int kRoundT = 512;                        // positions whose table entries are listed at a time
+constexpr int kWarps = 19;
+constexpr int kThreads = kWarps * 32;
+enum { kKU = 0, kSM = 4, kVU = 8, kSC = 12, kISS = 16, kISV = 17, kPR = 18 };   // first warp of every group
+// tensor-memory columns
 constexpr int kColK = 0;                            // key tile: d/2 columns (two fp16 per column)
-constexpr int kColS = 128;                          // scores: 16 columns
-constexpr int kColV = 144;                          // value tiles: 2 buffers x 2 pages x 2 halves x 8 columns
-constexpr int kColT = 0;                            // value products: 2 buffers x 2 pages x 2 halves x 16 columns, over the key
-                                                    // tile (dead once the scores are complete; every warp touches its own lanes only)
+constexpr int kColS = 128;                          // scores: 2 x 16 columns
+constexpr int kColV = 160;                          // value tiles: 2 buffers x 2 pages x 2 halves x 8 columns
+constexpr int kColT = 224;                          // value products: 4 buffers x 2 pages x 2 halves x 16 columns
+constexpr int kTBuf = 4;
+// mbarriers (index into the barrier array)
+enum {
+    kBarFull = 0,                                   // [kRing][kTile] records of a slot have landed (or the slot is unused)
+    kBarTileFree = kRing * kTile,                   // [kRing] all 16 consumer warps are done with the buffer
+    kBarKReady = kBarTileFree + kRing,              // [2] key tile stored (4 warps)
+    kBarSFull = kBarKReady + 2,                     // [2] scores complete (commit); also: key tile may be overwritten
+    kBarSFree = kBarSFull + 2,                      // [2] scores read (4 warps)
+    kBarPReady = kBarSFree + 2,                     // [2] P tiles, page sums and rescale factors written (4 warps)
+    kBarSCDone = kBarPReady + 2,                    // [2] scale warps are done with the tile (4 warps)
+    kBarVReady = kBarSCDone + 2,                    // [2] value tiles of a batch stored (4 warps)
+    kBarTFull = kBarVReady + 2,                     // [4] value products of a batch complete (commit); value tiles free
+    kBarTFree = kBarTFull + 4,                      // [4] value products read (4 warps)
+    kBarCount = kBarTFree + 4
+};
 
 template <int D>
 struct TG {
@@ -44,25 +58,25 @@ struct TG {
     static constexpr int TQ3_REC = 16 * D + 32;
     static constexpr int FP8_HALF = 16 * D;
     static constexpr int SLOT = (TQ3_REC + 127) / 128 * 128;
-    static constexpr int RING = kTeams * 2 * kTile * SLOT;             // per team two buffers of eight slots
+    static constexpr int RING = kRing * kTile * SLOT;
     static constexpr int QTILES = NB * 512;                            // query B tiles: 16 rows x 16 k x 2 bytes per block
     static constexpr int OFF_QT = RING;                                // rotated query (rows 0-7 high, 8-15 low halves)
     static constexpr int OFF_QF = OFF_QT + QTILES;                     // plain query (rows 0-7; rows 8-15 zero)
-    static constexpr int OFF_P = OFF_QF + QTILES;                      // per team: kTile P tiles of 512 bytes (rows 0-7 high, 8-15 low halves)
-    static constexpr int OFF_PS = OFF_P + kTeams * kTile * 512;        // per team: page sums [kTile][8] floats
-    static constexpr int OFF_BAR = OFF_PS + kTeams * kTile * 32;       // per team: 16 slot barriers, S, T0, T1 (32 x 8 bytes)
-    static constexpr int OFF_LIST = OFF_BAR + kTeams * 256;            // per team: Stale ids, FP8 ids | valid << 27
-    static constexpr int OFF_CNT = OFF_LIST + kTeams * 2 * kRoundT * 4;    // per team: n3, n8, 4 flags, 4 x 8 maxima
-    static constexpr int OFF_CUM = OFF_CNT + kTeams * 256;
+    static constexpr int OFF_P = OFF_QF + QTILES;                      // 2 x kTile P tiles of 512 bytes (rows 0-7 high, 8-15 low)
+    static constexpr int OFF_PS = OFF_P + 2 * kTile * 512;             // 2 x (page sums [kTile][8], rescale factors [8]) floats
+    static constexpr int OFF_BAR = OFF_PS + 2 * (kTile + 1) * 32;
+    static constexpr int OFF_LIST = OFF_BAR + ((kBarCount * 8 + 127) / 128) * 128;   // Stale ids, FP8 ids | valid << 27
+    static constexpr int OFF_CNT = OFF_LIST + 2 * kRoundT * 4;         // n3, n8, 4 flags, 4 x 8 maxima
+    static constexpr int OFF_CUM = OFF_CNT + 256;
     static constexpr int OFF_STRIDE = OFF_CUM + (kMaxBatch + 1) * 4;
     static constexpr int OFF_M = OFF_STRIDE + kMaxBatch * 4;
-    static constexpr int OFF_L = OFF_M + kTeams * 8 * 4;
-    static constexpr int OFF_PART = OFF_L + kTeams * 8 * 4;
+    static constexpr int OFF_L = OFF_M + 8 * 4;
+    static constexpr int OFF_PART = OFF_L + 8 * 4;
     static constexpr int OFF_LAST = OFF_PART + ((int)sizeof(Partition) + 15) / 16 * 16;
     static constexpr int OFF_TMEM = OFF_LAST + 16;
     static constexpr int SMEM = OFF_TMEM + 16;
     static_assert(D == 256, "column map and channel ownership are laid out for d = 256");
-    static_assert(RING >= kTeams * 8 * D * 4 + kMaxCtas * 16 * 4 + 64, "ring doubles as reduction and merge buffer");
+    static_assert(RING >= 8 * D * 4 + kMaxCtas * 16 * 4 + 64, "ring doubles as reduction and merge buffer");
 };
 
 // ---- tcgen05 wrappers ---------------------------------------------------------------------------
@@ -118,6 +132,14 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// try_wait that lets the hardware suspend the thread (up to `ns`) until the phase completes, instead of spinning
+__device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity, uint32_t ns)
+{
+    uint32_t ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(bar), "r"(parity), "r"(ns) : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ void bar_sync(int id, int count) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory"); }
 __device__ __forceinline__ void bar_arrive(int id, int count) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory"); }
 // B tile in shared memory: 16 rows x 16 k of fp16, K-major, no swizzle: 8-row x 16-byte core matrices, the two
@@ -133,6 +155,7 @@ constexpr uint32_t kIdesc = (1u << 4) | (uint32_t)(16 >> 3) << 17 | (uint32_t)(1
 // (2tq+8, 2tq+9) in columns 2tq and 2tq+1; Recent/Anchor fragments (ldmatrix) tokens 4tq .. 4tq+3
 __device__ __forceinline__ int k_of_token_tq3(int t) { return 4 * ((t & 7) >> 1) + (t & 1) + ((t >> 3) << 1); }
 
+
 }  // namespace tm
 
 template <int D>
@@ -140,7 +163,7 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
 {
     using namespace tm;
     using G = TG<D>;
-    constexpr int NB = G::NB, NT = kThreads, NU = kTeams, LW = 3 * NB / 4;
+    constexpr int NB = G::NB, NT = kThreads;
     constexpr uint32_t FULL = 0xffffffffu;
     extern __shared__ __align__(128) uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
@@ -151,20 +174,26 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
     Partition* pt = reinterpret_cast<Partition*>(smem + G::OFF_PART);
     int* last_s = reinterpret_cast<int*>(smem + G::OFF_LAST);
     uint32_t* tmem_s = reinterpret_cast<uint32_t*>(smem + G::OFF_TMEM);
-    float* red = reinterpret_cast<float*>(smem);            // [teams][D][8] over the ring, between segments
+    float* red = reinterpret_cast<float*>(smem);            // [D][8] over the ring, between segments
+    int* list3 = reinterpret_cast<int*>(smem + G::OFF_LIST);
+    int* list8 = list3 + kRoundT;
+    int* cnt = reinterpret_cast<int*>(smem + G::OFF_CNT);   // [0] n3, [1] n8, [4..7] flags, [8..39] maxima
+    float* ps_all = reinterpret_cast<float*>(smem + G::OFF_PS);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tq = lane & 3;
-    const bool worker = warp < kWorkerWarps;
-    const int team = worker ? warp >> 2 : warp - kWorkerWarps;
-    const int wq = warp & 3;                                 // worker: tensor-memory subpartition = quad of value blocks
-    const int ttid = (warp & 3) * 32 + lane;                 // worker: thread index inside the team
+    const int wq = warp & 3;                                 // tensor-memory subpartition of the warp (groups start at multiples of 4)
     const int hkv = P.hkv, GQ = P.group, hq = hkv * GQ;
-    // named barriers of the team: workers only; key tile ready; value tile ready (two, alternating); round hand-over
-    const int idW = 1 + 5 * team, idK = 2 + 5 * team, idK2 = 3 + 5 * team, idV0 = 4 + 5 * team, idR = 11 + team;
+    const uint32_t bars = sbase + G::OFF_BAR;
+    auto bar = [&](int idx) -> uint32_t { return bars + 8 * idx; };
 
     // ---- prologue -------------------------------------------------------------------------------
     if (tid == 0) {
-        for (int i = 0; i < kTeams * 32; ++i) mbar_init(sbase + G::OFF_BAR + 8 * i, 1);
+        for (int i = 0; i < kBarCount; ++i) {
+            int count = 1;
+            if (i >= kBarTileFree && i < kBarTileFree + kRing) count = 16;
+            else if ((i >= kBarKReady && i < kBarSFull) || (i >= kBarSFree && i < kBarVReady + 2) || i >= kBarTFree) count = 4;
+            mbar_init(bar(i), count);
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     for (int b = blockIdx.x; b < P.B; b += gridDim.x)
@@ -211,50 +240,57 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
     }
     __syncthreads();
     if ((int)blockIdx.x >= pt->blocks) return;             // more blocks than work (nothing allocated yet)
-    if (warp == kWorkerWarps) tmem_alloc(smem_u32(tmem_s), 512);
+    if (warp == kISS) tmem_alloc(smem_u32(tmem_s), 512);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_all = *tmem_s;
-    const uint32_t tb = tmem_all + team * kTeamCols;        // this team's columns (lane field zero)
-    const uint32_t my_lanes = (uint32_t)(32 * wq) << 16;    // worker: lanes of its subpartition
+    const uint32_t tb = *tmem_s;
+    const uint32_t my_lanes = (uint32_t)(32 * wq) << 16;    // lanes of this warp's subpartition
 
     int my_start, my_end;
     partition_range(pt, cum, hkv, P.B, blockIdx.x, my_start, my_end);
 
     bool failed = false;
-    const uint32_t bars = sbase + G::OFF_BAR + team * 256;  // slot barriers 0..15, S = 16, T0 = 17, T1 = 18
-    const uint32_t ring = sbase + team * 2 * kTile * G::SLOT;
-    const uint32_t ptiles = sbase + G::OFF_P + team * kTile * 512;
-    float* ps_s = reinterpret_cast<float*>(smem + G::OFF_PS) + team * kTile * 8;
-    int* list3 = reinterpret_cast<int*>(smem + G::OFF_LIST) + team * 2 * kRoundT;
-    int* list8 = list3 + kRoundT;
-    int* cnt = reinterpret_cast<int*>(smem + G::OFF_CNT) + team * 64;      // [0] n3, [1] n8, [4..7] flags, [8..39] maxima
     const float sc2 = P.scale * kLog2e;
-    uint32_t tcount = 0, scount = 0, tcnt0 = 0, tcnt1 = 0;   // tiles started, S and T completions waited for
+    uint32_t tcount = 0, bcount = 0;                         // tiles and value batches started so far (same in every warp)
 
-    auto wait_bar = [&](uint32_t bar, uint32_t parity) {     // bounded; on time-out flag the pool and carry on
-        if (failed || mbar_try_wait(bar, parity)) return;
-        unsigned long long t0, t1;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
-        int spins = 0;
-        while (!mbar_try_wait(bar, parity)) {
-            if ((++spins & 255) == 0) {
+    auto wait_bar = [&](int idx, uint32_t parity) {          // bounded; on time-out flag the pool and carry on
+        const uint32_t a = bar(idx);
+        if (failed || mbar_try_wait(a, parity)) return;
+        // a waiting warp must not eat the issue slots of the working ones: poll, then sleep a little, and
+        // look at the wall clock every 256 rounds
+        unsigned long long t0 = 0, t1;
+        for (int spins = 1;; ++spins) {
+            if (mbar_try_wait(a, parity)) return;
+            __nanosleep(spins < 4 ? 100 : 300);
+            if ((spins & 255) == 0) {
                 asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+                if (t0 == 0) t0 = t1;
                 if (t1 - t0 > 20000000ull) {
                     failed = true;
                     atomicOr(P.status, kStTimeout);
-                    break;
+                    return;
                 }
             }
         }
     };
+    // signal of a whole warp: its tensor-memory and shared-memory writes first, then one arrival
+    auto warp_arrive = [&](int idx) {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(idx));
+    };
+    auto wait_tile = [&](uint32_t t) {                       // all records of tile t are in its buffer
+        const uint32_t rb = t % kRing, par = (t / kRing) & 1;
+#pragma unroll 1
+        for (int s = 0; s < kTile; ++s) wait_bar(kBarFull + rb * kTile + s, par);
+    };
 
 #ifdef MKV_TIMELINE
-    unsigned long long tl_acc[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}, tl_last = tl_now(), tl_begin = tl_last;
-#define TM_STAMP(k) do { if (tid == 0) { const unsigned long long t__ = tl_now(); tl_acc[k] += t__ - tl_last; tl_last = t__; } } while (0)
+    long long tl_acc[4] = {0, 0, 0, 0}, tl_last = clock64();
+    const long long tl_begin = tl_last;
+#define TS(k) do { const long long t__ = clock64(); tl_acc[k] += t__ - tl_last; tl_last = t__; } while (0)
 #else
-#define TM_STAMP(k)
+#define TS(k)
 #endif
     int pos = my_start;
     int b = 0;
@@ -267,9 +303,7 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
         const int32_t* bt_row = P.bt + (size_t)b * P.max_pages;
         const uint8_t* tag_row = P.tags + (size_t)b * P.max_pages;
         const int stride = strides[b];
-        const int team_first = (int)(((unsigned)n_seg * (unsigned)team) / kTeams);
-        const int n_team = (int)(((unsigned)n_seg * (unsigned)(team + 1)) / kTeams) - team_first;
-        const int n_rounds = (n_team + kRoundT - 1) / kRoundT;
+        const int n_rounds = (n_seg + kRoundT - 1) / kRoundT;
         constexpr int EPL = D / 32;
         float qx[EPL];
 #pragma unroll
@@ -278,8 +312,8 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
         const uint8_t* tq3_base = P.tq3 + (size_t)h * G::TQ3_REC;
         const uint8_t* fp8_base = P.fp8 + (size_t)h * (2 * G::FP8_HALF);
 
-        // state of the team for this row (the same in all its worker threads): running maxima and row sums of
-        // the eight heads in log2 units; a worker thread's accumulators: channels (wq, lane) of the two halves
+        // softmax warps: running maxima of the eight heads (log2 units); scale warps: row sums and the accumulators
+        // of channels (wq, lane) of the two 128-channel halves
         float m_run[8], l_run[8], acc0[8], acc1[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) { m_run[i] = -CUDART_INF_F; l_run[i] = 0.f; acc0[i] = 0.f; acc1[i] = 0.f; }
@@ -329,210 +363,222 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
-        __syncthreads();
-        TM_STAMP(1);
 
         for (int round = 0; round < n_rounds; ++round) {
-            // ---- table entries of the round -> two id lists of the team ---------------------------------
-            if (worker) {
-                if (ttid == 0) { cnt[0] = 0; cnt[1] = 0; }
-                bar_sync(idW, 128);
-#pragma unroll 1
-                for (int k = 0; k < kRoundT / 128; ++k) {
-                    const int i = round * kRoundT + k * 128 + ttid;
-                    if (i < n_team) {
-                        const int pg = (int)(((unsigned)(pg0 + team_first + i) * (unsigned)stride) % (unsigned)n_pages);
-                        const int id = bt_row[pg], tag = tag_row[pg], valid = min(kPage, len - pg * kPage);
-                        int kind = 0;
-                        if (tag == MKV_TAG_STALE) kind = (id >= 0 && id < P.tq3_pages && valid == kPage) ? 1 : 0;
-                        else kind = (tag <= MKV_TAG_ANCHOR && id >= 0 && id < P.fp8_pages) ? 2 : 0;
-                        if (kind == 1) list3[atomicAdd(&cnt[0], 1)] = id;
-                        else if (kind == 2) list8[atomicAdd(&cnt[1], 1)] = id | ((valid & 15) << 27);
-                        else atomicOr(P.status, kStBounds);     // never dereferenced
-                    }
-                }
+            // ---- table entries of the round -> two id lists (all warps) ----------------------------------
+            if (tid == 0) { cnt[0] = 0; cnt[1] = 0; }
+            __syncthreads();
+            for (int i = round * kRoundT + tid; i < min(n_seg, (round + 1) * kRoundT); i += NT) {
+                const int pg = (int)(((unsigned)(pg0 + i) * (unsigned)stride) % (unsigned)n_pages);
+                const int id = bt_row[pg], tag = tag_row[pg], valid = min(kPage, len - pg * kPage);
+                int kind = 0;
+                if (tag == MKV_TAG_STALE) kind = (id >= 0 && id < P.tq3_pages && valid == kPage) ? 1 : 0;
+                else kind = (tag <= MKV_TAG_ANCHOR && id >= 0 && id < P.fp8_pages) ? 2 : 0;
+                if (kind == 1) list3[atomicAdd(&cnt[0], 1)] = id;
+                else if (kind == 2) list8[atomicAdd(&cnt[1], 1)] = id | ((valid & 15) << 27);
+                else atomicOr(P.status, kStBounds);     // never dereferenced
             }
-            bar_sync(idR, 160);                              // lists complete (workers and the issuing warp)
+            __syncthreads();                                 // lists (and, in the first round, the query tiles) complete
             const int n3 = cnt[0], n8 = cnt[1];
             const int tiles3 = (n3 + kTile - 1) / kTile, tiles8 = (n8 + kTile / 2 - 1) / (kTile / 2);
             const int n_tiles = tiles3 + tiles8;
-
-            // copies of tile ti into buffer `buf`: worker warp wq owns slots 2wq, 2wq + 1 (a Stale page each, or
-            // the key and the value half of one Recent/Anchor page); unused slots just complete their phase
-            auto issue_tile = [&](int ti, uint32_t buf) {
-                if (lane != 0) return;
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                const uint32_t s0 = 2 * wq, dst = ring + (buf * kTile + s0) * G::SLOT, bar0 = bars + 8 * (buf * kTile + s0);
-                if (ti < tiles3) {
-#pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        const int i = ti * kTile + s0 + e;
-                        if (i < n3) {
-                            mbar_expect_tx(bar0 + 8 * e, G::TQ3_REC);
-                            bulk_load(dst + e * G::SLOT, tq3_base + (size_t)list3[i] * hkv * G::TQ3_REC, G::TQ3_REC, bar0 + 8 * e);
-                        } else mbar_arrive(bar0 + 8 * e);
-                    }
-                } else {
-                    const int i = (ti - tiles3) * (kTile / 2) + wq;
-                    if (i < n8) {
-                        const uint8_t* rec = fp8_base + (size_t)(list8[i] & 0x7FFFFFF) * hkv * (2 * G::FP8_HALF);
-                        mbar_expect_tx(bar0, G::FP8_HALF);
-                        bulk_load(dst, rec, G::FP8_HALF, bar0);
-                        mbar_expect_tx(bar0 + 8, G::FP8_HALF);
-                        bulk_load(dst + G::SLOT, rec + G::FP8_HALF, G::FP8_HALF, bar0 + 8);
-                    } else { mbar_arrive(bar0); mbar_arrive(bar0 + 8); }
-                }
+            // tile ti of the round: format, first list entry, pages
+            auto tile_info = [&](int ti, bool& stale, int& first, int& np) {
+                stale = ti < tiles3;
+                first = stale ? ti * kTile : (ti - tiles3) * (kTile / 2);
+                np = stale ? min(kTile, n3 - first) : min(kTile / 2, n8 - first);
             };
 
-            if (!worker) {
-                // ================= issuing warp =================
+            if (warp == kPR) {
+                // ================= producer: records of a tile -> a tile buffer =================
+                if (lane == 0) {
+                    for (int ti = 0; ti < n_tiles; ++ti) {
+                        bool stale; int first, np;
+                        tile_info(ti, stale, first, np);
+                        const uint32_t t = tcount + ti, rb = t % kRing;
+                        TS(3);
+                        if (t >= kRing) wait_bar(kBarTileFree + rb, ((t / kRing) - 1) & 1);
+                        TS(0);
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        const uint32_t dst = sbase + rb * kTile * G::SLOT;
+                        for (int s = 0; s < kTile; ++s) {
+                            const uint32_t fb = bar(kBarFull + rb * kTile + s);
+                            if (stale) {
+                                if (s < np) {
+                                    mbar_expect_tx(fb, G::TQ3_REC);
+                                    bulk_load(dst + s * G::SLOT, tq3_base + (size_t)list3[first + s] * hkv * G::TQ3_REC, G::TQ3_REC, fb);
+                                } else mbar_arrive(fb);
+                            } else {
+                                if ((s >> 1) < np) {
+                                    const uint8_t* rec = fp8_base + (size_t)(list8[first + (s >> 1)] & 0x7FFFFFF) * hkv * (2 * G::FP8_HALF);
+                                    mbar_expect_tx(fb, G::FP8_HALF);
+                                    bulk_load(dst + s * G::SLOT, rec + (s & 1) * G::FP8_HALF, G::FP8_HALF, fb);
+                                } else mbar_arrive(fb);
+                            }
+                        }
+                    }
+                }
+                __syncwarp();
+            } else if (warp == kISS) {
+                // ================= score issue =================
                 for (int ti = 0; ti < n_tiles; ++ti) {
-                    const bool stale = ti < tiles3;
-                    const int np = stale ? min(kTile, n3 - ti * kTile) : min(kTile / 2, n8 - (ti - tiles3) * (kTile / 2));
-                    const uint32_t qtile = sbase + (stale ? G::OFF_QT : G::OFF_QF);
-                    bar_sync(idK, 160);                      // first half of the key tile stored
+                    bool stale; int first, np;
+                    tile_info(ti, stale, first, np);
+                    const uint32_t t = tcount + ti, kb2 = t & 1, par = (t >> 1) & 1;
+                    TS(3);
+                    wait_bar(kBarKReady + kb2, par);
+                    TS(0);
+                    if (t >= 2) wait_bar(kBarSFree + kb2, ((t >> 1) - 1) & 1);
+                    TS(1);
                     tc_fence_after();
                     if (lane == 0) {
+                        const uint32_t qtile = sbase + (stale ? G::OFF_QT : G::OFF_QF);
 #pragma unroll 1
-                        for (int kb = 0; kb < NB / 2; ++kb)
-                            mma_ts(tb + kColS, tb + kColK + 8 * kb, b_tile_desc(qtile + kb * 512), kIdesc, kb > 0);
+                        for (int kb = 0; kb < NB; ++kb)
+                            mma_ts(tb + kColS + 16 * kb2, tb + kColK + 8 * kb, b_tile_desc(qtile + kb * 512), kIdesc, kb > 0);
+                        mma_commit(bar(kBarSFull + kb2));
                     }
                     __syncwarp();
-                    bar_sync(idK2, 160);                     // second half
-                    tc_fence_after();
-                    if (lane == 0) {
-#pragma unroll 1
-                        for (int kb = NB / 2; kb < NB; ++kb)
-                            mma_ts(tb + kColS, tb + kColK + 8 * kb, b_tile_desc(qtile + kb * 512), kIdesc, 1);
-                        mma_commit(bars + 8 * 16);
-                    }
-                    __syncwarp();
+                }
+            } else if (warp == kISV) {
+                // ================= value issue =================
+                uint32_t bc = bcount;
+                for (int ti = 0; ti < n_tiles; ++ti) {
+                    bool stale; int first, np;
+                    tile_info(ti, stale, first, np);
+                    const uint32_t t = tcount + ti, pb = t & 1;
+                    TS(3);
+                    wait_bar(kBarPReady + pb, (t >> 1) & 1);
+                    TS(0);
                     const int nb = (np + 1) / 2;
-#pragma unroll 1
-                    for (int bi = 0; bi < nb; ++bi) {
-                        const uint32_t vb = bi & 1;
-                        bar_sync(idV0 + vb, 160);            // value tiles of the batch stored (and, for the first, all P tiles)
+                    for (int bi = 0; bi < nb; ++bi, ++bc) {
+                        const uint32_t vb = bc & 1, tbuf = bc % kTBuf;
+                        TS(3);
+                        wait_bar(kBarVReady + vb, (bc >> 1) & 1);
+                        TS(1);
+                        if (bc >= kTBuf) wait_bar(kBarTFree + tbuf, ((bc / kTBuf) - 1) & 1);
+                        TS(2);
                         tc_fence_after();
                         if (lane == 0) {
 #pragma unroll 1
                             for (int e = 0; e < 2; ++e) {
                                 const int p = 2 * bi + e;
                                 if (p >= np) break;
-                                const uint64_t dp = b_tile_desc(ptiles + p * 512);
+                                const uint64_t dp = b_tile_desc(sbase + G::OFF_P + (pb * kTile + p) * 512);
 #pragma unroll
                                 for (int m = 0; m < 2; ++m)
-                                    mma_ts(tb + kColT + vb * 64 + e * 32 + m * 16, tb + kColV + vb * 32 + e * 16 + m * 8, dp, kIdesc, 0);
+                                    mma_ts(tb + kColT + tbuf * 64 + e * 32 + m * 16, tb + kColV + vb * 32 + e * 16 + m * 8, dp, kIdesc, 0);
                             }
-                            mma_commit(bars + 8 * (17 + vb));
+                            mma_commit(bar(kBarTFull + tbuf));
                         }
                         __syncwarp();
                     }
                 }
-            } else {
-                // ================= worker warps =================
-                if (n_tiles > 0) issue_tile(0, tcount & 1);
+            } else if (warp < kSM) {
+                // ================= key unpack =================
                 for (int ti = 0; ti < n_tiles; ++ti) {
-                    const bool stale = ti < tiles3;
-                    const int first = stale ? ti * kTile : (ti - tiles3) * (kTile / 2);
-                    const int np = stale ? min(kTile, n3 - first) : min(kTile / 2, n8 - first);
-                    const uint32_t buf = tcount & 1, par = (tcount >> 1) & 1;
-                    ++tcount;
-                    const uint32_t tile = ring + buf * kTile * G::SLOT;
-                    // every worker of the team has finished the tile before: the other buffer can be refilled now
-                    bar_sync(idW, 128);
-                    if (ti + 1 < n_tiles) issue_tile(ti + 1, tcount & 1);
+                    bool stale; int first, np;
+                    tile_info(ti, stale, first, np);
+                    const uint32_t t = tcount + ti, rb = t % kRing, kb2 = t & 1;
+                    const uint32_t tile = sbase + rb * kTile * G::SLOT;
+                    TS(3);
+                    wait_tile(t);
+                    TS(0);
+                    if (t >= 1) wait_bar(kBarSFull + ((t - 1) & 1), ((t - 1) >> 1) & 1);      // the score products of the tile before have read it
+                    TS(1);
+                    tc_fence_after();
 #pragma unroll 1
-                    for (int s = 0; s < kTile; ++s) wait_bar(bars + 8 * (buf * kTile + s), par);
-                    failed = __any_sync(FULL, failed);
-                    TM_STAMP(2);
-
-                    // ---- keys of this warp's two pages -> tensor memory, in two halves of d ---------------------
+                    for (int e = 0; e < 2; ++e) {
+                        const int p = 2 * wq + e;
+                        if (p >= np) continue;
+                        const uint32_t dst = tb + kColK + my_lanes + ((uint32_t)(16 * e) << 16);
+                        if (stale) {
+                            const uint32_t sec = tile + p * G::SLOT + lane * 16;
 #pragma unroll 1
-                    for (int half = 0; half < 2; ++half) {
-#pragma unroll 1
-                        for (int e = 0; e < 2; ++e) {
-                            const int p = 2 * wq + e;
-                            if (p >= np) continue;
-                            const uint32_t dst = tb + kColK + my_lanes + ((uint32_t)(16 * e) << 16) + 64 * half;
-                            if (stale) {
-                                // words 6 half .. 6 half + 5 of the lane: two 16-byte chunks (the second half starts mid-chunk)
-                                const uint32_t sec = tile + p * G::SLOT + lane * 16;
-                                const uint4 c0 = lds128(sec + (half ? 512 : 0)), c1 = lds128(sec + (half ? 1024 : 512));
-                                const uint32_t kw[6] = {half ? c0.z : c0.x, half ? c0.w : c0.y, half ? c1.x : c0.z,
-                                                        half ? c1.y : c0.w, half ? c1.z : c1.x, half ? c1.w : c1.y};
+                            for (int j = 0; j < NB / 4; ++j) {
+                                // words 3j, 3j+1, 3j+2 of the lane (word i sits in chunk i / 4 at byte 4 (i % 4))
+                                uint32_t A, Bw, Cw;
+                                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(A) : "r"(sec + ((3 * j) >> 2) * 512 + ((3 * j) & 3) * 4));
+                                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(Bw) : "r"(sec + ((3 * j + 1) >> 2) * 512 + ((3 * j + 1) & 3) * 4));
+                                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(Cw) : "r"(sec + ((3 * j + 2) >> 2) * 512 + ((3 * j + 2) & 3) * 4));
+                                uint32_t sel[4], r[16];
+                                sel[0] = A & 0x77777777u;
+                                sel[1] = Bw & 0x77777777u;
+                                sel[2] = lop3_and_or(A >> 1, 0x44444444u, Cw & 0x33333333u);
+                                sel[3] = lop3_and_or(Bw >> 1, 0x44444444u, (Cw >> 2) & 0x33333333u);
 #pragma unroll
-                                for (int j = 0; j < 2; ++j) {
-                                    const uint32_t A = kw[3 * j], Bw = kw[3 * j + 1], Cw = kw[3 * j + 2];
-                                    uint32_t sel[4], r[16];
-                                    sel[0] = A & 0x77777777u;
-                                    sel[1] = Bw & 0x77777777u;
-                                    sel[2] = lop3_and_or(A >> 1, 0x44444444u, Cw & 0x33333333u);
-                                    sel[3] = lop3_and_or(Bw >> 1, 0x44444444u, (Cw >> 2) & 0x33333333u);
-#pragma unroll
-                                    for (int w = 0; w < 4; ++w) {
-                                        uint32_t a0, a1, a2, a3;
-                                        key_lut4(sel[w], a0, a1);
-                                        key_lut4(sel[w] >> 16, a2, a3);
-                                        r[4 * w] = a0; r[4 * w + 1] = a2; r[4 * w + 2] = a1; r[4 * w + 3] = a3;
-                                    }
-                                    tmem_st_frag4(dst + 32 * j, r);
+                                for (int w = 0; w < 4; ++w) {
+                                    uint32_t a0, a1, a2, a3;
+                                    key_lut4(sel[w], a0, a1);
+                                    key_lut4(sel[w] >> 16, a2, a3);
+                                    r[4 * w] = a0; r[4 * w + 1] = a2; r[4 * w + 2] = a1; r[4 * w + 3] = a3;
                                 }
-                            } else {
-                                const uint32_t kaddr = tile + 2 * p * G::SLOT;
+                                tmem_st_frag4(dst + 32 * j, r);
+                            }
+                        } else {
+                            const uint32_t kaddr = tile + 2 * p * G::SLOT;
+#pragma unroll 1
+                            for (int j = 0; j < D / 64; ++j) {
+                                const uint4 r0 = lds128(kaddr + g * D + 64 * j + 16 * tq);
+                                const uint4 r1 = lds128(kaddr + (g + 8) * D + 64 * j + 16 * tq);
+                                const uint32_t w0[4] = {r0.x, r0.y, r0.z, r0.w}, w1[4] = {r1.x, r1.y, r1.z, r1.w};
+                                uint32_t r[16];
 #pragma unroll
-                                for (int jj = 0; jj < 2; ++jj) {
-                                    const int j = 2 * half + jj;
-                                    const uint4 r0 = lds128(kaddr + g * D + 64 * j + 16 * tq);
-                                    const uint4 r1 = lds128(kaddr + (g + 8) * D + 64 * j + 16 * tq);
-                                    const uint32_t w0[4] = {r0.x, r0.y, r0.z, r0.w}, w1[4] = {r1.x, r1.y, r1.z, r1.w};
-                                    uint32_t r[16];
-#pragma unroll
-                                    for (int w = 0; w < 4; ++w) {
-                                        r[4 * w] = e4m3x2_to_f16x2((uint16_t)(w0[w] & 0xFFFFu));
-                                        r[4 * w + 1] = e4m3x2_to_f16x2((uint16_t)(w0[w] >> 16));
-                                        r[4 * w + 2] = e4m3x2_to_f16x2((uint16_t)(w1[w] & 0xFFFFu));
-                                        r[4 * w + 3] = e4m3x2_to_f16x2((uint16_t)(w1[w] >> 16));
-                                    }
-                                    tmem_st_frag4(dst + 32 * jj, r);
+                                for (int w = 0; w < 4; ++w) {
+                                    r[4 * w] = e4m3x2_to_f16x2((uint16_t)(w0[w] & 0xFFFFu));
+                                    r[4 * w + 1] = e4m3x2_to_f16x2((uint16_t)(w0[w] >> 16));
+                                    r[4 * w + 2] = e4m3x2_to_f16x2((uint16_t)(w1[w] & 0xFFFFu));
+                                    r[4 * w + 3] = e4m3x2_to_f16x2((uint16_t)(w1[w] >> 16));
                                 }
+                                tmem_st_frag4(dst + 32 * j, r);
                             }
                         }
-                        tmem_wait_st();
-                        tc_fence_before();
-                        bar_arrive(half ? idK2 : idK, 160);
                     }
-                    TM_STAMP(3);
-
-                    // ---- scores of this thread's token -------------------------------------------------------
+                    tmem_wait_st();
+                    tc_fence_before();
+                    warp_arrive(kBarKReady + kb2);
+                    warp_arrive(kBarTileFree + rb);
+                }
+            } else if (warp < kVU) {
+                // ================= softmax =================
+                for (int ti = 0; ti < n_tiles; ++ti) {
+                    bool stale; int first, np;
+                    tile_info(ti, stale, first, np);
+                    const uint32_t t = tcount + ti, rb = t % kRing, sb = t & 1, par = (t >> 1) & 1;
+                    const uint32_t tile = sbase + rb * kTile * G::SLOT;
                     const int p_me = 2 * wq + (lane >> 4), tok = lane & 15;
                     int valid = kPage;
                     if (!stale && p_me < np) { const int v = (list8[first + p_me] >> 27) & 15; valid = v ? v : kPage; }
                     const bool live = p_me < np && tok < valid;
-                    wait_bar(bars + 8 * 16, scount & 1);
-                    ++scount;
-                    failed = __any_sync(FULL, failed);
-                    TM_STAMP(4);
+                    TS(3);
+                    wait_tile(t);
+                    TS(0);
+                    float rsc = sc2 * P.k_scale;
+                    if (stale) rsc = __half2float(__ushort_as_half(lds16(tile + (p_me < np ? p_me : 0) * G::SLOT + 12 * D + 2 * tok))) * sc2;
+                    warp_arrive(kBarTileFree + rb);
+                    wait_bar(kBarSFull + sb, par);
+                    TS(1);
                     tc_fence_after();
                     float s[8];
                     {
                         float c[16];
-                        tmem_ld16(tb + kColS + my_lanes, c);
+                        tmem_ld16(tb + kColS + 16 * sb + my_lanes, c);
                         tmem_wait_ld();
-                        float rsc = sc2 * P.k_scale;
-                        if (stale) {
-                            const uint32_t gaddr = tile + (p_me < np ? p_me : 0) * G::SLOT + 12 * D;
-                            rsc = __half2float(__ushort_as_half(lds16(gaddr + 2 * tok))) * sc2;
-                        }
+                        tc_fence_before();
+                        warp_arrive(kBarSFree + sb);
 #pragma unroll
                         for (int i = 0; i < 8; ++i) s[i] = live ? (c[i] + c[8 + i]) * rsc : -CUDART_INF_F;
                     }
-                    // running maxima: raised (for the whole team) only when some score exceeds them by 2^kRescaleSlack
+                    // running maxima: raised only when some score of the tile exceeds them by 2^kRescaleSlack
+                    float fs[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) fs[i] = 1.f;
                     bool ex = false;
 #pragma unroll
                     for (int i = 0; i < 8; ++i) ex = ex || (s[i] > m_run[i] + kRescaleSlack);
                     ex = __any_sync(FULL, ex);
                     if (lane == 0) cnt[4 + wq] = ex ? 1 : 0;
-                    bar_sync(idW, 128);
+                    bar_sync(1, 128);
                     if (cnt[4] | cnt[5] | cnt[6] | cnt[7]) {
                         float mx[8];
 #pragma unroll
@@ -548,25 +594,26 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
                             for (int i = 1; i < 8; ++i) v = lane == i ? mx[i] : v;
                             reinterpret_cast<float*>(cnt)[8 + wq * 8 + lane] = v;
                         }
-                        bar_sync(idW, 128);
+                        bar_sync(1, 128);
 #pragma unroll
                         for (int i = 0; i < 8; ++i) {
                             const float* q4 = reinterpret_cast<const float*>(cnt) + 8 + i;
                             const float nm = fmaxf(fmaxf(q4[0], q4[8]), fmaxf(q4[16], q4[24]));
                             if (nm > m_run[i] + kRescaleSlack) {
-                                const float f = m_run[i] == -CUDART_INF_F ? 0.f : fast_exp2(m_run[i] - nm);
+                                fs[i] = m_run[i] == -CUDART_INF_F ? 0.f : fast_exp2(m_run[i] - nm);
                                 m_run[i] = nm;
-                                l_run[i] *= f;
-                                acc0[i] *= f;
-                                acc1[i] *= f;
                             }
                         }
-                        bar_sync(idW, 128);                  // the maxima are read before the next tile overwrites them
                     }
-                    // probabilities of this token -> B tile of its page (rows 0-7 high, 8-15 low fp16 halves), page sums
+                    bar_sync(1, 128);                        // flags and maxima are read; they may be rewritten for the next tile
+                    // the tile's P tiles, page sums and rescale factors go to set sb once the scale warps are done with it
+                    TS(3);
+                    if (t >= 2) wait_bar(kBarSCDone + sb, ((t >> 1) - 1) & 1);
+                    TS(2);
+                    float* ps_s = ps_all + sb * (kTile + 1) * 8;
                     {
                         const int kk = stale ? k_of_token_tq3(tok) : tok;
-                        const uint32_t tp = ptiles + (p_me & (kTile - 1)) * 512;
+                        const uint32_t tp = sbase + G::OFF_P + (sb * kTile + (p_me & (kTile - 1))) * 512;
                         float pv[8];
 #pragma unroll
                         for (int i = 0; i < 8; ++i) {
@@ -588,53 +635,32 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
                             *reinterpret_cast<float4*>(ps_s + p_me * 8) = make_float4(pv[0], pv[1], pv[2], pv[3]);
                             *reinterpret_cast<float4*>(ps_s + p_me * 8 + 4) = make_float4(pv[4], pv[5], pv[6], pv[7]);
                         }
+                        if (warp == kSM && lane == 0) {
+                            *reinterpret_cast<float4*>(ps_s + kTile * 8) = make_float4(fs[0], fs[1], fs[2], fs[3]);
+                            *reinterpret_cast<float4*>(ps_s + kTile * 8 + 4) = make_float4(fs[4], fs[5], fs[6], fs[7]);
+                        }
                         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     }
-                    bar_sync(idW, 128);                      // page sums and P tiles of all four warps are in place
-                    TM_STAMP(5);
-
-                    // ---- values: two pages at a time; the products of a batch run while the next one is unpacked -----
-                    auto scale_batch = [&](int bi) {
-                        const uint32_t vb = bi & 1;
-                        TM_STAMP(6);
-                        if (vb) { wait_bar(bars + 8 * 18, tcnt1 & 1); ++tcnt1; } else { wait_bar(bars + 8 * 17, tcnt0 & 1); ++tcnt0; }
-                        TM_STAMP(7);
-                        tc_fence_after();
-#pragma unroll 1
-                        for (int e = 0; e < 2; ++e) {
-                            const int p = 2 * bi + e;
-                            if (p >= np) break;
-                            float t0[16], t1[16];
-                            tmem_ld16(tb + kColT + vb * 64 + e * 32 + my_lanes, t0);
-                            tmem_ld16(tb + kColT + vb * 64 + e * 32 + 16 + my_lanes, t1);
-                            tmem_wait_ld();
-                            const float4 pa = *reinterpret_cast<const float4*>(ps_s + p * 8), pb = *reinterpret_cast<const float4*>(ps_s + p * 8 + 4);
-                            const float ps[8] = {pa.x, pa.y, pa.z, pa.w, pb.x, pb.y, pb.z, pb.w};
-                            float sc0 = P.v_scale, zp0 = 0.f, sc1 = P.v_scale, zp1 = 0.f;
-                            if (stale) {
-                                // channel 16 cb + row: halves (scale, zero) at ((cb/2) 64 + (row%8) 8 + 4 (cb%2) + row/8) and + 2
-                                const uint32_t meta = tile + p * G::SLOT + 12 * D + 32;
-                                const int row = lane & 15, cb0 = 4 * wq + (lane >> 4), cb1 = cb0 + 2;
-                                const uint32_t i0 = (cb0 >> 1) * 64 + (row & 7) * 8 + 4 * (cb0 & 1) + (row >> 3);
-                                const uint32_t i1 = (cb1 >> 1) * 64 + (row & 7) * 8 + 4 * (cb1 & 1) + (row >> 3);
-                                sc0 = __half2float(__ushort_as_half(lds16(meta + 2 * i0)));
-                                zp0 = __half2float(__ushort_as_half(lds16(meta + 2 * i0 + 4)));
-                                sc1 = __half2float(__ushort_as_half(lds16(meta + 2 * i1)));
-                                zp1 = __half2float(__ushort_as_half(lds16(meta + 2 * i1 + 4)));
-                            }
-#pragma unroll
-                            for (int i = 0; i < 8; ++i) {
-                                acc0[i] = fmaf(sc0, t0[i] + t0[8 + i], fmaf(zp0, ps[i], acc0[i]));
-                                acc1[i] = fmaf(sc1, t1[i] + t1[8 + i], fmaf(zp1, ps[i], acc1[i]));
-                                l_run[i] += ps[i];
-                            }
-                        }
-                        TM_STAMP(8);
-                    };
+                    warp_arrive(kBarPReady + sb);
+                }
+            } else if (warp < kSC) {
+                // ================= value unpack =================
+                uint32_t bc = bcount;
+                for (int ti = 0; ti < n_tiles; ++ti) {
+                    bool stale; int first, np;
+                    tile_info(ti, stale, first, np);
+                    const uint32_t t = tcount + ti, rb = t % kRing;
+                    const uint32_t tile = sbase + rb * kTile * G::SLOT;
+                    TS(2);
+                    wait_tile(t);
+                    TS(0);
                     const int nb = (np + 1) / 2;
-#pragma unroll 1
-                    for (int bi = 0; bi < nb; ++bi) {
-                        const uint32_t vb = bi & 1;
+                    for (int bi = 0; bi < nb; ++bi, ++bc) {
+                        const uint32_t vb = bc & 1;
+                        TS(2);
+                        if (bc >= 2) wait_bar(kBarTFull + (bc - 2) % kTBuf, ((bc - 2) / kTBuf) & 1);     // the products of the batch before last have read it
+                        TS(1);
+                        tc_fence_after();
 #pragma unroll 1
                         for (int e = 0; e < 2; ++e) {
                             const int p = 2 * bi + e;
@@ -672,46 +698,104 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
                                 }
                             }
                         }
+                        TS(3);
                         tmem_wait_st();
                         tc_fence_before();
-                        bar_arrive(idV0 + vb, 160);
-                        if (bi > 0) scale_batch(bi - 1);
+                        warp_arrive(kBarVReady + vb);
                     }
-                    if (nb > 0) scale_batch(nb - 1);
-                    failed = __any_sync(FULL, failed);
+                    warp_arrive(kBarTileFree + rb);
+                }
+            } else {
+                // ================= scale =================
+                uint32_t bc = bcount;
+                for (int ti = 0; ti < n_tiles; ++ti) {
+                    bool stale; int first, np;
+                    tile_info(ti, stale, first, np);
+                    const uint32_t t = tcount + ti, rb = t % kRing, pb = t & 1;
+                    const uint32_t tile = sbase + rb * kTile * G::SLOT;
+                    const float* ps_s = ps_all + pb * (kTile + 1) * 8;
+                    TS(3);
+                    wait_tile(t);
+                    wait_bar(kBarPReady + pb, (t >> 1) & 1);
+                    TS(0);
+                    {
+                        const float4 fa = *reinterpret_cast<const float4*>(ps_s + kTile * 8), fb = *reinterpret_cast<const float4*>(ps_s + kTile * 8 + 4);
+                        const float fsc[8] = {fa.x, fa.y, fa.z, fa.w, fb.x, fb.y, fb.z, fb.w};
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) { l_run[i] *= fsc[i]; acc0[i] *= fsc[i]; acc1[i] *= fsc[i]; }
+                    }
+                    const int nb = (np + 1) / 2;
+                    for (int bi = 0; bi < nb; ++bi, ++bc) {
+                        const uint32_t vb = bc % kTBuf;
+                        TS(3);
+                        wait_bar(kBarTFull + vb, (bc / kTBuf) & 1);
+                        TS(1);
+                        tc_fence_after();
+                        const int pn = min(2, np - 2 * bi);
+#pragma unroll 1
+                        for (int e = 0; e < pn; ++e) {
+                            float t0[16], t1[16];
+                            tmem_ld16(tb + kColT + vb * 64 + e * 32 + my_lanes, t0);
+                            tmem_ld16(tb + kColT + vb * 64 + e * 32 + 16 + my_lanes, t1);
+                            tmem_wait_ld();
+                            if (e == pn - 1) {
+                                tc_fence_before();
+                                warp_arrive(kBarTFree + vb);
+                            }
+                            const int p = 2 * bi + e;
+                            const float4 pa = *reinterpret_cast<const float4*>(ps_s + p * 8), pbv = *reinterpret_cast<const float4*>(ps_s + p * 8 + 4);
+                            const float ps[8] = {pa.x, pa.y, pa.z, pa.w, pbv.x, pbv.y, pbv.z, pbv.w};
+                            float sc0 = P.v_scale, zp0 = 0.f, sc1 = P.v_scale, zp1 = 0.f;
+                            if (stale) {
+                                // channel 16 cb + row: halves (scale, zero) at ((cb/2) 64 + (row%8) 8 + 4 (cb%2) + row/8) and + 2
+                                const uint32_t meta = tile + p * G::SLOT + 12 * D + 32;
+                                const int row = lane & 15, cb0 = 4 * wq + (lane >> 4), cb1 = cb0 + 2;
+                                const uint32_t i0 = (cb0 >> 1) * 64 + (row & 7) * 8 + 4 * (cb0 & 1) + (row >> 3);
+                                const uint32_t i1 = (cb1 >> 1) * 64 + (row & 7) * 8 + 4 * (cb1 & 1) + (row >> 3);
+                                sc0 = __half2float(__ushort_as_half(lds16(meta + 2 * i0)));
+                                zp0 = __half2float(__ushort_as_half(lds16(meta + 2 * i0 + 4)));
+                                sc1 = __half2float(__ushort_as_half(lds16(meta + 2 * i1)));
+                                zp1 = __half2float(__ushort_as_half(lds16(meta + 2 * i1 + 4)));
+                            }
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                acc0[i] = fmaf(sc0, t0[i] + t0[8 + i], fmaf(zp0, ps[i], acc0[i]));
+                                acc1[i] = fmaf(sc1, t1[i] + t1[8 + i], fmaf(zp1, ps[i], acc1[i]));
+                                l_run[i] += ps[i];
+                            }
+                        }
+                        TS(2);
+                    }
+                    warp_arrive(kBarTileFree + rb);
+                    warp_arrive(kBarSCDone + pb);
                 }
             }
-            bar_sync(idR, 160);                              // round finished: lists and counters may be rewritten
+            // every warp advances the counters by what the round held
+            for (int ti = 0; ti < n_tiles; ++ti) {
+                bool stale; int first, np;
+                tile_info(ti, stale, first, np);
+                bcount += (np + 1) / 2;
+            }
+            tcount += n_tiles;
+            failed = __any_sync(FULL, failed);
         }
 
-        // ---- combine the teams of the block (ring memory is idle now) -------------------------------------
-        TM_STAMP(9);
+        // ---- results of the row (ring memory is idle now) ------------------------------------------------
         tc_fence_before();
         __syncthreads();
-        TM_STAMP(10);
-        if (worker && ttid == 0) {
+        if (warp == kSM && lane == 0) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) sm_m[team * 8 + i] = m_run[i];
+            for (int i = 0; i < 8; ++i) sm_m[i] = m_run[i];
         }
-        __syncthreads();
-        if (worker) {
+        if (warp >= kSC && warp < kISS) {
             const int c0 = 16 * (4 * wq + (lane >> 4)) + (lane & 15), c1 = c0 + 32;
-            float f[8];
+            *reinterpret_cast<float4*>(red + c0 * 8) = make_float4(acc0[0], acc0[1], acc0[2], acc0[3]);
+            *reinterpret_cast<float4*>(red + c0 * 8 + 4) = make_float4(acc0[4], acc0[5], acc0[6], acc0[7]);
+            *reinterpret_cast<float4*>(red + c1 * 8) = make_float4(acc1[0], acc1[1], acc1[2], acc1[3]);
+            *reinterpret_cast<float4*>(red + c1 * 8 + 4) = make_float4(acc1[4], acc1[5], acc1[6], acc1[7]);
+            if (warp == kSC && lane == 0) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                float M = -CUDART_INF_F;
-#pragma unroll
-                for (int u = 0; u < NU; ++u) M = fmaxf(M, sm_m[u * 8 + i]);
-                f[i] = m_run[i] == -CUDART_INF_F ? 0.f : fast_exp2(m_run[i] - M);
-            }
-            float* mine = red + (size_t)team * D * 8;
-            *reinterpret_cast<float4*>(mine + c0 * 8) = make_float4(acc0[0] * f[0], acc0[1] * f[1], acc0[2] * f[2], acc0[3] * f[3]);
-            *reinterpret_cast<float4*>(mine + c0 * 8 + 4) = make_float4(acc0[4] * f[4], acc0[5] * f[5], acc0[6] * f[6], acc0[7] * f[7]);
-            *reinterpret_cast<float4*>(mine + c1 * 8) = make_float4(acc1[0] * f[0], acc1[1] * f[1], acc1[2] * f[2], acc1[3] * f[3]);
-            *reinterpret_cast<float4*>(mine + c1 * 8 + 4) = make_float4(acc1[4] * f[4], acc1[5] * f[5], acc1[6] * f[6], acc1[7] * f[7]);
-            if (ttid == 0) {
-#pragma unroll
-                for (int i = 0; i < 8; ++i) sm_l[team * 8 + i] = l_run[i] * f[i];
+                for (int i = 0; i < 8; ++i) sm_l[i] = l_run[i];
             }
         }
         __syncthreads();
@@ -721,38 +805,17 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
             for (int e = tid; e < 8 * D; e += NT) {
                 const int head = e & 7, ch = e >> 3;
                 if (head >= GQ) continue;
-                float acc = 0.f, l = 0.f;
-#pragma unroll
-                for (int u = 0; u < NU; ++u) {
-                    acc += red[(size_t)u * D * 8 + e];
-                    l += sm_l[u * 8 + head];
-                }
-                P.out[((size_t)b * hq + h * GQ + head) * D + ch] = l > 0.f ? acc / l : 0.f;
+                const float l = sm_l[head];
+                P.out[((size_t)b * hq + h * GQ + head) * D + ch] = l > 0.f ? red[e] / l : 0.f;
             }
-            if (P.lse && tid < GQ) {
-                float l = 0.f, M = -CUDART_INF_F;
-                for (int u = 0; u < NU; ++u) {
-                    l += sm_l[u * 8 + tid];
-                    M = fmaxf(M, sm_m[u * 8 + tid]);
-                }
-                P.lse[(size_t)b * hq + h * GQ + tid] = l > 0.f ? (M + log2f(l)) * kLn2 : -CUDART_INF_F;
-            }
+            if (P.lse && tid < GQ)
+                P.lse[(size_t)b * hq + h * GQ + tid] = sm_l[tid] > 0.f ? (sm_m[tid] + log2f(sm_l[tid])) * kLn2 : -CUDART_INF_F;
         } else {
             float* slot = P.partials + (size_t)(2 * blockIdx.x + (pos != my_start ? 1 : 0)) * (8 * D + 16);
-            for (int e = tid; e < 8 * D; e += NT) {
-                float acc = 0.f;
-#pragma unroll
-                for (int u = 0; u < NU; ++u) acc += red[(size_t)u * D * 8 + e];
-                slot[e] = acc;
-            }
+            for (int e = tid; e < 8 * D; e += NT) slot[e] = red[e];
             if (tid < 8) {
-                float l = 0.f, M = -CUDART_INF_F;
-                for (int u = 0; u < NU; ++u) {
-                    l += sm_l[u * 8 + tid];
-                    M = fmaxf(M, sm_m[u * 8 + tid]);
-                }
-                slot[8 * D + tid] = M;
-                slot[8 * D + 8 + tid] = l;
+                slot[8 * D + tid] = sm_m[tid];
+                slot[8 * D + 8 + tid] = sm_l[tid];
             }
             int c0, c1;
             partition_blocks_of_row(pt, cum, P.B, b * hkv + h, row_start, row_end, c0, c1);
@@ -769,22 +832,22 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
             if (*last_s) {
                 __threadfence();
                 const int first_slot = 2 * c0 + (row_start > partition_start(pt, cum, hkv, P.B, c0) ? 1 : 0);
-                merge_row<D, NT>(P, first_slot, 2 * c0, n_parts, red, b, h);
+                merge_row<D, NT, 16>(P, first_slot, 2 * c0, n_parts, red, b, h);
             }
         }
         __syncthreads();
-        TM_STAMP(11);
         pos += n_seg;
     }
 #ifdef MKV_TIMELINE
-    if (tid == 0) {
-        for (int k = 0; k < 12; ++k) g_timeline[blockIdx.x * 16 + k] = tl_acc[k];
-        g_timeline[blockIdx.x * 16 + 15] = tl_begin;
-        g_timeline[blockIdx.x * 16 + 14] = tl_now();
+    TS(3);
+    if (lane == 0 && wq == 0 || warp >= kISS && lane == 0) {
+        const int role = warp >= kISS ? 4 + (warp - kISS) : warp >> 2;
+        for (int k = 0; k < 4; ++k) g_warp_end[blockIdx.x * 32 + role * 4 + k] = tl_acc[k];
+        if (warp == 0) g_warp_end[blockIdx.x * 32 + 31] = clock64() - tl_begin;
     }
 #endif
     tc_fence_before();
     __syncthreads();
-    if (warp == kWorkerWarps) tmem_dealloc(tmem_all, 512);
+    if (warp == kISS) tmem_dealloc(tb, 512);
 }
-#undef TM_STAMP
+#undef TS
