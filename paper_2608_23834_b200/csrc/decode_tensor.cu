@@ -227,7 +227,7 @@ __device__ __forceinline__ void affine_accumulate(float (&acc)[4], const float (
 }
 
 // ------------------------------------------------------------------------------------------------
-// Work partition, shared by the scan and the merge kernel
+// Work partition (the scan and the merge of split rows use the same cut)
 // ------------------------------------------------------------------------------------------------
 // Work = (request, KV head, page) triples in row-major order; cum[b] = index of the first triple of
 // request b.  Two ways to cut it into one contiguous range per block:
