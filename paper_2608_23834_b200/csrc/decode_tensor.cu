@@ -413,13 +413,14 @@ __device__ __forceinline__ void softmax_page(WarpAcc<NB>& acc, const float (&s)[
 {
     constexpr uint32_t FULL = 0xffffffffu;
     float mx0 = fmaxf(s[0], s[2]), mx1 = fmaxf(s[1], s[3]);
+    // the page maximum is only needed when some score exceeds the running maximum by more than the slack
+    if (__any_sync(FULL, mx0 > acc.m[0] + kRescaleSlack || mx1 > acc.m[1] + kRescaleSlack)) {
 #pragma unroll
-    for (int o = 4; o < 32; o <<= 1) {
-        mx0 = fmaxf(mx0, __shfl_xor_sync(FULL, mx0, o));
-        mx1 = fmaxf(mx1, __shfl_xor_sync(FULL, mx1, o));
-    }
-    const bool up0 = mx0 > acc.m[0] + kRescaleSlack, up1 = mx1 > acc.m[1] + kRescaleSlack;
-    if (__any_sync(FULL, up0 || up1)) {
+        for (int o = 4; o < 32; o <<= 1) {
+            mx0 = fmaxf(mx0, __shfl_xor_sync(FULL, mx0, o));
+            mx1 = fmaxf(mx1, __shfl_xor_sync(FULL, mx1, o));
+        }
+        const bool up0 = mx0 > acc.m[0] + kRescaleSlack, up1 = mx1 > acc.m[1] + kRescaleSlack;
         const float f0 = up0 ? fast_exp2(acc.m[0] - mx0) : 1.f, f1 = up1 ? fast_exp2(acc.m[1] - mx1) : 1.f;
         if (up0) acc.m[0] = mx0;
         if (up1) acc.m[1] = mx1;
