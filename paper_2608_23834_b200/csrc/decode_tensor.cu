@@ -408,8 +408,9 @@ struct PFrag {
     float ps0, ps1;
 };
 
+// First half: raise the running maximum (and rescale the accumulators) if the page asks for it.
 template <int NB>
-__device__ __forceinline__ void softmax_page(WarpAcc<NB>& acc, const float (&s)[4], PFrag& pf)
+__device__ __forceinline__ void softmax_rescale(WarpAcc<NB>& acc, const float (&s)[4])
 {
     constexpr uint32_t FULL = 0xffffffffu;
     float mx0 = fmaxf(s[0], s[2]), mx1 = fmaxf(s[1], s[3]);
@@ -432,6 +433,12 @@ __device__ __forceinline__ void softmax_page(WarpAcc<NB>& acc, const float (&s)[
         acc.l[0] *= f0;
         acc.l[1] *= f1;
     }
+}
+
+// Second half, branch-free (so that it can be scheduled into the unpack work of the next page): P and its row sums.
+template <int NB>
+__device__ __forceinline__ void softmax_probs(WarpAcc<NB>& acc, const float (&s)[4], PFrag& pf)
+{
     const float p0 = fast_exp2(s[0] - acc.m[0]), p1 = fast_exp2(s[1] - acc.m[1]);
     const float p2 = fast_exp2(s[2] - acc.m[0]), p3 = fast_exp2(s[3] - acc.m[1]);
     const uint32_t ph01 = pack_f16x2(p0, p1), ph23 = pack_f16x2(p2, p3);
@@ -449,6 +456,13 @@ __device__ __forceinline__ void softmax_page(WarpAcc<NB>& acc, const float (&s)[
     pf.ps1 = ps[1];
     acc.l[0] += ps[0];
     acc.l[1] += ps[1];
+}
+
+template <int NB>
+__device__ __forceinline__ void softmax_page(WarpAcc<NB>& acc, const float (&s)[4], PFrag& pf)
+{
+    softmax_rescale<NB>(acc, s);
+    softmax_probs<NB>(acc, s, pf);
 }
 
 // Scored variant (Section 3.1): log2 of the page's exponential sum, referred to an absolute origin
@@ -553,7 +567,7 @@ __device__ __forceinline__ void tq3_value_quad(float (&o0)[4], float (&o1)[4], f
 // one instruction stream, so that table lookups, half-precision FMAs, fp32 FMAs and MMAs of the two
 // phases overlap.  DO_V / DO_K switch the halves off for the first and the last page.
 template <int D, bool DO_V, bool DO_K>
-__device__ __forceinline__ void tq3_step(WarpAcc<D / 16>& acc, uint32_t rec_v, const PFrag& pf, uint32_t rec_k,
+__device__ __forceinline__ void tq3_step(WarpAcc<D / 16>& acc, uint32_t rec_v, const float (&s_cur)[4], PFrag& pf, uint32_t rec_k,
                                          uint32_t qt_lane, float sc2, int lane, float (&s_next)[4])
 {
     constexpr int NB = D / 16, LW = 3 * NB / 4;
@@ -562,6 +576,7 @@ __device__ __forceinline__ void tq3_step(WarpAcc<D / 16>& acc, uint32_t rec_v, c
     float S0[4] = {0.f, 0.f, 0.f, 0.f}, S1[4] = {0.f, 0.f, 0.f, 0.f};
     if constexpr (DO_K) load_lane_words<D>(rec_k, lane, kw);
     if constexpr (DO_V) load_lane_words<D>(rec_v + 6 * D, lane, vw);
+    if constexpr (DO_V) softmax_probs<NB>(acc, s_cur, pf);     // in one block with the key unpack of the next page
     const uint32_t meta = rec_v + 12 * D + 32 + g * 16;
 #pragma unroll
     for (int j = 0; j < NB / 4; ++j) {
@@ -1032,23 +1047,23 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                 float s_cur[4], s_next[4];
                 PFrag pf;
                 wait_slot(0);
-                if (!failed) tq3_step<D, false, true>(acc, 0, pf, ring, qt_lane, sc2, lane, s_cur);
+                if (!failed) tq3_step<D, false, true>(acc, 0, s_cur, pf, ring, qt_lane, sc2, lane, s_cur);
                 for (int i = 0; i + 1 < n3 && !failed; ++i) {
                     const uint32_t cur = (uint32_t)i % NSTAGE, nxt = (uint32_t)(i + 1) % NSTAGE;
                     wait_slot(nxt);
                     if (failed) break;
-                    softmax_page<NB>(acc, s_cur, pf);
+                    softmax_rescale<NB>(acc, s_cur);
+                    tq3_step<D, true, true>(acc, ring + cur * G::SLOT, s_cur, pf, ring + nxt * G::SLOT, qt_lane, sc2, lane, s_next);
                     if constexpr (SCORED) store_page_mass<NB>(acc, pf, mass_row + lpg3[i], P.max_pages, GQ, lane);
-                    tq3_step<D, true, true>(acc, ring + cur * G::SLOT, pf, ring + nxt * G::SLOT, qt_lane, sc2, lane, s_next);
 #pragma unroll
                     for (int e = 0; e < 4; ++e) s_cur[e] = s_next[e];
                     __syncwarp();
                     if (i + NSTAGE < n3) issue_tq3(i + NSTAGE);
                 }
                 if (!failed) {
-                    softmax_page<NB>(acc, s_cur, pf);
+                    softmax_rescale<NB>(acc, s_cur);
+                    tq3_step<D, true, false>(acc, ring + ((uint32_t)(n3 - 1) % NSTAGE) * G::SLOT, s_cur, pf, 0, qt_lane, sc2, lane, s_next);
                     if constexpr (SCORED) store_page_mass<NB>(acc, pf, mass_row + lpg3[n3 - 1], P.max_pages, GQ, lane);
-                    tq3_step<D, true, false>(acc, ring + ((uint32_t)(n3 - 1) % NSTAGE) * G::SLOT, pf, 0, qt_lane, sc2, lane, s_next);
                 }
                 __syncwarp();
             }
