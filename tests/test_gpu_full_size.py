@@ -64,3 +64,45 @@ def test_config3_ragged_batch_sampled_requests():
     # a request whose pages are all zero records attends uniformly to zeros
     other = [b for b in range(spec.batch) if b not in sample][0]
     assert not out[other].any()
+
+
+def test_long_rows_many_rounds_kernels_agree():
+    """Rows long enough that every block lists its pages in several rounds (thousands of pages per block and
+    row): the two tensor-core kernels must agree with each other (2.8 M token-heads),
+    and a sampled (request, KV head) row is checked against the oracle on its own."""
+    spec = W.config(2, seq_lens=(16 * 24000 - 3, 16 * 20000), n_layers=1, recent_tokens=4096, anchor_prefix=512,
+                    anchor_spans=3, anchor_span_tokens=640)
+    tab = W.tables(spec)
+    d, hkv = spec.head_dim, spec.n_kv_heads
+    # pages: random valid records (any byte pattern is a valid record for the kernels except NaN bytes 0x7F/0xFF
+    # in FP8 records and fp16 specials in the TQ3 metadata, which the generator below avoids)
+    g = torch.Generator(device="cuda").manual_seed(7)
+    pool = M.Pool(d, hkv, spec.n_q_heads, tab.fp8_pages, tab.tq3_pages, W.rotation_signs(spec, 0), max_batch=spec.batch)
+    fp8 = torch.randint(0, 0x48, (tab.fp8_pages, hkv, 32 * d), generator=g, device="cuda", dtype=torch.uint8)      # |x| < 4
+    fp8 |= (torch.randint(0, 2, fp8.shape, generator=g, device="cuda", dtype=torch.uint8) << 7)
+    tq3 = torch.randint(0, 256, (tab.tq3_pages, hkv, 16 * d + 32), generator=g, device="cuda", dtype=torch.uint8)
+    meta16 = tq3[:, :, 12 * d:].view(torch.int16)              # key norms, value scales and zeros: fp16 in (-2, 2)
+    meta16 &= -16385                                             # clear the top exponent bit (0x4000): |x| < 2, never inf/nan
+    pool.fp8_arena.view(torch.uint8)[:fp8.numel()].copy_(fp8.reshape(-1))
+    pool.tq3_arena.view(torch.uint8)[:tq3.numel()].copy_(tq3.reshape(-1))
+    q = bf16_tensor(W.query(spec, 0))
+    bt = torch.from_numpy(tab.block_table).cuda()
+    tg = torch.from_numpy(tab.tier_tag).cuda()
+    ln = torch.from_numpy(tab.seq_lens).cuda()
+    outs = {}
+    for name, variant in (("tensor", M.DECODE_TENSOR), ("tmem", M.DECODE_TMEM)):
+        pool.set_decode_variant(variant)
+        lse = torch.empty((spec.batch, spec.n_q_heads), dtype=torch.float32, device="cuda")
+        outs[name] = (pool.decode_attention(q, bt, tg, ln, spec.scale, lse=lse).cpu().numpy(), lse.cpu().numpy())
+        torch.cuda.synchronize()
+        assert pool.status() == M.OK
+    a, b = outs["tensor"], outs["tmem"]
+    assert np.isfinite(a[0]).all() and np.isfinite(b[0]).all()
+    assert np.abs(a[0] - b[0]).max() <= 2e-4 * max(1.0, np.abs(a[0]).max())
+    assert np.abs(a[1] - b[1]).max() <= 1e-4
+    # one row against the oracle, which gets the same arenas
+    ref, ref_lse = oracle.decode_attention(fp8.cpu().numpy(), tq3.cpu().numpy(), d, hkv, spec.group, W.rotation_signs(spec, 0),
+                                           W.query(spec, 0), tab.block_table, tab.tier_tag, tab.seq_lens, spec.scale,
+                                           only_b=1, only_h=2)
+    G = spec.group
+    check_close(a[0][1, 2 * G:3 * G], ref[1, 2 * G:3 * G], "long row, request 1, KV head 2")
