@@ -22,7 +22,8 @@ def needs_build() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    deps = sources() + [os.path.join(CSRC, "mkv_internal.cuh"), os.path.join(ROOT, "include", "mkv.h")]
+    deps = sources() + [os.path.join(CSRC, "mkv_internal.cuh"), os.path.join(CSRC, "decode_tmem.cuh"),
+                        os.path.join(ROOT, "include", "mkv.h")]
     return any(os.path.getmtime(d) > t for d in deps)
 
 

@@ -12,6 +12,15 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200); run with -m gpu")
 
 
+def pytest_sessionstart(session):
+    """The library and the C oracle are built in-tree and not kept in the history: (re)build them when
+    they are missing or older than their sources (nvcc cross-compiles without a GPU)."""
+    from paper_2608_23834_b200 import build as mkv_build
+    mkv_build.build(force=False)
+    import oracle
+    oracle.build()
+
+
 def pytest_collection_modifyitems(config, items):
     # GPU tests are skipped (not failed) where no device exists, so that `pytest tests/` is green
     # on a CPU-only box; on a GPU box they must run through the CUDA library.
