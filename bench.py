@@ -497,6 +497,85 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------- lifecycle kernels
+def run_lifecycle(args):
+    """`--lifecycle`: bulk throughput of Append, Demote and Promote (Algorithm 1's state changes) for the
+    head geometry of the chosen config, each timed alone with CUDA events over data larger than L2.
+    Prints its own JSON line; the decode benchmark above is the contract's line."""
+    import torch
+    import paper_2608_23834_b200 as M
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    device = torch.device("cuda:%d" % int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(device)
+    M.lib()
+    spec = workload_spec(args)
+    d, hkv, hq = spec.head_dim, spec.n_kv_heads, spec.n_q_heads
+    fp8_page, tq3_page = 32 * d * hkv, (16 * d + 32) * hkv
+    P = max(1024, (384 << 20) // fp8_page)               # FP8 pages converted per call: 384 MB, 3 x L2
+    pool = M.Pool(d, hkv, hq, 2 * P + 8, P + 8, W.rotation_signs(spec, 0), max_batch=1, device=device)
+    gen = torch.Generator(device=device)
+    gen.manual_seed(spec.seed)
+    T = 16 * P
+    k = torch.randn((T, hkv, d), generator=gen, device=device, dtype=torch.float32)
+    k[:, :, torch.from_numpy(W.outlier_channels(spec, 0, 0)).to(device)] *= 8.0
+    k = k.to(torch.bfloat16)
+    v = torch.randn((T, hkv, d), generator=gen, device=device, dtype=torch.float32).to(torch.bfloat16)
+    slots = torch.arange(T, dtype=torch.int32, device=device)
+    ids = torch.arange(P, dtype=torch.int32, device=device)
+    ids_hi = ids + P
+    stream = torch.cuda.current_stream()
+    reps, warm = max(3, min(args.steps, 10)), 3
+    peaks, peak_kind = measured_peaks()
+    peak = float(peaks["hbm_gbs"])
+
+    def timed(fn):
+        for _ in range(warm):
+            fn()
+        torch.cuda.synchronize(device)
+        evs = []
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn()
+            b.record(stream)
+            evs.append((a, b))
+        torch.cuda.synchronize(device)
+        return statistics.median(x.elapsed_time(y) for x, y in evs)
+
+    def line(ms, units, unit_name, bytes_moved):
+        gbs = bytes_moved / (ms * 1e-3) / 1e9
+        return {"ms_per_call": ms, unit_name + "_per_s": units / (ms * 1e-3), "GB_per_s_in_plus_out": gbs,
+                "frac_of_%s_copy_bandwidth" % peak_kind: gbs / peak}
+
+    with ClockSampler(device.index or 0) as clocks:
+        ms_append = timed(lambda: pool.append(k, v, slots))                       # bf16 K,V in; e4m3 records out
+        ms_demote = timed(lambda: pool.demote(ids, ids))                          # FP8 pages in; TQ3 pages out
+        ms_promote = timed(lambda: pool.promote(ids, ids_hi))                     # TQ3 pages in; FP8 pages out
+    if pool.status() != M.OK:
+        raise RuntimeError("device status word set during the lifecycle run")
+    new = [torch.randn((spec.batch, hkv, d), generator=gen, device=device).to(torch.bfloat16) for _ in range(2)]
+    step_slots = (torch.arange(spec.batch, dtype=torch.int32, device=device) * 16 + 5)
+    ms_step_append = timed(lambda: pool.append(new[0], new[1], step_slots))
+    src1, dst1 = ids[:spec.batch].contiguous(), ids[:spec.batch].contiguous()
+    ms_step_demote = timed(lambda: pool.demote(src1, dst1))
+    print(json.dumps({
+        "mode": "lifecycle", "data": "synthetic", "n_gpus": 1,
+        "config": {"workload": "Append / Demote / Promote alone, head geometry of " + workload_name(spec),
+                   "head_dim": d, "kv_heads": hkv, "pages_per_call": P, "tokens_per_append_call": T,
+                   "fp8_page_bytes": fp8_page, "tq3_page_bytes": tq3_page, "repetitions": reps,
+                   "l2": "every call moves more than 3 x L2"},
+        "append": line(ms_append, T, "tokens", T * hkv * d * (4 + 2)),
+        "demote": line(ms_demote, P, "pages", P * (fp8_page + tq3_page)),
+        "promote": line(ms_promote, P, "pages", P * (fp8_page + tq3_page)),
+        "decode_step_calls": {"append_%d_tokens_ms" % spec.batch: ms_step_append,
+                              "demote_%d_pages_ms" % spec.batch: ms_step_demote,
+                              "note": "launch-bound sizes of one decode step, event-timed from Python"},
+        "peak": peak, "peak_source": peak_kind + " copy bandwidth", "clocks": clocks.summary(),
+    }))
+
+
 # ---------------------------------------------------------------------------------------- oracle arm
 def workload_spec(args):
     over = {"n_layers": args.layers} if args.layers > 0 else {}
@@ -595,11 +674,15 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="config 4 only: requests of the lifecycle cell (default 8)")
     ap.add_argument("--stale", type=float, default=0.5, help="config 4 only: Stale fraction of the lifecycle cell")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--lifecycle", action="store_true",
+                    help="time Append, Demote and Promote alone (bulk throughput) instead of the decode step")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
+    elif args.lifecycle:
+        run_lifecycle(args)
     else:
         run_ours(args)
 

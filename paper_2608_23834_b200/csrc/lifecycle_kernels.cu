@@ -27,6 +27,28 @@ __device__ __forceinline__ uint16_t f32_to_f16_sat_bits(float x)
 }
 
 // ------------------------------------------------------------------------------------------ append
+// One token of one KV head: thread i converts elements 2i, 2i+1 of K and V (scale, round to nearest
+// even, saturate to +-448) and stores K token-major, V channel-major.
+template <int D>
+__device__ __forceinline__ void append_token(uint8_t* __restrict__ rec, int slot, float inv_k_scale, float inv_v_scale,
+                                             const __nv_bfloat162* __restrict__ k, const __nv_bfloat162* __restrict__ v,
+                                             int pair)
+{
+    float2 kf = __bfloat1622float2(k[pair]);
+    float2 vf = __bfloat1622float2(v[pair]);
+    kf.x = __fmul_rn(kf.x, inv_k_scale);
+    kf.y = __fmul_rn(kf.y, inv_k_scale);
+    vf.x = __fmul_rn(vf.x, inv_v_scale);
+    vf.y = __fmul_rn(vf.y, inv_v_scale);
+    const __nv_fp8x2_storage_t kq = __nv_cvt_float2_to_fp8x2(kf, __NV_SATFINITE, __NV_E4M3);
+    const __nv_fp8x2_storage_t vq = __nv_cvt_float2_to_fp8x2(vf, __NV_SATFINITE, __NV_E4M3);
+    const int i = 2 * pair;
+    *reinterpret_cast<uint16_t*>(rec + slot * D + i) = kq;             // K: token-major
+    rec[16 * D + i * kPage + slot] = (uint8_t)(vq & 0xFF);             // V: channel-major
+    rec[16 * D + (i + 1) * kPage + slot] = (uint8_t)(vq >> 8);
+}
+
+// Decode-sized calls: one block per (token, KV head).
 template <int D>
 __global__ void __launch_bounds__(D / 2) append_kernel(uint8_t* __restrict__ fp8, int fp8_pages, int hkv,
                                                         float inv_k_scale, float inv_v_scale,
@@ -35,7 +57,7 @@ __global__ void __launch_bounds__(D / 2) append_kernel(uint8_t* __restrict__ fp8
                                                         const int32_t* __restrict__ slots,
                                                         uint32_t* __restrict__ status)
 {
-    const int tok = blockIdx.x, h = blockIdx.y, i = threadIdx.x * 2;
+    const int tok = blockIdx.x, h = blockIdx.y;
     const int sm = slots[tok];
     if (sm < 0) return;
     const int page = sm >> 4, slot = sm & 15;
@@ -44,40 +66,140 @@ __global__ void __launch_bounds__(D / 2) append_kernel(uint8_t* __restrict__ fp8
         return;
     }
     uint8_t* rec = fp8 + ((size_t)page * hkv + h) * fp8_record_bytes(D);
-    const size_t src = ((size_t)tok * hkv + h) * (D / 2) + threadIdx.x;
-    float2 kf = __bfloat1622float2(k[src]);
-    float2 vf = __bfloat1622float2(v[src]);
-    kf.x = __fmul_rn(kf.x, inv_k_scale);
-    kf.y = __fmul_rn(kf.y, inv_k_scale);
-    vf.x = __fmul_rn(vf.x, inv_v_scale);
-    vf.y = __fmul_rn(vf.y, inv_v_scale);
-    // round to nearest even, saturate to +-448
-    __nv_fp8x2_storage_t kq = __nv_cvt_float2_to_fp8x2(kf, __NV_SATFINITE, __NV_E4M3);
-    __nv_fp8x2_storage_t vq = __nv_cvt_float2_to_fp8x2(vf, __NV_SATFINITE, __NV_E4M3);
-    *reinterpret_cast<uint16_t*>(rec + slot * D + i) = kq;             // K: token-major
-    rec[16 * D + i * kPage + slot] = (uint8_t)(vq & 0xFF);             // V: channel-major
-    rec[16 * D + (i + 1) * kPage + slot] = (uint8_t)(vq >> 8);
+    const size_t src = ((size_t)tok * hkv + h) * (D / 2);
+    append_token<D>(rec, slot, inv_k_scale, inv_v_scale, k + src, v + src, threadIdx.x);
+}
+
+// eight bf16 (one 16-byte load) -> eight e4m3 bytes
+__device__ __forceinline__ uint2 bf16x8_to_e4m3x8(uint4 in, float inv_scale)
+{
+    const uint32_t w[4] = {in.x, in.y, in.z, in.w};
+    uint32_t q[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[i]));
+        f.x = __fmul_rn(f.x, inv_scale);
+        f.y = __fmul_rn(f.y, inv_scale);
+        q[i] = __nv_cvt_float2_to_fp8x2(f, __NV_SATFINITE, __NV_E4M3);
+    }
+    return make_uint2(q[0] | (q[1] << 16), q[2] | (q[3] << 16));
+}
+
+// Prefill-sized calls: one block per (16 consecutive input tokens, KV head).  Where the 16 tokens fill
+// one page front to back (slot_mapping[t0 + i] = 16 page + i), K rows leave with 8-byte stores and V
+// is transposed through shared memory so that every channel's 16 tokens leave as one 16-byte store;
+// any other group (skipped tokens, a run that starts inside a page, the tail) takes the per-token path.
+template <int D>
+__global__ void __launch_bounds__(128) append_run_kernel(uint8_t* __restrict__ fp8, int fp8_pages, int hkv,
+                                                          float inv_k_scale, float inv_v_scale,
+                                                          const __nv_bfloat162* __restrict__ k,
+                                                          const __nv_bfloat162* __restrict__ v,
+                                                          const int32_t* __restrict__ slots, int n,
+                                                          uint32_t* __restrict__ status)
+{
+    constexpr int VROW = D + 4;                      // padded token row of the transposition tile
+    __shared__ __align__(16) uint8_t vt[kPage * VROW];
+    __shared__ int32_t slot_s[kPage];
+    __shared__ int run_s;
+    const int t0 = blockIdx.x * kPage, h = blockIdx.y, tid = threadIdx.x;
+    const int cnt = min(kPage, n - t0);
+    if (tid < kPage) slot_s[tid] = tid < cnt ? slots[t0 + tid] : -1;
+    __syncthreads();
+    if (tid == 0) {
+        const int s0 = slot_s[0];
+        bool run = cnt == kPage && s0 >= 0 && (s0 & 15) == 0 && (s0 >> 4) < fp8_pages;
+        for (int i = 1; run && i < kPage; ++i) run = slot_s[i] == s0 + i;
+        run_s = run ? 1 : 0;
+    }
+    __syncthreads();
+    if (run_s) {
+        uint8_t* rec = fp8 + ((size_t)(slot_s[0] >> 4) * hkv + h) * fp8_record_bytes(D);
+        constexpr int CPT = D / 8;                   // 16-byte input chunks per token
+        for (int c = tid; c < kPage * CPT; c += 128) {
+            const int t = c / CPT, c8 = c % CPT;
+            const size_t at = ((size_t)(t0 + t) * hkv + h) * (D / 8) + c8;
+            const uint2 kq = bf16x8_to_e4m3x8(reinterpret_cast<const uint4*>(k)[at], inv_k_scale);
+            const uint2 vq = bf16x8_to_e4m3x8(reinterpret_cast<const uint4*>(v)[at], inv_v_scale);
+            *reinterpret_cast<uint2*>(rec + t * D + 8 * c8) = kq;
+            *reinterpret_cast<uint32_t*>(vt + t * VROW + 8 * c8) = vq.x;
+            *reinterpret_cast<uint32_t*>(vt + t * VROW + 8 * c8 + 4) = vq.y;
+        }
+        __syncthreads();
+        // thread c4 owns channels 4 c4 .. 4 c4 + 3: 16 words (one per token) -> 4 x 16 bytes
+        for (int c4 = tid; c4 < D / 4; c4 += 128) {
+            uint32_t w[kPage];
+#pragma unroll
+            for (int t = 0; t < kPage; ++t) w[t] = *reinterpret_cast<const uint32_t*>(vt + t * VROW + 4 * c4);
+#pragma unroll
+            for (int ch = 0; ch < 4; ++ch) {
+                uint32_t o[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const uint32_t lo = __byte_perm(w[4 * q], w[4 * q + 1], 0x0040 + 0x0011 * ch);   // bytes ch of t, t+1
+                    const uint32_t hi = __byte_perm(w[4 * q + 2], w[4 * q + 3], 0x0040 + 0x0011 * ch);
+                    o[q] = __byte_perm(lo, hi, 0x5410);
+                }
+                *reinterpret_cast<uint4*>(rec + 16 * D + (4 * c4 + ch) * kPage) = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+        }
+        return;
+    }
+    for (int t = 0; t < cnt; ++t) {
+        const int sm = slot_s[t];
+        if (sm < 0) continue;
+        if ((sm >> 4) >= fp8_pages) {
+            if (tid == 0) atomicOr(status, kStBounds);
+            continue;
+        }
+        uint8_t* rec = fp8 + ((size_t)(sm >> 4) * hkv + h) * fp8_record_bytes(D);
+        const size_t src = ((size_t)(t0 + t) * hkv + h) * (D / 2);
+        if (tid < D / 2) append_token<D>(rec, sm & 15, inv_k_scale, inv_v_scale, k + src, v + src, tid);
+    }
 }
 
 int32_t launch_append(mkv_pool* p, const void* k, const void* v, const int32_t* slots, int n, cudaStream_t s)
 {
-    dim3 grid(n, p->hkv);
     const float ik = 1.0f / p->cfg.k_scale, iv = 1.0f / p->cfg.v_scale;
-    if (p->d == 128)
-        append_kernel<128><<<grid, 64, 0, s>>>(p->fp8, p->cfg.fp8_pages, p->hkv, ik, iv,
-                                               (const __nv_bfloat162*)k, (const __nv_bfloat162*)v, slots,
-                                               p->status_dev);
-    else
-        append_kernel<256><<<grid, 128, 0, s>>>(p->fp8, p->cfg.fp8_pages, p->hkv, ik, iv,
-                                                (const __nv_bfloat162*)k, (const __nv_bfloat162*)v, slots,
-                                                p->status_dev);
+    const __nv_bfloat162* kk = (const __nv_bfloat162*)k;
+    const __nv_bfloat162* vv = (const __nv_bfloat162*)v;
+    if (n >= 2 * kPage) {
+        dim3 grid((n + kPage - 1) / kPage, p->hkv);
+        if (p->d == 128)
+            append_run_kernel<128><<<grid, 128, 0, s>>>(p->fp8, p->cfg.fp8_pages, p->hkv, ik, iv, kk, vv, slots, n,
+                                                        p->status_dev);
+        else
+            append_run_kernel<256><<<grid, 128, 0, s>>>(p->fp8, p->cfg.fp8_pages, p->hkv, ik, iv, kk, vv, slots, n,
+                                                        p->status_dev);
+    } else {
+        dim3 grid(n, p->hkv);
+        if (p->d == 128)
+            append_kernel<128><<<grid, 64, 0, s>>>(p->fp8, p->cfg.fp8_pages, p->hkv, ik, iv, kk, vv, slots, p->status_dev);
+        else
+            append_kernel<256><<<grid, 128, 0, s>>>(p->fp8, p->cfg.fp8_pages, p->hkv, ik, iv, kk, vv, slots, p->status_dev);
+    }
     MKV_CUDA(cudaGetLastError());
     return MKV_OK;
 }
 
 // ------------------------------------------------------------------------------------------ demote
 // One block per page; loops over the KV heads.  Warps encode key vectors (one token each), threads
-// encode value channels, then all threads assemble the packed words from the codes in shared memory.
+// encode value channels; the 3-bit codes meet in shared memory, where every thread assembles one
+// word triple of the record image; the image leaves with 16-byte stores.
+//
+// Shared layout: key codes [token][D + 8] (the 8 pad bytes spread the token rows over the banks for
+// the packers, which read rows g and g + 8), value codes [channel][16 tokens], and two record images
+// (alternating per head, so that the copy-out of one head overlaps the encoding of the next).
+
+// two e4m3 bytes (low byte first) -> two fp32
+__device__ __forceinline__ float2 e4m3x2_to_f32(uint32_t two_bytes)
+{
+    const __half2_raw h = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)two_bytes, __NV_E4M3);
+    return __half22float2(__half2(h));
+}
+
+// nibble pairs of two bytes -> one byte: (x & 0x000F) | ((x & 0x0F00) >> 4)
+__device__ __forceinline__ uint32_t squeeze_nibbles(uint32_t x) { return (x & 0xFu) | ((x >> 4) & 0xF0u); }
+
 template <int D>
 __global__ void __launch_bounds__(256) demote_kernel(const uint8_t* __restrict__ fp8, uint8_t* __restrict__ tq3,
                                                       int fp8_pages, int tq3_pages, int hkv, float k_scale,
@@ -88,11 +210,12 @@ __global__ void __launch_bounds__(256) demote_kernel(const uint8_t* __restrict__
                                                       uint32_t* __restrict__ status)
 {
     constexpr int EPL = D / 32;          // key elements per lane
-    constexpr int LW = 3 * (D / 16) / 4; // packed words per lane and section
-    __shared__ uint8_t kcode[kPage][D];
-    __shared__ uint8_t vcode[kPage][D];
-    __shared__ uint16_t g_s[kPage];
-    __shared__ uint16_t sc_s[D], zp_s[D];
+    constexpr int NJ = D / 64;           // word triples per lane and section
+    constexpr int KROW = D + 8;          // padded row of the key-code tile
+    constexpr int REC = 16 * D + 32;     // bytes of one TQ3 record
+    __shared__ __align__(16) uint8_t kcode[kPage * KROW];
+    __shared__ __align__(16) uint8_t vcode[D * kPage];
+    __shared__ __align__(16) uint8_t image[2][REC];
 
     const int page = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int src = src_ids[page], dst = dst_ids[page];
@@ -100,21 +223,43 @@ __global__ void __launch_bounds__(256) demote_kernel(const uint8_t* __restrict__
         if (tid == 0) atomicOr(status, kStBounds);
         return;
     }
-    const float C[4] = {MKV_C0, MKV_C1, MKV_C2, MKV_C3};
+    // squared levels (single fp32 products, as the record's norm correction defines them)
+    const float c0sq = __fmul_rn(MKV_C0, MKV_C0), c1sq = __fmul_rn(MKV_C1, MKV_C1),
+                c2sq = __fmul_rn(MKV_C2, MKV_C2), c3sq = __fmul_rn(MKV_C3, MKV_C3);
+    // rotation signs of this lane's key elements, as fp32 sign-bit masks
+    uint32_t flip[EPL];
+#pragma unroll
+    for (int r = 0; r < EPL; ++r) {
+        const int i = lane * EPL + r;
+        flip[r] = ((sigma.w[i >> 5] >> (i & 31)) & 1u) << 31;
+    }
+    uint32_t neg[5];                      // butterfly stage m: lanes with bit m set subtract
+#pragma unroll
+    for (int b = 0; b < 5; ++b) neg[b] = ((lane >> b) & 1u) << 31;
 
     for (int h = 0; h < hkv; ++h) {
         const uint8_t* rec8 = fp8 + ((size_t)src * hkv + h) * fp8_record_bytes(D);
         uint8_t* rec3 = tq3 + ((size_t)dst * hkv + h) * tq3_record_bytes(D);
+        uint8_t* img = image[h & 1];
 
         // ---- keys: warp w encodes tokens w and w + 8 ------------------------------------------
         for (int tok = warp; tok < kPage; tok += 8) {
             float x[EPL], a[EPL];
-            const uint8_t* row = rec8 + tok * D + lane * EPL;
+            uint32_t raw[EPL / 4];
+            if constexpr (EPL == 8) {
+                const uint2 u = *reinterpret_cast<const uint2*>(rec8 + tok * D + lane * EPL);
+                raw[0] = u.x;
+                raw[1] = u.y;
+            } else {
+                raw[0] = *reinterpret_cast<const uint32_t*>(rec8 + tok * D + lane * EPL);
+            }
 #pragma unroll
-            for (int r = 0; r < EPL; ++r) {
-                const int i = lane * EPL + r;
-                x[r] = __fmul_rn(e4m3_to_f32(row[r]), k_scale);
-                a[r] = ((sigma.w[i >> 5] >> (i & 31)) & 1u) ? -x[r] : x[r];
+            for (int r = 0; r < EPL; r += 2) {
+                const float2 f = e4m3x2_to_f32((raw[r >> 2] >> (8 * (r & 3))) & 0xFFFFu);
+                x[r] = __fmul_rn(f.x, k_scale);
+                x[r + 1] = __fmul_rn(f.y, k_scale);
+                a[r] = __uint_as_float(__float_as_uint(x[r]) ^ flip[r]);
+                a[r + 1] = __uint_as_float(__float_as_uint(x[r + 1]) ^ flip[r + 1]);
             }
             // Walsh-Hadamard butterflies, strides ascending: inside the lane, then across lanes
 #pragma unroll
@@ -127,11 +272,12 @@ __global__ void __launch_bounds__(256) demote_kernel(const uint8_t* __restrict__
                         a[r + hh] = __fsub_rn(u, w);
                     }
 #pragma unroll
-            for (int m = 1; m < 32; m <<= 1)
+            for (int b = 0; b < 5; ++b)
 #pragma unroll
                 for (int r = 0; r < EPL; ++r) {
-                    const float o = __shfl_xor_sync(0xffffffffu, a[r], m);
-                    a[r] = (lane & m) ? __fsub_rn(o, a[r]) : __fadd_rn(a[r], o);
+                    // lower lane: a + o; upper lane: o - a (the same single addition either way)
+                    const float o = __shfl_xor_sync(0xffffffffu, a[r], 1 << b);
+                    a[r] = __fadd_rn(o, __uint_as_float(__float_as_uint(a[r]) ^ neg[b]));
                 }
             // |x|^2: pairwise tree in index order (every element of the butterfly ends equal)
             float e[EPL];
@@ -147,14 +293,22 @@ __global__ void __launch_bounds__(256) demote_kernel(const uint8_t* __restrict__
             const float nx = __fsqrt_rn(n2);
             const float t1 = __fmul_rn(MKV_B0, nx), t2 = __fmul_rn(MKV_B1, nx), t3 = __fmul_rn(MKV_B2, nx);
             float f[EPL];
+            uint32_t packed[EPL / 4];
+#pragma unroll
+            for (int r = 0; r < EPL / 4; ++r) packed[r] = 0;
 #pragma unroll
             for (int r = 0; r < EPL; ++r) {
                 const float w = fabsf(a[r]);
-                const int mag = (w > t1) + (w > t2) + (w > t3);
-                const int sgn = a[r] < 0.0f ? 1 : 0;
-                kcode[tok][lane * EPL + r] = (uint8_t)(mag | (sgn << 2));
-                f[r] = __fmul_rn(C[mag], C[mag]);
+                const bool g1 = w > t1, g2 = w > t2, g3 = w > t3;
+                const uint32_t code = (uint32_t)g1 + (uint32_t)g2 + (uint32_t)g3 + ((__float_as_uint(a[r]) >> 29) & 4u);
+                // a[r] < 0 is the sign bit except for -0, which cannot meet a threshold test either way
+                packed[r >> 2] |= (a[r] == 0.0f ? (code & 3u) : code) << (8 * (r & 3));
+                f[r] = g2 ? (g3 ? c3sq : c2sq) : (g1 ? c1sq : c0sq);
             }
+            if constexpr (EPL == 8)
+                *reinterpret_cast<uint2*>(kcode + tok * KROW + lane * EPL) = make_uint2(packed[0], packed[1]);
+            else
+                *reinterpret_cast<uint32_t*>(kcode + tok * KROW + lane * EPL) = packed[0];
 #pragma unroll
             for (int hh = 1; hh < EPL; hh <<= 1)
 #pragma unroll
@@ -163,16 +317,22 @@ __global__ void __launch_bounds__(256) demote_kernel(const uint8_t* __restrict__
 #pragma unroll
             for (int m = 1; m < 32; m <<= 1) nc2 = __fadd_rn(nc2, __shfl_xor_sync(0xffffffffu, nc2, m));
             const float nc = __fsqrt_rn(nc2);
-            if (lane == 0) g_s[tok] = (nx == 0.0f) ? (uint16_t)0 : f32_to_f16_sat_bits(__fdiv_rn(nx, nc));
+            if (lane == 0)
+                *reinterpret_cast<uint16_t*>(img + 12 * D + 2 * tok) =
+                    (nx == 0.0f) ? (uint16_t)0 : f32_to_f16_sat_bits(__fdiv_rn(nx, nc));
         }
 
         // ---- values: one thread per channel, 16 tokens of the page ------------------------------
         for (int c = tid; c < D; c += 256) {
             const uint4 raw = *reinterpret_cast<const uint4*>(rec8 + 16 * D + c * kPage);
-            const uint8_t* bytes = reinterpret_cast<const uint8_t*>(&raw);
+            const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
             float val[kPage];
 #pragma unroll
-            for (int t = 0; t < kPage; ++t) val[t] = __fmul_rn(e4m3_to_f32(bytes[t]), v_scale);
+            for (int t = 0; t < kPage; t += 2) {
+                const float2 f = e4m3x2_to_f32((rw[t >> 2] >> (8 * (t & 3))) & 0xFFFFu);
+                val[t] = __fmul_rn(f.x, v_scale);
+                val[t + 1] = __fmul_rn(f.y, v_scale);
+            }
             float mn = val[0], mx = val[0];
 #pragma unroll
             for (int t = 1; t < kPage; ++t) {
@@ -182,78 +342,77 @@ __global__ void __launch_bounds__(256) demote_kernel(const uint8_t* __restrict__
             const uint16_t sc = f32_to_f16_sat_bits(__fdiv_rn(__fsub_rn(mx, mn), 7.0f));
             const uint16_t zp = f32_to_f16_sat_bits(mn);
             const float scf = __half2float(__ushort_as_half(sc)), zpf = __half2float(__ushort_as_half(zp));
-            sc_s[c] = sc;
-            zp_s[c] = zp;
+            {
+                const int cb = c >> 4, row = c & 15;
+                uint16_t* meta = reinterpret_cast<uint16_t*>(img + 12 * D + 32);
+                const int hi = (cb >> 1) * 64 + (row & 7) * 8 + 4 * (cb & 1) + (row >> 3);
+                meta[hi] = sc;
+                meta[hi + 2] = zp;
+            }
+            // q = clamp(rint((val - zp) / sc), 0, 7), 0 when sc == 0.  The division is the correctly
+            // rounded one; a zero numerator (the channel's minimum) or a zero scale is replaced by
+            // operands whose quotient is not used, which keeps the divider on its short path.
+            const float den = scf != 0.0f ? scf : 1.0f;
+            uint32_t q4[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
             for (int t = 0; t < kPage; ++t) {
-                int q = 0;
-                if (scf != 0.0f) {
-                    float r = rintf(__fdiv_rn(__fsub_rn(val[t], zpf), scf));   // half to even
-                    r = r < 0.0f ? 0.0f : r;
-                    r = r > 7.0f ? 7.0f : r;
-                    q = (int)r;
-                }
-                vcode[t][c] = (uint8_t)q;
+                const float num = __fsub_rn(val[t], zpf);
+                float r = rintf(__fdiv_rn(num != 0.0f ? num : den, den));   // half to even
+                r = r < 0.0f ? 0.0f : r;
+                r = r > 7.0f ? 7.0f : r;
+                const uint32_t q = (num != 0.0f && scf != 0.0f) ? (uint32_t)(int)r : 0u;
+                q4[t >> 2] |= q << (8 * (t & 3));
             }
+            *reinterpret_cast<uint4*>(vcode + c * kPage) = make_uint4(q4[0], q4[1], q4[2], q4[3]);
         }
         __syncthreads();
 
-        // ---- pack: every thread assembles whole 32-bit words of the two code sections ----------
-        for (int idx = tid; idx < 2 * 32 * LW; idx += 256) {
-            const int section = idx / (32 * LW), L = (idx / LW) & 31, w = idx % LW;
-            const int g = L >> 2, tq = L & 3, j = w / 3, kind = w % 3;
-            uint32_t word = 0;
+        // ---- pack: one thread per (section, triple j, fragment lane L) --------------------------
+        for (int item = tid; item < 2 * NJ * 32; item += 256) {
+            const int L = item & 31, j = (item >> 5) % NJ, section = item / (32 * NJ);
+            const int g = L >> 2, tq = L & 3;
+            uint32_t w0 = 0, w1 = 0, w2 = 0;
             if (section == 0) {
-                // key codes: nibble n = 2r + half holds row g + 8(r&1), slot 2tq + 8(r>>1) + half
+                // key codes: nibble n = 2r + half holds row g + 8(r&1), slot 2tq + 8(r>>1) + half.
+                // A: block 4j with the signs of block 4j+2; B: block 4j+1 with the signs of 4j+3;
+                // C: magnitudes of blocks 4j+2 (low pair) and 4j+3 (high pair).
 #pragma unroll
-                for (int n = 0; n < 8; ++n) {
-                    const int r = n >> 1, half = n & 1;
-                    const int t = g + 8 * (r & 1), s = 2 * tq + 8 * (r >> 1) + half;
-                    if (kind < 2) {   // A: block 4j (+ signs of block 4j+2); B: block 4j+1 (+ signs of 4j+3)
-                        const uint32_t own = kcode[t][16 * (4 * j + kind) + s];
-                        const uint32_t other = kcode[t][16 * (4 * j + kind + 2) + s];
-                        word |= (own | ((other >> 2) << 3)) << (4 * n);
-                    } else {          // C: magnitudes of blocks 4j+2 (low pair) and 4j+3 (high pair)
-                        const uint32_t lo = kcode[t][16 * (4 * j + 2) + s] & 3u;
-                        const uint32_t hi = kcode[t][16 * (4 * j + 3) + s] & 3u;
-                        word |= (lo | (hi << 2)) << (4 * n);
-                    }
+                for (int r = 0; r < 4; ++r) {
+                    const uint8_t* at = kcode + (g + 8 * (r & 1)) * KROW + 64 * j + 2 * tq + 8 * (r >> 1);
+                    const uint32_t b0 = *reinterpret_cast<const uint16_t*>(at);        // (half 0, half 1)
+                    const uint32_t b1 = *reinterpret_cast<const uint16_t*>(at + 16);
+                    const uint32_t b2 = *reinterpret_cast<const uint16_t*>(at + 32);
+                    const uint32_t b3 = *reinterpret_cast<const uint16_t*>(at + 48);
+                    w0 |= squeeze_nibbles(b0 | ((b2 & 0x0404u) << 1)) << (8 * r);
+                    w1 |= squeeze_nibbles(b1 | ((b3 & 0x0404u) << 1)) << (8 * r);
+                    w2 |= squeeze_nibbles((b2 & 0x0303u) | ((b3 & 0x0303u) << 2)) << (8 * r);
                 }
             } else {
-                // value codes: four 24-bit streams (group, half) per triple, spread over 3 words
-                uint32_t S[2][2];
+                // value codes: four 24-bit streams (group, half) per triple; stream code k is
+                // channel block 4j + 2 grp + (k>>2), row g + 8(k&1), token 2tq + 8((k>>1)&1) + half
+                uint32_t S[2][2] = {{0u, 0u}, {0u, 0u}};
 #pragma unroll
                 for (int grp = 0; grp < 2; ++grp)
 #pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        uint32_t st = 0;
-#pragma unroll
-                        for (int k = 0; k < 8; ++k) {
-                            const int cb = 4 * j + 2 * grp + (k >> 2), r = k & 3;
-                            const int row = g + 8 * (r & 1), t = 2 * tq + 8 * (r >> 1) + half;
-                            st |= (uint32_t)vcode[t][16 * cb + row] << (3 * k);
-                        }
-                        S[grp][half] = st;
+                    for (int k = 0; k < 8; ++k) {
+                        const int cb = 4 * j + 2 * grp + (k >> 2), r = k & 3;
+                        const uint32_t two = *reinterpret_cast<const uint16_t*>(
+                            vcode + (16 * cb + g + 8 * (r & 1)) * kPage + 2 * tq + 8 * (r >> 1));
+                        S[grp][0] |= (two & 7u) << (3 * k);
+                        S[grp][1] |= (two >> 8) << (3 * k);
                     }
-                auto byte = [](uint32_t st, int b) { return (st >> (8 * b)) & 0xFFu; };
-                if (kind == 0)
-                    word = byte(S[0][0], 0) | byte(S[0][0], 1) << 8 | byte(S[0][1], 0) << 16 | byte(S[0][1], 1) << 24;
-                else if (kind == 1)
-                    word = byte(S[0][0], 2) | byte(S[1][0], 0) << 8 | byte(S[0][1], 2) << 16 | byte(S[1][1], 0) << 24;
-                else
-                    word = byte(S[1][0], 1) | byte(S[1][0], 2) << 8 | byte(S[1][1], 1) << 16 | byte(S[1][1], 2) << 24;
+                w0 = (S[0][0] & 0xFFFFu) | (S[0][1] << 16);
+                w1 = (S[0][0] >> 16) | ((S[1][0] & 0xFFu) << 8) | ((S[0][1] >> 16) << 16) | (S[1][1] << 24);
+                w2 = (S[1][0] >> 8) | ((S[1][1] >> 8) << 16);
             }
-            *reinterpret_cast<uint32_t*>(rec3 + section * 6 * D + lane_word_offset(D, L, w)) = word;
-        }
-        if (tid < kPage) *reinterpret_cast<uint16_t*>(rec3 + 12 * D + 2 * tid) = g_s[tid];
-        for (int c = tid; c < D; c += 256) {
-            const int cb = c >> 4, row = c & 15;
-            const int hi = (cb >> 1) * 64 + (row & 7) * 8 + 4 * (cb & 1) + (row >> 3);
-            uint16_t* meta = reinterpret_cast<uint16_t*>(rec3 + 12 * D + 32);
-            meta[hi] = sc_s[c];
-            meta[hi + 2] = zp_s[c];
+            uint8_t* sec = img + section * 6 * D;
+            *reinterpret_cast<uint32_t*>(sec + lane_word_offset(D, L, 3 * j)) = w0;
+            *reinterpret_cast<uint32_t*>(sec + lane_word_offset(D, L, 3 * j + 1)) = w1;
+            *reinterpret_cast<uint32_t*>(sec + lane_word_offset(D, L, 3 * j + 2)) = w2;
         }
         __syncthreads();
+        for (int i = tid; i < REC / 16; i += 256)
+            reinterpret_cast<uint4*>(rec3)[i] = reinterpret_cast<const uint4*>(img)[i];
     }
 
     // copy-before-publish: the record is complete and visible before its id and tag appear

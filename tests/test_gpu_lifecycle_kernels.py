@@ -58,6 +58,56 @@ def test_append_is_bit_exact(d, hkv, k_scale, v_scale):
     assert not pool.page_read_raw(M.FMT_FP8, int(np.setdiff1d(np.arange(n_pages), page_of)[0])).any()
 
 
+@pytest.mark.parametrize("d,hkv,k_scale,v_scale", [(128, 2, 1.0, 1.0), (256, 4, 0.5, 2.0)])
+def test_prefill_sized_append_is_bit_exact(d, hkv, k_scale, v_scale):
+    """One call of many tokens: groups of 16 input tokens that fill a page front to back take the
+    transposing path, every other group (a skipped token, a run that starts inside a page, a page that
+    does not exist, the ragged tail) the per-token path; both must write the same bytes."""
+    rng = np.random.default_rng(7 * d + hkv)
+    n_pages = 12
+    pool = M.Pool(d, hkv, hkv * 2, n_pages, 1, np.ones(d, np.int8), k_scale, v_scale)
+    page_of = rng.permutation(n_pages)
+    plan = []                                            # (page, first slot, tokens) per input group, in input order
+    plan += [(int(page_of[i]), 0, 16) for i in range(4)]             # whole pages
+    plan += [(int(page_of[4]), 0, 16)]                               # whole page with one skipped token (below)
+    plan += [(int(page_of[5]), 0, 16)]                               # whole page, slots permuted (below)
+    plan += [(n_pages + 3, 0, 16)]                                   # a page beyond the arena: flagged, not written
+    plan += [(int(page_of[6]), 8, 8), (int(page_of[7]), 0, 8)]       # one input group over two half pages
+    plan += [(int(page_of[8]), 0, 16)]                               # aligned again
+    plan += [(int(page_of[9]), 0, 5)]                                # ragged tail
+    slots = np.concatenate([p * 16 + s0 + np.arange(n) for p, s0, n in plan]).astype(np.int32)
+    skipped = 4 * 16 + 9
+    slots[skipped] = -1
+    perm = 5 * 16 + rng.permutation(16)
+    slots[5 * 16:6 * 16] = slots[perm]
+    n_tok = len(slots)
+    k_bits, v_bits = special_bf16(rng, (n_tok, hkv, d)), special_bf16(rng, (n_tok, hkv, d))
+    pool.append(bf16_tensor(k_bits), bf16_tensor(v_bits), torch.from_numpy(slots).cuda())
+    torch.cuda.synchronize()
+    assert pool.status() == M.E_BOUNDS and pool.status() == M.OK
+    kf, vf = oracle.bf16_bits_to_f32(k_bits), oracle.bf16_bits_to_f32(v_bits)
+    want = {}                                            # page -> (k [16][d], v [16][d], filled slots) per head
+    for t, sm in enumerate(slots):
+        if sm < 0 or sm // 16 >= n_pages:
+            continue
+        kk, vv, used = want.setdefault(int(sm) // 16, (np.zeros((hkv, 16, d), np.float32), np.zeros((hkv, 16, d), np.float32), set()))
+        kk[:, sm % 16], vv[:, sm % 16] = kf[t], vf[t]
+        used.add(int(sm) % 16)
+    assert len(want) == 10
+    for page in range(n_pages):
+        got = pool.page_read_raw(M.FMT_FP8, page).reshape(hkv, 32 * d)
+        if page not in want:
+            assert not got.any()
+            continue
+        kk, vv, used = want[page]
+        for h in range(hkv):
+            ref = oracle.fp8_pack_record(kk[h], vv[h], 16, k_scale, v_scale).copy()
+            for s in set(range(16)) - used:              # slots never written stay zero
+                ref[:16 * d].reshape(16, d)[s] = 0
+                ref[16 * d:].reshape(d, 16)[:, s] = 0
+            assert np.array_equal(got[h], ref), (page, h)
+
+
 @pytest.mark.parametrize("d,hkv,k_scale,v_scale", [(128, 2, 1.0, 1.0), (256, 4, 1.0, 1.0), (256, 1, 0.25, 4.0)])
 def test_demote_is_bit_exact_and_publishes_after_the_copy(d, hkv, k_scale, v_scale):
     rng = np.random.default_rng(100 + d + hkv)
