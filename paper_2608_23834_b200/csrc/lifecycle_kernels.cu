@@ -201,7 +201,7 @@ __device__ __forceinline__ float2 e4m3x2_to_f32(uint32_t two_bytes)
 __device__ __forceinline__ uint32_t squeeze_nibbles(uint32_t x) { return (x & 0xFu) | ((x >> 4) & 0xF0u); }
 
 template <int D>
-__global__ void __launch_bounds__(256) demote_kernel(const uint8_t* __restrict__ fp8, uint8_t* __restrict__ tq3,
+__global__ void __launch_bounds__(D) demote_kernel(const uint8_t* __restrict__ fp8, uint8_t* __restrict__ tq3,
                                                       int fp8_pages, int tq3_pages, int hkv, float k_scale,
                                                       float v_scale, SigmaBits sigma,
                                                       const int32_t* __restrict__ src_ids,
@@ -213,6 +213,7 @@ __global__ void __launch_bounds__(256) demote_kernel(const uint8_t* __restrict__
     constexpr int NJ = D / 64;           // word triples per lane and section
     constexpr int KROW = D + 8;          // padded row of the key-code tile
     constexpr int REC = 16 * D + 32;     // bytes of one TQ3 record
+    constexpr int NT = D;                // threads: one per value channel, one per packed word triple
     __shared__ __align__(16) uint8_t kcode[kPage * KROW];
     __shared__ __align__(16) uint8_t vcode[D * kPage];
     __shared__ __align__(16) uint8_t image[2][REC];
@@ -242,8 +243,8 @@ __global__ void __launch_bounds__(256) demote_kernel(const uint8_t* __restrict__
         uint8_t* rec3 = tq3 + ((size_t)dst * hkv + h) * tq3_record_bytes(D);
         uint8_t* img = image[h & 1];
 
-        // ---- keys: warp w encodes tokens w and w + 8 ------------------------------------------
-        for (int tok = warp; tok < kPage; tok += 8) {
+        // ---- keys: warp w encodes tokens w, w + NT/32, ... ------------------------------------------
+        for (int tok = warp; tok < kPage; tok += NT / 32) {
             float x[EPL], a[EPL];
             uint32_t raw[EPL / 4];
             if constexpr (EPL == 8) {
@@ -323,7 +324,7 @@ __global__ void __launch_bounds__(256) demote_kernel(const uint8_t* __restrict__
         }
 
         // ---- values: one thread per channel, 16 tokens of the page ------------------------------
-        for (int c = tid; c < D; c += 256) {
+        for (int c = tid; c < D; c += NT) {
             const uint4 raw = *reinterpret_cast<const uint4*>(rec8 + 16 * D + c * kPage);
             const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
             float val[kPage];
@@ -368,7 +369,7 @@ __global__ void __launch_bounds__(256) demote_kernel(const uint8_t* __restrict__
         __syncthreads();
 
         // ---- pack: one thread per (section, triple j, fragment lane L) --------------------------
-        for (int item = tid; item < 2 * NJ * 32; item += 256) {
+        for (int item = tid; item < 2 * NJ * 32; item += NT) {
             const int L = item & 31, j = (item >> 5) % NJ, section = item / (32 * NJ);
             const int g = L >> 2, tq = L & 3;
             uint32_t w0 = 0, w1 = 0, w2 = 0;
@@ -411,7 +412,7 @@ __global__ void __launch_bounds__(256) demote_kernel(const uint8_t* __restrict__
             *reinterpret_cast<uint32_t*>(sec + lane_word_offset(D, L, 3 * j + 2)) = w2;
         }
         __syncthreads();
-        for (int i = tid; i < REC / 16; i += 256)
+        for (int i = tid; i < REC / 16; i += NT)
             reinterpret_cast<uint4*>(rec3)[i] = reinterpret_cast<const uint4*>(img)[i];
     }
 
@@ -432,7 +433,7 @@ int32_t launch_demote(mkv_pool* p, const int32_t* src, const int32_t* dst, int n
                       const int64_t* entry, cudaStream_t s)
 {
     if (p->d == 128)
-        demote_kernel<128><<<n, 256, 0, s>>>(p->fp8, p->tq3, p->cfg.fp8_pages, p->cfg.tq3_pages, p->hkv,
+        demote_kernel<128><<<n, 128, 0, s>>>(p->fp8, p->tq3, p->cfg.fp8_pages, p->cfg.tq3_pages, p->hkv,
                                              p->cfg.k_scale, p->cfg.v_scale, p->sigma, src, dst, bt, tags, entry,
                                              p->status_dev);
     else
@@ -445,75 +446,89 @@ int32_t launch_demote(mkv_pool* p, const int32_t* src, const int32_t* dst, int n
 
 // ------------------------------------------------------------------------------------------ promote
 // Promote (Algorithm 1 step 3): reconstruct a Stale page into a newly allocated FP8 page, then publish
-// it as Anchor.  One block per page, loops over the KV heads.  Warps rebuild key vectors (signed
-// levels, shuffle Walsh-Hadamard, norm correction, sign), threads rebuild value channels; the fp32
-// operation order is fixed so that the written bytes are reproducible.
+// it as Anchor.  One block per page, loops over the KV heads.  The record is staged in shared memory;
+// warps rebuild key vectors (signed levels, shuffle Walsh-Hadamard, norm correction, sign), threads
+// rebuild value channels; the fp32 operation order is fixed so that the written bytes are reproducible.
+//
+// Reading the code sections back (inverse of the packer in demote_kernel): fragment lane
+// L = 4 (row % 8) + (slot % 8) / 2 holds, in nibble 2 rr + slot % 2 with rr = row / 8 + 2 (slot / 8),
+// the entry (row, slot) of every 16 x 16 block; for keys row = token and slot = channel % 16, for
+// values row = channel % 16 and slot = token.
 template <int D>
-__device__ __forceinline__ uint32_t tq3_lane_word(const uint8_t* section, int lane, int w)
-{
-    return *reinterpret_cast<const uint32_t*>(section + lane_word_offset(D, lane, w));
-}
-
-template <int D>
-__device__ int tq3_key_code_at(const uint8_t* rec, int t, int i)
-{
-    const int kb = i >> 4, s = i & 15;
-    const int lane = 4 * (t & 7) + ((s & 7) >> 1), r = (t >> 3) + 2 * (s >> 3), n = 2 * r + (s & 1), j = kb >> 2;
-    const uint32_t A = tq3_lane_word<D>(rec, lane, 3 * j), Bw = tq3_lane_word<D>(rec, lane, 3 * j + 1),
-                   Cw = tq3_lane_word<D>(rec, lane, 3 * j + 2);
-    switch (kb & 3) {
-    case 0: return (A >> (4 * n)) & 7;
-    case 1: return (Bw >> (4 * n)) & 7;
-    case 2: return ((Cw >> (4 * n)) & 3) | (((A >> (4 * n + 3)) & 1) << 2);
-    default: return ((Cw >> (4 * n + 2)) & 3) | (((Bw >> (4 * n + 3)) & 1) << 2);
-    }
-}
-
-template <int D>
-__device__ int tq3_value_code_at(const uint8_t* rec, int t, int c)
-{
-    const int cb = c >> 4, row = c & 15;
-    const int lane = 4 * (row & 7) + ((t & 7) >> 1), r = (row >> 3) + 2 * (t >> 3), half = t & 1;
-    const int j = cb >> 2, grp = (cb & 3) >> 1, k = 4 * (cb & 1) + r;
-    const uint8_t* sec = rec + 6 * D;
-    const uint32_t W0 = tq3_lane_word<D>(sec, lane, 3 * j), W1 = tq3_lane_word<D>(sec, lane, 3 * j + 1),
-                   W2 = tq3_lane_word<D>(sec, lane, 3 * j + 2);
-    auto by = [](uint32_t w, int b) { return (w >> (8 * b)) & 0xFFu; };
-    uint32_t st;
-    if (grp == 0)
-        st = half == 0 ? (by(W0, 0) | by(W0, 1) << 8 | by(W1, 0) << 16) : (by(W0, 2) | by(W0, 3) << 8 | by(W1, 2) << 16);
-    else
-        st = half == 0 ? (by(W1, 1) | by(W2, 0) << 8 | by(W2, 1) << 16) : (by(W1, 3) | by(W2, 2) << 8 | by(W2, 3) << 16);
-    return (st >> (3 * k)) & 7;
-}
-
-template <int D>
-__global__ void __launch_bounds__(256) promote_kernel(const uint8_t* __restrict__ tq3, uint8_t* __restrict__ fp8,
-                                                       int tq3_pages, int fp8_pages, int hkv, float inv_k_scale,
-                                                       float inv_v_scale, float rs, SigmaBits sigma,
-                                                       const int32_t* __restrict__ src_ids,
-                                                       const int32_t* __restrict__ dst_ids, int32_t* block_table,
-                                                       uint8_t* tier_tag, const int64_t* entry_index,
-                                                       uint32_t* __restrict__ status)
+__global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ tq3, uint8_t* __restrict__ fp8,
+                                                     int tq3_pages, int fp8_pages, int hkv, float inv_k_scale,
+                                                     float inv_v_scale, float rs, SigmaBits sigma,
+                                                     const int32_t* __restrict__ src_ids,
+                                                     const int32_t* __restrict__ dst_ids, int32_t* block_table,
+                                                     uint8_t* tier_tag, const int64_t* entry_index,
+                                                     uint32_t* __restrict__ status)
 {
     constexpr int EPL = D / 32;
+    constexpr int NT = D;
+    constexpr int REC = 16 * D + 32;
+    __shared__ __align__(16) uint8_t image[2][REC];
+    __shared__ float level[8];            // signed key levels by 3-bit code
+
     const int page = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int src = src_ids[page], dst = dst_ids[page];
     if (src < 0 || src >= tq3_pages || dst < 0 || dst >= fp8_pages) {
         if (tid == 0) atomicOr(status, kStBounds);
         return;
     }
-    const float C[4] = {MKV_C0, MKV_C1, MKV_C2, MKV_C3};
+    if (tid < 8) {
+        const float c = (tid & 3) == 0 ? MKV_C0 : (tid & 3) == 1 ? MKV_C1 : (tid & 3) == 2 ? MKV_C2 : MKV_C3;
+        level[tid] = (tid & 4) ? -c : c;
+    }
+    // ---- per-lane constants of the key path: this lane rebuilds channels lane*EPL .. +EPL-1
+    const int kb = (lane * EPL) >> 4, s0 = (lane * EPL) & 15;       // 16-channel block, first slot in it
+    const int kj = kb >> 2, kind = kb & 3;
+    const int w_sgn = 3 * kj + (kind & 1);                          // word A or B: codes of kinds 0/1, signs of 2/3
+    const int w_mag = kind < 2 ? w_sgn : 3 * kj + 2;                // word C holds the magnitudes of kinds 2/3
+    const int off_sgn = lane_word_offset(D, 0, w_sgn), off_mag = lane_word_offset(D, 0, w_mag);
+    const int str_sgn = lane_word_offset(D, 1, w_sgn) - off_sgn, str_mag = lane_word_offset(D, 1, w_mag) - off_mag;
+    const int mag_extra = kind == 3 ? 2 : 0;                        // high pair of the C nibble
+    const uint32_t mag_mask = kind < 2 ? 7u : 3u;                   // kinds 0/1 read sign and magnitude at once
+    const uint32_t sgn_mask = kind < 2 ? 0u : 4u;
+    uint32_t flip[EPL];
+#pragma unroll
+    for (int r = 0; r < EPL; ++r) {
+        const int i = lane * EPL + r;
+        flip[r] = ((sigma.w[i >> 5] >> (i & 31)) & 1u) << 31;
+    }
+    uint32_t neg[5];
+#pragma unroll
+    for (int b = 0; b < 5; ++b) neg[b] = ((lane >> b) & 1u) << 31;
+    // ---- per-thread constants of the value path: this thread rebuilds channel tid
+    const int cb = tid >> 4, row = tid & 15;
+    const int vj = cb >> 2, grp = (cb & 3) >> 1, k0 = 4 * (cb & 1) + (row >> 3);
+    const int off_v = 6 * D + lane_word_offset(D, 4 * (row & 7), 3 * vj + grp);
+    const int off_v1 = 6 * D + lane_word_offset(D, 4 * (row & 7), 3 * vj + grp + 1);
+    const int str_v = lane_word_offset(D, 1, 3 * vj + grp) - lane_word_offset(D, 0, 3 * vj + grp);
+    const int str_v1 = lane_word_offset(D, 1, 3 * vj + grp + 1) - lane_word_offset(D, 0, 3 * vj + grp + 1);
+    const uint32_t sel0 = grp == 0 ? 0x0410u : 0x0541u, sel1 = grp == 0 ? 0x0632u : 0x0763u;
+    const int meta_i = (cb >> 1) * 64 + (row & 7) * 8 + 4 * (cb & 1) + (row >> 3);
+
     for (int h = 0; h < hkv; ++h) {
         const uint8_t* rec3 = tq3 + ((size_t)src * hkv + h) * tq3_record_bytes(D);
         uint8_t* rec8 = fp8 + ((size_t)dst * hkv + h) * fp8_record_bytes(D);
-        // ---- keys: warp w rebuilds tokens w and w + 8
-        for (int tok = warp; tok < kPage; tok += 8) {
+        uint8_t* img = image[h & 1];
+        for (int i = tid; i < REC / 16; i += NT)
+            reinterpret_cast<uint4*>(img)[i] = reinterpret_cast<const uint4*>(rec3)[i];
+        __syncthreads();
+
+        // ---- keys: warp w rebuilds tokens w, w + NT/32, ...
+        for (int tok = warp; tok < kPage; tok += NT / 32) {
             float y[EPL];
 #pragma unroll
-            for (int r = 0; r < EPL; ++r) {
-                const int kc = tq3_key_code_at<D>(rec3, tok, lane * EPL + r);
-                y[r] = (kc & 4) ? -C[kc & 3] : C[kc & 3];
+            for (int r2 = 0; r2 < EPL; r2 += 2) {
+                const int s = s0 + r2;                                    // even slot; s + 1 shares the word
+                const int L = 4 * (tok & 7) + ((s & 7) >> 1), n = 2 * ((tok >> 3) + 2 * (s >> 3));
+                const uint32_t ws = *reinterpret_cast<const uint32_t*>(img + off_sgn + L * str_sgn) >> (4 * n);
+                const uint32_t wm = *reinterpret_cast<const uint32_t*>(img + off_mag + L * str_mag) >> (4 * n + mag_extra);
+                const uint32_t c_even = (wm & mag_mask) | ((ws >> 1) & sgn_mask);
+                const uint32_t c_odd = ((wm >> 4) & mag_mask) | ((ws >> 5) & sgn_mask);
+                y[r2] = level[c_even];
+                y[r2 + 1] = level[c_odd];
             }
 #pragma unroll
             for (int hh = 1; hh < EPL; hh <<= 1)
@@ -525,36 +540,54 @@ __global__ void __launch_bounds__(256) promote_kernel(const uint8_t* __restrict_
                         y[r + hh] = __fsub_rn(u, w);
                     }
 #pragma unroll
-            for (int m = 1; m < 32; m <<= 1)
+            for (int b = 0; b < 5; ++b)
 #pragma unroll
                 for (int r = 0; r < EPL; ++r) {
-                    const float o = __shfl_xor_sync(0xffffffffu, y[r], m);
-                    y[r] = (lane & m) ? __fsub_rn(o, y[r]) : __fadd_rn(y[r], o);
+                    const float o = __shfl_xor_sync(0xffffffffu, y[r], 1 << b);
+                    y[r] = __fadd_rn(o, __uint_as_float(__float_as_uint(y[r]) ^ neg[b]));
                 }
-            const float g = __half2float(reinterpret_cast<const __half*>(rec3 + 12 * D)[tok]);
+            const float g = __half2float(reinterpret_cast<const __half*>(img + 12 * D)[tok]);
             const float gr = __fmul_rn(g, rs);
+            uint32_t out[EPL / 4];
 #pragma unroll
-            for (int r = 0; r < EPL; ++r) {
-                const int i = lane * EPL + r;
-                float k = __fmul_rn(gr, y[r]);
-                if ((sigma.w[i >> 5] >> (i & 31)) & 1u) k = -k;
-                rec8[tok * D + i] = (uint8_t)__nv_cvt_float_to_fp8(__fmul_rn(k, inv_k_scale), __NV_SATFINITE, __NV_E4M3);
+            for (int r = 0; r < EPL / 4; ++r) out[r] = 0;
+#pragma unroll
+            for (int r = 0; r < EPL; r += 2) {
+                float2 kk;
+                kk.x = __fmul_rn(__uint_as_float(__float_as_uint(__fmul_rn(gr, y[r])) ^ flip[r]), inv_k_scale);
+                kk.y = __fmul_rn(__uint_as_float(__float_as_uint(__fmul_rn(gr, y[r + 1])) ^ flip[r + 1]), inv_k_scale);
+                out[r >> 2] |= (uint32_t)__nv_cvt_float2_to_fp8x2(kk, __NV_SATFINITE, __NV_E4M3) << (8 * (r & 3));
             }
+            if constexpr (EPL == 8)
+                *reinterpret_cast<uint2*>(rec8 + tok * D + lane * EPL) = make_uint2(out[0], out[1]);
+            else
+                *reinterpret_cast<uint32_t*>(rec8 + tok * D + lane * EPL) = out[0];
         }
-        // ---- values: one thread per channel
-        for (int c = tid; c < D; c += 256) {
-            const int cb = c >> 4, row = c & 15;
-            const __half* meta = reinterpret_cast<const __half*>(rec3 + 12 * D + 32);
-            const int mi = (cb >> 1) * 64 + (row & 7) * 8 + 4 * (cb & 1) + (row >> 3);
-            const float sc = __half2float(meta[mi]), zp = __half2float(meta[mi + 2]);
+        // ---- values: one thread per channel; fragment lane 4 (row % 8) + q holds tokens 2q, 2q+1, 2q+8, 2q+9
+        {
+            const __half* meta = reinterpret_cast<const __half*>(img + 12 * D + 32);
+            const float sc = __half2float(meta[meta_i]), zp = __half2float(meta[meta_i + 2]);
+            uint32_t code[kPage];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const uint32_t lo = *reinterpret_cast<const uint32_t*>(img + off_v + q * str_v);
+                const uint32_t hi = *reinterpret_cast<const uint32_t*>(img + off_v1 + q * str_v1);
+                const uint32_t st0 = __byte_perm(lo, hi, sel0) >> (3 * k0);          // stream of the even tokens
+                const uint32_t st1 = __byte_perm(lo, hi, sel1) >> (3 * k0);          // stream of the odd tokens
+                code[2 * q] = st0 & 7u;
+                code[2 * q + 1] = st1 & 7u;
+                code[2 * q + 8] = (st0 >> 6) & 7u;
+                code[2 * q + 9] = (st1 >> 6) & 7u;
+            }
             uint32_t out[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
-            for (int t = 0; t < kPage; ++t) {
-                const float v = __fadd_rn(__fmul_rn(sc, (float)tq3_value_code_at<D>(rec3, t, c)), zp);
-                const uint32_t b = (uint32_t)__nv_cvt_float_to_fp8(__fmul_rn(v, inv_v_scale), __NV_SATFINITE, __NV_E4M3);
-                out[t >> 2] |= b << (8 * (t & 3));
+            for (int t = 0; t < kPage; t += 2) {
+                float2 vv;
+                vv.x = __fmul_rn(__fadd_rn(__fmul_rn(sc, (float)code[t]), zp), inv_v_scale);
+                vv.y = __fmul_rn(__fadd_rn(__fmul_rn(sc, (float)code[t + 1]), zp), inv_v_scale);
+                out[t >> 2] |= (uint32_t)__nv_cvt_float2_to_fp8x2(vv, __NV_SATFINITE, __NV_E4M3) << (8 * (t & 3));
             }
-            *reinterpret_cast<uint4*>(rec8 + 16 * D + c * kPage) = make_uint4(out[0], out[1], out[2], out[3]);
+            *reinterpret_cast<uint4*>(rec8 + 16 * D + tid * kPage) = make_uint4(out[0], out[1], out[2], out[3]);
         }
     }
     // copy-before-publish
@@ -576,7 +609,7 @@ int32_t launch_promote(mkv_pool* p, const int32_t* src, const int32_t* dst, int 
     const float ik = 1.0f / p->cfg.k_scale, iv = 1.0f / p->cfg.v_scale;
     const float rs = (float)(1.0 / sqrt((double)p->d));
     if (p->d == 128)
-        promote_kernel<128><<<n, 256, 0, s>>>(p->tq3, p->fp8, p->cfg.tq3_pages, p->cfg.fp8_pages, p->hkv, ik, iv, rs,
+        promote_kernel<128><<<n, 128, 0, s>>>(p->tq3, p->fp8, p->cfg.tq3_pages, p->cfg.fp8_pages, p->hkv, ik, iv, rs,
                                               p->sigma, src, dst, bt, tags, entry, p->status_dev);
     else
         promote_kernel<256><<<n, 256, 0, s>>>(p->tq3, p->fp8, p->cfg.tq3_pages, p->cfg.fp8_pages, p->hkv, ik, iv, rs,
