@@ -181,10 +181,60 @@ int32_t launch_append(mkv_pool* p, const void* k, const void* v, const int32_t* 
     return MKV_OK;
 }
 
+// ---- thread-block cluster helpers (Demote and Promote run one cluster per page) ------------------
+__device__ __forceinline__ uint32_t cluster_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_size()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+    return r;
+}
+// Every thread of every block of the cluster arrives exactly once; no block leaves early.
+__device__ __forceinline__ void cluster_barrier()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+// Blocks per page.  A call of few pages (the retier of a decode step) is latency-bound: the heads of a
+// page go to the blocks of a cluster, the largest divisor of the head count that a portable cluster
+// allows.  A call that fills the GPU with one block per page anyway keeps the heads in one block, which
+// amortises the per-block set-up and overlaps one head's copy-out with the next head's encoding.
+static int heads_cluster(int hkv, int n_pages)
+{
+    if (n_pages > 2 * 148) return 1;
+    for (int c = 8; c > 1; --c)
+        if (hkv % c == 0) return c;
+    return 1;
+}
+
+template <typename Kernel, typename... Args>
+static cudaError_t launch_clustered(Kernel kernel, int n_pages, int csize, int threads, cudaStream_t s, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)n_pages * csize);
+    cfg.blockDim = dim3(threads);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = csize;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 // ------------------------------------------------------------------------------------------ demote
-// One block per page; loops over the KV heads.  Warps encode key vectors (one token each), threads
-// encode value channels; the 3-bit codes meet in shared memory, where every thread assembles one
-// word triple of the record image; the image leaves with 16-byte stores.
+// One thread-block cluster per page, its blocks sharing out the KV heads (block r takes heads r,
+// r + cluster size, ...); the cluster's barrier orders every head's record before the page is
+// published.  Warps encode key vectors (one token each), threads encode value channels; the 3-bit
+// codes meet in shared memory, where every thread assembles one word triple of the record image; the
+// image leaves with 16-byte stores.
 //
 // Shared layout: key codes [token][D + 8] (the 8 pad bytes spread the token rows over the banks for
 // the packers, which read rows g and g + 8), value codes [channel][16 tokens], and two record images
@@ -218,12 +268,11 @@ __global__ void __launch_bounds__(D) demote_kernel(const uint8_t* __restrict__ f
     __shared__ __align__(16) uint8_t vcode[D * kPage];
     __shared__ __align__(16) uint8_t image[2][REC];
 
-    const int page = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int csize = (int)cluster_size(), crank = (int)cluster_rank();
+    const int page = blockIdx.x / csize, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int src = src_ids[page], dst = dst_ids[page];
-    if (src < 0 || src >= fp8_pages || dst < 0 || dst >= tq3_pages) {
-        if (tid == 0) atomicOr(status, kStBounds);
-        return;
-    }
+    const bool valid = src >= 0 && src < fp8_pages && dst >= 0 && dst < tq3_pages;
+    if (!valid && tid == 0 && crank == 0) atomicOr(status, kStBounds);
     // squared levels (single fp32 products, as the record's norm correction defines them)
     const float c0sq = __fmul_rn(MKV_C0, MKV_C0), c1sq = __fmul_rn(MKV_C1, MKV_C1),
                 c2sq = __fmul_rn(MKV_C2, MKV_C2), c3sq = __fmul_rn(MKV_C3, MKV_C3);
@@ -238,10 +287,10 @@ __global__ void __launch_bounds__(D) demote_kernel(const uint8_t* __restrict__ f
 #pragma unroll
     for (int b = 0; b < 5; ++b) neg[b] = ((lane >> b) & 1u) << 31;
 
-    for (int h = 0; h < hkv; ++h) {
+    for (int h = crank, it = 0; valid && h < hkv; h += csize, ++it) {
         const uint8_t* rec8 = fp8 + ((size_t)src * hkv + h) * fp8_record_bytes(D);
         uint8_t* rec3 = tq3 + ((size_t)dst * hkv + h) * tq3_record_bytes(D);
-        uint8_t* img = image[h & 1];
+        uint8_t* img = image[it & 1];
 
         // ---- keys: warp w encodes tokens w, w + NT/32, ... ------------------------------------------
         for (int tok = warp; tok < kPage; tok += NT / 32) {
@@ -416,10 +465,10 @@ __global__ void __launch_bounds__(D) demote_kernel(const uint8_t* __restrict__ f
             reinterpret_cast<uint4*>(rec3)[i] = reinterpret_cast<const uint4*>(img)[i];
     }
 
-    // copy-before-publish: the record is complete and visible before its id and tag appear
+    // copy-before-publish: every head's record is complete and visible before the id and tag appear
     __threadfence();
-    __syncthreads();
-    if (tid == 0 && entry_index != nullptr) {
+    cluster_barrier();
+    if (valid && crank == 0 && tid == 0 && entry_index != nullptr) {
         const int64_t e = entry_index[page];
         if (e >= 0) {
             block_table[e] = dst;
@@ -432,21 +481,22 @@ __global__ void __launch_bounds__(D) demote_kernel(const uint8_t* __restrict__ f
 int32_t launch_demote(mkv_pool* p, const int32_t* src, const int32_t* dst, int n, int32_t* bt, uint8_t* tags,
                       const int64_t* entry, cudaStream_t s)
 {
+    const int c = heads_cluster(p->hkv, n);
     if (p->d == 128)
-        demote_kernel<128><<<n, 128, 0, s>>>(p->fp8, p->tq3, p->cfg.fp8_pages, p->cfg.tq3_pages, p->hkv,
-                                             p->cfg.k_scale, p->cfg.v_scale, p->sigma, src, dst, bt, tags, entry,
-                                             p->status_dev);
+        MKV_CUDA(launch_clustered(demote_kernel<128>, n, c, 128, s, (const uint8_t*)p->fp8, p->tq3, p->cfg.fp8_pages,
+                                  p->cfg.tq3_pages, p->hkv, p->cfg.k_scale, p->cfg.v_scale, p->sigma, src, dst, bt, tags,
+                                  entry, p->status_dev));
     else
-        demote_kernel<256><<<n, 256, 0, s>>>(p->fp8, p->tq3, p->cfg.fp8_pages, p->cfg.tq3_pages, p->hkv,
-                                             p->cfg.k_scale, p->cfg.v_scale, p->sigma, src, dst, bt, tags, entry,
-                                             p->status_dev);
-    MKV_CUDA(cudaGetLastError());
+        MKV_CUDA(launch_clustered(demote_kernel<256>, n, c, 256, s, (const uint8_t*)p->fp8, p->tq3, p->cfg.fp8_pages,
+                                  p->cfg.tq3_pages, p->hkv, p->cfg.k_scale, p->cfg.v_scale, p->sigma, src, dst, bt, tags,
+                                  entry, p->status_dev));
     return MKV_OK;
 }
 
 // ------------------------------------------------------------------------------------------ promote
 // Promote (Algorithm 1 step 3): reconstruct a Stale page into a newly allocated FP8 page, then publish
-// it as Anchor.  One block per page, loops over the KV heads.  The record is staged in shared memory;
+// it as Anchor.  One cluster per page, its blocks sharing out the KV heads as in demote_kernel.  The
+// record is staged in shared memory;
 // warps rebuild key vectors (signed levels, shuffle Walsh-Hadamard, norm correction, sign), threads
 // rebuild value channels; the fp32 operation order is fixed so that the written bytes are reproducible.
 //
@@ -469,12 +519,11 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
     __shared__ __align__(16) uint8_t image[2][REC];
     __shared__ float level[8];            // signed key levels by 3-bit code
 
-    const int page = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int csize = (int)cluster_size(), crank = (int)cluster_rank();
+    const int page = blockIdx.x / csize, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int src = src_ids[page], dst = dst_ids[page];
-    if (src < 0 || src >= tq3_pages || dst < 0 || dst >= fp8_pages) {
-        if (tid == 0) atomicOr(status, kStBounds);
-        return;
-    }
+    const bool valid = src >= 0 && src < tq3_pages && dst >= 0 && dst < fp8_pages;
+    if (!valid && tid == 0 && crank == 0) atomicOr(status, kStBounds);
     if (tid < 8) {
         const float c = (tid & 3) == 0 ? MKV_C0 : (tid & 3) == 1 ? MKV_C1 : (tid & 3) == 2 ? MKV_C2 : MKV_C3;
         level[tid] = (tid & 4) ? -c : c;
@@ -508,10 +557,10 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
     const uint32_t sel0 = grp == 0 ? 0x0410u : 0x0541u, sel1 = grp == 0 ? 0x0632u : 0x0763u;
     const int meta_i = (cb >> 1) * 64 + (row & 7) * 8 + 4 * (cb & 1) + (row >> 3);
 
-    for (int h = 0; h < hkv; ++h) {
+    for (int h = crank, it = 0; valid && h < hkv; h += csize, ++it) {
         const uint8_t* rec3 = tq3 + ((size_t)src * hkv + h) * tq3_record_bytes(D);
         uint8_t* rec8 = fp8 + ((size_t)dst * hkv + h) * fp8_record_bytes(D);
-        uint8_t* img = image[h & 1];
+        uint8_t* img = image[it & 1];
         for (int i = tid; i < REC / 16; i += NT)
             reinterpret_cast<uint4*>(img)[i] = reinterpret_cast<const uint4*>(rec3)[i];
         __syncthreads();
@@ -592,8 +641,8 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
     }
     // copy-before-publish
     __threadfence();
-    __syncthreads();
-    if (tid == 0 && entry_index != nullptr) {
+    cluster_barrier();
+    if (valid && crank == 0 && tid == 0 && entry_index != nullptr) {
         const int64_t e = entry_index[page];
         if (e >= 0) {
             block_table[e] = dst;
@@ -608,13 +657,13 @@ int32_t launch_promote(mkv_pool* p, const int32_t* src, const int32_t* dst, int 
 {
     const float ik = 1.0f / p->cfg.k_scale, iv = 1.0f / p->cfg.v_scale;
     const float rs = (float)(1.0 / sqrt((double)p->d));
+    const int c = heads_cluster(p->hkv, n);
     if (p->d == 128)
-        promote_kernel<128><<<n, 128, 0, s>>>(p->tq3, p->fp8, p->cfg.tq3_pages, p->cfg.fp8_pages, p->hkv, ik, iv, rs,
-                                              p->sigma, src, dst, bt, tags, entry, p->status_dev);
+        MKV_CUDA(launch_clustered(promote_kernel<128>, n, c, 128, s, (const uint8_t*)p->tq3, p->fp8, p->cfg.tq3_pages,
+                                  p->cfg.fp8_pages, p->hkv, ik, iv, rs, p->sigma, src, dst, bt, tags, entry, p->status_dev));
     else
-        promote_kernel<256><<<n, 256, 0, s>>>(p->tq3, p->fp8, p->cfg.tq3_pages, p->cfg.fp8_pages, p->hkv, ik, iv, rs,
-                                              p->sigma, src, dst, bt, tags, entry, p->status_dev);
-    MKV_CUDA(cudaGetLastError());
+        MKV_CUDA(launch_clustered(promote_kernel<256>, n, c, 256, s, (const uint8_t*)p->tq3, p->fp8, p->cfg.tq3_pages,
+                                  p->cfg.fp8_pages, p->hkv, ik, iv, rs, p->sigma, src, dst, bt, tags, entry, p->status_dev));
     return MKV_OK;
 }
 

@@ -218,3 +218,75 @@ def test_promote_is_bit_exact_and_publishes_anchor(d, hkv, k_scale, v_scale):
     assert (btc[0::2] == -1).all() and (tc[0::2] == 2).all()
     pool.promote(torch.tensor([99], dtype=torch.int32, device="cuda:0"), torch.tensor([0], dtype=torch.int32, device="cuda:0"))
     assert pool.status() == M.E_BOUNDS
+
+
+@pytest.mark.parametrize("d,hkv", [(128, 1), (128, 3), (256, 6), (128, 12), (256, 16)])
+def test_demote_then_promote_for_every_head_split(d, hkv):
+    """The blocks of a page's cluster share out the KV heads (1, 3, 6 blocks of one head; 6 blocks of two;
+    8 blocks of two): every head's record is bit-exact both ways and both calls publish once."""
+    rng = np.random.default_rng(300 + d + hkv)
+    n = 5
+    sigma = (rng.integers(0, 2, d) * 2 - 1).astype(np.int8)
+    pool = M.Pool(d, hkv, hkv, 2 * n, n, sigma)
+    recs = np.zeros((n, hkv, 32 * d), np.uint8)
+    for p in range(n):
+        for h in range(hkv):
+            k = rng.standard_normal((16, d)).astype(np.float32) * (1 + h)
+            v = rng.standard_normal((16, d)).astype(np.float32)
+            v[:, rng.integers(0, d, 2)] *= 8
+            recs[p, h] = oracle.fp8_pack_record(k, v, 16, 1.0, 1.0)
+        pool.page_write_raw(M.FMT_FP8, p, recs[p])
+    ids = torch.arange(n, dtype=torch.int32, device="cuda:0")
+    bt = torch.full((1, n), -1, dtype=torch.int32, device="cuda:0")
+    tags = torch.zeros((1, n), dtype=torch.uint8, device="cuda:0")
+    entry = torch.arange(n, dtype=torch.int64, device="cuda:0")
+    pool.demote(ids, ids.flip(0).contiguous(), bt, tags, entry)
+    torch.cuda.synchronize()
+    assert pool.status() == M.OK
+    assert bt.cpu().numpy().tolist() == [list(range(n - 1, -1, -1))] and (tags.cpu().numpy() == M.TAG_STALE).all()
+    stale = np.zeros((n, hkv, 16 * d + 32), np.uint8)
+    for p in range(n):
+        stale[p] = pool.page_read_raw(M.FMT_TQ3, n - 1 - p).reshape(hkv, -1)
+        for h in range(hkv):
+            assert np.array_equal(stale[p, h], oracle.demote_record(recs[p, h], d, sigma, 1.0, 1.0)), (p, h)
+    pool.promote(ids.flip(0).contiguous(), ids + n, bt, tags, entry)
+    torch.cuda.synchronize()
+    assert pool.status() == M.OK
+    assert bt.cpu().numpy().tolist() == [list(range(n, 2 * n))] and (tags.cpu().numpy() == M.TAG_ANCHOR).all()
+    for p in range(n):
+        got = pool.page_read_raw(M.FMT_FP8, n + p).reshape(hkv, 32 * d)
+        for h in range(hkv):
+            assert np.array_equal(got[h], oracle.promote_record(stale[p, h], d, sigma, 1.0, 1.0)), (p, h)
+
+
+@pytest.mark.parametrize("d,hkv", [(128, 8), (256, 4)])
+def test_bulk_calls_write_the_same_bytes_as_small_calls(d, hkv):
+    """A call of hundreds of pages keeps a page's heads in one block, a call of a few pages spreads them
+    over a cluster: both layouts of the work must produce identical arenas (and match the oracle)."""
+    rng = np.random.default_rng(400 + d)
+    n = 320
+    sigma = (rng.integers(0, 2, d) * 2 - 1).astype(np.int8)
+    pool = M.Pool(d, hkv, hkv, 2 * n, 2 * n, sigma)
+    k, v = bf16_tensor(special_bf16(rng, (16 * n, hkv, d))), bf16_tensor(special_bf16(rng, (16 * n, hkv, d)))
+    pool.append(k, v, torch.arange(16 * n, dtype=torch.int32, device="cuda:0"))
+    ids = torch.arange(n, dtype=torch.int32, device="cuda:0")
+    pool.demote(ids, ids)                                   # one bulk call -> TQ3 pages 0 .. n-1
+    for lo in range(0, n, 8):                               # small calls -> TQ3 pages n .. 2n-1
+        pool.demote(ids[lo:lo + 8], (ids[lo:lo + 8] + n).contiguous())
+    pool.promote(ids, (ids + n).contiguous())               # bulk -> FP8 pages n .. 2n-1
+    torch.cuda.synchronize()
+    assert pool.status() == M.OK
+    rec3 = hkv * (16 * d + 32)
+    tq3 = pool.tq3_arena[:2 * n * rec3].view(2, n * rec3)
+    assert torch.equal(tq3[0], tq3[1])
+    rec8 = hkv * 32 * d
+    bulk_fp8 = pool.fp8_arena[n * rec8:2 * n * rec8].clone()
+    for lo in range(0, n, 8):                               # small promote calls over the same target pages
+        pool.promote((ids[lo:lo + 8] + n).contiguous(), (ids[lo:lo + 8] + n).contiguous())
+    torch.cuda.synchronize()
+    assert torch.equal(bulk_fp8, pool.fp8_arena[n * rec8:2 * n * rec8])
+    for p in (0, 157, n - 1):
+        src = pool.page_read_raw(M.FMT_FP8, p).reshape(hkv, 32 * d)
+        got = pool.page_read_raw(M.FMT_TQ3, p).reshape(hkv, -1)
+        for h in range(hkv):
+            assert np.array_equal(got[h], oracle.demote_record(src[h], d, sigma, 1.0, 1.0)), (p, h)
