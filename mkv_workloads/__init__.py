@@ -55,6 +55,7 @@ class Spec:
     recent_tokens: int              # Recent window at the end of the context
     n_outlier: int                  # channels scaled x8, drawn per layer and per tensor
     stale_fraction: Optional[float] = None   # lifecycle sweep: oldest floor(f*P) pages Stale, rest Recent
+    page_tokens: int = T            # tokens per page: 16, or 16 M for the paper-scale blocks (1,792 / 832)
 
     @property
     def n_q_heads(self) -> int:
@@ -65,7 +66,11 @@ class Spec:
         return float(1.0 / np.sqrt(np.float64(self.head_dim)))
 
     def n_pages(self, b: int) -> int:
-        return (self.seq_lens[b] + T - 1) // T
+        return (self.seq_lens[b] + self.page_tokens - 1) // self.page_tokens
+
+    @property
+    def tiles_per_page(self) -> int:
+        return self.page_tokens // T
 
     @property
     def max_pages(self) -> int:
@@ -92,8 +97,13 @@ def config(idx: int, **over) -> Spec:
         frac = over.pop("stale_fraction", 0.5)
         s = Spec(f"cfg4_lifecycle_b{batch}_c{ctx}_f{frac}", 4, batch, 1, 128, 8, 4, (ctx,) * batch,
                  0, 0, 0, 0, 3, stale_fraction=frac)
+    elif idx == 5:
+        # the canary's shape with pages of 1,792 tokens (the block size its byte counters were taken at):
+        # 33 pages per request = 1 first-tokens Anchor + 3 Anchor spans + 6 Recent (FP8) + 23 Stale (TQ3)
+        s = Spec("cfg5_canary_blocks_1792", 5, 2, 1, 256, 4, 6, (59008,) * 2, 1792, 3, 1792, 5 * 1792, 5,
+                 page_tokens=1792)
     else:
-        raise ValueError("config index 0..4")
+        raise ValueError("config index 0..5")
     if "seq_lens" in over:
         over["seq_lens"] = tuple(int(x) for x in over["seq_lens"])
         over.setdefault("batch", len(over["seq_lens"]))
@@ -107,18 +117,19 @@ def tier_tags(spec: Spec, b: int) -> np.ndarray:
     """Tier tag (0 Recent, 1 Anchor, 2 Stale) of every logical page of request b."""
     n = spec.n_pages(b)
     ln = spec.seq_lens[b]
+    Tp = spec.page_tokens
     tags = np.full(n, TAG_STALE, np.uint8)
     if spec.stale_fraction is not None:
         n_stale = int(np.floor(spec.stale_fraction * n))
         tags[n_stale:] = TAG_RECENT
     else:
         rng = _rng(spec.seed, 1, b)
-        n_anchor = min(n, spec.anchor_prefix // T)
+        n_anchor = min(n, spec.anchor_prefix // Tp)
         tags[:n_anchor] = TAG_ANCHOR
-        first_recent = max(0, ln - spec.recent_tokens) // T   # pages covering the last tokens
+        first_recent = max(0, ln - spec.recent_tokens) // Tp   # pages covering the last tokens
         tags[first_recent:] = TAG_RECENT
         n_spans = spec.anchor_spans if spec.anchor_spans >= 0 else int(rng.integers(1, 5))
-        span = spec.anchor_span_tokens // T
+        span = spec.anchor_span_tokens // Tp
         placed, tries = 0, 0
         while placed < n_spans and span > 0 and tries < 1000:
             tries += 1
@@ -128,7 +139,7 @@ def tier_tags(spec: Spec, b: int) -> np.ndarray:
             if np.all(tags[start:start + span] == TAG_STALE):      # re-draw on collision
                 tags[start:start + span] = TAG_ANCHOR
                 placed += 1
-    if ln % T != 0 and n and tags[-1] == TAG_STALE:
+    if ln % Tp != 0 and n and tags[-1] == TAG_STALE:
         tags[-1] = TAG_RECENT        # a partial (still open) page is never Stale
     return tags
 
@@ -202,11 +213,12 @@ def new_token_kv(spec: Spec, layer: int, step: int = 0) -> Tuple[np.ndarray, np.
 
 def kv_bytes(spec: Spec, tab: Tables) -> int:
     """Algorithmic KV bytes one decode step of ONE layer must read: 2*d bytes per valid FP8 token and
-    16*d + 32 bytes per Stale page, per KV head (queries, outputs, tables and workspace excluded)."""
-    d, total = spec.head_dim, 0
+    M (12 d + 32) + 4 d bytes per Stale page of 16 M tokens (16 d + 32 at M = 1), per KV head (queries,
+    outputs, tables and workspace excluded)."""
+    d, total, M = spec.head_dim, 0, spec.tiles_per_page
     for b in range(spec.batch):
         n = spec.n_pages(b)
         stale = int((tab.tier_tag[b, :n] == TAG_STALE).sum())
-        fp8_tokens = spec.seq_lens[b] - stale * T
-        total += spec.n_kv_heads * (fp8_tokens * 2 * d + stale * (16 * d + 32))
+        fp8_tokens = spec.seq_lens[b] - stale * spec.page_tokens
+        total += spec.n_kv_heads * (fp8_tokens * 2 * d + stale * (M * (12 * d + 32) + 4 * d))
     return total

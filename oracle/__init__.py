@@ -94,6 +94,33 @@ def lib():
         L.orc_encode_request.restype = C.c_int
         L.orc_encode_request.argtypes = [C.c_int, C.c_int, C.c_int, u16p, u16p, i32p, u8p, i8p,
                                          C.c_float, C.c_float, u8p, u8p]
+        L.orc_fp8_block_bytes.restype = C.c_int64
+        L.orc_fp8_block_bytes.argtypes = [C.c_int, C.c_int]
+        L.orc_tq3_block_bytes.restype = C.c_int64
+        L.orc_tq3_block_bytes.argtypes = [C.c_int, C.c_int]
+        L.orc_tq3_encode_value_block.restype = None
+        L.orc_tq3_encode_value_block.argtypes = [f32p, C.c_int, C.c_int, u8p, u16p, u16p]
+        L.orc_tq3_pack_block.restype = None
+        L.orc_tq3_pack_block.argtypes = [C.c_int, C.c_int, u8p, u16p, u8p, u16p, u16p, u8p]
+        L.orc_tq3_unpack_block.restype = None
+        L.orc_tq3_unpack_block.argtypes = [C.c_int, C.c_int, u8p, u8p, u16p, u8p, u16p, u16p]
+        L.orc_tq3_block_from_f32.restype = None
+        L.orc_tq3_block_from_f32.argtypes = [C.c_int, C.c_int, f32p, f32p, i8p, u8p]
+        L.orc_fp8_pack_block.restype = None
+        L.orc_fp8_pack_block.argtypes = [C.c_int, C.c_int, f32p, f32p, C.c_int, C.c_float, C.c_float, u8p]
+        L.orc_fp8_unpack_block_f32.restype = None
+        L.orc_fp8_unpack_block_f32.argtypes = [C.c_int, C.c_int, u8p, C.c_float, C.c_float, f32p, f32p]
+        L.orc_demote_block.restype = None
+        L.orc_demote_block.argtypes = [C.c_int, C.c_int, u8p, C.c_float, C.c_float, i8p, u8p]
+        L.orc_promote_block.restype = None
+        L.orc_promote_block.argtypes = [C.c_int, C.c_int, u8p, C.c_float, C.c_float, i8p, u8p]
+        L.orc_decode_attention_blocks.restype = C.c_int
+        L.orc_decode_attention_blocks.argtypes = [u8p, C.c_int64, u8p, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int,
+                                                  C.c_float, C.c_float, i8p, u16p, i32p, u8p, i32p, C.c_int,
+                                                  C.c_int, C.c_double, f64p, f64p, C.c_int, C.c_int, C.c_int]
+        L.orc_encode_request_blocks.restype = C.c_int
+        L.orc_encode_request_blocks.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, u16p, u16p, i32p, u8p, i8p,
+                                                C.c_float, C.c_float, u8p, u8p]
         L.orc_kv_bytes_per_token.restype = C.c_int64
         L.orc_kv_bytes_per_token.argtypes = [C.c_int] * 4
         L.orc_page_bytes_dense.restype = C.c_int64
@@ -266,6 +293,92 @@ def tq3_record_from_f32(k: np.ndarray, v: np.ndarray, sigma: np.ndarray) -> np.n
     return out
 
 
+# ---------------------------------------------------------------------------- pages of 16 M tokens
+def fp8_block_bytes(d: int, M: int) -> int:
+    return lib().orc_fp8_block_bytes(d, M)
+
+
+def tq3_block_bytes(d: int, M: int) -> int:
+    """M (12 d + 32) + 4 d: M tiles of key codes, value codes and g, one scale/zero set per page."""
+    return lib().orc_tq3_block_bytes(d, M)
+
+
+def tq3_encode_value_block(v: np.ndarray):
+    """Values of one full page (fp32 [T][d], any T) -> (codes uint8 [T][d], scale fp16 bits [d], zero fp16 bits [d]);
+    one scale/zero per channel over all T tokens."""
+    v = _c(v, np.float32)
+    Tn, d = v.shape
+    code = np.zeros((Tn, d), np.uint8)
+    sc = np.zeros(d, np.uint16)
+    zp = np.zeros(d, np.uint16)
+    lib().orc_tq3_encode_value_block(_p(v, C.c_float), d, Tn, _p(code, C.c_uint8), _p(sc, C.c_uint16), _p(zp, C.c_uint16))
+    return code, sc, zp
+
+
+def tq3_pack_block(kcode, g, vcode, sc, zp) -> np.ndarray:
+    kcode, vcode = _c(kcode, np.uint8), _c(vcode, np.uint8)
+    g, sc, zp = _c(g, np.uint16), _c(sc, np.uint16), _c(zp, np.uint16)
+    Tn, d = kcode.shape
+    assert Tn % T == 0
+    rec = np.zeros(tq3_block_bytes(d, Tn // T), np.uint8)
+    lib().orc_tq3_pack_block(d, Tn // T, _p(kcode, C.c_uint8), _p(g, C.c_uint16), _p(vcode, C.c_uint8),
+                             _p(sc, C.c_uint16), _p(zp, C.c_uint16), _p(rec, C.c_uint8))
+    return rec
+
+
+def tq3_unpack_block(rec: np.ndarray, d: int, M: int):
+    rec = _c(rec, np.uint8)
+    kcode = np.zeros((T * M, d), np.uint8)
+    vcode = np.zeros((T * M, d), np.uint8)
+    g = np.zeros(T * M, np.uint16)
+    sc = np.zeros(d, np.uint16)
+    zp = np.zeros(d, np.uint16)
+    lib().orc_tq3_unpack_block(d, M, _p(rec, C.c_uint8), _p(kcode, C.c_uint8), _p(g, C.c_uint16),
+                               _p(vcode, C.c_uint8), _p(sc, C.c_uint16), _p(zp, C.c_uint16))
+    return kcode, g, vcode, sc, zp
+
+
+def tq3_block_from_f32(k: np.ndarray, v: np.ndarray, sigma: np.ndarray) -> np.ndarray:
+    k, v, sigma = _c(k, np.float32), _c(v, np.float32), _c(sigma, np.int8)
+    Tn, d = k.shape
+    assert Tn % T == 0 and v.shape == k.shape
+    out = np.zeros(tq3_block_bytes(d, Tn // T), np.uint8)
+    lib().orc_tq3_block_from_f32(d, Tn // T, _p(k, C.c_float), _p(v, C.c_float), _p(sigma, C.c_int8), _p(out, C.c_uint8))
+    return out
+
+
+def fp8_pack_block(k: np.ndarray, v: np.ndarray, n_valid=None, k_scale=1.0, v_scale=1.0) -> np.ndarray:
+    k, v = _c(k, np.float32), _c(v, np.float32)
+    Tn, d = k.shape
+    assert Tn % T == 0
+    out = np.zeros(fp8_block_bytes(d, Tn // T), np.uint8)
+    lib().orc_fp8_pack_block(d, Tn // T, _p(k, C.c_float), _p(v, C.c_float), Tn if n_valid is None else n_valid,
+                             k_scale, v_scale, _p(out, C.c_uint8))
+    return out
+
+
+def fp8_unpack_block_f32(rec: np.ndarray, d: int, M: int, k_scale=1.0, v_scale=1.0):
+    rec = _c(rec, np.uint8)
+    k = np.zeros((T * M, d), np.float32)
+    v = np.zeros((T * M, d), np.float32)
+    lib().orc_fp8_unpack_block_f32(d, M, _p(rec, C.c_uint8), k_scale, v_scale, _p(k, C.c_float), _p(v, C.c_float))
+    return k, v
+
+
+def demote_block(fp8_block: np.ndarray, d: int, M: int, sigma: np.ndarray, k_scale=1.0, v_scale=1.0) -> np.ndarray:
+    fp8_block, sigma = _c(fp8_block, np.uint8), _c(sigma, np.int8)
+    out = np.zeros(tq3_block_bytes(d, M), np.uint8)
+    lib().orc_demote_block(d, M, _p(fp8_block, C.c_uint8), k_scale, v_scale, _p(sigma, C.c_int8), _p(out, C.c_uint8))
+    return out
+
+
+def promote_block(tq3_block: np.ndarray, d: int, M: int, sigma: np.ndarray, k_scale=1.0, v_scale=1.0) -> np.ndarray:
+    tq3_block, sigma = _c(tq3_block, np.uint8), _c(sigma, np.int8)
+    out = np.zeros(fp8_block_bytes(d, M), np.uint8)
+    lib().orc_promote_block(d, M, _p(tq3_block, C.c_uint8), k_scale, v_scale, _p(sigma, C.c_int8), _p(out, C.c_uint8))
+    return out
+
+
 # ---------------------------------------------------------------------------- bulk page encoding
 def encode_fp8_pages(k_bits: np.ndarray, v_bits: np.ndarray, n_valid: int = T, k_scale=1.0,
                      v_scale=1.0) -> np.ndarray:
@@ -288,8 +401,9 @@ def encode_tq3_pages(k_bits: np.ndarray, v_bits: np.ndarray, sigma: np.ndarray) 
     return out
 
 
-def encode_request(k_bits, v_bits, row, tags, sigma, fp8_arena, tq3_arena, k_scale=1.0, v_scale=1.0):
-    """Write all pages of one request (bf16 bits [len][hkv][d]) into the uint8 arenas in place."""
+def encode_request(k_bits, v_bits, row, tags, sigma, fp8_arena, tq3_arena, k_scale=1.0, v_scale=1.0, page_tokens=T):
+    """Write all pages of one request (bf16 bits [len][hkv][d]) into the uint8 arenas in place
+    (pages of `page_tokens` = 16 M tokens)."""
     k_bits = _c(k_bits, np.uint16)
     v_bits = _c(v_bits, np.uint16)
     row = _c(row, np.int32)
@@ -299,7 +413,8 @@ def encode_request(k_bits, v_bits, row, tags, sigma, fp8_arena, tq3_arena, k_sca
     assert fp8_arena.dtype == np.uint8 and fp8_arena.flags.c_contiguous
     assert tq3_arena.dtype == np.uint8 and tq3_arena.flags.c_contiguous
     dummy = np.zeros(16, np.uint8)
-    rc = lib().orc_encode_request(d, hkv, ln, _p(k_bits, C.c_uint16), _p(v_bits, C.c_uint16),
+    assert page_tokens % T == 0 and page_tokens >= T
+    rc = lib().orc_encode_request_blocks(d, hkv, ln, page_tokens // T, _p(k_bits, C.c_uint16), _p(v_bits, C.c_uint16),
                                   _p(row, C.c_int32), _p(tags, C.c_uint8), _p(sigma, C.c_int8),
                                   k_scale, v_scale,
                                   _p(fp8_arena if fp8_arena.size else dummy, C.c_uint8),
@@ -310,13 +425,15 @@ def encode_request(k_bits, v_bits, row, tags, sigma, fp8_arena, tq3_arena, k_sca
 
 # ---------------------------------------------------------------------------- attention
 def decode_attention(fp8_arena, tq3_arena, d, hkv, group, sigma, q_bits, block_table, tier_tag,
-                     seq_lens, scale, k_scale=1.0, v_scale=1.0, mode=0, only_b=-1, only_h=-1):
+                     seq_lens, scale, k_scale=1.0, v_scale=1.0, mode=0, only_b=-1, only_h=-1, page_tokens=T):
     """Dequantise-then-attend in fp64 (Section 3.3).  Returns (out [B][Hq][d], lse [B][Hq]).
 
     fp8_arena: uint8 [fp8_pages][hkv][32d]; tq3_arena: uint8 [tq3_pages][hkv][16d+32];
     q_bits: bf16 bits [B][Hq][d]; block_table int32 [B][max_pages]; tier_tag uint8 [B][max_pages].
     mode 0 = one softmax; 1 = Eq. (softmax-merge) over the two format partitions;
     n >= 2 = Eq. (softmax-merge) over n contiguous ranges.
+    page_tokens = 16 M: pages of M tiles (arenas then hold [pages][hkv][M * 32d] and
+    [pages][hkv][M * (12d + 32) + 4d] bytes).
     """
     fp8_arena = _c(fp8_arena, np.uint8)
     tq3_arena = _c(tq3_arena, np.uint8)
@@ -328,14 +445,16 @@ def decode_attention(fp8_arena, tq3_arena, d, hkv, group, sigma, q_bits, block_t
     B, max_pages = block_table.shape
     Hq = hkv * group
     assert q_bits.shape == (B, Hq, d)
-    fp8_pages = fp8_arena.size // (hkv * fp8_record_bytes(d)) if fp8_arena.size else 0
-    tq3_pages = tq3_arena.size // (hkv * tq3_record_bytes(d)) if tq3_arena.size else 0
+    assert page_tokens % T == 0 and page_tokens >= T
+    M = page_tokens // T
+    fp8_pages = fp8_arena.size // (hkv * fp8_block_bytes(d, M)) if fp8_arena.size else 0
+    tq3_pages = tq3_arena.size // (hkv * tq3_block_bytes(d, M)) if tq3_arena.size else 0
     out = np.zeros((B, Hq, d), np.float64)
     lse = np.zeros((B, Hq), np.float64)
     dummy = np.zeros(16, np.uint8)
-    rc = lib().orc_decode_attention(
+    rc = lib().orc_decode_attention_blocks(
         _p(fp8_arena if fp8_arena.size else dummy, C.c_uint8), fp8_pages,
-        _p(tq3_arena if tq3_arena.size else dummy, C.c_uint8), tq3_pages, d, hkv, group,
+        _p(tq3_arena if tq3_arena.size else dummy, C.c_uint8), tq3_pages, d, hkv, group, M,
         k_scale, v_scale, _p(sigma, C.c_int8), _p(q_bits, C.c_uint16), _p(block_table, C.c_int32),
         _p(tier_tag, C.c_uint8), _p(seq_lens, C.c_int32), B, max_pages, float(scale),
         _p(out, C.c_double), _p(lse, C.c_double), mode, only_b, only_h)

@@ -11,24 +11,26 @@ import numpy as np
 
 import mkv_workloads as W
 
-from . import encode_request, fp8_record_bytes, tq3_record_bytes
+from . import encode_request, fp8_block_bytes, tq3_block_bytes
 
 
 @dataclass
 class LayerArrays:
-    fp8_arena: np.ndarray     # uint8 [fp8_pages][hkv][32d]
-    tq3_arena: np.ndarray     # uint8 [tq3_pages][hkv][16d+32]
+    fp8_arena: np.ndarray     # uint8 [fp8_pages][hkv][M * 32d]            (M = tiles of 16 tokens per page)
+    tq3_arena: np.ndarray     # uint8 [tq3_pages][hkv][M * (12d + 32) + 4d]  (16d + 32 at M = 1)
     sigma: np.ndarray         # int8 [d]
     q_bits: np.ndarray        # uint16 [B][Hq][d]
 
 
 def build_layer(spec: W.Spec, tab: W.Tables, layer: int = 0, requests=None) -> LayerArrays:
     d, hkv = spec.head_dim, spec.n_kv_heads
-    fp8 = np.zeros((max(tab.fp8_pages, 1), hkv, fp8_record_bytes(d)), np.uint8)
-    tq3 = np.zeros((max(tab.tq3_pages, 1), hkv, tq3_record_bytes(d)), np.uint8)
+    M = spec.tiles_per_page
+    fp8 = np.zeros((max(tab.fp8_pages, 1), hkv, fp8_block_bytes(d, M)), np.uint8)
+    tq3 = np.zeros((max(tab.tq3_pages, 1), hkv, tq3_block_bytes(d, M)), np.uint8)
     sigma = W.rotation_signs(spec, layer)
     for b in (range(spec.batch) if requests is None else requests):
         k_bits, v_bits = W.kv(spec, layer, b)
         n = spec.n_pages(b)
-        encode_request(k_bits, v_bits, tab.block_table[b, :n], tab.tier_tag[b, :n], sigma, fp8, tq3)
+        encode_request(k_bits, v_bits, tab.block_table[b, :n], tab.tier_tag[b, :n], sigma, fp8, tq3,
+                       page_tokens=spec.page_tokens)
     return LayerArrays(fp8, tq3, sigma, W.query(spec, layer))

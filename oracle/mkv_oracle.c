@@ -184,16 +184,17 @@ void orc_tq3_decode_key(const uint8_t* code, uint16_t g, int d, const int8_t* si
     for (i = 0; i < d; ++i) out[i] = gg * rs * (sigma[i] < 0 ? -y[i] : y[i]);
 }
 
-/* TQ3 value encoder for one full page: v[t*d + c], t < 16.  Asymmetric uniform 3-bit quantiser
- * per channel over the 16 tokens of the page; scale and zero stored as fp16. */
-void orc_tq3_encode_value_page(const float* v, int d, uint8_t* code /*[16*d] token-major*/,
-                               uint16_t* sc /*[d]*/, uint16_t* zp /*[d]*/)
+/* TQ3 value encoder for one full page of T tokens: v[t*d + c], t < T.  Asymmetric uniform 3-bit
+ * quantiser per channel over ALL tokens of the page; scale and zero stored as fp16 (Section 4.1:
+ * "three-bit value codes, and FP16 scale/zero" per Stale page and KV head). */
+void orc_tq3_encode_value_block(const float* v, int d, int T, uint8_t* code /*[T*d] token-major*/,
+                                uint16_t* sc /*[d]*/, uint16_t* zp /*[d]*/)
 {
     int c, t;
     for (c = 0; c < d; ++c) {
         float mn = v[c], mx = v[c], scf, zpf;
-        for (t = 1; t < ORC_T; ++t) {
-            float u = v[t * d + c];
+        for (t = 1; t < T; ++t) {
+            float u = v[(int64_t)t * d + c];
             if (u < mn) mn = u;
             if (u > mx) mx = u;
         }
@@ -201,17 +202,24 @@ void orc_tq3_encode_value_page(const float* v, int d, uint8_t* code /*[16*d] tok
         zp[c] = orc_f32_to_f16_sat(mn);
         scf = orc_f16_to_f32(sc[c]);
         zpf = orc_f16_to_f32(zp[c]);
-        for (t = 0; t < ORC_T; ++t) {
+        for (t = 0; t < T; ++t) {
             int q = 0;
             if (scf != 0.0f) {
-                float r = rintf((v[t * d + c] - zpf) / scf); /* half to even */
+                float r = rintf((v[(int64_t)t * d + c] - zpf) / scf); /* half to even */
                 if (r < 0.0f) r = 0.0f;
                 if (r > 7.0f) r = 7.0f;
                 q = (int)r;
             }
-            code[t * d + c] = (uint8_t)q;
+            code[(int64_t)t * d + c] = (uint8_t)q;
         }
     }
+}
+
+/* the 16-token page */
+void orc_tq3_encode_value_page(const float* v, int d, uint8_t* code /*[16*d] token-major*/,
+                               uint16_t* sc /*[d]*/, uint16_t* zp /*[d]*/)
+{
+    orc_tq3_encode_value_block(v, d, ORC_T, code, sc, zp);
 }
 
 double orc_tq3_decode_value(uint8_t code, uint16_t sc, uint16_t zp)
@@ -424,6 +432,117 @@ void orc_tq3_record_from_f32(int d, const float* k, const float* v, const int8_t
 }
 
 /* ------------------------------------------------------------------------------------------
+ * Pages of T = 16 M tokens (Section 4.1: the measured prototype stores blocks of 1,792 tokens,
+ * the fast-arithmetic one blocks of 832; Section 5.4 counts their physical bytes).  A page is M
+ * tiles of 16 tokens.  Keys are coded per token, so a key tile is the key part of the 16-token
+ * record; value scale and zero are per channel over ALL T tokens of the page (one scale/zero
+ * pair per channel and page, which is what amortises the value metadata to ~3.04 bit/scalar).
+ *
+ *   FP8 page of (page, kv head), M * 32 d bytes: tile m = the 16-token FP8 record of tokens
+ *       [16 m, 16 m + 16) at offset m * 32 d.
+ *   TQ3 page of (page, kv head), M * (12 d + 32) + 4 d bytes: tile m at offset m * (12 d + 32)
+ *       = [key codes 6 d | value codes 6 d | g[16] 32 B] of its 16 tokens, laid out as in the
+ *       16-token record; then the page's value scale/zero (4 d bytes, same order as there).
+ *   M = 1 gives exactly the 16-token records.
+ * ---------------------------------------------------------------------------------------- */
+int64_t orc_fp8_block_bytes(int d, int M) { return (int64_t)M * orc_fp8_record_bytes(d); }
+int64_t orc_tq3_tile_bytes(int d) { return 12 * (int64_t)d + 32; }
+int64_t orc_tq3_block_bytes(int d, int M) { return M * orc_tq3_tile_bytes(d) + 4 * (int64_t)d; }
+
+void orc_tq3_pack_block(int d, int M, const uint8_t* kcode /*[16M][d]*/, const uint16_t* g /*[16M]*/,
+                        const uint8_t* vcode /*[16M][d]*/, const uint16_t* sc, const uint16_t* zp, uint8_t* rec)
+{
+    uint8_t* tmp = (uint8_t*)malloc((size_t)orc_tq3_record_bytes(d));
+    int64_t tile = orc_tq3_tile_bytes(d);
+    int m;
+    for (m = 0; m < M; ++m) {
+        orc_tq3_pack_record(d, kcode + (int64_t)m * ORC_T * d, g + m * ORC_T, vcode + (int64_t)m * ORC_T * d, sc, zp, tmp);
+        memcpy(rec + m * tile, tmp, (size_t)tile);
+    }
+    memcpy(rec + M * tile, tmp + tile, (size_t)(4 * d));     /* scale/zero: the same in every tile's record */
+    free(tmp);
+}
+
+void orc_tq3_unpack_block(int d, int M, const uint8_t* rec, uint8_t* kcode, uint16_t* g, uint8_t* vcode,
+                          uint16_t* sc, uint16_t* zp)
+{
+    uint8_t* tmp = (uint8_t*)malloc((size_t)orc_tq3_record_bytes(d));
+    int64_t tile = orc_tq3_tile_bytes(d);
+    int m;
+    for (m = 0; m < M; ++m) {
+        memcpy(tmp, rec + m * tile, (size_t)tile);
+        memcpy(tmp + tile, rec + M * tile, (size_t)(4 * d));
+        orc_tq3_unpack_record(d, tmp, kcode + (int64_t)m * ORC_T * d, g + m * ORC_T, vcode + (int64_t)m * ORC_T * d, sc, zp);
+    }
+    free(tmp);
+}
+
+/* TQ3 page straight from fp32 K,V of a full page of 16 M tokens (k[t*d+i], v[t*d+c]) */
+void orc_tq3_block_from_f32(int d, int M, const float* k, const float* v, const int8_t* sigma, uint8_t* rec)
+{
+    int T = ORC_T * M, t;
+    uint8_t* kc = (uint8_t*)malloc((size_t)T * d);
+    uint8_t* vc = (uint8_t*)malloc((size_t)T * d);
+    uint16_t* g = (uint16_t*)malloc(sizeof(uint16_t) * (size_t)T);
+    uint16_t sc[ORC_MAXD], zp[ORC_MAXD];
+    for (t = 0; t < T; ++t) orc_tq3_encode_key(k + (int64_t)t * d, d, sigma, kc + (int64_t)t * d, &g[t]);
+    orc_tq3_encode_value_block(v, d, T, vc, sc, zp);
+    orc_tq3_pack_block(d, M, kc, g, vc, sc, zp, rec);
+    free(kc); free(vc); free(g);
+}
+
+void orc_fp8_pack_block(int d, int M, const float* k, const float* v, int n_valid, float k_scale, float v_scale,
+                        uint8_t* rec)
+{
+    int m;
+    for (m = 0; m < M; ++m) {
+        int n = n_valid - m * ORC_T;
+        n = n < 0 ? 0 : (n > ORC_T ? ORC_T : n);
+        orc_fp8_pack_record(d, k + (int64_t)m * ORC_T * d, v + (int64_t)m * ORC_T * d, n, k_scale, v_scale,
+                            rec + m * orc_fp8_record_bytes(d));
+    }
+}
+
+void orc_fp8_unpack_block_f32(int d, int M, const uint8_t* rec, float k_scale, float v_scale, float* k, float* v)
+{
+    int m;
+    for (m = 0; m < M; ++m)
+        orc_fp8_unpack_record_f32(d, rec + m * orc_fp8_record_bytes(d), k_scale, v_scale, k + (int64_t)m * ORC_T * d,
+                                  v + (int64_t)m * ORC_T * d);
+}
+
+/* Retier(p, TQ3), data part, for a page of 16 M tokens */
+void orc_demote_block(int d, int M, const uint8_t* fp8_block, float k_scale, float v_scale, const int8_t* sigma,
+                      uint8_t* tq3_block)
+{
+    int T = ORC_T * M;
+    float* k = (float*)malloc(sizeof(float) * (size_t)T * d);
+    float* v = (float*)malloc(sizeof(float) * (size_t)T * d);
+    orc_fp8_unpack_block_f32(d, M, fp8_block, k_scale, v_scale, k, v);
+    orc_tq3_block_from_f32(d, M, k, v, sigma, tq3_block);
+    free(k); free(v);
+}
+
+void orc_promote_record(int d, const uint8_t* tq3_rec, float k_scale, float v_scale, const int8_t* sigma,
+                        uint8_t* fp8_rec);
+
+/* Promote(p), data part, for a page of 16 M tokens: every tile is rebuilt like a 16-token record
+ * whose scale/zero are the page's */
+void orc_promote_block(int d, int M, const uint8_t* tq3_block, float k_scale, float v_scale, const int8_t* sigma,
+                       uint8_t* fp8_block)
+{
+    uint8_t* tmp = (uint8_t*)malloc((size_t)orc_tq3_record_bytes(d));
+    int64_t tile = orc_tq3_tile_bytes(d);
+    int m;
+    for (m = 0; m < M; ++m) {
+        memcpy(tmp, tq3_block + m * tile, (size_t)tile);
+        memcpy(tmp + tile, tq3_block + M * tile, (size_t)(4 * d));
+        orc_promote_record(d, tmp, k_scale, v_scale, sigma, fp8_block + m * orc_fp8_record_bytes(d));
+    }
+    free(tmp);
+}
+
+/* ------------------------------------------------------------------------------------------
  * Dequantise-then-attend (Section 3.3).  For request b and KV head h the logical cache is the
  * concatenation, in block-table order, of the pages of the row; a page with tag 0 (Recent) or
  * 1 (Anchor) is an FP8 record of the FP8 arena, tag 2 (Stale) a TQ3 record of the TQ3 arena.
@@ -433,6 +552,7 @@ typedef struct {
     const uint8_t* tq3_arena;
     int64_t fp8_pages, tq3_pages;
     int d, hkv, group;
+    int M;                      /* 16-token tiles per page (page = 16 M tokens) */
     float k_scale, v_scale;
     const int8_t* sigma;
 } orc_pool;
@@ -442,38 +562,43 @@ typedef struct {
 static int materialise(const orc_pool* p, const int32_t* row, const uint8_t* tags, int len, int h,
                        double* K, double* V)
 {
-    int d = p->d, n_pages = (len + ORC_T - 1) / ORC_T, pg, t, i;
-    uint8_t* kc = (uint8_t*)malloc(ORC_T * (size_t)d);
-    uint8_t* vc = (uint8_t*)malloc(ORC_T * (size_t)d);
-    uint16_t g[ORC_T], sc[ORC_MAXD], zp[ORC_MAXD];
+    int d = p->d, M = p->M, T = ORC_T * M, n_pages = (len + T - 1) / T, pg, t, i, m;
+    uint8_t* kc = (uint8_t*)malloc((size_t)T * d);
+    uint8_t* vc = (uint8_t*)malloc((size_t)T * d);
+    uint16_t* g = (uint16_t*)malloc(sizeof(uint16_t) * (size_t)T);
+    uint16_t sc[ORC_MAXD], zp[ORC_MAXD];
     int rc = 0;
     for (pg = 0; pg < n_pages && rc == 0; ++pg) {
-        int valid = len - pg * ORC_T < ORC_T ? len - pg * ORC_T : ORC_T;
+        int valid = len - pg * T < T ? len - pg * T : T;
         int64_t id = row[pg];
         if (tags[pg] <= 1) {
-            const uint8_t* rec;
+            const uint8_t* blk;
             if (id < 0 || id >= p->fp8_pages) { rc = -1; break; }
-            rec = p->fp8_arena + (id * p->hkv + h) * orc_fp8_record_bytes(d);
-            for (t = 0; t < valid; ++t)
+            blk = p->fp8_arena + (id * p->hkv + h) * orc_fp8_block_bytes(d, M);
+            for (t = 0; t < valid; ++t) {
+                const uint8_t* rec = blk + (int64_t)(t / ORC_T) * orc_fp8_record_bytes(d);   /* tile of the token */
+                int s = t % ORC_T;
                 for (i = 0; i < d; ++i) {
-                    K[(int64_t)(pg * ORC_T + t) * d + i] = orc_e4m3_decode(rec[t * d + i]) * (double)p->k_scale;
-                    V[(int64_t)(pg * ORC_T + t) * d + i] = orc_e4m3_decode(rec[16 * d + i * ORC_T + t]) * (double)p->v_scale;
+                    K[((int64_t)pg * T + t) * d + i] = orc_e4m3_decode(rec[s * d + i]) * (double)p->k_scale;
+                    V[((int64_t)pg * T + t) * d + i] = orc_e4m3_decode(rec[16 * d + i * ORC_T + s]) * (double)p->v_scale;
                 }
+            }
         } else if (tags[pg] == 2) {
-            const uint8_t* rec;
-            if (id < 0 || id >= p->tq3_pages || valid != ORC_T) { rc = -1; break; }
-            rec = p->tq3_arena + (id * p->hkv + h) * orc_tq3_record_bytes(d);
-            orc_tq3_unpack_record(d, rec, kc, g, vc, sc, zp);
-            for (t = 0; t < ORC_T; ++t) {
-                orc_tq3_decode_key(kc + t * d, g[t], d, p->sigma, K + (int64_t)(pg * ORC_T + t) * d);
+            const uint8_t* blk;
+            if (id < 0 || id >= p->tq3_pages || valid != T) { rc = -1; break; }
+            blk = p->tq3_arena + (id * p->hkv + h) * orc_tq3_block_bytes(d, M);
+            orc_tq3_unpack_block(d, M, blk, kc, g, vc, sc, zp);
+            for (t = 0; t < T; ++t) {
+                orc_tq3_decode_key(kc + (int64_t)t * d, g[t], d, p->sigma, K + ((int64_t)pg * T + t) * d);
                 for (i = 0; i < d; ++i)
-                    V[(int64_t)(pg * ORC_T + t) * d + i] = orc_tq3_decode_value(vc[t * d + i], sc[i], zp[i]);
+                    V[((int64_t)pg * T + t) * d + i] = orc_tq3_decode_value(vc[(int64_t)t * d + i], sc[i], zp[i]);
             }
         } else {
             rc = -1;
         }
     }
-    free(kc); free(vc);
+    (void)m;
+    free(kc); free(vc); free(g);
     return rc;
 }
 
@@ -516,18 +641,19 @@ static void attend_range(const double* q, const double* K, const double* V, int 
  *   mode >= 2: Eq. (softmax-merge) over `mode` contiguous token ranges of equal size.
  *   only_b / only_h >= 0 restrict the work to one request / one KV head (other outputs untouched).
  * Returns 0, or -1 if a table entry is invalid. */
-int orc_decode_attention(const uint8_t* fp8_arena, int64_t fp8_pages, const uint8_t* tq3_arena,
-                         int64_t tq3_pages, int d, int hkv, int group, float k_scale, float v_scale,
-                         const int8_t* sigma, const uint16_t* q, const int32_t* block_table,
-                         const uint8_t* tier_tag, const int32_t* seq_lens, int B, int max_pages,
-                         double scale, double* out, double* lse, int mode, int only_b, int only_h)
+int orc_decode_attention_blocks(const uint8_t* fp8_arena, int64_t fp8_pages, const uint8_t* tq3_arena,
+                                int64_t tq3_pages, int d, int hkv, int group, int M, float k_scale, float v_scale,
+                                const int8_t* sigma, const uint16_t* q, const int32_t* block_table,
+                                const uint8_t* tier_tag, const int32_t* seq_lens, int B, int max_pages,
+                                double scale, double* out, double* lse, int mode, int only_b, int only_h)
 {
     orc_pool pool;
     int Hq = hkv * group, unit, rc = 0;
     pool.fp8_arena = fp8_arena; pool.tq3_arena = tq3_arena;
     pool.fp8_pages = fp8_pages; pool.tq3_pages = tq3_pages;
-    pool.d = d; pool.hkv = hkv; pool.group = group;
+    pool.d = d; pool.hkv = hkv; pool.group = group; pool.M = M;
     pool.k_scale = k_scale; pool.v_scale = v_scale; pool.sigma = sigma;
+    if (M < 1) return -1;
 
 #pragma omp parallel for schedule(dynamic, 1)
     for (unit = 0; unit < B * hkv; ++unit) {
@@ -572,7 +698,7 @@ int orc_decode_attention(const uint8_t* fp8_arena, int64_t fp8_pages, const uint
                         double* Vp = (double*)malloc(sizeof(double) * (size_t)len * d);
                         int n = 0, i;
                         for (i = 0; i < len; ++i)
-                            if ((tags[i / ORC_T] == 2) == (j == 1)) {
+                            if ((tags[i / (ORC_T * M)] == 2) == (j == 1)) {
                                 memcpy(Kp + (int64_t)n * d, K + (int64_t)i * d, sizeof(double) * d);
                                 memcpy(Vp + (int64_t)n * d, V + (int64_t)i * d, sizeof(double) * d);
                                 ++n;
@@ -606,6 +732,18 @@ int orc_decode_attention(const uint8_t* fp8_arena, int64_t fp8_pages, const uint
     return rc;
 }
 
+/* the 16-token page (M = 1) */
+int orc_decode_attention(const uint8_t* fp8_arena, int64_t fp8_pages, const uint8_t* tq3_arena,
+                         int64_t tq3_pages, int d, int hkv, int group, float k_scale, float v_scale,
+                         const int8_t* sigma, const uint16_t* q, const int32_t* block_table,
+                         const uint8_t* tier_tag, const int32_t* seq_lens, int B, int max_pages,
+                         double scale, double* out, double* lse, int mode, int only_b, int only_h)
+{
+    return orc_decode_attention_blocks(fp8_arena, fp8_pages, tq3_arena, tq3_pages, d, hkv, group, 1, k_scale, v_scale,
+                                       sigma, q, block_table, tier_tag, seq_lens, B, max_pages, scale, out, lse, mode,
+                                       only_b, only_h);
+}
+
 /* ------------------------------------------------------------------------------------------
  * Globally normalised page mass (Section 3.1, Eq. score-partial, Eq. score-global-weight,
  * Eq. attention-score).  For query head h the tokens are split into partitions j by physical
@@ -625,7 +763,7 @@ int orc_page_mass(const uint8_t* fp8_arena, int64_t fp8_pages, const uint8_t* tq
     int Hq = hkv * group, unit, rc = 0;
     pool.fp8_arena = fp8_arena; pool.tq3_arena = tq3_arena;
     pool.fp8_pages = fp8_pages; pool.tq3_pages = tq3_pages;
-    pool.d = d; pool.hkv = hkv; pool.group = group;
+    pool.d = d; pool.hkv = hkv; pool.group = group; pool.M = 1;
     pool.k_scale = k_scale; pool.v_scale = v_scale; pool.sigma = sigma;
 
 #pragma omp parallel for schedule(dynamic, 1)
@@ -746,37 +884,47 @@ double orc_effective_bits(double p_R, double p_A, double p_S, double b_S, double
  *   Stale pages: TQ3 encoded from the bf16 originals (must be full).
  * Returns 0, or -1 on an invalid tag or a partial Stale page.
  * ---------------------------------------------------------------------------------------- */
-int orc_encode_request(int d, int hkv, int len, const uint16_t* k_bits, const uint16_t* v_bits,
-                       const int32_t* row, const uint8_t* tags, const int8_t* sigma, float k_scale,
-                       float v_scale, uint8_t* fp8_arena, uint8_t* tq3_arena)
+int orc_encode_request_blocks(int d, int hkv, int len, int M, const uint16_t* k_bits, const uint16_t* v_bits,
+                              const int32_t* row, const uint8_t* tags, const int8_t* sigma, float k_scale,
+                              float v_scale, uint8_t* fp8_arena, uint8_t* tq3_arena)
 {
-    int n_pages = (len + ORC_T - 1) / ORC_T, pg, rc = 0;
+    int T = ORC_T * M, n_pages = (len + T - 1) / T, pg, rc = 0;
 #pragma omp parallel for schedule(dynamic, 8)
     for (pg = 0; pg < n_pages; ++pg) {
-        int valid = len - pg * ORC_T < ORC_T ? len - pg * ORC_T : ORC_T, h, t, i;
-        float k[ORC_T * ORC_MAXD], v[ORC_T * ORC_MAXD];
+        int valid = len - pg * T < T ? len - pg * T : T, h, t, i;
+        float* k = (float*)malloc(sizeof(float) * (size_t)T * d);
+        float* v = (float*)malloc(sizeof(float) * (size_t)T * d);
         for (h = 0; h < hkv; ++h) {
-            memset(k, 0, sizeof k);
-            memset(v, 0, sizeof v);
+            memset(k, 0, sizeof(float) * (size_t)T * d);
+            memset(v, 0, sizeof(float) * (size_t)T * d);
             for (t = 0; t < valid; ++t)
                 for (i = 0; i < d; ++i) {
-                    int64_t src = ((int64_t)(pg * ORC_T + t) * hkv + h) * d + i;
-                    k[t * d + i] = orc_bf16_to_f32(k_bits[src]);
-                    v[t * d + i] = orc_bf16_to_f32(v_bits[src]);
+                    int64_t src = (((int64_t)pg * T + t) * hkv + h) * d + i;
+                    k[(int64_t)t * d + i] = orc_bf16_to_f32(k_bits[src]);
+                    v[(int64_t)t * d + i] = orc_bf16_to_f32(v_bits[src]);
                 }
             if (tags[pg] <= 1) {
-                orc_fp8_pack_record(d, k, v, valid, k_scale, v_scale,
-                                    fp8_arena + ((int64_t)row[pg] * hkv + h) * orc_fp8_record_bytes(d));
-            } else if (tags[pg] == 2 && valid == ORC_T) {
-                orc_tq3_record_from_f32(d, k, v, sigma,
-                                        tq3_arena + ((int64_t)row[pg] * hkv + h) * orc_tq3_record_bytes(d));
+                orc_fp8_pack_block(d, M, k, v, valid, k_scale, v_scale,
+                                   fp8_arena + ((int64_t)row[pg] * hkv + h) * orc_fp8_block_bytes(d, M));
+            } else if (tags[pg] == 2 && valid == T) {
+                orc_tq3_block_from_f32(d, M, k, v, sigma,
+                                       tq3_arena + ((int64_t)row[pg] * hkv + h) * orc_tq3_block_bytes(d, M));
             } else {
 #pragma omp atomic write
                 rc = -1;
             }
         }
+        free(k); free(v);
     }
     return rc;
+}
+
+int orc_encode_request(int d, int hkv, int len, const uint16_t* k_bits, const uint16_t* v_bits,
+                       const int32_t* row, const uint8_t* tags, const int8_t* sigma, float k_scale,
+                       float v_scale, uint8_t* fp8_arena, uint8_t* tq3_arena)
+{
+    return orc_encode_request_blocks(d, hkv, len, 1, k_bits, v_bits, row, tags, sigma, k_scale, v_scale, fp8_arena,
+                                     tq3_arena);
 }
 
 /* ------------------------------------------------------------------------------------------
