@@ -11,8 +11,9 @@
  * cache is ever built.
  *
  * Conventions
- *   - page = 16 tokens; head_dim d in {128, 256}; query head h reads KV head h / (n_q/n_kv);
- *     at most 8 query heads per KV head.
+ *   - page = 16 tokens by default, or 16 M tokens, M <= 256 (Section 4.1 stores blocks of 1,792 and of
+ *     832 tokens); head_dim d in {128, 256}; query head h reads KV head h / (n_q/n_kv); at most 8
+ *     query heads per KV head.
  *   - "device" pointers are CUDA device memory owned by the caller, 16-byte aligned (arenas and
  *     workspace 256-byte aligned); "host" pointers are ordinary host memory.  The library
  *     allocates no device memory: the caller hands it arenas and workspace.
@@ -33,6 +34,16 @@
  *       [0, 6d)   key codes,   [6d, 12d) value codes,   [12d, 12d+32) norm correction g[16],
  *       [12d+32, 16d+32) value scale/zero.  Bit positions are those of the tensor-core
  *     fragment that consumes them; mkv_page_read_raw() returns the bytes as stored.
+ *   Pages of 16 M tokens (page_size = 16 M) are M tiles of 16 tokens:
+ *     FP8 page, M * 32*d bytes: tile m is the FP8 record of tokens [16 m, 16 m + 16) at m * 32*d.
+ *     TQ3 page, M * (12*d + 32) + 4*d bytes: tile m at m * (12*d + 32) holds [key codes | value codes |
+ *       g[16]] of its 16 tokens as in the 16-token record; the value scale/zero of the PAGE (one pair per
+ *       channel over all 16 M tokens) follow the tiles.  M = 1 is the 16-token record.  At M = 112,
+ *       d = 256 this is 348,672 bytes per page and head: the 3.04 bit/scalar of Section 5.4.
+ *     Block-table rows have one entry per page; slot_mapping = page * page_size + position.  With M > 1
+ *     mkv_decode_attention() runs the tensor-core kernel (MKV_DECODE_SCALAR / _TMEM, the scored call and
+ *     the no-allocation entry point with a scored output are refused with MKV_E_INVALID); mkv_demote()
+ *     and mkv_promote() take three resp. two launches (page scale/zero, tiles, publication).
  */
 #ifndef MKV_H_
 #define MKV_H_
@@ -68,7 +79,7 @@ enum { MKV_FMT_FP8 = 0, MKV_FMT_TQ3 = 1 };
 enum { MKV_DECODE_TENSOR = 0, MKV_DECODE_SCALAR = 1, MKV_DECODE_TMEM = 2 };
 
 typedef struct {
-    int32_t page_size;          /* must be 16                                                   */
+    int32_t page_size;          /* tokens per page: 16, or a multiple of 16 up to 4096          */
     int32_t head_dim;           /* 128 or 256                                                   */
     int32_t n_kv_heads;
     int32_t n_q_heads;          /* multiple of n_kv_heads, at most 8 per KV head                */

@@ -125,9 +125,10 @@ def _stream(stream: Optional[torch.cuda.Stream]):
     return C.c_void_p(s.cuda_stream)
 
 
-def make_config(head_dim, n_kv_heads, n_q_heads, fp8_pages, tq3_pages, sigma: np.ndarray, k_scale=1.0, v_scale=1.0):
+def make_config(head_dim, n_kv_heads, n_q_heads, fp8_pages, tq3_pages, sigma: np.ndarray, k_scale=1.0, v_scale=1.0,
+                page_tokens=16):
     sig = np.ascontiguousarray(sigma, dtype=np.int8)
-    cfg = PoolConfig(16, head_dim, n_kv_heads, n_q_heads, fp8_pages, tq3_pages, k_scale, v_scale,
+    cfg = PoolConfig(page_tokens, head_dim, n_kv_heads, n_q_heads, fp8_pages, tq3_pages, k_scale, v_scale,
                      sig.ctypes.data_as(C.POINTER(C.c_int8)))
     cfg._keepalive = sig
     return cfg
@@ -150,14 +151,17 @@ class Pool:
     """One layer's page pool.  Owns the torch buffers handed to the library (arenas, workspace)."""
 
     def __init__(self, head_dim, n_kv_heads, n_q_heads, fp8_pages, tq3_pages, sigma, k_scale=1.0, v_scale=1.0,
-                 max_batch=64, device="cuda:0"):
+                 max_batch=64, device="cuda:0", page_tokens=16):
         L = lib()
         self.device = torch.device(device)
         self.d, self.hkv, self.hq = head_dim, n_kv_heads, n_q_heads
         self.group = n_q_heads // n_kv_heads
-        self.cfg = make_config(head_dim, n_kv_heads, n_q_heads, fp8_pages, tq3_pages, sigma, k_scale, v_scale)
+        self.cfg = make_config(head_dim, n_kv_heads, n_q_heads, fp8_pages, tq3_pages, sigma, k_scale, v_scale, page_tokens)
         fp8_bytes, tq3_bytes = mkv_pool_query(self.cfg)
-        self.fp8_rec, self.tq3_rec = 32 * head_dim, 16 * head_dim + 32
+        # bytes of one page and KV head: a page is page_tokens / 16 tiles (16 d + 32 bytes of TQ3 at one tile)
+        self.page_tokens, self.tiles = page_tokens, page_tokens // 16
+        self.fp8_rec = self.tiles * 32 * head_dim
+        self.tq3_rec = self.tiles * (12 * head_dim + 32) + 4 * head_dim
         with torch.cuda.device(self.device):
             self.fp8_arena = torch.empty(fp8_bytes, dtype=torch.uint8, device=self.device)
             self.tq3_arena = torch.empty(tq3_bytes, dtype=torch.uint8, device=self.device)

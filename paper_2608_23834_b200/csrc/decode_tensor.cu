@@ -55,6 +55,7 @@ struct DecodeParams {
     const uint8_t* tags;
     const int32_t* lens;
     int B, max_pages;
+    int tiles;             // 16-token tiles per page (page = 16 * tiles tokens); table entries are per page
     float scale;
     float* out;
     float* lse;
@@ -776,7 +777,7 @@ __device__ __forceinline__ void merge_row(const DecodeParams& P, int first_slot,
         P.lse[(size_t)b * hq + h * GQ + tid] = ml_s[8 + tid] > 0.f ? (ml_s[tid] + log2f(ml_s[8 + tid])) * kLn2 : -CUDART_INF_F;
 }
 
-template <int D, int NW, int NSTAGE, int MINB, bool SCORED>
+template <int D, int NW, int NSTAGE, int MINB, bool SCORED, bool TILED>
 __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const DecodeParams P)
 {
 #ifdef MKV_TIMELINE
@@ -915,6 +916,10 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
         float* mass_row = SCORED ? P.mass + ((size_t)b * hq + (size_t)h * GQ) * P.max_pages : nullptr;
         const uint8_t* tq3_base = P.tq3 + (size_t)h * G::TQ3_REC;
         const uint8_t* fp8_base = P.fp8 + (size_t)h * (2 * G::FP8_HALF);
+        // pages of several tiles: a TQ3 page is tiles * (12 D + 32) bytes of tiles, then 4 D bytes of value
+        // scale/zero shared by its tiles; an FP8 page is `tiles` consecutive 16-token records
+        constexpr int TQ3_TILE = 12 * D + 32, TQ3_META = 4 * D;
+        const size_t tq3_page = (size_t)P.tiles * TQ3_TILE + TQ3_META;
 
         // Table entries of up to G::ROUND of the warp's pages are compacted into two id lists, one per
         // format (entry i of a 32-page chunk is read by lane i; ballots give the positions).
@@ -927,14 +932,17 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                 int kind = 0, id = 0, valid = kPage, pg = 0;
                 if (i < n_my) {
                     pg = (int)(((unsigned)(pg0 + warp_first + i) * (unsigned)stride) % (unsigned)n_pages);   // < 2^32: max_pages <= 65535
-                    id = bt_row[pg];
-                    const int tag = tag_row[pg];
+                    // `pg` counts 16-token tiles of the row; the table has one entry per page of P.tiles tiles
+                    const int entry = TILED ? pg / P.tiles : pg;
+                    id = bt_row[entry];
+                    const int tag = tag_row[entry];
                     valid = min(kPage, len - pg * kPage);
                     if (tag == MKV_TAG_STALE)
                         kind = (id >= 0 && id < P.tq3_pages && valid == kPage) ? 1 : 0;
                     else
                         kind = (tag <= MKV_TAG_ANCHOR && id >= 0 && id < P.fp8_pages) ? 2 : 0;
                     if (kind == 0) atomicOr(P.status, kStBounds);     // never dereferenced
+                    if constexpr (TILED) id = id * P.tiles + (pg - entry * P.tiles);   // tile index inside the arena
                 }
                 const uint32_t m3 = __ballot_sync(FULL, kind == 1), m8 = __ballot_sync(FULL, kind == 2);
                 const uint32_t lt = (1u << lane) - 1u;
@@ -954,13 +962,27 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                 const uint32_t s = (uint32_t)i % NSTAGE;
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 mbar_expect_tx(bars + 8 * s, G::TQ3_REC);
-                bulk_load(ring + s * G::SLOT, tq3_base + (size_t)list3[i] * hkv * G::TQ3_REC, G::TQ3_REC, bars + 8 * s);
+                if constexpr (!TILED) {
+                    bulk_load(ring + s * G::SLOT, tq3_base + (size_t)list3[i] * hkv * G::TQ3_REC, G::TQ3_REC, bars + 8 * s);
+                } else {   // the tile, then the page's scale/zero behind it: the slot then reads like a 16-token record
+                    const int page = list3[i] / P.tiles, m = list3[i] - page * P.tiles;
+                    const uint8_t* pbase = P.tq3 + ((size_t)page * hkv + h) * tq3_page;
+                    bulk_load(ring + s * G::SLOT, pbase + (size_t)m * TQ3_TILE, TQ3_TILE, bars + 8 * s);
+                    bulk_load(ring + s * G::SLOT + TQ3_TILE, pbase + (size_t)P.tiles * TQ3_TILE, TQ3_META, bars + 8 * s);
+                }
             }
         };
         auto issue_fp8 = [&](int i) {      // copy FP8 page i of the round into the slot pair 2 (i % (NSTAGE/2))
             if (lane == 0) {
                 const uint32_t s = (uint32_t)(2 * i) % NSTAGE;
-                const uint8_t* rec = fp8_base + (size_t)(list8[i] & 0x7FFFFFF) * hkv * (2 * G::FP8_HALF);
+                const int e8 = list8[i] & 0x7FFFFFF;
+                const uint8_t* rec;
+                if constexpr (!TILED) {
+                    rec = fp8_base + (size_t)e8 * hkv * (2 * G::FP8_HALF);
+                } else {
+                    const int page = e8 / P.tiles, m = e8 - page * P.tiles;
+                    rec = P.fp8 + (((size_t)page * hkv + h) * P.tiles + m) * (2 * G::FP8_HALF);
+                }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 mbar_expect_tx(bars + 8 * s, G::FP8_HALF);
                 bulk_load(ring + s * G::SLOT, rec, G::FP8_HALF, bars + 8 * s);
@@ -1216,11 +1238,11 @@ static int32_t run_tmem(mkv_pool* p, DecodeParams& prm, cudaStream_t s)
     return MKV_OK;
 }
 
-template <int D, int NW, int NSTAGE, int MINB, bool SCORED = false>
+template <int D, int NW, int NSTAGE, int MINB, bool SCORED = false, bool TILED = false>
 static int32_t run_tensor(mkv_pool* p, DecodeParams& prm, cudaStream_t s)
 {
     using G = Geo<D, NW, NSTAGE>;
-    auto kern = decode_tensor_kernel<D, NW, NSTAGE, MINB, SCORED>;
+    auto kern = decode_tensor_kernel<D, NW, NSTAGE, MINB, SCORED, TILED>;
     static int grid_cache[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     int dev = p->device & 7;
     if (grid_cache[dev] == 0) {
@@ -1341,11 +1363,16 @@ int32_t launch_decode_tensor_at(mkv_pool* p, const void* q, const int32_t* bt, c
                                 float* partials, uint32_t* tickets, int max_blocks, float* mass, cudaStream_t s)
 {
     if (B > kMaxBatch) return MKV_E_INVALID;
-    if (max_pages > 65535) {            // the strided page order multiplies two page indices in 32 bits
-        set_last_error("mkv_decode_attention: max_pages above 65535 (1,048,560 tokens per request)");
+    if ((int64_t)max_pages * p->tiles > 65535) {   // the strided order multiplies two 16-token tile indices in 32 bits
+        set_last_error("mkv_decode_attention: more than 65535 16-token tiles per table row (1,048,560 tokens per request)");
+        return MKV_E_INVALID;
+    }
+    if (p->tiles > 1 && (mass || p->variant == MKV_DECODE_TMEM)) {
+        set_last_error("mkv_decode_attention: pages of several tiles are served by the tensor-core kernel without page mass");
         return MKV_E_INVALID;
     }
     DecodeParams prm;
+    prm.tiles = p->tiles;
     prm.fp8 = p->fp8; prm.tq3 = p->tq3;
     prm.fp8_pages = p->cfg.fp8_pages; prm.tq3_pages = p->cfg.tq3_pages;
     prm.hkv = p->hkv; prm.group = p->group;
@@ -1365,6 +1392,8 @@ int32_t launch_decode_tensor_at(mkv_pool* p, const void* q, const int32_t* bt, c
         if (rc != MKV_OK) return rc;
         return launch_page_mass_finish(mass, lse, lens, B, p->hkv * p->group, max_pages, s);
     }
+    if (p->tiles > 1)                    // pages of several tiles: the default launch shapes only
+        return p->d == 128 ? run_tensor<128, 12, 4, 1, false, true>(p, prm, s) : run_tensor<256, 8, 4, 1, false, true>(p, prm, s);
     if (p->variant == MKV_DECODE_TMEM && p->d == 256) return run_tmem<256>(p, prm, s);
     // Launch shapes (warps per block, ring slots per warp, blocks per SM); MKV_DECODE_SHAPE selects the
     // alternatives for profiling.

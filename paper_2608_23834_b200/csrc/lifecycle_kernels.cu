@@ -50,7 +50,7 @@ __device__ __forceinline__ void append_token(uint8_t* __restrict__ rec, int slot
 
 // Decode-sized calls: one block per (token, KV head).
 template <int D>
-__global__ void __launch_bounds__(D / 2) append_kernel(uint8_t* __restrict__ fp8, int fp8_pages, int hkv,
+__global__ void __launch_bounds__(D / 2) append_kernel(uint8_t* __restrict__ fp8, int fp8_pages, int hkv, int tiles,
                                                         float inv_k_scale, float inv_v_scale,
                                                         const __nv_bfloat162* __restrict__ k,
                                                         const __nv_bfloat162* __restrict__ v,
@@ -60,12 +60,13 @@ __global__ void __launch_bounds__(D / 2) append_kernel(uint8_t* __restrict__ fp8
     const int tok = blockIdx.x, h = blockIdx.y;
     const int sm = slots[tok];
     if (sm < 0) return;
-    const int page = sm >> 4, slot = sm & 15;
+    // slot_mapping = page * page_tokens + position; a page is `tiles` consecutive 16-token records per head
+    const int gt = sm >> 4, slot = sm & 15, page = gt / tiles, m = gt - page * tiles;
     if (page >= fp8_pages) {
         if (threadIdx.x == 0) atomicOr(status, kStBounds);
         return;
     }
-    uint8_t* rec = fp8 + ((size_t)page * hkv + h) * fp8_record_bytes(D);
+    uint8_t* rec = fp8 + (((size_t)page * hkv + h) * tiles + m) * fp8_record_bytes(D);
     const size_t src = ((size_t)tok * hkv + h) * (D / 2);
     append_token<D>(rec, slot, inv_k_scale, inv_v_scale, k + src, v + src, threadIdx.x);
 }
@@ -90,7 +91,7 @@ __device__ __forceinline__ uint2 bf16x8_to_e4m3x8(uint4 in, float inv_scale)
 // is transposed through shared memory so that every channel's 16 tokens leave as one 16-byte store;
 // any other group (skipped tokens, a run that starts inside a page, the tail) takes the per-token path.
 template <int D>
-__global__ void __launch_bounds__(128) append_run_kernel(uint8_t* __restrict__ fp8, int fp8_pages, int hkv,
+__global__ void __launch_bounds__(128) append_run_kernel(uint8_t* __restrict__ fp8, int fp8_pages, int hkv, int tiles,
                                                           float inv_k_scale, float inv_v_scale,
                                                           const __nv_bfloat162* __restrict__ k,
                                                           const __nv_bfloat162* __restrict__ v,
@@ -107,13 +108,14 @@ __global__ void __launch_bounds__(128) append_run_kernel(uint8_t* __restrict__ f
     __syncthreads();
     if (tid == 0) {
         const int s0 = slot_s[0];
-        bool run = cnt == kPage && s0 >= 0 && (s0 & 15) == 0 && (s0 >> 4) < fp8_pages;
+        bool run = cnt == kPage && s0 >= 0 && (s0 & 15) == 0 && (s0 >> 4) / tiles < fp8_pages;
         for (int i = 1; run && i < kPage; ++i) run = slot_s[i] == s0 + i;
         run_s = run ? 1 : 0;
     }
     __syncthreads();
     if (run_s) {
-        uint8_t* rec = fp8 + ((size_t)(slot_s[0] >> 4) * hkv + h) * fp8_record_bytes(D);
+        const int gt = slot_s[0] >> 4, page = gt / tiles;
+        uint8_t* rec = fp8 + (((size_t)page * hkv + h) * tiles + (gt - page * tiles)) * fp8_record_bytes(D);
         constexpr int CPT = D / 8;                   // 16-byte input chunks per token
         for (int c = tid; c < kPage * CPT; c += 128) {
             const int t = c / CPT, c8 = c % CPT;
@@ -147,11 +149,12 @@ __global__ void __launch_bounds__(128) append_run_kernel(uint8_t* __restrict__ f
     for (int t = 0; t < cnt; ++t) {
         const int sm = slot_s[t];
         if (sm < 0) continue;
-        if ((sm >> 4) >= fp8_pages) {
+        const int gt = sm >> 4, page = gt / tiles;
+        if (page >= fp8_pages) {
             if (tid == 0) atomicOr(status, kStBounds);
             continue;
         }
-        uint8_t* rec = fp8 + ((size_t)(sm >> 4) * hkv + h) * fp8_record_bytes(D);
+        uint8_t* rec = fp8 + (((size_t)page * hkv + h) * tiles + (gt - page * tiles)) * fp8_record_bytes(D);
         const size_t src = ((size_t)(t0 + t) * hkv + h) * (D / 2);
         if (tid < D / 2) append_token<D>(rec, sm & 15, inv_k_scale, inv_v_scale, k + src, v + src, tid);
     }
@@ -165,17 +168,17 @@ int32_t launch_append(mkv_pool* p, const void* k, const void* v, const int32_t* 
     if (n >= 2 * kPage) {
         dim3 grid((n + kPage - 1) / kPage, p->hkv);
         if (p->d == 128)
-            append_run_kernel<128><<<grid, 128, 0, s>>>(p->fp8, p->cfg.fp8_pages, p->hkv, ik, iv, kk, vv, slots, n,
+            append_run_kernel<128><<<grid, 128, 0, s>>>(p->fp8, p->cfg.fp8_pages, p->hkv, p->tiles, ik, iv, kk, vv, slots, n,
                                                         p->status_dev);
         else
-            append_run_kernel<256><<<grid, 128, 0, s>>>(p->fp8, p->cfg.fp8_pages, p->hkv, ik, iv, kk, vv, slots, n,
+            append_run_kernel<256><<<grid, 128, 0, s>>>(p->fp8, p->cfg.fp8_pages, p->hkv, p->tiles, ik, iv, kk, vv, slots, n,
                                                         p->status_dev);
     } else {
         dim3 grid(n, p->hkv);
         if (p->d == 128)
-            append_kernel<128><<<grid, 64, 0, s>>>(p->fp8, p->cfg.fp8_pages, p->hkv, ik, iv, kk, vv, slots, p->status_dev);
+            append_kernel<128><<<grid, 64, 0, s>>>(p->fp8, p->cfg.fp8_pages, p->hkv, p->tiles, ik, iv, kk, vv, slots, p->status_dev);
         else
-            append_kernel<256><<<grid, 128, 0, s>>>(p->fp8, p->cfg.fp8_pages, p->hkv, ik, iv, kk, vv, slots, p->status_dev);
+            append_kernel<256><<<grid, 128, 0, s>>>(p->fp8, p->cfg.fp8_pages, p->hkv, p->tiles, ik, iv, kk, vv, slots, p->status_dev);
     }
     MKV_CUDA(cudaGetLastError());
     return MKV_OK;
@@ -250,17 +253,225 @@ __device__ __forceinline__ float2 e4m3x2_to_f32(uint32_t two_bytes)
 // nibble pairs of two bytes -> one byte: (x & 0x000F) | ((x & 0x0F00) >> 4)
 __device__ __forceinline__ uint32_t squeeze_nibbles(uint32_t x) { return (x & 0xFu) | ((x >> 4) & 0xF0u); }
 
+// Constants of the key encoder that depend only on the lane.
 template <int D>
+struct DemoteLane {
+    float c0sq, c1sq, c2sq, c3sq;     // squared levels (single fp32 products, as the record's norm correction defines them)
+    uint32_t flip[D / 32];            // rotation signs of this lane's key elements, as fp32 sign-bit masks
+    uint32_t neg[5];                  // butterfly stage m: lanes with bit m set subtract
+    __device__ __forceinline__ void init(const SigmaBits& sigma, int lane)
+    {
+        c0sq = __fmul_rn(MKV_C0, MKV_C0);
+        c1sq = __fmul_rn(MKV_C1, MKV_C1);
+        c2sq = __fmul_rn(MKV_C2, MKV_C2);
+        c3sq = __fmul_rn(MKV_C3, MKV_C3);
+#pragma unroll
+        for (int r = 0; r < D / 32; ++r) {
+            const int i = lane * (D / 32) + r;
+            flip[r] = ((sigma.w[i >> 5] >> (i & 31)) & 1u) << 31;
+        }
+#pragma unroll
+        for (int b = 0; b < 5; ++b) neg[b] = ((lane >> b) & 1u) << 31;
+    }
+};
+
+// Encodes the 16 tokens of one FP8 record (rec8) into the record image img = [key codes | value codes | g |
+// scale/zero] in shared memory; all D threads of the block call it.  OWN_META: the value scale and zero come
+// from these 16 tokens (16-token pages); otherwise thread c passes the page's scale/zero of channel c.
+template <int D, bool OWN_META>
+__device__ __forceinline__ void demote_tile(const uint8_t* __restrict__ rec8, uint8_t* img, uint8_t* kcode, uint8_t* vcode,
+                                            const DemoteLane<D>& K, float k_scale, float v_scale, uint16_t sc_page,
+                                            uint16_t zp_page)
+{
+    constexpr int EPL = D / 32, NJ = D / 64, KROW = D + 8, NT = D;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const float c0sq = K.c0sq, c1sq = K.c1sq, c2sq = K.c2sq, c3sq = K.c3sq;
+    const uint32_t (&flip)[EPL] = K.flip;
+    const uint32_t (&neg)[5] = K.neg;
+    // ---- keys: warp w encodes tokens w, w + NT/32, ... ------------------------------------------
+    for (int tok = warp; tok < kPage; tok += NT / 32) {
+        float x[EPL], a[EPL];
+        uint32_t raw[EPL / 4];
+        if constexpr (EPL == 8) {
+            const uint2 u = *reinterpret_cast<const uint2*>(rec8 + tok * D + lane * EPL);
+            raw[0] = u.x;
+            raw[1] = u.y;
+        } else {
+            raw[0] = *reinterpret_cast<const uint32_t*>(rec8 + tok * D + lane * EPL);
+        }
+#pragma unroll
+        for (int r = 0; r < EPL; r += 2) {
+            const float2 f = e4m3x2_to_f32((raw[r >> 2] >> (8 * (r & 3))) & 0xFFFFu);
+            x[r] = __fmul_rn(f.x, k_scale);
+            x[r + 1] = __fmul_rn(f.y, k_scale);
+            a[r] = __uint_as_float(__float_as_uint(x[r]) ^ flip[r]);
+            a[r + 1] = __uint_as_float(__float_as_uint(x[r + 1]) ^ flip[r + 1]);
+        }
+        // Walsh-Hadamard butterflies, strides ascending: inside the lane, then across lanes
+#pragma unroll
+        for (int hh = 1; hh < EPL; hh <<= 1)
+#pragma unroll
+            for (int r = 0; r < EPL; ++r)
+                if ((r & hh) == 0) {
+                    const float u = a[r], w = a[r + hh];
+                    a[r] = __fadd_rn(u, w);
+                    a[r + hh] = __fsub_rn(u, w);
+                }
+#pragma unroll
+        for (int b = 0; b < 5; ++b)
+#pragma unroll
+            for (int r = 0; r < EPL; ++r) {
+                // lower lane: a + o; upper lane: o - a (the same single addition either way)
+                const float o = __shfl_xor_sync(0xffffffffu, a[r], 1 << b);
+                a[r] = __fadd_rn(o, __uint_as_float(__float_as_uint(a[r]) ^ neg[b]));
+            }
+        // |x|^2: pairwise tree in index order (every element of the butterfly ends equal)
+        float e[EPL];
+#pragma unroll
+        for (int r = 0; r < EPL; ++r) e[r] = __fmul_rn(x[r], x[r]);
+#pragma unroll
+        for (int hh = 1; hh < EPL; hh <<= 1)
+#pragma unroll
+            for (int r = 0; r < EPL; r += 2 * hh) e[r] = __fadd_rn(e[r], e[r + hh]);
+        float n2 = e[0];
+#pragma unroll
+        for (int m = 1; m < 32; m <<= 1) n2 = __fadd_rn(n2, __shfl_xor_sync(0xffffffffu, n2, m));
+        const float nx = __fsqrt_rn(n2);
+        const float t1 = __fmul_rn(MKV_B0, nx), t2 = __fmul_rn(MKV_B1, nx), t3 = __fmul_rn(MKV_B2, nx);
+        float f[EPL];
+        uint32_t packed[EPL / 4];
+#pragma unroll
+        for (int r = 0; r < EPL / 4; ++r) packed[r] = 0;
+#pragma unroll
+        for (int r = 0; r < EPL; ++r) {
+            const float w = fabsf(a[r]);
+            const bool g1 = w > t1, g2 = w > t2, g3 = w > t3;
+            const uint32_t code = (uint32_t)g1 + (uint32_t)g2 + (uint32_t)g3 + ((__float_as_uint(a[r]) >> 29) & 4u);
+            // a[r] < 0 is the sign bit except for -0, which cannot meet a threshold test either way
+            packed[r >> 2] |= (a[r] == 0.0f ? (code & 3u) : code) << (8 * (r & 3));
+            f[r] = g2 ? (g3 ? c3sq : c2sq) : (g1 ? c1sq : c0sq);
+        }
+        if constexpr (EPL == 8)
+            *reinterpret_cast<uint2*>(kcode + tok * KROW + lane * EPL) = make_uint2(packed[0], packed[1]);
+        else
+            *reinterpret_cast<uint32_t*>(kcode + tok * KROW + lane * EPL) = packed[0];
+#pragma unroll
+        for (int hh = 1; hh < EPL; hh <<= 1)
+#pragma unroll
+            for (int r = 0; r < EPL; r += 2 * hh) f[r] = __fadd_rn(f[r], f[r + hh]);
+        float nc2 = f[0];
+#pragma unroll
+        for (int m = 1; m < 32; m <<= 1) nc2 = __fadd_rn(nc2, __shfl_xor_sync(0xffffffffu, nc2, m));
+        const float nc = __fsqrt_rn(nc2);
+        if (lane == 0)
+            *reinterpret_cast<uint16_t*>(img + 12 * D + 2 * tok) =
+                (nx == 0.0f) ? (uint16_t)0 : f32_to_f16_sat_bits(__fdiv_rn(nx, nc));
+    }
+
+    // ---- values: one thread per channel, 16 tokens of the page ------------------------------
+    for (int c = tid; c < D; c += NT) {
+        const uint4 raw = *reinterpret_cast<const uint4*>(rec8 + 16 * D + c * kPage);
+        const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
+        float val[kPage];
+#pragma unroll
+        for (int t = 0; t < kPage; t += 2) {
+            const float2 f = e4m3x2_to_f32((rw[t >> 2] >> (8 * (t & 3))) & 0xFFFFu);
+            val[t] = __fmul_rn(f.x, v_scale);
+            val[t + 1] = __fmul_rn(f.y, v_scale);
+        }
+        // scale and zero of the channel: from this tile's 16 tokens (16-token pages), or the page's (given)
+        uint16_t sc = sc_page, zp = zp_page;
+        if constexpr (OWN_META) {
+            float mn = val[0], mx = val[0];
+#pragma unroll
+            for (int t = 1; t < kPage; ++t) {
+                if (val[t] < mn) mn = val[t];
+                if (val[t] > mx) mx = val[t];
+            }
+            sc = f32_to_f16_sat_bits(__fdiv_rn(__fsub_rn(mx, mn), 7.0f));
+            zp = f32_to_f16_sat_bits(mn);
+        }
+        const float scf = __half2float(__ushort_as_half(sc)), zpf = __half2float(__ushort_as_half(zp));
+        {
+            const int cb = c >> 4, row = c & 15;
+            uint16_t* meta = reinterpret_cast<uint16_t*>(img + 12 * D + 32);
+            const int hi = (cb >> 1) * 64 + (row & 7) * 8 + 4 * (cb & 1) + (row >> 3);
+            meta[hi] = sc;
+            meta[hi + 2] = zp;
+        }
+        // q = clamp(rint((val - zp) / sc), 0, 7), 0 when sc == 0.  The division is the correctly
+        // rounded one; a zero numerator (the channel's minimum) or a zero scale is replaced by
+        // operands whose quotient is not used, which keeps the divider on its short path.
+        const float den = scf != 0.0f ? scf : 1.0f;
+        uint32_t q4[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+        for (int t = 0; t < kPage; ++t) {
+            const float num = __fsub_rn(val[t], zpf);
+            float r = rintf(__fdiv_rn(num != 0.0f ? num : den, den));   // half to even
+            r = r < 0.0f ? 0.0f : r;
+            r = r > 7.0f ? 7.0f : r;
+            const uint32_t q = (num != 0.0f && scf != 0.0f) ? (uint32_t)(int)r : 0u;
+            q4[t >> 2] |= q << (8 * (t & 3));
+        }
+        *reinterpret_cast<uint4*>(vcode + c * kPage) = make_uint4(q4[0], q4[1], q4[2], q4[3]);
+    }
+    __syncthreads();
+
+    // ---- pack: one thread per (section, triple j, fragment lane L) --------------------------
+    for (int item = tid; item < 2 * NJ * 32; item += NT) {
+        const int L = item & 31, j = (item >> 5) % NJ, section = item / (32 * NJ);
+        const int g = L >> 2, tq = L & 3;
+        uint32_t w0 = 0, w1 = 0, w2 = 0;
+        if (section == 0) {
+            // key codes: nibble n = 2r + half holds row g + 8(r&1), slot 2tq + 8(r>>1) + half.
+            // A: block 4j with the signs of block 4j+2; B: block 4j+1 with the signs of 4j+3;
+            // C: magnitudes of blocks 4j+2 (low pair) and 4j+3 (high pair).
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                const uint8_t* at = kcode + (g + 8 * (r & 1)) * KROW + 64 * j + 2 * tq + 8 * (r >> 1);
+                const uint32_t b0 = *reinterpret_cast<const uint16_t*>(at);        // (half 0, half 1)
+                const uint32_t b1 = *reinterpret_cast<const uint16_t*>(at + 16);
+                const uint32_t b2 = *reinterpret_cast<const uint16_t*>(at + 32);
+                const uint32_t b3 = *reinterpret_cast<const uint16_t*>(at + 48);
+                w0 |= squeeze_nibbles(b0 | ((b2 & 0x0404u) << 1)) << (8 * r);
+                w1 |= squeeze_nibbles(b1 | ((b3 & 0x0404u) << 1)) << (8 * r);
+                w2 |= squeeze_nibbles((b2 & 0x0303u) | ((b3 & 0x0303u) << 2)) << (8 * r);
+            }
+        } else {
+            // value codes: four 24-bit streams (group, half) per triple; stream code k is
+            // channel block 4j + 2 grp + (k>>2), row g + 8(k&1), token 2tq + 8((k>>1)&1) + half
+            uint32_t S[2][2] = {{0u, 0u}, {0u, 0u}};
+#pragma unroll
+            for (int grp = 0; grp < 2; ++grp)
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const int cb = 4 * j + 2 * grp + (k >> 2), r = k & 3;
+                    const uint32_t two = *reinterpret_cast<const uint16_t*>(
+                        vcode + (16 * cb + g + 8 * (r & 1)) * kPage + 2 * tq + 8 * (r >> 1));
+                    S[grp][0] |= (two & 7u) << (3 * k);
+                    S[grp][1] |= (two >> 8) << (3 * k);
+                }
+            w0 = (S[0][0] & 0xFFFFu) | (S[0][1] << 16);
+            w1 = (S[0][0] >> 16) | ((S[1][0] & 0xFFu) << 8) | ((S[0][1] >> 16) << 16) | (S[1][1] << 24);
+            w2 = (S[1][0] >> 8) | ((S[1][1] >> 8) << 16);
+        }
+        uint8_t* sec = img + section * 6 * D;
+        *reinterpret_cast<uint32_t*>(sec + lane_word_offset(D, L, 3 * j)) = w0;
+        *reinterpret_cast<uint32_t*>(sec + lane_word_offset(D, L, 3 * j + 1)) = w1;
+        *reinterpret_cast<uint32_t*>(sec + lane_word_offset(D, L, 3 * j + 2)) = w2;
+    }
+    __syncthreads();
+}
+
+template <int D, bool BIG>
 __global__ void __launch_bounds__(D) demote_kernel(const uint8_t* __restrict__ fp8, uint8_t* __restrict__ tq3,
-                                                      int fp8_pages, int tq3_pages, int hkv, float k_scale,
+                                                      int fp8_pages, int tq3_pages, int hkv, int tiles, float k_scale,
                                                       float v_scale, SigmaBits sigma,
                                                       const int32_t* __restrict__ src_ids,
                                                       const int32_t* __restrict__ dst_ids, int32_t* block_table,
                                                       uint8_t* tier_tag, const int64_t* entry_index,
                                                       uint32_t* __restrict__ status)
 {
-    constexpr int EPL = D / 32;          // key elements per lane
-    constexpr int NJ = D / 64;           // word triples per lane and section
     constexpr int KROW = D + 8;          // padded row of the key-code tile
     constexpr int REC = 16 * D + 32;     // bytes of one TQ3 record
     constexpr int NT = D;                // threads: one per value channel, one per packed word triple
@@ -269,200 +480,39 @@ __global__ void __launch_bounds__(D) demote_kernel(const uint8_t* __restrict__ f
     __shared__ __align__(16) uint8_t image[2][REC];
 
     const int csize = (int)cluster_size(), crank = (int)cluster_rank();
-    const int page = blockIdx.x / csize, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int page = blockIdx.x / csize, tid = threadIdx.x, lane = tid & 31;
     const int src = src_ids[page], dst = dst_ids[page];
     const bool valid = src >= 0 && src < fp8_pages && dst >= 0 && dst < tq3_pages;
-    if (!valid && tid == 0 && crank == 0) atomicOr(status, kStBounds);
-    // squared levels (single fp32 products, as the record's norm correction defines them)
-    const float c0sq = __fmul_rn(MKV_C0, MKV_C0), c1sq = __fmul_rn(MKV_C1, MKV_C1),
-                c2sq = __fmul_rn(MKV_C2, MKV_C2), c3sq = __fmul_rn(MKV_C3, MKV_C3);
-    // rotation signs of this lane's key elements, as fp32 sign-bit masks
-    uint32_t flip[EPL];
-#pragma unroll
-    for (int r = 0; r < EPL; ++r) {
-        const int i = lane * EPL + r;
-        flip[r] = ((sigma.w[i >> 5] >> (i & 31)) & 1u) << 31;
-    }
-    uint32_t neg[5];                      // butterfly stage m: lanes with bit m set subtract
-#pragma unroll
-    for (int b = 0; b < 5; ++b) neg[b] = ((lane >> b) & 1u) << 31;
+    if (!valid && tid == 0 && crank == 0 && blockIdx.y == 0) atomicOr(status, kStBounds);
+    DemoteLane<D> lane_consts;
+    lane_consts.init(sigma, lane);
 
-    for (int h = crank, it = 0; valid && h < hkv; h += csize, ++it) {
-        const uint8_t* rec8 = fp8 + ((size_t)src * hkv + h) * fp8_record_bytes(D);
-        uint8_t* rec3 = tq3 + ((size_t)dst * hkv + h) * tq3_record_bytes(D);
-        uint8_t* img = image[it & 1];
-
-        // ---- keys: warp w encodes tokens w, w + NT/32, ... ------------------------------------------
-        for (int tok = warp; tok < kPage; tok += NT / 32) {
-            float x[EPL], a[EPL];
-            uint32_t raw[EPL / 4];
-            if constexpr (EPL == 8) {
-                const uint2 u = *reinterpret_cast<const uint2*>(rec8 + tok * D + lane * EPL);
-                raw[0] = u.x;
-                raw[1] = u.y;
-            } else {
-                raw[0] = *reinterpret_cast<const uint32_t*>(rec8 + tok * D + lane * EPL);
+    int it = 0;
+    for (int h = crank; valid && h < hkv; h += csize) {
+        if constexpr (!BIG) {
+            const uint8_t* rec8 = fp8 + ((size_t)src * hkv + h) * fp8_record_bytes(D);
+            uint8_t* rec3 = tq3 + ((size_t)dst * hkv + h) * tq3_record_bytes(D);
+            uint8_t* img = image[it++ & 1];
+            demote_tile<D, true>(rec8, img, kcode, vcode, lane_consts, k_scale, v_scale, 0, 0);
+            for (int i = tid; i < REC / 16; i += NT)
+                reinterpret_cast<uint4*>(rec3)[i] = reinterpret_cast<const uint4*>(img)[i];
+        } else {
+            // pages of several tiles: the page's scale/zero were written by demote_minmax_kernel; the blocks of
+            // grid row y take tiles y, y + gridDim.y, ... and write the tile part of the image only
+            constexpr int TILE = 12 * D + 32;
+            uint8_t* page3 = tq3 + ((size_t)dst * hkv + h) * tq3_page_bytes(D, tiles);
+            const uint16_t* meta = reinterpret_cast<const uint16_t*>(page3 + (size_t)tiles * TILE);
+            const int cb = tid >> 4, row = tid & 15;
+            const int hi = (cb >> 1) * 64 + (row & 7) * 8 + 4 * (cb & 1) + (row >> 3);
+            const uint16_t sc = meta[hi], zp = meta[hi + 2];
+            for (int m = blockIdx.y; m < tiles; m += gridDim.y) {
+                const uint8_t* rec8 = fp8 + (((size_t)src * hkv + h) * tiles + m) * fp8_record_bytes(D);
+                uint8_t* img = image[it++ & 1];
+                demote_tile<D, false>(rec8, img, kcode, vcode, lane_consts, k_scale, v_scale, sc, zp);
+                uint4* out = reinterpret_cast<uint4*>(page3 + (size_t)m * TILE);
+                for (int i = tid; i < TILE / 16; i += NT) out[i] = reinterpret_cast<const uint4*>(img)[i];
             }
-#pragma unroll
-            for (int r = 0; r < EPL; r += 2) {
-                const float2 f = e4m3x2_to_f32((raw[r >> 2] >> (8 * (r & 3))) & 0xFFFFu);
-                x[r] = __fmul_rn(f.x, k_scale);
-                x[r + 1] = __fmul_rn(f.y, k_scale);
-                a[r] = __uint_as_float(__float_as_uint(x[r]) ^ flip[r]);
-                a[r + 1] = __uint_as_float(__float_as_uint(x[r + 1]) ^ flip[r + 1]);
-            }
-            // Walsh-Hadamard butterflies, strides ascending: inside the lane, then across lanes
-#pragma unroll
-            for (int hh = 1; hh < EPL; hh <<= 1)
-#pragma unroll
-                for (int r = 0; r < EPL; ++r)
-                    if ((r & hh) == 0) {
-                        const float u = a[r], w = a[r + hh];
-                        a[r] = __fadd_rn(u, w);
-                        a[r + hh] = __fsub_rn(u, w);
-                    }
-#pragma unroll
-            for (int b = 0; b < 5; ++b)
-#pragma unroll
-                for (int r = 0; r < EPL; ++r) {
-                    // lower lane: a + o; upper lane: o - a (the same single addition either way)
-                    const float o = __shfl_xor_sync(0xffffffffu, a[r], 1 << b);
-                    a[r] = __fadd_rn(o, __uint_as_float(__float_as_uint(a[r]) ^ neg[b]));
-                }
-            // |x|^2: pairwise tree in index order (every element of the butterfly ends equal)
-            float e[EPL];
-#pragma unroll
-            for (int r = 0; r < EPL; ++r) e[r] = __fmul_rn(x[r], x[r]);
-#pragma unroll
-            for (int hh = 1; hh < EPL; hh <<= 1)
-#pragma unroll
-                for (int r = 0; r < EPL; r += 2 * hh) e[r] = __fadd_rn(e[r], e[r + hh]);
-            float n2 = e[0];
-#pragma unroll
-            for (int m = 1; m < 32; m <<= 1) n2 = __fadd_rn(n2, __shfl_xor_sync(0xffffffffu, n2, m));
-            const float nx = __fsqrt_rn(n2);
-            const float t1 = __fmul_rn(MKV_B0, nx), t2 = __fmul_rn(MKV_B1, nx), t3 = __fmul_rn(MKV_B2, nx);
-            float f[EPL];
-            uint32_t packed[EPL / 4];
-#pragma unroll
-            for (int r = 0; r < EPL / 4; ++r) packed[r] = 0;
-#pragma unroll
-            for (int r = 0; r < EPL; ++r) {
-                const float w = fabsf(a[r]);
-                const bool g1 = w > t1, g2 = w > t2, g3 = w > t3;
-                const uint32_t code = (uint32_t)g1 + (uint32_t)g2 + (uint32_t)g3 + ((__float_as_uint(a[r]) >> 29) & 4u);
-                // a[r] < 0 is the sign bit except for -0, which cannot meet a threshold test either way
-                packed[r >> 2] |= (a[r] == 0.0f ? (code & 3u) : code) << (8 * (r & 3));
-                f[r] = g2 ? (g3 ? c3sq : c2sq) : (g1 ? c1sq : c0sq);
-            }
-            if constexpr (EPL == 8)
-                *reinterpret_cast<uint2*>(kcode + tok * KROW + lane * EPL) = make_uint2(packed[0], packed[1]);
-            else
-                *reinterpret_cast<uint32_t*>(kcode + tok * KROW + lane * EPL) = packed[0];
-#pragma unroll
-            for (int hh = 1; hh < EPL; hh <<= 1)
-#pragma unroll
-                for (int r = 0; r < EPL; r += 2 * hh) f[r] = __fadd_rn(f[r], f[r + hh]);
-            float nc2 = f[0];
-#pragma unroll
-            for (int m = 1; m < 32; m <<= 1) nc2 = __fadd_rn(nc2, __shfl_xor_sync(0xffffffffu, nc2, m));
-            const float nc = __fsqrt_rn(nc2);
-            if (lane == 0)
-                *reinterpret_cast<uint16_t*>(img + 12 * D + 2 * tok) =
-                    (nx == 0.0f) ? (uint16_t)0 : f32_to_f16_sat_bits(__fdiv_rn(nx, nc));
         }
-
-        // ---- values: one thread per channel, 16 tokens of the page ------------------------------
-        for (int c = tid; c < D; c += NT) {
-            const uint4 raw = *reinterpret_cast<const uint4*>(rec8 + 16 * D + c * kPage);
-            const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
-            float val[kPage];
-#pragma unroll
-            for (int t = 0; t < kPage; t += 2) {
-                const float2 f = e4m3x2_to_f32((rw[t >> 2] >> (8 * (t & 3))) & 0xFFFFu);
-                val[t] = __fmul_rn(f.x, v_scale);
-                val[t + 1] = __fmul_rn(f.y, v_scale);
-            }
-            float mn = val[0], mx = val[0];
-#pragma unroll
-            for (int t = 1; t < kPage; ++t) {
-                if (val[t] < mn) mn = val[t];
-                if (val[t] > mx) mx = val[t];
-            }
-            const uint16_t sc = f32_to_f16_sat_bits(__fdiv_rn(__fsub_rn(mx, mn), 7.0f));
-            const uint16_t zp = f32_to_f16_sat_bits(mn);
-            const float scf = __half2float(__ushort_as_half(sc)), zpf = __half2float(__ushort_as_half(zp));
-            {
-                const int cb = c >> 4, row = c & 15;
-                uint16_t* meta = reinterpret_cast<uint16_t*>(img + 12 * D + 32);
-                const int hi = (cb >> 1) * 64 + (row & 7) * 8 + 4 * (cb & 1) + (row >> 3);
-                meta[hi] = sc;
-                meta[hi + 2] = zp;
-            }
-            // q = clamp(rint((val - zp) / sc), 0, 7), 0 when sc == 0.  The division is the correctly
-            // rounded one; a zero numerator (the channel's minimum) or a zero scale is replaced by
-            // operands whose quotient is not used, which keeps the divider on its short path.
-            const float den = scf != 0.0f ? scf : 1.0f;
-            uint32_t q4[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-            for (int t = 0; t < kPage; ++t) {
-                const float num = __fsub_rn(val[t], zpf);
-                float r = rintf(__fdiv_rn(num != 0.0f ? num : den, den));   // half to even
-                r = r < 0.0f ? 0.0f : r;
-                r = r > 7.0f ? 7.0f : r;
-                const uint32_t q = (num != 0.0f && scf != 0.0f) ? (uint32_t)(int)r : 0u;
-                q4[t >> 2] |= q << (8 * (t & 3));
-            }
-            *reinterpret_cast<uint4*>(vcode + c * kPage) = make_uint4(q4[0], q4[1], q4[2], q4[3]);
-        }
-        __syncthreads();
-
-        // ---- pack: one thread per (section, triple j, fragment lane L) --------------------------
-        for (int item = tid; item < 2 * NJ * 32; item += NT) {
-            const int L = item & 31, j = (item >> 5) % NJ, section = item / (32 * NJ);
-            const int g = L >> 2, tq = L & 3;
-            uint32_t w0 = 0, w1 = 0, w2 = 0;
-            if (section == 0) {
-                // key codes: nibble n = 2r + half holds row g + 8(r&1), slot 2tq + 8(r>>1) + half.
-                // A: block 4j with the signs of block 4j+2; B: block 4j+1 with the signs of 4j+3;
-                // C: magnitudes of blocks 4j+2 (low pair) and 4j+3 (high pair).
-#pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    const uint8_t* at = kcode + (g + 8 * (r & 1)) * KROW + 64 * j + 2 * tq + 8 * (r >> 1);
-                    const uint32_t b0 = *reinterpret_cast<const uint16_t*>(at);        // (half 0, half 1)
-                    const uint32_t b1 = *reinterpret_cast<const uint16_t*>(at + 16);
-                    const uint32_t b2 = *reinterpret_cast<const uint16_t*>(at + 32);
-                    const uint32_t b3 = *reinterpret_cast<const uint16_t*>(at + 48);
-                    w0 |= squeeze_nibbles(b0 | ((b2 & 0x0404u) << 1)) << (8 * r);
-                    w1 |= squeeze_nibbles(b1 | ((b3 & 0x0404u) << 1)) << (8 * r);
-                    w2 |= squeeze_nibbles((b2 & 0x0303u) | ((b3 & 0x0303u) << 2)) << (8 * r);
-                }
-            } else {
-                // value codes: four 24-bit streams (group, half) per triple; stream code k is
-                // channel block 4j + 2 grp + (k>>2), row g + 8(k&1), token 2tq + 8((k>>1)&1) + half
-                uint32_t S[2][2] = {{0u, 0u}, {0u, 0u}};
-#pragma unroll
-                for (int grp = 0; grp < 2; ++grp)
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        const int cb = 4 * j + 2 * grp + (k >> 2), r = k & 3;
-                        const uint32_t two = *reinterpret_cast<const uint16_t*>(
-                            vcode + (16 * cb + g + 8 * (r & 1)) * kPage + 2 * tq + 8 * (r >> 1));
-                        S[grp][0] |= (two & 7u) << (3 * k);
-                        S[grp][1] |= (two >> 8) << (3 * k);
-                    }
-                w0 = (S[0][0] & 0xFFFFu) | (S[0][1] << 16);
-                w1 = (S[0][0] >> 16) | ((S[1][0] & 0xFFu) << 8) | ((S[0][1] >> 16) << 16) | (S[1][1] << 24);
-                w2 = (S[1][0] >> 8) | ((S[1][1] >> 8) << 16);
-            }
-            uint8_t* sec = img + section * 6 * D;
-            *reinterpret_cast<uint32_t*>(sec + lane_word_offset(D, L, 3 * j)) = w0;
-            *reinterpret_cast<uint32_t*>(sec + lane_word_offset(D, L, 3 * j + 1)) = w1;
-            *reinterpret_cast<uint32_t*>(sec + lane_word_offset(D, L, 3 * j + 2)) = w2;
-        }
-        __syncthreads();
-        for (int i = tid; i < REC / 16; i += NT)
-            reinterpret_cast<uint4*>(rec3)[i] = reinterpret_cast<const uint4*>(img)[i];
     }
 
     // copy-before-publish: every head's record is complete and visible before the id and tag appear
@@ -478,19 +528,114 @@ __global__ void __launch_bounds__(D) demote_kernel(const uint8_t* __restrict__ f
     }
 }
 
+// Pages of several tiles, first pass of Demote: thread c finds the minimum and maximum of value channel c
+// over all tokens of the page and writes the page's scale and zero (same arithmetic and order of the
+// halves as in the 16-token record).  One block per (page, KV head).
+template <int D>
+__global__ void __launch_bounds__(D) demote_minmax_kernel(const uint8_t* __restrict__ fp8, uint8_t* __restrict__ tq3,
+                                                           int fp8_pages, int tq3_pages, int hkv, int tiles,
+                                                           float v_scale, const int32_t* __restrict__ src_ids,
+                                                           const int32_t* __restrict__ dst_ids)
+{
+    const int page = blockIdx.x / hkv, h = blockIdx.x % hkv, c = threadIdx.x;
+    const int src = src_ids[page], dst = dst_ids[page];
+    if (src < 0 || src >= fp8_pages || dst < 0 || dst >= tq3_pages) return;      // flagged by demote_kernel
+    const uint8_t* page8 = fp8 + ((size_t)src * hkv + h) * fp8_page_bytes(D, tiles);
+    float mn = 0.f, mx = 0.f;
+    for (int m = 0; m < tiles; ++m) {
+        const uint4 raw = *reinterpret_cast<const uint4*>(page8 + (size_t)m * fp8_record_bytes(D) + 16 * D + c * kPage);
+        const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+        for (int t = 0; t < kPage; t += 2) {
+            const float2 f = e4m3x2_to_f32((rw[t >> 2] >> (8 * (t & 3))) & 0xFFFFu);
+            const float a = __fmul_rn(f.x, v_scale), b = __fmul_rn(f.y, v_scale);
+            if (m == 0 && t == 0) mn = mx = a;
+            if (a < mn) mn = a;
+            if (a > mx) mx = a;
+            if (b < mn) mn = b;
+            if (b > mx) mx = b;
+        }
+    }
+    uint16_t* meta = reinterpret_cast<uint16_t*>(tq3 + ((size_t)dst * hkv + h) * tq3_page_bytes(D, tiles) +
+                                                 (size_t)tiles * (12 * D + 32));
+    const int cb = c >> 4, row = c & 15;
+    const int hi = (cb >> 1) * 64 + (row & 7) * 8 + 4 * (cb & 1) + (row >> 3);
+    meta[hi] = f32_to_f16_sat_bits(__fdiv_rn(__fsub_rn(mx, mn), 7.0f));
+    meta[hi + 2] = f32_to_f16_sat_bits(mn);
+}
+
+// Pages of several tiles, last pass of Demote / Promote: the kernels before it in the stream have written the
+// whole page, so its id and tag may appear (copy-before-publish by stream order).
+__global__ void publish_kernel(int n, const int32_t* __restrict__ src_ids, const int32_t* __restrict__ dst_ids,
+                               int src_cap, int dst_cap, int32_t* block_table, uint8_t* tier_tag,
+                               const int64_t* __restrict__ entry_index, int tag)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int src = src_ids[i], dst = dst_ids[i];
+    if (src < 0 || src >= src_cap || dst < 0 || dst >= dst_cap) return;
+    const int64_t e = entry_index[i];
+    if (e >= 0) {
+        block_table[e] = dst;
+        __threadfence();
+        tier_tag[e] = (uint8_t)tag;
+    }
+}
+
+// grid rows of the tile-parallel passes
+static int tile_rows(int tiles) { return tiles < 16 ? tiles : 16; }
+
+template <typename Kernel, typename... Args>
+static cudaError_t launch_clustered_rows(Kernel kernel, int n_pages, int csize, int rows, int threads, cudaStream_t s,
+                                         Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)n_pages * csize, rows);
+    cfg.blockDim = dim3(threads);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = csize;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
+template <int D>
+static int32_t launch_demote_d(mkv_pool* p, const int32_t* src, const int32_t* dst, int n, int32_t* bt, uint8_t* tags,
+                               const int64_t* entry, cudaStream_t s)
+{
+    const int c = heads_cluster(p->hkv, n);
+    if (p->tiles == 1) {
+        MKV_CUDA(launch_clustered(demote_kernel<D, false>, n, c, D, s, (const uint8_t*)p->fp8, p->tq3, p->cfg.fp8_pages,
+                                  p->cfg.tq3_pages, p->hkv, 1, p->cfg.k_scale, p->cfg.v_scale, p->sigma, src, dst, bt,
+                                  tags, entry, p->status_dev));
+        return MKV_OK;
+    }
+    // pages of several tiles: scale/zero of the page, then the tiles in parallel, then the publication
+    demote_minmax_kernel<D><<<n * p->hkv, D, 0, s>>>(p->fp8, p->tq3, p->cfg.fp8_pages, p->cfg.tq3_pages, p->hkv, p->tiles,
+                                                     p->cfg.v_scale, src, dst);
+    MKV_CUDA(cudaGetLastError());
+    MKV_CUDA(launch_clustered_rows(demote_kernel<D, true>, n, heads_cluster(p->hkv, 0), tile_rows(p->tiles), D, s,
+                                   (const uint8_t*)p->fp8, p->tq3, p->cfg.fp8_pages, p->cfg.tq3_pages, p->hkv, p->tiles,
+                                   p->cfg.k_scale, p->cfg.v_scale, p->sigma, src, dst, (int32_t*)nullptr,
+                                   (uint8_t*)nullptr, (const int64_t*)nullptr, p->status_dev));
+    if (entry) {
+        publish_kernel<<<(n + 127) / 128, 128, 0, s>>>(n, src, dst, p->cfg.fp8_pages, p->cfg.tq3_pages, bt, tags, entry,
+                                                       MKV_TAG_STALE);
+        MKV_CUDA(cudaGetLastError());
+    }
+    (void)c;
+    return MKV_OK;
+}
+
 int32_t launch_demote(mkv_pool* p, const int32_t* src, const int32_t* dst, int n, int32_t* bt, uint8_t* tags,
                       const int64_t* entry, cudaStream_t s)
 {
-    const int c = heads_cluster(p->hkv, n);
-    if (p->d == 128)
-        MKV_CUDA(launch_clustered(demote_kernel<128>, n, c, 128, s, (const uint8_t*)p->fp8, p->tq3, p->cfg.fp8_pages,
-                                  p->cfg.tq3_pages, p->hkv, p->cfg.k_scale, p->cfg.v_scale, p->sigma, src, dst, bt, tags,
-                                  entry, p->status_dev));
-    else
-        MKV_CUDA(launch_clustered(demote_kernel<256>, n, c, 256, s, (const uint8_t*)p->fp8, p->tq3, p->cfg.fp8_pages,
-                                  p->cfg.tq3_pages, p->hkv, p->cfg.k_scale, p->cfg.v_scale, p->sigma, src, dst, bt, tags,
-                                  entry, p->status_dev));
-    return MKV_OK;
+    return p->d == 128 ? launch_demote_d<128>(p, src, dst, n, bt, tags, entry, s)
+                       : launch_demote_d<256>(p, src, dst, n, bt, tags, entry, s);
 }
 
 // ------------------------------------------------------------------------------------------ promote
@@ -504,9 +649,9 @@ int32_t launch_demote(mkv_pool* p, const int32_t* src, const int32_t* dst, int n
 // L = 4 (row % 8) + (slot % 8) / 2 holds, in nibble 2 rr + slot % 2 with rr = row / 8 + 2 (slot / 8),
 // the entry (row, slot) of every 16 x 16 block; for keys row = token and slot = channel % 16, for
 // values row = channel % 16 and slot = token.
-template <int D>
+template <int D, bool BIG>
 __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ tq3, uint8_t* __restrict__ fp8,
-                                                     int tq3_pages, int fp8_pages, int hkv, float inv_k_scale,
+                                                     int tq3_pages, int fp8_pages, int hkv, int tiles, float inv_k_scale,
                                                      float inv_v_scale, float rs, SigmaBits sigma,
                                                      const int32_t* __restrict__ src_ids,
                                                      const int32_t* __restrict__ dst_ids, int32_t* block_table,
@@ -523,7 +668,7 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
     const int page = blockIdx.x / csize, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int src = src_ids[page], dst = dst_ids[page];
     const bool valid = src >= 0 && src < tq3_pages && dst >= 0 && dst < fp8_pages;
-    if (!valid && tid == 0 && crank == 0) atomicOr(status, kStBounds);
+    if (!valid && tid == 0 && crank == 0 && blockIdx.y == 0) atomicOr(status, kStBounds);
     if (tid < 8) {
         const float c = (tid & 3) == 0 ? MKV_C0 : (tid & 3) == 1 ? MKV_C1 : (tid & 3) == 2 ? MKV_C2 : MKV_C3;
         level[tid] = (tid & 4) ? -c : c;
@@ -557,12 +702,26 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
     const uint32_t sel0 = grp == 0 ? 0x0410u : 0x0541u, sel1 = grp == 0 ? 0x0632u : 0x0763u;
     const int meta_i = (cb >> 1) * 64 + (row & 7) * 8 + 4 * (cb & 1) + (row >> 3);
 
-    for (int h = crank, it = 0; valid && h < hkv; h += csize, ++it) {
-        const uint8_t* rec3 = tq3 + ((size_t)src * hkv + h) * tq3_record_bytes(D);
-        uint8_t* rec8 = fp8 + ((size_t)dst * hkv + h) * fp8_record_bytes(D);
-        uint8_t* img = image[it & 1];
-        for (int i = tid; i < REC / 16; i += NT)
-            reinterpret_cast<uint4*>(img)[i] = reinterpret_cast<const uint4*>(rec3)[i];
+    // 16-token pages: one record per head.  Pages of several tiles: the blocks of grid row y take tiles y,
+    // y + gridDim.y, ...; a tile and the page's scale/zero behind it form the same image as a 16-token record.
+    constexpr int TILE = 12 * D + 32;
+    const int m_first = BIG ? (int)blockIdx.y : 0, m_step = BIG ? (int)gridDim.y : 1, m_end = BIG ? tiles : 1;
+    int it = 0;
+    for (int h = crank; valid && h < hkv; h += csize)
+    for (int m = m_first; m < m_end; m += m_step) {
+        const uint8_t* rec3 = tq3 + ((size_t)src * hkv + h) * tq3_page_bytes(D, tiles) + (size_t)m * TILE;
+        uint8_t* rec8 = fp8 + (((size_t)dst * hkv + h) * tiles + m) * fp8_record_bytes(D);
+        uint8_t* img = image[it++ & 1];
+        if constexpr (!BIG) {
+            for (int i = tid; i < REC / 16; i += NT)
+                reinterpret_cast<uint4*>(img)[i] = reinterpret_cast<const uint4*>(rec3)[i];
+        } else {
+            const uint8_t* meta = tq3 + ((size_t)src * hkv + h) * tq3_page_bytes(D, tiles) + (size_t)tiles * TILE;
+            for (int i = tid; i < TILE / 16; i += NT)
+                reinterpret_cast<uint4*>(img)[i] = reinterpret_cast<const uint4*>(rec3)[i];
+            for (int i = tid; i < 4 * D / 16; i += NT)
+                reinterpret_cast<uint4*>(img + TILE)[i] = reinterpret_cast<const uint4*>(meta)[i];
+        }
         __syncthreads();
 
         // ---- keys: warp w rebuilds tokens w, w + NT/32, ...
@@ -652,19 +811,35 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
     }
 }
 
-int32_t launch_promote(mkv_pool* p, const int32_t* src, const int32_t* dst, int n, int32_t* bt, uint8_t* tags,
-                       const int64_t* entry, cudaStream_t s)
+template <int D>
+static int32_t launch_promote_d(mkv_pool* p, const int32_t* src, const int32_t* dst, int n, int32_t* bt, uint8_t* tags,
+                                const int64_t* entry, cudaStream_t s)
 {
     const float ik = 1.0f / p->cfg.k_scale, iv = 1.0f / p->cfg.v_scale;
     const float rs = (float)(1.0 / sqrt((double)p->d));
-    const int c = heads_cluster(p->hkv, n);
-    if (p->d == 128)
-        MKV_CUDA(launch_clustered(promote_kernel<128>, n, c, 128, s, (const uint8_t*)p->tq3, p->fp8, p->cfg.tq3_pages,
-                                  p->cfg.fp8_pages, p->hkv, ik, iv, rs, p->sigma, src, dst, bt, tags, entry, p->status_dev));
-    else
-        MKV_CUDA(launch_clustered(promote_kernel<256>, n, c, 256, s, (const uint8_t*)p->tq3, p->fp8, p->cfg.tq3_pages,
-                                  p->cfg.fp8_pages, p->hkv, ik, iv, rs, p->sigma, src, dst, bt, tags, entry, p->status_dev));
+    if (p->tiles == 1) {
+        MKV_CUDA(launch_clustered(promote_kernel<D, false>, n, heads_cluster(p->hkv, n), D, s, (const uint8_t*)p->tq3, p->fp8,
+                                  p->cfg.tq3_pages, p->cfg.fp8_pages, p->hkv, 1, ik, iv, rs, p->sigma, src, dst, bt, tags,
+                                  entry, p->status_dev));
+        return MKV_OK;
+    }
+    MKV_CUDA(launch_clustered_rows(promote_kernel<D, true>, n, heads_cluster(p->hkv, 0), tile_rows(p->tiles), D, s,
+                                   (const uint8_t*)p->tq3, p->fp8, p->cfg.tq3_pages, p->cfg.fp8_pages, p->hkv, p->tiles, ik,
+                                   iv, rs, p->sigma, src, dst, (int32_t*)nullptr, (uint8_t*)nullptr,
+                                   (const int64_t*)nullptr, p->status_dev));
+    if (entry) {
+        publish_kernel<<<(n + 127) / 128, 128, 0, s>>>(n, src, dst, p->cfg.tq3_pages, p->cfg.fp8_pages, bt, tags, entry,
+                                                       MKV_TAG_ANCHOR);
+        MKV_CUDA(cudaGetLastError());
+    }
     return MKV_OK;
+}
+
+int32_t launch_promote(mkv_pool* p, const int32_t* src, const int32_t* dst, int n, int32_t* bt, uint8_t* tags,
+                       const int64_t* entry, cudaStream_t s)
+{
+    return p->d == 128 ? launch_promote_d<128>(p, src, dst, n, bt, tags, entry, s)
+                       : launch_promote_d<256>(p, src, dst, n, bt, tags, entry, s);
 }
 
 // ------------------------------------------------------------------------------------------ anchor

@@ -33,6 +33,14 @@ struct SigmaBits {
 
 __host__ __device__ inline size_t fp8_record_bytes(int d) { return (size_t)32 * d; }
 __host__ __device__ inline size_t tq3_record_bytes(int d) { return (size_t)16 * d + 32; }
+// Pages of `tiles` 16-token tiles (Section 4.1 stores blocks of 1,792 / 832 tokens): an FP8 page is `tiles`
+// consecutive 16-token records; a TQ3 page is `tiles` tile records (key codes, value codes, g: 12 d + 32
+// bytes each) followed by ONE set of value scale/zero (4 d bytes) shared by all its tokens.  tiles = 1 gives
+// the 16-token records above.
+__host__ __device__ inline size_t tq3_tile_bytes(int d) { return (size_t)12 * d + 32; }
+__host__ __device__ inline size_t fp8_page_bytes(int d, int tiles) { return (size_t)tiles * 32 * d; }
+__host__ __device__ inline size_t tq3_page_bytes(int d, int tiles) { return (size_t)tiles * (12 * d + 32) + (size_t)4 * d; }
+constexpr int kMaxTiles = 256;       // pages of at most 4,096 tokens
 
 // ---- TQ3 record geometry -------------------------------------------------------------------
 // The code sections are laid out for the m16n8k16 A-fragment: "lane" L = 4*g + tq owns rows
@@ -55,6 +63,7 @@ struct Device {
 struct mkv_pool {
     mkv_pool_config cfg;
     int d, hkv, hq, group;
+    int tiles;                   // 16-token tiles per page (cfg.page_size / 16)
     uint8_t* fp8;
     uint8_t* tq3;
     uint32_t* status_dev;

@@ -24,7 +24,7 @@ static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 static int32_t check_cfg(const mkv_pool_config* c)
 {
     if (!c) return MKV_E_INVALID;
-    if (c->page_size != kPage) return MKV_E_INVALID;
+    if (c->page_size < kPage || c->page_size % kPage || c->page_size > kPage * kMaxTiles) return MKV_E_INVALID;
     if (c->head_dim != 128 && c->head_dim != 256) return MKV_E_INVALID;
     if (c->n_kv_heads < 1 || c->n_q_heads < c->n_kv_heads) return MKV_E_INVALID;
     if (c->n_q_heads % c->n_kv_heads) return MKV_E_INVALID;
@@ -55,8 +55,9 @@ int32_t mkv_pool_query(const mkv_pool_config* cfg, size_t* fp8_bytes, size_t* tq
     int32_t rc = check_cfg(cfg);
     if (rc) return rc;
     if (!fp8_bytes || !tq3_bytes) return MKV_E_INVALID;
-    *fp8_bytes = (size_t)cfg->fp8_pages * cfg->n_kv_heads * fp8_record_bytes(cfg->head_dim) + kStatusTail;
-    *tq3_bytes = (size_t)cfg->tq3_pages * cfg->n_kv_heads * tq3_record_bytes(cfg->head_dim);
+    const int tiles = cfg->page_size / kPage;
+    *fp8_bytes = (size_t)cfg->fp8_pages * cfg->n_kv_heads * fp8_page_bytes(cfg->head_dim, tiles) + kStatusTail;
+    *tq3_bytes = (size_t)cfg->tq3_pages * cfg->n_kv_heads * tq3_page_bytes(cfg->head_dim, tiles);
     if (*tq3_bytes == 0) *tq3_bytes = 256;
     return MKV_OK;
 }
@@ -104,6 +105,7 @@ static mkv_pool* new_pool(const mkv_pool_config* cfg, void* fp8_arena, void* tq3
     p->hkv = cfg->n_kv_heads;
     p->hq = cfg->n_q_heads;
     p->group = cfg->n_q_heads / cfg->n_kv_heads;
+    p->tiles = cfg->page_size / kPage;
     p->fp8 = static_cast<uint8_t*>(fp8_arena);
     p->tq3 = static_cast<uint8_t*>(tq3_arena);
     p->variant = MKV_DECODE_TENSOR;
@@ -200,9 +202,9 @@ int32_t mkv_pool_stats(const mkv_pool* pool, mkv_stats* out)
     out->tq3_pages_total = p->cfg.tq3_pages;
     out->fp8_pages_used = p->cfg.fp8_pages - (int64_t)p->free_list[0].size();
     out->tq3_pages_used = p->cfg.tq3_pages - (int64_t)p->free_list[1].size();
-    out->fp8_bytes_used = out->fp8_pages_used * p->hkv * (int64_t)fp8_record_bytes(p->d);
-    out->tq3_bytes_used = out->tq3_pages_used * p->hkv * (int64_t)tq3_record_bytes(p->d);
-    out->bf16_bytes_equivalent = (out->fp8_pages_used + out->tq3_pages_used) * p->hkv * (int64_t)kPage * p->d * 4;
+    out->fp8_bytes_used = out->fp8_pages_used * p->hkv * (int64_t)fp8_page_bytes(p->d, p->tiles);
+    out->tq3_bytes_used = out->tq3_pages_used * p->hkv * (int64_t)tq3_page_bytes(p->d, p->tiles);
+    out->bf16_bytes_equivalent = (out->fp8_pages_used + out->tq3_pages_used) * p->hkv * (int64_t)p->cfg.page_size * p->d * 4;
     return MKV_OK;
 }
 
@@ -235,7 +237,7 @@ static int32_t raw_span(mkv_pool* pool, int32_t fmt, int32_t id, uint8_t** ptr, 
     if (!pool || !pool->fp8 || (fmt != MKV_FMT_FP8 && fmt != MKV_FMT_TQ3)) return MKV_E_INVALID;
     int cap = fmt == MKV_FMT_FP8 ? pool->cfg.fp8_pages : pool->cfg.tq3_pages;
     if (id < 0 || id >= cap) return MKV_E_BOUNDS;
-    size_t rec = fmt == MKV_FMT_FP8 ? fp8_record_bytes(pool->d) : tq3_record_bytes(pool->d);
+    size_t rec = fmt == MKV_FMT_FP8 ? fp8_page_bytes(pool->d, pool->tiles) : tq3_page_bytes(pool->d, pool->tiles);
     *bytes = rec * pool->hkv;
     *ptr = (fmt == MKV_FMT_FP8 ? pool->fp8 : pool->tq3) + (size_t)id * *bytes;
     return MKV_OK;
@@ -313,6 +315,10 @@ int32_t mkv_decode_attention(mkv_pool* pool, const void* q, const int32_t* bt, c
     size_t need;
     if (mkv_decode_workspace_bytes(&pool->cfg, B, &need) != MKV_OK || ws_bytes < need) return MKV_E_INVALID;
     if (!(scale == scale)) return MKV_E_INVALID;
+    if (pool->variant == MKV_DECODE_SCALAR && pool->tiles > 1) {
+        set_last_error("mkv_decode_attention: pages of several tiles are served by the tensor-core kernel only");
+        return MKV_E_INVALID;
+    }
     if (pool->variant == MKV_DECODE_SCALAR)
         return launch_decode_scalar(pool, q, bt, tags, lens, B, max_pages, scale, out, lse, ws, ws_bytes,
                                     (cudaStream_t)stream);
@@ -378,7 +384,8 @@ int32_t mkv_seq_finish(mkv_seq* seq)
 int32_t mkv_seq_append(mkv_seq* seq, int32_t* page_id, int32_t* slot, int32_t* opened)
 {
     if (!seq || !page_id || !slot) return MKV_E_INVALID;
-    bool open = seq->len % kPage == 0;
+    const int T = seq->pool->cfg.page_size;
+    bool open = seq->len % T == 0;
     if (open) {
         int32_t id;
         int32_t rc = mkv_page_alloc(seq->pool, MKV_FMT_FP8, &id, 1);
@@ -387,7 +394,7 @@ int32_t mkv_seq_append(mkv_seq* seq, int32_t* page_id, int32_t* slot, int32_t* o
         seq->tags.push_back(MKV_TAG_RECENT);
     }
     *page_id = seq->ids.back();
-    *slot = seq->len % kPage;
+    *slot = seq->len % T;
     if (opened) *opened = open ? 1 : 0;
     seq->len += 1;
     return MKV_OK;
@@ -408,7 +415,7 @@ int32_t mkv_seq_demote(mkv_seq* seq, int32_t lp, int32_t* src, int32_t* dst)
     if (!seq || !src || !dst) return MKV_E_INVALID;
     if (lp < 0 || (size_t)lp >= seq->ids.size()) return MKV_E_BOUNDS;
     if (seq->tags[lp] == MKV_TAG_STALE) return MKV_E_STATE;
-    if ((lp + 1) * kPage > seq->len) return MKV_E_STATE;   // only full pages may become TQ3
+    if ((int64_t)(lp + 1) * seq->pool->cfg.page_size > seq->len) return MKV_E_STATE;   // only full pages may become TQ3
     int32_t id;
     int32_t rc = mkv_page_alloc(seq->pool, MKV_FMT_TQ3, &id, 1);
     if (rc) return rc;
@@ -438,11 +445,12 @@ int32_t mkv_seq_age(mkv_seq* seq, int32_t recent_tokens, int32_t* lps, int32_t* 
                     int32_t cap, int32_t* n)
 {
     if (!seq || !n || recent_tokens < 0 || cap < 0) return MKV_E_INVALID;
-    int first_recent = (seq->len - recent_tokens > 0 ? seq->len - recent_tokens : 0) / kPage;
+    const int T = seq->pool->cfg.page_size;
+    int first_recent = (seq->len - recent_tokens > 0 ? seq->len - recent_tokens : 0) / T;
     if ((size_t)first_recent > seq->ids.size()) first_recent = (int)seq->ids.size();
     int need = 0;
     for (int lp = 0; lp < first_recent; ++lp)
-        if (seq->tags[lp] == MKV_TAG_RECENT && (lp + 1) * kPage <= seq->len) ++need;
+        if (seq->tags[lp] == MKV_TAG_RECENT && (int64_t)(lp + 1) * T <= seq->len) ++need;
     if (need > cap || (need > 0 && (!lps || !srcs || !dsts))) return MKV_E_INVALID;
     {
         std::lock_guard<std::mutex> lk(seq->pool->mu);
@@ -450,7 +458,7 @@ int32_t mkv_seq_age(mkv_seq* seq, int32_t recent_tokens, int32_t* lps, int32_t* 
     }
     int k = 0;
     for (int lp = 0; lp < first_recent; ++lp)
-        if (seq->tags[lp] == MKV_TAG_RECENT && (lp + 1) * kPage <= seq->len) {
+        if (seq->tags[lp] == MKV_TAG_RECENT && (int64_t)(lp + 1) * T <= seq->len) {
             int32_t rc = mkv_seq_demote(seq, lp, &srcs[k], &dsts[k]);
             if (rc) return rc;
             lps[k++] = lp;

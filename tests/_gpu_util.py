@@ -21,7 +21,8 @@ class Case:
         self.tab = W.tables(spec, extra_fp8, extra_tq3)
         self.L = build_layer(spec, self.tab, layer)
         self.pool = M.Pool(spec.head_dim, spec.n_kv_heads, spec.n_q_heads, max(self.tab.fp8_pages, 1),
-                           max(self.tab.tq3_pages, 1), self.L.sigma, k_scale, v_scale, max_batch=spec.batch)
+                           max(self.tab.tq3_pages, 1), self.L.sigma, k_scale, v_scale, max_batch=spec.batch,
+                           page_tokens=spec.page_tokens)
         self.pool.upload_arenas(self.L.fp8_arena, self.L.tq3_arena)
         self.q = bf16_tensor(self.L.q_bits)
         self.bt = torch.from_numpy(self.tab.block_table).cuda()
@@ -40,7 +41,8 @@ class Case:
         s = self.spec
         return oracle.decode_attention(self.L.fp8_arena, self.L.tq3_arena, s.head_dim, s.n_kv_heads, s.group,
                                        self.L.sigma, self.L.q_bits, self.tab.block_table, self.tab.tier_tag,
-                                       self.tab.seq_lens, s.scale, only_b=only_b, only_h=only_h)
+                                       self.tab.seq_lens, s.scale, only_b=only_b, only_h=only_h,
+                                       page_tokens=s.page_tokens)
 
 
 def check_close(got, ref, what=""):

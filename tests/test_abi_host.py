@@ -44,9 +44,14 @@ def test_query_and_argument_validation_without_a_device():
             M.mkv_pool_query(c)
         assert e.value.code == M.E_INVALID
     c = M.make_config(128, 1, 1, 1, 1, np.ones(128, np.int8))
-    c.page_size = 32
-    with pytest.raises(M.MkvError):
-        M.mkv_pool_query(c)
+    for bad_page in (0, 8, 24, 4112):                       # a page is 16 M tokens, M <= 256
+        c.page_size = bad_page
+        with pytest.raises(M.MkvError):
+            M.mkv_pool_query(c)
+    # pages of 1,792 tokens, 4 KV heads, d = 256: the block sizes behind the paper's byte counters (Section 5.4)
+    c = M.make_config(256, 4, 24, 18, 47, np.ones(256, np.int8), page_tokens=1792)
+    fp8, tq3 = M.mkv_pool_query(c)
+    assert fp8 - 256 + tq3 == 131_610_624
     # device calls on a bookkeeping-only pool are refused, not attempted
     hp = M.HostPool(128, 2, 8, 4, 4)
     L = M.lib()
