@@ -124,13 +124,15 @@ def build_layers(spec, steps_total, device, M, torch):
     """Pools of every layer filled through the library's own Append and Demote kernels from seeded
     synthetic bf16 K/V, plus the tables, slots and retier plan of every timed step."""
     B, d, hkv, hq = spec.batch, spec.head_dim, spec.n_kv_heads, spec.n_q_heads
+    T = spec.page_tokens                      # 16, or 16 M for the paper-scale pages
+    stage_pages = max(1, STAGE_PAGES * 16 // T)
     final_lens = [n + steps_total for n in spec.seq_lens]
-    max_pages = max((n + 15) // 16 for n in final_lens) + 1
+    max_pages = max((n + T - 1) // T for n in final_lens) + 1
     tab0 = W.tables(spec)
     n_fp8_0, n_tq3_0 = tab0.fp8_pages, tab0.tq3_pages
-    extra_pages = sum((fl + 15) // 16 - (n + 15) // 16 for fl, n in zip(final_lens, spec.seq_lens))
-    demotes_per_req = steps_total // 16 + 2
-    fp8_cap = n_fp8_0 + extra_pages + STAGE_PAGES + 8
+    extra_pages = sum((fl + T - 1) // T - (n + T - 1) // T for fl, n in zip(final_lens, spec.seq_lens))
+    demotes_per_req = steps_total // T + 2
+    fp8_cap = n_fp8_0 + extra_pages + stage_pages + 8
     tq3_cap = n_tq3_0 + B * demotes_per_req + 8
 
     # host plan shared by all layers: table, tags, per-step slots and retier events
@@ -140,7 +142,7 @@ def build_layers(spec, steps_total, device, M, torch):
     tg[:, :tab0.tier_tag.shape[1]] = tab0.tier_tag
     next_fp8, next_tq3 = n_fp8_0, n_tq3_0
     lens = np.array(spec.seq_lens, np.int64)
-    n_pages = (lens + 15) // 16
+    n_pages = (lens + T - 1) // T
     slots = np.zeros((steps_total, B), np.int32)
     lens_steps = np.zeros((steps_total, B), np.int32)
     events = []              # per step: list of (b, logical page, src fp8 id, dst tq3 id)
@@ -148,16 +150,16 @@ def build_layers(spec, steps_total, device, M, torch):
     for st in range(steps_total):
         ev = []
         for b in range(B):
-            if lens[b] % 16 == 0:                       # Append opens a Recent page
+            if lens[b] % T == 0:                        # Append opens a Recent page
                 bt[b, n_pages[b]] = next_fp8
                 tg[b, n_pages[b]] = W.TAG_RECENT
                 next_fp8 += 1
                 n_pages[b] += 1
-            slots[st, b] = bt[b, lens[b] // 16] * 16 + lens[b] % 16
+            slots[st, b] = bt[b, lens[b] // T] * T + lens[b] % T
             lens[b] += 1
             lens_steps[st, b] = lens[b]
             # age: a full Recent page wholly before the window is demoted (tags tracked on the host too)
-            first_recent = max(0, lens[b] - recent) // 16
+            first_recent = max(0, lens[b] - recent) // T
             for lp in range(max(0, first_recent - 2), first_recent):
                 if tg[b, lp] == W.TAG_RECENT:
                     ev.append((b, lp, int(bt[b, lp]), next_tq3))
@@ -165,14 +167,14 @@ def build_layers(spec, steps_total, device, M, torch):
                     bt[b, lp] = next_tq3
                     next_tq3 += 1
         events.append(ev)
-    assert next_fp8 <= fp8_cap - STAGE_PAGES and next_tq3 <= tq3_cap
+    assert next_fp8 <= fp8_cap - stage_pages and next_tq3 <= tq3_cap
 
     layers = []
     gen = torch.Generator(device=device)
     for layer in range(spec.n_layers):
         L = LayerState()
         sigma = W.rotation_signs(spec, layer)
-        L.pool = M.Pool(d, hkv, hq, fp8_cap, tq3_cap, sigma, max_batch=B, device=device)
+        L.pool = M.Pool(d, hkv, hq, fp8_cap, tq3_cap, sigma, max_batch=B, device=device, page_tokens=T)
         gen.manual_seed(1000 * spec.seed + layer)
         k_out = torch.from_numpy(W.outlier_channels(spec, layer, 0)).to(device)
         v_out = torch.from_numpy(W.outlier_channels(spec, layer, 1)).to(device)
@@ -184,25 +186,25 @@ def build_layers(spec, steps_total, device, M, torch):
             v[:, :, v_out] *= 8.0
             return k.to(torch.bfloat16).contiguous(), v.to(torch.bfloat16).contiguous()
 
-        stage0 = fp8_cap - STAGE_PAGES
+        stage0 = fp8_cap - stage_pages
         for b in range(B):
-            npg = (spec.seq_lens[b] + 15) // 16
+            npg = (spec.seq_lens[b] + T - 1) // T
             tags_b, ids_b = tab0.tier_tag[b, :npg], tab0.block_table[b, :npg]
             fp8_lp = np.nonzero(tags_b != W.TAG_STALE)[0]
             # Recent/Anchor pages: append straight into their pages
-            tok = np.concatenate([np.arange(lp * 16, min(lp * 16 + 16, spec.seq_lens[b])) for lp in fp8_lp]) \
+            tok = np.concatenate([np.arange(lp * T, min(lp * T + T, spec.seq_lens[b])) for lp in fp8_lp]) \
                 if len(fp8_lp) else np.zeros(0, np.int64)
             if len(tok):
-                sm = (ids_b[tok // 16].astype(np.int64) * 16 + tok % 16).astype(np.int32)
+                sm = (ids_b[tok // T].astype(np.int64) * T + tok % T).astype(np.int32)
                 k, v = synth(len(tok))
                 L.pool.append(k, v, torch.from_numpy(sm).to(device))
             # Stale pages: append into staging FP8 pages, demote into their TQ3 pages, reuse the staging pages
             st_lp = np.nonzero(tags_b == W.TAG_STALE)[0]
-            for c0 in range(0, len(st_lp), STAGE_PAGES):
-                chunk = st_lp[c0:c0 + STAGE_PAGES]
+            for c0 in range(0, len(st_lp), stage_pages):
+                chunk = st_lp[c0:c0 + stage_pages]
                 n = len(chunk)
-                sm = ((stage0 + np.arange(n))[:, None] * 16 + np.arange(16)[None, :]).reshape(-1).astype(np.int32)
-                k, v = synth(16 * n)
+                sm = ((stage0 + np.arange(n))[:, None] * T + np.arange(T)[None, :]).reshape(-1).astype(np.int32)
+                k, v = synth(T * n)
                 L.pool.append(k, v, torch.from_numpy(sm).to(device))
                 src = torch.arange(stage0, stage0 + n, dtype=torch.int32, device=device)
                 dst = torch.from_numpy(ids_b[chunk].astype(np.int32)).to(device)
@@ -253,12 +255,13 @@ def initial_tags(tab0, tg_final):
 
 
 def kv_bytes_at(spec, tags_host_rows, lens_row):
-    """Algorithmic KV bytes of one decode launch: 2d per valid FP8 token + (16d + 32) per Stale page, per KV head."""
-    d, total = spec.head_dim, 0
+    """Algorithmic KV bytes of one decode launch: 2d per valid FP8 token + M (12d + 32) + 4d per Stale page of
+    16 M tokens (16d + 32 at M = 1), per KV head."""
+    d, total, T, Mt = spec.head_dim, 0, spec.page_tokens, spec.tiles_per_page
     for b, ln in enumerate(lens_row):
-        npg = (int(ln) + 15) // 16
+        npg = (int(ln) + T - 1) // T
         stale = int((tags_host_rows[b, :npg] == W.TAG_STALE).sum())
-        total += spec.n_kv_heads * ((int(ln) - 16 * stale) * 2 * d + stale * (16 * d + 32))
+        total += spec.n_kv_heads * ((int(ln) - T * stale) * 2 * d + stale * (Mt * (12 * d + 32) + 4 * d))
     return total
 
 
@@ -470,7 +473,7 @@ def run_ours(args):
         "warmup": Wm, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "u8 codes (e4m3 / 3-bit TQ3) -> f16 tensor-core operands, f32 accumulate", "data": "synthetic",
         "config": {"workload": workload_name(spec), "batch": B, "context_tokens": list(spec.seq_lens)[:4],
-                   "layers": spec.n_layers, "head_dim": d, "kv_heads": hkv, "q_heads": hq, "page_tokens": 16,
+                   "layers": spec.n_layers, "head_dim": d, "kv_heads": hkv, "q_heads": hq, "page_tokens": spec.page_tokens,
                    "parallelism": "replicas only" if world > 1 else "single GPU",
                    "l2": "inputs larger than L2 (%.0f MB of KV per step)" % (step_bytes / 1e6),
                    "step": "append + demote at its natural cadence + decode attention, every layer",
@@ -583,11 +586,15 @@ def workload_spec(args):
         over["seq_lens"] = (args.ctx,) * W.config(args.config).batch
     if args.config == 4:
         return W.config(4, batch=args.batch or 8, ctx=args.ctx or 32768, stale_fraction=args.stale, **over)
+    if args.config == 5 and args.layers <= 0:
+        over["n_layers"] = 16                      # the canary's 16 full-attention layers
     return W.config(args.config, **over)
 
 
 def workload_name(spec):
-    return {"cfg2_canary_59k": "configs[2]: 2 x 59,008 tokens, 16 layers, d=256, 4 KV x 6 q heads, ~96% TQ3 pages"}.get(
+    return {"cfg2_canary_59k": "configs[2]: 2 x 59,008 tokens, 16 layers, d=256, 4 KV x 6 q heads, ~96% TQ3 pages",
+            "cfg5_canary_blocks_1792": "the configs[2] shape with pages of 1,792 tokens (paper-scale blocks): 2 x 59,008 "
+                                       "tokens, d=256, 4 KV x 6 q heads, 10 FP8 + 23 TQ3 pages per request"}.get(
         spec.name, spec.name)
 
 
@@ -599,7 +606,8 @@ def oracle_sample(spec, seconds_hint=20.0):
     sub = W.config(0, seq_lens=[spec.seq_lens[b] for b in reqs], head_dim=spec.head_dim, n_kv_heads=spec.n_kv_heads,
                    group=spec.group, anchor_prefix=spec.anchor_prefix, anchor_spans=max(spec.anchor_spans, 0),
                    anchor_span_tokens=spec.anchor_span_tokens, recent_tokens=spec.recent_tokens,
-                   n_outlier=spec.n_outlier, seed=spec.seed, stale_fraction=spec.stale_fraction)
+                   n_outlier=spec.n_outlier, seed=spec.seed, stale_fraction=spec.stale_fraction,
+                   page_tokens=spec.page_tokens)
     tab = W.tables(sub)
     L = build_layer(sub, tab)
     return oracle, sub, tab, L
@@ -611,7 +619,7 @@ def time_oracle(spec, reps=3):
     for _ in range(reps):
         t0 = time.perf_counter()
         oracle.decode_attention(L.fp8_arena, L.tq3_arena, sub.head_dim, sub.n_kv_heads, sub.group, L.sigma, L.q_bits,
-                                tab.block_table, tab.tier_tag, tab.seq_lens, sub.scale)
+                                tab.block_table, tab.tier_tag, tab.seq_lens, sub.scale, page_tokens=sub.page_tokens)
         times.append(time.perf_counter() - t0)
     layer_s = sum(times) / len(times)
     # one decode step = all layers over the whole batch; the sample covers one layer of `sub.batch` requests
@@ -640,7 +648,7 @@ def run_reference(args):
     def one():
         t0 = time.perf_counter()
         oracle.decode_attention(L.fp8_arena, L.tq3_arena, sub.head_dim, sub.n_kv_heads, sub.group, L.sigma, L.q_bits,
-                                tab.block_table, tab.tier_tag, tab.seq_lens, sub.scale)
+                                tab.block_table, tab.tier_tag, tab.seq_lens, sub.scale, page_tokens=sub.page_tokens)
         return time.perf_counter() - t0
     for _ in range(Wm):
         one()
