@@ -582,6 +582,8 @@ def run_lifecycle(args):
 # ---------------------------------------------------------------------------------------- oracle arm
 def workload_spec(args):
     over = {"n_layers": args.layers} if args.layers > 0 else {}
+    if args.page_tokens > 0:
+        over["page_tokens"] = args.page_tokens
     if args.ctx > 0 and args.config != 4:
         over["seq_lens"] = (args.ctx,) * W.config(args.config).batch
     if args.config == 4:
@@ -592,6 +594,8 @@ def workload_spec(args):
 
 
 def workload_name(spec):
+    if spec.page_tokens != 16 and spec.name != "cfg5_canary_blocks_1792":
+        return "%s with pages of %d tokens" % (spec.name, spec.page_tokens)
     return {"cfg2_canary_59k": "configs[2]: 2 x 59,008 tokens, 16 layers, d=256, 4 KV x 6 q heads, ~96% TQ3 pages",
             "cfg5_canary_blocks_1792": "the configs[2] shape with pages of 1,792 tokens (paper-scale blocks): 2 x 59,008 "
                                        "tokens, d=256, 4 KV x 6 q heads, 10 FP8 + 23 TQ3 pages per request"}.get(
@@ -681,6 +685,8 @@ def main():
     ap.add_argument("--ctx", type=int, default=0, help="override the context length of every request (profiling)")
     ap.add_argument("--batch", type=int, default=0, help="config 4 only: requests of the lifecycle cell (default 8)")
     ap.add_argument("--stale", type=float, default=0.5, help="config 4 only: Stale fraction of the lifecycle cell")
+    ap.add_argument("--page-tokens", type=int, default=0,
+                    help="override the page size (a multiple of 16; 1792 and 832 are the paper's block sizes)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--lifecycle", action="store_true",
                     help="time Append, Demote and Promote alone (bulk throughput) instead of the decode step")

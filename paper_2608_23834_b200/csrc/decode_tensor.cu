@@ -337,7 +337,7 @@ __device__ __forceinline__ void partition_blocks_of_row(const Partition* pt, con
 // kernel
 // ------------------------------------------------------------------------------------------------
 
-template <int D, int NW, int NSTAGE>
+template <int D, int NW, int NSTAGE, bool SHORT_ROUNDS = false>
 struct Geo {
     static constexpr int NB = D / 16;                       // 16-wide blocks along d
     static constexpr int LW = 3 * NB / 4;                   // packed words per lane and code section
@@ -345,7 +345,7 @@ struct Geo {
     static constexpr int FP8_HALF = 16 * D;
     static constexpr int SLOT = (TQ3_REC + 127) / 128 * 128;
     // pages of one warp whose table entries are compacted at a time (fewer where the ring leaves little room)
-    static constexpr int ROUND = NW * NSTAGE * SLOT > 190000 ? 64 : 128;
+    static constexpr int ROUND = (NW * NSTAGE * SLOT > 190000 || SHORT_ROUNDS) ? 64 : 128;
     static constexpr int RING = NW * NSTAGE * SLOT;
     static constexpr int QROT = NB * 32 * 16;               // rotated query B fragments, hi and lo interleaved
     static constexpr int QPLAIN = NB * 32 * 8;              // plain query B fragments (FP8 pages)
@@ -398,6 +398,11 @@ struct WarpAcc {
     float o[NB][4];
     float l[2];
     float m[2];
+    // pages of several tiles only: while the tiles of one Stale page are scanned, o holds sum p * code of
+    // that page (the page's scale/zero are applied once, when the page is left), lp its row sums, and the
+    // output accumulated before sits in shared memory, to be multiplied by pk (the rescales since then)
+    float lp[2];
+    float pk[2];
 };
 
 // Scores of one page -> probabilities.  s[0..1] = token g, s[2..3] = token g+8 (heads 2tq, 2tq+1).
@@ -410,7 +415,7 @@ struct PFrag {
 };
 
 // First half: raise the running maximum (and rescale the accumulators) if the page asks for it.
-template <int NB>
+template <int NB, bool TILED = false>
 __device__ __forceinline__ void softmax_rescale(WarpAcc<NB>& acc, const float (&s)[4])
 {
     constexpr uint32_t FULL = 0xffffffffu;
@@ -433,6 +438,10 @@ __device__ __forceinline__ void softmax_rescale(WarpAcc<NB>& acc, const float (&
         }
         acc.l[0] *= f0;
         acc.l[1] *= f1;
+        if constexpr (TILED) {
+            acc.lp[0] *= f0; acc.lp[1] *= f1;
+            acc.pk[0] *= f0; acc.pk[1] *= f1;
+        }
     }
 }
 
@@ -520,11 +529,29 @@ __device__ __forceinline__ void tq3_key_quad(float (&S0)[4], float (&S1)[4], uin
 
 // Output update of the four channel blocks 4j..4j+3 of a Stale page: integer codes through the tensor
 // core, then the fp16 scale and zero of every channel applied to the 16x8 result in fp32.
+template <bool DEFER = false>
 __device__ __forceinline__ void tq3_value_quad(float (&o0)[4], float (&o1)[4], float (&o2)[4], float (&o3)[4],
                                                uint32_t W0, uint32_t W1, uint32_t W2, uint32_t meta_quad, const PFrag& pf)
 {
     float t[4];
     uint32_t a[4];
+    if constexpr (DEFER) {
+        // sum p * code only: the accumulators are in code units until the page is left
+        const uint32_t X1 = prmt(W0, W1, 0x6341u), X0 = prmt(W1, W2, 0x6341u), X2 = W2 >> 8;
+        a[0] = value_code<0>(W0); a[1] = value_code<3>(W0); a[2] = value_code<6>(W0); a[3] = value_code<1>(X1);
+        mma16816(o0, a, pf.b0, pf.b1);
+        mma16816(o0, a, pf.c0, pf.c1);
+        a[0] = value_code<4>(X1); a[1] = value_code<7>(X1); a[2] = value_code<2>(W1); a[3] = value_code<5>(W1);
+        mma16816(o1, a, pf.b0, pf.b1);
+        mma16816(o1, a, pf.c0, pf.c1);
+        a[0] = value_code<0>(X0); a[1] = value_code<3>(X0); a[2] = value_code<6>(X0); a[3] = value_code<1>(W2);
+        mma16816(o2, a, pf.b0, pf.b1);
+        mma16816(o2, a, pf.c0, pf.c1);
+        a[0] = value_code<4>(W2); a[1] = value_code<7>(W2); a[2] = value_code<2>(X2); a[3] = value_code<5>(X2);
+        mma16816(o3, a, pf.b0, pf.b1);
+        mma16816(o3, a, pf.c0, pf.c1);
+        return;
+    }
     {   // blocks 4j, 4j+1
         const uint4 mt = lds128(meta_quad);
         const uint32_t X1 = prmt(W0, W1, 0x6341u);
@@ -567,7 +594,7 @@ __device__ __forceinline__ void tq3_value_quad(float (&o0)[4], float (&o1)[4], f
 // probabilities pf) and the score phase of the next page (record rec_k) are issued quad by quad in
 // one instruction stream, so that table lookups, half-precision FMAs, fp32 FMAs and MMAs of the two
 // phases overlap.  DO_V / DO_K switch the halves off for the first and the last page.
-template <int D, bool DO_V, bool DO_K>
+template <int D, bool DO_V, bool DO_K, bool DEFER = false>
 __device__ __forceinline__ void tq3_step(WarpAcc<D / 16>& acc, uint32_t rec_v, const float (&s_cur)[4], PFrag& pf, uint32_t rec_k,
                                          uint32_t qt_lane, float sc2, int lane, float (&s_next)[4])
 {
@@ -578,13 +605,17 @@ __device__ __forceinline__ void tq3_step(WarpAcc<D / 16>& acc, uint32_t rec_v, c
     if constexpr (DO_K) load_lane_words<D>(rec_k, lane, kw);
     if constexpr (DO_V) load_lane_words<D>(rec_v + 6 * D, lane, vw);
     if constexpr (DO_V) softmax_probs<NB>(acc, s_cur, pf);     // in one block with the key unpack of the next page
+    if constexpr (DO_V && DEFER) {
+        acc.lp[0] += pf.ps0;
+        acc.lp[1] += pf.ps1;
+    }
     const uint32_t meta = rec_v + 12 * D + 32 + g * 16;
 #pragma unroll
     for (int j = 0; j < NB / 4; ++j) {
         if constexpr (DO_K) tq3_key_quad(S0, S1, kw[3 * j], kw[3 * j + 1], kw[3 * j + 2], qt_lane + j * 2048);
         if constexpr (DO_V)
-            tq3_value_quad(acc.o[4 * j], acc.o[4 * j + 1], acc.o[4 * j + 2], acc.o[4 * j + 3], vw[3 * j], vw[3 * j + 1],
-                           vw[3 * j + 2], meta + j * 256, pf);
+            tq3_value_quad<DEFER>(acc.o[4 * j], acc.o[4 * j + 1], acc.o[4 * j + 2], acc.o[4 * j + 3], vw[3 * j], vw[3 * j + 1],
+                                  vw[3 * j + 2], meta + j * 256, pf);
     }
     if constexpr (DO_K) {
         const uint32_t gaddr = rec_k + 12 * D;
@@ -784,7 +815,7 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
     unsigned long long tl_last = 0;
 #endif
     MKV_STAMP(0);
-    using G = Geo<D, NW, NSTAGE>;
+    using G = Geo<D, NW, NSTAGE, TILED>;     // pages of several tiles: short rounds leave room for the parked rows
     constexpr int NB = G::NB, NBH = NB, NU = NW;
     constexpr uint32_t FULL = 0xffffffffu;
     extern __shared__ __align__(128) uint8_t smem[];
@@ -843,7 +874,8 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
             const int len = P.lens[b], n = (len + kPage - 1) / kPage;
             int st = (int)((float)n * 0.6180339f);
             if (st < 1) st = 1;
-            for (; n > 1; ++st) {
+            if constexpr (TILED) st = 1;          // consecutive tiles: a warp's run stays inside one or two pages
+            for (; n > 1 && !TILED; ++st) {
                 int a = st, c = n;
                 while (c) { const int t = a % c; a = c; c = t; }
                 if (a == 1) break;
@@ -942,13 +974,13 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                     else
                         kind = (tag <= MKV_TAG_ANCHOR && id >= 0 && id < P.fp8_pages) ? 2 : 0;
                     if (kind == 0) atomicOr(P.status, kStBounds);     // never dereferenced
-                    if constexpr (TILED) id = id * P.tiles + (pg - entry * P.tiles);   // tile index inside the arena
+                    if constexpr (TILED) pg -= entry * P.tiles;   // from here on: the tile's index inside its page (kept in the second list)
                 }
                 const uint32_t m3 = __ballot_sync(FULL, kind == 1), m8 = __ballot_sync(FULL, kind == 2);
                 const uint32_t lt = (1u << lane) - 1u;
                 if (kind == 1) list3[n3 + __popc(m3 & lt)] = id;
                 if (kind == 2) list8[n8 + __popc(m8 & lt)] = id | ((valid & 15) << 27);
-                if constexpr (SCORED) {
+                if constexpr (SCORED || TILED) {     // logical page (scored output) or tile inside the page (pages of several tiles)
                     if (kind == 1) lpg3[n3 + __popc(m3 & lt)] = pg;
                     if (kind == 2) lpg8[n8 + __popc(m8 & lt)] = pg;
                 }
@@ -961,14 +993,14 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
             if (lane == 0) {
                 const uint32_t s = (uint32_t)i % NSTAGE;
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                mbar_expect_tx(bars + 8 * s, G::TQ3_REC);
                 if constexpr (!TILED) {
+                    mbar_expect_tx(bars + 8 * s, G::TQ3_REC);
                     bulk_load(ring + s * G::SLOT, tq3_base + (size_t)list3[i] * hkv * G::TQ3_REC, G::TQ3_REC, bars + 8 * s);
-                } else {   // the tile, then the page's scale/zero behind it: the slot then reads like a 16-token record
-                    const int page = list3[i] / P.tiles, m = list3[i] - page * P.tiles;
+                } else {   // the tile only: the page's scale/zero are applied once, when the scan leaves the page
+                    const int page = list3[i], m = lpg3[i];
                     const uint8_t* pbase = P.tq3 + ((size_t)page * hkv + h) * tq3_page;
+                    mbar_expect_tx(bars + 8 * s, TQ3_TILE);
                     bulk_load(ring + s * G::SLOT, pbase + (size_t)m * TQ3_TILE, TQ3_TILE, bars + 8 * s);
-                    bulk_load(ring + s * G::SLOT + TQ3_TILE, pbase + (size_t)P.tiles * TQ3_TILE, TQ3_META, bars + 8 * s);
                 }
             }
         };
@@ -980,8 +1012,7 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                 if constexpr (!TILED) {
                     rec = fp8_base + (size_t)e8 * hkv * (2 * G::FP8_HALF);
                 } else {
-                    const int page = e8 / P.tiles, m = e8 - page * P.tiles;
-                    rec = P.fp8 + (((size_t)page * hkv + h) * P.tiles + m) * (2 * G::FP8_HALF);
+                    rec = P.fp8 + (((size_t)e8 * hkv + h) * P.tiles + lpg8[i]) * (2 * G::FP8_HALF);
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 mbar_expect_tx(bars + 8 * s, G::FP8_HALF);
@@ -995,6 +1026,49 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
         int tl_n3 = 0, tl_n8 = 0;
 #endif
         WarpAcc<NB> acc;
+        // Pages of several tiles.  While the scan is inside a Stale page, acc.o holds sum p * code and the
+        // output gathered before waits in this warp's shared-memory rows ("parked"); leaving the page adds
+        // scale * acc.o + zero * acc.lp to it (fold).  The scale/zero halves come straight from the page's
+        // metadata in global memory, in the order of the 16-token record.
+        float* park = reinterpret_cast<float*>(smem + G::SMEM) + (size_t)warp * NB * 128;
+        auto park_store = [&]() {
+#pragma unroll
+            for (int i = 0; i < NB; ++i)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    park[(i * 4 + e) * 32 + lane] = acc.o[i][e];
+                    acc.o[i][e] = 0.f;
+                }
+            acc.pk[0] = acc.pk[1] = 1.f;
+            acc.lp[0] = acc.lp[1] = 0.f;
+        };
+        auto fold = [&](int page, bool to_regs) {
+            const uint4* meta = reinterpret_cast<const uint4*>(P.tq3 + ((size_t)page * hkv + h) * tq3_page +
+                                                                (size_t)P.tiles * TQ3_TILE + g * 16);
+#pragma unroll
+            for (int j = 0; j < NB / 4; ++j) {
+                const uint4 m01 = __ldg(meta + j * 16), m23 = __ldg(meta + j * 16 + 8);
+                const uint32_t scp[4] = {m01.x, m01.z, m23.x, m23.z}, zpp[4] = {m01.y, m01.w, m23.y, m23.w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int i = 4 * j + q;
+                    const float2 sc = half2_to_float2(scp[q]), zp = half2_to_float2(zpp[q]);
+                    float r[4];
+                    r[0] = fmaf(park[(i * 4 + 0) * 32 + lane], acc.pk[0], fmaf(sc.x, acc.o[i][0], zp.x * acc.lp[0]));
+                    r[1] = fmaf(park[(i * 4 + 1) * 32 + lane], acc.pk[1], fmaf(sc.x, acc.o[i][1], zp.x * acc.lp[1]));
+                    r[2] = fmaf(park[(i * 4 + 2) * 32 + lane], acc.pk[0], fmaf(sc.y, acc.o[i][2], zp.y * acc.lp[0]));
+                    r[3] = fmaf(park[(i * 4 + 3) * 32 + lane], acc.pk[1], fmaf(sc.y, acc.o[i][3], zp.y * acc.lp[1]));
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        if (to_regs) acc.o[i][e] = r[e];
+                        else { park[(i * 4 + e) * 32 + lane] = r[e]; acc.o[i][e] = 0.f; }
+                    }
+                }
+            }
+            acc.pk[0] = acc.pk[1] = 1.f;
+            acc.lp[0] = acc.lp[1] = 0.f;
+        };
+        (void)park_store; (void)fold;
 #pragma unroll
         for (int i = 0; i < NB; ++i) acc.o[i][0] = acc.o[i][1] = acc.o[i][2] = acc.o[i][3] = 0.f;
         acc.l[0] = acc.l[1] = 0.f;
@@ -1068,14 +1142,26 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
             if (n3 > 0) {
                 float s_cur[4], s_next[4];
                 PFrag pf;
+                int cur_page = 0;
+                if constexpr (TILED) {
+                    park_store();
+                    cur_page = list3[0];
+                }
                 wait_slot(0);
-                if (!failed) tq3_step<D, false, true>(acc, 0, s_cur, pf, ring, qt_lane, sc2, lane, s_cur);
+                if (!failed) tq3_step<D, false, true, TILED>(acc, 0, s_cur, pf, ring, qt_lane, sc2, lane, s_cur);
                 for (int i = 0; i + 1 < n3 && !failed; ++i) {
                     const uint32_t cur = (uint32_t)i % NSTAGE, nxt = (uint32_t)(i + 1) % NSTAGE;
                     wait_slot(nxt);
                     if (failed) break;
-                    softmax_rescale<NB>(acc, s_cur);
-                    tq3_step<D, true, true>(acc, ring + cur * G::SLOT, s_cur, pf, ring + nxt * G::SLOT, qt_lane, sc2, lane, s_next);
+                    softmax_rescale<NB, TILED>(acc, s_cur);
+                    if constexpr (TILED) {
+                        const int pg_i = list3[i];
+                        if (pg_i != cur_page) {
+                            fold(cur_page, false);
+                            cur_page = pg_i;
+                        }
+                    }
+                    tq3_step<D, true, true, TILED>(acc, ring + cur * G::SLOT, s_cur, pf, ring + nxt * G::SLOT, qt_lane, sc2, lane, s_next);
                     if constexpr (SCORED) store_page_mass<NB>(acc, pf, mass_row + lpg3[i], P.max_pages, GQ, lane);
 #pragma unroll
                     for (int e = 0; e < 4; ++e) s_cur[e] = s_next[e];
@@ -1083,9 +1169,17 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                     if (i + NSTAGE < n3) issue_tq3(i + NSTAGE);
                 }
                 if (!failed) {
-                    softmax_rescale<NB>(acc, s_cur);
-                    tq3_step<D, true, false>(acc, ring + ((uint32_t)(n3 - 1) % NSTAGE) * G::SLOT, s_cur, pf, 0, qt_lane, sc2, lane, s_next);
+                    softmax_rescale<NB, TILED>(acc, s_cur);
+                    if constexpr (TILED) {
+                        const int pg_i = list3[n3 - 1];
+                        if (pg_i != cur_page) {
+                            fold(cur_page, false);
+                            cur_page = pg_i;
+                        }
+                    }
+                    tq3_step<D, true, false, TILED>(acc, ring + ((uint32_t)(n3 - 1) % NSTAGE) * G::SLOT, s_cur, pf, 0, qt_lane, sc2, lane, s_next);
                     if constexpr (SCORED) store_page_mass<NB>(acc, pf, mass_row + lpg3[n3 - 1], P.max_pages, GQ, lane);
+                    if constexpr (TILED) fold(cur_page, true);        // back to output units for the FP8 pages and the reduction
                 }
                 __syncwarp();
             }
@@ -1241,20 +1335,23 @@ static int32_t run_tmem(mkv_pool* p, DecodeParams& prm, cudaStream_t s)
 template <int D, int NW, int NSTAGE, int MINB, bool SCORED = false, bool TILED = false>
 static int32_t run_tensor(mkv_pool* p, DecodeParams& prm, cudaStream_t s)
 {
-    using G = Geo<D, NW, NSTAGE>;
+    using G = Geo<D, NW, NSTAGE, TILED>;
     auto kern = decode_tensor_kernel<D, NW, NSTAGE, MINB, SCORED, TILED>;
+    // pages of several tiles: one row of parked accumulators (8 D floats) per warp behind the usual layout
+    constexpr int SMEM = G::SMEM + (TILED ? NW * 8 * D * 4 : 0);
+    static_assert(SMEM <= 232448, "dynamic shared memory of one block");
     static int grid_cache[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     int dev = p->device & 7;
     if (grid_cache[dev] == 0) {
-        MKV_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM));
+        MKV_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM));
         int per_sm = 0;
-        MKV_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, NW * 32, G::SMEM));
+        MKV_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, NW * 32, SMEM));
         if (per_sm < 1) return MKV_E_INVALID;
         int grid = p->dev.sm_count * per_sm;
         grid_cache[dev] = grid > kMaxCtas ? kMaxCtas : grid;
     }
     if (grid_cache[dev] > prm.max_blocks) return MKV_E_INVALID;
-    kern<<<grid_cache[dev], NW * 32, G::SMEM, s>>>(prm);
+    kern<<<grid_cache[dev], NW * 32, SMEM, s>>>(prm);
     MKV_CUDA(cudaGetLastError());
     return MKV_OK;
 }
@@ -1406,9 +1503,8 @@ int32_t launch_decode_tensor_at(mkv_pool* p, const void* q, const int32_t* bt, c
         }
     }
     switch (shape) {
-    case 1: return run_tensor<256, 8, 6, 1>(p, prm, s);
     case 2: return run_tensor<256, 10, 4, 1>(p, prm, s);
-    default: return run_tensor<256, 8, 4, 1>(p, prm, s);
+    default: return run_tensor<256, 8, 4, 1>(p, prm, s);     // a ring of 6 slots per warp no longer fits beside the page lists
     }
 }
 
