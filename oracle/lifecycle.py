@@ -30,7 +30,8 @@ class LifecycleError(Exception):
 
 
 class PoolModel:
-    def __init__(self, fp8_pages: int, tq3_pages: int):
+    def __init__(self, fp8_pages: int, tq3_pages: int, page_tokens: int = T):
+        self.T = page_tokens               # tokens per page (16, or 16 M for the paper-scale blocks)
         self.capacity = {FMT_FP8: fp8_pages, FMT_TQ3: tq3_pages}
         self.free = {FMT_FP8: list(range(fp8_pages - 1, -1, -1)),
                      FMT_TQ3: list(range(tq3_pages - 1, -1, -1))}
@@ -71,7 +72,7 @@ class PoolModel:
         is mapped twice, or both mapped and free."""
         seen = set()
         for s in self.seqs.values():
-            assert len(s.pages) == (s.len + T - 1) // T
+            assert len(s.pages) == (s.len + self.T - 1) // self.T
             for tag, pid in s.pages:
                 fmt = FMT_TQ3 if tag == STALE else FMT_FP8
                 assert 0 <= pid < self.capacity[fmt]
@@ -94,17 +95,17 @@ class SeqModel:
     # Append(q, p): allocate a request-owned Recent page when the previous one is full, write KV,
     # then publish the mapping.  Returns (physical id, slot, opened_new_page).
     def append(self):
-        opened = self.len % T == 0
+        opened = self.len % self.pool.T == 0
         if opened:
             pid = self.pool.alloc(FMT_FP8, self.handle)
             self.pages.append((RECENT, pid))
         tag, pid = self.pages[-1]
-        slot = self.len % T
+        slot = self.len % self.pool.T
         self.len += 1
         return pid, slot, opened
 
     def _full(self, lp: int) -> bool:
-        return (lp + 1) * T <= self.len
+        return (lp + 1) * self.pool.T <= self.len
 
     def protect(self, lp: int):
         tag, pid = self._get(lp)
@@ -144,7 +145,7 @@ class SeqModel:
     def age(self, recent_tokens: int):
         """Demote every full Recent page that lies wholly before the last `recent_tokens` tokens."""
         moved = []
-        first_recent = max(0, self.len - recent_tokens) // T
+        first_recent = max(0, self.len - recent_tokens) // self.pool.T
         for lp in range(min(first_recent, len(self.pages))):
             if self.pages[lp][0] == RECENT and self._full(lp):
                 moved.append((lp,) + self.demote(lp))

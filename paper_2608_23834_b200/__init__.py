@@ -319,9 +319,10 @@ def decode_attention_static(pool: "Pool", q, block_table, tier_tag, seq_lens, sc
 class HostPool:
     """Bookkeeping-only pool (no device): free lists, sequence rows, statistics."""
 
-    def __init__(self, head_dim, n_kv_heads, n_q_heads, fp8_pages, tq3_pages):
+    def __init__(self, head_dim, n_kv_heads, n_q_heads, fp8_pages, tq3_pages, page_tokens=16):
         self.d, self.hkv, self.hq = head_dim, n_kv_heads, n_q_heads
-        self.cfg = make_config(head_dim, n_kv_heads, n_q_heads, fp8_pages, tq3_pages, np.ones(head_dim, np.int8))
+        self.cfg = make_config(head_dim, n_kv_heads, n_q_heads, fp8_pages, tq3_pages, np.ones(head_dim, np.int8),
+                               page_tokens=page_tokens)
         h = C.c_void_p()
         _check(lib().mkv_pool_create_host_only(C.byref(self.cfg), C.byref(h)), "mkv_pool_create_host_only")
         self.handle = h

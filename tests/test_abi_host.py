@@ -88,12 +88,14 @@ def test_free_lists_hand_out_ids_in_order_and_reject_misuse():
 CODES = {"MKV_E_OOM_FP8": M.E_OOM_FP8, "MKV_E_OOM_TQ3": M.E_OOM_TQ3, "MKV_E_STATE": M.E_STATE, "MKV_E_BOUNDS": M.E_BOUNDS}
 
 
-def test_sequence_bookkeeping_agrees_with_the_lifecycle_model_on_a_random_walk():
+@pytest.mark.parametrize("page_tokens", [16, 48])
+def test_sequence_bookkeeping_agrees_with_the_lifecycle_model_on_a_random_walk(page_tokens):
     """Same transitions on the library's mkv_seq_* and on the oracle's model of Algorithm 1: same
-    rows (tags and physical ids), same failures, same pool occupancy, after every step."""
-    rnd = random.Random(1)
-    hp = M.HostPool(128, 2, 8, 24, 24)
-    model = PoolModel(24, 24)
+    rows (tags and physical ids), same failures, same pool occupancy, after every step (pages of 16
+    tokens, and pages of three 16-token tiles)."""
+    rnd = random.Random(page_tokens)
+    hp = M.HostPool(128, 2, 8, 24, 24, page_tokens=page_tokens)
+    model = PoolModel(24, 24, page_tokens)
     seqs = []          # (library Seq, model SeqModel)
     for step in range(3000):
         r = rnd.random()
@@ -113,7 +115,7 @@ def test_sequence_bookkeeping_agrees_with_the_lifecycle_model_on_a_random_walk()
         elif r < 0.90:
             op = ("protect", lp, rnd.random() < 0.7)
         elif r < 0.96:
-            op = ("age", rnd.choice([16, 40, 100]))
+            op = ("age", rnd.choice([16, 40, 100]) * page_tokens // 16)
         else:
             op = ("finish",)
         got = want = None
