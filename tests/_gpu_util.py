@@ -16,10 +16,12 @@ def bf16_tensor(bits: np.ndarray, device="cuda:0") -> torch.Tensor:
 
 
 class Case:
-    def __init__(self, spec, layer=0, extra_fp8=0, extra_tq3=0, k_scale=1.0, v_scale=1.0):
+    def __init__(self, spec, layer=0, extra_fp8=0, extra_tq3=0, k_scale=1.0, v_scale=1.0, requests=None):
+        """requests: encode only these requests' pages (the others stay zero-filled records: valid input,
+        compared nowhere) to keep the oracle's share of a full-size case short."""
         self.spec = spec
         self.tab = W.tables(spec, extra_fp8, extra_tq3)
-        self.L = build_layer(spec, self.tab, layer)
+        self.L = build_layer(spec, self.tab, layer, requests=requests)
         self.pool = M.Pool(spec.head_dim, spec.n_kv_heads, spec.n_q_heads, max(self.tab.fp8_pages, 1),
                            max(self.tab.tq3_pages, 1), self.L.sigma, k_scale, v_scale, max_batch=spec.batch,
                            page_tokens=spec.page_tokens)

@@ -120,3 +120,19 @@ def test_canary_shape_with_1792_token_pages_full_size():
     assert np.isfinite(out).all() and out.any()
     # physical bytes of the layer: 20 FP8 + 46 TQ3 pages of 4 heads
     assert case.pool.fp8_rec * 4 * 20 + case.pool.tq3_rec * 4 * 46 == 4 * (20 * 917_504 + 46 * 348_672)
+
+
+def test_runs_longer_than_a_round_park_and_fold_across_rounds():
+    """8 x 32,256 tokens, d = 128, 8 KV heads, pages of 1,792 tokens, half of them Stale: every warp scans more than
+    64 tiles, so its page lists are rebuilt and the parked accumulators carried from round to round."""
+    spec = W.config(4, batch=8, ctx=18 * 1792, stale_fraction=0.5, page_tokens=1792)
+    case = Case(spec, requests=[3])
+    n_units = sum((n + 15) // 16 for n in spec.seq_lens) * spec.n_kv_heads
+    assert n_units / (148 * 12) > 64
+    out, lse = case.run()
+    ref, ref_lse = case.reference(only_b=3, only_h=5)
+    g = spec.group
+    for hq in range(5 * g, 6 * g):
+        check_close(out[3, hq], ref[3, hq], f"b=3 hq={hq}")
+        assert abs(lse[3, hq] - ref_lse[3, hq]) < 2e-3
+    assert np.isfinite(out).all()
