@@ -15,10 +15,13 @@ from _gpu_util import Case, MAX_ABS, REL_L2, bf16_tensor
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("cfg", ["d256", "d128"])
+@pytest.mark.parametrize("cfg", ["d256", "d128", "d256_pages_of_832"])
 def test_static_scratch_entry_matches_the_workspace_entry_twice_in_a_row(cfg):
     if cfg == "d256":
         spec = W.config(2, seq_lens=(9008, 7600), recent_tokens=512, n_layers=1)
+    elif cfg == "d256_pages_of_832":
+        spec = W.config(2, seq_lens=(9 * 832 + 100, 7 * 832), anchor_prefix=832, recent_tokens=900, n_layers=1,
+                        page_tokens=832)
     else:
         spec = W.config(1, seq_lens=(3000, 1500, 4100, 16), recent_tokens=256, anchor_span_tokens=64)
     case = Case(spec, extra_fp8=3, extra_tq3=3)
@@ -42,7 +45,7 @@ def test_static_scratch_entry_matches_the_workspace_entry_twice_in_a_row(cfg):
     s = spec
     ref64, _ = oracle.decode_attention(case.L.fp8_arena, case.L.tq3_arena, s.head_dim, s.n_kv_heads, s.group, case.L.sigma,
                                        W.query(spec, layer=1), case.tab.block_table, case.tab.tier_tag, case.tab.seq_lens,
-                                       s.scale)
+                                       s.scale, page_tokens=s.page_tokens)
     assert np.abs(got - ref64).max() <= MAX_ABS and np.linalg.norm(got - ref64) / np.linalg.norm(ref64) <= REL_L2
 
 
