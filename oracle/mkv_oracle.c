@@ -20,13 +20,15 @@
  * The paper fixes the structure of TQ3 but not its constants; the readings used here (rotation =
  * randomised Walsh-Hadamard, Lloyd-Max N(0,1) codebook rounded to fp16, norm correction
  * g = |x|/|c|, per-channel asymmetric 3-bit values, fp32 encoder with a fixed operation order)
- * are listed in the design doc.  Parity status per function:
+ * are stated where they are used below.  Parity status per function:
  *   pinned by the paper / mathematics / a library: e4m3 codec, fp16 conversion, byte accounting,
  *     codebook values (Lloyd-Max), key round trip and norm preservation, value round-trip
  *     bounds, attention (dense special case, brute force, partition invariance, indexing).
- *   parity unpinned (fixed only by the readings in the design doc): choice of rotation, definition of
+ *   pinned by the paper's byte counters (Section 6.3): the sizes of pages of 16 M tokens, i.e. one
+ *     value scale/zero pair per channel and PAGE.
+ *   parity unpinned (fixed only by the readings made here): choice of rotation, definition of
  *     the norm correction, value quantiser being un-rotated, tie-breaking, FP8 scale handling,
- *     bit positions of the packed records.
+ *     bit positions of the packed records, order of tiles and metadata inside a page of 16 M tokens.
  *
  * Floating point: the encoder works in fp32, one IEEE round-to-nearest operation at a time
  * (compile with -ffp-contract=off, no fast-math).  Dequantisation and attention work in fp64.
@@ -36,7 +38,7 @@
 #include <stdlib.h>
 #include <string.h>
 
-#define ORC_T 16 /* tokens per page (all BASELINE configs) */
+#define ORC_T 16 /* tokens per page, and per tile of a page of 16 M tokens */
 #define ORC_MAXD 256
 
 /* ------------------------------------------------------------------------------------------
