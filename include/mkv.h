@@ -41,9 +41,10 @@
  *       channel over all 16 M tokens) follow the tiles.  M = 1 is the 16-token record.  At M = 112,
  *       d = 256 this is 348,672 bytes per page and head: the 3.04 bit/scalar of Section 5.4.
  *     Block-table rows have one entry per page; slot_mapping = page * page_size + position.  With M > 1
- *     mkv_decode_attention() runs the tensor-core kernel (MKV_DECODE_SCALAR / _TMEM, the scored call and
- *     the no-allocation entry point with a scored output are refused with MKV_E_INVALID); mkv_demote()
- *     and mkv_promote() take three resp. two launches (page scale/zero, tiles, publication).
+ *     mkv_decode_attention() and mkv_decode_attention_scored() run the tensor-core kernel
+ *     (MKV_DECODE_SCALAR / _TMEM are refused with MKV_E_INVALID); the page mass is per page of 16 M
+ *     tokens; mkv_demote() and mkv_promote() take three resp. two launches (page scale/zero, tiles,
+ *     publication).
  */
 #ifndef MKV_H_
 #define MKV_H_
@@ -262,6 +263,12 @@ int32_t mkv_decode_attention_scored(mkv_pool* pool, const void* q_dev, const int
 int32_t mkv_page_score_update(const float* page_mass_dev, const int32_t* seq_lens_dev, int32_t B,
                               int32_t n_q_heads, int32_t max_pages, uint64_t head_mask, float beta,
                               float* score_dev, void* stream);
+
+/* The same for pools whose pages hold page_size tokens (a multiple of 16): a request of len tokens has
+ * ceil(len / page_size) pages.  mkv_page_score_update() is this call with page_size = 16. */
+int32_t mkv_page_score_update_paged(const float* page_mass_dev, const int32_t* seq_lens_dev, int32_t B,
+                                    int32_t n_q_heads, int32_t max_pages, int32_t page_size, uint64_t head_mask,
+                                    float beta, float* score_dev, void* stream);
 
 /* ---- host-side sequence bookkeeping (Algorithm 1; no device work) ------------------------- */
 

@@ -91,6 +91,11 @@ def lib():
                                     i8p, u16p, i32p, u8p, i32p, C.c_int, C.c_int, C.c_double, f64p]
         L.orc_page_score_update.restype = None
         L.orc_page_score_update.argtypes = [f64p, i32p, C.c_int, C.c_int, C.c_int, C.c_uint64, C.c_double, f64p]
+        L.orc_page_score_update_blocks.restype = None
+        L.orc_page_score_update_blocks.argtypes = [f64p, i32p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_uint64, C.c_double, f64p]
+        L.orc_page_mass_blocks.restype = C.c_int
+        L.orc_page_mass_blocks.argtypes = [u8p, C.c_int64, u8p, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_float,
+                                           C.c_float, i8p, u16p, i32p, u8p, i32p, C.c_int, C.c_int, C.c_double, f64p]
         L.orc_encode_request.restype = C.c_int
         L.orc_encode_request.argtypes = [C.c_int, C.c_int, C.c_int, u16p, u16p, i32p, u8p, i8p,
                                          C.c_float, C.c_float, u8p, u8p]
@@ -464,7 +469,7 @@ def decode_attention(fp8_arena, tq3_arena, d, hkv, group, sigma, q_bits, block_t
 
 
 def page_mass(fp8_arena, tq3_arena, d, hkv, group, sigma, q_bits, block_table, tier_tag, seq_lens, scale,
-              k_scale=1.0, v_scale=1.0):
+              k_scale=1.0, v_scale=1.0, page_tokens=T):
     """Globally normalised attention mass of every page, q~ [B][Hq][max_pages] in fp64 (Eq. score-partial,
     Eq. score-global-weight with the two format partitions).  Arguments as decode_attention."""
     fp8_arena = _c(fp8_arena, np.uint8)
@@ -477,13 +482,14 @@ def page_mass(fp8_arena, tq3_arena, d, hkv, group, sigma, q_bits, block_table, t
     B, max_pages = block_table.shape
     Hq = hkv * group
     assert q_bits.shape == (B, Hq, d)
-    fp8_pages = fp8_arena.size // (hkv * fp8_record_bytes(d)) if fp8_arena.size else 0
-    tq3_pages = tq3_arena.size // (hkv * tq3_record_bytes(d)) if tq3_arena.size else 0
+    M = page_tokens // T
+    fp8_pages = fp8_arena.size // (hkv * fp8_block_bytes(d, M)) if fp8_arena.size else 0
+    tq3_pages = tq3_arena.size // (hkv * tq3_block_bytes(d, M)) if tq3_arena.size else 0
     mass = np.zeros((B, Hq, max_pages), np.float64)
     dummy = np.zeros(16, np.uint8)
-    rc = lib().orc_page_mass(
+    rc = lib().orc_page_mass_blocks(
         _p(fp8_arena if fp8_arena.size else dummy, C.c_uint8), fp8_pages,
-        _p(tq3_arena if tq3_arena.size else dummy, C.c_uint8), tq3_pages, d, hkv, group,
+        _p(tq3_arena if tq3_arena.size else dummy, C.c_uint8), tq3_pages, d, hkv, group, M,
         k_scale, v_scale, _p(sigma, C.c_int8), _p(q_bits, C.c_uint16), _p(block_table, C.c_int32),
         _p(tier_tag, C.c_uint8), _p(seq_lens, C.c_int32), B, max_pages, float(scale), _p(mass, C.c_double))
     if rc != 0:
@@ -491,15 +497,15 @@ def page_mass(fp8_arena, tq3_arena, d, hkv, group, sigma, q_bits, block_table, t
     return mass
 
 
-def page_score_update(mass, seq_lens, head_mask, beta, score):
+def page_score_update(mass, seq_lens, head_mask, beta, score, page_tokens=T):
     """Eq. (attention-score): returns beta * score + (1 - beta) * mean_{h in head set} mass[:, h, :] for the
     pages below each request's length (other entries unchanged).  score: [B][max_pages] fp64."""
     mass = _c(mass, np.float64)
     seq_lens = _c(seq_lens, np.int32)
     out = np.array(score, np.float64, copy=True, order="C")
     B, Hq, max_pages = mass.shape
-    lib().orc_page_score_update(_p(mass, C.c_double), _p(seq_lens, C.c_int32), B, Hq, max_pages,
-                                C.c_uint64(int(head_mask)), float(beta), _p(out, C.c_double))
+    lib().orc_page_score_update_blocks(_p(mass, C.c_double), _p(seq_lens, C.c_int32), B, Hq, max_pages, int(page_tokens),
+                                       C.c_uint64(int(head_mask)), float(beta), _p(out, C.c_double))
     return out
 
 

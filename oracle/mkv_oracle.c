@@ -756,22 +756,23 @@ int orc_decode_attention(const uint8_t* fp8_arena, int64_t fp8_pages, const uint
  *      q_p = w_j rho_p,   q~_p = q_p / sum_p' q_p'   (no sink state here: every page is addressable).
  * mass[b][hq][p] receives q~ (0 for pages beyond the request's length).
  * Returns 0, or -1 if a table entry is invalid. */
-int orc_page_mass(const uint8_t* fp8_arena, int64_t fp8_pages, const uint8_t* tq3_arena, int64_t tq3_pages,
-                  int d, int hkv, int group, float k_scale, float v_scale, const int8_t* sigma,
-                  const uint16_t* q, const int32_t* block_table, const uint8_t* tier_tag,
-                  const int32_t* seq_lens, int B, int max_pages, double scale, double* mass)
+int orc_page_mass_blocks(const uint8_t* fp8_arena, int64_t fp8_pages, const uint8_t* tq3_arena, int64_t tq3_pages,
+                         int d, int hkv, int group, int M, float k_scale, float v_scale, const int8_t* sigma,
+                         const uint16_t* q, const int32_t* block_table, const uint8_t* tier_tag,
+                         const int32_t* seq_lens, int B, int max_pages, double scale, double* mass)
 {
     orc_pool pool;
-    int Hq = hkv * group, unit, rc = 0;
+    int Hq = hkv * group, unit, rc = 0, T = ORC_T * M;      /* pages of T = 16 M tokens */
     pool.fp8_arena = fp8_arena; pool.tq3_arena = tq3_arena;
     pool.fp8_pages = fp8_pages; pool.tq3_pages = tq3_pages;
-    pool.d = d; pool.hkv = hkv; pool.group = group; pool.M = 1;
+    pool.d = d; pool.hkv = hkv; pool.group = group; pool.M = M;
     pool.k_scale = k_scale; pool.v_scale = v_scale; pool.sigma = sigma;
+    if (M < 1) return -1;
 
 #pragma omp parallel for schedule(dynamic, 1)
     for (unit = 0; unit < B * hkv; ++unit) {
         int b = unit / hkv, h = unit % hkv, len = seq_lens[b], gq, c, i, pg, j;
-        int n_pages = len > 0 ? (len + ORC_T - 1) / ORC_T : 0;
+        int n_pages = len > 0 ? (len + T - 1) / T : 0;
         const int32_t* row = block_table + (int64_t)b * max_pages;
         const uint8_t* tags = tier_tag + (int64_t)b * max_pages;
         double *K, *V, *s;
@@ -796,18 +797,18 @@ int orc_page_mass(const uint8_t* fp8_arena, int64_t fp8_pages, const uint8_t* tq
                 for (c = 0; c < d; ++c)
                     acc += (double)orc_bf16_to_f32(q[((int64_t)b * Hq + hq) * d + c]) * K[(int64_t)i * d + c];
                 s[i] = scale * acc;
-                j = tags[i / ORC_T] == 2;
+                j = tags[i / T] == 2;
                 if (s[i] > mj[j]) mj[j] = s[i];
             }
             for (i = 0; i < len; ++i) {
-                j = tags[i / ORC_T] == 2;
+                j = tags[i / T] == 2;
                 lj[j] += exp(s[i] - mj[j]);
             }
             m = mj[0] > mj[1] ? mj[0] : mj[1];
             l = 0.0;
             for (j = 0; j < 2; ++j) if (lj[j] > 0.0) l += exp(mj[j] - m) * lj[j];
             for (pg = 0; pg < n_pages; ++pg) {
-                int lo = pg * ORC_T, hi = lo + ORC_T < len ? lo + ORC_T : len;
+                int lo = pg * T, hi = lo + T < len ? lo + T : len;
                 double rho = 0.0, w;
                 j = tags[pg] == 2;
                 for (i = lo; i < hi; ++i) rho += exp(s[i] - mj[j]);
@@ -823,16 +824,25 @@ int orc_page_mass(const uint8_t* fp8_arena, int64_t fp8_pages, const uint8_t* tq
     return rc;
 }
 
+int orc_page_mass(const uint8_t* fp8_arena, int64_t fp8_pages, const uint8_t* tq3_arena, int64_t tq3_pages,
+                  int d, int hkv, int group, float k_scale, float v_scale, const int8_t* sigma,
+                  const uint16_t* q, const int32_t* block_table, const uint8_t* tier_tag,
+                  const int32_t* seq_lens, int B, int max_pages, double scale, double* mass)
+{
+    return orc_page_mass_blocks(fp8_arena, fp8_pages, tq3_arena, tq3_pages, d, hkv, group, 1, k_scale, v_scale, sigma, q,
+                                block_table, tier_tag, seq_lens, B, max_pages, scale, mass);
+}
+
 /* Eq. (attention-score): r_p = mean over the sampled head set of q~_{h,p}; a_p <- beta a_p + (1 - beta) r_p.
  * head_mask bit hq selects query head hq (at least one bit set among the first Hq).  mass is
  * [B][Hq][max_pages], score is [B][max_pages] and is updated in place for pages below the length. */
-void orc_page_score_update(const double* mass, const int32_t* seq_lens, int B, int Hq, int max_pages,
-                           uint64_t head_mask, double beta, double* score)
+void orc_page_score_update_blocks(const double* mass, const int32_t* seq_lens, int B, int Hq, int max_pages,
+                                  int page_tokens, uint64_t head_mask, double beta, double* score)
 {
     int b, pg, hq, n_heads = 0;
     for (hq = 0; hq < Hq; ++hq) if ((head_mask >> hq) & 1u) ++n_heads;
     for (b = 0; b < B; ++b) {
-        int n_pages = seq_lens[b] > 0 ? (seq_lens[b] + ORC_T - 1) / ORC_T : 0;
+        int n_pages = seq_lens[b] > 0 ? (seq_lens[b] + page_tokens - 1) / page_tokens : 0;
         for (pg = 0; pg < n_pages; ++pg) {
             double r = 0.0;
             for (hq = 0; hq < Hq; ++hq)
@@ -841,6 +851,12 @@ void orc_page_score_update(const double* mass, const int32_t* seq_lens, int B, i
             score[(int64_t)b * max_pages + pg] = beta * score[(int64_t)b * max_pages + pg] + (1.0 - beta) * r;
         }
     }
+}
+
+void orc_page_score_update(const double* mass, const int32_t* seq_lens, int B, int Hq, int max_pages,
+                           uint64_t head_mask, double beta, double* score)
+{
+    orc_page_score_update_blocks(mass, seq_lens, B, Hq, max_pages, ORC_T, head_mask, beta, score);
 }
 
 /* ------------------------------------------------------------------------------------------

@@ -33,7 +33,7 @@ EXPORTS = [
     "mkv_set_anchor", "mkv_decode_attention", "mkv_seq_create", "mkv_seq_finish", "mkv_seq_append",
     "mkv_seq_protect", "mkv_seq_demote", "mkv_seq_age", "mkv_seq_len", "mkv_seq_row",
     "mkv_decode_attention_static", "mkv_promote", "mkv_seq_promote",
-    "mkv_decode_attention_scored", "mkv_page_score_update",
+    "mkv_decode_attention_scored", "mkv_page_score_update", "mkv_page_score_update_paged",
 ]
 
 
@@ -92,6 +92,8 @@ def lib():
             "mkv_decode_attention_scored": [vp, vp, vp, vp, vp, C.c_int32, C.c_int32, C.c_float, f32p, f32p, f32p, vp,
                                             C.c_size_t, vp],
             "mkv_page_score_update": [f32p, vp, C.c_int32, C.c_int32, C.c_int32, C.c_uint64, C.c_float, f32p, vp],
+            "mkv_page_score_update_paged": [f32p, vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_uint64, C.c_float,
+                                            f32p, vp],
             "mkv_seq_create": [vp, C.POINTER(vp)],
             "mkv_seq_finish": [vp],
             "mkv_seq_append": [vp, i32p, i32p, i32p],
@@ -288,15 +290,20 @@ class Pool:
         return out, lse, page_mass
 
 
-def page_score_update(page_mass, seq_lens, head_mask, beta, score, stream=None):
-    """mkv_page_score_update (Eq. attention-score): score <- beta * score + (1 - beta) * mean over the heads in
-    head_mask of page_mass, in place, for the pages below each request's length."""
+def page_score_update(page_mass, seq_lens, head_mask, beta, score, stream=None, page_tokens=16):
+    """mkv_page_score_update[_paged] (Eq. attention-score): score <- beta * score + (1 - beta) * mean over the
+    heads in head_mask of page_mass, in place, for the pages below each request's length."""
     B, hq, max_pages = page_mass.shape
     assert page_mass.dtype == torch.float32 and page_mass.is_contiguous()
     assert score.dtype == torch.float32 and score.is_contiguous() and score.shape == (B, max_pages)
     assert seq_lens.dtype == torch.int32 and seq_lens.numel() == B
-    _check(lib().mkv_page_score_update(_ptr(page_mass), _ptr(seq_lens), B, hq, max_pages, C.c_uint64(int(head_mask)),
-                                       float(beta), _ptr(score), _stream(stream)), "mkv_page_score_update")
+    if page_tokens == 16:
+        _check(lib().mkv_page_score_update(_ptr(page_mass), _ptr(seq_lens), B, hq, max_pages, C.c_uint64(int(head_mask)),
+                                           float(beta), _ptr(score), _stream(stream)), "mkv_page_score_update")
+    else:
+        _check(lib().mkv_page_score_update_paged(_ptr(page_mass), _ptr(seq_lens), B, hq, max_pages, int(page_tokens),
+                                                 C.c_uint64(int(head_mask)), float(beta), _ptr(score), _stream(stream)),
+               "mkv_page_score_update_paged")
     return score
 
 

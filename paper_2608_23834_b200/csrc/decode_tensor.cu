@@ -479,14 +479,36 @@ __device__ __forceinline__ void softmax_page(WarpAcc<NB>& acc, const float (&s)[
 // (row sum relative to the running maximum, plus that maximum), for the two heads this lane owns.
 // mass_pg points at (request, first head of the group, this page); heads are mass_stride apart.
 // The finishing kernel turns it into the globally normalised mass with the row's log-sum-exp.
-template <int NB>
-__device__ __forceinline__ void store_page_mass(const WarpAcc<NB>& acc, const PFrag& pf, float* mass_pg, int mass_stride,
+// *addr <- log2(2^*addr + 2^v): several warps add their parts of one page's exponential sum (pages of several
+// tiles); the entries start at -inf.
+__device__ __forceinline__ void atomic_log2_add(float* addr, float v)
+{
+    int* ia = reinterpret_cast<int*>(addr);
+    int old = *reinterpret_cast<volatile int*>(ia), assumed;
+    do {
+        assumed = old;
+        const float a = __int_as_float(assumed);
+        const float hi = fmaxf(a, v), lo = fminf(a, v);
+        const float nv = lo == -CUDART_INF_F ? hi : hi + __log2f(1.f + fast_exp2(lo - hi));
+        old = atomicCAS(ia, assumed, __float_as_int(nv));
+    } while (old != assumed);
+}
+
+// ACCUMULATE: the entry receives a part of the page (a tile, or a run of tiles) and is added to, not stored.
+template <int NB, bool ACCUMULATE = false>
+__device__ __forceinline__ void store_page_mass(const WarpAcc<NB>& acc, float ps0, float ps1, float* mass_pg, int mass_stride,
                                                 int GQ, int lane)
 {
     if (lane < 4) {                  // g == 0: one lane per head pair
         const int h0 = 2 * lane;
-        if (h0 < GQ) mass_pg[(size_t)h0 * mass_stride] = __log2f(pf.ps0) + acc.m[0];
-        if (h0 + 1 < GQ) mass_pg[(size_t)(h0 + 1) * mass_stride] = __log2f(pf.ps1) + acc.m[1];
+        const float v0 = __log2f(ps0) + acc.m[0], v1 = __log2f(ps1) + acc.m[1];
+        if constexpr (ACCUMULATE) {
+            if (h0 < GQ) atomic_log2_add(mass_pg + (size_t)h0 * mass_stride, v0);
+            if (h0 + 1 < GQ) atomic_log2_add(mass_pg + (size_t)(h0 + 1) * mass_stride, v1);
+        } else {
+            if (h0 < GQ) mass_pg[(size_t)h0 * mass_stride] = v0;
+            if (h0 + 1 < GQ) mass_pg[(size_t)(h0 + 1) * mass_stride] = v1;
+        }
     }
 }
 
@@ -642,7 +664,7 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_
 // fragments can be fetched with ldmatrix: a lane then holds the four consecutive tokens 4tq .. 4tq+3 of
 // its two channel rows, which is the order P^T has after the transposition of a score tile whose rows
 // are permuted this way.
-template <int D, bool SCORED>
+template <int D, bool SCORED, bool ACCUMULATE = false>
 __device__ __forceinline__ void fp8_page(WarpAcc<D / 16>& acc, uint32_t kaddr, uint32_t vaddr, uint32_t qf_lane,
                                          float score_scale, float v_scale, int valid, int lane, float* mass_pg,
                                          int mass_stride, int GQ)
@@ -680,7 +702,7 @@ __device__ __forceinline__ void fp8_page(WarpAcc<D / 16>& acc, uint32_t kaddr, u
     }
     PFrag pf;
     softmax_page<NB>(acc, s, pf);
-    if constexpr (SCORED) store_page_mass<NB>(acc, pf, mass_pg, mass_stride, GQ, lane);
+    if constexpr (SCORED) store_page_mass<NB, ACCUMULATE>(acc, pf.ps0, pf.ps1, mass_pg, mass_stride, GQ, lane);
     const bool scale_v = v_scale != 1.0f;
 #pragma unroll
     for (int cb = 0; cb < NB; cb += 2) {
@@ -974,7 +996,7 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                     else
                         kind = (tag <= MKV_TAG_ANCHOR && id >= 0 && id < P.fp8_pages) ? 2 : 0;
                     if (kind == 0) atomicOr(P.status, kStBounds);     // never dereferenced
-                    if constexpr (TILED) pg -= entry * P.tiles;   // from here on: the tile's index inside its page (kept in the second list)
+                    if constexpr (TILED) pg = (pg - entry * P.tiles) | (entry << 16);   // second list: tile inside its page | logical page << 16
                 }
                 const uint32_t m3 = __ballot_sync(FULL, kind == 1), m8 = __ballot_sync(FULL, kind == 2);
                 const uint32_t lt = (1u << lane) - 1u;
@@ -997,7 +1019,7 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                     mbar_expect_tx(bars + 8 * s, G::TQ3_REC);
                     bulk_load(ring + s * G::SLOT, tq3_base + (size_t)list3[i] * hkv * G::TQ3_REC, G::TQ3_REC, bars + 8 * s);
                 } else {   // the tile only: the page's scale/zero are applied once, when the scan leaves the page
-                    const int page = list3[i], m = lpg3[i];
+                    const int page = list3[i], m = lpg3[i] & 0xFFFF;
                     const uint8_t* pbase = P.tq3 + ((size_t)page * hkv + h) * tq3_page;
                     mbar_expect_tx(bars + 8 * s, TQ3_TILE);
                     bulk_load(ring + s * G::SLOT, pbase + (size_t)m * TQ3_TILE, TQ3_TILE, bars + 8 * s);
@@ -1012,7 +1034,7 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                 if constexpr (!TILED) {
                     rec = fp8_base + (size_t)e8 * hkv * (2 * G::FP8_HALF);
                 } else {
-                    rec = P.fp8 + (((size_t)e8 * hkv + h) * P.tiles + lpg8[i]) * (2 * G::FP8_HALF);
+                    rec = P.fp8 + (((size_t)e8 * hkv + h) * P.tiles + (lpg8[i] & 0xFFFF)) * (2 * G::FP8_HALF);
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 mbar_expect_tx(bars + 8 * s, G::FP8_HALF);
@@ -1042,7 +1064,9 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
             acc.pk[0] = acc.pk[1] = 1.f;
             acc.lp[0] = acc.lp[1] = 0.f;
         };
-        auto fold = [&](int page, bool to_regs) {
+        auto fold = [&](int page, bool to_regs, int logical_page) {
+            if constexpr (SCORED)      // this warp's part of the page's exponential sum
+                store_page_mass<NB, true>(acc, acc.lp[0], acc.lp[1], mass_row + logical_page, P.max_pages, GQ, lane);
             const uint4* meta = reinterpret_cast<const uint4*>(P.tq3 + ((size_t)page * hkv + h) * tq3_page +
                                                                 (size_t)P.tiles * TQ3_TILE + g * 16);
 #pragma unroll
@@ -1142,10 +1166,11 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
             if (n3 > 0) {
                 float s_cur[4], s_next[4];
                 PFrag pf;
-                int cur_page = 0;
+                int cur_page = 0, cur_lp = 0;             // physical id and logical index of the Stale page being scanned
                 if constexpr (TILED) {
                     park_store();
                     cur_page = list3[0];
+                    cur_lp = lpg3[0] >> 16;
                 }
                 wait_slot(0);
                 if (!failed) tq3_step<D, false, true, TILED>(acc, 0, s_cur, pf, ring, qt_lane, sc2, lane, s_cur);
@@ -1157,12 +1182,13 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                     if constexpr (TILED) {
                         const int pg_i = list3[i];
                         if (pg_i != cur_page) {
-                            fold(cur_page, false);
+                            fold(cur_page, false, cur_lp);
                             cur_page = pg_i;
+                            cur_lp = lpg3[i] >> 16;
                         }
                     }
                     tq3_step<D, true, true, TILED>(acc, ring + cur * G::SLOT, s_cur, pf, ring + nxt * G::SLOT, qt_lane, sc2, lane, s_next);
-                    if constexpr (SCORED) store_page_mass<NB>(acc, pf, mass_row + lpg3[i], P.max_pages, GQ, lane);
+                    if constexpr (SCORED && !TILED) store_page_mass<NB>(acc, pf.ps0, pf.ps1, mass_row + lpg3[i], P.max_pages, GQ, lane);
 #pragma unroll
                     for (int e = 0; e < 4; ++e) s_cur[e] = s_next[e];
                     __syncwarp();
@@ -1173,13 +1199,14 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                     if constexpr (TILED) {
                         const int pg_i = list3[n3 - 1];
                         if (pg_i != cur_page) {
-                            fold(cur_page, false);
+                            fold(cur_page, false, cur_lp);
                             cur_page = pg_i;
+                            cur_lp = lpg3[n3 - 1] >> 16;
                         }
                     }
                     tq3_step<D, true, false, TILED>(acc, ring + ((uint32_t)(n3 - 1) % NSTAGE) * G::SLOT, s_cur, pf, 0, qt_lane, sc2, lane, s_next);
-                    if constexpr (SCORED) store_page_mass<NB>(acc, pf, mass_row + lpg3[n3 - 1], P.max_pages, GQ, lane);
-                    if constexpr (TILED) fold(cur_page, true);        // back to output units for the FP8 pages and the reduction
+                    if constexpr (SCORED && !TILED) store_page_mass<NB>(acc, pf.ps0, pf.ps1, mass_row + lpg3[n3 - 1], P.max_pages, GQ, lane);
+                    if constexpr (TILED) fold(cur_page, true, cur_lp);   // back to output units for the FP8 pages and the reduction
                 }
                 __syncwarp();
             }
@@ -1193,8 +1220,9 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                     if (failed) break;
                     const int e = list8[i];
                     const int valid = (e >> 27) & 15;
-                    fp8_page<D, SCORED>(acc, ring + s * G::SLOT, ring + (s + 1) * G::SLOT, qf_lane, sc2 * P.k_scale, P.v_scale,
-                                        valid ? valid : kPage, lane, SCORED ? mass_row + lpg8[i] : nullptr, P.max_pages, GQ);
+                    fp8_page<D, SCORED, TILED>(acc, ring + s * G::SLOT, ring + (s + 1) * G::SLOT, qf_lane, sc2 * P.k_scale, P.v_scale,
+                                               valid ? valid : kPage, lane,
+                                               SCORED ? mass_row + (TILED ? (lpg8[i] >> 16) : lpg8[i]) : nullptr, P.max_pages, GQ);
                     __syncwarp();
                     if (i + NSTAGE / 2 < n8) issue_fp8(i + NSTAGE / 2);
                 }
@@ -1396,11 +1424,11 @@ int decode_tensor_partial_floats(int d) { return 8 * d + 16; }
 // (Eq. score-global-weight and the normalisation over page-addressable mass that follows it).
 // One block per (query head, request); entries beyond the request's pages are set to zero.
 __global__ void __launch_bounds__(256) page_mass_finish_kernel(float* mass, const float* lse, const int32_t* lens,
-                                                              int hq, int max_pages)
+                                                              int hq, int max_pages, int page_tokens)
 {
     __shared__ float red[8];
     const int b = blockIdx.y, h = blockIdx.x, tid = threadIdx.x;
-    const int len = lens[b], n_pages = len > 0 ? (len + kPage - 1) / kPage : 0;
+    const int len = lens[b], n_pages = len > 0 ? (len + page_tokens - 1) / page_tokens : 0;
     float* row = mass + ((size_t)b * hq + h) * max_pages;
     const float lse2 = n_pages > 0 ? lse[(size_t)b * hq + h] * kLog2e : 0.f;
     float sum = 0.f;
@@ -1423,10 +1451,10 @@ __global__ void __launch_bounds__(256) page_mass_finish_kernel(float* mass, cons
 // Eq. (attention-score): r_p = mean over the sampled heads of q~_{h,p}; a_p <- beta a_p + (1 - beta) r_p.
 __global__ void __launch_bounds__(256) page_score_kernel(const float* mass, const int32_t* lens, int hq, int max_pages,
                                                          unsigned long long head_mask, float beta, float inv_heads,
-                                                         float* score)
+                                                         float* score, int page_tokens)
 {
     const int b = blockIdx.y, p = blockIdx.x * 256 + threadIdx.x;
-    const int len = lens[b], n_pages = len > 0 ? (len + kPage - 1) / kPage : 0;
+    const int len = lens[b], n_pages = len > 0 ? (len + page_tokens - 1) / page_tokens : 0;
     if (p >= n_pages) return;
     float r = 0.f;
     for (int h = 0; h < hq; ++h)
@@ -1435,22 +1463,29 @@ __global__ void __launch_bounds__(256) page_score_kernel(const float* mass, cons
     *a = beta * *a + (1.f - beta) * (r * inv_heads);
 }
 
-int32_t launch_page_mass_finish(float* mass, const float* lse, const int32_t* lens, int B, int hq, int max_pages,
-                                cudaStream_t s)
+// pages of several tiles: the scan adds parts of a page's sum to its entry, which therefore starts at -inf
+__global__ void page_mass_clear_kernel(float* mass, size_t n)
 {
-    page_mass_finish_kernel<<<dim3(hq, B), 256, 0, s>>>(mass, lse, lens, hq, max_pages);
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) mass[i] = -CUDART_INF_F;
+}
+
+int32_t launch_page_mass_finish(float* mass, const float* lse, const int32_t* lens, int B, int hq, int max_pages,
+                                int page_tokens, cudaStream_t s)
+{
+    page_mass_finish_kernel<<<dim3(hq, B), 256, 0, s>>>(mass, lse, lens, hq, max_pages, page_tokens);
     MKV_CUDA(cudaGetLastError());
     return MKV_OK;
 }
 
 int32_t launch_page_score(const float* mass, const int32_t* lens, int B, int hq, int max_pages, uint64_t head_mask,
-                          float beta, float* score, cudaStream_t s)
+                          float beta, float* score, int page_tokens, cudaStream_t s)
 {
     int n = 0;
     for (int h = 0; h < hq; ++h) n += (int)((head_mask >> h) & 1ull);
     if (n == 0) return MKV_E_INVALID;
     page_score_kernel<<<dim3((max_pages + 255) / 256, B), 256, 0, s>>>(mass, lens, hq, max_pages, head_mask, beta,
-                                                                         1.f / (float)n, score);
+                                                                         1.f / (float)n, score, page_tokens);
     MKV_CUDA(cudaGetLastError());
     return MKV_OK;
 }
@@ -1464,8 +1499,8 @@ int32_t launch_decode_tensor_at(mkv_pool* p, const void* q, const int32_t* bt, c
         set_last_error("mkv_decode_attention: more than 65535 16-token tiles per table row (1,048,560 tokens per request)");
         return MKV_E_INVALID;
     }
-    if (p->tiles > 1 && (mass || p->variant == MKV_DECODE_TMEM)) {
-        set_last_error("mkv_decode_attention: pages of several tiles are served by the tensor-core kernel without page mass");
+    if (p->tiles > 1 && p->variant == MKV_DECODE_TMEM) {
+        set_last_error("mkv_decode_attention: pages of several tiles are served by the tensor-core kernel");
         return MKV_E_INVALID;
     }
     DecodeParams prm;
@@ -1485,9 +1520,17 @@ int32_t launch_decode_tensor_at(mkv_pool* p, const void* q, const int32_t* bt, c
     prm.mass = mass;
     prm.status = p->status_dev;
     if (mass) {                          // scored variant: the default launch shapes only
-        const int32_t rc = p->d == 128 ? run_tensor<128, 12, 4, 1, true>(p, prm, s) : run_tensor<256, 8, 4, 1, true>(p, prm, s);
+        int32_t rc;
+        if (p->tiles > 1) {
+            const size_t n = (size_t)B * p->hkv * p->group * max_pages;
+            page_mass_clear_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(mass, n);
+            MKV_CUDA(cudaGetLastError());
+            rc = p->d == 128 ? run_tensor<128, 12, 4, 1, true, true>(p, prm, s) : run_tensor<256, 8, 4, 1, true, true>(p, prm, s);
+        } else {
+            rc = p->d == 128 ? run_tensor<128, 12, 4, 1, true>(p, prm, s) : run_tensor<256, 8, 4, 1, true>(p, prm, s);
+        }
         if (rc != MKV_OK) return rc;
-        return launch_page_mass_finish(mass, lse, lens, B, p->hkv * p->group, max_pages, s);
+        return launch_page_mass_finish(mass, lse, lens, B, p->hkv * p->group, max_pages, p->cfg.page_size, s);
     }
     if (p->tiles > 1)                    // pages of several tiles: the default launch shapes only
         return p->d == 128 ? run_tensor<128, 12, 4, 1, false, true>(p, prm, s) : run_tensor<256, 8, 4, 1, false, true>(p, prm, s);

@@ -107,7 +107,7 @@ int32_t launch_decode_tensor_at(mkv_pool* p, const void* q, const int32_t* bt, c
                                 const int32_t* lens, int B, int max_pages, float scale, float* out, float* lse,
                                 float* partials, uint32_t* tickets, int max_blocks, float* mass, cudaStream_t s);
 int32_t launch_page_score(const float* mass, const int32_t* lens, int B, int hq, int max_pages, uint64_t head_mask,
-                          float beta, float* score, cudaStream_t s);
+                          float beta, float* score, int page_tokens, cudaStream_t s);
 constexpr int kMaxCtas = 512;        // upper bound of the decode scan's persistent grid (sizes workspace and tickets)
 int decode_tensor_partial_floats(int d);
 void set_last_error(const char* msg);

@@ -345,14 +345,23 @@ int32_t mkv_decode_attention_scored(mkv_pool* pool, const void* q, const int32_t
                                    page_mass, (cudaStream_t)stream);
 }
 
-int32_t mkv_page_score_update(const float* page_mass, const int32_t* lens, int32_t B, int32_t n_q_heads,
-                              int32_t max_pages, uint64_t head_mask, float beta, float* score, void* stream)
+int32_t mkv_page_score_update_paged(const float* page_mass, const int32_t* lens, int32_t B, int32_t n_q_heads,
+                                    int32_t max_pages, int32_t page_size, uint64_t head_mask, float beta, float* score,
+                                    void* stream)
 {
     if (B < 0 || max_pages < 0 || n_q_heads < 1 || n_q_heads > 64) return MKV_E_INVALID;
+    if (page_size < kPage || page_size % kPage || page_size > kPage * kMaxTiles) return MKV_E_INVALID;
     if (B == 0 || max_pages == 0) return MKV_OK;
     if (!page_mass || !lens || !score || !(beta >= 0.f && beta <= 1.f)) return MKV_E_INVALID;
     if (n_q_heads < 64) head_mask &= (1ull << n_q_heads) - 1ull;
-    return launch_page_score(page_mass, lens, B, n_q_heads, max_pages, head_mask, beta, score, (cudaStream_t)stream);
+    return launch_page_score(page_mass, lens, B, n_q_heads, max_pages, head_mask, beta, score, page_size,
+                             (cudaStream_t)stream);
+}
+
+int32_t mkv_page_score_update(const float* page_mass, const int32_t* lens, int32_t B, int32_t n_q_heads,
+                              int32_t max_pages, uint64_t head_mask, float beta, float* score, void* stream)
+{
+    return mkv_page_score_update_paged(page_mass, lens, B, n_q_heads, max_pages, kPage, head_mask, beta, score, stream);
 }
 
 // ---- sequence rows (Algorithm 1, host bookkeeping only) ----------------------------------------

@@ -105,8 +105,6 @@ def test_decode_over_big_pages_matches_the_oracle(d, hkv, group, page_tokens, le
     with pytest.raises(M.MkvError):
         case.pool.decode_attention(case.q, case.bt, case.tags, case.lens, spec.scale)
     case.pool.set_decode_variant(M.DECODE_TENSOR)
-    with pytest.raises(M.MkvError):
-        case.pool.decode_attention_scored(case.q, case.bt, case.tags, case.lens, spec.scale)
     # the refusals launched nothing and left the pool usable
     out2, _ = case.run()
     assert np.array_equal(out, out2)

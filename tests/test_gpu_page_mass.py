@@ -22,13 +22,20 @@ CASES = {
     "cfg3": lambda: W.config(3, seq_lens=[int(1024 * 8 ** u) for u in np.random.default_rng(3).random(12)], recent_tokens=200),
     "cfg4_f95": lambda: W.config(4, batch=3, ctx=1024, stale_fraction=0.95),
     "ragged": lambda: W.config(1, seq_lens=(1, 17, 0, 1000, 16, 333), recent_tokens=40, anchor_spans=0),
+    # pages of several 16-token tiles: a page's mass is gathered from the warps and blocks that scan its tiles
+    "pages_of_48": lambda: W.config(0, seq_lens=(21 * 48 + 37, 4 * 48, 0, 17), head_dim=128, n_kv_heads=2, group=4,
+                                    anchor_prefix=48, anchor_spans=2, anchor_span_tokens=96, recent_tokens=150, page_tokens=48,
+                                    seed=31),
+    "pages_of_832_d256": lambda: W.config(2, seq_lens=(11 * 832 + 500, 9 * 832), anchor_prefix=832, recent_tokens=1700,
+                                          n_layers=1, page_tokens=832),
 }
 
 
 def oracle_mass(case):
     s = case.spec
     return oracle.page_mass(case.L.fp8_arena, case.L.tq3_arena, s.head_dim, s.n_kv_heads, s.group, case.L.sigma,
-                            case.L.q_bits, case.tab.block_table, case.tab.tier_tag, case.tab.seq_lens, s.scale)
+                            case.L.q_bits, case.tab.block_table, case.tab.tier_tag, case.tab.seq_lens, s.scale,
+                            page_tokens=s.page_tokens)
 
 
 @pytest.mark.parametrize("name", list(CASES))
@@ -54,8 +61,9 @@ def test_page_mass_matches_oracle(name):
     assert torch.equal(out, out2)
 
 
-def test_score_update_matches_oracle_over_two_steps():
-    case = Case(CASES["cfg2"]())
+@pytest.mark.parametrize("name", ["cfg2", "pages_of_832_d256"])
+def test_score_update_matches_oracle_over_two_steps(name):
+    case = Case(CASES[name]())
     spec = case.spec
     _, _, mass = case.pool.decode_attention_scored(case.q, case.bt, case.tags, case.lens, spec.scale)
     P = case.bt.shape[1]
@@ -65,8 +73,8 @@ def test_score_update_matches_oracle_over_two_steps():
     mask = 0b100100100100100100100101                                              # a sampled head set
     ref_mass = oracle_mass(case)
     for beta in (0.9, 0.5):
-        M.page_score_update(mass, case.lens, mask, beta, score)
-        ref = oracle.page_score_update(ref_mass, case.tab.seq_lens, mask, beta, ref)
+        M.page_score_update(mass, case.lens, mask, beta, score, page_tokens=spec.page_tokens)
+        ref = oracle.page_score_update(ref_mass, case.tab.seq_lens, mask, beta, ref, page_tokens=spec.page_tokens)
     torch.cuda.synchronize()
     got = score.cpu().numpy().astype(np.float64)
     assert np.abs(got - ref).max() <= 2e-6

@@ -157,3 +157,54 @@ def test_all_fp8_blocks_and_16_token_pages_hold_the_same_cache():
         outs.append(oracle.decode_attention(L.fp8_arena, L.tq3_arena, 128, 1, 4, L.sigma, L.q_bits, tab.block_table,
                                             tab.tier_tag, tab.seq_lens, spec.scale, page_tokens=pt)[0])
     assert np.abs(outs[0] - outs[1]).max() < 1e-13 and np.abs(outs[0] - outs[2]).max() < 1e-13
+
+
+def test_page_mass_of_blocks_is_the_softmax_probability_summed_over_the_page():
+    """Eq. (score-partial) / (score-global-weight) with the two format partitions collapse to: the mass of a page is the
+    sum of the global softmax probabilities of its tokens.  Checked against an independent evaluation, and, for an
+    all-FP8 cache, against the 16-token page masses of the same cache added up per block."""
+    pt = 80
+    spec = W.config(0, seq_lens=(6 * pt + 33, 3 * pt), head_dim=128, n_kv_heads=2, group=2, anchor_prefix=pt, anchor_spans=0,
+                    recent_tokens=pt + 1, page_tokens=pt, seed=13)
+    tab = W.tables(spec)
+    L = build_layer(spec, tab)
+    mass = oracle.page_mass(L.fp8_arena, L.tq3_arena, 128, 2, 2, L.sigma, L.q_bits, tab.block_table, tab.tier_tag, tab.seq_lens,
+                            spec.scale, page_tokens=pt)
+    assert mass.shape == (2, 4, tab.block_table.shape[1])
+    assert np.abs(mass.sum(-1) - 1).max() < 1e-12
+    for b, hq in ((0, 1), (1, 3)):
+        d, M = 128, pt // 16
+        h, ln = hq // spec.group, spec.seq_lens[b]
+        K = np.zeros((spec.n_pages(b) * pt, d))
+        for pg in range(spec.n_pages(b)):
+            pid = tab.block_table[b, pg]
+            if tab.tier_tag[b, pg] == W.TAG_STALE:
+                kc, g, _, _, _ = oracle.tq3_unpack_block(L.tq3_arena[pid, h], d, M)
+                for t in range(pt):
+                    K[pg * pt + t] = oracle.tq3_decode_key(kc[t], int(g[t]), L.sigma)
+            else:
+                K[pg * pt:(pg + 1) * pt] = oracle.fp8_unpack_block_f32(L.fp8_arena[pid, h], d, M)[0]
+        q = oracle.bf16_bits_to_f32(L.q_bits[b, hq]).astype(np.float64)
+        s = (K[:ln] @ q) * spec.scale
+        p = np.exp(s - s.max())
+        p /= p.sum()
+        want = np.array([p[pg * pt:(pg + 1) * pt].sum() for pg in range(spec.n_pages(b))])
+        assert np.abs(mass[b, hq, :spec.n_pages(b)] - want).max() < 1e-13
+        assert not mass[b, hq, spec.n_pages(b):].any()
+    # Eq. (attention-score) over blocks: pages are counted in units of the page size
+    prev = np.full((2, mass.shape[2]), 0.25)
+    got = oracle.page_score_update(mass, tab.seq_lens, 0b0101, 0.5, prev, page_tokens=pt)
+    n0 = spec.n_pages(0)
+    assert np.abs(got[0, :n0] - (0.125 + 0.5 * (mass[0, 0, :n0] + mass[0, 2, :n0]) / 2)).max() < 1e-15
+    assert np.array_equal(got[0, n0:], prev[0, n0:])
+    # all-FP8: the same cache in 16-token pages; block masses are sums of page masses
+    base = dict(seq_lens=(5 * pt + 7,), head_dim=128, n_kv_heads=1, group=4, anchor_prefix=0, anchor_spans=0, recent_tokens=10 ** 6, seed=5)
+    sb, s16 = W.config(0, page_tokens=pt, **base), W.config(0, **base)
+    tb, t16 = W.tables(sb), W.tables(s16)
+    Lb, L16 = build_layer(sb, tb), build_layer(s16, t16)
+    mb = oracle.page_mass(Lb.fp8_arena, Lb.tq3_arena, 128, 1, 4, Lb.sigma, Lb.q_bits, tb.block_table, tb.tier_tag, tb.seq_lens,
+                          sb.scale, page_tokens=pt)
+    m16 = oracle.page_mass(L16.fp8_arena, L16.tq3_arena, 128, 1, 4, L16.sigma, L16.q_bits, t16.block_table, t16.tier_tag,
+                           t16.seq_lens, s16.scale)
+    for pg in range(sb.n_pages(0)):
+        assert np.abs(mb[0, :, pg] - m16[0, :, pg * 5:(pg + 1) * 5].sum(-1)).max() < 1e-13
