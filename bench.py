@@ -515,12 +515,13 @@ def run_lifecycle(args):
     M.lib()
     spec = workload_spec(args)
     d, hkv, hq = spec.head_dim, spec.n_kv_heads, spec.n_q_heads
-    fp8_page, tq3_page = 32 * d * hkv, (16 * d + 32) * hkv
-    P = max(1024, (384 << 20) // fp8_page)               # FP8 pages converted per call: 384 MB, 3 x L2
-    pool = M.Pool(d, hkv, hq, 2 * P + 8, P + 8, W.rotation_signs(spec, 0), max_batch=1, device=device)
+    Tp, Mt = spec.page_tokens, spec.tiles_per_page
+    fp8_page, tq3_page = Mt * 32 * d * hkv, (Mt * (12 * d + 32) + 4 * d) * hkv
+    P = max(1024 // Mt, (384 << 20) // fp8_page)         # FP8 pages converted per call: 384 MB, 3 x L2
+    pool = M.Pool(d, hkv, hq, 2 * P + 8, P + 8, W.rotation_signs(spec, 0), max_batch=1, device=device, page_tokens=Tp)
     gen = torch.Generator(device=device)
     gen.manual_seed(spec.seed)
-    T = 16 * P
+    T = Tp * P
     k = torch.randn((T, hkv, d), generator=gen, device=device, dtype=torch.float32)
     k[:, :, torch.from_numpy(W.outlier_channels(spec, 0, 0)).to(device)] *= 8.0
     k = k.to(torch.bfloat16)
@@ -559,14 +560,14 @@ def run_lifecycle(args):
     if pool.status() != M.OK:
         raise RuntimeError("device status word set during the lifecycle run")
     new = [torch.randn((spec.batch, hkv, d), generator=gen, device=device).to(torch.bfloat16) for _ in range(2)]
-    step_slots = (torch.arange(spec.batch, dtype=torch.int32, device=device) * 16 + 5)
+    step_slots = (torch.arange(spec.batch, dtype=torch.int32, device=device) * Tp + 5)
     ms_step_append = timed(lambda: pool.append(new[0], new[1], step_slots))
     src1, dst1 = ids[:spec.batch].contiguous(), ids[:spec.batch].contiguous()
     ms_step_demote = timed(lambda: pool.demote(src1, dst1))
     print(json.dumps({
         "mode": "lifecycle", "data": "synthetic", "n_gpus": 1,
         "config": {"workload": "Append / Demote / Promote alone, head geometry of " + workload_name(spec),
-                   "head_dim": d, "kv_heads": hkv, "pages_per_call": P, "tokens_per_append_call": T,
+                   "head_dim": d, "kv_heads": hkv, "page_tokens": Tp, "pages_per_call": P, "tokens_per_append_call": T,
                    "fp8_page_bytes": fp8_page, "tq3_page_bytes": tq3_page, "repetitions": reps,
                    "l2": "every call moves more than 3 x L2"},
         "append": line(ms_append, T, "tokens", T * hkv * d * (4 + 2)),

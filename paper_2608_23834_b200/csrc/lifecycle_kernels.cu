@@ -532,29 +532,53 @@ __global__ void __launch_bounds__(D) demote_kernel(const uint8_t* __restrict__ f
 // over all tokens of the page and writes the page's scale and zero (same arithmetic and order of the
 // halves as in the 16-token record).  One block per (page, KV head).
 template <int D>
-__global__ void __launch_bounds__(D) demote_minmax_kernel(const uint8_t* __restrict__ fp8, uint8_t* __restrict__ tq3,
-                                                           int fp8_pages, int tq3_pages, int hkv, int tiles,
-                                                           float v_scale, const int32_t* __restrict__ src_ids,
-                                                           const int32_t* __restrict__ dst_ids)
+__global__ void __launch_bounds__(1024) demote_minmax_kernel(const uint8_t* __restrict__ fp8, uint8_t* __restrict__ tq3,
+                                                              int fp8_pages, int tq3_pages, int hkv, int tiles,
+                                                              float v_scale, const int32_t* __restrict__ src_ids,
+                                                              const int32_t* __restrict__ dst_ids)
 {
-    const int page = blockIdx.x / hkv, h = blockIdx.x % hkv, c = threadIdx.x;
+    constexpr int R = 1024 / D;                 // tile groups: thread (c, r) scans tiles r, r + R, ...
+    // The minimum and maximum are those a scan in token order with strict comparisons finds: of equal values
+    // (+0 and -0) the earliest token counts, so every candidate carries its token index.
+    __shared__ float mn_s[R][D], mx_s[R][D];
+    __shared__ int mni_s[R][D], mxi_s[R][D];
+    const int page = blockIdx.x / hkv, h = blockIdx.x % hkv, c = threadIdx.x % D, r = threadIdx.x / D;
     const int src = src_ids[page], dst = dst_ids[page];
     if (src < 0 || src >= fp8_pages || dst < 0 || dst >= tq3_pages) return;      // flagged by demote_kernel
     const uint8_t* page8 = fp8 + ((size_t)src * hkv + h) * fp8_page_bytes(D, tiles);
-    float mn = 0.f, mx = 0.f;
-    for (int m = 0; m < tiles; ++m) {
+    // every group starts from the page's first token, so that an empty group (fewer tiles than groups) is neutral
+    float mn, mx;
+    int mni = 0, mxi = 0;
+    {
+        const uint32_t first = *reinterpret_cast<const uint32_t*>(page8 + 16 * D + c * kPage);
+        mn = mx = __fmul_rn(e4m3x2_to_f32(first & 0xFFFFu).x, v_scale);
+    }
+    for (int m = r; m < tiles; m += R) {
         const uint4 raw = *reinterpret_cast<const uint4*>(page8 + (size_t)m * fp8_record_bytes(D) + 16 * D + c * kPage);
         const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
         for (int t = 0; t < kPage; t += 2) {
             const float2 f = e4m3x2_to_f32((rw[t >> 2] >> (8 * (t & 3))) & 0xFFFFu);
             const float a = __fmul_rn(f.x, v_scale), b = __fmul_rn(f.y, v_scale);
-            if (m == 0 && t == 0) mn = mx = a;
-            if (a < mn) mn = a;
-            if (a > mx) mx = a;
-            if (b < mn) mn = b;
-            if (b > mx) mx = b;
+            const int ia = m * kPage + t;
+            if (a < mn) { mn = a; mni = ia; }
+            if (a > mx) { mx = a; mxi = ia; }
+            if (b < mn) { mn = b; mni = ia + 1; }
+            if (b > mx) { mx = b; mxi = ia + 1; }
         }
+    }
+    mn_s[r][c] = mn;
+    mx_s[r][c] = mx;
+    mni_s[r][c] = mni;
+    mxi_s[r][c] = mxi;
+    __syncthreads();
+    if (r != 0) return;
+#pragma unroll
+    for (int k = 1; k < R; ++k) {
+        const float a = mn_s[k][c], b = mx_s[k][c];
+        const int ia = mni_s[k][c], ib = mxi_s[k][c];
+        if (a < mn || (a == mn && ia < mni)) { mn = a; mni = ia; }
+        if (b > mx || (b == mx && ib < mxi)) { mx = b; mxi = ib; }
     }
     uint16_t* meta = reinterpret_cast<uint16_t*>(tq3 + ((size_t)dst * hkv + h) * tq3_page_bytes(D, tiles) +
                                                  (size_t)tiles * (12 * D + 32));
@@ -582,8 +606,13 @@ __global__ void publish_kernel(int n, const int32_t* __restrict__ src_ids, const
     }
 }
 
-// grid rows of the tile-parallel passes
-static int tile_rows(int tiles) { return tiles < 16 ? tiles : 16; }
+// grid rows of the tile-parallel passes: at least 16, and enough to fill the GPU when few pages are converted
+static int tile_rows(int tiles, int n_pages, int hkv)
+{
+    int rows = (4 * 148 + n_pages * hkv - 1) / (n_pages * hkv);
+    if (rows < 16) rows = 16;
+    return rows < tiles ? rows : tiles;
+}
 
 template <typename Kernel, typename... Args>
 static cudaError_t launch_clustered_rows(Kernel kernel, int n_pages, int csize, int rows, int threads, cudaStream_t s,
@@ -615,10 +644,10 @@ static int32_t launch_demote_d(mkv_pool* p, const int32_t* src, const int32_t* d
         return MKV_OK;
     }
     // pages of several tiles: scale/zero of the page, then the tiles in parallel, then the publication
-    demote_minmax_kernel<D><<<n * p->hkv, D, 0, s>>>(p->fp8, p->tq3, p->cfg.fp8_pages, p->cfg.tq3_pages, p->hkv, p->tiles,
+    demote_minmax_kernel<D><<<n * p->hkv, 1024, 0, s>>>(p->fp8, p->tq3, p->cfg.fp8_pages, p->cfg.tq3_pages, p->hkv, p->tiles,
                                                      p->cfg.v_scale, src, dst);
     MKV_CUDA(cudaGetLastError());
-    MKV_CUDA(launch_clustered_rows(demote_kernel<D, true>, n, heads_cluster(p->hkv, 0), tile_rows(p->tiles), D, s,
+    MKV_CUDA(launch_clustered_rows(demote_kernel<D, true>, n, heads_cluster(p->hkv, 0), tile_rows(p->tiles, n, p->hkv), D, s,
                                    (const uint8_t*)p->fp8, p->tq3, p->cfg.fp8_pages, p->cfg.tq3_pages, p->hkv, p->tiles,
                                    p->cfg.k_scale, p->cfg.v_scale, p->sigma, src, dst, (int32_t*)nullptr,
                                    (uint8_t*)nullptr, (const int64_t*)nullptr, p->status_dev));
@@ -823,7 +852,7 @@ static int32_t launch_promote_d(mkv_pool* p, const int32_t* src, const int32_t* 
                                   entry, p->status_dev));
         return MKV_OK;
     }
-    MKV_CUDA(launch_clustered_rows(promote_kernel<D, true>, n, heads_cluster(p->hkv, 0), tile_rows(p->tiles), D, s,
+    MKV_CUDA(launch_clustered_rows(promote_kernel<D, true>, n, heads_cluster(p->hkv, 0), tile_rows(p->tiles, n, p->hkv), D, s,
                                    (const uint8_t*)p->tq3, p->fp8, p->cfg.tq3_pages, p->cfg.fp8_pages, p->hkv, p->tiles, ik,
                                    iv, rs, p->sigma, src, dst, (int32_t*)nullptr, (uint8_t*)nullptr,
                                    (const int64_t*)nullptr, p->status_dev));

@@ -30,6 +30,13 @@ def test_append_demote_promote_of_big_pages_are_bit_exact(d, hkv, page_tokens):
     assert pool.fp8_rec == oracle.fp8_block_bytes(d, Mt) and pool.tq3_rec == oracle.tq3_block_bytes(d, Mt)
     n_tok = n_pages * page_tokens
     k_bits, v_bits = _kv_bits(rng, n_tok, hkv, d)
+    # channels whose extremes are zeros of both signs (the sign of the earliest one goes into the record), a
+    # constant channel, and an all-zero key vector
+    v_bits[:, :, 9] = np.where(np.arange(n_tok) % 5 == 1, 0x8000, 0x0000).astype(np.uint16)[:, None]
+    v_bits[:, :, 10] = np.where(np.arange(n_tok) % 7 == 0, 0x0000, 0x8000).astype(np.uint16)[:, None]
+    v_bits[:, :, 11] = W.f32_to_bf16_bits(np.float32([1.5]))[0]
+    v_bits[:, :, 12] = np.where(np.arange(n_tok) % 3 == 2, 0x8000, W.f32_to_bf16_bits(np.float32([-2.0]))[0]).astype(np.uint16)[:, None]
+    k_bits[page_tokens + 3] = 0
     page_of = rng.permutation(2 * n_pages + 1)[:n_pages]
     slots = np.concatenate([p * page_tokens + np.arange(page_tokens) for p in page_of]).astype(np.int32)
     # one prefill-sized call for most tokens, the last 20 tokens one decode-sized call each way
