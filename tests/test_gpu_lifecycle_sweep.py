@@ -15,17 +15,19 @@ from oracle.lifecycle import PoolModel, STALE
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("frac,ctx,batch", [(0.5, 512, 2), (0.95, 320, 3), (0.0, 256, 2)])
-def test_append_demote_decode_cell(frac, ctx, batch):
-    spec = W.config(4, batch=batch, ctx=ctx, stale_fraction=frac, n_kv_heads=2)
+@pytest.mark.parametrize("frac,ctx,batch,T", [(0.5, 512, 2, 16), (0.95, 320, 3, 16), (0.0, 256, 2, 16), (0.5, 12 * 48, 2, 48)])
+def test_append_demote_decode_cell(frac, ctx, batch, T):
+    """T: tokens per page (16, or three 16-token tiles with one value scale/zero set per page)."""
+    spec = W.config(4, batch=batch, ctx=ctx, stale_fraction=frac, n_kv_heads=2, page_tokens=T)
     d, hkv, hq = spec.head_dim, spec.n_kv_heads, spec.n_q_heads
-    n_pages = ctx // 16
+    Mt = T // 16
+    n_pages = ctx // T
     cap = batch * (n_pages + 2)
     sigma = W.rotation_signs(spec)
-    pool = M.Pool(d, hkv, hq, cap, cap, sigma, max_batch=batch)
-    model = PoolModel(cap, cap)
-    fp8 = np.zeros((cap, hkv, 32 * d), np.uint8)          # the oracle's own arenas
-    tq3 = np.zeros((cap, hkv, 16 * d + 32), np.uint8)
+    pool = M.Pool(d, hkv, hq, cap, cap, sigma, max_batch=batch, page_tokens=T)
+    model = PoolModel(cap, cap, T)
+    fp8 = np.zeros((cap, hkv, oracle.fp8_block_bytes(d, Mt)), np.uint8)          # the oracle's own arenas
+    tq3 = np.zeros((cap, hkv, oracle.tq3_block_bytes(d, Mt)), np.uint8)
     seqs = [M.Seq(pool) for _ in range(batch)]
     mods = [model.new_seq() for _ in range(batch)]
     max_pages = n_pages + 2
@@ -41,12 +43,13 @@ def test_append_demote_decode_cell(frac, ctx, batch):
                 assert (pid, sl, opened) == mods[b].append()
                 if opened:
                     bt[b, len(mods[b].pages) - 1] = pid       # publish the new Recent page
-                slots.append(pid * 16 + sl)
+                slots.append(pid * T + sl)
                 kf, vf = oracle.bf16_bits_to_f32(k_bits[t, b]), oracle.bf16_bits_to_f32(v_bits[t, b])
                 for h in range(hkv):
-                    rec = fp8[pid, h]
-                    rec[sl * d:(sl + 1) * d] = [oracle.e4m3_encode(x) for x in kf[h]]
-                    rec[16 * d + sl:32 * d:16] = [oracle.e4m3_encode(x) for x in vf[h]]
+                    rec = fp8[pid, h, (sl // 16) * 32 * d:(sl // 16 + 1) * 32 * d]     # the 16-token tile of the slot
+                    s16 = sl % 16
+                    rec[s16 * d:(s16 + 1) * d] = [oracle.e4m3_encode(x) for x in kf[h]]
+                    rec[16 * d + s16:32 * d:16] = [oracle.e4m3_encode(x) for x in vf[h]]
         kk = bf16_tensor(k_bits.reshape(-1, hkv, d))
         vv = bf16_tensor(v_bits.reshape(-1, hkv, d))
         pool.append(kk, vv, torch.tensor(slots, dtype=torch.int32, device="cuda:0"))
@@ -57,7 +60,7 @@ def test_append_demote_decode_cell(frac, ctx, batch):
             return
         for b, lp, s, t in pairs:
             for h in range(hkv):
-                tq3[t, h] = oracle.demote_record(fp8[s, h], d, sigma)
+                tq3[t, h] = oracle.demote_block(fp8[s, h], d, Mt, sigma)
         src = torch.tensor([p[2] for p in pairs], dtype=torch.int32, device="cuda:0")
         dst = torch.tensor([p[3] for p in pairs], dtype=torch.int32, device="cuda:0")
         ent = torch.tensor([p[0] * max_pages + p[1] for p in pairs], dtype=torch.int64, device="cuda:0")
@@ -79,7 +82,7 @@ def test_append_demote_decode_cell(frac, ctx, batch):
     # ---- the cell: append one token, demote the page leaving the Recent window, protect one, decode ----
     k1, v1 = W.new_token_kv(spec, 0)
     append_tokens(k1[None], v1[None])
-    recent = max(16, ctx - int(np.floor(frac * n_pages)) * 16 - 16)   # the window shrinks by one page
+    recent = max(T, ctx - int(np.floor(frac * n_pages)) * T - T)   # the window shrinks by one page
     pairs = []
     for b in range(batch):
         moved = seqs[b].age(recent)
@@ -117,8 +120,9 @@ def test_append_demote_decode_cell(frac, ctx, batch):
 
     lens = np.array([m.len for m in mods], np.int32)
     q_bits = W.query(spec)
-    ref, ref_lse = oracle.decode_attention(fp8, tq3, d, hkv, spec.group, sigma, q_bits, bt_h, tg_h, lens, spec.scale)
-    for variant in (M.DECODE_TENSOR, M.DECODE_SCALAR):
+    ref, ref_lse = oracle.decode_attention(fp8, tq3, d, hkv, spec.group, sigma, q_bits, bt_h, tg_h, lens, spec.scale,
+                                           page_tokens=T)
+    for variant in ((M.DECODE_TENSOR, M.DECODE_SCALAR) if T == 16 else (M.DECODE_TENSOR,)):
         pool.set_decode_variant(variant)
         out = pool.decode_attention(bf16_tensor(q_bits), bt, tags, torch.from_numpy(lens).cuda(), spec.scale)
         torch.cuda.synchronize()
@@ -135,7 +139,7 @@ def test_append_demote_decode_cell(frac, ctx, batch):
     if pairs:
         for b, lp, s_id, t_id in pairs:
             for h in range(hkv):
-                fp8[t_id, h] = oracle.promote_record(tq3[s_id, h], d, sigma)
+                fp8[t_id, h] = oracle.promote_block(tq3[s_id, h], d, Mt, sigma)
         src = torch.tensor([p[2] for p in pairs], dtype=torch.int32, device="cuda:0")
         dst = torch.tensor([p[3] for p in pairs], dtype=torch.int32, device="cuda:0")
         ent = torch.tensor([p[0] * max_pages + p[1] for p in pairs], dtype=torch.int64, device="cuda:0")
@@ -146,7 +150,8 @@ def test_append_demote_decode_cell(frac, ctx, batch):
         for b, lp, s_id, t_id in pairs:
             assert bt_h[b, lp] == t_id and tg_h[b, lp] == M.TAG_ANCHOR
             assert np.array_equal(pool.page_read_raw(M.FMT_FP8, t_id).reshape(hkv, -1), fp8[t_id])
-        ref, _ = oracle.decode_attention(fp8, tq3, d, hkv, spec.group, sigma, q_bits, bt_h, tg_h, lens, spec.scale)
+        ref, _ = oracle.decode_attention(fp8, tq3, d, hkv, spec.group, sigma, q_bits, bt_h, tg_h, lens, spec.scale,
+                                         page_tokens=T)
         pool.set_decode_variant(M.DECODE_TENSOR)
         out = pool.decode_attention(bf16_tensor(q_bits), bt, tags, torch.from_numpy(lens).cuda(), spec.scale)
         check_close(out.cpu().numpy(), ref, f"cell f={frac} after promote")
