@@ -41,8 +41,8 @@
  *       channel over all 16 M tokens) follow the tiles.  M = 1 is the 16-token record.  At M = 112,
  *       d = 256 this is 348,672 bytes per page and head: the 3.04 bit/scalar of Section 5.4.
  *     Block-table rows have one entry per page; slot_mapping = page * page_size + position.  With M > 1
- *     mkv_decode_attention() and mkv_decode_attention_scored() run the tensor-core kernel
- *     (MKV_DECODE_SCALAR / _TMEM are refused with MKV_E_INVALID); the page mass is per page of 16 M
+ *     mkv_decode_attention() and mkv_decode_attention_scored() run the tensor-core kernel or, if
+ *     selected, the CUDA-core kernel (MKV_DECODE_TMEM is refused with MKV_E_INVALID); the page mass is per page of 16 M
  *     tokens; mkv_demote() and mkv_promote() take three resp. two launches (page scale/zero, tiles,
  *     publication).
  */

@@ -74,7 +74,7 @@ __global__ void __launch_bounds__(D) decode_scalar_kernel(
     const uint8_t* __restrict__ fp8, const uint8_t* __restrict__ tq3, int fp8_pages, int tq3_pages, int hkv, int G,
     float k_scale, float v_scale, SigmaBits sigma, const __nv_bfloat16* __restrict__ q,
     const int32_t* __restrict__ bt, const uint8_t* __restrict__ tags, const int32_t* __restrict__ lens,
-    int max_pages, float scale, int n_splits, float* __restrict__ part, uint32_t* __restrict__ status)
+    int max_pages, int tiles, float scale, int n_splits, float* __restrict__ part, uint32_t* __restrict__ status)
 {
     extern __shared__ float smem[];
     float* qs = smem;                       // [8][D] query
@@ -113,8 +113,10 @@ __global__ void __launch_bounds__(D) decode_scalar_kernel(
     float O[8], m[8], l[8];
     for (int g = 0; g < 8; ++g) { O[g] = 0.f; m[g] = -CUDART_INF_F; l[g] = 0.f; }
 
+    // `pg` counts 16-token tiles; the table has one entry per page of `tiles` tiles (tiles = 1: 16-token pages)
     for (int pg = lo; pg < hi; ++pg) {
-        const int tag = tags[(size_t)b * max_pages + pg], id = bt[(size_t)b * max_pages + pg];
+        const int entry = pg / tiles, tile = pg - entry * tiles;
+        const int tag = tags[(size_t)b * max_pages + entry], id = bt[(size_t)b * max_pages + entry];
         const int valid = min(kPage, len - pg * kPage);
         const bool is_tq3 = tag == MKV_TAG_STALE;
         const bool ok = is_tq3 ? (id >= 0 && id < tq3_pages && valid == kPage)
@@ -124,9 +126,12 @@ __global__ void __launch_bounds__(D) decode_scalar_kernel(
             continue;
         }
         if (is_tq3) {
-            const uint8_t* rec = tq3 + ((size_t)id * hkv + h) * tq3_record_bytes(D);
+            // one tile of the page: key codes, value codes and g as in a 16-token record; the value scale/zero
+            // of the page follow its last tile
+            const uint8_t* page = tq3 + ((size_t)id * hkv + h) * tq3_page_bytes(D, tiles);
+            const uint8_t* rec = page + (size_t)tile * tq3_tile_bytes(D);
             const int cb = tid >> 4, row = tid & 15;
-            const __half* meta = reinterpret_cast<const __half*>(rec + 12 * D + 32);
+            const __half* meta = reinterpret_cast<const __half*>(page + (size_t)tiles * tq3_tile_bytes(D));
             const int mi = (cb >> 1) * 64 + (row & 7) * 8 + 4 * (cb & 1) + (row >> 3);
             const float vsc = __half2float(meta[mi]), vzp = __half2float(meta[mi + 2]);
             for (int t = 0; t < kPage; ++t) {
@@ -136,7 +141,7 @@ __global__ void __launch_bounds__(D) decode_scalar_kernel(
             }
             if (tid < kPage) gn[tid] = __half2float(reinterpret_cast<const __half*>(rec + 12 * D)[tid]);
         } else {
-            const uint8_t* rec = fp8 + ((size_t)id * hkv + h) * fp8_record_bytes(D);
+            const uint8_t* rec = fp8 + (((size_t)id * hkv + h) * tiles + tile) * fp8_record_bytes(D);
             for (int t = 0; t < kPage; ++t) {
                 Ks[t * (D + 1) + tid] = e4m3_f32(rec[t * D + tid]) * k_scale;
                 Vs[t * D + tid] = e4m3_f32(rec[16 * D + tid * kPage + t]) * v_scale;
@@ -224,7 +229,7 @@ static int32_t run_scalar(mkv_pool* p, const void* q, const int32_t* bt, const u
     dim3 grid(S, p->hkv, B);
     decode_scalar_kernel<D><<<grid, D, smem, s>>>(p->fp8, p->tq3, p->cfg.fp8_pages, p->cfg.tq3_pages, p->hkv,
                                                   p->group, p->cfg.k_scale, p->cfg.v_scale, p->sigma,
-                                                  (const __nv_bfloat16*)q, bt, tags, lens, max_pages, scale, S,
+                                                  (const __nv_bfloat16*)q, bt, tags, lens, max_pages, p->tiles, scale, S,
                                                   part, p->status_dev);
     MKV_CUDA(cudaGetLastError());
     merge_scalar_kernel<D><<<dim3(p->hq, B), D, 0, s>>>(part, S, p->hq, out, lse);

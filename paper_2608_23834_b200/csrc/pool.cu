@@ -315,10 +315,6 @@ int32_t mkv_decode_attention(mkv_pool* pool, const void* q, const int32_t* bt, c
     size_t need;
     if (mkv_decode_workspace_bytes(&pool->cfg, B, &need) != MKV_OK || ws_bytes < need) return MKV_E_INVALID;
     if (!(scale == scale)) return MKV_E_INVALID;
-    if (pool->variant == MKV_DECODE_SCALAR && pool->tiles > 1) {
-        set_last_error("mkv_decode_attention: pages of several tiles are served by the tensor-core kernel only");
-        return MKV_E_INVALID;
-    }
     if (pool->variant == MKV_DECODE_SCALAR)
         return launch_decode_scalar(pool, q, bt, tags, lens, B, max_pages, scale, out, lse, ws, ws_bytes,
                                     (cudaStream_t)stream);

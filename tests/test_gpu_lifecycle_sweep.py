@@ -122,7 +122,7 @@ def test_append_demote_decode_cell(frac, ctx, batch, T):
     q_bits = W.query(spec)
     ref, ref_lse = oracle.decode_attention(fp8, tq3, d, hkv, spec.group, sigma, q_bits, bt_h, tg_h, lens, spec.scale,
                                            page_tokens=T)
-    for variant in ((M.DECODE_TENSOR, M.DECODE_SCALAR) if T == 16 else (M.DECODE_TENSOR,)):
+    for variant in (M.DECODE_TENSOR, M.DECODE_SCALAR):
         pool.set_decode_variant(variant)
         out = pool.decode_attention(bf16_tensor(q_bits), bt, tags, torch.from_numpy(lens).cuda(), spec.scale)
         torch.cuda.synchronize()
