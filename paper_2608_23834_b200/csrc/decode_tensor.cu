@@ -232,7 +232,7 @@ __device__ __forceinline__ void affine_accumulate(float (&acc)[4], const float (
 // ------------------------------------------------------------------------------------------------
 // Work = (request, KV head, page) triples in row-major order; cum[b] = index of the first triple of
 // request b.  Two ways to cut it into one contiguous range per block:
-//   row-aligned (few rows: B * hkv <= grid / 12): every row gets a whole number of blocks in proportion
+//   row-aligned (few rows: B * hkv <= grid / 4): every row gets a whole number of blocks in proportion
 //     to its pages (cumulative rounding), so that no block straddles two rows and pays the per-row set-up
 //     and reduction twice;
 //   linear (many rows): grid equal ranges that may cross row boundaries.
@@ -252,8 +252,10 @@ __device__ __forceinline__ void build_partition(Partition* pt, const int* cum, c
     const long long W = cum[B];
     const int rows = B * hkv;
     int blocks = (int)(W < (long long)grid ? W : (long long)grid);
-    // with k blocks per row the rows that get one block fewer run 1/k longer: worth it from about twelve
-    int aligned = (rows * 12 <= grid && rows <= kMaxAlignedRows && W >= grid) ? 1 : 0;
+    // With k blocks per row the rows that get one block fewer run 1/k longer, but a block that straddles two rows
+    // pays the per-row set-up, reduction and partial twice (about 8 us, a quarter of a block's pages at config-1
+    // sizes).  Measured: from four blocks per row on, whole blocks per row win (16 rows: 71 -> 66 us, 32 rows: 74 -> 71).
+    int aligned = (rows * 4 <= grid && rows <= kMaxAlignedRows && W >= grid) ? 1 : 0;
     if (aligned) {
         // block boundaries at the rounded cumulative share of the rows: base[r] = round(grid * first_page(r) / W);
         // every row must end up with at least one block, otherwise the linear cut is used
