@@ -147,3 +147,34 @@ def test_runs_longer_than_a_round_park_and_fold_across_rounds():
         check_close(out[3, hq], ref[3, hq], f"b=3 hq={hq}")
         assert abs(lse[3, hq] - ref_lse[3, hq]) < 2e-3
     assert np.isfinite(out).all()
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_page_sizes_lengths_and_tier_mixes(seed):
+    """Drawn shapes: page size, head geometry, ragged lengths (empty, shorter than a tile, partial last pages), tier
+    mix; the tensor-core kernel and the CUDA-core kernel against the oracle, plus the page mass."""
+    rng = np.random.default_rng(1000 + seed)
+    page_tokens = int(rng.choice([32, 48, 80, 160, 256, 1024]))
+    d = int(rng.choice([128, 256]))
+    hkv = int(rng.choice([1, 2, 3]))
+    group = int(rng.choice([1, 4, 6, 8]))
+    batch = int(rng.integers(1, 5))
+    lens = [int(rng.choice([0, 5, page_tokens, int(rng.integers(1, 9 * page_tokens))])) for _ in range(batch)]
+    lens[0] = int(rng.integers(3 * page_tokens, 12 * page_tokens))
+    spec = W.config(0, seq_lens=lens, head_dim=d, n_kv_heads=hkv, group=group, anchor_prefix=page_tokens * int(rng.integers(0, 2)),
+                    anchor_spans=int(rng.integers(0, 3)), anchor_span_tokens=page_tokens,
+                    recent_tokens=int(rng.integers(1, 3 * page_tokens)), page_tokens=page_tokens, seed=50 + seed)
+    case = Case(spec, extra_fp8=1, extra_tq3=1)
+    out, lse = case.run()
+    ref, ref_lse = case.reference()
+    check_case(case, out, lse, ref, ref_lse)
+    out_s, lse_s = case.run(M.DECODE_SCALAR)
+    check_case(case, out_s, lse_s, ref, ref_lse)
+    case.pool.set_decode_variant(M.DECODE_TENSOR)
+    _, _, mass = case.pool.decode_attention_scored(case.q, case.bt, case.tags, case.lens, spec.scale)
+    torch.cuda.synchronize()
+    assert case.pool.status() == M.OK
+    want = oracle.page_mass(case.L.fp8_arena, case.L.tq3_arena, d, hkv, group, case.L.sigma, case.L.q_bits, case.tab.block_table,
+                            case.tab.tier_tag, case.tab.seq_lens, spec.scale, page_tokens=page_tokens)
+    got = mass.cpu().numpy().astype(np.float64)
+    assert (np.abs(got - want) <= 1e-6 + 1e-4 * want).all(), np.abs(got - want).max()
