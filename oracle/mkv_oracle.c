@@ -564,7 +564,7 @@ typedef struct {
 static int materialise(const orc_pool* p, const int32_t* row, const uint8_t* tags, int len, int h,
                        double* K, double* V)
 {
-    int d = p->d, M = p->M, T = ORC_T * M, n_pages = (len + T - 1) / T, pg, t, i, m;
+    int d = p->d, M = p->M, T = ORC_T * M, n_pages = (len + T - 1) / T, pg, t, i;
     uint8_t* kc = (uint8_t*)malloc((size_t)T * d);
     uint8_t* vc = (uint8_t*)malloc((size_t)T * d);
     uint16_t* g = (uint16_t*)malloc(sizeof(uint16_t) * (size_t)T);
@@ -599,7 +599,6 @@ static int materialise(const orc_pool* p, const int32_t* row, const uint8_t* tag
             rc = -1;
         }
     }
-    (void)m;
     free(kc); free(vc); free(g);
     return rc;
 }
