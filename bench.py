@@ -37,7 +37,7 @@ METRIC = "decode attention tokens/s and achieved KV HBM GB/s (% of B200 peak) at
 UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode_tensor_kernel launch on the default
 # workload, from the ncu capture summarised under profiles/; None until captured.
-TRAFFIC_BYTES_PER_LAUNCH = 126854656 + 4088832   # dram read + write of one decode launch (ncu, config 2; profiles/decode_tensor_cfg2.md)
+TRAFFIC_BYTES_PER_LAUNCH = 126853120 + 3811072   # dram read + write of one decode launch (ncu, config 2; profiles/decode_tensor_cfg2.md)
 FALLBACK_HBM_GBS = 6650.0
 STAGE_PAGES = 512
 
