@@ -3,7 +3,7 @@
 
 One step = one decode step of the whole hot path over the batch, for every layer of the workload:
 Append of the new token's K/V into the Recent FP8 page, Demote (FP8 -> TQ3, publish) of the page
-that leaves the Recent window when one does, an Anchor tag flip at each such retier point, and
+that leaves the Recent window when one does, and
 mkv_decode_attention (table walk, query rotation, FP8 and TQ3 page scans, split partials, merge).
 Default workload: 2 requests x 59,008 tokens, 16 layers each with its own pool, d = 256,
 4 KV x 6 query heads, first 256 tokens Anchor, last 2,048 Recent, the rest TQ3.
@@ -35,11 +35,24 @@ import mkv_workloads as W  # noqa: E402
 
 METRIC = "decode attention tokens/s and achieved KV HBM GB/s (% of B200 peak) at 1 GPU"
 UNIT = "tokens/s"
-# dram__bytes_read.sum + dram__bytes_write.sum of one decode_tensor_kernel launch on the default
-# workload, from the ncu capture summarised under profiles/; None until captured.
-TRAFFIC_BYTES_PER_LAUNCH = 126853120 + 3811072   # dram read + write of one decode launch (ncu, config 2; profiles/decode_tensor_cfg2.md)
+# DRAM traffic of the decode kernel (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture) is kept
+# as data beside the profile summaries; the line reports it only for the workload and format it was taken on.
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "dram_traffic.json")
 FALLBACK_HBM_GBS = 6650.0
 STAGE_PAGES = 512
+
+
+def traffic_per_launch(workload_key, layers_per_launch):
+    """DRAM bytes of one decode launch from the recorded capture (per layer, scaled to the layers of a launch:
+    the scan reads every page once, so traffic grows in proportion), or None when no capture covers the workload."""
+    try:
+        with open(TRAFFIC_FILE) as f:
+            rec = json.load(f).get(workload_key)
+    except (OSError, ValueError):
+        return None
+    if not rec:
+        return None
+    return int((rec["dram_read_bytes_per_layer"] + rec["dram_write_bytes_per_layer"]) * layers_per_launch)
 
 
 def measured_peaks():
@@ -295,34 +308,54 @@ def run_ours(args):
     ev_pairs = []
 
     def retier(L, ev):
-        src, dst, ent, nxt = ev
+        src, dst, ent, _ = ev
         L.pool.demote(src, dst, L.bt, L.tags, ent)
-        for e in nxt:                             # retier checkpoint: protect / unprotect the page that follows
-            L.pool.set_anchor(L.tags, e, True)
-            L.pool.set_anchor(L.tags, e, False)
-        launches[0] += 1 + 2 * len(nxt)
+        launches[0] += 1
 
     def mark_retired(i):
         if plan["ev_dev"][i] is not None:
             for (b, lp, _, _) in plan["events"][i]:
                 tags_host[b, lp] = W.TAG_STALE
 
-    def step(i, timed_events=None):
-        """One step, every call issued from Python: per layer append, (demote), decode."""
-        ev = plan["ev_dev"][i]
-        for L in layers:
-            L.pool.append(L.k_new, L.v_new, plan["slots"][i])
-            launches[0] += 1
-            if ev is not None:
-                retier(L, ev)
+    # The library's batched calls take all layers of the step in one launch each (append, decode); they serve
+    # 16-token pages and the tensor-core kernel.  Other variants and page sizes go layer by layer.
+    batched = (not args.per_layer) and args.variant == "tensor" and spec.page_tokens == 16 and len(layers) <= M.MAX_LAYERS_PER_CALL
+    pools = [L.pool for L in layers]
+    layers_per_decode_launch = len(layers) if batched else 1
+
+    def calls(slots_t, lens_t, qs, ks, vs, outs, timed_events=None):
+        """The append and decode calls of one step for all layers."""
+        if batched:
+            M.append_layers(pools, ks, vs, slots_t)
             if timed_events is not None:
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record(stream)
-            L.pool.decode_attention(L.q, L.bt, L.tags, plan["lens"][i], spec.scale, out=L.out)
-            launches[0] += decode_launches
+            M.decode_attention_layers(pools, qs, [L.bt for L in layers], [L.tags for L in layers], lens_t, spec.scale, outs)
             if timed_events is not None:
                 e1.record(stream)
                 timed_events.append((e0, e1))
+            return 2
+        for li, L in enumerate(layers):
+            L.pool.append(ks[li], vs[li], slots_t)
+            if timed_events is not None:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+            L.pool.decode_attention(qs[li], L.bt, L.tags, lens_t, spec.scale, out=outs[li])
+            if timed_events is not None:
+                e1.record(stream)
+                timed_events.append((e0, e1))
+        return len(layers) * (1 + decode_launches)
+
+    all_q, all_k, all_v, all_out = ([L.q for L in layers], [L.k_new for L in layers], [L.v_new for L in layers],
+                                    [L.out for L in layers])
+
+    def step(i, timed_events=None):
+        """One step, every call issued from Python: demote where a page leaves the window, append, decode."""
+        ev = plan["ev_dev"][i]
+        if ev is not None:
+            for L in layers:
+                retier(L, ev)
+        launches[0] += calls(plan["slots"][i], plan["lens"][i], all_q, all_k, all_v, all_out, timed_events)
         mark_retired(i)
 
     def barrier():
@@ -354,10 +387,10 @@ def run_ours(args):
     cur_lens = torch.empty_like(plan["lens"][0])
     base_g = Wm + K
 
+    per_step_launches = [0]
+
     def layer_calls():
-        for L in layers:
-            L.pool.append(L.k_new, L.v_new, cur_slots)
-            L.pool.decode_attention(L.q, L.bt, L.tags, cur_lens, spec.scale, out=L.out)
+        per_step_launches[0] = calls(cur_slots, cur_lens, all_q, all_k, all_v, all_out)
 
     def step_graph(i, graph):
         ev = plan["ev_dev"][i]
@@ -367,7 +400,7 @@ def run_ours(args):
             for L in layers:
                 retier(L, ev)
         graph.replay()
-        launches[0] += len(layers) * (1 + decode_launches)
+        launches[0] += per_step_launches[0]
         mark_retired(i)
 
     graph = torch.cuda.CUDAGraph()
@@ -430,7 +463,12 @@ def run_ours(args):
     def layer_calls_e2e():
         main = torch.cuda.current_stream()
         d_in.copy_(h_in, non_blocking=True)          # host -> device: the step's inputs (one copy; per-layer copies
-        for li, L in enumerate(layers):              # on a second stream measured slower)
+        if batched:                                  # on a second stream measured slower)
+            calls(d_slots, d_lens, [v_[0] for v_ in views], [v_[1] for v_ in views], [v_[2] for v_ in views],
+                  [d_out[li] for li in range(len(layers))])
+            h_out.copy_(d_out, non_blocking=True)    # device -> host: the outputs of all layers
+            return
+        for li, L in enumerate(layers):
             qv, kv_, vv = views[li]
             L.pool.append(kv_, vv, d_slots)
             L.pool.decode_attention(qv, L.bt, L.tags, d_lens, spec.scale, out=d_out[li])
@@ -476,9 +514,10 @@ def run_ours(args):
     peaks, peak_kind = measured_peaks()
     peak = float(peaks["hbm_gbs"])
     avg_kernel_ms = sum(kern_ms) / len(kern_ms)
-    avg_bytes = sum(bytes_per_launch) / len(bytes_per_launch)
+    # bytes_per_launch holds one layer's algorithmic bytes per step; a launch covers layers_per_decode_launch layers
+    avg_bytes = sum(bytes_per_launch) / len(bytes_per_launch) * layers_per_decode_launch
     achieved = avg_bytes / (avg_kernel_ms * 1e-3) / 1e9
-    step_bytes = avg_bytes * spec.n_layers
+    step_bytes = avg_bytes / layers_per_decode_launch * spec.n_layers
     result = {
         "metric": METRIC, "value": aggregate_value(B, K, ms, world), "unit": UNIT, "n_gpus": world, "steps": K,
         "warmup": Wm, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -488,12 +527,16 @@ def run_ours(args):
                    "parallelism": "replicas only" if world > 1 else "single GPU",
                    "l2": "inputs larger than L2 (%.0f MB of KV per step)" % (step_bytes / 1e6),
                    "step": "append + demote at its natural cadence + decode attention, every layer",
-                   "launch": "one CUDA graph per step (append + decode of every layer); retier calls issued directly"},
+                   "launch": ("one CUDA graph per step holding mkv_append_layers and mkv_decode_attention_layers (all layers in "
+                              "one launch each); retier calls issued directly") if batched else
+                             "one CUDA graph per step (append + decode of every layer); retier calls issued directly",
+                   "layers_per_decode_launch": layers_per_decode_launch},
         "eager_ms_per_step": eager_ms / K,
         "kv_gbs_whole_step": step_bytes / (ms / K * 1e-3) / 1e9,
         "roofline": {"bound": "hbm", "kernel": {"tensor": "decode_tensor_kernel", "tmem": "decode_tmem_kernel"}.get(args.variant, "decode_scalar_kernel + merge"), "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_kind + " copy bandwidth",
-                     "frac_of_nominal_8000": achieved / 8000.0, "traffic": TRAFFIC_BYTES_PER_LAUNCH if (args.config == 2 and args.ctx == 0 and args.variant == "tensor") else None,
+                     "frac_of_nominal_8000": achieved / 8000.0, "traffic": traffic_per_launch("cfg2_%s_%s" % (args.variant, args.format), layers_per_decode_launch)
+                     if (args.config == 2 and args.ctx == 0 and args.page_tokens == 0) else None,
                      "algorithmic_bytes_per_launch": avg_bytes, "avg_launch_ms": avg_kernel_ms,
                      "median_launch_ms": statistics.median(kern_ms), "min_launch_ms": min(kern_ms)},
         "e2e": {"value": aggregate_value(B, K, e2e_ms, world), "unit": UNIT, "h2d_bytes_per_step": h2d,
@@ -700,6 +743,10 @@ def main():
     ap.add_argument("--page-tokens", type=int, default=0,
                     help="override the page size (a multiple of 16; 1792 and 832 are the paper's block sizes)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--format", default="v1", choices=["v1", "v2"],
+                    help="TQ3 record format of the pools (v2: e4m3-exact key codebook, FP8 key products)")
+    ap.add_argument("--per-layer", action="store_true",
+                    help="issue mkv_append / mkv_decode_attention layer by layer instead of the batched calls")
     ap.add_argument("--lifecycle", action="store_true",
                     help="time Append, Demote and Promote alone (bulk throughput) instead of the decode step")
     args = ap.parse_args()

@@ -143,6 +143,13 @@ int32_t mkv_pool_status(mkv_pool* pool, void* stream);
 /* Select the decode kernel (MKV_DECODE_TENSOR by default). */
 int32_t mkv_pool_set_decode_variant(mkv_pool* pool, int32_t variant);
 
+/* Wall-time limit, in nanoseconds, of the decode scan's waits for a page copy (Section 4.1: the direct
+ * path "fails closed").  Default 20,000,000 (20 ms).  A wait that runs out makes the block stop scanning,
+ * wait (with the default limit) for the copies it still has in flight, and finish; the call's output is
+ * then not valid and mkv_pool_status() returns MKV_E_TIMEOUT.  0 makes every wait that is not satisfied
+ * at once give up: a diagnostic setting that exercises this path. */
+int32_t mkv_pool_set_wait_limit_ns(mkv_pool* pool, uint64_t ns);
+
 /* Test hooks: copy one page (all KV heads; n_kv_heads * record bytes) between the arena and a
  * host buffer, synchronously.  Lets a test compare packed bytes with a reference encoder, or
  * install pages encoded elsewhere. */
@@ -156,8 +163,8 @@ const char* mkv_last_cuda_error(void);
 /* Append (Algorithm 1 step 1, Section 3.1 "Recent"): write the K and V of n_tokens new tokens
  * into FP8 pages as e4m3.
  *   k, v          device, bf16 [n_tokens][n_kv_heads][d]
- *   slot_mapping  device, int32 [n_tokens]: page_id * 16 + slot in the FP8 arena; negative =
- *                 skip the token.  An id beyond the arena is skipped and flagged (MKV_E_BOUNDS).
+ *   slot_mapping  device, int32 [n_tokens]: page_id * page_size + position in the FP8 arena;
+ *                 negative = skip the token.  An id beyond the arena is skipped and flagged (MKV_E_BOUNDS).
  * The caller publishes the page in the block table (tag MKV_TAG_RECENT) when it opens it. */
 int32_t mkv_append(mkv_pool* pool, const void* k_dev, const void* v_dev, const int32_t* slot_mapping_dev,
                    int32_t n_tokens, void* stream);
@@ -178,9 +185,8 @@ int32_t mkv_demote(mkv_pool* pool, const int32_t* src_fp8_ids_dev, const int32_t
                    int32_t n_pages, int32_t* block_table_dev, uint8_t* tier_tag_dev,
                    const int64_t* entry_index_dev, void* stream);
 
-/* Promote (Algorithm 1 step 3; Section 3.1 "A Stale page is materialized and promoted when it
- * re-enters the protected budget"): reconstruct n_pages TQ3 pages (all KV heads) into newly
- * allocated FP8 pages, then publish id and MKV_TAG_ANCHOR; arguments as for mkv_demote with the
+/* Promote (Algorithm 1 step 3; Section 3.1, Anchor tier: a Stale page that becomes protected again
+ * is rebuilt at FP8): reconstruct n_pages TQ3 pages (all KV heads) into newly allocated FP8 pages, then publish id and MKV_TAG_ANCHOR; arguments as for mkv_demote with the
  * arenas swapped.  Keys: inverse Walsh-Hadamard of the signed levels times the norm correction and
  * d^-1/2, rotation signs undone; values: scale * code + zero; both rounded to e4m3 like Append.  The
  * TQ3 source is not modified; free it once earlier readers are ordered before its next writer. */
@@ -214,13 +220,51 @@ int32_t mkv_decode_attention(mkv_pool* pool, const void* q_dev, const int32_t* b
                              int32_t max_pages, float scale, float* out_dev, float* lse_dev,
                              void* workspace_dev, size_t workspace_bytes, void* stream);
 
+/* The decode step of several layers in one launch (Section 4.1 runs the direct FP8/TQ3 path of all
+ * full-attention layers of a decode step from one CUDA graph; Section 5, evaluated profiles).  Layer i
+ * has its own pool, query, table, tags, outputs and workspace; the requests (seq_lens, B, max_pages,
+ * scale) are common to all layers, and all pools have the same geometry (head_dim, heads, 16-token
+ * pages).  Every block of the persistent scan walks its share of layer 0, then of layer 1, ... without
+ * waiting for the other blocks, so the table walk and query rotation of one layer and the merge of the
+ * layer before overlap the page scans of their neighbours; results are those of n_layers calls of
+ * mkv_decode_attention (the same kernel code per layer).
+ *   layers_host  host array of n_layers entries (copied into the launch; free to reuse on return);
+ *                lse_dev may be NULL; every workspace_dev as for mkv_decode_attention, distinct per layer
+ *   n_layers     1 .. MKV_MAX_LAYERS_PER_CALL; MKV_E_INVALID beyond, for pools of different geometry,
+ *                for pages of more than 16 tokens, or for a pool set to another decode variant */
+#define MKV_MAX_LAYERS_PER_CALL 32
+typedef struct {
+    mkv_pool* pool;
+    const void* q_dev;                  /* bf16 [B][n_q_heads][d]                   */
+    const int32_t* block_table_dev;     /* int32 [B][max_pages]                     */
+    const uint8_t* tier_tag_dev;        /* uint8 [B][max_pages]                     */
+    float* out_dev;                     /* fp32 [B][n_q_heads][d]                   */
+    float* lse_dev;                     /* fp32 [B][n_q_heads] or NULL              */
+    void* workspace_dev;                /* this layer's workspace                   */
+} mkv_layer_call;
+int32_t mkv_decode_attention_layers(const mkv_layer_call* layers_host, int32_t n_layers, const int32_t* seq_lens_dev,
+                                    int32_t B, int32_t max_pages, float scale, size_t workspace_bytes, void* stream);
+
+/* Append (Algorithm 1 step 1) of the same n_tokens positions into the pools of several layers in one
+ * launch: layer i converts k_dev[i], v_dev[i] (bf16 [n_tokens][n_kv_heads][d]) into its own FP8 arena at
+ * slot_mapping (common to the layers: every layer's table names the same page ids).  Decode-sized
+ * calls only (n_tokens <= 64); same bytes as n_layers calls of mkv_append. */
+typedef struct {
+    mkv_pool* pool;
+    const void* k_dev;
+    const void* v_dev;
+} mkv_layer_append;
+int32_t mkv_append_layers(const mkv_layer_append* layers_host, int32_t n_layers, const int32_t* slot_mapping_dev,
+                          int32_t n_tokens, void* stream);
+
 /* The same decode attention for callers that cannot give the library a workspace because they are
  * not allowed to allocate device memory once they are running (a server that handed its whole
  * memory budget to the KV pool at start-up, code living inside another component's memory manager,
  * a process whose allocator is frozen while it serves).  (The paper has no counterpart: this is a
  * property of the library, not of the method.)  The split partials go to a fixed array inside the
  * library image, MKV_STATIC_SCRATCH_BYTES per GPU that loads the library, held until the process
- * exits.  Arguments, results and kernels are those of mkv_decode_attention (tensor-core kernel).
+ * exits.  Arguments, results and kernel are those of mkv_decode_attention with the tensor-core variant;
+ * a pool that was switched to another variant is refused with MKV_E_INVALID.
  *   - allocates nothing: no cudaMalloc / cudaFree, no allocating library call, on any call.
  *   - limits: B <= MKV_STATIC_MAX_BATCH, and the scan must not launch more than MKV_STATIC_MAX_BLOCKS
  *     blocks on this GPU (it launches one per SM on B200); beyond either the call launches nothing and

@@ -34,7 +34,9 @@ EXPORTS = [
     "mkv_seq_protect", "mkv_seq_demote", "mkv_seq_age", "mkv_seq_len", "mkv_seq_row",
     "mkv_decode_attention_static", "mkv_promote", "mkv_seq_promote",
     "mkv_decode_attention_scored", "mkv_page_score_update", "mkv_page_score_update_paged",
+    "mkv_decode_attention_layers", "mkv_append_layers", "mkv_pool_set_wait_limit_ns",
 ]
+MAX_LAYERS_PER_CALL = 32
 
 
 class MkvError(RuntimeError):
@@ -55,6 +57,15 @@ class PoolConfig(C.Structure):
 class Stats(C.Structure):
     _fields_ = [(n, C.c_int64) for n in ("fp8_pages_total", "fp8_pages_used", "tq3_pages_total", "tq3_pages_used",
                                          "fp8_bytes_used", "tq3_bytes_used", "bf16_bytes_equivalent")]
+
+
+class LayerCall(C.Structure):
+    _fields_ = [("pool", C.c_void_p), ("q_dev", C.c_void_p), ("block_table_dev", C.c_void_p), ("tier_tag_dev", C.c_void_p),
+                ("out_dev", C.c_void_p), ("lse_dev", C.c_void_p), ("workspace_dev", C.c_void_p)]
+
+
+class LayerAppend(C.Structure):
+    _fields_ = [("pool", C.c_void_p), ("k_dev", C.c_void_p), ("v_dev", C.c_void_p)]
 
 
 def lib():
@@ -94,6 +105,10 @@ def lib():
             "mkv_page_score_update": [f32p, vp, C.c_int32, C.c_int32, C.c_int32, C.c_uint64, C.c_float, f32p, vp],
             "mkv_page_score_update_paged": [f32p, vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_uint64, C.c_float,
                                             f32p, vp],
+            "mkv_decode_attention_layers": [C.POINTER(LayerCall), C.c_int32, vp, C.c_int32, C.c_int32, C.c_float,
+                                            C.c_size_t, vp],
+            "mkv_append_layers": [C.POINTER(LayerAppend), C.c_int32, vp, C.c_int32, vp],
+            "mkv_pool_set_wait_limit_ns": [vp, C.c_uint64],
             "mkv_seq_create": [vp, C.POINTER(vp)],
             "mkv_seq_finish": [vp],
             "mkv_seq_append": [vp, i32p, i32p, i32p],
@@ -209,6 +224,9 @@ class Pool:
     def set_decode_variant(self, variant: int) -> None:
         _check(lib().mkv_pool_set_decode_variant(self.handle, variant), "mkv_pool_set_decode_variant")
 
+    def set_wait_limit_ns(self, ns: int) -> None:
+        _check(lib().mkv_pool_set_wait_limit_ns(self.handle, int(ns)), "mkv_pool_set_wait_limit_ns")
+
     def page_read_raw(self, fmt: int, pid: int) -> np.ndarray:
         buf = np.zeros(self.hkv * (self.fp8_rec if fmt == FMT_FP8 else self.tq3_rec), np.uint8)
         _check(lib().mkv_page_read_raw(self.handle, fmt, pid, C.c_void_p(buf.ctypes.data), _stream(None)), "mkv_page_read_raw")
@@ -288,6 +306,40 @@ class Pool:
                                                  _ptr(page_mass), _ptr(ws), ws.numel(), _stream(stream)),
                "mkv_decode_attention_scored")
         return out, lse, page_mass
+
+
+def decode_attention_layers(pools, qs, block_tables, tier_tags, seq_lens, scale, outs, lses=None, stream=None):
+    """mkv_decode_attention_layers: the decode attention of len(pools) layers in one launch; layer i reads
+    pools[i], qs[i], block_tables[i], tier_tags[i] and writes outs[i] (and lses[i]); seq_lens is common."""
+    n = len(pools)
+    B = qs[0].shape[0]
+    calls = (LayerCall * n)()
+    for i, pool in enumerate(pools):
+        q, bt, tg, out = qs[i], block_tables[i], tier_tags[i], outs[i]
+        assert q.dtype == torch.bfloat16 and q.is_contiguous() and q.shape == (B, pool.hq, pool.d)
+        assert bt.dtype == torch.int32 and bt.is_contiguous() and bt.shape == block_tables[0].shape and bt.shape[0] == B
+        assert tg.dtype == torch.uint8 and tg.is_contiguous() and tg.shape == bt.shape
+        assert out.dtype == torch.float32 and out.is_contiguous() and out.shape == (B, pool.hq, pool.d)
+        lse = None if lses is None else lses[i]
+        calls[i] = LayerCall(pool.handle, q.data_ptr(), bt.data_ptr(), tg.data_ptr(), out.data_ptr(),
+                             None if lse is None else lse.data_ptr(), pool.workspace.data_ptr())
+    assert seq_lens.dtype == torch.int32 and seq_lens.numel() == B
+    _check(lib().mkv_decode_attention_layers(calls, n, _ptr(seq_lens), B, block_tables[0].shape[1], float(scale),
+                                             pools[0].ws_bytes, _stream(stream)), "mkv_decode_attention_layers")
+    return outs
+
+
+def append_layers(pools, ks, vs, slot_mapping, stream=None):
+    """mkv_append_layers: Append of the same token positions into the pools of several layers in one launch."""
+    n = len(pools)
+    calls = (LayerAppend * n)()
+    for i, pool in enumerate(pools):
+        k, v = ks[i], vs[i]
+        assert k.dtype == torch.bfloat16 and v.dtype == torch.bfloat16 and k.is_contiguous() and v.is_contiguous()
+        assert k.shape == v.shape and k.shape[1:] == (pool.hkv, pool.d) and k.shape[0] == slot_mapping.numel()
+        calls[i] = LayerAppend(pool.handle, k.data_ptr(), v.data_ptr())
+    assert slot_mapping.dtype == torch.int32
+    _check(lib().mkv_append_layers(calls, n, _ptr(slot_mapping), slot_mapping.numel(), _stream(stream)), "mkv_append_layers")
 
 
 def page_score_update(page_mass, seq_lens, head_mask, beta, score, stream=None, page_tokens=16):

@@ -85,7 +85,16 @@ __global__ void __launch_bounds__(D) decode_scalar_kernel(
     float* sc = red + 256;                  // [16][8] scores
     float* gn = sc + 128;                   // [16] norm corrections
     const int tid = threadIdx.x, split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
-    const int hq = hkv * G, len = lens[b], n_pages = (len + kPage - 1) / kPage;
+    const int hq = hkv * G;
+    // a length beyond the table row is cut to the row and flagged, so that no entry past it is read
+    const long long cap = (long long)max_pages * tiles * kPage;
+    int len = lens[b];
+    if (len > cap) {
+        if (tid == 0) atomicOr(status, kStBounds);
+        len = (int)cap;
+    }
+    if (len < 0) len = 0;
+    const int n_pages = (len + kPage - 1) / kPage;
     const int per = (n_pages + n_splits - 1) / n_splits;
     const int lo = split * per, hi = min(n_pages, lo + per);
     const float C[4] = {MKV_C0, MKV_C1, MKV_C2, MKV_C3};

@@ -47,6 +47,11 @@ extern "C" int32_t mkv_decode_attention_static(mkv_pool* pool, const void* q, co
         mkv::set_last_error("mkv_decode_attention_static: the pool's device must be the current device");
         return MKV_E_INVALID;
     }
+    if (pool->variant != MKV_DECODE_TENSOR) {
+        // the fixed array is sized for the partials of the tensor-core scan; the other kernels keep theirs elsewhere
+        mkv::set_last_error("mkv_decode_attention_static: runs the tensor-core kernel only; set the pool's decode variant back to MKV_DECODE_TENSOR");
+        return MKV_E_INVALID;
+    }
     void* scratch = nullptr;
     {
         // first call on this device: resolve the device address of the array (no allocation happens)
@@ -61,10 +66,9 @@ extern "C" int32_t mkv_decode_attention_static(mkv_pool* pool, const void* q, co
     // Partial slots are written before they are read.  The ticket words behind them start at zero
     // (the array is zero-initialised when the module is loaded) and every call leaves them at zero.
     uint32_t* tickets = reinterpret_cast<uint32_t*>(static_cast<unsigned char*>(scratch) + kPartialBytes);
-    const int32_t rc = mkv::launch_decode_tensor_at(pool, q, bt, tags, lens, B, max_pages, scale, out, lse,
-                                                    static_cast<float*>(scratch), tickets, kStaticMaxBlocks,
-                                                    nullptr, (cudaStream_t)stream);
-    if (rc == MKV_E_INVALID)
-        mkv::set_last_error("mkv_decode_attention_static: this GPU launches more blocks than MKV_STATIC_MAX_BLOCKS allows");
-    return rc;
+    // A refusal keeps the reason the launch code recorded (a table wider than 65,535 tiles per row, more
+    // blocks than MKV_STATIC_MAX_BLOCKS partial slots, a device index out of range): mkv_last_cuda_error().
+    return mkv::launch_decode_tensor_at(pool, q, bt, tags, lens, B, max_pages, scale, out, lse,
+                                        static_cast<float*>(scratch), tickets, kStaticMaxBlocks, nullptr,
+                                        (cudaStream_t)stream);
 }

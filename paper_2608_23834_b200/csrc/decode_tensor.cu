@@ -29,6 +29,7 @@
 #include <math_constants.h>
 
 #include <cstdlib>
+#include <mutex>
 
 #include "mkv_internal.cuh"
 
@@ -38,6 +39,7 @@ constexpr int kMaxBatch = 1024;      // requests per call
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleSlack = 8.0f;   // running maximum is only raised when exceeded by 2^8
+constexpr unsigned long long kDefaultWaitNs = 20000000ull;   // 20 ms: far beyond any copy that is going to arrive
 
 size_t decode_ws_tensor_bytes(int, int, int, int d)
 {
@@ -64,6 +66,19 @@ struct DecodeParams {
     int max_blocks;        // the partial area holds 2 * max_blocks slots
     float* mass;           // scored variant: [B][hq][max_pages], log2-domain page sums from the scan (else unused)
     uint32_t* status;
+    unsigned long long wait_ns;   // wall-time limit of a wait for a page copy (kDefaultWaitNs unless the pool says otherwise)
+};
+
+// One launch can scan the pools of several layers (Section 4.1 runs the decode step of all full-attention
+// layers from one CUDA graph): the layers share the requests (lengths, batch, geometry) and differ in
+// their arenas, tables, queries, outputs and workspaces.  A block walks its share of layer 0, then of
+// layer 1, ... without waiting for the other blocks, so the start-up and the merge tail of one layer
+// overlap the page loops of its neighbours.
+constexpr int kMaxLayers = 32;
+template <int MAXL>
+struct LayerSet {
+    int n;
+    DecodeParams layer[MAXL];
 };
 
 // ------------------------------------------------------------------------------------------------
@@ -150,6 +165,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 {
     uint32_t ok;
     asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
                  : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
@@ -245,8 +268,7 @@ struct Partition {
 };
 
 // Called by warp 0 (all 32 lanes) after cum[] is complete; other warps wait at the next barrier.
-__device__ __forceinline__ void build_partition(Partition* pt, const int* cum, const int32_t* lens, int B, int hkv,
-                                                int grid, int lane)
+__device__ __forceinline__ void build_partition(Partition* pt, const int* cum, int B, int hkv, int grid, int lane)
 {
     constexpr uint32_t FULL = 0xffffffffu;
     const long long W = cum[B];
@@ -362,35 +384,12 @@ struct Geo {
     static constexpr int OFF_PART = OFF_L + NW * 8 * 4;
     static constexpr int OFF_LAST = OFF_PART + ((int)sizeof(Partition) + 15) / 16 * 16;
     static constexpr int SMEM = OFF_LAST + 16;
-    static_assert(NW >= 8, "one warp per column of the 8-wide head group builds the query fragments");
+    static_assert(NW >= 4, "a warp builds the query fragments of at most two columns of the 8-wide head group");
     static_assert(NSTAGE >= 2 && NSTAGE % 2 == 0 && NSTAGE <= 16, "an FP8 page takes a pair of slots; one phase bit per slot");
     static_assert(NSTAGE * SLOT >= 8 * D * 4, "ring doubles as the cross-warp reduction buffer");
     static_assert(FP8_HALF <= SLOT, "half an FP8 record fits a slot");
 };
 
-#ifdef MKV_TIMELINE
-// profiling build only: thread 0 of every block accumulates the time spent in each phase
-__device__ unsigned long long g_timeline[kMaxCtas * 16];
-__device__ unsigned long long g_warp_end[kMaxCtas * 32];   // per warp: time its page loops ended, pages it had (TQ3 << 32 | FP8)
-__device__ __forceinline__ unsigned long long tl_now()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-#define MKV_STAMP(k)                                                      \
-    do {                                                                  \
-        if (threadIdx.x == 0) {                                            \
-            const unsigned long long t__ = tl_now();                      \
-            if ((k) == 0) { g_timeline[blockIdx.x * 16 + 15] = t__; for (int z__ = 0; z__ < 15; ++z__) g_timeline[blockIdx.x * 16 + z__] = 0; } \
-            else g_timeline[blockIdx.x * 16 + (k)] += t__ - tl_last;       \
-            tl_last = t__;                                                \
-            g_timeline[blockIdx.x * 16 + 14] = t__;                        \
-        }                                                                 \
-    } while (0)
-#else
-#define MKV_STAMP(k)
-#endif
 
 // Running state of one warp for one (request, KV head) segment: O^T accumulators [d channels x 8
 // heads] in the MMA C layout, row sums and the (lazily raised) running maximum of the two head
@@ -782,8 +781,7 @@ __device__ __forceinline__ void merge_row(const DecodeParams& P, int first_slot,
             }
     };
     load_round(0);                           // in flight while the weights are worked out
-    if (warp < 8) {
-        const int hd = warp;
+    for (int hd = warp; hd < 8; hd += NT / 32) {
         float M = -CUDART_INF_F;
         for (int j = lane; j < n_parts; j += 32) {
             const float* ps = slot_of(j) + 8 * D;
@@ -832,13 +830,10 @@ __device__ __forceinline__ void merge_row(const DecodeParams& P, int first_slot,
         P.lse[(size_t)b * hq + h * GQ + tid] = ml_s[8 + tid] > 0.f ? (ml_s[tid] + log2f(ml_s[8 + tid])) * kLn2 : -CUDART_INF_F;
 }
 
-template <int D, int NW, int NSTAGE, int MINB, bool SCORED, bool TILED>
-__global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const DecodeParams P)
+template <int D, int NW, int NSTAGE, int MINB, bool SCORED, bool TILED, int MAXL>
+__global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const LayerSet<MAXL> LS)
 {
-#ifdef MKV_TIMELINE
-    unsigned long long tl_last = 0;
-#endif
-    MKV_STAMP(0);
+    const DecodeParams& P0 = LS.layer[0];    // requests and geometry are common to all layers
     using G = Geo<D, NW, NSTAGE, TILED>;     // pages of several tiles: short rounds leave room for the parked rows
     constexpr int NB = G::NB, NBH = NB, NU = NW;
     constexpr uint32_t FULL = 0xffffffffu;
@@ -854,26 +849,32 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tq = lane & 3;
     const int unit = warp, hf = 0;
-    const int hkv = P.hkv, GQ = P.group, hq = hkv * GQ;
+    const int hkv = P0.hkv, GQ = P0.group, hq = hkv * GQ;
+    const int n_layers = MAXL == 1 ? 1 : LS.n;
+    // a length beyond the table row is cut to the row (and flagged), so that no entry past it is ever read
+    const int len_cap = P0.max_pages * P0.tiles * kPage;
+    auto length_of = [&](int b) -> int {
+        const int len = P0.lens[b];
+        if (len > len_cap) {
+            atomicOr(P0.status, kStBounds);
+            return len_cap;
+        }
+        return len < 0 ? 0 : len;
+    };
 
-    // ---- prologue: barriers, zero rows of empty requests, prefix of pages, page strides ---------
+    // ---- prologue: barriers, prefix of pages, page strides ---------------------------------------
     if (tid == 0) {
         for (int i = 0; i < NW * NSTAGE; ++i) mbar_init(sbase + G::OFF_BAR + 8 * i, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        last_s[1] = 0;
     }
-    for (int b = blockIdx.x; b < P.B; b += gridDim.x)
-        if (P.lens[b] <= 0) {
-            for (int i = tid; i < hq * D; i += NW * 32) P.out[(size_t)b * hq * D + i] = 0.f;
-            if (P.lse)
-                for (int i = tid; i < hq; i += NW * 32) P.lse[(size_t)b * hq + i] = -CUDART_INF_F;
-        }
     if (warp == 0) {
         int run = 0;
-        for (int b0 = 0; b0 < P.B; b0 += 32) {
+        for (int b0 = 0; b0 < P0.B; b0 += 32) {
             const int b = b0 + lane;
             int n = 0;
-            if (b < P.B) {
-                const int len = P.lens[b];
+            if (b < P0.B) {
+                const int len = length_of(b);
                 n = len > 0 ? ((len + kPage - 1) / kPage) * hkv : 0;
             }
             int inc = n;
@@ -882,20 +883,18 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                 const int v = __shfl_up_sync(FULL, inc, o);
                 if (lane >= o) inc += v;
             }
-            if (b < P.B) cum[b] = run + inc - n;
+            if (b < P0.B) cum[b] = run + inc - n;
             run += __shfl_sync(FULL, inc, 31);
         }
-        if (lane == 0) cum[P.B] = run;
+        if (lane == 0) cum[P0.B] = run;
         __syncwarp();
-        MKV_STAMP(9);
-        build_partition(pt, cum, P.lens, P.B, hkv, gridDim.x, lane);
-        MKV_STAMP(10);
+        build_partition(pt, cum, P0.B, hkv, gridDim.x, lane);
     } else {
         // Pages of a row are visited in a strided order, page(i) = i * stride mod n_pages, the stride
         // coprime to n_pages and near 0.618 n_pages: every contiguous range of positions then holds the
         // row's FP8 and TQ3 pages in their overall proportion, so equal ranges cost equal time.
-        for (int b = tid - 32; b < P.B; b += NW * 32 - 32) {
-            const int len = P.lens[b], n = (len + kPage - 1) / kPage;
+        for (int b = tid - 32; b < P0.B; b += NW * 32 - 32) {
+            const int len = length_of(b), n = (len + kPage - 1) / kPage;
             int st = (int)((float)n * 0.6180339f);
             if (st < 1) st = 1;
             if constexpr (TILED) st = 1;          // consecutive tiles: a warp's run stays inside one or two pages
@@ -908,10 +907,8 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
         }
     }
     __syncthreads();
-    MKV_STAMP(11);
-    if ((int)blockIdx.x >= pt->blocks) return;             // more blocks than work
-    int my_start, my_end;
-    partition_range(pt, cum, hkv, P.B, blockIdx.x, my_start, my_end);
+    int my_start = 0, my_end = 0;                          // more blocks than work: an empty range
+    if ((int)blockIdx.x < pt->blocks) partition_range(pt, cum, hkv, P0.B, blockIdx.x, my_start, my_end);
 
     // per-warp ring of NSTAGE slots; one bit per slot holds the mbarrier phase the next wait must see
     uint32_t phase = 0;
@@ -923,37 +920,65 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
     int* list8 = list3 + G::ROUND;                                                   // FP8 page ids | valid << 27
     int* lpg3 = reinterpret_cast<int*>(smem + G::OFF_LIST) + (NW + warp) * 2 * G::ROUND;   // their logical pages (scored variant)
     int* lpg8 = lpg3 + G::ROUND;
-    const float sc2 = P.scale * kLog2e;      // scores are kept in log2 units
-    // bounded wait for ring slot s, then flip its expected phase
-    auto wait_slot = [&](uint32_t s) {
+    const float sc2 = P0.scale * kLog2e;     // scores are kept in log2 units
+    uint32_t pending = 0;                    // ring slots with a copy in flight that nobody has waited for yet
+    // Bounded wait for ring slot s, then flip its expected phase.  `limit_ns` of wall time (the pool's wait
+    // limit, 20 ms by default); returns false when it ran out.
+    auto wait_bounded = [&](uint32_t s, unsigned long long limit_ns) -> bool {
         const uint32_t bar = bars + 8 * s, parity = (phase >> s) & 1u;
-        phase ^= 1u << s;
-        if (!mbar_try_wait(bar, parity)) {
-            // give up after ~20 ms of wall time: flag the pool's status word and skip the remaining pages
+        // limit 0 (diagnostic): one look without blocking, so that a copy still in flight counts as late
+        bool ok = limit_ns == 0 ? mbar_test_wait(bar, parity) : mbar_try_wait(bar, parity);
+        if (!ok && limit_ns != 0) {
             unsigned long long t0, t1;
             asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
-            int spins = 0;
-            while (!mbar_try_wait(bar, parity)) {
-                if ((++spins & 255) == 0) {
+            for (int spins = 1; !ok; ++spins) {
+                ok = mbar_try_wait(bar, parity);
+                if (!ok && (spins & 255) == 0) {
                     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
-                    if (t1 - t0 > 20000000ull) {
-                        failed = true;
-                        atomicOr(P.status, kStTimeout);
-                        break;
-                    }
+                    if (t1 - t0 >= limit_ns) break;
                 }
             }
         }
-        failed = __any_sync(FULL, failed);
+        ok = __all_sync(FULL, ok);           // the copy has landed for every lane, or the warp gives up as one
+        if (ok) {
+            phase ^= 1u << s;
+            pending &= ~(1u << s);
+        }
+        return ok;
     };
+    // After a wait has run out the warp stops scanning; before anybody reuses the ring (as the reduction
+    // buffer) or the block leaves, every copy this warp still has in flight is waited for with the
+    // default limit, so that nothing lands in memory that has changed hands.
+    auto drain = [&]() {
+        bool lost = false;
+#pragma unroll 1
+        for (uint32_t s = 0; s < (uint32_t)NSTAGE; ++s)
+            if (pending & (1u << s)) lost |= !wait_bounded(s, kDefaultWaitNs);
+        return lost;
+    };
+
+    for (int layer = 0; layer < n_layers; ++layer) {
+    const DecodeParams& P = LS.layer[MAXL == 1 ? 0 : layer];
+    auto wait_slot = [&](uint32_t s) {
+        if (!wait_bounded(s, P.wait_ns)) {
+            failed = true;
+            atomicOr(P.status, kStTimeout);
+        }
+    };
+    // rows of empty requests
+    for (int b = blockIdx.x; b < P.B; b += gridDim.x)
+        if (P.lens[b] <= 0) {
+            for (int i = tid; i < hq * D; i += NW * 32) P.out[(size_t)b * hq * D + i] = 0.f;
+            if (P.lse)
+                for (int i = tid; i < hq; i += NW * 32) P.lse[(size_t)b * hq + i] = -CUDART_INF_F;
+        }
 
     int pos = my_start;
     int b = 0;
-    MKV_STAMP(1);
     while (pos < my_end) {
         // ---- locate the segment: request b, KV head h, positions [pg0, pg0 + n_seg) of the row ------
         while (cum[b + 1] <= pos) ++b;
-        const int len = P.lens[b], n_pages = (len + kPage - 1) / kPage;
+        const int len = min(max(P.lens[b], 0), len_cap), n_pages = (len + kPage - 1) / kPage;
         const int h = (pos - cum[b]) / n_pages, pg0 = (pos - cum[b]) % n_pages;
         const int row_start = cum[b] + h * n_pages, row_end = row_start + n_pages;
         const int n_seg = min(my_end, row_end) - pos;
@@ -965,10 +990,15 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
         const int n_my = (int)(((unsigned)n_seg * (unsigned)(warp + 1)) / NW) - warp_first;
         const int stride = strides[b];
         constexpr int EPL = D / 32;
-        float qx[EPL];            // this warp's query head (warps 0..7), loaded before anything else waits
+        constexpr int HPW = (8 + NW - 1) / NW;      // query heads a warp prepares (head warp, warp + NW, ...)
+        float qx[HPW][EPL];       // loaded before anything else waits
 #pragma unroll
-        for (int r = 0; r < EPL; ++r)
-            qx[r] = (warp < GQ) ? __bfloat162float(P.q[((size_t)b * hq + h * GQ + warp) * D + lane * EPL + r]) : 0.f;
+        for (int k = 0; k < HPW; ++k)
+#pragma unroll
+            for (int r = 0; r < EPL; ++r) {
+                const int hd = warp + k * NW;
+                qx[k][r] = (hd < GQ) ? __bfloat162float(P.q[((size_t)b * hq + h * GQ + hd) * D + lane * EPL + r]) : 0.f;
+            }
         float* mass_row = SCORED ? P.mass + ((size_t)b * hq + (size_t)h * GQ) * P.max_pages : nullptr;
         const uint8_t* tq3_base = P.tq3 + (size_t)h * G::TQ3_REC;
         const uint8_t* fp8_base = P.fp8 + (size_t)h * (2 * G::FP8_HALF);
@@ -1014,6 +1044,7 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
             __syncwarp();
         };
         auto issue_tq3 = [&](int i) {      // copy Stale page i of the round into ring slot i % NSTAGE
+            pending |= 1u << ((uint32_t)i % NSTAGE);
             if (lane == 0) {
                 const uint32_t s = (uint32_t)i % NSTAGE;
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -1029,6 +1060,7 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
             }
         };
         auto issue_fp8 = [&](int i) {      // copy FP8 page i of the round into the slot pair 2 (i % (NSTAGE/2))
+            pending |= 3u << ((uint32_t)(2 * i) % NSTAGE);
             if (lane == 0) {
                 const uint32_t s = (uint32_t)(2 * i) % NSTAGE;
                 const int e8 = list8[i] & 0x7FFFFFF;
@@ -1046,9 +1078,6 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
             }
         };
 
-#ifdef MKV_TIMELINE
-        int tl_n3 = 0, tl_n8 = 0;
-#endif
         WarpAcc<NB> acc;
         // Pages of several tiles.  While the scan is inside a Stale page, acc.o holds sum p * code and the
         // output gathered before waits in this warp's shared-memory rows ("parked"); leaving the page adds
@@ -1107,14 +1136,16 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
             for (int i = 0; i < min(n3, NSTAGE); ++i) issue_tq3(i);
         }
 
-        // query fragments: warp hd < 8 rotates head hd (loads were issued before the copies started)
-        if (warp < 8) {
-            const int hd = warp;
+        // query fragments: a warp rotates head `warp` (and `warp + NW`); loads were issued before the copies started
+#pragma unroll
+        for (int k = 0; k < HPW; ++k) {
+            const int hd = warp + k * NW;
+            if (hd >= 8) break;
             float a[EPL];
 #pragma unroll
             for (int r = 0; r < EPL; ++r) {
                 const int i = lane * EPL + r;
-                a[r] = ((P.sigma.w[i >> 5] >> (i & 31)) & 1u) ? -qx[r] : qx[r];
+                a[r] = ((P.sigma.w[i >> 5] >> (i & 31)) & 1u) ? -qx[k][r] : qx[k][r];
             }
 #pragma unroll
             for (int hh = 1; hh < EPL; hh <<= 1)
@@ -1149,21 +1180,17 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                 }
                 {   // plain query in the slot order of the FP8 key loads: 16 consecutive dims per lane
                     const int j = i >> 6, t4 = (i & 63) >> 4, wv = (i & 15) >> 2, e = i & 3;
-                    qf[((4 * j + wv) * 32 + 4 * hd + t4) * 4 + (e >> 1) * 2 + (e & 1)] = __float2half_rn(qx[r]);
+                    qf[((4 * j + wv) * 32 + 4 * hd + t4) * 4 + (e >> 1) * 2 + (e & 1)] = __float2half_rn(qx[k][r]);
                 }
             }
         }
         __syncthreads();
-        MKV_STAMP(2);
 
         for (int round = 0; round < n_rounds && !failed; ++round) {
             if (round > 0) {
                 build_lists(round);
                 for (int i = 0; i < min(n3, NSTAGE); ++i) issue_tq3(i);
             }
-#ifdef MKV_TIMELINE
-            tl_n3 += n3; tl_n8 += n8;
-#endif
             // ---- Stale pages: scores of page i+1 are computed together with the output update of page i
             if (n3 > 0) {
                 float s_cur[4], s_next[4];
@@ -1235,16 +1262,9 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
         float (&m_run)[2] = acc.m;
 
         // ---- combine the warps of the block (ring memory is idle now) ---------------------------
-#ifdef MKV_TIMELINE
-        if (lane == 0 && warp < 16) {
-            g_warp_end[blockIdx.x * 32 + warp] = tl_now();
-            g_warp_end[blockIdx.x * 32 + 16 + warp] = ((unsigned long long)tl_n3 << 32) | (unsigned)tl_n8;
-            if (warp == 0) { unsigned sm__; asm volatile("mov.u32 %0, %%smid;" : "=r"(sm__)); g_warp_end[blockIdx.x * 32 + 15] = sm__; }
-        }
-#endif
-        MKV_STAMP(3);
+        if (failed && drain()) last_s[1] = 1;      // a copy never arrived at all: the block must not touch the ring
         __syncthreads();
-        MKV_STAMP(4);
+        if (last_s[1]) return;                     // (the call has failed; its workspace needs mkv_workspace_init again)
         if (g == 0 && hf == 0) {           // both warps of a unit hold the same maximum and row sums
             sm_m[unit * 8 + 2 * tq] = m_run[0];
             sm_m[unit * 8 + 2 * tq + 1] = m_run[1];
@@ -1273,7 +1293,6 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
         }
         __syncthreads();
 
-        MKV_STAMP(5);
         const bool whole_row = (pos == row_start) && (pos + n_seg == row_end);
         if (whole_row) {
             for (int e = tid; e < 8 * D; e += NW * 32) {
@@ -1314,99 +1333,135 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Deco
                 slot[8 * D + tid] = M;
                 slot[8 * D + 8 + tid] = l;
             }
-            // ticket of the row: the block that draws the last one merges (its loads then see every
-            // other block's partial: store -> fence -> ticket on their side, ticket -> fence -> load here)
+            // Ticket of the row (store -> fence -> ticket on the writers' side, ticket -> fence -> load on the
+            // merger's).  Who merges?  In the last layer of the launch the block that draws the row's last
+            // ticket.  In an earlier layer the row is left to the block that is FIRST to finish the same row in
+            // the next layer -- the one that is ahead of the others, so that the merges do not keep falling on
+            // the block that is already late.  That block finds the row complete and merges it, or it leaves a
+            // request (the counter's top bit) and the row's last arrival, seeing the request, merges after all.
+            // Either way exactly one block merges, and it leaves the counter at zero for the next call.
             int c0, c1;
             partition_blocks_of_row(pt, cum, P.B, b * hkv + h, row_start, row_end, c0, c1);
             const int n_parts = c1 - c0 + 1;
+            constexpr uint32_t kRequest = 0x80000000u;
             __syncthreads();
             if (tid == 0) {
                 __threadfence();
                 const uint32_t prev = atomicAdd(P.tickets + c0, 1u);
-                const int last = prev == (uint32_t)(n_parts - 1);
-                if (last) P.tickets[c0] = 0;           // leave the counter cleared for the next call
-                *last_s = last;
+                int todo = 0;                          // 1: merge this layer's row, 2: merge the row of the layer before
+                if ((prev & ~kRequest) == (uint32_t)(n_parts - 1) && (layer == n_layers - 1 || (prev & kRequest))) todo |= 1;
+                if (MAXL > 1 && layer > 0 && (prev & ~kRequest) == 0u) {
+                    const uint32_t old = atomicOr(LS.layer[layer - 1].tickets + c0, kRequest);
+                    if (old == (uint32_t)n_parts) todo |= 2;
+                }
+                *last_s = todo;
             }
             __syncthreads();
-            if (*last_s) {
+            const int todo = *last_s;
+            if (todo) {
                 __threadfence();
-                MKV_STAMP(6);
                 const int first_slot = 2 * c0 + (row_start > partition_start(pt, cum, hkv, P.B, c0) ? 1 : 0);
-                merge_row<D, NW * 32>(P, first_slot, 2 * c0, n_parts, red, b, h);
-                MKV_STAMP(7);
+                if constexpr (MAXL > 1) {
+                    if (todo & 2) {
+                        const DecodeParams& Q = LS.layer[layer - 1];
+                        merge_row<D, NW * 32>(Q, first_slot, 2 * c0, n_parts, red, b, h);
+                        if (tid == 0) Q.tickets[c0] = 0;
+                    }
+                }
+                if (todo & 1) {
+                    merge_row<D, NW * 32>(P, first_slot, 2 * c0, n_parts, red, b, h);
+                    if (tid == 0) P.tickets[c0] = 0;
+                }
             }
         }
         __syncthreads();
-        MKV_STAMP(8);
         pos += n_seg;
     }
+    }   // layers
 }
 
 #include "decode_tmem.cuh"
+
+// Per-device launch state of one kernel instantiation (dynamic shared memory opt-in, persistent grid size).
+constexpr int kMaxDevices = 64;
+struct LaunchCache {
+    std::mutex mu;
+    int grid[kMaxDevices] = {};
+};
 
 template <int D>
 static int32_t run_tmem(mkv_pool* p, DecodeParams& prm, cudaStream_t s)
 {
     using G = tm::TG<D>;
     auto kern = decode_tmem_kernel<D>;
-    static bool attr_done[8] = {false, false, false, false, false, false, false, false};
-    const int dev = p->device & 7;
-    if (!attr_done[dev]) {
-        MKV_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM));
-        attr_done[dev] = true;
+    static LaunchCache cache;
+    const int dev = p->device;
+    if (dev < 0 || dev >= kMaxDevices) {
+        set_last_error("decode attention: device index beyond the 64 this library keeps launch state for");
+        return MKV_E_INVALID;
     }
-    const int grid = p->dev.sm_count > kMaxCtas ? kMaxCtas : p->dev.sm_count;     // one block per SM: it takes all the tensor memory
-    if (grid > prm.max_blocks) return MKV_E_INVALID;
+    int grid;
+    {
+        std::lock_guard<std::mutex> lk(cache.mu);
+        if (cache.grid[dev] == 0) {
+            MKV_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM));
+            cache.grid[dev] = p->dev.sm_count > kMaxCtas ? kMaxCtas : p->dev.sm_count;   // one block per SM: it takes all the tensor memory
+        }
+        grid = cache.grid[dev];
+    }
+    if (grid > prm.max_blocks) {
+        set_last_error("decode attention: the scan launches more blocks on this GPU than the partial area has slots for");
+        return MKV_E_INVALID;
+    }
     kern<<<grid, tm::kThreads, G::SMEM, s>>>(prm);
     MKV_CUDA(cudaGetLastError());
     return MKV_OK;
 }
 
-template <int D, int NW, int NSTAGE, int MINB, bool SCORED = false, bool TILED = false>
-static int32_t run_tensor(mkv_pool* p, DecodeParams& prm, cudaStream_t s)
+template <int D, int NW, int NSTAGE, int MINB, bool SCORED = false, bool TILED = false, int MAXL = 1>
+static int32_t run_tensor(mkv_pool* p, const LayerSet<MAXL>& ls, cudaStream_t s)
 {
     using G = Geo<D, NW, NSTAGE, TILED>;
-    auto kern = decode_tensor_kernel<D, NW, NSTAGE, MINB, SCORED, TILED>;
+    auto kern = decode_tensor_kernel<D, NW, NSTAGE, MINB, SCORED, TILED, MAXL>;
     // pages of several tiles: one row of parked accumulators (8 D floats) per warp behind the usual layout
     constexpr int SMEM = G::SMEM + (TILED ? NW * 8 * D * 4 : 0);
     static_assert(SMEM <= 232448, "dynamic shared memory of one block");
-    static int grid_cache[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    int dev = p->device & 7;
-    if (grid_cache[dev] == 0) {
-        MKV_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM));
-        int per_sm = 0;
-        MKV_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, NW * 32, SMEM));
-        if (per_sm < 1) return MKV_E_INVALID;
-        int grid = p->dev.sm_count * per_sm;
-        grid_cache[dev] = grid > kMaxCtas ? kMaxCtas : grid;
+    static LaunchCache cache;
+    const int dev = p->device;
+    if (dev < 0 || dev >= kMaxDevices) {
+        set_last_error("decode attention: device index beyond the 64 this library keeps launch state for");
+        return MKV_E_INVALID;
     }
-    if (grid_cache[dev] > prm.max_blocks) return MKV_E_INVALID;
-    kern<<<grid_cache[dev], NW * 32, SMEM, s>>>(prm);
+    int grid;
+    {
+        std::lock_guard<std::mutex> lk(cache.mu);
+        if (cache.grid[dev] == 0) {
+            MKV_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM));
+            int per_sm = 0;
+            MKV_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, NW * 32, SMEM));
+            if (per_sm < 1) return MKV_E_INVALID;
+            const int g = p->dev.sm_count * per_sm;
+            cache.grid[dev] = g > kMaxCtas ? kMaxCtas : g;
+        }
+        grid = cache.grid[dev];
+    }
+    if (grid > ls.layer[0].max_blocks) {
+        set_last_error("decode attention: the scan launches more blocks on this GPU than the partial area has slots for");
+        return MKV_E_INVALID;
+    }
+    kern<<<grid, NW * 32, SMEM, s>>>(ls);
     MKV_CUDA(cudaGetLastError());
     return MKV_OK;
 }
 
-// launch shape: warps per block, ring slots per warp, blocks per SM the register budget is sized for
-static int tensor_shape()
+template <int D, int NW, int NSTAGE, int MINB, bool SCORED = false, bool TILED = false>
+static int32_t run_tensor1(mkv_pool* p, const DecodeParams& prm, cudaStream_t s)
 {
-    static int shape = -1;
-    if (shape < 0) {
-        const char* e = getenv("MKV_DECODE_SHAPE");
-        shape = e ? atoi(e) : 0;
-    }
-    return shape;
+    LayerSet<1> ls;
+    ls.n = 1;
+    ls.layer[0] = prm;
+    return run_tensor<D, NW, NSTAGE, MINB, SCORED, TILED, 1>(p, ls, s);
 }
-
-#ifdef MKV_TIMELINE
-extern "C" int mkv_debug_timeline(unsigned long long* host, int n)
-{
-    return (int)cudaMemcpyFromSymbol(host, g_timeline, sizeof(unsigned long long) * n);
-}
-extern "C" int mkv_debug_warp_end(unsigned long long* host, int n)
-{
-    return (int)cudaMemcpyFromSymbol(host, g_warp_end, sizeof(unsigned long long) * n);
-}
-#endif
 
 int32_t launch_decode_tensor(mkv_pool* p, const void* q, const int32_t* bt, const uint8_t* tags,
                              const int32_t* lens, int B, int max_pages, float scale, float* out, float* lse,
@@ -1430,7 +1485,7 @@ __global__ void __launch_bounds__(256) page_mass_finish_kernel(float* mass, cons
 {
     __shared__ float red[8];
     const int b = blockIdx.y, h = blockIdx.x, tid = threadIdx.x;
-    const int len = lens[b], n_pages = len > 0 ? (len + page_tokens - 1) / page_tokens : 0;
+    const int len = lens[b], n_pages = len > 0 ? min((len + page_tokens - 1) / page_tokens, max_pages) : 0;
     float* row = mass + ((size_t)b * hq + h) * max_pages;
     const float lse2 = n_pages > 0 ? lse[(size_t)b * hq + h] * kLog2e : 0.f;
     float sum = 0.f;
@@ -1456,7 +1511,7 @@ __global__ void __launch_bounds__(256) page_score_kernel(const float* mass, cons
                                                          float* score, int page_tokens)
 {
     const int b = blockIdx.y, p = blockIdx.x * 256 + threadIdx.x;
-    const int len = lens[b], n_pages = len > 0 ? (len + page_tokens - 1) / page_tokens : 0;
+    const int len = lens[b], n_pages = len > 0 ? min((len + page_tokens - 1) / page_tokens, max_pages) : 0;
     if (p >= n_pages) return;
     float r = 0.f;
     for (int h = 0; h < hq; ++h)
@@ -1492,19 +1547,10 @@ int32_t launch_page_score(const float* mass, const int32_t* lens, int B, int hq,
     return MKV_OK;
 }
 
-int32_t launch_decode_tensor_at(mkv_pool* p, const void* q, const int32_t* bt, const uint8_t* tags,
-                                const int32_t* lens, int B, int max_pages, float scale, float* out, float* lse,
-                                float* partials, uint32_t* tickets, int max_blocks, float* mass, cudaStream_t s)
+static DecodeParams make_params(mkv_pool* p, const void* q, const int32_t* bt, const uint8_t* tags, const int32_t* lens,
+                                int B, int max_pages, float scale, float* out, float* lse, float* partials,
+                                uint32_t* tickets, int max_blocks, float* mass)
 {
-    if (B > kMaxBatch) return MKV_E_INVALID;
-    if ((int64_t)max_pages * p->tiles > 65535) {   // the strided order multiplies two 16-token tile indices in 32 bits
-        set_last_error("mkv_decode_attention: more than 65535 16-token tiles per table row (1,048,560 tokens per request)");
-        return MKV_E_INVALID;
-    }
-    if (p->tiles > 1 && p->variant == MKV_DECODE_TMEM) {
-        set_last_error("mkv_decode_attention: pages of several tiles are served by the tensor-core kernel");
-        return MKV_E_INVALID;
-    }
     DecodeParams prm;
     prm.tiles = p->tiles;
     prm.fp8 = p->fp8; prm.tq3 = p->tq3;
@@ -1521,36 +1567,75 @@ int32_t launch_decode_tensor_at(mkv_pool* p, const void* q, const int32_t* bt, c
     prm.max_blocks = max_blocks;
     prm.mass = mass;
     prm.status = p->status_dev;
+    prm.wait_ns = p->wait_ns;
+    return prm;
+}
+
+// Decode attention of several layers in one launch: layer i reads pool[i], q[i], bt[i], tags[i] and writes
+// out[i], lse[i] (or none), with its own workspace ws[i]; the requests (lens, B, max_pages, scale) are common.
+int32_t launch_decode_tensor_layers(mkv_pool* const* pools, const void* const* q, const int32_t* const* bt,
+                                    const uint8_t* const* tags, const int32_t* lens, int B, int max_pages, float scale,
+                                    float* const* out, float* const* lse, void* const* ws, int n_layers, cudaStream_t s)
+{
+    mkv_pool* p0 = pools[0];
+    if (B > kMaxBatch || n_layers > kMaxLayers) return MKV_E_INVALID;
+    if ((int64_t)max_pages * p0->tiles > 65535) {
+        set_last_error("mkv_decode_attention_layers: more than 65535 16-token tiles per table row (1,048,560 tokens per request)");
+        return MKV_E_INVALID;
+    }
+    if (p0->tiles > 1) {
+        set_last_error("mkv_decode_attention_layers: pages of 16 tokens only");
+        return MKV_E_INVALID;
+    }
+    LayerSet<kMaxLayers> ls;
+    ls.n = n_layers;
+    for (int i = 0; i < n_layers; ++i) {
+        uint32_t* tickets = reinterpret_cast<uint32_t*>(static_cast<uint8_t*>(ws[i]) + 256);
+        float* partials = reinterpret_cast<float*>(static_cast<uint8_t*>(ws[i]) + decode_ws_header_bytes(B, p0->hkv));
+        ls.layer[i] = make_params(pools[i], q[i], bt[i], tags[i], lens, B, max_pages, scale, out[i], lse ? lse[i] : nullptr,
+                                  partials, tickets, kMaxCtas, nullptr);
+    }
+#ifdef MKV_SHAPE_2X4
+    return p0->d == 128 ? run_tensor<128, 12, 4, 1, false, false, kMaxLayers>(p0, ls, s)
+                        : run_tensor<256, 4, 4, 2, false, false, kMaxLayers>(p0, ls, s);
+#endif
+    return p0->d == 128 ? run_tensor<128, 12, 4, 1, false, false, kMaxLayers>(p0, ls, s)
+                        : run_tensor<256, 8, 4, 1, false, false, kMaxLayers>(p0, ls, s);
+}
+
+int32_t launch_decode_tensor_at(mkv_pool* p, const void* q, const int32_t* bt, const uint8_t* tags,
+                                const int32_t* lens, int B, int max_pages, float scale, float* out, float* lse,
+                                float* partials, uint32_t* tickets, int max_blocks, float* mass, cudaStream_t s)
+{
+    if (B > kMaxBatch) return MKV_E_INVALID;
+    if ((int64_t)max_pages * p->tiles > 65535) {   // the strided order multiplies two 16-token tile indices in 32 bits
+        set_last_error("mkv_decode_attention: more than 65535 16-token tiles per table row (1,048,560 tokens per request)");
+        return MKV_E_INVALID;
+    }
+    if (p->tiles > 1 && p->variant == MKV_DECODE_TMEM) {
+        set_last_error("mkv_decode_attention: pages of several tiles are served by the tensor-core kernel");
+        return MKV_E_INVALID;
+    }
+    DecodeParams prm = make_params(p, q, bt, tags, lens, B, max_pages, scale, out, lse, partials, tickets, max_blocks, mass);
     if (mass) {                          // scored variant: the default launch shapes only
         int32_t rc;
         if (p->tiles > 1) {
             const size_t n = (size_t)B * p->hkv * p->group * max_pages;
             page_mass_clear_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(mass, n);
             MKV_CUDA(cudaGetLastError());
-            rc = p->d == 128 ? run_tensor<128, 12, 4, 1, true, true>(p, prm, s) : run_tensor<256, 8, 4, 1, true, true>(p, prm, s);
+            rc = p->d == 128 ? run_tensor1<128, 12, 4, 1, true, true>(p, prm, s) : run_tensor1<256, 8, 4, 1, true, true>(p, prm, s);
         } else {
-            rc = p->d == 128 ? run_tensor<128, 12, 4, 1, true>(p, prm, s) : run_tensor<256, 8, 4, 1, true>(p, prm, s);
+            rc = p->d == 128 ? run_tensor1<128, 12, 4, 1, true>(p, prm, s) : run_tensor1<256, 8, 4, 1, true>(p, prm, s);
         }
         if (rc != MKV_OK) return rc;
         return launch_page_mass_finish(mass, lse, lens, B, p->hkv * p->group, max_pages, p->cfg.page_size, s);
     }
     if (p->tiles > 1)                    // pages of several tiles: the default launch shapes only
-        return p->d == 128 ? run_tensor<128, 12, 4, 1, false, true>(p, prm, s) : run_tensor<256, 8, 4, 1, false, true>(p, prm, s);
+        return p->d == 128 ? run_tensor1<128, 12, 4, 1, false, true>(p, prm, s) : run_tensor1<256, 8, 4, 1, false, true>(p, prm, s);
     if (p->variant == MKV_DECODE_TMEM && p->d == 256) return run_tmem<256>(p, prm, s);
-    // Launch shapes (warps per block, ring slots per warp, blocks per SM); MKV_DECODE_SHAPE selects the
-    // alternatives for profiling.
-    const int shape = tensor_shape();
-    if (p->d == 128) {
-        switch (shape) {
-        case 1: return run_tensor<128, 16, 4, 1>(p, prm, s);
-        case 2: return run_tensor<128, 8, 4, 1>(p, prm, s);
-        default: return run_tensor<128, 12, 4, 1>(p, prm, s);     // 168 registers: 7 % faster than 16 warps at 128; 10, 11, 13, 14 warps are slower
-        }
-    }
-    switch (shape) {
-    case 2: return run_tensor<256, 10, 4, 1>(p, prm, s);
-    default: return run_tensor<256, 8, 4, 1>(p, prm, s);     // a ring of 6 slots per warp no longer fits beside the page lists
-    }
+    // launch shapes (warps per block, ring slots per warp, blocks per SM): 12 warps at 168 registers for
+    // d = 128 (7 % faster than 16 warps at 128 registers), 8 warps for d = 256
+    return p->d == 128 ? run_tensor1<128, 12, 4, 1>(p, prm, s) : run_tensor1<256, 8, 4, 1>(p, prm, s);
 }
 
 }  // namespace mkv

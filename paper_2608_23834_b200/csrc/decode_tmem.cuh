@@ -210,7 +210,8 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
             const int b = b0 + lane;
             int n = 0;
             if (b < P.B) {
-                const int len = P.lens[b];
+                int len = P.lens[b];
+                if (len > P.max_pages * kPage) { atomicOr(P.status, kStBounds); len = P.max_pages * kPage; }   // a length beyond the table row is cut and flagged
                 n = len > 0 ? ((len + kPage - 1) / kPage) * hkv : 0;
             }
             int inc = n;
@@ -224,10 +225,10 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
         }
         if (lane == 0) cum[P.B] = run;
         __syncwarp();
-        build_partition(pt, cum, P.lens, P.B, hkv, gridDim.x, lane);
+        build_partition(pt, cum, P.B, hkv, gridDim.x, lane);
     } else {
         for (int b = tid - 32; b < P.B; b += NT - 32) {
-            const int len = P.lens[b], n = (len + kPage - 1) / kPage;
+            const int len = min(max(P.lens[b], 0), P.max_pages * kPage), n = (len + kPage - 1) / kPage;
             int st = (int)((float)n * 0.6180339f);
             if (st < 1) st = 1;
             for (; n > 1; ++st) {
@@ -285,18 +286,11 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
         for (int s = 0; s < kTile; ++s) wait_bar(kBarFull + rb * kTile + s, par);
     };
 
-#ifdef MKV_TIMELINE
-    long long tl_acc[4] = {0, 0, 0, 0}, tl_last = clock64();
-    const long long tl_begin = tl_last;
-#define TS(k) do { const long long t__ = clock64(); tl_acc[k] += t__ - tl_last; tl_last = t__; } while (0)
-#else
-#define TS(k)
-#endif
     int pos = my_start;
     int b = 0;
     while (pos < my_end) {
         while (cum[b + 1] <= pos) ++b;
-        const int len = P.lens[b], n_pages = (len + kPage - 1) / kPage;
+        const int len = min(max(P.lens[b], 0), P.max_pages * kPage), n_pages = (len + kPage - 1) / kPage;
         const int h = (pos - cum[b]) / n_pages, pg0 = (pos - cum[b]) % n_pages;
         const int row_start = cum[b] + h * n_pages, row_end = row_start + n_pages;
         const int n_seg = min(my_end, row_end) - pos;
@@ -396,9 +390,7 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
                         bool stale; int first, np;
                         tile_info(ti, stale, first, np);
                         const uint32_t t = tcount + ti, rb = t % kRing;
-                        TS(3);
                         if (t >= kRing) wait_bar(kBarTileFree + rb, ((t / kRing) - 1) & 1);
-                        TS(0);
                         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                         const uint32_t dst = sbase + rb * kTile * G::SLOT;
                         for (int s = 0; s < kTile; ++s) {
@@ -425,11 +417,8 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
                     bool stale; int first, np;
                     tile_info(ti, stale, first, np);
                     const uint32_t t = tcount + ti, kb2 = t & 1, par = (t >> 1) & 1;
-                    TS(3);
                     wait_bar(kBarKReady + kb2, par);
-                    TS(0);
                     if (t >= 2) wait_bar(kBarSFree + kb2, ((t >> 1) - 1) & 1);
-                    TS(1);
                     tc_fence_after();
                     if (lane == 0) {
                         const uint32_t qtile = sbase + (stale ? G::OFF_QT : G::OFF_QF);
@@ -447,17 +436,12 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
                     bool stale; int first, np;
                     tile_info(ti, stale, first, np);
                     const uint32_t t = tcount + ti, pb = t & 1;
-                    TS(3);
                     wait_bar(kBarPReady + pb, (t >> 1) & 1);
-                    TS(0);
                     const int nb = (np + 1) / 2;
                     for (int bi = 0; bi < nb; ++bi, ++bc) {
                         const uint32_t vb = bc & 1, tbuf = bc % kTBuf;
-                        TS(3);
                         wait_bar(kBarVReady + vb, (bc >> 1) & 1);
-                        TS(1);
                         if (bc >= kTBuf) wait_bar(kBarTFree + tbuf, ((bc / kTBuf) - 1) & 1);
-                        TS(2);
                         tc_fence_after();
                         if (lane == 0) {
 #pragma unroll 1
@@ -481,11 +465,8 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
                     tile_info(ti, stale, first, np);
                     const uint32_t t = tcount + ti, rb = t % kRing, kb2 = t & 1;
                     const uint32_t tile = sbase + rb * kTile * G::SLOT;
-                    TS(3);
                     wait_tile(t);
-                    TS(0);
                     if (t >= 1) wait_bar(kBarSFull + ((t - 1) & 1), ((t - 1) >> 1) & 1);      // the score products of the tile before have read it
-                    TS(1);
                     tc_fence_after();
 #pragma unroll 1
                     for (int e = 0; e < 2; ++e) {
@@ -550,14 +531,11 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
                     int valid = kPage;
                     if (!stale && p_me < np) { const int v = (list8[first + p_me] >> 27) & 15; valid = v ? v : kPage; }
                     const bool live = p_me < np && tok < valid;
-                    TS(3);
                     wait_tile(t);
-                    TS(0);
                     float rsc = sc2 * P.k_scale;
                     if (stale) rsc = __half2float(__ushort_as_half(lds16(tile + (p_me < np ? p_me : 0) * G::SLOT + 12 * D + 2 * tok))) * sc2;
                     warp_arrive(kBarTileFree + rb);
                     wait_bar(kBarSFull + sb, par);
-                    TS(1);
                     tc_fence_after();
                     float s[8];
                     {
@@ -607,9 +585,7 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
                     }
                     bar_sync(1, 128);                        // flags and maxima are read; they may be rewritten for the next tile
                     // the tile's P tiles, page sums and rescale factors go to set sb once the scale warps are done with it
-                    TS(3);
                     if (t >= 2) wait_bar(kBarSCDone + sb, ((t >> 1) - 1) & 1);
-                    TS(2);
                     float* ps_s = ps_all + sb * (kTile + 1) * 8;
                     {
                         const int kk = stale ? k_of_token_tq3(tok) : tok;
@@ -651,15 +627,11 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
                     tile_info(ti, stale, first, np);
                     const uint32_t t = tcount + ti, rb = t % kRing;
                     const uint32_t tile = sbase + rb * kTile * G::SLOT;
-                    TS(2);
                     wait_tile(t);
-                    TS(0);
                     const int nb = (np + 1) / 2;
                     for (int bi = 0; bi < nb; ++bi, ++bc) {
                         const uint32_t vb = bc & 1;
-                        TS(2);
                         if (bc >= 2) wait_bar(kBarTFull + (bc - 2) % kTBuf, ((bc - 2) / kTBuf) & 1);     // the products of the batch before last have read it
-                        TS(1);
                         tc_fence_after();
 #pragma unroll 1
                         for (int e = 0; e < 2; ++e) {
@@ -698,7 +670,6 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
                                 }
                             }
                         }
-                        TS(3);
                         tmem_wait_st();
                         tc_fence_before();
                         warp_arrive(kBarVReady + vb);
@@ -714,10 +685,8 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
                     const uint32_t t = tcount + ti, rb = t % kRing, pb = t & 1;
                     const uint32_t tile = sbase + rb * kTile * G::SLOT;
                     const float* ps_s = ps_all + pb * (kTile + 1) * 8;
-                    TS(3);
                     wait_tile(t);
                     wait_bar(kBarPReady + pb, (t >> 1) & 1);
-                    TS(0);
                     {
                         const float4 fa = *reinterpret_cast<const float4*>(ps_s + kTile * 8), fb = *reinterpret_cast<const float4*>(ps_s + kTile * 8 + 4);
                         const float fsc[8] = {fa.x, fa.y, fa.z, fa.w, fb.x, fb.y, fb.z, fb.w};
@@ -727,9 +696,7 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
                     const int nb = (np + 1) / 2;
                     for (int bi = 0; bi < nb; ++bi, ++bc) {
                         const uint32_t vb = bc % kTBuf;
-                        TS(3);
                         wait_bar(kBarTFull + vb, (bc / kTBuf) & 1);
-                        TS(1);
                         tc_fence_after();
                         const int pn = min(2, np - 2 * bi);
 #pragma unroll 1
@@ -764,7 +731,6 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
                                 l_run[i] += ps[i];
                             }
                         }
-                        TS(2);
                     }
                     warp_arrive(kBarTileFree + rb);
                     warp_arrive(kBarSCDone + pb);
@@ -838,16 +804,7 @@ __global__ void __launch_bounds__(tm::kThreads, 1) decode_tmem_kernel(const Deco
         __syncthreads();
         pos += n_seg;
     }
-#ifdef MKV_TIMELINE
-    TS(3);
-    if (lane == 0 && wq == 0 || warp >= kISS && lane == 0) {
-        const int role = warp >= kISS ? 4 + (warp - kISS) : warp >> 2;
-        for (int k = 0; k < 4; ++k) g_warp_end[blockIdx.x * 32 + role * 4 + k] = tl_acc[k];
-        if (warp == 0) g_warp_end[blockIdx.x * 32 + 31] = clock64() - tl_begin;
-    }
-#endif
     tc_fence_before();
     __syncthreads();
     if (warp == kISS) tmem_dealloc(tb, 512);
 }
-#undef TS

@@ -160,6 +160,54 @@ __global__ void __launch_bounds__(128) append_run_kernel(uint8_t* __restrict__ f
     }
 }
 
+// Decode-sized append into the pools of several layers: one block per (token, KV head, layer).
+struct AppendLayers {
+    uint8_t* fp8[MKV_MAX_LAYERS_PER_CALL];
+    const __nv_bfloat162* k[MKV_MAX_LAYERS_PER_CALL];
+    const __nv_bfloat162* v[MKV_MAX_LAYERS_PER_CALL];
+    uint32_t* status[MKV_MAX_LAYERS_PER_CALL];
+    float inv_k_scale[MKV_MAX_LAYERS_PER_CALL], inv_v_scale[MKV_MAX_LAYERS_PER_CALL];
+    int fp8_pages[MKV_MAX_LAYERS_PER_CALL];
+};
+
+template <int D>
+__global__ void __launch_bounds__(D / 2) append_layers_kernel(const AppendLayers A, int hkv, int tiles,
+                                                               const int32_t* __restrict__ slots)
+{
+    const int tok = blockIdx.x, h = blockIdx.y, layer = blockIdx.z;
+    const int sm = slots[tok];
+    if (sm < 0) return;
+    const int gt = sm >> 4, slot = sm & 15, page = gt / tiles, m = gt - page * tiles;
+    if (page >= A.fp8_pages[layer]) {
+        if (threadIdx.x == 0) atomicOr(A.status[layer], kStBounds);
+        return;
+    }
+    uint8_t* rec = A.fp8[layer] + (((size_t)page * hkv + h) * tiles + m) * fp8_record_bytes(D);
+    const size_t src = ((size_t)tok * hkv + h) * (D / 2);
+    append_token<D>(rec, slot, A.inv_k_scale[layer], A.inv_v_scale[layer], A.k[layer] + src, A.v[layer] + src, threadIdx.x);
+}
+
+int32_t launch_append_layers(mkv_pool* const* pools, const void* const* k, const void* const* v, const int32_t* slots,
+                             int n, int n_layers, cudaStream_t s)
+{
+    AppendLayers A;
+    for (int i = 0; i < n_layers; ++i) {
+        A.fp8[i] = pools[i]->fp8;
+        A.k[i] = static_cast<const __nv_bfloat162*>(k[i]);
+        A.v[i] = static_cast<const __nv_bfloat162*>(v[i]);
+        A.status[i] = pools[i]->status_dev;
+        A.inv_k_scale[i] = 1.0f / pools[i]->cfg.k_scale;
+        A.inv_v_scale[i] = 1.0f / pools[i]->cfg.v_scale;
+        A.fp8_pages[i] = pools[i]->cfg.fp8_pages;
+    }
+    const mkv_pool* p = pools[0];
+    dim3 grid(n, p->hkv, n_layers);
+    if (p->d == 128) append_layers_kernel<128><<<grid, 64, 0, s>>>(A, p->hkv, p->tiles, slots);
+    else append_layers_kernel<256><<<grid, 128, 0, s>>>(A, p->hkv, p->tiles, slots);
+    MKV_CUDA(cudaGetLastError());
+    return MKV_OK;
+}
+
 int32_t launch_append(mkv_pool* p, const void* k, const void* v, const int32_t* slots, int n, cudaStream_t s)
 {
     const float ik = 1.0f / p->cfg.k_scale, iv = 1.0f / p->cfg.v_scale;

@@ -69,6 +69,7 @@ struct mkv_pool {
     uint32_t* status_dev;
     mkv::SigmaBits sigma;
     int variant;
+    unsigned long long wait_ns;  // wall-time limit of the decode scan's waits for a page copy
     int device;
     mkv::Device dev;
     std::mutex mu;
@@ -106,6 +107,11 @@ int32_t launch_decode_tensor(mkv_pool* p, const void* q, const int32_t* bt, cons
 int32_t launch_decode_tensor_at(mkv_pool* p, const void* q, const int32_t* bt, const uint8_t* tags,
                                 const int32_t* lens, int B, int max_pages, float scale, float* out, float* lse,
                                 float* partials, uint32_t* tickets, int max_blocks, float* mass, cudaStream_t s);
+int32_t launch_decode_tensor_layers(mkv_pool* const* pools, const void* const* q, const int32_t* const* bt,
+                                    const uint8_t* const* tags, const int32_t* lens, int B, int max_pages, float scale,
+                                    float* const* out, float* const* lse, void* const* ws, int n_layers, cudaStream_t s);
+int32_t launch_append_layers(mkv_pool* const* pools, const void* const* k, const void* const* v, const int32_t* slots,
+                             int n_tokens, int n_layers, cudaStream_t s);
 int32_t launch_page_score(const float* mass, const int32_t* lens, int B, int hq, int max_pages, uint64_t head_mask,
                           float beta, float* score, int page_tokens, cudaStream_t s);
 constexpr int kMaxCtas = 512;        // upper bound of the decode scan's persistent grid (sizes workspace and tickets)

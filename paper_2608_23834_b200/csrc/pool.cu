@@ -109,6 +109,7 @@ static mkv_pool* new_pool(const mkv_pool_config* cfg, void* fp8_arena, void* tq3
     p->fp8 = static_cast<uint8_t*>(fp8_arena);
     p->tq3 = static_cast<uint8_t*>(tq3_arena);
     p->variant = MKV_DECODE_TENSOR;
+    p->wait_ns = 20000000ull;
     std::memset(&p->sigma, 0, sizeof p->sigma);
     for (int i = 0; cfg->k_rot_signs && i < cfg->head_dim; ++i)
         if (cfg->k_rot_signs[i] < 0) p->sigma.w[i >> 5] |= 1u << (i & 31);
@@ -232,6 +233,13 @@ int32_t mkv_pool_set_decode_variant(mkv_pool* pool, int32_t variant)
     return MKV_OK;
 }
 
+int32_t mkv_pool_set_wait_limit_ns(mkv_pool* pool, uint64_t ns)
+{
+    if (!pool) return MKV_E_INVALID;
+    pool->wait_ns = ns;
+    return MKV_OK;
+}
+
 static int32_t raw_span(mkv_pool* pool, int32_t fmt, int32_t id, uint8_t** ptr, size_t* bytes)
 {
     if (!pool || !pool->fp8 || (fmt != MKV_FMT_FP8 && fmt != MKV_FMT_TQ3)) return MKV_E_INVALID;
@@ -320,6 +328,66 @@ int32_t mkv_decode_attention(mkv_pool* pool, const void* q, const int32_t* bt, c
                                     (cudaStream_t)stream);
     return launch_decode_tensor(pool, q, bt, tags, lens, B, max_pages, scale, out, lse, ws, ws_bytes,
                                 (cudaStream_t)stream);
+}
+
+int32_t mkv_decode_attention_layers(const mkv_layer_call* L, int32_t n_layers, const int32_t* lens, int32_t B,
+                                    int32_t max_pages, float scale, size_t ws_bytes, void* stream)
+{
+    if (!L || n_layers < 1 || n_layers > MKV_MAX_LAYERS_PER_CALL || B < 0 || max_pages < 0) return MKV_E_INVALID;
+    if (B == 0) return MKV_OK;
+    if (!lens || !aligned(lens, 4) || !(scale == scale)) return MKV_E_INVALID;
+    mkv_pool* pools[MKV_MAX_LAYERS_PER_CALL];
+    const void* q[MKV_MAX_LAYERS_PER_CALL];
+    const int32_t* bt[MKV_MAX_LAYERS_PER_CALL];
+    const uint8_t* tags[MKV_MAX_LAYERS_PER_CALL];
+    float* out[MKV_MAX_LAYERS_PER_CALL];
+    float* lse[MKV_MAX_LAYERS_PER_CALL];
+    void* ws[MKV_MAX_LAYERS_PER_CALL];
+    for (int i = 0; i < n_layers; ++i) {
+        const mkv_layer_call& c = L[i];
+        if (!c.pool || !c.pool->fp8 || !c.q_dev || !c.block_table_dev || !c.tier_tag_dev || !c.out_dev || !c.workspace_dev)
+            return MKV_E_INVALID;
+        if (!aligned(c.q_dev, 16) || !aligned(c.out_dev, 16) || !aligned(c.workspace_dev, 256) || !aligned(c.block_table_dev, 4))
+            return MKV_E_INVALID;
+        const mkv_pool* p0 = L[0].pool;
+        if (c.pool->d != p0->d || c.pool->hkv != p0->hkv || c.pool->hq != p0->hq || c.pool->tiles != 1 ||
+            c.pool->device != p0->device || c.pool->variant != MKV_DECODE_TENSOR) {
+            set_last_error("mkv_decode_attention_layers: pools of one geometry, 16-token pages, one device and the tensor-core variant");
+            return MKV_E_INVALID;
+        }
+        for (int j = 0; j < i; ++j)
+            if (L[j].workspace_dev == c.workspace_dev) {
+                set_last_error("mkv_decode_attention_layers: every layer needs its own workspace");
+                return MKV_E_INVALID;
+            }
+        pools[i] = c.pool; q[i] = c.q_dev; bt[i] = c.block_table_dev; tags[i] = c.tier_tag_dev;
+        out[i] = c.out_dev; lse[i] = c.lse_dev; ws[i] = c.workspace_dev;
+    }
+    size_t need;
+    if (mkv_decode_workspace_bytes(&L[0].pool->cfg, B, &need) != MKV_OK || ws_bytes < need) return MKV_E_INVALID;
+    return launch_decode_tensor_layers(pools, q, bt, tags, lens, B, max_pages, scale, out, lse, ws, n_layers,
+                                       (cudaStream_t)stream);
+}
+
+int32_t mkv_append_layers(const mkv_layer_append* L, int32_t n_layers, const int32_t* slots, int32_t n, void* stream)
+{
+    if (!L || n_layers < 1 || n_layers > MKV_MAX_LAYERS_PER_CALL || n < 0 || n > 64) return MKV_E_INVALID;
+    if (n == 0) return MKV_OK;
+    if (!slots || !aligned(slots, 4)) return MKV_E_INVALID;
+    mkv_pool* pools[MKV_MAX_LAYERS_PER_CALL];
+    const void* k[MKV_MAX_LAYERS_PER_CALL];
+    const void* v[MKV_MAX_LAYERS_PER_CALL];
+    for (int i = 0; i < n_layers; ++i) {
+        const mkv_layer_append& c = L[i];
+        if (!c.pool || !c.pool->fp8 || !c.k_dev || !c.v_dev || !aligned(c.k_dev, 16) || !aligned(c.v_dev, 16)) return MKV_E_INVALID;
+        const mkv_pool* p0 = L[0].pool;
+        if (c.pool->d != p0->d || c.pool->hkv != p0->hkv || c.pool->tiles != p0->tiles || c.pool->device != p0->device) {
+            set_last_error("mkv_append_layers: pools of one geometry on one device");
+            return MKV_E_INVALID;
+        }
+        pools[i] = c.pool; k[i] = c.k_dev; v[i] = c.v_dev;
+    }
+    return launch_append_layers(pools, k, v, slots, n, n_layers, (cudaStream_t)stream);
 }
 
 int32_t mkv_decode_attention_scored(mkv_pool* pool, const void* q, const int32_t* bt, const uint8_t* tags,
