@@ -52,6 +52,10 @@ def lib():
         L.orc_f32_to_f16_sat.argtypes = [C.c_float]
         L.orc_f16_to_f32.restype = C.c_float
         L.orc_f16_to_f32.argtypes = [C.c_uint16]
+        L.orc_set_format.restype = C.c_int
+        L.orc_set_format.argtypes = [C.c_int]
+        L.orc_get_format.restype = C.c_int
+        L.orc_get_format.argtypes = []
         L.orc_codebook_level.restype = C.c_float
         L.orc_codebook_level.argtypes = [C.c_int]
         L.orc_codebook_threshold.restype = C.c_float
@@ -138,6 +142,32 @@ def lib():
         L.orc_effective_bits.argtypes = [C.c_double] * 5
         _lib = L
     return _lib
+
+
+def set_format(fmt: int) -> None:
+    """Select the TQ3 record format (1: fp16 Lloyd-Max codebook; 2: e4m3-exact codebook and the re-cut key
+    section) that every oracle function uses from now on."""
+    if lib().orc_set_format(int(fmt)) != 0:
+        raise ValueError("record format must be 1 or 2")
+
+
+def get_format() -> int:
+    return lib().orc_get_format()
+
+
+class record_format:
+    """with oracle.record_format(2): ...  -- run a block under one record format, then restore."""
+
+    def __init__(self, fmt: int):
+        self.fmt = fmt
+
+    def __enter__(self):
+        self.prev = get_format()
+        set_format(self.fmt)
+        return self
+
+    def __exit__(self, *exc):
+        set_format(self.prev)
 
 
 def _p(a: np.ndarray, ty):

@@ -86,9 +86,15 @@ def test_brute_force_softmax_on_tiny_inputs():
                 assert np.array_equal(out[0, g], v0)
 
 
-def test_tq3_pages_match_numpy_dense_attention_on_decoded_codes():
+@pytest.fixture(params=[1, 2])
+def record_format(request):
+    with oracle.record_format(request.param):
+        yield request.param
+
+
+def test_tq3_pages_match_numpy_dense_attention_on_decoded_codes(record_format):
     """Stale pages: decode the packed codes with an explicit Hadamard matrix (k^ = g d^-1/2 sigma.(H c),
-    v^ = scale*code + zero) and attend densely in numpy."""
+    v^ = scale*code + zero) and attend densely in numpy; in both record formats."""
     spec = small_spec(0, (16 * 9 + 5,), anchor_prefix=16, recent_tokens=40)
     tab = W.tables(spec)
     assert (tab.tier_tag[0, :spec.n_pages(0)] == W.TAG_STALE).sum() >= 5
