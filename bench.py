@@ -133,7 +133,7 @@ class LayerState:
     pass
 
 
-def build_layers(spec, steps_total, device, M, torch):
+def build_layers(spec, steps_total, device, M, torch, spec_format=1):
     """Pools of every layer filled through the library's own Append and Demote kernels from seeded
     synthetic bf16 K/V, plus the tables, slots and retier plan of every timed step."""
     B, d, hkv, hq = spec.batch, spec.head_dim, spec.n_kv_heads, spec.n_q_heads
@@ -187,7 +187,8 @@ def build_layers(spec, steps_total, device, M, torch):
     for layer in range(spec.n_layers):
         L = LayerState()
         sigma = W.rotation_signs(spec, layer)
-        L.pool = M.Pool(d, hkv, hq, fp8_cap, tq3_cap, sigma, max_batch=B, device=device, page_tokens=T)
+        L.pool = M.Pool(d, hkv, hq, fp8_cap, tq3_cap, sigma, max_batch=B, device=device, page_tokens=T,
+                        tq3_format=spec_format)
         gen.manual_seed(1000 * spec.seed + layer)
         k_out = torch.from_numpy(W.outlier_channels(spec, layer, 0)).to(device)
         v_out = torch.from_numpy(W.outlier_channels(spec, layer, 1)).to(device)
@@ -296,7 +297,8 @@ def run_ours(args):
     spec = workload_spec(args)
     K, Wm = args.steps, args.warmup
     total = 3 * (K + Wm)                       # eager run (per-launch events), graph run (timed), end-to-end run
-    layers, plan, tab0 = build_layers(spec, total, device, M, torch)
+    fmt = 2 if args.format == "v2" else 1
+    layers, plan, tab0 = build_layers(spec, total, device, M, torch, fmt)
     for L in layers:
         L.pool.set_decode_variant({"scalar": M.DECODE_SCALAR, "tmem": M.DECODE_TMEM}.get(args.variant, M.DECODE_TENSOR))
     B, d, hq, hkv = spec.batch, spec.head_dim, spec.n_q_heads, spec.n_kv_heads
@@ -521,9 +523,10 @@ def run_ours(args):
     result = {
         "metric": METRIC, "value": aggregate_value(B, K, ms, world), "unit": UNIT, "n_gpus": world, "steps": K,
         "warmup": Wm, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "u8 codes (e4m3 / 3-bit TQ3) -> f16 tensor-core operands, f32 accumulate", "data": "synthetic",
+        "dtype": ("u8 codes (e4m3 / 3-bit TQ3); key products e4m3 x e4m3, value products f16 x f16, f32 accumulate" if fmt == 2 else
+                  "u8 codes (e4m3 / 3-bit TQ3) -> f16 tensor-core operands, f32 accumulate"), "data": "synthetic",
         "config": {"workload": workload_name(spec), "batch": B, "context_tokens": list(spec.seq_lens)[:4],
-                   "layers": spec.n_layers, "head_dim": d, "kv_heads": hkv, "q_heads": hq, "page_tokens": spec.page_tokens,
+                   "tq3_record_format": fmt, "layers": spec.n_layers, "head_dim": d, "kv_heads": hkv, "q_heads": hq, "page_tokens": spec.page_tokens,
                    "parallelism": "replicas only" if world > 1 else "single GPU",
                    "l2": "inputs larger than L2 (%.0f MB of KV per step)" % (step_bytes / 1e6),
                    "step": "append + demote at its natural cadence + decode attention, every layer",

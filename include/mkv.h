@@ -34,6 +34,14 @@
  *       [0, 6d)   key codes,   [6d, 12d) value codes,   [12d, 12d+32) norm correction g[16],
  *       [12d+32, 16d+32) value scale/zero.  Bit positions are those of the tensor-core
  *     fragment that consumes them; mkv_page_read_raw() returns the bytes as stored.
+ *   TQ3 record format 2 (mkv_pool_config.tq3_format = 2; Section 3.1 fixes neither codebook nor layout):
+ *     the four key magnitudes are the e4m3 numbers nearest to the Lloyd-Max levels (0.25, 0.75, 1.375,
+ *     2.25; thresholds 0.5, 1.0625, 1.8125; about 1 % more Gaussian distortion), and the key section is
+ *     cut so that four consecutive dims of a token are the nibbles of one half-word.  The decode scan then
+ *     turns four codes into four 8-bit floats with one byte-table lookup and multiplies them as FP8 tensor-
+ *     core operands against the rotated query carried as four e4m3 terms.  Value codes, norm corrections,
+ *     scale/zero, sizes and every other encoder step are those of format 1.  A pool has one format; pages
+ *     written under one format must not be read under the other.  MKV_DECODE_TMEM serves format 1 only.
  *   Pages of 16 M tokens (page_size = 16 M) are M tiles of 16 tokens:
  *     FP8 page, M * 32*d bytes: tile m is the FP8 record of tokens [16 m, 16 m + 16) at m * 32*d.
  *     TQ3 page, M * (12*d + 32) + 4*d bytes: tile m at m * (12*d + 32) holds [key codes | value codes |
@@ -90,6 +98,7 @@ typedef struct {
     float v_scale;              /* FP8 value scale                                              */
     const int8_t* k_rot_signs;  /* host, head_dim entries of +1/-1: diagonal of the randomised  */
                                 /* Hadamard rotation applied to keys before 3-bit quantisation  */
+    int32_t tq3_format;         /* TQ3 record format: 1 (0 means 1), or 2 (see "Record formats") */
 } mkv_pool_config;
 
 typedef struct {

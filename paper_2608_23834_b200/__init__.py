@@ -51,7 +51,8 @@ class MkvError(RuntimeError):
 class PoolConfig(C.Structure):
     _fields_ = [("page_size", C.c_int32), ("head_dim", C.c_int32), ("n_kv_heads", C.c_int32),
                 ("n_q_heads", C.c_int32), ("fp8_pages", C.c_int32), ("tq3_pages", C.c_int32),
-                ("k_scale", C.c_float), ("v_scale", C.c_float), ("k_rot_signs", C.POINTER(C.c_int8))]
+                ("k_scale", C.c_float), ("v_scale", C.c_float), ("k_rot_signs", C.POINTER(C.c_int8)),
+                ("tq3_format", C.c_int32)]
 
 
 class Stats(C.Structure):
@@ -143,10 +144,10 @@ def _stream(stream: Optional[torch.cuda.Stream]):
 
 
 def make_config(head_dim, n_kv_heads, n_q_heads, fp8_pages, tq3_pages, sigma: np.ndarray, k_scale=1.0, v_scale=1.0,
-                page_tokens=16):
+                page_tokens=16, tq3_format=1):
     sig = np.ascontiguousarray(sigma, dtype=np.int8)
     cfg = PoolConfig(page_tokens, head_dim, n_kv_heads, n_q_heads, fp8_pages, tq3_pages, k_scale, v_scale,
-                     sig.ctypes.data_as(C.POINTER(C.c_int8)))
+                     sig.ctypes.data_as(C.POINTER(C.c_int8)), tq3_format)
     cfg._keepalive = sig
     return cfg
 
@@ -168,12 +169,14 @@ class Pool:
     """One layer's page pool.  Owns the torch buffers handed to the library (arenas, workspace)."""
 
     def __init__(self, head_dim, n_kv_heads, n_q_heads, fp8_pages, tq3_pages, sigma, k_scale=1.0, v_scale=1.0,
-                 max_batch=64, device="cuda:0", page_tokens=16):
+                 max_batch=64, device="cuda:0", page_tokens=16, tq3_format=1):
         L = lib()
+        self.tq3_format = tq3_format
         self.device = torch.device(device)
         self.d, self.hkv, self.hq = head_dim, n_kv_heads, n_q_heads
         self.group = n_q_heads // n_kv_heads
-        self.cfg = make_config(head_dim, n_kv_heads, n_q_heads, fp8_pages, tq3_pages, sigma, k_scale, v_scale, page_tokens)
+        self.cfg = make_config(head_dim, n_kv_heads, n_q_heads, fp8_pages, tq3_pages, sigma, k_scale, v_scale, page_tokens,
+                               tq3_format)
         fp8_bytes, tq3_bytes = mkv_pool_query(self.cfg)
         # bytes of one page and KV head: a page is page_tokens / 16 tiles (16 d + 32 bytes of TQ3 at one tile)
         self.page_tokens, self.tiles = page_tokens, page_tokens // 16

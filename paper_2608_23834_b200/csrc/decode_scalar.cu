@@ -36,8 +36,21 @@ __device__ __forceinline__ uint32_t lane_word(const uint8_t* section, int lane, 
 
 // 3-bit key code of (token t, rotated dim i): magnitude in bits 0-1, sign in bit 2
 template <int D>
-__device__ int tq3_key_code(const uint8_t* rec, int t, int i)
+__device__ int tq3_key_code(const uint8_t* rec, int t, int i, int fmt)
 {
+    if (fmt == 2) {
+        // record format 2: step i/32, K slot k = i%32; lane 4 (t%8) + (k%16)/4, register e = 4 (step%2) + 2 (t/8) + k/16
+        // of word triple step/2, nibble 4 (e%2) + k%4
+        const int st = i >> 5, k = i & 31;
+        const int lane = 4 * (t & 7) + ((k & 15) >> 2), j = st >> 1, e = 4 * (st & 1) + 2 * (t >> 3) + (k >> 4);
+        const int n = 4 * (e & 1) + (k & 3);
+        const uint32_t A = lane_word<D>(rec, lane, 3 * j), Bw = lane_word<D>(rec, lane, 3 * j + 1),
+                       Cw = lane_word<D>(rec, lane, 3 * j + 2);
+        if (e < 2) return (A >> (4 * n)) & 7;
+        if (e < 4) return (Bw >> (4 * n)) & 7;
+        if (e < 6) return ((Cw >> (4 * n)) & 3) | (((A >> (4 * n + 3)) & 1) << 2);
+        return ((Cw >> (4 * n + 2)) & 3) | (((Bw >> (4 * n + 3)) & 1) << 2);
+    }
     const int kb = i >> 4, s = i & 15;
     const int lane = 4 * (t & 7) + ((s & 7) >> 1), r = (t >> 3) + 2 * (s >> 3), n = 2 * r + (s & 1), j = kb >> 2;
     const uint32_t A = lane_word<D>(rec, lane, 3 * j), Bw = lane_word<D>(rec, lane, 3 * j + 1),
@@ -74,7 +87,7 @@ __global__ void __launch_bounds__(D) decode_scalar_kernel(
     const uint8_t* __restrict__ fp8, const uint8_t* __restrict__ tq3, int fp8_pages, int tq3_pages, int hkv, int G,
     float k_scale, float v_scale, SigmaBits sigma, const __nv_bfloat16* __restrict__ q,
     const int32_t* __restrict__ bt, const uint8_t* __restrict__ tags, const int32_t* __restrict__ lens,
-    int max_pages, int tiles, float scale, int n_splits, float* __restrict__ part, uint32_t* __restrict__ status)
+    int max_pages, int tiles, int fmt, float scale, int n_splits, float* __restrict__ part, uint32_t* __restrict__ status)
 {
     extern __shared__ float smem[];
     float* qs = smem;                       // [8][D] query
@@ -97,7 +110,8 @@ __global__ void __launch_bounds__(D) decode_scalar_kernel(
     const int n_pages = (len + kPage - 1) / kPage;
     const int per = (n_pages + n_splits - 1) / n_splits;
     const int lo = split * per, hi = min(n_pages, lo + per);
-    const float C[4] = {MKV_C0, MKV_C1, MKV_C2, MKV_C3};
+    const float C[4] = {fmt == 2 ? KeyCodebook<2>::C0 : KeyCodebook<1>::C0, fmt == 2 ? KeyCodebook<2>::C1 : KeyCodebook<1>::C1,
+                        fmt == 2 ? KeyCodebook<2>::C2 : KeyCodebook<1>::C2, fmt == 2 ? KeyCodebook<2>::C3 : KeyCodebook<1>::C3};
 
     for (int g = 0; g < 8; ++g) {
         float x = g < G ? __bfloat162float(q[((size_t)b * hq + h * G + g) * D + tid]) : 0.f;
@@ -144,7 +158,7 @@ __global__ void __launch_bounds__(D) decode_scalar_kernel(
             const int mi = (cb >> 1) * 64 + (row & 7) * 8 + 4 * (cb & 1) + (row >> 3);
             const float vsc = __half2float(meta[mi]), vzp = __half2float(meta[mi + 2]);
             for (int t = 0; t < kPage; ++t) {
-                const int kc = tq3_key_code<D>(rec, t, tid);
+                const int kc = tq3_key_code<D>(rec, t, tid, fmt);
                 Ks[t * (D + 1) + tid] = (kc & 4) ? -C[kc & 3] : C[kc & 3];
                 Vs[t * D + tid] = fmaf(vsc, (float)tq3_value_code<D>(rec, t, tid), vzp);
             }
@@ -238,7 +252,7 @@ static int32_t run_scalar(mkv_pool* p, const void* q, const int32_t* bt, const u
     dim3 grid(S, p->hkv, B);
     decode_scalar_kernel<D><<<grid, D, smem, s>>>(p->fp8, p->tq3, p->cfg.fp8_pages, p->cfg.tq3_pages, p->hkv,
                                                   p->group, p->cfg.k_scale, p->cfg.v_scale, p->sigma,
-                                                  (const __nv_bfloat16*)q, bt, tags, lens, max_pages, p->tiles, scale, S,
+                                                  (const __nv_bfloat16*)q, bt, tags, lens, max_pages, p->tiles, p->fmt, scale, S,
                                                   part, p->status_dev);
     MKV_CUDA(cudaGetLastError());
     merge_scalar_kernel<D><<<dim3(p->hq, B), D, 0, s>>>(part, S, p->hq, out, lse);

@@ -26,6 +26,7 @@
 //     waits for another, and there is no second launch.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
+#include <cuda_fp8.h>
 #include <math_constants.h>
 
 #include <cstdlib>
@@ -114,6 +115,24 @@ __device__ __forceinline__ void mma16816_zero(float (&d)[4], const uint32_t (&a)
     asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
                  : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.f));
+}
+
+// D += A B with signed 8-bit integer operands and 32-bit integer accumulators: A 16 x 32 (row-major fragment),
+// B 32 x 8.  (Measured on B200: this legacy integer MMA is one native instruction at the rate of the fp16
+// m16n8k16 one, i.e. twice its products per instruction; the e4m3 form of mma.sync is expanded by the compiler
+// into conversions and fp16 MMAs and is slower than the fp16 path it was meant to replace.)
+__device__ __forceinline__ void mma16832_s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1)
+{
+    asm("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t lds32(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
 }
 
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x)
@@ -383,7 +402,8 @@ struct Geo {
     static constexpr int OFF_L = OFF_M + NW * 8 * 4;
     static constexpr int OFF_PART = OFF_L + NW * 8 * 4;
     static constexpr int OFF_LAST = OFF_PART + ((int)sizeof(Partition) + 15) / 16 * 16;
-    static constexpr int SMEM = OFF_LAST + 16;
+    static constexpr int OFF_QS = OFF_LAST + 16;             // record format 2: digit unit of the rotated query, per head
+    static constexpr int SMEM = OFF_QS + 32;
     static_assert(NW >= 4, "a warp builds the query fragments of at most two columns of the 8-wide head group");
     static_assert(NSTAGE >= 2 && NSTAGE % 2 == 0 && NSTAGE <= 16, "an FP8 page takes a pair of slots; one phase bit per slot");
     static_assert(NSTAGE * SLOT >= 8 * D * 4, "ring doubles as the cross-warp reduction buffer");
@@ -404,6 +424,10 @@ struct WarpAcc {
     // output accumulated before sits in shared memory, to be multiplied by pk (the rescales since then)
     float lp[2];
     float pk[2];
+    // record format 2: its score tile has the heads in the rows, so the lane also keeps the running maximum
+    // of head g (`mr`); m[] (heads 2tq, 2tq+1: the columns of the output tile) stays the master copy that the
+    // Recent/Anchor pages, the page mass and the reduction use, and the two are brought in line on every change
+    float mr;
 };
 
 // Scores of one page -> probabilities.  s[0..1] = token g, s[2..3] = token g+8 (heads 2tq, 2tq+1).
@@ -613,11 +637,121 @@ __device__ __forceinline__ void tq3_value_quad(float (&o0)[4], float (&o1)[4], f
     }
 }
 
+// ---- record format 2 ---------------------------------------------------------------------------------
+// The key levels of format 2 are eighths of small integers (2, 6, 11, 18), and four consecutive dims of a
+// token are the four nibbles of one half-word: one byte-table lookup turns four codes into four signed bytes,
+// and the products run as integer MMAs with the roles swapped: A = the rotated query (16 rows = 8 heads x 2
+// of its 3 digits per MMA), B = the keys of eight tokens (32 dims per step).  S[head g][tokens 2tq, 2tq+1]
+// then sits in the lane that needs exactly these probabilities as the B fragment of the value product: no
+// transposition.
+//
+// Rotated query of head h: q' = delta_h (2^14 t0 + 2^7 t1 + t2), digits in [-64, 63], delta_h = max|q'| / (63 2^14):
+// 21 bits below the largest coordinate (one fp16, 11 bits, is not enough for the 2e-3 bound; two int8 digits,
+// 15 bits, fail it on short peaked rows by simulation).  The integer sums are exact.
+
+// Two 32-dim steps (2j, 2j+1) of a Stale page: word triple (A, B, C) of the lane -> eight B registers
+// (step, token half u, K half), then per step and token half one MMA for digits 0,1 and one for digit 2.
+// q_pair: shared-memory address of this lane's query fragments of step 2j (digits 0,1 at +0, digit 2 at +512,
+// step 2j+1 at +1024).
+__device__ __forceinline__ void tq3_key_pair_v2(int (&Sa0)[4], int (&Sb0)[4], int (&Sa1)[4], int (&Sb1)[4],
+                                                uint32_t A, uint32_t Bw, uint32_t Cw, uint32_t q_pair)
+{
+    // signed levels +-{2, 6, 11, 18} (eight times the codebook) as bytes, indexed by code = magnitude | sign << 2
+    constexpr uint32_t T0 = 0x120B0602u, T1 = 0xEEF5FAFEu;
+    uint32_t sel[4], r[8];
+    sel[0] = A & 0x77777777u;
+    sel[1] = Bw & 0x77777777u;
+    sel[2] = lop3_and_or(A >> 1, 0x44444444u, Cw & 0x33333333u);
+    sel[3] = lop3_and_or(Bw >> 1, 0x44444444u, (Cw >> 2) & 0x33333333u);
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+        r[2 * w] = prmt(T0, T1, sel[w]);
+        r[2 * w + 1] = prmt(T0, T1, sel[w] >> 16);
+    }
+#pragma unroll
+    for (int st = 0; st < 2; ++st) {
+        const uint4 qa = lds128(q_pair + st * 1024);
+        const uint2 qb = lds64(q_pair + st * 1024 + 512);
+        mma16832_s8(Sa0, qa.x, qa.y, qa.z, qa.w, r[4 * st], r[4 * st + 1]);
+        mma16832_s8(Sb0, qb.x, 0u, qb.y, 0u, r[4 * st], r[4 * st + 1]);
+        mma16832_s8(Sa1, qa.x, qa.y, qa.z, qa.w, r[4 * st + 2], r[4 * st + 3]);
+        mma16832_s8(Sb1, qb.x, 0u, qb.y, 0u, r[4 * st + 2], r[4 * st + 3]);
+    }
+}
+
+// head g, one token: exact integer sums of the three digits -> the score in units of delta_h / 8
+__device__ __forceinline__ float digits_to_score(int hi, int mid, int lo)
+{
+    return fmaf((float)hi, 16384.f, (float)(mid * 128 + lo));
+}
+
+// row form of the maximum from the column form and back (lanes 4h .. 4h+3 hold head h's row value; lane
+// (g, tq) holds the column values of heads 2tq, 2tq+1)
+template <int NB>
+__device__ __forceinline__ void max_rows_from_columns(WarpAcc<NB>& acc, int lane)
+{
+    const int g = lane >> 2;
+    const float a = __shfl_sync(0xffffffffu, acc.m[0], g >> 1), b = __shfl_sync(0xffffffffu, acc.m[1], g >> 1);
+    acc.mr = (g & 1) ? b : a;
+}
+
+// Scores s[0..1] = tokens 2tq, 2tq+1, s[2..3] = tokens 2tq+8, 2tq+9, all of head g.  Raises the running
+// maximum of head g when it is exceeded by more than the slack and rescales the accumulator columns.
+template <int NB, bool TILED = false>
+__device__ __forceinline__ void softmax_rescale_v2(WarpAcc<NB>& acc, const float (&s)[4], int lane)
+{
+    constexpr uint32_t FULL = 0xffffffffu;
+    float mx = fmaxf(fmaxf(s[0], s[1]), fmaxf(s[2], s[3]));
+    if (__any_sync(FULL, mx > acc.mr + kRescaleSlack)) {
+        mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, 2));
+        const bool up = mx > acc.mr + kRescaleSlack;
+        const float f = up ? fast_exp2(acc.mr - mx) : 1.f;
+        if (up) acc.mr = mx;
+        const int tq = lane & 3;
+        const float f0 = __shfl_sync(FULL, f, 8 * tq), f1 = __shfl_sync(FULL, f, 8 * tq + 4);
+        acc.m[0] = __shfl_sync(FULL, acc.mr, 8 * tq);
+        acc.m[1] = __shfl_sync(FULL, acc.mr, 8 * tq + 4);
+#pragma unroll
+        for (int i = 0; i < NB; ++i) {
+            acc.o[i][0] *= f0; acc.o[i][2] *= f0;
+            acc.o[i][1] *= f1; acc.o[i][3] *= f1;
+        }
+        acc.l[0] *= f0;
+        acc.l[1] *= f1;
+        if constexpr (TILED) {
+            acc.lp[0] *= f0; acc.lp[1] *= f1;
+            acc.pk[0] *= f0; acc.pk[1] *= f1;
+        }
+    }
+}
+
+// P of head g for the lane's four tokens is the B fragment of the value product as it stands.
+template <int NB>
+__device__ __forceinline__ void softmax_probs_v2(WarpAcc<NB>& acc, const float (&s)[4], PFrag& pf)
+{
+    const float p0 = fast_exp2(s[0] - acc.mr), p1 = fast_exp2(s[1] - acc.mr);
+    const float p2 = fast_exp2(s[2] - acc.mr), p3 = fast_exp2(s[3] - acc.mr);
+    pf.b0 = pack_f16x2(p0, p1);
+    pf.b1 = pack_f16x2(p2, p3);
+    const float2 h01 = half2_to_float2(pf.b0), h23 = half2_to_float2(pf.b1);
+    pf.c0 = pack_f16x2(p0 - h01.x, p1 - h01.y);
+    pf.c1 = pack_f16x2(p2 - h23.x, p3 - h23.y);
+    const uint32_t ones[4] = {0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u};
+    float ps[4];
+    mma16816_zero(ps, ones, pf.b0, pf.b1);
+    mma16816(ps, ones, pf.c0, pf.c1);
+    pf.ps0 = ps[0];
+    pf.ps1 = ps[1];
+    acc.l[0] += ps[0];
+    acc.l[1] += ps[1];
+}
+
 // Software-pipelined step over Stale pages: the value phase of the current page (record rec_v, its
 // probabilities pf) and the score phase of the next page (record rec_k) are issued quad by quad in
 // one instruction stream, so that table lookups, half-precision FMAs, fp32 FMAs and MMAs of the two
 // phases overlap.  DO_V / DO_K switch the halves off for the first and the last page.
-template <int D, bool DO_V, bool DO_K, bool DEFER = false>
+template <int D, bool DO_V, bool DO_K, bool DEFER = false, int FMT = 1>
 __device__ __forceinline__ void tq3_step(WarpAcc<D / 16>& acc, uint32_t rec_v, const float (&s_cur)[4], PFrag& pf, uint32_t rec_k,
                                          uint32_t qt_lane, float sc2, int lane, float (&s_next)[4])
 {
@@ -625,9 +759,13 @@ __device__ __forceinline__ void tq3_step(WarpAcc<D / 16>& acc, uint32_t rec_v, c
     const int g = lane >> 2;
     uint32_t kw[LW], vw[LW];
     float S0[4] = {0.f, 0.f, 0.f, 0.f}, S1[4] = {0.f, 0.f, 0.f, 0.f};
+    int I0[4] = {0, 0, 0, 0}, I1[4] = {0, 0, 0, 0}, I2[4] = {0, 0, 0, 0}, I3[4] = {0, 0, 0, 0};   // format 2: (digits 0,1 | 2) x (tokens g | g+8)
     if constexpr (DO_K) load_lane_words<D>(rec_k, lane, kw);
     if constexpr (DO_V) load_lane_words<D>(rec_v + 6 * D, lane, vw);
-    if constexpr (DO_V) softmax_probs<NB>(acc, s_cur, pf);     // in one block with the key unpack of the next page
+    if constexpr (DO_V) {      // in one block with the key unpack of the next page
+        if constexpr (FMT == 2) softmax_probs_v2<NB>(acc, s_cur, pf);
+        else softmax_probs<NB>(acc, s_cur, pf);
+    }
     if constexpr (DO_V && DEFER) {
         acc.lp[0] += pf.ps0;
         acc.lp[1] += pf.ps1;
@@ -635,12 +773,27 @@ __device__ __forceinline__ void tq3_step(WarpAcc<D / 16>& acc, uint32_t rec_v, c
     const uint32_t meta = rec_v + 12 * D + 32 + g * 16;
 #pragma unroll
     for (int j = 0; j < NB / 4; ++j) {
-        if constexpr (DO_K) tq3_key_quad(S0, S1, kw[3 * j], kw[3 * j + 1], kw[3 * j + 2], qt_lane + j * 2048);
+        if constexpr (DO_K) {
+            if constexpr (FMT == 2) tq3_key_pair_v2(I0, I1, I2, I3, kw[3 * j], kw[3 * j + 1], kw[3 * j + 2], qt_lane + j * 2048);
+            else tq3_key_quad(S0, S1, kw[3 * j], kw[3 * j + 1], kw[3 * j + 2], qt_lane + j * 2048);
+        }
         if constexpr (DO_V)
             tq3_value_quad<DEFER>(acc.o[4 * j], acc.o[4 * j + 1], acc.o[4 * j + 2], acc.o[4 * j + 3], vw[3 * j], vw[3 * j + 1],
                                   vw[3 * j + 2], meta + j * 256, pf);
     }
-    if constexpr (DO_K) {
+    if constexpr (DO_K && FMT == 2) {
+        // head g, tokens 2tq, 2tq+1 (I0 | I1) and 2tq+8, 2tq+9 (I2 | I3): the three query digits, then the token's
+        // norm correction
+        const int tq = lane & 3;
+        const uint32_t gaddr = rec_k + 12 * D + 4 * tq;
+        const float2 ga = half2_to_float2(lds32(gaddr)), gb = half2_to_float2(lds32(gaddr + 16));
+        // (sc2 carries the head's digit unit delta_h / 8 here)
+        s_next[0] = digits_to_score(I0[0], I0[2], I1[0]) * (ga.x * sc2);
+        s_next[1] = digits_to_score(I0[1], I0[3], I1[1]) * (ga.y * sc2);
+        s_next[2] = digits_to_score(I2[0], I2[2], I3[0]) * (gb.x * sc2);
+        s_next[3] = digits_to_score(I2[1], I2[3], I3[1]) * (gb.y * sc2);
+    }
+    if constexpr (DO_K && FMT == 1) {
         const uint32_t gaddr = rec_k + 12 * D;
         const float r0 = __half2float(__ushort_as_half(lds16(gaddr + 2 * g))) * sc2;
         const float r1 = __half2float(__ushort_as_half(lds16(gaddr + 2 * g + 16))) * sc2;
@@ -830,7 +983,7 @@ __device__ __forceinline__ void merge_row(const DecodeParams& P, int first_slot,
         P.lse[(size_t)b * hq + h * GQ + tid] = ml_s[8 + tid] > 0.f ? (ml_s[tid] + log2f(ml_s[8 + tid])) * kLn2 : -CUDART_INF_F;
 }
 
-template <int D, int NW, int NSTAGE, int MINB, bool SCORED, bool TILED, int MAXL>
+template <int D, int NW, int NSTAGE, int MINB, bool SCORED, bool TILED, int MAXL, int FMT>
 __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const LayerSet<MAXL> LS)
 {
     const DecodeParams& P0 = LS.layer[0];    // requests and geometry are common to all layers
@@ -1128,6 +1281,7 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Laye
         for (int i = 0; i < NB; ++i) acc.o[i][0] = acc.o[i][1] = acc.o[i][2] = acc.o[i][3] = 0.f;
         acc.l[0] = acc.l[1] = 0.f;
         acc.m[0] = acc.m[1] = -CUDART_INF_F;
+        acc.mr = -CUDART_INF_F;
 
         // first round: start the copies, then build the query fragments while they fly
         const int n_rounds = (n_my + G::ROUND - 1) / G::ROUND;
@@ -1166,10 +1320,42 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Laye
             const float rs = rsqrtf((float)D);
             __half* qt = reinterpret_cast<__half*>(smem + G::OFF_QT);
             __half* qf = reinterpret_cast<__half*>(smem + G::OFF_QF);
+            if constexpr (FMT == 2) {
+                // rotated query as three balanced base-128 digits in the A-fragment order of the integer key
+                // products: dim i sits in step i/32 at K slot k = i%32 of fragment lane 4 hd + (k%16)/4, byte k%4;
+                // digits 0,1 in registers 2 (k/16) + digit of the step's first 512 bytes, digit 2 in register k/16 of
+                // the second 512 bytes (16 bytes per lane, the upper eight unused)
+                uint8_t* qt8 = smem + G::OFF_QT;
+                float amax = 0.f;
+#pragma unroll
+                for (int r = 0; r < EPL; ++r) amax = fmaxf(amax, fabsf(a[r] * rs));
+#pragma unroll
+                for (int m = 16; m > 0; m >>= 1) amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, m));
+                const float delta = amax > 0.f ? amax * (1.f / (63.f * 16384.f)) : 1.f, inv_delta = 1.f / delta;
+                if (lane == 0) reinterpret_cast<float*>(smem + G::OFF_QS)[hd] = delta * 0.125f;   // key levels are eighths
+#pragma unroll
+                for (int r0 = 0; r0 < EPL; r0 += 4) {
+                    uint32_t word[3] = {0u, 0u, 0u};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int Q = __float2int_rn(a[r0 + e] * rs * inv_delta);
+                        const int t2 = ((Q + 64) & 127) - 64, Q1 = (Q - t2) >> 7;
+                        const int t1 = ((Q1 + 64) & 127) - 64, t0 = (Q1 - t1) >> 7;
+                        word[0] |= (uint32_t)(t0 & 0xFF) << (8 * e);
+                        word[1] |= (uint32_t)(t1 & 0xFF) << (8 * e);
+                        word[2] |= (uint32_t)(t2 & 0xFF) << (8 * e);
+                    }
+                    const int i0 = lane * EPL + r0, st = i0 >> 5, k = i0 & 31;
+                    const int L = 4 * hd + ((k & 15) >> 2);
+                    *reinterpret_cast<uint32_t*>(qt8 + ((st * 2) * 32 + L) * 16 + (2 * (k >> 4)) * 4) = word[0];
+                    *reinterpret_cast<uint32_t*>(qt8 + ((st * 2) * 32 + L) * 16 + (2 * (k >> 4) + 1) * 4) = word[1];
+                    *reinterpret_cast<uint32_t*>(qt8 + ((st * 2 + 1) * 32 + L) * 16 + (k >> 4) * 4) = word[2];
+                }
+            }
 #pragma unroll
             for (int r = 0; r < EPL; ++r) {
                 const int i = lane * EPL + r;
-                {   // rotated query, natural slot order: block i/16, slot s = i%16; per lane {hi b0, hi b1, lo b0, lo b1}
+                if constexpr (FMT == 1) {   // rotated query, natural slot order: block i/16, slot s = i%16; per lane {hi b0, hi b1, lo b0, lo b1}
                     const int kb = i >> 4, s = i & 15;
                     const int at = (kb * 32 + 4 * hd + ((s & 7) >> 1)) * 8 + (s >> 3) * 2 + (s & 1);
                     // fp16 pair hi + lo carries the rotated query to ~2^-22
@@ -1185,6 +1371,8 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Laye
             }
         }
         __syncthreads();
+        // score unit of the Stale pages: record format 2 counts in digit units of this lane's head g
+        const float sc2k = FMT == 2 ? sc2 * reinterpret_cast<const float*>(smem + G::OFF_QS)[g] : sc2;
 
         for (int round = 0; round < n_rounds && !failed; ++round) {
             if (round > 0) {
@@ -1202,12 +1390,13 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Laye
                     cur_lp = lpg3[0] >> 16;
                 }
                 wait_slot(0);
-                if (!failed) tq3_step<D, false, true, TILED>(acc, 0, s_cur, pf, ring, qt_lane, sc2, lane, s_cur);
+                if (!failed) tq3_step<D, false, true, TILED, FMT>(acc, 0, s_cur, pf, ring, qt_lane, sc2k, lane, s_cur);
                 for (int i = 0; i + 1 < n3 && !failed; ++i) {
                     const uint32_t cur = (uint32_t)i % NSTAGE, nxt = (uint32_t)(i + 1) % NSTAGE;
                     wait_slot(nxt);
                     if (failed) break;
-                    softmax_rescale<NB, TILED>(acc, s_cur);
+                    if constexpr (FMT == 2) softmax_rescale_v2<NB, TILED>(acc, s_cur, lane);
+                    else softmax_rescale<NB, TILED>(acc, s_cur);
                     if constexpr (TILED) {
                         const int pg_i = list3[i];
                         if (pg_i != cur_page) {
@@ -1216,7 +1405,7 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Laye
                             cur_lp = lpg3[i] >> 16;
                         }
                     }
-                    tq3_step<D, true, true, TILED>(acc, ring + cur * G::SLOT, s_cur, pf, ring + nxt * G::SLOT, qt_lane, sc2, lane, s_next);
+                    tq3_step<D, true, true, TILED, FMT>(acc, ring + cur * G::SLOT, s_cur, pf, ring + nxt * G::SLOT, qt_lane, sc2k, lane, s_next);
                     if constexpr (SCORED && !TILED) store_page_mass<NB>(acc, pf.ps0, pf.ps1, mass_row + lpg3[i], P.max_pages, GQ, lane);
 #pragma unroll
                     for (int e = 0; e < 4; ++e) s_cur[e] = s_next[e];
@@ -1224,7 +1413,8 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Laye
                     if (i + NSTAGE < n3) issue_tq3(i + NSTAGE);
                 }
                 if (!failed) {
-                    softmax_rescale<NB, TILED>(acc, s_cur);
+                    if constexpr (FMT == 2) softmax_rescale_v2<NB, TILED>(acc, s_cur, lane);
+                    else softmax_rescale<NB, TILED>(acc, s_cur);
                     if constexpr (TILED) {
                         const int pg_i = list3[n3 - 1];
                         if (pg_i != cur_page) {
@@ -1233,7 +1423,7 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Laye
                             cur_lp = lpg3[n3 - 1] >> 16;
                         }
                     }
-                    tq3_step<D, true, false, TILED>(acc, ring + ((uint32_t)(n3 - 1) % NSTAGE) * G::SLOT, s_cur, pf, 0, qt_lane, sc2, lane, s_next);
+                    tq3_step<D, true, false, TILED, FMT>(acc, ring + ((uint32_t)(n3 - 1) % NSTAGE) * G::SLOT, s_cur, pf, 0, qt_lane, sc2k, lane, s_next);
                     if constexpr (SCORED && !TILED) store_page_mass<NB>(acc, pf.ps0, pf.ps1, mass_row + lpg3[n3 - 1], P.max_pages, GQ, lane);
                     if constexpr (TILED) fold(cur_page, true, cur_lp);   // back to output units for the FP8 pages and the reduction
                 }
@@ -1252,6 +1442,7 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Laye
                     fp8_page<D, SCORED, TILED>(acc, ring + s * G::SLOT, ring + (s + 1) * G::SLOT, qf_lane, sc2 * P.k_scale, P.v_scale,
                                                valid ? valid : kPage, lane,
                                                SCORED ? mass_row + (TILED ? (lpg8[i] >> 16) : lpg8[i]) : nullptr, P.max_pages, GQ);
+                    if constexpr (FMT == 2) max_rows_from_columns<NB>(acc, lane);     // the page may have raised the maxima
                     __syncwarp();
                     if (i + NSTAGE / 2 < n8) issue_fp8(i + NSTAGE / 2);
                 }
@@ -1418,11 +1609,11 @@ static int32_t run_tmem(mkv_pool* p, DecodeParams& prm, cudaStream_t s)
     return MKV_OK;
 }
 
-template <int D, int NW, int NSTAGE, int MINB, bool SCORED = false, bool TILED = false, int MAXL = 1>
-static int32_t run_tensor(mkv_pool* p, const LayerSet<MAXL>& ls, cudaStream_t s)
+template <int D, int NW, int NSTAGE, int MINB, bool SCORED, bool TILED, int MAXL, int FMT>
+static int32_t run_tensor_fmt(mkv_pool* p, const LayerSet<MAXL>& ls, cudaStream_t s)
 {
     using G = Geo<D, NW, NSTAGE, TILED>;
-    auto kern = decode_tensor_kernel<D, NW, NSTAGE, MINB, SCORED, TILED, MAXL>;
+    auto kern = decode_tensor_kernel<D, NW, NSTAGE, MINB, SCORED, TILED, MAXL, FMT>;
     // pages of several tiles: one row of parked accumulators (8 D floats) per warp behind the usual layout
     constexpr int SMEM = G::SMEM + (TILED ? NW * 8 * D * 4 : 0);
     static_assert(SMEM <= 232448, "dynamic shared memory of one block");
@@ -1452,6 +1643,14 @@ static int32_t run_tensor(mkv_pool* p, const LayerSet<MAXL>& ls, cudaStream_t s)
     kern<<<grid, NW * 32, SMEM, s>>>(ls);
     MKV_CUDA(cudaGetLastError());
     return MKV_OK;
+}
+
+// the pool's record format selects the instantiation
+template <int D, int NW, int NSTAGE, int MINB, bool SCORED = false, bool TILED = false, int MAXL = 1>
+static int32_t run_tensor(mkv_pool* p, const LayerSet<MAXL>& ls, cudaStream_t s)
+{
+    return p->fmt == 2 ? run_tensor_fmt<D, NW, NSTAGE, MINB, SCORED, TILED, MAXL, 2>(p, ls, s)
+                       : run_tensor_fmt<D, NW, NSTAGE, MINB, SCORED, TILED, MAXL, 1>(p, ls, s);
 }
 
 template <int D, int NW, int NSTAGE, int MINB, bool SCORED = false, bool TILED = false>
@@ -1595,10 +1794,6 @@ int32_t launch_decode_tensor_layers(mkv_pool* const* pools, const void* const* q
         ls.layer[i] = make_params(pools[i], q[i], bt[i], tags[i], lens, B, max_pages, scale, out[i], lse ? lse[i] : nullptr,
                                   partials, tickets, kMaxCtas, nullptr);
     }
-#ifdef MKV_SHAPE_2X4
-    return p0->d == 128 ? run_tensor<128, 12, 4, 1, false, false, kMaxLayers>(p0, ls, s)
-                        : run_tensor<256, 4, 4, 2, false, false, kMaxLayers>(p0, ls, s);
-#endif
     return p0->d == 128 ? run_tensor<128, 12, 4, 1, false, false, kMaxLayers>(p0, ls, s)
                         : run_tensor<256, 8, 4, 1, false, false, kMaxLayers>(p0, ls, s);
 }
@@ -1614,6 +1809,10 @@ int32_t launch_decode_tensor_at(mkv_pool* p, const void* q, const int32_t* bt, c
     }
     if (p->tiles > 1 && p->variant == MKV_DECODE_TMEM) {
         set_last_error("mkv_decode_attention: pages of several tiles are served by the tensor-core kernel");
+        return MKV_E_INVALID;
+    }
+    if (p->fmt == 2 && p->variant == MKV_DECODE_TMEM) {
+        set_last_error("mkv_decode_attention: record format 2 is served by the tensor-core and the CUDA-core kernels");
         return MKV_E_INVALID;
     }
     DecodeParams prm = make_params(p, q, bt, tags, lens, B, max_pages, scale, out, lse, partials, tickets, max_blocks, mass);

@@ -301,18 +301,25 @@ __device__ __forceinline__ float2 e4m3x2_to_f32(uint32_t two_bytes)
 // nibble pairs of two bytes -> one byte: (x & 0x000F) | ((x & 0x0F00) >> 4)
 __device__ __forceinline__ uint32_t squeeze_nibbles(uint32_t x) { return (x & 0xFu) | ((x >> 4) & 0xF0u); }
 
-// Constants of the key encoder that depend only on the lane.
-template <int D>
+// four code bytes -> four nibbles
+__device__ __forceinline__ uint32_t squeeze4(uint32_t x)
+{
+    return (x & 0xFu) | ((x >> 4) & 0xF0u) | ((x >> 8) & 0xF00u) | ((x >> 12) & 0xF000u);
+}
+
+// Constants of the key encoder that depend only on the lane (FMT: the record format's codebook).
+template <int D, int FMT>
 struct DemoteLane {
     float c0sq, c1sq, c2sq, c3sq;     // squared levels (single fp32 products, as the record's norm correction defines them)
     uint32_t flip[D / 32];            // rotation signs of this lane's key elements, as fp32 sign-bit masks
     uint32_t neg[5];                  // butterfly stage m: lanes with bit m set subtract
     __device__ __forceinline__ void init(const SigmaBits& sigma, int lane)
     {
-        c0sq = __fmul_rn(MKV_C0, MKV_C0);
-        c1sq = __fmul_rn(MKV_C1, MKV_C1);
-        c2sq = __fmul_rn(MKV_C2, MKV_C2);
-        c3sq = __fmul_rn(MKV_C3, MKV_C3);
+        using CB = KeyCodebook<FMT>;
+        c0sq = __fmul_rn(CB::C0, CB::C0);
+        c1sq = __fmul_rn(CB::C1, CB::C1);
+        c2sq = __fmul_rn(CB::C2, CB::C2);
+        c3sq = __fmul_rn(CB::C3, CB::C3);
 #pragma unroll
         for (int r = 0; r < D / 32; ++r) {
             const int i = lane * (D / 32) + r;
@@ -326,11 +333,12 @@ struct DemoteLane {
 // Encodes the 16 tokens of one FP8 record (rec8) into the record image img = [key codes | value codes | g |
 // scale/zero] in shared memory; all D threads of the block call it.  OWN_META: the value scale and zero come
 // from these 16 tokens (16-token pages); otherwise thread c passes the page's scale/zero of channel c.
-template <int D, bool OWN_META>
+template <int D, bool OWN_META, int FMT>
 __device__ __forceinline__ void demote_tile(const uint8_t* __restrict__ rec8, uint8_t* img, uint8_t* kcode, uint8_t* vcode,
-                                            const DemoteLane<D>& K, float k_scale, float v_scale, uint16_t sc_page,
+                                            const DemoteLane<D, FMT>& K, float k_scale, float v_scale, uint16_t sc_page,
                                             uint16_t zp_page)
 {
+    using CB = KeyCodebook<FMT>;
     constexpr int EPL = D / 32, NJ = D / 64, KROW = D + 8, NT = D;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const float c0sq = K.c0sq, c1sq = K.c1sq, c2sq = K.c2sq, c3sq = K.c3sq;
@@ -385,7 +393,7 @@ __device__ __forceinline__ void demote_tile(const uint8_t* __restrict__ rec8, ui
 #pragma unroll
         for (int m = 1; m < 32; m <<= 1) n2 = __fadd_rn(n2, __shfl_xor_sync(0xffffffffu, n2, m));
         const float nx = __fsqrt_rn(n2);
-        const float t1 = __fmul_rn(MKV_B0, nx), t2 = __fmul_rn(MKV_B1, nx), t3 = __fmul_rn(MKV_B2, nx);
+        const float t1 = __fmul_rn(CB::B0, nx), t2 = __fmul_rn(CB::B1, nx), t3 = __fmul_rn(CB::B2, nx);
         float f[EPL];
         uint32_t packed[EPL / 4];
 #pragma unroll
@@ -470,7 +478,21 @@ __device__ __forceinline__ void demote_tile(const uint8_t* __restrict__ rec8, ui
         const int L = item & 31, j = (item >> 5) % NJ, section = item / (32 * NJ);
         const int g = L >> 2, tq = L & 3;
         uint32_t w0 = 0, w1 = 0, w2 = 0;
-        if (section == 0) {
+        if (section == 0 && FMT == 2) {
+            // record format 2: register e = 4 (step % 2) + 2 u + b of the triple holds, in its four nibbles, the
+            // codes of token g + 8u at dims 32 step + 16 b + 4 tq .. + 3 (steps 2j, 2j+1).  A: registers 0,1 with
+            // the signs of 4,5; B: registers 2,3 with the signs of 6,7; C: magnitudes of 4,5 (low pair), 6,7 (high).
+            uint32_t x[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+                x[e] = *reinterpret_cast<const uint32_t*>(kcode + (g + 8 * ((e >> 1) & 1)) * KROW + 32 * (2 * j + (e >> 2)) +
+                                                          16 * (e & 1) + 4 * tq);
+            auto signs = [](uint32_t v) { return squeeze4((v >> 2) & 0x01010101u) << 3; };
+            auto mags = [](uint32_t v) { return squeeze4(v & 0x03030303u); };
+            w0 = squeeze4(x[0]) | (squeeze4(x[1]) << 16) | signs(x[4]) | (signs(x[5]) << 16);
+            w1 = squeeze4(x[2]) | (squeeze4(x[3]) << 16) | signs(x[6]) | (signs(x[7]) << 16);
+            w2 = mags(x[4]) | (mags(x[5]) << 16) | ((mags(x[6]) | (mags(x[7]) << 16)) << 2);
+        } else if (section == 0) {
             // key codes: nibble n = 2r + half holds row g + 8(r&1), slot 2tq + 8(r>>1) + half.
             // A: block 4j with the signs of block 4j+2; B: block 4j+1 with the signs of 4j+3;
             // C: magnitudes of blocks 4j+2 (low pair) and 4j+3 (high pair).
@@ -511,7 +533,7 @@ __device__ __forceinline__ void demote_tile(const uint8_t* __restrict__ rec8, ui
     __syncthreads();
 }
 
-template <int D, bool BIG>
+template <int D, bool BIG, int FMT>
 __global__ void __launch_bounds__(D) demote_kernel(const uint8_t* __restrict__ fp8, uint8_t* __restrict__ tq3,
                                                       int fp8_pages, int tq3_pages, int hkv, int tiles, float k_scale,
                                                       float v_scale, SigmaBits sigma,
@@ -532,7 +554,7 @@ __global__ void __launch_bounds__(D) demote_kernel(const uint8_t* __restrict__ f
     const int src = src_ids[page], dst = dst_ids[page];
     const bool valid = src >= 0 && src < fp8_pages && dst >= 0 && dst < tq3_pages;
     if (!valid && tid == 0 && crank == 0 && blockIdx.y == 0) atomicOr(status, kStBounds);
-    DemoteLane<D> lane_consts;
+    DemoteLane<D, FMT> lane_consts;
     lane_consts.init(sigma, lane);
 
     int it = 0;
@@ -541,7 +563,7 @@ __global__ void __launch_bounds__(D) demote_kernel(const uint8_t* __restrict__ f
             const uint8_t* rec8 = fp8 + ((size_t)src * hkv + h) * fp8_record_bytes(D);
             uint8_t* rec3 = tq3 + ((size_t)dst * hkv + h) * tq3_record_bytes(D);
             uint8_t* img = image[it++ & 1];
-            demote_tile<D, true>(rec8, img, kcode, vcode, lane_consts, k_scale, v_scale, 0, 0);
+            demote_tile<D, true, FMT>(rec8, img, kcode, vcode, lane_consts, k_scale, v_scale, 0, 0);
             for (int i = tid; i < REC / 16; i += NT)
                 reinterpret_cast<uint4*>(rec3)[i] = reinterpret_cast<const uint4*>(img)[i];
         } else {
@@ -556,7 +578,7 @@ __global__ void __launch_bounds__(D) demote_kernel(const uint8_t* __restrict__ f
             for (int m = blockIdx.y; m < tiles; m += gridDim.y) {
                 const uint8_t* rec8 = fp8 + (((size_t)src * hkv + h) * tiles + m) * fp8_record_bytes(D);
                 uint8_t* img = image[it++ & 1];
-                demote_tile<D, false>(rec8, img, kcode, vcode, lane_consts, k_scale, v_scale, sc, zp);
+                demote_tile<D, false, FMT>(rec8, img, kcode, vcode, lane_consts, k_scale, v_scale, sc, zp);
                 uint4* out = reinterpret_cast<uint4*>(page3 + (size_t)m * TILE);
                 for (int i = tid; i < TILE / 16; i += NT) out[i] = reinterpret_cast<const uint4*>(img)[i];
             }
@@ -680,13 +702,13 @@ static cudaError_t launch_clustered_rows(Kernel kernel, int n_pages, int csize, 
     return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
-template <int D>
+template <int D, int FMT>
 static int32_t launch_demote_d(mkv_pool* p, const int32_t* src, const int32_t* dst, int n, int32_t* bt, uint8_t* tags,
                                const int64_t* entry, cudaStream_t s)
 {
     const int c = heads_cluster(p->hkv, n);
     if (p->tiles == 1) {
-        MKV_CUDA(launch_clustered(demote_kernel<D, false>, n, c, D, s, (const uint8_t*)p->fp8, p->tq3, p->cfg.fp8_pages,
+        MKV_CUDA(launch_clustered(demote_kernel<D, false, FMT>, n, c, D, s, (const uint8_t*)p->fp8, p->tq3, p->cfg.fp8_pages,
                                   p->cfg.tq3_pages, p->hkv, 1, p->cfg.k_scale, p->cfg.v_scale, p->sigma, src, dst, bt,
                                   tags, entry, p->status_dev));
         return MKV_OK;
@@ -695,7 +717,7 @@ static int32_t launch_demote_d(mkv_pool* p, const int32_t* src, const int32_t* d
     demote_minmax_kernel<D><<<n * p->hkv, 1024, 0, s>>>(p->fp8, p->tq3, p->cfg.fp8_pages, p->cfg.tq3_pages, p->hkv, p->tiles,
                                                      p->cfg.v_scale, src, dst);
     MKV_CUDA(cudaGetLastError());
-    MKV_CUDA(launch_clustered_rows(demote_kernel<D, true>, n, heads_cluster(p->hkv, 0), tile_rows(p->tiles, n, p->hkv), D, s,
+    MKV_CUDA(launch_clustered_rows(demote_kernel<D, true, FMT>, n, heads_cluster(p->hkv, 0), tile_rows(p->tiles, n, p->hkv), D, s,
                                    (const uint8_t*)p->fp8, p->tq3, p->cfg.fp8_pages, p->cfg.tq3_pages, p->hkv, p->tiles,
                                    p->cfg.k_scale, p->cfg.v_scale, p->sigma, src, dst, (int32_t*)nullptr,
                                    (uint8_t*)nullptr, (const int64_t*)nullptr, p->status_dev));
@@ -711,8 +733,11 @@ static int32_t launch_demote_d(mkv_pool* p, const int32_t* src, const int32_t* d
 int32_t launch_demote(mkv_pool* p, const int32_t* src, const int32_t* dst, int n, int32_t* bt, uint8_t* tags,
                       const int64_t* entry, cudaStream_t s)
 {
-    return p->d == 128 ? launch_demote_d<128>(p, src, dst, n, bt, tags, entry, s)
-                       : launch_demote_d<256>(p, src, dst, n, bt, tags, entry, s);
+    if (p->fmt == 2)
+        return p->d == 128 ? launch_demote_d<128, 2>(p, src, dst, n, bt, tags, entry, s)
+                           : launch_demote_d<256, 2>(p, src, dst, n, bt, tags, entry, s);
+    return p->d == 128 ? launch_demote_d<128, 1>(p, src, dst, n, bt, tags, entry, s)
+                       : launch_demote_d<256, 1>(p, src, dst, n, bt, tags, entry, s);
 }
 
 // ------------------------------------------------------------------------------------------ promote
@@ -726,7 +751,7 @@ int32_t launch_demote(mkv_pool* p, const int32_t* src, const int32_t* dst, int n
 // L = 4 (row % 8) + (slot % 8) / 2 holds, in nibble 2 rr + slot % 2 with rr = row / 8 + 2 (slot / 8),
 // the entry (row, slot) of every 16 x 16 block; for keys row = token and slot = channel % 16, for
 // values row = channel % 16 and slot = token.
-template <int D, bool BIG>
+template <int D, bool BIG, int FMT>
 __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ tq3, uint8_t* __restrict__ fp8,
                                                      int tq3_pages, int fp8_pages, int hkv, int tiles, float inv_k_scale,
                                                      float inv_v_scale, float rs, SigmaBits sigma,
@@ -747,7 +772,8 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
     const bool valid = src >= 0 && src < tq3_pages && dst >= 0 && dst < fp8_pages;
     if (!valid && tid == 0 && crank == 0 && blockIdx.y == 0) atomicOr(status, kStBounds);
     if (tid < 8) {
-        const float c = (tid & 3) == 0 ? MKV_C0 : (tid & 3) == 1 ? MKV_C1 : (tid & 3) == 2 ? MKV_C2 : MKV_C3;
+        using CB = KeyCodebook<FMT>;
+        const float c = (tid & 3) == 0 ? CB::C0 : (tid & 3) == 1 ? CB::C1 : (tid & 3) == 2 ? CB::C2 : CB::C3;
         level[tid] = (tid & 4) ? -c : c;
     }
     // ---- per-lane constants of the key path: this lane rebuilds channels lane*EPL .. +EPL-1
@@ -804,8 +830,27 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
         // ---- keys: warp w rebuilds tokens w, w + NT/32, ...
         for (int tok = warp; tok < kPage; tok += NT / 32) {
             float y[EPL];
+            if constexpr (FMT == 2) {
+                // record format 2: four consecutive dims are the nibbles of one half-word of register
+                // e = 4 (step % 2) + 2 (token / 8) + (k / 16) in the triple step / 2 of fragment lane 4 (token % 8) + (k % 16) / 4
 #pragma unroll
-            for (int r2 = 0; r2 < EPL; r2 += 2) {
+                for (int gi = 0; gi < EPL / 4; ++gi) {
+                    const int i0 = lane * EPL + 4 * gi, st = i0 >> 5, k = i0 & 31, j = st >> 1;
+                    const int e = 4 * (st & 1) + 2 * (tok >> 3) + (k >> 4), L = 4 * (tok & 7) + ((k & 15) >> 2), sh = 16 * (e & 1);
+                    const uint32_t A = *reinterpret_cast<const uint32_t*>(img + lane_word_offset(D, L, 3 * j));
+                    const uint32_t Bw = *reinterpret_cast<const uint32_t*>(img + lane_word_offset(D, L, 3 * j + 1));
+                    const uint32_t Cw = *reinterpret_cast<const uint32_t*>(img + lane_word_offset(D, L, 3 * j + 2));
+                    uint32_t nib;
+                    if (e < 2) nib = (A >> sh) & 0x7777u;
+                    else if (e < 4) nib = (Bw >> sh) & 0x7777u;
+                    else if (e < 6) nib = ((Cw >> sh) & 0x3333u) | ((A >> (sh + 1)) & 0x4444u);
+                    else nib = ((Cw >> (sh + 2)) & 0x3333u) | ((Bw >> (sh + 1)) & 0x4444u);
+#pragma unroll
+                    for (int x = 0; x < 4; ++x) y[4 * gi + x] = level[(nib >> (4 * x)) & 7u];
+                }
+            }
+#pragma unroll
+            for (int r2 = 0; r2 < (FMT == 2 ? 0 : EPL); r2 += 2) {
                 const int s = s0 + r2;                                    // even slot; s + 1 shares the word
                 const int L = 4 * (tok & 7) + ((s & 7) >> 1), n = 2 * ((tok >> 3) + 2 * (s >> 3));
                 const uint32_t ws = *reinterpret_cast<const uint32_t*>(img + off_sgn + L * str_sgn) >> (4 * n);
@@ -888,19 +933,19 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
     }
 }
 
-template <int D>
+template <int D, int FMT>
 static int32_t launch_promote_d(mkv_pool* p, const int32_t* src, const int32_t* dst, int n, int32_t* bt, uint8_t* tags,
                                 const int64_t* entry, cudaStream_t s)
 {
     const float ik = 1.0f / p->cfg.k_scale, iv = 1.0f / p->cfg.v_scale;
     const float rs = (float)(1.0 / sqrt((double)p->d));
     if (p->tiles == 1) {
-        MKV_CUDA(launch_clustered(promote_kernel<D, false>, n, heads_cluster(p->hkv, n), D, s, (const uint8_t*)p->tq3, p->fp8,
+        MKV_CUDA(launch_clustered(promote_kernel<D, false, FMT>, n, heads_cluster(p->hkv, n), D, s, (const uint8_t*)p->tq3, p->fp8,
                                   p->cfg.tq3_pages, p->cfg.fp8_pages, p->hkv, 1, ik, iv, rs, p->sigma, src, dst, bt, tags,
                                   entry, p->status_dev));
         return MKV_OK;
     }
-    MKV_CUDA(launch_clustered_rows(promote_kernel<D, true>, n, heads_cluster(p->hkv, 0), tile_rows(p->tiles, n, p->hkv), D, s,
+    MKV_CUDA(launch_clustered_rows(promote_kernel<D, true, FMT>, n, heads_cluster(p->hkv, 0), tile_rows(p->tiles, n, p->hkv), D, s,
                                    (const uint8_t*)p->tq3, p->fp8, p->cfg.tq3_pages, p->cfg.fp8_pages, p->hkv, p->tiles, ik,
                                    iv, rs, p->sigma, src, dst, (int32_t*)nullptr, (uint8_t*)nullptr,
                                    (const int64_t*)nullptr, p->status_dev));
@@ -915,8 +960,11 @@ static int32_t launch_promote_d(mkv_pool* p, const int32_t* src, const int32_t* 
 int32_t launch_promote(mkv_pool* p, const int32_t* src, const int32_t* dst, int n, int32_t* bt, uint8_t* tags,
                        const int64_t* entry, cudaStream_t s)
 {
-    return p->d == 128 ? launch_promote_d<128>(p, src, dst, n, bt, tags, entry, s)
-                       : launch_promote_d<256>(p, src, dst, n, bt, tags, entry, s);
+    if (p->fmt == 2)
+        return p->d == 128 ? launch_promote_d<128, 2>(p, src, dst, n, bt, tags, entry, s)
+                           : launch_promote_d<256, 2>(p, src, dst, n, bt, tags, entry, s);
+    return p->d == 128 ? launch_promote_d<128, 1>(p, src, dst, n, bt, tags, entry, s)
+                       : launch_promote_d<256, 1>(p, src, dst, n, bt, tags, entry, s);
 }
 
 // ------------------------------------------------------------------------------------------ anchor

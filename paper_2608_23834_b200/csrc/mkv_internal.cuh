@@ -27,6 +27,19 @@ constexpr uint32_t kStBounds = 1u, kStState = 2u, kStTimeout = 4u;
 #define MKV_B1 1.0498046875f
 #define MKV_B2 1.748046875f
 
+// Record format 2: the same quantiser with its levels on the nearest e4m3 numbers (0.25, 0.75, 1.375, 2.25), so
+// that a reader feeds the codes to FP8 arithmetic exactly; thresholds are again the midpoints.
+template <int FMT>
+struct KeyCodebook {
+    static constexpr float C0 = MKV_C0, C1 = MKV_C1, C2 = MKV_C2, C3 = MKV_C3;
+    static constexpr float B0 = MKV_B0, B1 = MKV_B1, B2 = MKV_B2;
+};
+template <>
+struct KeyCodebook<2> {
+    static constexpr float C0 = 0.25f, C1 = 0.75f, C2 = 1.375f, C3 = 2.25f;
+    static constexpr float B0 = 0.5f, B1 = 1.0625f, B2 = 1.8125f;
+};
+
 struct SigmaBits {
     uint32_t w[8];   // bit i set <=> rotation sign of dim i is -1
 };
@@ -64,6 +77,7 @@ struct mkv_pool {
     mkv_pool_config cfg;
     int d, hkv, hq, group;
     int tiles;                   // 16-token tiles per page (cfg.page_size / 16)
+    int fmt;                     // TQ3 record format: 1 or 2 (cfg.tq3_format, 0 meaning 1)
     uint8_t* fp8;
     uint8_t* tq3;
     uint32_t* status_dev;

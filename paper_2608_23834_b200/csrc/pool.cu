@@ -31,6 +31,7 @@ static int32_t check_cfg(const mkv_pool_config* c)
     if (c->n_q_heads / c->n_kv_heads > kMaxGroup) return MKV_E_INVALID;
     if (c->fp8_pages < 0 || c->tq3_pages < 0) return MKV_E_INVALID;
     if (!(c->k_scale > 0.f) || !(c->v_scale > 0.f)) return MKV_E_INVALID;
+    if (c->tq3_format < 0 || c->tq3_format > 2) return MKV_E_INVALID;
     return MKV_OK;
 }
 
@@ -106,6 +107,7 @@ static mkv_pool* new_pool(const mkv_pool_config* cfg, void* fp8_arena, void* tq3
     p->hq = cfg->n_q_heads;
     p->group = cfg->n_q_heads / cfg->n_kv_heads;
     p->tiles = cfg->page_size / kPage;
+    p->fmt = cfg->tq3_format == 2 ? 2 : 1;
     p->fp8 = static_cast<uint8_t*>(fp8_arena);
     p->tq3 = static_cast<uint8_t*>(tq3_arena);
     p->variant = MKV_DECODE_TENSOR;
@@ -351,8 +353,8 @@ int32_t mkv_decode_attention_layers(const mkv_layer_call* L, int32_t n_layers, c
             return MKV_E_INVALID;
         const mkv_pool* p0 = L[0].pool;
         if (c.pool->d != p0->d || c.pool->hkv != p0->hkv || c.pool->hq != p0->hq || c.pool->tiles != 1 ||
-            c.pool->device != p0->device || c.pool->variant != MKV_DECODE_TENSOR) {
-            set_last_error("mkv_decode_attention_layers: pools of one geometry, 16-token pages, one device and the tensor-core variant");
+            c.pool->device != p0->device || c.pool->variant != MKV_DECODE_TENSOR || c.pool->fmt != p0->fmt) {
+            set_last_error("mkv_decode_attention_layers: pools of one geometry, record format, 16-token pages, one device and the tensor-core variant");
             return MKV_E_INVALID;
         }
         for (int j = 0; j < i; ++j)

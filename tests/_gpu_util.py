@@ -22,9 +22,11 @@ class Case:
         self.spec = spec
         self.tab = W.tables(spec, extra_fp8, extra_tq3)
         self.L = build_layer(spec, self.tab, layer, requests=requests)
+        # the pool reads its Stale pages in the record format the oracle wrote them in
+        self.fmt = oracle.get_format()
         self.pool = M.Pool(spec.head_dim, spec.n_kv_heads, spec.n_q_heads, max(self.tab.fp8_pages, 1),
                            max(self.tab.tq3_pages, 1), self.L.sigma, k_scale, v_scale, max_batch=spec.batch,
-                           page_tokens=spec.page_tokens)
+                           page_tokens=spec.page_tokens, tq3_format=self.fmt)
         self.pool.upload_arenas(self.L.fp8_arena, self.L.tq3_arena)
         self.q = bf16_tensor(self.L.q_bits)
         self.bt = torch.from_numpy(self.tab.block_table).cuda()
@@ -41,6 +43,7 @@ class Case:
 
     def reference(self, only_b=-1, only_h=-1):
         s = self.spec
+        assert oracle.get_format() == self.fmt
         return oracle.decode_attention(self.L.fp8_arena, self.L.tq3_arena, s.head_dim, s.n_kv_heads, s.group,
                                        self.L.sigma, self.L.q_bits, self.tab.block_table, self.tab.tier_tag,
                                        self.tab.seq_lens, s.scale, only_b=only_b, only_h=only_h,
