@@ -670,12 +670,13 @@ __device__ __forceinline__ void tq3_key_pair_v2(int (&Sa0)[4], int (&Sb0)[4], in
     }
 #pragma unroll
     for (int st = 0; st < 2; ++st) {
-        const uint4 qa = lds128(q_pair + st * 1024);
-        const uint2 qb = lds64(q_pair + st * 1024 + 512);
+        // (the second fragment's rows 8-15 are stored as zeros: a full 16-byte load keeps the four operand
+        // registers together, where building {x, 0, y, 0} cost two moves per MMA)
+        const uint4 qa = lds128(q_pair + st * 1024), qb = lds128(q_pair + st * 1024 + 512);
         mma16832_s8(Sa0, qa.x, qa.y, qa.z, qa.w, r[4 * st], r[4 * st + 1]);
-        mma16832_s8(Sb0, qb.x, 0u, qb.y, 0u, r[4 * st], r[4 * st + 1]);
+        mma16832_s8(Sb0, qb.x, qb.y, qb.z, qb.w, r[4 * st], r[4 * st + 1]);
         mma16832_s8(Sa1, qa.x, qa.y, qa.z, qa.w, r[4 * st + 2], r[4 * st + 3]);
-        mma16832_s8(Sb1, qb.x, 0u, qb.y, 0u, r[4 * st + 2], r[4 * st + 3]);
+        mma16832_s8(Sb1, qb.x, qb.y, qb.z, qb.w, r[4 * st + 2], r[4 * st + 3]);
     }
 }
 
@@ -1323,8 +1324,8 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Laye
             if constexpr (FMT == 2) {
                 // rotated query as three balanced base-128 digits in the A-fragment order of the integer key
                 // products: dim i sits in step i/32 at K slot k = i%32 of fragment lane 4 hd + (k%16)/4, byte k%4;
-                // digits 0,1 in registers 2 (k/16) + digit of the step's first 512 bytes, digit 2 in register k/16 of
-                // the second 512 bytes (16 bytes per lane, the upper eight unused)
+                // digits 0,1 in registers 2 (k/16) + digit of the step's first 512 bytes, digit 2 in register 2 (k/16)
+                // of the second 512 bytes, whose odd registers (fragment rows 8-15) are zero
                 uint8_t* qt8 = smem + G::OFF_QT;
                 float amax = 0.f;
 #pragma unroll
@@ -1349,7 +1350,7 @@ __global__ void __launch_bounds__(NW * 32, MINB) decode_tensor_kernel(const Laye
                     const int L = 4 * hd + ((k & 15) >> 2);
                     *reinterpret_cast<uint32_t*>(qt8 + ((st * 2) * 32 + L) * 16 + (2 * (k >> 4)) * 4) = word[0];
                     *reinterpret_cast<uint32_t*>(qt8 + ((st * 2) * 32 + L) * 16 + (2 * (k >> 4) + 1) * 4) = word[1];
-                    *reinterpret_cast<uint32_t*>(qt8 + ((st * 2 + 1) * 32 + L) * 16 + (k >> 4) * 4) = word[2];
+                    *reinterpret_cast<uint2*>(qt8 + ((st * 2 + 1) * 32 + L) * 16 + (k >> 4) * 8) = make_uint2(word[2], 0u);
                 }
             }
 #pragma unroll
