@@ -128,6 +128,14 @@ __device__ __forceinline__ void mma16832_s8(int (&c)[4], uint32_t a0, uint32_t a
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// the same product with a zero accumulator
+__device__ __forceinline__ void mma16832_s8_zero(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1)
+{
+    asm("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+                 : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(0));
+}
+
 __device__ __forceinline__ uint32_t lds32(uint32_t addr)
 {
     uint32_t v;
@@ -653,6 +661,7 @@ __device__ __forceinline__ void tq3_value_quad(float (&o0)[4], float (&o1)[4], f
 // (step, token half u, K half), then per step and token half one MMA for digits 0,1 and one for digit 2.
 // q_pair: shared-memory address of this lane's query fragments of step 2j (digits 0,1 at +0, digit 2 at +512,
 // step 2j+1 at +1024).
+template <bool FIRST>      // FIRST: the page's first two steps start the four sums
 __device__ __forceinline__ void tq3_key_pair_v2(int (&Sa0)[4], int (&Sb0)[4], int (&Sa1)[4], int (&Sb1)[4],
                                                 uint32_t A, uint32_t Bw, uint32_t Cw, uint32_t q_pair)
 {
@@ -673,6 +682,13 @@ __device__ __forceinline__ void tq3_key_pair_v2(int (&Sa0)[4], int (&Sb0)[4], in
         // (the second fragment's rows 8-15 are stored as zeros: a full 16-byte load keeps the four operand
         // registers together, where building {x, 0, y, 0} cost two moves per MMA)
         const uint4 qa = lds128(q_pair + st * 1024), qb = lds128(q_pair + st * 1024 + 512);
+        if (FIRST && st == 0) {
+            mma16832_s8_zero(Sa0, qa.x, qa.y, qa.z, qa.w, r[0], r[1]);
+            mma16832_s8_zero(Sb0, qb.x, qb.y, qb.z, qb.w, r[0], r[1]);
+            mma16832_s8_zero(Sa1, qa.x, qa.y, qa.z, qa.w, r[2], r[3]);
+            mma16832_s8_zero(Sb1, qb.x, qb.y, qb.z, qb.w, r[2], r[3]);
+            continue;
+        }
         mma16832_s8(Sa0, qa.x, qa.y, qa.z, qa.w, r[4 * st], r[4 * st + 1]);
         mma16832_s8(Sb0, qb.x, qb.y, qb.z, qb.w, r[4 * st], r[4 * st + 1]);
         mma16832_s8(Sa1, qa.x, qa.y, qa.z, qa.w, r[4 * st + 2], r[4 * st + 3]);
@@ -760,7 +776,7 @@ __device__ __forceinline__ void tq3_step(WarpAcc<D / 16>& acc, uint32_t rec_v, c
     const int g = lane >> 2;
     uint32_t kw[LW], vw[LW];
     float S0[4] = {0.f, 0.f, 0.f, 0.f}, S1[4] = {0.f, 0.f, 0.f, 0.f};
-    int I0[4] = {0, 0, 0, 0}, I1[4] = {0, 0, 0, 0}, I2[4] = {0, 0, 0, 0}, I3[4] = {0, 0, 0, 0};   // format 2: (digits 0,1 | 2) x (tokens g | g+8)
+    int I0[4], I1[4], I2[4], I3[4];     // format 2: (digits 0,1 | 2) x (tokens g | g+8), started by the first pair of steps
     if constexpr (DO_K) load_lane_words<D>(rec_k, lane, kw);
     if constexpr (DO_V) load_lane_words<D>(rec_v + 6 * D, lane, vw);
     if constexpr (DO_V) {      // in one block with the key unpack of the next page
@@ -775,7 +791,10 @@ __device__ __forceinline__ void tq3_step(WarpAcc<D / 16>& acc, uint32_t rec_v, c
 #pragma unroll
     for (int j = 0; j < NB / 4; ++j) {
         if constexpr (DO_K) {
-            if constexpr (FMT == 2) tq3_key_pair_v2(I0, I1, I2, I3, kw[3 * j], kw[3 * j + 1], kw[3 * j + 2], qt_lane + j * 2048);
+            if constexpr (FMT == 2) {
+                if (j == 0) tq3_key_pair_v2<true>(I0, I1, I2, I3, kw[0], kw[1], kw[2], qt_lane);
+                else tq3_key_pair_v2<false>(I0, I1, I2, I3, kw[3 * j], kw[3 * j + 1], kw[3 * j + 2], qt_lane + j * 2048);
+            }
             else tq3_key_quad(S0, S1, kw[3 * j], kw[3 * j + 1], kw[3 * j + 2], qt_lane + j * 2048);
         }
         if constexpr (DO_V)
