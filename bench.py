@@ -523,17 +523,9 @@ def run_ours(args):
     result = {
         "metric": METRIC, "value": aggregate_value(B, K, ms, world), "unit": UNIT, "n_gpus": world, "steps": K,
         "warmup": Wm, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": ("u8 codes (e4m3 / 3-bit TQ3); key products e4m3 x e4m3, value products f16 x f16, f32 accumulate" if fmt == 2 else
+        "dtype": ("u8 codes (e4m3 / 3-bit TQ3); Stale key products s8 x s8 -> s32, other products f16 x f16 -> f32" if fmt == 2 else
                   "u8 codes (e4m3 / 3-bit TQ3) -> f16 tensor-core operands, f32 accumulate"), "data": "synthetic",
-        "config": {"workload": workload_name(spec), "batch": B, "context_tokens": list(spec.seq_lens)[:4],
-                   "tq3_record_format": fmt, "layers": spec.n_layers, "head_dim": d, "kv_heads": hkv, "q_heads": hq, "page_tokens": spec.page_tokens,
-                   "parallelism": "replicas only" if world > 1 else "single GPU",
-                   "l2": "inputs larger than L2 (%.0f MB of KV per step)" % (step_bytes / 1e6),
-                   "step": "append + demote at its natural cadence + decode attention, every layer",
-                   "launch": ("one CUDA graph per step holding mkv_append_layers and mkv_decode_attention_layers (all layers in "
-                              "one launch each); retier calls issued directly") if batched else
-                             "one CUDA graph per step (append + decode of every layer); retier calls issued directly",
-                   "layers_per_decode_launch": layers_per_decode_launch},
+        "config": config_dict(spec, args, world, step_bytes, batched, layers_per_decode_launch),
         "eager_ms_per_step": eager_ms / K,
         "kv_gbs_whole_step": step_bytes / (ms / K * 1e-3) / 1e9,
         "roofline": {"bound": "hbm", "kernel": {"tensor": "decode_tensor_kernel", "tmem": "decode_tmem_kernel"}.get(args.variant, "decode_scalar_kernel + merge"), "achieved": achieved, "peak": peak,
@@ -549,7 +541,7 @@ def run_ours(args):
     }
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
-            result["cpu_baseline"] = cpu_baseline(spec)
+            result["cpu_baseline"] = cpu_baseline(spec, fmt)
         print(json.dumps(result))
     if world > 1:
         import torch.distributed as dist
@@ -637,6 +629,94 @@ def run_lifecycle(args):
     }))
 
 
+# ------------------------------------------------------------------------------- lifecycle sweep
+def run_sweep(args):
+    """`--config 4 --sweep`: the 27 cells batch {1, 8, 32} x context {4K, 32K, 128K} x Stale fraction {0, 0.5, 0.95}
+    (head_dim 128, 8 KV x 4 query heads, 16-token pages).  Per cell, each on its own and summed: Append of one
+    token per request, Demote of the page that leaves the Recent window of every request (FP8 -> TQ3 encode),
+    decode attention.  Every repetition starts from a flushed L2 (a 256 MB buffer is rewritten before it) and is
+    timed with a CUDA-event pair on the launching stream; the median is reported with its roofline fraction
+    (bytes the step must move / time / measured copy bandwidth)."""
+    import torch
+    import paper_2608_23834_b200 as M
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    device = torch.device("cuda:%d" % int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(device)
+    M.lib()
+    fmt = 2 if args.format == "v2" else 1
+    peaks, peak_kind = measured_peaks()
+    peak = float(peaks["hbm_gbs"])
+    stream = torch.cuda.current_stream()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+    reps = max(5, min(args.steps, 20))
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        evs = []
+        for _ in range(reps):
+            flush.zero_()                               # L2 (126 MB) holds nothing of the pool afterwards
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn()
+            b.record(stream)
+            evs.append((a, b))
+        torch.cuda.synchronize(device)
+        return statistics.median(x.elapsed_time(y) for x, y in evs) * 1e3        # microseconds
+
+    def entry(us, nbytes, **extra):
+        gbs = nbytes / (us * 1e-6) / 1e9
+        out = {"us": us, "bytes": nbytes, "GB_per_s": gbs, "frac_of_%s_copy_bandwidth" % peak_kind: gbs / peak}
+        out.update(extra)
+        return out
+
+    cells = []
+    with ClockSampler(device.index or 0) as clocks:
+        for B in (1, 8, 32):
+            for ctx in (4096, 32768, 131072):
+                for f in (0.0, 0.5, 0.95):
+                    spec = W.config(4, batch=B, ctx=ctx, stale_fraction=f)
+                    d, hkv, T = spec.head_dim, spec.n_kv_heads, spec.page_tokens
+                    layers, plan, tab0 = build_layers(spec, 4, device, M, torch, fmt)
+                    L = layers[0]
+                    tags_host = initial_tags(tab0, np.zeros((B, plan["max_pages"]), np.uint8))
+                    n_stale = int((tags_host[0] == W.TAG_STALE).sum())
+                    # Demote: the oldest FP8 page of every request into spare TQ3 pages (not published: the table
+                    # stays as it is, so every repetition converts the same pages)
+                    src = torch.from_numpy(np.ascontiguousarray(tab0.block_table[:, n_stale]).astype(np.int32)).to(device)
+                    dst = torch.arange(tab0.tq3_pages, tab0.tq3_pages + B, dtype=torch.int32, device=device)
+                    us_append = timed(lambda: L.pool.append(L.k_new, L.v_new, plan["slots"][0]))
+                    us_demote = timed(lambda: L.pool.demote(src, dst))
+                    us_decode = timed(lambda: L.pool.decode_attention(L.q, L.bt, L.tags, plan["lens"][0], spec.scale, out=L.out))
+                    if L.pool.status() != M.OK:
+                        raise RuntimeError("device status word set in cell %s" % spec.name)
+                    kv = kv_bytes_at(spec, tags_host, plan["lens_host"][0])
+                    cell = {
+                        "mode": "sweep_cell", "cell": {"batch": B, "context_tokens": ctx, "stale_fraction": f},
+                        "tq3_record_format": fmt,
+                        "append": entry(us_append, B * hkv * d * (4 + 2), tokens=B),
+                        "demote": entry(us_demote, B * hkv * (32 * d + 16 * d + 32), pages=B,
+                                        pages_per_s=B / (us_demote * 1e-6)),
+                        "decode": entry(us_decode, kv, tokens_per_s=B / (us_decode * 1e-6)),
+                        "sum_us": us_append + us_demote + us_decode,
+                        "tokens_per_s_whole_cell": B / ((us_append + us_demote + us_decode) * 1e-6),
+                    }
+                    cells.append(cell)
+                    print(json.dumps(cell), flush=True)
+                    del layers, L, plan
+                    torch.cuda.empty_cache()
+    summary = {"mode": "sweep", "metric": METRIC, "data": "synthetic", "n_gpus": 1, "repetitions": reps,
+               "config": {"workload": "configs[4]: lifecycle sweep, 27 cells, head_dim 128, 8 KV x 4 q heads, 16-token pages",
+                          "tq3_record_format": fmt, "l2": "L2 flushed (256 MB rewritten) before every timed repetition"},
+               "peak": peak, "peak_source": peak_kind + " copy bandwidth", "clocks": clocks.summary(), "cells": cells}
+    if args.out:
+        with open(args.out, "w") as fh:
+            json.dump(summary, fh, indent=1)
+    print(json.dumps({k: v for k, v in summary.items() if k != "cells"}))
+
+
 # ---------------------------------------------------------------------------------------- oracle arm
 def workload_spec(args):
     over = {"n_layers": args.layers} if args.layers > 0 else {}
@@ -658,6 +738,23 @@ def workload_name(spec):
             "cfg5_canary_blocks_1792": "the configs[2] shape with pages of 1,792 tokens (paper-scale blocks): 2 x 59,008 "
                                        "tokens, d=256, 4 KV x 6 q heads, 10 FP8 + 23 TQ3 pages per request"}.get(
         spec.name, spec.name)
+
+
+def config_dict(spec, args, world, step_bytes=None, batched=None, layers_per_launch=None):
+    """The `config` object of the JSON line; both arms print the same workload keys."""
+    fmt = 2 if args.format == "v2" else 1
+    cfg = {"workload": workload_name(spec), "batch": spec.batch, "context_tokens": list(spec.seq_lens)[:4],
+           "tq3_record_format": fmt, "layers": spec.n_layers, "head_dim": spec.head_dim, "kv_heads": spec.n_kv_heads,
+           "q_heads": spec.n_q_heads, "page_tokens": spec.page_tokens,
+           "parallelism": "replicas only" if world > 1 else "single GPU"}
+    if step_bytes is not None:
+        cfg["l2"] = "inputs larger than L2 (%.0f MB of KV per step)" % (step_bytes / 1e6)
+        cfg["step"] = "append + demote at its natural cadence + decode attention, every layer"
+        cfg["launch"] = ("one CUDA graph per step holding mkv_append_layers and mkv_decode_attention_layers (all layers in "
+                         "one launch each); retier calls issued directly") if batched else \
+                        "one CUDA graph per step (append + decode of every layer); retier calls issued directly"
+        cfg["layers_per_decode_launch"] = layers_per_launch
+    return cfg
 
 
 def oracle_sample(spec, seconds_hint=20.0):
@@ -693,8 +790,39 @@ def time_oracle(spec, reps=3):
             "kv_gbs": W.kv_bytes(sub, tab) / layer_s / 1e9}
 
 
-def cpu_baseline(spec):
-    return time_oracle(spec)
+def time_oracle_lifecycle(spec, seconds=3.0):
+    """The oracle's own Append (bf16 -> e4m3 record) and Demote (FP8 record -> TQ3 record) per page and KV head,
+    single-threaded as the oracle is written, on seeded data of the workload's head geometry."""
+    import oracle
+    d = spec.head_dim
+    rng = np.random.default_rng(spec.seed)
+    k = rng.standard_normal((16, d)).astype(np.float32)
+    v = rng.standard_normal((16, d)).astype(np.float32)
+    sigma = W.rotation_signs(spec, 0)
+    out = {}
+    for name, fn in (("append", lambda: oracle.fp8_pack_record(k, v)),
+                     ("demote", None)):
+        if name == "demote":
+            rec8 = oracle.fp8_pack_record(k, v)
+            fn = lambda: oracle.demote_record(rec8, d, sigma)
+        n, t0 = 0, time.perf_counter()
+        while time.perf_counter() - t0 < seconds:
+            fn()
+            n += 1
+        dt = time.perf_counter() - t0
+        out[name + "_page_heads_per_s"] = n / dt
+    out["append_tokens_per_s_all_heads"] = out["append_page_heads_per_s"] * 16 / spec.n_kv_heads
+    out["demote_pages_per_s_all_heads"] = out["demote_page_heads_per_s"] / spec.n_kv_heads
+    out["threads"] = 1
+    return out
+
+
+def cpu_baseline(spec, fmt=1):
+    import oracle
+    with oracle.record_format(fmt):
+        res = time_oracle(spec)
+        res["lifecycle"] = time_oracle_lifecycle(spec)
+    return res
 
 
 def run_reference(args):
@@ -702,10 +830,10 @@ def run_reference(args):
     if rank != 0:
         return
     spec = workload_spec(args)
+    import oracle as _o
+    _o.set_format(2 if args.format == "v2" else 1)
     oracle, sub, tab, L = oracle_sample(spec)
     K, Wm = args.steps, args.warmup
-    K = min(K, 5)
-    Wm = min(Wm, 1)
 
     def one():
         t0 = time.perf_counter()
@@ -723,7 +851,7 @@ def run_reference(args):
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": K, "warmup": Wm,
         "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-        "data": "synthetic", "config": {"workload": workload_name(spec)},
+        "data": "synthetic", "config": config_dict(spec, args, 1),
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -746,17 +874,38 @@ def main():
     ap.add_argument("--page-tokens", type=int, default=0,
                     help="override the page size (a multiple of 16; 1792 and 832 are the paper's block sizes)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--format", default="v1", choices=["v1", "v2"],
+    ap.add_argument("--format", default="v2", choices=["v1", "v2"],
                     help="TQ3 record format of the pools (v2: e4m3-exact key codebook, FP8 key products)")
     ap.add_argument("--per-layer", action="store_true",
                     help="issue mkv_append / mkv_decode_attention layer by layer instead of the batched calls")
+    ap.add_argument("--sweep", action="store_true",
+                    help="config 4 only: all 27 cells (batch x context x Stale fraction), each timing Append, Demote and "
+                         "decode separately; one JSON line per cell and a summary, also written to --out")
+    ap.add_argument("--out", default="", help="--sweep: file that receives the results as JSON")
     ap.add_argument("--lifecycle", action="store_true",
                     help="time Append, Demote and Promote alone (bulk throughput) instead of the decode step")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
+    # --gpus N: N independent replicas, one process per GPU.  Under torchrun WORLD_SIZE must agree with N; started
+    # plainly with N > 1 the script re-launches itself under torch.distributed.run on this node.
+    world_env = os.environ.get("WORLD_SIZE")
+    if world_env is not None and int(world_env) != args.gpus:
+        sys.stderr.write("bench.py: --gpus %d but WORLD_SIZE=%s; launch with --nproc-per-node equal to --gpus\n"
+                         % (args.gpus, world_env))
+        sys.exit(2)
+    if world_env is None and args.gpus > 1 and not args.lifecycle and not args.sweep:
+        import socket
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        os.execv(sys.executable, cmd)
     if args.impl == "reference":
         run_reference(args)
+    elif args.sweep:
+        run_sweep(args)
     elif args.lifecycle:
         run_lifecycle(args)
     else:

@@ -6,7 +6,10 @@ Follows Algorithm 1 (ownership-aware page-transition protocol) and Fig. "lifecyc
     Anchor --demote------> Stale      Stale  --promote--> Anchor
 
 with the copy-before-publish rule (a destination is populated before its tag and physical id are
-published; the source is released afterwards) and per-format free lists.  SealPrefix and the
+published; the source is released afterwards) and per-format free lists.  "Afterwards" is a point the
+planner cannot see: Algorithm 1 releases a source only once its readers and the conversion have cleared.
+So Retier and Promote leave the source RETIRING -- owned by the request, mapped nowhere, on no free list,
+never handed out -- until the caller says that point has passed (SeqModel.release).  SealPrefix and the
 prefix cache are outside the modelled path.  No transition ever drops a logical page of a live
 request.
 
@@ -35,7 +38,8 @@ class PoolModel:
         self.capacity = {FMT_FP8: fp8_pages, FMT_TQ3: tq3_pages}
         self.free = {FMT_FP8: list(range(fp8_pages - 1, -1, -1)),
                      FMT_TQ3: list(range(tq3_pages - 1, -1, -1))}
-        self.owner: Dict[Tuple[int, int], int] = {}    # (fmt, id) -> sequence handle
+        self.owner: Dict[Tuple[int, int], int] = {}    # (fmt, id) -> sequence handle (mapped pages)
+        self.retiring: Dict[Tuple[int, int], int] = {} # (fmt, id) -> sequence handle (sources awaiting release)
         self.seqs: Dict[int, "SeqModel"] = {}
         self._next = 0
 
@@ -52,6 +56,20 @@ class PoolModel:
         del self.owner[(fmt, pid)]
         self.free[fmt].append(pid)
 
+    def retire(self, fmt: int, pid: int):
+        """A conversion's source: no longer mapped, not yet reusable."""
+        if (fmt, pid) not in self.owner:
+            raise LifecycleError("MKV_E_STATE", "not an owned page")
+        self.retiring[(fmt, pid)] = self.owner.pop((fmt, pid))
+
+    def release_retired(self, fmt: int, pid: int, owner: int):
+        if not 0 <= pid < self.capacity[fmt]:
+            raise LifecycleError("MKV_E_BOUNDS", "page id out of range")
+        if self.retiring.get((fmt, pid)) != owner:
+            raise LifecycleError("MKV_E_STATE", "page is not retiring for this request")
+        del self.retiring[(fmt, pid)]
+        self.free[fmt].append(pid)
+
     def new_seq(self) -> "SeqModel":
         s = SeqModel(self, self._next)
         self.seqs[self._next] = s
@@ -65,6 +83,8 @@ class PoolModel:
             for tag, pid in s.pages:
                 tiers[tag] += 1
                 used[FMT_TQ3 if tag == STALE else FMT_FP8] += 1
+        for fmt, _ in self.retiring:          # a retiring source still occupies its arena
+            used[fmt] += 1
         return used, tiers
 
     def check_invariants(self):
@@ -81,8 +101,14 @@ class PoolModel:
                 assert self.owner.get((fmt, pid)) == s.handle
                 assert pid not in self.free[fmt], "mapped page on a free list"
         assert seen == set(self.owner.keys()), "owned page not mapped (leak)"
+        for (fmt, pid), h in self.retiring.items():
+            assert h in self.seqs, "retiring page of a finished request"
+            assert (fmt, pid) not in seen, "retiring page still mapped"
+            assert pid not in self.free[fmt], "retiring page handed back before its release"
         for fmt in (FMT_FP8, FMT_TQ3):
-            assert len(self.free[fmt]) + sum(1 for f, _ in self.owner if f == fmt) == self.capacity[fmt]
+            assert len(set(self.free[fmt])) == len(self.free[fmt])
+            assert (len(self.free[fmt]) + sum(1 for f, _ in self.owner if f == fmt) +
+                    sum(1 for f, _ in self.retiring if f == fmt)) == self.capacity[fmt]
 
 
 class SeqModel:
@@ -119,8 +145,8 @@ class SeqModel:
             raise LifecycleError("MKV_E_STATE", "page is not Anchor")
         self.pages[lp] = (RECENT, pid)
 
-    # Retier(p, TQ3): retain the source, allocate and populate the destination, publish tag + id,
-    # then release the source.  Returns (source fp8 id, destination tq3 id).
+    # Retier(p, TQ3): retain the source, allocate and populate the destination, publish tag + id;
+    # the source is retiring until release().  Returns (source fp8 id, destination tq3 id).
     def demote(self, lp: int):
         tag, src = self._get(lp)
         if tag == STALE:
@@ -129,7 +155,7 @@ class SeqModel:
             raise LifecycleError("MKV_E_STATE", "only full pages may become TQ3")
         dst = self.pool.alloc(FMT_TQ3, self.handle)
         self.pages[lp] = (STALE, dst)      # publish (after the destination is populated)
-        self.pool.release(FMT_FP8, src)    # release after readers and the conversion cleared
+        self.pool.retire(FMT_FP8, src)     # released only after readers and the conversion cleared
         return src, dst
 
     # Promote(p): reconstruct into a newly allocated FP8 page, publish, retire the TQ3 page.
@@ -139,8 +165,13 @@ class SeqModel:
             raise LifecycleError("MKV_E_STATE", "not Stale")
         dst = self.pool.alloc(FMT_FP8, self.handle)
         self.pages[lp] = (ANCHOR, dst)
-        self.pool.release(FMT_TQ3, src)
+        self.pool.retire(FMT_TQ3, src)
         return src, dst
+
+    # The point Algorithm 1 waits for has passed (earlier readers and the conversion are ordered before
+    # any later writer of the page): the retiring source goes back to its free list.
+    def release(self, fmt: int, pid: int):
+        self.pool.release_retired(fmt, pid, self.handle)
 
     def age(self, recent_tokens: int):
         """Demote every full Recent page that lies wholly before the last `recent_tokens` tokens."""
@@ -155,6 +186,9 @@ class SeqModel:
     def finish(self):
         for tag, pid in self.pages:
             self.pool.release(FMT_TQ3 if tag == STALE else FMT_FP8, pid)
+        for (fmt, pid), h in sorted(self.pool.retiring.items()):     # in (format, id) order
+            if h == self.handle:
+                self.pool.release_retired(fmt, pid, h)
         self.pages = []
         self.len = 0
         del self.pool.seqs[self.handle]

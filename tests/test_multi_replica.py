@@ -45,3 +45,14 @@ def test_single_process_passthrough():
     import bench
     assert bench.max_over_ranks([1.5, 2.5]) == [1.5, 2.5]
     assert bench.aggregate_value(2, 40, 50.0, 1) == 1600.0
+
+
+def test_gpus_flag_must_agree_with_the_launched_world_size():
+    """`--gpus N` means N replicas: under a launcher whose WORLD_SIZE differs the script refuses to run
+    (exit code 2) instead of silently timing another number of replicas."""
+    import subprocess
+    env = dict(os.environ, WORLD_SIZE="1", RANK="0", LOCAL_RANK="0")
+    for impl in ("ours", "reference"):
+        r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", impl, "--steps", "1"],
+                           env=env, capture_output=True, text=True, timeout=120)
+        assert r.returncode == 2 and "WORLD_SIZE" in r.stderr, (impl, r.returncode, r.stderr[-300:])

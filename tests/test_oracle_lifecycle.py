@@ -25,13 +25,25 @@ def test_transitions_of_the_lifecycle_graph():
     s.protect(0)                                   # Recent -> Anchor
     assert s.pages[0][0] == ANCHOR
     src, dst = s.demote(1)                         # Recent -> Stale (age)
-    assert s.pages[1] == (STALE, dst) and src in pool.free[FMT_FP8]
+    assert s.pages[1] == (STALE, dst)
+    # the source is retiring: not mapped, not free, and the next page a request opens is another one
+    assert (FMT_FP8, src) in pool.retiring and src not in pool.free[FMT_FP8]
+    other = pool.new_seq()
+    assert other.append()[0] != src
+    with pytest.raises(LifecycleError) as e:
+        other.release(FMT_FP8, src)                # only the owning request releases it
+    assert e.value.code == "MKV_E_STATE"
+    s.release(FMT_FP8, src)
+    assert src in pool.free[FMT_FP8] and not pool.retiring
+    with pytest.raises(LifecycleError):
+        s.release(FMT_FP8, src)                    # once
+    other.finish()
     s.demote(0)                                    # Anchor -> Stale (demote)
     with pytest.raises(LifecycleError) as e:
         s.protect(0)                               # Stale cannot be tagged; it must be promoted
     assert e.value.code == "MKV_E_STATE"
     src, dst = s.promote(0)                        # Stale -> Anchor through a new FP8 page
-    assert s.pages[0] == (ANCHOR, dst) and src in pool.free[FMT_TQ3]
+    assert s.pages[0] == (ANCHOR, dst) and (FMT_TQ3, src) in pool.retiring and src not in pool.free[FMT_TQ3]
     with pytest.raises(LifecycleError):
         s.demote(3)                                # the open, partial page never becomes TQ3
     with pytest.raises(LifecycleError):
@@ -95,8 +107,12 @@ def test_random_walk_keeps_every_invariant():
                 s = rnd.choice(seqs)
                 if s.pages:
                     s.protect(rnd.randrange(len(s.pages)))
-            elif r < 0.96:
+            elif r < 0.94:
                 rnd.choice(seqs).age(rnd.choice([16, 48, 100]))
+            elif r < 0.96:
+                if pool.retiring:                  # the stream point of some conversion has passed
+                    (fmt, pid), h = rnd.choice(sorted(pool.retiring.items()))
+                    pool.seqs[h].release(fmt, pid)
             else:
                 s = seqs.pop(rnd.randrange(len(seqs)))
                 s.finish()
