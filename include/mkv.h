@@ -137,7 +137,8 @@ int32_t mkv_pool_destroy(mkv_pool* pool);
 /* Per-format free lists (Section 4.4: "per-kind free list").  ids is a host array of n entries.
  * alloc: all-or-nothing; MKV_E_OOM_* leaves the lists untouched.  A fresh list hands out
  * 0, 1, 2, ...; a freed id is reused first.  free: MKV_E_BOUNDS for a bad id, MKV_E_STATE for a
- * page that is not allocated; nothing is freed in either case. */
+ * page that is not allocated or is the retiring source of a planned conversion (mkv_seq_release);
+ * nothing is freed in either case. */
 int32_t mkv_page_alloc(mkv_pool* pool, int32_t fmt, int32_t* ids_host, int32_t n);
 int32_t mkv_page_free(mkv_pool* pool, int32_t fmt, const int32_t* ids_host, int32_t n);
 
@@ -334,14 +335,23 @@ int32_t mkv_seq_finish(mkv_seq* seq);
 int32_t mkv_seq_append(mkv_seq* seq, int32_t* page_id, int32_t* slot, int32_t* opened_page);
 /* Recent <-> Anchor tag of a logical page (MKV_E_STATE if it is Stale). */
 int32_t mkv_seq_protect(mkv_seq* seq, int32_t logical_page, int32_t flag);
-/* Retier to TQ3: allocates the destination, updates the row, releases the source id.  Only full,
- * non-Stale pages qualify (MKV_E_STATE otherwise).  The caller then enqueues mkv_demote(). */
+/* Retier to TQ3 (Algorithm 1 step 2): allocates the destination and updates the row.  Only full, non-Stale
+ * pages qualify (MKV_E_STATE otherwise).  The caller then enqueues mkv_demote().  The source FP8 id leaves
+ * the row but is RETIRING: it is on no free list and is handed to nobody until mkv_seq_release(), which the
+ * caller issues once every reader enqueued before the conversion, and the conversion itself, are ordered
+ * before any later writer of that page (on one stream: as soon as mkv_demote() has been enqueued; across
+ * streams: after the event that marks it).  mkv_pool_stats() counts retiring pages as used. */
 int32_t mkv_seq_demote(mkv_seq* seq, int32_t logical_page, int32_t* src_fp8_id, int32_t* dst_tq3_id);
-/* Promote: Stale -> Anchor through a newly allocated FP8 page (MKV_E_STATE if the page is not Stale,
- * MKV_E_OOM_FP8 if none is free).  The caller then enqueues mkv_promote(). */
+/* Promote (Algorithm 1 step 3): Stale -> Anchor through a newly allocated FP8 page (MKV_E_STATE if the page
+ * is not Stale, MKV_E_OOM_FP8 if none is free).  The caller then enqueues mkv_promote(); the TQ3 source is
+ * retiring until mkv_seq_release(), as for mkv_seq_demote(). */
 int32_t mkv_seq_promote(mkv_seq* seq, int32_t logical_page, int32_t* src_tq3_id, int32_t* dst_fp8_id);
+/* Release a retiring source (Algorithm 1: "after readers and the conversion event clear") to its free list.
+ * MKV_E_STATE if (fmt, id) is not a retiring source of this sequence, MKV_E_BOUNDS for a bad id.
+ * mkv_seq_finish() releases what is still retiring. */
+int32_t mkv_seq_release(mkv_seq* seq, int32_t fmt, int32_t id);
 /* Age: plan the demotion of every full Recent page wholly before the last `recent_tokens`
- * tokens.  Writes up to `cap` triples and returns their number in *n (MKV_E_INVALID if more
+ * tokens (their sources become retiring, as with mkv_seq_demote).  Writes up to `cap` triples and returns their number in *n (MKV_E_INVALID if more
  * would be needed; nothing changes then). */
 int32_t mkv_seq_age(mkv_seq* seq, int32_t recent_tokens, int32_t* logical_pages, int32_t* src_fp8_ids,
                     int32_t* dst_tq3_ids, int32_t cap, int32_t* n);

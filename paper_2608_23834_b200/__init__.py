@@ -34,7 +34,7 @@ EXPORTS = [
     "mkv_seq_protect", "mkv_seq_demote", "mkv_seq_age", "mkv_seq_len", "mkv_seq_row",
     "mkv_decode_attention_static", "mkv_promote", "mkv_seq_promote",
     "mkv_decode_attention_scored", "mkv_page_score_update", "mkv_page_score_update_paged",
-    "mkv_decode_attention_layers", "mkv_append_layers", "mkv_pool_set_wait_limit_ns",
+    "mkv_decode_attention_layers", "mkv_append_layers", "mkv_pool_set_wait_limit_ns", "mkv_seq_release",
 ]
 MAX_LAYERS_PER_CALL = 32
 
@@ -116,6 +116,7 @@ def lib():
             "mkv_seq_protect": [vp, C.c_int32, C.c_int32],
             "mkv_seq_demote": [vp, C.c_int32, i32p, i32p],
             "mkv_seq_age": [vp, C.c_int32, i32p, i32p, i32p, C.c_int32, i32p],
+            "mkv_seq_release": [vp, C.c_int32, C.c_int32],
             "mkv_seq_len": [vp, i32p, i32p],
             "mkv_seq_row": [vp, i32p, u8p, C.c_int32],
         }
@@ -425,6 +426,10 @@ class Seq:
         a, b = C.c_int32(), C.c_int32()
         _check(lib().mkv_seq_promote(self.handle, lp, C.byref(a), C.byref(b)), "mkv_seq_promote")
         return a.value, b.value
+
+    def release(self, fmt: int, pid: int):
+        """mkv_seq_release: the stream point of a planned conversion has passed; its source may be reused."""
+        _check(lib().mkv_seq_release(self.handle, int(fmt), int(pid)), "mkv_seq_release")
 
     def age(self, recent_tokens: int):
         _, n_pages = self.len()

@@ -4,6 +4,7 @@
 #include <stdint.h>
 
 #include <mutex>
+#include <utility>
 #include <vector>
 
 #include "mkv.h"
@@ -88,7 +89,7 @@ struct mkv_pool {
     mkv::Device dev;
     std::mutex mu;
     std::vector<int32_t> free_list[2];
-    std::vector<uint8_t> allocated[2];
+    std::vector<uint8_t> allocated[2];   // 0 free, 1 allocated, 2 retiring (source of a planned conversion)
 };
 
 struct mkv_seq {
@@ -96,6 +97,7 @@ struct mkv_seq {
     int32_t len;
     std::vector<int32_t> ids;
     std::vector<uint8_t> tags;
+    std::vector<std::pair<int32_t, int32_t>> retiring;   // (format, id) of conversion sources awaiting mkv_seq_release
 };
 
 namespace mkv {

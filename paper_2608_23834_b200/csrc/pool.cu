@@ -1,6 +1,7 @@
 // Host side of libmkv: pool bookkeeping, per-format free lists, sequence rows (Algorithm 1),
 // argument validation and the C ABI entry points.  No arithmetic of the method lives here.
 #include <cstdio>
+#include <algorithm>
 #include <cstring>
 #include <new>
 #include <string>
@@ -185,7 +186,7 @@ int32_t mkv_page_free(mkv_pool* pool, int32_t fmt, const int32_t* ids, int32_t n
     auto& al = pool->allocated[fmt];
     for (int i = 0; i < n; ++i) {
         if (ids[i] < 0 || (size_t)ids[i] >= al.size()) return MKV_E_BOUNDS;
-        if (!al[ids[i]]) return MKV_E_STATE;
+        if (al[ids[i]] != 1) return MKV_E_STATE;          // free already, or retiring (mkv_seq_release frees those)
         for (int j = 0; j < i; ++j)
             if (ids[j] == ids[i]) return MKV_E_STATE;
     }
@@ -452,6 +453,13 @@ int32_t mkv_seq_finish(mkv_seq* seq)
         int32_t r = mkv_page_free(seq->pool, fmt, &seq->ids[i], 1);
         if (r != MKV_OK) rc = r;
     }
+    // sources still retiring go back too, in (format, id) order
+    std::sort(seq->retiring.begin(), seq->retiring.end());
+    while (!seq->retiring.empty()) {
+        const std::pair<int32_t, int32_t> e = seq->retiring.front();
+        int32_t r = mkv_seq_release(seq, e.first, e.second);
+        if (r != MKV_OK) { rc = r; break; }
+    }
     delete seq;
     return rc;
 }
@@ -485,6 +493,16 @@ int32_t mkv_seq_protect(mkv_seq* seq, int32_t lp, int32_t flag)
     return MKV_OK;
 }
 
+// The source of a planned conversion: it leaves the row but stays out of the free list (state 2) until the
+// caller reports, with mkv_seq_release, that earlier readers and the conversion are ordered before any later writer.
+static int32_t retire_source(mkv_seq* seq, int32_t fmt, int32_t id)
+{
+    std::lock_guard<std::mutex> lk(seq->pool->mu);
+    seq->pool->allocated[fmt][id] = 2;
+    seq->retiring.emplace_back(fmt, id);
+    return MKV_OK;
+}
+
 int32_t mkv_seq_demote(mkv_seq* seq, int32_t lp, int32_t* src, int32_t* dst)
 {
     if (!seq || !src || !dst) return MKV_E_INVALID;
@@ -498,7 +516,7 @@ int32_t mkv_seq_demote(mkv_seq* seq, int32_t lp, int32_t* src, int32_t* dst)
     *dst = id;
     seq->ids[lp] = id;
     seq->tags[lp] = MKV_TAG_STALE;
-    return mkv_page_free(seq->pool, MKV_FMT_FP8, src, 1);
+    return retire_source(seq, MKV_FMT_FP8, *src);
 }
 
 int32_t mkv_seq_promote(mkv_seq* seq, int32_t lp, int32_t* src, int32_t* dst)
@@ -513,7 +531,23 @@ int32_t mkv_seq_promote(mkv_seq* seq, int32_t lp, int32_t* src, int32_t* dst)
     *dst = id;
     seq->ids[lp] = id;
     seq->tags[lp] = MKV_TAG_ANCHOR;
-    return mkv_page_free(seq->pool, MKV_FMT_TQ3, src, 1);
+    return retire_source(seq, MKV_FMT_TQ3, *src);
+}
+
+int32_t mkv_seq_release(mkv_seq* seq, int32_t fmt, int32_t id)
+{
+    if (!seq || (fmt != MKV_FMT_FP8 && fmt != MKV_FMT_TQ3)) return MKV_E_INVALID;
+    mkv_pool* pool = seq->pool;
+    std::lock_guard<std::mutex> lk(pool->mu);
+    if (id < 0 || (size_t)id >= pool->allocated[fmt].size()) return MKV_E_BOUNDS;
+    for (size_t i = 0; i < seq->retiring.size(); ++i)
+        if (seq->retiring[i].first == fmt && seq->retiring[i].second == id) {
+            seq->retiring.erase(seq->retiring.begin() + (long)i);
+            pool->allocated[fmt][id] = 0;
+            pool->free_list[fmt].push_back(id);
+            return MKV_OK;
+        }
+    return MKV_E_STATE;                                    // not a retiring source of this sequence
 }
 
 int32_t mkv_seq_age(mkv_seq* seq, int32_t recent_tokens, int32_t* lps, int32_t* srcs, int32_t* dsts,

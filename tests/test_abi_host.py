@@ -114,8 +114,12 @@ def test_sequence_bookkeeping_agrees_with_the_lifecycle_model_on_a_random_walk(p
             op = ("promote", lp)
         elif r < 0.90:
             op = ("protect", lp, rnd.random() < 0.7)
-        elif r < 0.96:
+        elif r < 0.94:
             op = ("age", rnd.choice([16, 40, 100]) * page_tokens // 16)
+        elif r < 0.97:
+            # the stream point of a planned conversion has passed: release one retiring source of this request
+            mine = sorted(k for k, h in model.retiring.items() if h == m.handle)
+            op = ("release",) + (rnd.choice(mine) if mine and rnd.random() < 0.9 else (rnd.randrange(2), rnd.randrange(26)))
         else:
             op = ("finish",)
         got = want = None
@@ -130,6 +134,8 @@ def test_sequence_bookkeeping_agrees_with_the_lifecycle_model_on_a_random_walk(p
                 want = m.protect(op[1]) if op[2] else m.unprotect(op[1])
             elif op[0] == "age":
                 want = m.age(op[1])
+            elif op[0] == "release":
+                want = m.release(op[1], op[2])
             else:
                 m.finish()
         except LifecycleError as e:
@@ -145,6 +151,8 @@ def test_sequence_bookkeeping_agrees_with_the_lifecycle_model_on_a_random_walk(p
                 got = s.protect(op[1], op[2])
             elif op[0] == "age":
                 got = s.age(op[1])
+            elif op[0] == "release":
+                got = s.release(op[1], op[2])
             else:
                 s.finish()
         except M.MkvError as e:

@@ -10,7 +10,7 @@ import mkv_workloads as W
 import oracle
 import paper_2608_23834_b200 as M
 from _gpu_util import bf16_tensor, check_close
-from oracle.lifecycle import PoolModel, STALE
+from oracle.lifecycle import FMT_FP8, FMT_TQ3, PoolModel, STALE
 
 pytestmark = pytest.mark.gpu
 
@@ -65,6 +65,11 @@ def test_append_demote_decode_cell(frac, ctx, batch, T):
         dst = torch.tensor([p[3] for p in pairs], dtype=torch.int32, device="cuda:0")
         ent = torch.tensor([p[0] * max_pages + p[1] for p in pairs], dtype=torch.int64, device="cuda:0")
         pool.demote(src, dst, bt, tags, ent)
+        # everything runs on one stream: once the conversion is enqueued, later writers of the sources are ordered
+        # after it and after every earlier reader, so the retiring sources can go back to their free list
+        for b, lp, s, t in pairs:
+            seqs[b].release(M.FMT_FP8, s)
+            mods[b].release(FMT_FP8, s)
 
     # ---- bring the cell to its starting state: ctx tokens, oldest floor(f*P) pages Stale ----
     rng = np.random.default_rng(4)
@@ -146,6 +151,14 @@ def test_append_demote_decode_cell(frac, ctx, batch, T):
         pool.promote(src, dst, bt, tags, ent)
         torch.cuda.synchronize()
         assert pool.status() == M.OK
+        # the Stale sources are retiring (counted as used, handed to nobody) until they are released
+        st, (used, _) = pool.stats(), model.stats()
+        assert (st.fp8_pages_used, st.tq3_pages_used) == (used[0], used[1])
+        for b_, lp_, s_id, t_id in pairs:
+            seqs[b_].release(M.FMT_TQ3, s_id)
+            mods[b_].release(FMT_TQ3, s_id)
+        model.check_invariants()
+        assert pool.stats().tq3_pages_used == st.tq3_pages_used - len(pairs)
         bt_h, tg_h = bt.cpu().numpy(), tags.cpu().numpy()
         for b, lp, s_id, t_id in pairs:
             assert bt_h[b, lp] == t_id and tg_h[b, lp] == M.TAG_ANCHOR
