@@ -185,6 +185,8 @@ int32_t mkv_append(mkv_pool* pool, const void* k_dev, const void* v_dev, const i
  *   block_table, tier_tag      device tables to publish into, or NULL
  *   entry_index                device, int64 [n_pages]: flat index of each page's entry in the two
  *                              tables (negative = do not publish), or NULL
+ *   table_entries              number of entries of block_table / tier_tag (ignored when entry_index is
+ *                              NULL); an index at or beyond it is not written and flags MKV_E_BOUNDS
  * For every page the TQ3 record is complete and fenced before its id and MKV_TAG_STALE are
  * written (copy-before-publish).  The FP8 source is not modified; return it to its free list with
  * mkv_page_free() once every reader enqueued before this call has been ordered before the next
@@ -193,7 +195,7 @@ int32_t mkv_append(mkv_pool* pool, const void* k_dev, const void* v_dev, const i
  * over the page's 16 tokens, asymmetric 3-bit codes with fp16 scale and zero. */
 int32_t mkv_demote(mkv_pool* pool, const int32_t* src_fp8_ids_dev, const int32_t* dst_tq3_ids_dev,
                    int32_t n_pages, int32_t* block_table_dev, uint8_t* tier_tag_dev,
-                   const int64_t* entry_index_dev, void* stream);
+                   const int64_t* entry_index_dev, int64_t table_entries, void* stream);
 
 /* Promote (Algorithm 1 step 3; Section 3.1, Anchor tier: a Stale page that becomes protected again
  * is rebuilt at FP8): reconstruct n_pages TQ3 pages (all KV heads) into newly allocated FP8 pages, then publish id and MKV_TAG_ANCHOR; arguments as for mkv_demote with the
@@ -202,13 +204,17 @@ int32_t mkv_demote(mkv_pool* pool, const int32_t* src_fp8_ids_dev, const int32_t
  * TQ3 source is not modified; free it once earlier readers are ordered before its next writer. */
 int32_t mkv_promote(mkv_pool* pool, const int32_t* src_tq3_ids_dev, const int32_t* dst_fp8_ids_dev,
                     int32_t n_pages, int32_t* block_table_dev, uint8_t* tier_tag_dev,
-                    const int64_t* entry_index_dev, void* stream);
+                    const int64_t* entry_index_dev, int64_t table_entries, void* stream);
 
 /* Protect / unprotect (Fig. lifecycle: Recent -> Anchor): set the tag of one table entry to
  * MKV_TAG_ANCHOR (flag != 0) or MKV_TAG_RECENT (flag == 0).  No data moves.  If the entry is
  * Stale the tag is left alone and MKV_E_STATE is recorded in the status word (a Stale page is
- * promoted into a new FP8 page with mkv_promote instead). */
-int32_t mkv_set_anchor(mkv_pool* pool, uint8_t* tier_tag_dev, int64_t entry_index, int32_t flag, void* stream);
+ * promoted into a new FP8 page with mkv_promote instead).  entry_index >= table_entries (the number of
+ * entries of tier_tag) returns MKV_E_BOUNDS without launching.
+ * Publication writes the id, then the tag, as two stores: a reader on ANOTHER stream must be ordered after
+ * the publishing call (an event), readers on the same stream are by stream order. */
+int32_t mkv_set_anchor(mkv_pool* pool, uint8_t* tier_tag_dev, int64_t table_entries, int64_t entry_index, int32_t flag,
+                       void* stream);
 
 /* Decode attention (Section 3.3; Section 4.1 "fused decode path"): for every request b and query
  * head h, softmax(scale * q K^T) V over the seq_lens[b] tokens of row b, where each page is read

@@ -94,10 +94,10 @@ def lib():
             "mkv_page_read_raw": [vp, C.c_int32, C.c_int32, vp, vp],
             "mkv_page_write_raw": [vp, C.c_int32, C.c_int32, vp, vp],
             "mkv_append": [vp, vp, vp, vp, C.c_int32, vp],
-            "mkv_demote": [vp, vp, vp, C.c_int32, vp, vp, vp, vp],
-            "mkv_promote": [vp, vp, vp, C.c_int32, vp, vp, vp, vp],
+            "mkv_demote": [vp, vp, vp, C.c_int32, vp, vp, vp, C.c_int64, vp],
+            "mkv_promote": [vp, vp, vp, C.c_int32, vp, vp, vp, C.c_int64, vp],
             "mkv_seq_promote": [vp, C.c_int32, i32p, i32p],
-            "mkv_set_anchor": [vp, vp, C.c_int64, C.c_int32, vp],
+            "mkv_set_anchor": [vp, vp, C.c_int64, C.c_int64, C.c_int32, vp],
             "mkv_decode_attention": [vp, vp, vp, vp, vp, C.c_int32, C.c_int32, C.c_float, f32p, f32p, vp,
                                      C.c_size_t, vp],
             "mkv_decode_attention_static": [vp, vp, vp, vp, vp, C.c_int32, C.c_int32, C.c_float, f32p, f32p, vp],
@@ -262,7 +262,8 @@ class Pool:
         if entry_index is not None:
             assert entry_index.dtype == torch.int64 and block_table.dtype == torch.int32 and tier_tag.dtype == torch.uint8
         _check(lib().mkv_demote(self.handle, _ptr(src_ids), _ptr(dst_ids), src_ids.numel(), _ptr(block_table),
-                                _ptr(tier_tag), _ptr(entry_index), _stream(stream)), "mkv_demote")
+                                _ptr(tier_tag), _ptr(entry_index), 0 if tier_tag is None else tier_tag.numel(),
+                                _stream(stream)), "mkv_demote")
 
     def promote(self, src_ids: torch.Tensor, dst_ids: torch.Tensor, block_table=None, tier_tag=None, entry_index=None,
                 stream=None) -> None:
@@ -270,11 +271,12 @@ class Pool:
         if entry_index is not None:
             assert entry_index.dtype == torch.int64 and block_table.dtype == torch.int32 and tier_tag.dtype == torch.uint8
         _check(lib().mkv_promote(self.handle, _ptr(src_ids), _ptr(dst_ids), src_ids.numel(), _ptr(block_table),
-                                 _ptr(tier_tag), _ptr(entry_index), _stream(stream)), "mkv_promote")
+                                 _ptr(tier_tag), _ptr(entry_index), 0 if tier_tag is None else tier_tag.numel(),
+                                 _stream(stream)), "mkv_promote")
 
     def set_anchor(self, tier_tag: torch.Tensor, entry_index: int, flag: bool, stream=None) -> None:
-        _check(lib().mkv_set_anchor(self.handle, _ptr(tier_tag), int(entry_index), int(bool(flag)), _stream(stream)),
-               "mkv_set_anchor")
+        _check(lib().mkv_set_anchor(self.handle, _ptr(tier_tag), tier_tag.numel(), int(entry_index), int(bool(flag)),
+                                    _stream(stream)), "mkv_set_anchor")
 
     def decode_attention(self, q, block_table, tier_tag, seq_lens, scale, out=None, lse=None, workspace=None, stream=None):
         B = q.shape[0]

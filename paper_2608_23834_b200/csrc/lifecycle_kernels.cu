@@ -539,7 +539,7 @@ __global__ void __launch_bounds__(D) demote_kernel(const uint8_t* __restrict__ f
                                                       float v_scale, SigmaBits sigma,
                                                       const int32_t* __restrict__ src_ids,
                                                       const int32_t* __restrict__ dst_ids, int32_t* block_table,
-                                                      uint8_t* tier_tag, const int64_t* entry_index,
+                                                      uint8_t* tier_tag, const int64_t* entry_index, int64_t n_entries,
                                                       uint32_t* __restrict__ status)
 {
     constexpr int KROW = D + 8;          // padded row of the key-code tile
@@ -590,7 +590,8 @@ __global__ void __launch_bounds__(D) demote_kernel(const uint8_t* __restrict__ f
     cluster_barrier();
     if (valid && crank == 0 && tid == 0 && entry_index != nullptr) {
         const int64_t e = entry_index[page];
-        if (e >= 0) {
+        if (e >= n_entries) atomicOr(status, kStBounds);      // an entry beyond the tables: flagged, nothing published
+        else if (e >= 0) {
             block_table[e] = dst;
             __threadfence();
             tier_tag[e] = (uint8_t)MKV_TAG_STALE;
@@ -662,14 +663,15 @@ __global__ void __launch_bounds__(1024) demote_minmax_kernel(const uint8_t* __re
 // whole page, so its id and tag may appear (copy-before-publish by stream order).
 __global__ void publish_kernel(int n, const int32_t* __restrict__ src_ids, const int32_t* __restrict__ dst_ids,
                                int src_cap, int dst_cap, int32_t* block_table, uint8_t* tier_tag,
-                               const int64_t* __restrict__ entry_index, int tag)
+                               const int64_t* __restrict__ entry_index, int64_t n_entries, int tag, uint32_t* status)
 {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     const int src = src_ids[i], dst = dst_ids[i];
     if (src < 0 || src >= src_cap || dst < 0 || dst >= dst_cap) return;
     const int64_t e = entry_index[i];
-    if (e >= 0) {
+    if (e >= n_entries) atomicOr(status, kStBounds);
+    else if (e >= 0) {
         block_table[e] = dst;
         __threadfence();
         tier_tag[e] = (uint8_t)tag;
@@ -704,13 +706,13 @@ static cudaError_t launch_clustered_rows(Kernel kernel, int n_pages, int csize, 
 
 template <int D, int FMT>
 static int32_t launch_demote_d(mkv_pool* p, const int32_t* src, const int32_t* dst, int n, int32_t* bt, uint8_t* tags,
-                               const int64_t* entry, cudaStream_t s)
+                               const int64_t* entry, int64_t n_entries, cudaStream_t s)
 {
     const int c = heads_cluster(p->hkv, n);
     if (p->tiles == 1) {
         MKV_CUDA(launch_clustered(demote_kernel<D, false, FMT>, n, c, D, s, (const uint8_t*)p->fp8, p->tq3, p->cfg.fp8_pages,
                                   p->cfg.tq3_pages, p->hkv, 1, p->cfg.k_scale, p->cfg.v_scale, p->sigma, src, dst, bt,
-                                  tags, entry, p->status_dev));
+                                  tags, entry, n_entries, p->status_dev));
         return MKV_OK;
     }
     // pages of several tiles: scale/zero of the page, then the tiles in parallel, then the publication
@@ -720,10 +722,10 @@ static int32_t launch_demote_d(mkv_pool* p, const int32_t* src, const int32_t* d
     MKV_CUDA(launch_clustered_rows(demote_kernel<D, true, FMT>, n, heads_cluster(p->hkv, 0), tile_rows(p->tiles, n, p->hkv), D, s,
                                    (const uint8_t*)p->fp8, p->tq3, p->cfg.fp8_pages, p->cfg.tq3_pages, p->hkv, p->tiles,
                                    p->cfg.k_scale, p->cfg.v_scale, p->sigma, src, dst, (int32_t*)nullptr,
-                                   (uint8_t*)nullptr, (const int64_t*)nullptr, p->status_dev));
+                                   (uint8_t*)nullptr, (const int64_t*)nullptr, (int64_t)0, p->status_dev));
     if (entry) {
         publish_kernel<<<(n + 127) / 128, 128, 0, s>>>(n, src, dst, p->cfg.fp8_pages, p->cfg.tq3_pages, bt, tags, entry,
-                                                       MKV_TAG_STALE);
+                                                       n_entries, MKV_TAG_STALE, p->status_dev);
         MKV_CUDA(cudaGetLastError());
     }
     (void)c;
@@ -731,13 +733,13 @@ static int32_t launch_demote_d(mkv_pool* p, const int32_t* src, const int32_t* d
 }
 
 int32_t launch_demote(mkv_pool* p, const int32_t* src, const int32_t* dst, int n, int32_t* bt, uint8_t* tags,
-                      const int64_t* entry, cudaStream_t s)
+                      const int64_t* entry, int64_t n_entries, cudaStream_t s)
 {
     if (p->fmt == 2)
-        return p->d == 128 ? launch_demote_d<128, 2>(p, src, dst, n, bt, tags, entry, s)
-                           : launch_demote_d<256, 2>(p, src, dst, n, bt, tags, entry, s);
-    return p->d == 128 ? launch_demote_d<128, 1>(p, src, dst, n, bt, tags, entry, s)
-                       : launch_demote_d<256, 1>(p, src, dst, n, bt, tags, entry, s);
+        return p->d == 128 ? launch_demote_d<128, 2>(p, src, dst, n, bt, tags, entry, n_entries, s)
+                           : launch_demote_d<256, 2>(p, src, dst, n, bt, tags, entry, n_entries, s);
+    return p->d == 128 ? launch_demote_d<128, 1>(p, src, dst, n, bt, tags, entry, n_entries, s)
+                       : launch_demote_d<256, 1>(p, src, dst, n, bt, tags, entry, n_entries, s);
 }
 
 // ------------------------------------------------------------------------------------------ promote
@@ -757,7 +759,7 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
                                                      float inv_v_scale, float rs, SigmaBits sigma,
                                                      const int32_t* __restrict__ src_ids,
                                                      const int32_t* __restrict__ dst_ids, int32_t* block_table,
-                                                     uint8_t* tier_tag, const int64_t* entry_index,
+                                                     uint8_t* tier_tag, const int64_t* entry_index, int64_t n_entries,
                                                      uint32_t* __restrict__ status)
 {
     constexpr int EPL = D / 32;
@@ -925,7 +927,8 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
     cluster_barrier();
     if (valid && crank == 0 && tid == 0 && entry_index != nullptr) {
         const int64_t e = entry_index[page];
-        if (e >= 0) {
+        if (e >= n_entries) atomicOr(status, kStBounds);
+        else if (e >= 0) {
             block_table[e] = dst;
             __threadfence();
             tier_tag[e] = (uint8_t)MKV_TAG_ANCHOR;
@@ -935,36 +938,36 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
 
 template <int D, int FMT>
 static int32_t launch_promote_d(mkv_pool* p, const int32_t* src, const int32_t* dst, int n, int32_t* bt, uint8_t* tags,
-                                const int64_t* entry, cudaStream_t s)
+                                const int64_t* entry, int64_t n_entries, cudaStream_t s)
 {
     const float ik = 1.0f / p->cfg.k_scale, iv = 1.0f / p->cfg.v_scale;
     const float rs = (float)(1.0 / sqrt((double)p->d));
     if (p->tiles == 1) {
         MKV_CUDA(launch_clustered(promote_kernel<D, false, FMT>, n, heads_cluster(p->hkv, n), D, s, (const uint8_t*)p->tq3, p->fp8,
                                   p->cfg.tq3_pages, p->cfg.fp8_pages, p->hkv, 1, ik, iv, rs, p->sigma, src, dst, bt, tags,
-                                  entry, p->status_dev));
+                                  entry, n_entries, p->status_dev));
         return MKV_OK;
     }
     MKV_CUDA(launch_clustered_rows(promote_kernel<D, true, FMT>, n, heads_cluster(p->hkv, 0), tile_rows(p->tiles, n, p->hkv), D, s,
                                    (const uint8_t*)p->tq3, p->fp8, p->cfg.tq3_pages, p->cfg.fp8_pages, p->hkv, p->tiles, ik,
                                    iv, rs, p->sigma, src, dst, (int32_t*)nullptr, (uint8_t*)nullptr,
-                                   (const int64_t*)nullptr, p->status_dev));
+                                   (const int64_t*)nullptr, (int64_t)0, p->status_dev));
     if (entry) {
         publish_kernel<<<(n + 127) / 128, 128, 0, s>>>(n, src, dst, p->cfg.tq3_pages, p->cfg.fp8_pages, bt, tags, entry,
-                                                       MKV_TAG_ANCHOR);
+                                                       n_entries, MKV_TAG_ANCHOR, p->status_dev);
         MKV_CUDA(cudaGetLastError());
     }
     return MKV_OK;
 }
 
 int32_t launch_promote(mkv_pool* p, const int32_t* src, const int32_t* dst, int n, int32_t* bt, uint8_t* tags,
-                       const int64_t* entry, cudaStream_t s)
+                       const int64_t* entry, int64_t n_entries, cudaStream_t s)
 {
     if (p->fmt == 2)
-        return p->d == 128 ? launch_promote_d<128, 2>(p, src, dst, n, bt, tags, entry, s)
-                           : launch_promote_d<256, 2>(p, src, dst, n, bt, tags, entry, s);
-    return p->d == 128 ? launch_promote_d<128, 1>(p, src, dst, n, bt, tags, entry, s)
-                       : launch_promote_d<256, 1>(p, src, dst, n, bt, tags, entry, s);
+        return p->d == 128 ? launch_promote_d<128, 2>(p, src, dst, n, bt, tags, entry, n_entries, s)
+                           : launch_promote_d<256, 2>(p, src, dst, n, bt, tags, entry, n_entries, s);
+    return p->d == 128 ? launch_promote_d<128, 1>(p, src, dst, n, bt, tags, entry, n_entries, s)
+                       : launch_promote_d<256, 1>(p, src, dst, n, bt, tags, entry, n_entries, s);
 }
 
 // ------------------------------------------------------------------------------------------ anchor

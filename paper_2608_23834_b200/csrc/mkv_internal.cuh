@@ -110,9 +110,9 @@ int32_t cuda_fail(cudaError_t e, const char* what);
 
 int32_t launch_append(mkv_pool* p, const void* k, const void* v, const int32_t* slots, int n, cudaStream_t s);
 int32_t launch_demote(mkv_pool* p, const int32_t* src, const int32_t* dst, int n, int32_t* bt, uint8_t* tags,
-                      const int64_t* entry, cudaStream_t s);
+                      const int64_t* entry, int64_t n_entries, cudaStream_t s);
 int32_t launch_promote(mkv_pool* p, const int32_t* src, const int32_t* dst, int n, int32_t* bt, uint8_t* tags,
-                       const int64_t* entry, cudaStream_t s);
+                       const int64_t* entry, int64_t n_entries, cudaStream_t s);
 int32_t launch_set_anchor(mkv_pool* p, uint8_t* tags, int64_t entry, int flag, cudaStream_t s);
 int32_t launch_decode_scalar(mkv_pool* p, const void* q, const int32_t* bt, const uint8_t* tags,
                              const int32_t* lens, int B, int max_pages, float scale, float* out, float* lse,

@@ -289,28 +289,29 @@ int32_t mkv_append(mkv_pool* pool, const void* k, const void* v, const int32_t* 
 }
 
 int32_t mkv_demote(mkv_pool* pool, const int32_t* src, const int32_t* dst, int32_t n, int32_t* bt,
-                   uint8_t* tags, const int64_t* entry, void* stream)
+                   uint8_t* tags, const int64_t* entry, int64_t table_entries, void* stream)
 {
     if (!pool || !pool->fp8 || n < 0) return MKV_E_INVALID;
     if (n == 0) return MKV_OK;
     if (!src || !dst) return MKV_E_INVALID;
-    if (entry && (!bt || !tags)) return MKV_E_INVALID;
-    return launch_demote(pool, src, dst, n, bt, tags, entry, (cudaStream_t)stream);
+    if (entry && (!bt || !tags || table_entries < 1)) return MKV_E_INVALID;
+    return launch_demote(pool, src, dst, n, bt, tags, entry, table_entries, (cudaStream_t)stream);
 }
 
 int32_t mkv_promote(mkv_pool* pool, const int32_t* src, const int32_t* dst, int32_t n, int32_t* bt, uint8_t* tags,
-                    const int64_t* entry, void* stream)
+                    const int64_t* entry, int64_t table_entries, void* stream)
 {
     if (!pool || !pool->fp8 || n < 0) return MKV_E_INVALID;
     if (n == 0) return MKV_OK;
     if (!src || !dst) return MKV_E_INVALID;
-    if (entry && (!bt || !tags)) return MKV_E_INVALID;
-    return launch_promote(pool, src, dst, n, bt, tags, entry, (cudaStream_t)stream);
+    if (entry && (!bt || !tags || table_entries < 1)) return MKV_E_INVALID;
+    return launch_promote(pool, src, dst, n, bt, tags, entry, table_entries, (cudaStream_t)stream);
 }
 
-int32_t mkv_set_anchor(mkv_pool* pool, uint8_t* tags, int64_t entry, int32_t flag, void* stream)
+int32_t mkv_set_anchor(mkv_pool* pool, uint8_t* tags, int64_t table_entries, int64_t entry, int32_t flag, void* stream)
 {
-    if (!pool || !pool->fp8 || !tags || entry < 0) return MKV_E_INVALID;
+    if (!pool || !pool->fp8 || !tags || entry < 0 || table_entries < 1) return MKV_E_INVALID;
+    if (entry >= table_entries) return MKV_E_BOUNDS;
     return launch_set_anchor(pool, tags, entry, flag, (cudaStream_t)stream);
 }
 

@@ -167,6 +167,29 @@ def test_out_of_range_ids_are_flagged_not_dereferenced():
     assert pool.status() == M.E_BOUNDS
 
 
+def test_an_entry_index_beyond_the_tables_is_flagged_and_nothing_is_published():
+    d, hkv, n = 128, 2, 3
+    pool = M.Pool(d, hkv, hkv, 2 * n, 2 * n, np.ones(d, np.int8))
+    k = torch.randn((16 * n, hkv, d), device="cuda:0").to(torch.bfloat16)
+    pool.append(k, k, torch.arange(16 * n, dtype=torch.int32, device="cuda:0"))
+    ids = torch.arange(n, dtype=torch.int32, device="cuda:0")
+    buf_bt = torch.full((8 + 16,), -7, dtype=torch.int32, device="cuda:0")       # the tables are the first 8 entries
+    buf_tg = torch.full((8 + 16,), 9, dtype=torch.uint8, device="cuda:0")
+    bt, tags = buf_bt[:8], buf_tg[:8]
+    entry = torch.tensor([2, 8, 10 ** 9], dtype=torch.int64, device="cuda:0")     # one good, two beyond the tables
+    pool.demote(ids, ids, bt, tags, entry)
+    torch.cuda.synchronize()
+    assert pool.status() == M.E_BOUNDS
+    assert buf_bt.cpu().tolist() == [-7, -7, 0] + [-7] * 21 and buf_tg.cpu().tolist() == [9, 9, M.TAG_STALE] + [9] * 21
+    pool.promote(ids, (ids + n).contiguous(), bt, tags, entry)
+    torch.cuda.synchronize()
+    assert pool.status() == M.E_BOUNDS
+    assert buf_bt.cpu().tolist() == [-7, -7, n] + [-7] * 21 and buf_tg.cpu().tolist() == [9, 9, M.TAG_ANCHOR] + [9] * 21
+    with pytest.raises(M.MkvError) as e:
+        pool.set_anchor(tags, 8, True)
+    assert e.value.code == M.E_BOUNDS
+
+
 def test_set_anchor_flips_fp8_tags_and_refuses_stale():
     pool = M.Pool(128, 1, 4, 4, 4, np.ones(128, np.int8))
     tags = torch.tensor([[0, 0, 2, 1]], dtype=torch.uint8, device="cuda:0")

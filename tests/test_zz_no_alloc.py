@@ -26,14 +26,26 @@ def test_static_scratch_entry_matches_the_workspace_entry_twice_in_a_row(cfg):
         spec = W.config(1, seq_lens=(3000, 1500, 4100, 16), recent_tokens=256, anchor_span_tokens=64)
     case = Case(spec, extra_fp8=3, extra_tq3=3)
     case.pool.set_decode_variant(M.DECODE_TENSOR)
+    # set-up call: the first call on a device resolves the scratch array's address (the CUDA runtime may load the
+    # library's image on that occasion); a caller makes it at start-up, before its memory budget is frozen
+    M.decode_attention_static(case.pool, case.q, case.bt, case.tags, case.lens, spec.scale)
+    torch.cuda.synchronize()
     for call in range(2):
         # a different query on the second call: the shared scratch still holds the first call's partials
         q = bf16_tensor(W.query(spec, layer=call))
         lse_ref = torch.empty((spec.batch, spec.n_q_heads), dtype=torch.float32, device="cuda:0")
         lse_got = torch.empty_like(lse_ref)
         ref = case.pool.decode_attention(q, case.bt, case.tags, case.lens, spec.scale, lse=lse_ref)
-        got = M.decode_attention_static(case.pool, q, case.bt, case.tags, case.lens, spec.scale, lse=lse_got)
+        out_got = torch.empty_like(ref)                 # the caller's output buffer exists before the call
         torch.cuda.synchronize()
+        free_before, _ = torch.cuda.mem_get_info()
+        torch_before = torch.cuda.memory_allocated()
+        got = M.decode_attention_static(case.pool, q, case.bt, case.tags, case.lens, spec.scale, out=out_got, lse=lse_got)
+        torch.cuda.synchronize()
+        # the property in the entry point's name: the device has exactly as much free memory as before the call
+        # (the first call on the device resolves the scratch array's address, which allocates nothing either)
+        assert torch.cuda.mem_get_info()[0] == free_before and torch.cuda.memory_allocated() == torch_before
+        assert got.data_ptr() == out_got.data_ptr()
         assert case.pool.status() == M.OK
         ref, got = ref.cpu().numpy().astype(np.float64), got.cpu().numpy().astype(np.float64)
         assert np.isfinite(got).all()
@@ -61,3 +73,13 @@ def test_static_scratch_entry_refuses_sizes_beyond_its_maximum():
         M.decode_attention_static(case.pool, q, bt, tags, lens, spec.scale)
     assert e.value.code == M.E_INVALID
     assert b"MKV_STATIC_MAX_BATCH" in M.lib().mkv_last_cuda_error()
+    # a refusal names its real cause: a table wider than the scan can index, or a pool set to another kernel
+    wide_bt = torch.zeros((1, 65536), dtype=torch.int32, device="cuda:0")
+    wide_tg = torch.zeros((1, 65536), dtype=torch.uint8, device="cuda:0")
+    with pytest.raises(M.MkvError) as e:
+        M.decode_attention_static(case.pool, case.q, wide_bt, wide_tg, case.lens, spec.scale)
+    assert e.value.code == M.E_INVALID and b"65535" in M.lib().mkv_last_cuda_error()
+    case.pool.set_decode_variant(M.DECODE_TMEM)
+    with pytest.raises(M.MkvError) as e:
+        M.decode_attention_static(case.pool, case.q, case.bt, case.tags, case.lens, spec.scale)
+    assert e.value.code == M.E_INVALID and b"tensor-core kernel only" in M.lib().mkv_last_cuda_error()
