@@ -250,15 +250,22 @@ __device__ __forceinline__ void key_lut4(uint32_t sel, uint32_t& r0, uint32_t& r
 // (x & mask) | 0x6400 is the fp16 number 1024 + code * 2^POS; one FMA recovers the code exactly.
 // The per-channel scale and zero are applied in fp32 after the token sum:
 //   sum_t p_t (scale*code_t + zero) = scale * (sum_t p_t code_t) + zero * (sum_t p_t).
-template <int POS>
+// The multiplier of the value unpack is read from the constant bank.  Written as a literal it needs a register
+// (the inline PTX takes register operands) beside the one of the addend, and the scan is short of registers: the
+// compiler then rebuilds literals with a move before every use.  Measured: 2 % of a layer's time; doing the same
+// to the masks of the LOP3s, or writing these operations as plain expressions, made the scan slower.
+// 2^-POS as fp16 pairs (exponent arithmetic on 1.0 = 0x3C00)
+__constant__ uint32_t kValueMul[8] = {0x3C003C00u, 0x38003800u, 0x34003400u, 0x30003000u,
+                                      0x2C002C00u, 0x28002800u, 0x24002400u, 0x20002000u};
+template <int POS, bool CB = false>      // CB: multiplier from the constant bank (it pays in the format-2 scan only)
 __device__ __forceinline__ uint32_t value_code(uint32_t x)
 {
     constexpr uint32_t mask = 0x00070007u << POS;
     const uint32_t u = lop3_and_or(x, mask, 0x64006400u);
-    // 2^-POS and -1024 * 2^-POS as fp16 bit patterns (exponent arithmetic on 1.0 = 0x3C00, -1024 = 0xE400)
+    // 2^-POS and -1024 * 2^-POS as fp16 pairs (exponent arithmetic on 1.0 = 0x3C00, -1024 = 0xE400)
     constexpr uint32_t mul = (0x3C00u - (POS << 10)) * 0x00010001u;
     constexpr uint32_t add = (0xE400u - (POS << 10)) * 0x00010001u;
-    return hfma2_u32(u, mul, add);
+    return hfma2_u32(u, CB ? kValueMul[POS] : mul, add);
 }
 
 __device__ __forceinline__ float2 half2_to_float2(uint32_t x)
@@ -584,7 +591,7 @@ __device__ __forceinline__ void tq3_key_quad(float (&S0)[4], float (&S1)[4], uin
 
 // Output update of the four channel blocks 4j..4j+3 of a Stale page: integer codes through the tensor
 // core, then the fp16 scale and zero of every channel applied to the 16x8 result in fp32.
-template <bool DEFER = false>
+template <bool DEFER = false, bool CB = false>
 __device__ __forceinline__ void tq3_value_quad(float (&o0)[4], float (&o1)[4], float (&o2)[4], float (&o3)[4],
                                                uint32_t W0, uint32_t W1, uint32_t W2, uint32_t meta_quad, const PFrag& pf)
 {
@@ -593,16 +600,16 @@ __device__ __forceinline__ void tq3_value_quad(float (&o0)[4], float (&o1)[4], f
     if constexpr (DEFER) {
         // sum p * code only: the accumulators are in code units until the page is left
         const uint32_t X1 = prmt(W0, W1, 0x6341u), X0 = prmt(W1, W2, 0x6341u), X2 = W2 >> 8;
-        a[0] = value_code<0>(W0); a[1] = value_code<3>(W0); a[2] = value_code<6>(W0); a[3] = value_code<1>(X1);
+        a[0] = value_code<0, CB>(W0); a[1] = value_code<3, CB>(W0); a[2] = value_code<6, CB>(W0); a[3] = value_code<1, CB>(X1);
         mma16816(o0, a, pf.b0, pf.b1);
         mma16816(o0, a, pf.c0, pf.c1);
-        a[0] = value_code<4>(X1); a[1] = value_code<7>(X1); a[2] = value_code<2>(W1); a[3] = value_code<5>(W1);
+        a[0] = value_code<4, CB>(X1); a[1] = value_code<7, CB>(X1); a[2] = value_code<2, CB>(W1); a[3] = value_code<5, CB>(W1);
         mma16816(o1, a, pf.b0, pf.b1);
         mma16816(o1, a, pf.c0, pf.c1);
-        a[0] = value_code<0>(X0); a[1] = value_code<3>(X0); a[2] = value_code<6>(X0); a[3] = value_code<1>(W2);
+        a[0] = value_code<0, CB>(X0); a[1] = value_code<3, CB>(X0); a[2] = value_code<6, CB>(X0); a[3] = value_code<1, CB>(W2);
         mma16816(o2, a, pf.b0, pf.b1);
         mma16816(o2, a, pf.c0, pf.c1);
-        a[0] = value_code<4>(W2); a[1] = value_code<7>(W2); a[2] = value_code<2>(X2); a[3] = value_code<5>(X2);
+        a[0] = value_code<4, CB>(W2); a[1] = value_code<7, CB>(W2); a[2] = value_code<2, CB>(X2); a[3] = value_code<5, CB>(X2);
         mma16816(o3, a, pf.b0, pf.b1);
         mma16816(o3, a, pf.c0, pf.c1);
         return;
@@ -610,17 +617,17 @@ __device__ __forceinline__ void tq3_value_quad(float (&o0)[4], float (&o1)[4], f
     {   // blocks 4j, 4j+1
         const uint4 mt = lds128(meta_quad);
         const uint32_t X1 = prmt(W0, W1, 0x6341u);
-        a[0] = value_code<0>(W0);
-        a[1] = value_code<3>(W0);
-        a[2] = value_code<6>(W0);
-        a[3] = value_code<1>(X1);
+        a[0] = value_code<0, CB>(W0);
+        a[1] = value_code<3, CB>(W0);
+        a[2] = value_code<6, CB>(W0);
+        a[3] = value_code<1, CB>(X1);
         mma16816_zero(t, a, pf.b0, pf.b1);
         mma16816(t, a, pf.c0, pf.c1);
         affine_accumulate(o0, t, mt.x, mt.y, pf.ps0, pf.ps1);
-        a[0] = value_code<4>(X1);
-        a[1] = value_code<7>(X1);
-        a[2] = value_code<2>(W1);
-        a[3] = value_code<5>(W1);
+        a[0] = value_code<4, CB>(X1);
+        a[1] = value_code<7, CB>(X1);
+        a[2] = value_code<2, CB>(W1);
+        a[3] = value_code<5, CB>(W1);
         mma16816_zero(t, a, pf.b0, pf.b1);
         mma16816(t, a, pf.c0, pf.c1);
         affine_accumulate(o1, t, mt.z, mt.w, pf.ps0, pf.ps1);
@@ -628,17 +635,17 @@ __device__ __forceinline__ void tq3_value_quad(float (&o0)[4], float (&o1)[4], f
     {   // blocks 4j+2, 4j+3
         const uint4 mt = lds128(meta_quad + 128);
         const uint32_t X0 = prmt(W1, W2, 0x6341u), X2 = W2 >> 8;
-        a[0] = value_code<0>(X0);
-        a[1] = value_code<3>(X0);
-        a[2] = value_code<6>(X0);
-        a[3] = value_code<1>(W2);
+        a[0] = value_code<0, CB>(X0);
+        a[1] = value_code<3, CB>(X0);
+        a[2] = value_code<6, CB>(X0);
+        a[3] = value_code<1, CB>(W2);
         mma16816_zero(t, a, pf.b0, pf.b1);
         mma16816(t, a, pf.c0, pf.c1);
         affine_accumulate(o2, t, mt.x, mt.y, pf.ps0, pf.ps1);
-        a[0] = value_code<4>(W2);
-        a[1] = value_code<7>(W2);
-        a[2] = value_code<2>(X2);
-        a[3] = value_code<5>(X2);
+        a[0] = value_code<4, CB>(W2);
+        a[1] = value_code<7, CB>(W2);
+        a[2] = value_code<2, CB>(X2);
+        a[3] = value_code<5, CB>(X2);
         mma16816_zero(t, a, pf.b0, pf.b1);
         mma16816(t, a, pf.c0, pf.c1);
         affine_accumulate(o3, t, mt.z, mt.w, pf.ps0, pf.ps1);
@@ -798,7 +805,7 @@ __device__ __forceinline__ void tq3_step(WarpAcc<D / 16>& acc, uint32_t rec_v, c
             else tq3_key_quad(S0, S1, kw[3 * j], kw[3 * j + 1], kw[3 * j + 2], qt_lane + j * 2048);
         }
         if constexpr (DO_V)
-            tq3_value_quad<DEFER>(acc.o[4 * j], acc.o[4 * j + 1], acc.o[4 * j + 2], acc.o[4 * j + 3], vw[3 * j], vw[3 * j + 1],
+            tq3_value_quad<DEFER, FMT == 2>(acc.o[4 * j], acc.o[4 * j + 1], acc.o[4 * j + 2], acc.o[4 * j + 3], vw[3 * j], vw[3 * j + 1],
                                   vw[3 * j + 2], meta + j * 256, pf);
     }
     if constexpr (DO_K && FMT == 2) {
