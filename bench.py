@@ -320,8 +320,8 @@ def run_ours(args):
                 tags_host[b, lp] = W.TAG_STALE
 
     # The library's batched calls take all layers of the step in one launch each (append, decode); they serve
-    # 16-token pages and the tensor-core kernel.  Other variants and page sizes go layer by layer.
-    batched = (not args.per_layer) and args.variant == "tensor" and spec.page_tokens == 16 and len(layers) <= M.MAX_LAYERS_PER_CALL
+    # the tensor-core kernel.  Other variants go layer by layer.
+    batched = (not args.per_layer) and args.variant == "tensor" and len(layers) <= M.MAX_LAYERS_PER_CALL
     pools = [L.pool for L in layers]
     layers_per_decode_launch = len(layers) if batched else 1
 

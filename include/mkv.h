@@ -37,9 +37,10 @@
  *   TQ3 record format 2 (mkv_pool_config.tq3_format = 2; Section 3.1 fixes neither codebook nor layout):
  *     the four key magnitudes are the e4m3 numbers nearest to the Lloyd-Max levels (0.25, 0.75, 1.375,
  *     2.25; thresholds 0.5, 1.0625, 1.8125; about 1 % more Gaussian distortion), and the key section is
- *     cut so that four consecutive dims of a token are the nibbles of one half-word.  The decode scan then
- *     turns four codes into four 8-bit floats with one byte-table lookup and multiplies them as FP8 tensor-
- *     core operands against the rotated query carried as four e4m3 terms.  Value codes, norm corrections,
+ *     cut so that four consecutive dims of a token are the nibbles of one half-word.  All levels are
+ *     eighths of small integers (2, 6, 11, 18), so the decode scan turns four codes into four signed bytes
+ *     with one byte-table lookup and multiplies them in integer tensor-core instructions against the rotated
+ *     query carried as three base-128 digits per head (exact integer sums).  Value codes, norm corrections,
  *     scale/zero, sizes and every other encoder step are those of format 1.  A pool has one format; pages
  *     written under one format must not be read under the other.  MKV_DECODE_TMEM serves format 1 only.
  *   Pages of 16 M tokens (page_size = 16 M) are M tiles of 16 tokens:
@@ -239,15 +240,15 @@ int32_t mkv_decode_attention(mkv_pool* pool, const void* q_dev, const int32_t* b
 /* The decode step of several layers in one launch (Section 4.1 runs the direct FP8/TQ3 path of all
  * full-attention layers of a decode step from one CUDA graph; Section 5, evaluated profiles).  Layer i
  * has its own pool, query, table, tags, outputs and workspace; the requests (seq_lens, B, max_pages,
- * scale) are common to all layers, and all pools have the same geometry (head_dim, heads, 16-token
- * pages).  Every block of the persistent scan walks its share of layer 0, then of layer 1, ... without
+ * scale) are common to all layers, and all pools have the same geometry (head_dim, heads, page_size,
+ * record format).  Every block of the persistent scan walks its share of layer 0, then of layer 1, ... without
  * waiting for the other blocks, so the table walk and query rotation of one layer and the merge of the
  * layer before overlap the page scans of their neighbours; results are those of n_layers calls of
  * mkv_decode_attention (the same kernel code per layer).
  *   layers_host  host array of n_layers entries (copied into the launch; free to reuse on return);
  *                lse_dev may be NULL; every workspace_dev as for mkv_decode_attention, distinct per layer
  *   n_layers     1 .. MKV_MAX_LAYERS_PER_CALL; MKV_E_INVALID beyond, for pools of different geometry,
- *                for pages of more than 16 tokens, or for a pool set to another decode variant */
+ *                page size or record format, or for a pool set to another decode variant */
 #define MKV_MAX_LAYERS_PER_CALL 32
 typedef struct {
     mkv_pool* pool;

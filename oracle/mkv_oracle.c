@@ -251,7 +251,7 @@ double orc_tq3_decode_value(uint8_t code, uint16_t sc, uint16_t zp)
 }
 
 /* ------------------------------------------------------------------------------------------
- * Packed records ("packed codes, scales, and required metadata are stored next to the page").
+ * Packed records (Section 4.1: a Stale page's codes, scales and metadata sit in one record per page).
  * The values (codes, g, scale, zero) are the semantics; the positions below are a wire choice
  * that the paper does not print.  All sections start on 16-byte boundaries.
  *
@@ -281,7 +281,7 @@ double orc_tq3_decode_value(uint8_t code, uint16_t sc, uint16_t zp)
  *    e = 4,5: C bits [4n,4n+1] = mag, A bit 4n+3 = sign
  *    e = 6,7: C bits [4n+2,4n+3] = mag, B bit 4n+3 = sign
  *    (four consecutive dims of one token are the four nibbles of one half-word: a reader turns them
- *    into four 8-bit floats with one byte-table lookup)
+ *    into four 8-bit operands with one byte-table lookup)
  * V code of token t, channel c (both formats):  block cb = c/16, row = c%16.
  *    lane = 4*(row%8) + (t%8)/2 ; register r = (row/8) + 2*(t/8) ; half = t%2
  *    word triple j = cb/4; group = (cb%4)/2; field k = 4*(cb%2) + r; stream bit = 3k + bit

@@ -419,6 +419,8 @@ struct Geo {
     static constexpr int OFF_LAST = OFF_PART + ((int)sizeof(Partition) + 15) / 16 * 16;
     static constexpr int OFF_QS = OFF_LAST + 16;             // record format 2: digit unit of the rotated query, per head
     static constexpr int SMEM = OFF_QS + 32;
+    static_assert(SLOT % 128 == 0 && OFF_QT % 16 == 0 && OFF_QF % 16 == 0 && OFF_BAR % 8 == 0,
+                  "slots are bulk-copy destinations; query fragments are read with 16- and 8-byte loads");
     static_assert(NW >= 4, "a warp builds the query fragments of at most two columns of the 8-wide head group");
     static_assert(NSTAGE >= 2 && NSTAGE % 2 == 0 && NSTAGE <= 16, "an FP8 page takes a pair of slots; one phase bit per slot");
     static_assert(NSTAGE * SLOT >= 8 * D * 4, "ring doubles as the cross-warp reduction buffer");
@@ -1809,10 +1811,6 @@ int32_t launch_decode_tensor_layers(mkv_pool* const* pools, const void* const* q
         set_last_error("mkv_decode_attention_layers: more than 65535 16-token tiles per table row (1,048,560 tokens per request)");
         return MKV_E_INVALID;
     }
-    if (p0->tiles > 1) {
-        set_last_error("mkv_decode_attention_layers: pages of 16 tokens only");
-        return MKV_E_INVALID;
-    }
     LayerSet<kMaxLayers> ls;
     ls.n = n_layers;
     for (int i = 0; i < n_layers; ++i) {
@@ -1821,6 +1819,9 @@ int32_t launch_decode_tensor_layers(mkv_pool* const* pools, const void* const* q
         ls.layer[i] = make_params(pools[i], q[i], bt[i], tags[i], lens, B, max_pages, scale, out[i], lse ? lse[i] : nullptr,
                                   partials, tickets, kMaxCtas, nullptr);
     }
+    if (p0->tiles > 1)                   // pages of several tiles (all pools of the call have the same page size)
+        return p0->d == 128 ? run_tensor<128, 12, 4, 1, false, true, kMaxLayers>(p0, ls, s)
+                            : run_tensor<256, 8, 4, 1, false, true, kMaxLayers>(p0, ls, s);
     return p0->d == 128 ? run_tensor<128, 12, 4, 1, false, false, kMaxLayers>(p0, ls, s)
                         : run_tensor<256, 8, 4, 1, false, false, kMaxLayers>(p0, ls, s);
 }

@@ -354,9 +354,9 @@ int32_t mkv_decode_attention_layers(const mkv_layer_call* L, int32_t n_layers, c
         if (!aligned(c.q_dev, 16) || !aligned(c.out_dev, 16) || !aligned(c.workspace_dev, 256) || !aligned(c.block_table_dev, 4))
             return MKV_E_INVALID;
         const mkv_pool* p0 = L[0].pool;
-        if (c.pool->d != p0->d || c.pool->hkv != p0->hkv || c.pool->hq != p0->hq || c.pool->tiles != 1 ||
+        if (c.pool->d != p0->d || c.pool->hkv != p0->hkv || c.pool->hq != p0->hq || c.pool->tiles != p0->tiles ||
             c.pool->device != p0->device || c.pool->variant != MKV_DECODE_TENSOR || c.pool->fmt != p0->fmt) {
-            set_last_error("mkv_decode_attention_layers: pools of one geometry, record format, 16-token pages, one device and the tensor-core variant");
+            set_last_error("mkv_decode_attention_layers: pools of one geometry, page size, record format, one device and the tensor-core variant");
             return MKV_E_INVALID;
         }
         for (int j = 0; j < i; ++j)

@@ -16,12 +16,16 @@ def _layer_cases(n_layers, spec_fn):
     return [Case(spec_fn(), layer=i, extra_fp8=4) for i in range(n_layers)]
 
 
-@pytest.mark.parametrize("name", ["cfg2", "cfg1", "edge"])
+@pytest.mark.parametrize("name", ["cfg2", "cfg1", "edge", "pages_of_832", "pages_of_48_d128"])
 def test_layers_call_equals_per_layer_calls(name):
     """Section 4.1: the decode step of all layers runs as one unit.  One launch over three pools must give,
     bit for bit, what three calls give (the per-layer arithmetic is the same code), and match the oracle."""
     fn = {"cfg2": lambda: W.config(2, seq_lens=(5008, 4432), recent_tokens=512, n_layers=3),
           "cfg1": lambda: W.config(1, seq_lens=(2048 + 16 * i for i in range(8)), recent_tokens=256, anchor_span_tokens=64),
+          "pages_of_832": lambda: W.config(2, seq_lens=(9 * 832 + 100, 7 * 832), anchor_prefix=832, recent_tokens=900,
+                                           n_layers=3, page_tokens=832),
+          "pages_of_48_d128": lambda: W.config(1, seq_lens=(48 * 21 + 5, 48 * 30, 47, 48 * 9 + 47), anchor_prefix=48,
+                                               recent_tokens=100, anchor_span_tokens=96, page_tokens=48),
           "edge": lambda: W.config(0, seq_lens=(0, 1, 15, 16, 17, 33, 16 * 20 + 9, 300), head_dim=128, n_kv_heads=2, group=4,
                                    anchor_prefix=16, recent_tokens=40, n_outlier=3)}[name]
     cases = _layer_cases(3, fn)
