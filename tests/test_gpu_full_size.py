@@ -106,3 +106,68 @@ def test_long_rows_many_rounds_kernels_agree():
                                            only_b=1, only_h=2)
     G = spec.group
     check_close(a[0][1, 2 * G:3 * G], ref[1, 2 * G:3 * G], "long row, request 1, KV head 2")
+
+
+def _layers_call(cases, lse=True):
+    """The call bench.py times: all layers in one launch (mkv_decode_attention_layers)."""
+    spec = cases[0].spec
+    outs = [torch.full((spec.batch, spec.n_q_heads, spec.head_dim), 7.0, dtype=torch.float32, device="cuda:0") for _ in cases]
+    lses = [torch.full((spec.batch, spec.n_q_heads), 7.0, dtype=torch.float32, device="cuda:0") for _ in cases] if lse else None
+    M.decode_attention_layers([c.pool for c in cases], [c.q for c in cases], [c.bt for c in cases],
+                              [c.tags for c in cases], cases[0].lens, spec.scale, outs, lses)
+    torch.cuda.synchronize()
+    for c in cases:
+        assert c.pool.status() == M.OK
+    return [o.cpu().numpy() for o in outs], ([l.cpu().numpy() for l in lses] if lse else None)
+
+
+def test_config2_record_format2_two_full_layers_in_one_launch_every_output():
+    """The benchmark's default: pools of record format 2, the layers of the step in one launch.  Two full
+    layers of config 2 (different pages, tables' ids and queries per layer), every output of both."""
+    with oracle.record_format(2):
+        spec = W.config(2, n_layers=2)
+        cases = [Case(spec, layer=i) for i in range(2)]
+        outs, lses = _layers_call(cases)
+        for i, c in enumerate(cases):
+            ref, ref_lse = c.reference()
+            check_case(c, outs[i], lses[i], ref, ref_lse)
+
+
+def test_config3_one_request_per_length_decile():
+    """Config 3 as specified (64 ragged requests, 1,024 .. 131,072 tokens), record format 2, through the call the
+    benchmark times; the oracle computes the shortest, the longest and one request per decile of the length order
+    (the test above covers record format 1 and the single-layer call on a smaller sample)."""
+    with oracle.record_format(2):
+        spec = W.config(3)
+        order = np.argsort(spec.seq_lens)
+        sample = sorted({int(order[min(63, round(6.3 * k))]) for k in range(11)})
+        assert len(sample) == 11 and int(order[0]) in sample and int(order[-1]) in sample
+        case = Case(spec, requests=sample)
+        (out,), (lse,) = _layers_call([case])
+        assert np.isfinite(out).all()
+        for b in sample:
+            ref, ref_lse = case.reference(only_b=b)
+            check_close(out[b], ref[b], f"config 3 request {b} len {spec.seq_lens[b]}")
+            assert np.abs(lse[b] - ref_lse[b]).max() < 2e-3
+        other = [b for b in range(spec.batch) if b not in sample][0]
+        assert not out[other].any()
+
+
+CORNERS = [(b, c, f) for b in (1, 32) for c in (4096, 131072) for f in (0.0, 0.95)]
+
+
+@pytest.mark.parametrize("batch,ctx,frac", CORNERS)
+def test_config4_corner_cells_at_full_size(batch, ctx, frac):
+    """The eight corners of the config-4 sweep (batch x context x Stale fraction) at their full sizes, record
+    format 2, through the call the benchmark times.  The oracle computes every request of the small cells and
+    two sampled requests of the 32-request cells (the pages of the others are zero records)."""
+    with oracle.record_format(2):
+        spec = W.config(4, batch=batch, ctx=ctx, stale_fraction=frac)
+        sample = list(range(batch)) if batch * ctx <= 262144 else [5, 31] if ctx <= 4096 * 8 else [17]
+        case = Case(spec, requests=sample)
+        (out,), (lse,) = _layers_call([case])
+        assert np.isfinite(out).all()
+        for b in sample:
+            ref, ref_lse = case.reference(only_b=b)
+            check_close(out[b], ref[b], f"{spec.name} request {b}")
+            assert np.abs(lse[b] - ref_lse[b]).max() < 2e-3
