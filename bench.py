@@ -567,7 +567,9 @@ def run_lifecycle(args):
     Tp, Mt = spec.page_tokens, spec.tiles_per_page
     fp8_page, tq3_page = Mt * 32 * d * hkv, (Mt * (12 * d + 32) + 4 * d) * hkv
     P = max(1024 // Mt, (384 << 20) // fp8_page)         # FP8 pages converted per call: 384 MB, 3 x L2
-    pool = M.Pool(d, hkv, hq, 2 * P + 8, P + 8, W.rotation_signs(spec, 0), max_batch=1, device=device, page_tokens=Tp)
+    fmt = 2 if args.format == "v2" else 1
+    pool = M.Pool(d, hkv, hq, 2 * P + 8, P + 8, W.rotation_signs(spec, 0), max_batch=1, device=device, page_tokens=Tp,
+                  tq3_format=fmt)
     gen = torch.Generator(device=device)
     gen.manual_seed(spec.seed)
     T = Tp * P
@@ -616,6 +618,7 @@ def run_lifecycle(args):
     print(json.dumps({
         "mode": "lifecycle", "data": "synthetic", "n_gpus": 1,
         "config": {"workload": "Append / Demote / Promote alone, head geometry of " + workload_name(spec),
+                   "tq3_record_format": fmt,
                    "head_dim": d, "kv_heads": hkv, "page_tokens": Tp, "pages_per_call": P, "tokens_per_append_call": T,
                    "fp8_page_bytes": fp8_page, "tq3_page_bytes": tq3_page, "repetitions": reps,
                    "l2": "every call moves more than 3 x L2"},
@@ -875,7 +878,7 @@ def main():
                     help="override the page size (a multiple of 16; 1792 and 832 are the paper's block sizes)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--format", default="v2", choices=["v1", "v2"],
-                    help="TQ3 record format of the pools (v2: e4m3-exact key codebook, FP8 key products)")
+                    help="TQ3 record format of the pools (v2: key codebook of exact small integers, integer key products)")
     ap.add_argument("--per-layer", action="store_true",
                     help="issue mkv_append / mkv_decode_attention layer by layer instead of the batched calls")
     ap.add_argument("--sweep", action="store_true",

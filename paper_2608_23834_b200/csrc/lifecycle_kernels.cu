@@ -312,7 +312,7 @@ template <int D, int FMT>
 struct DemoteLane {
     float c0sq, c1sq, c2sq, c3sq;     // squared levels (single fp32 products, as the record's norm correction defines them)
     uint32_t flip[D / 32];            // rotation signs of this lane's key elements, as fp32 sign-bit masks
-    uint32_t neg[5];                  // butterfly stage m: lanes with bit m set subtract
+    float sgn[5];                     // butterfly stage m: lanes with bit m set subtract (-1.0f), the others add (+1.0f)
     __device__ __forceinline__ void init(const SigmaBits& sigma, int lane)
     {
         using CB = KeyCodebook<FMT>;
@@ -326,7 +326,7 @@ struct DemoteLane {
             flip[r] = ((sigma.w[i >> 5] >> (i & 31)) & 1u) << 31;
         }
 #pragma unroll
-        for (int b = 0; b < 5; ++b) neg[b] = ((lane >> b) & 1u) << 31;
+        for (int b = 0; b < 5; ++b) sgn[b] = ((lane >> b) & 1) ? -1.0f : 1.0f;
     }
 };
 
@@ -343,7 +343,7 @@ __device__ __forceinline__ void demote_tile(const uint8_t* __restrict__ rec8, ui
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const float c0sq = K.c0sq, c1sq = K.c1sq, c2sq = K.c2sq, c3sq = K.c3sq;
     const uint32_t (&flip)[EPL] = K.flip;
-    const uint32_t (&neg)[5] = K.neg;
+    const float (&sgn)[5] = K.sgn;
     // ---- keys: warp w encodes tokens w, w + NT/32, ... ------------------------------------------
     for (int tok = warp; tok < kPage; tok += NT / 32) {
         float x[EPL], a[EPL];
@@ -358,11 +358,15 @@ __device__ __forceinline__ void demote_tile(const uint8_t* __restrict__ rec8, ui
 #pragma unroll
         for (int r = 0; r < EPL; r += 2) {
             const float2 f = e4m3x2_to_f32((raw[r >> 2] >> (8 * (r & 3))) & 0xFFFFu);
-            x[r] = __fmul_rn(f.x, k_scale);
-            x[r + 1] = __fmul_rn(f.y, k_scale);
-            a[r] = __uint_as_float(__float_as_uint(x[r]) ^ flip[r]);
-            a[r + 1] = __uint_as_float(__float_as_uint(x[r + 1]) ^ flip[r + 1]);
+            x[r] = f.x;
+            x[r + 1] = f.y;
         }
+        if (k_scale != 1.0f) {           // a product with 1 is the factor itself: the common case skips it
+#pragma unroll
+            for (int r = 0; r < EPL; ++r) x[r] = __fmul_rn(x[r], k_scale);
+        }
+#pragma unroll
+        for (int r = 0; r < EPL; ++r) a[r] = __uint_as_float(__float_as_uint(x[r]) ^ flip[r]);
         // Walsh-Hadamard butterflies, strides ascending: inside the lane, then across lanes
 #pragma unroll
         for (int hh = 1; hh < EPL; hh <<= 1)
@@ -377,9 +381,10 @@ __device__ __forceinline__ void demote_tile(const uint8_t* __restrict__ rec8, ui
         for (int b = 0; b < 5; ++b)
 #pragma unroll
             for (int r = 0; r < EPL; ++r) {
-                // lower lane: a + o; upper lane: o - a (the same single addition either way)
+                // lower lane: o + a; upper lane: o - a.  The product with +-1 is exact, so the fused form rounds
+                // once, exactly like the single addition it stands for (zero signs included)
                 const float o = __shfl_xor_sync(0xffffffffu, a[r], 1 << b);
-                a[r] = __fadd_rn(o, __uint_as_float(__float_as_uint(a[r]) ^ neg[b]));
+                a[r] = __fmaf_rn(a[r], sgn[b], o);
             }
         // |x|^2: pairwise tree in index order (every element of the butterfly ends equal)
         float e[EPL];
@@ -396,28 +401,47 @@ __device__ __forceinline__ void demote_tile(const uint8_t* __restrict__ rec8, ui
         const float t1 = __fmul_rn(CB::B0, nx), t2 = __fmul_rn(CB::B1, nx), t3 = __fmul_rn(CB::B2, nx);
         float f[EPL];
         uint32_t packed[EPL / 4];
+        uint32_t sq64 = 4u * EPL;          // record format 2: 64 x the sum of this lane's squared levels (4, 36, 121, 324)
 #pragma unroll
         for (int r = 0; r < EPL / 4; ++r) packed[r] = 0;
 #pragma unroll
         for (int r = 0; r < EPL; ++r) {
             const float w = fabsf(a[r]);
             const bool g1 = w > t1, g2 = w > t2, g3 = w > t3;
-            const uint32_t code = (uint32_t)g1 + (uint32_t)g2 + (uint32_t)g3 + ((__float_as_uint(a[r]) >> 29) & 4u);
-            // a[r] < 0 is the sign bit except for -0, which cannot meet a threshold test either way
-            packed[r >> 2] |= (a[r] == 0.0f ? (code & 3u) : code) << (8 * (r & 3));
-            f[r] = g2 ? (g3 ? c3sq : c2sq) : (g1 ? c1sq : c0sq);
+            // sign bit of the code: a[r] < 0 (a zero of either sign is positive)
+            uint32_t code = a[r] < 0.0f ? 4u : 0u;
+            if (g1) code += 1u;
+            if (g2) code += 1u;
+            if (g3) code += 1u;
+            packed[r >> 2] |= code << (8 * (r & 3));
+            if constexpr (FMT == 2) {
+                if (g1) sq64 += 32u;
+                if (g2) sq64 += 85u;
+                if (g3) sq64 += 203u;
+            } else {
+                f[r] = g2 ? (g3 ? c3sq : c2sq) : (g1 ? c1sq : c0sq);
+            }
         }
         if constexpr (EPL == 8)
             *reinterpret_cast<uint2*>(kcode + tok * KROW + lane * EPL) = make_uint2(packed[0], packed[1]);
         else
             *reinterpret_cast<uint32_t*>(kcode + tok * KROW + lane * EPL) = packed[0];
+        float nc2;
+        if constexpr (FMT == 2) {
+            // The squared levels of format 2 are multiples of 1/64 and d of them sum to at most 5.0625 d, so every
+            // partial sum of the pairwise tree is exact in fp32: any order gives the same bits, and the sum can be
+            // taken in integers (one warp reduction) instead.
+            static_assert(324 * D < (1 << 24), "exact in fp32");
+            nc2 = __fmul_rn((float)__reduce_add_sync(0xffffffffu, sq64), 0.015625f);
+        } else {
 #pragma unroll
-        for (int hh = 1; hh < EPL; hh <<= 1)
+            for (int hh = 1; hh < EPL; hh <<= 1)
 #pragma unroll
-            for (int r = 0; r < EPL; r += 2 * hh) f[r] = __fadd_rn(f[r], f[r + hh]);
-        float nc2 = f[0];
+                for (int r = 0; r < EPL; r += 2 * hh) f[r] = __fadd_rn(f[r], f[r + hh]);
+            nc2 = f[0];
 #pragma unroll
-        for (int m = 1; m < 32; m <<= 1) nc2 = __fadd_rn(nc2, __shfl_xor_sync(0xffffffffu, nc2, m));
+            for (int m = 1; m < 32; m <<= 1) nc2 = __fadd_rn(nc2, __shfl_xor_sync(0xffffffffu, nc2, m));
+        }
         const float nc = __fsqrt_rn(nc2);
         if (lane == 0)
             *reinterpret_cast<uint16_t*>(img + 12 * D + 2 * tok) =
@@ -432,17 +456,32 @@ __device__ __forceinline__ void demote_tile(const uint8_t* __restrict__ rec8, ui
 #pragma unroll
         for (int t = 0; t < kPage; t += 2) {
             const float2 f = e4m3x2_to_f32((rw[t >> 2] >> (8 * (t & 3))) & 0xFFFFu);
-            val[t] = __fmul_rn(f.x, v_scale);
-            val[t + 1] = __fmul_rn(f.y, v_scale);
+            val[t] = f.x;
+            val[t + 1] = f.y;
+        }
+        if (v_scale != 1.0f) {
+#pragma unroll
+            for (int t = 0; t < kPage; ++t) val[t] = __fmul_rn(val[t], v_scale);
         }
         // scale and zero of the channel: from this tile's 16 tokens (16-token pages), or the page's (given)
         uint16_t sc = sc_page, zp = zp_page;
         if constexpr (OWN_META) {
+            // minimum and maximum by strict comparison in token order.  The min/max instructions give the same
+            // value except for the sign of a zero extreme and a leading NaN; those cases take the literal loop
             float mn = val[0], mx = val[0];
 #pragma unroll
             for (int t = 1; t < kPage; ++t) {
-                if (val[t] < mn) mn = val[t];
-                if (val[t] > mx) mx = val[t];
+                mn = fminf(mn, val[t]);
+                mx = fmaxf(mx, val[t]);
+            }
+            if (!(mn != 0.0f && mx != 0.0f) || val[0] != val[0]) {
+                mn = val[0];
+                mx = val[0];
+#pragma unroll
+                for (int t = 1; t < kPage; ++t) {
+                    if (val[t] < mn) mn = val[t];
+                    if (val[t] > mx) mx = val[t];
+                }
             }
             sc = f32_to_f16_sat_bits(__fdiv_rn(__fsub_rn(mx, mn), 7.0f));
             zp = f32_to_f16_sat_bits(mn);
@@ -455,19 +494,37 @@ __device__ __forceinline__ void demote_tile(const uint8_t* __restrict__ rec8, ui
             meta[hi] = sc;
             meta[hi + 2] = zp;
         }
-        // q = clamp(rint((val - zp) / sc), 0, 7), 0 when sc == 0.  The division is the correctly
-        // rounded one; a zero numerator (the channel's minimum) or a zero scale is replaced by
-        // operands whose quotient is not used, which keeps the divider on its short path.
+        // q = clamp(rint((val - zp) / sc), 0, 7), 0 when sc == 0, the division correctly rounded.
+        // The correctly rounded quotient d = RN(num / sc) without the divider: with y = RN(1 / sc) (one correctly
+        // rounded reciprocal per channel), q0 = RN(num y) is within 1.5 ulp of the quotient, one residual step
+        // q1 = RN(q0 + (num - sc q0) y) makes it faithful, and for a faithful q1 the second step gives exactly d
+        // (Markstein's theorem; the residuals are exact in an FMA).  No intermediate can overflow or underflow when
+        // the value scale is between 2^-20 and 2^20 (numerators are 0 or at least 2^-52 and below 2^30, scales are
+        // fp16 numbers); other scales take the divider.  A zero scale gives y = 0 and code 0, a zero numerator code 0,
+        // a NaN input code 0, all as the quotient form does.
         const float den = scf != 0.0f ? scf : 1.0f;
         uint32_t q4[4] = {0u, 0u, 0u, 0u};
+        if (v_scale >= 9.5367431640625e-07f && v_scale <= 1048576.0f) {
+            const float y = scf != 0.0f ? __frcp_rn(scf) : 0.0f;
 #pragma unroll
-        for (int t = 0; t < kPage; ++t) {
-            const float num = __fsub_rn(val[t], zpf);
-            float r = rintf(__fdiv_rn(num != 0.0f ? num : den, den));   // half to even
-            r = r < 0.0f ? 0.0f : r;
-            r = r > 7.0f ? 7.0f : r;
-            const uint32_t q = (num != 0.0f && scf != 0.0f) ? (uint32_t)(int)r : 0u;
-            q4[t >> 2] |= q << (8 * (t & 3));
+            for (int t = 0; t < kPage; ++t) {
+                const float num = __fsub_rn(val[t], zpf);
+                const float q0 = __fmul_rn(num, y);
+                const float q1 = __fmaf_rn(__fmaf_rn(-den, q0, num), y, q0);
+                const float d = __fmaf_rn(__fmaf_rn(-den, q1, num), y, q1);
+                const float r = fminf(fmaxf(rintf(d), 0.0f), 7.0f);          // half to even; NaN -> 0
+                q4[t >> 2] |= (uint32_t)(int)r << (8 * (t & 3));
+            }
+        } else {
+#pragma unroll
+            for (int t = 0; t < kPage; ++t) {
+                const float num = __fsub_rn(val[t], zpf);
+                float r = rintf(__fdiv_rn(num != 0.0f ? num : den, den));   // half to even
+                r = r < 0.0f ? 0.0f : r;
+                r = r > 7.0f ? 7.0f : r;
+                const uint32_t q = (num != 0.0f && scf != 0.0f) ? (uint32_t)(int)r : 0u;
+                q4[t >> 2] |= q << (8 * (t & 3));
+            }
         }
         *reinterpret_cast<uint4*>(vcode + c * kPage) = make_uint4(q4[0], q4[1], q4[2], q4[3]);
     }
@@ -794,9 +851,10 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
         const int i = lane * EPL + r;
         flip[r] = ((sigma.w[i >> 5] >> (i & 31)) & 1u) << 31;
     }
-    uint32_t neg[5];
+    float sgn[5];                           // butterfly stage b: lanes with bit b set subtract
 #pragma unroll
-    for (int b = 0; b < 5; ++b) neg[b] = ((lane >> b) & 1u) << 31;
+    for (int b = 0; b < 5; ++b) sgn[b] = ((lane >> b) & 1) ? -1.0f : 1.0f;
+    const bool unit_k = inv_k_scale == 1.0f, unit_v = inv_v_scale == 1.0f;   // a product with 1 is skipped
     // ---- per-thread constants of the value path: this thread rebuilds channel tid
     const int cb = tid >> 4, row = tid & 15;
     const int vj = cb >> 2, grp = (cb & 3) >> 1, k0 = 4 * (cb & 1) + (row >> 3);
@@ -875,8 +933,9 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
             for (int b = 0; b < 5; ++b)
 #pragma unroll
                 for (int r = 0; r < EPL; ++r) {
+                    // o + y or o - y: the product with +-1 is exact, one rounding as in the single addition
                     const float o = __shfl_xor_sync(0xffffffffu, y[r], 1 << b);
-                    y[r] = __fadd_rn(o, __uint_as_float(__float_as_uint(y[r]) ^ neg[b]));
+                    y[r] = __fmaf_rn(y[r], sgn[b], o);
                 }
             const float g = __half2float(reinterpret_cast<const __half*>(img + 12 * D)[tok]);
             const float gr = __fmul_rn(g, rs);
@@ -886,8 +945,12 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
 #pragma unroll
             for (int r = 0; r < EPL; r += 2) {
                 float2 kk;
-                kk.x = __fmul_rn(__uint_as_float(__float_as_uint(__fmul_rn(gr, y[r])) ^ flip[r]), inv_k_scale);
-                kk.y = __fmul_rn(__uint_as_float(__float_as_uint(__fmul_rn(gr, y[r + 1])) ^ flip[r + 1]), inv_k_scale);
+                kk.x = __uint_as_float(__float_as_uint(__fmul_rn(gr, y[r])) ^ flip[r]);
+                kk.y = __uint_as_float(__float_as_uint(__fmul_rn(gr, y[r + 1])) ^ flip[r + 1]);
+                if (!unit_k) {
+                    kk.x = __fmul_rn(kk.x, inv_k_scale);
+                    kk.y = __fmul_rn(kk.y, inv_k_scale);
+                }
                 out[r >> 2] |= (uint32_t)__nv_cvt_float2_to_fp8x2(kk, __NV_SATFINITE, __NV_E4M3) << (8 * (r & 3));
             }
             if constexpr (EPL == 8)
@@ -915,8 +978,12 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
 #pragma unroll
             for (int t = 0; t < kPage; t += 2) {
                 float2 vv;
-                vv.x = __fmul_rn(__fadd_rn(__fmul_rn(sc, (float)code[t]), zp), inv_v_scale);
-                vv.y = __fmul_rn(__fadd_rn(__fmul_rn(sc, (float)code[t + 1]), zp), inv_v_scale);
+                vv.x = __fadd_rn(__fmul_rn(sc, (float)code[t]), zp);
+                vv.y = __fadd_rn(__fmul_rn(sc, (float)code[t + 1]), zp);
+                if (!unit_v) {
+                    vv.x = __fmul_rn(vv.x, inv_v_scale);
+                    vv.y = __fmul_rn(vv.y, inv_v_scale);
+                }
                 out[t >> 2] |= (uint32_t)__nv_cvt_float2_to_fp8x2(vv, __NV_SATFINITE, __NV_E4M3) << (8 * (t & 3));
             }
             *reinterpret_cast<uint4*>(rec8 + 16 * D + tid * kPage) = make_uint4(out[0], out[1], out[2], out[3]);

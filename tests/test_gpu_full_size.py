@@ -160,10 +160,10 @@ CORNERS = [(b, c, f) for b in (1, 32) for c in (4096, 131072) for f in (0.0, 0.9
 def test_config4_corner_cells_at_full_size(batch, ctx, frac):
     """The eight corners of the config-4 sweep (batch x context x Stale fraction) at their full sizes, record
     format 2, through the call the benchmark times.  The oracle computes every request of the small cells and
-    two sampled requests of the 32-request cells (the pages of the others are zero records)."""
+    two sampled requests of the large 32-request cells (the pages of the others are zero records)."""
     with oracle.record_format(2):
         spec = W.config(4, batch=batch, ctx=ctx, stale_fraction=frac)
-        sample = list(range(batch)) if batch * ctx <= 262144 else [5, 31] if ctx <= 4096 * 8 else [17]
+        sample = list(range(batch)) if batch * ctx <= 262144 else [5, 31] if ctx <= 4096 * 8 else [3, 17]
         case = Case(spec, requests=sample)
         (out,), (lse,) = _layers_call([case])
         assert np.isfinite(out).all()
