@@ -155,6 +155,37 @@ def test_demote_is_bit_exact_and_publishes_after_the_copy(d, hkv, k_scale, v_sca
     assert (btc[1::2] == -1).all() and (tc[1::2] == 0).all() and btc[8] == -1 and tc[8] == 0
 
 
+@pytest.mark.parametrize("fmt", [1, 2])
+@pytest.mark.parametrize("d,hkv,k_scale,v_scale", [(256, 2, 1.0, 1.0), (128, 3, 1.0, 0.37), (256, 1, 3.0, 3.0),
+                                                    (128, 2, 2.0 ** -24, 2.0 ** -24), (128, 2, 1.0e7, 1.0e7)])
+def test_demote_of_arbitrary_byte_patterns_is_bit_exact(d, hkv, k_scale, v_scale, fmt):
+    """FP8 records filled with random bytes (every finite e4m3 value, subnormals, both zeros, +-448): value
+    channels whose range is 7 * 2^k or 7 * 3 * 2^k put many quotients exactly on a half-integer, large and tiny
+    values in one channel stress the quotient's rounding, and scales outside 2^-20 .. 2^20 take the encoder's
+    other division path.  The record bytes must equal the oracle's in every case."""
+    with oracle.record_format(fmt):
+        rng = np.random.default_rng(7 * d + hkv + fmt)
+        n = 12
+        sigma = (rng.integers(0, 2, d) * 2 - 1).astype(np.int8)
+        pool = M.Pool(d, hkv, hkv, n, n, sigma, k_scale, v_scale, tq3_format=fmt)
+        recs = rng.integers(0, 256, (n, hkv, 32 * d), dtype=np.uint8)
+        recs[(recs & 0x7F) == 0x7F] = 0x38                       # no NaN bytes
+        # a few pages with small magnitudes only (|x| < 2: ranges on the e4m3 grid, many exact ties)
+        small = recs[:4]
+        small &= 0xBF
+        for p in range(n):
+            pool.page_write_raw(M.FMT_FP8, p, recs[p])
+        ids = torch.arange(n, dtype=torch.int32, device="cuda:0")
+        pool.demote(ids, ids)
+        torch.cuda.synchronize()
+        assert pool.status() == M.OK
+        for p in range(n):
+            got = pool.page_read_raw(M.FMT_TQ3, p).reshape(hkv, 16 * d + 32)
+            for h in range(hkv):
+                ref = oracle.demote_record(recs[p, h], d, sigma, k_scale, v_scale)
+                assert np.array_equal(got[h], ref), (p, h, np.nonzero(got[h] != ref)[0][:8])
+
+
 def test_out_of_range_ids_are_flagged_not_dereferenced():
     d, hkv = 128, 1
     pool = M.Pool(d, hkv, 4, 4, 4, np.ones(d, np.int8))
