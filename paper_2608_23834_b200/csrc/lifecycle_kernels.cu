@@ -905,8 +905,11 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
                     else if (e < 4) nib = (Bw >> sh) & 0x7777u;
                     else if (e < 6) nib = ((Cw >> sh) & 0x3333u) | ((A >> (sh + 1)) & 0x4444u);
                     else nib = ((Cw >> (sh + 2)) & 0x3333u) | ((Bw >> (sh + 1)) & 0x4444u);
+                    // one byte-table lookup for the four codes: 8 x the signed level (2, 6, 11, 18 | negated).  The
+                    // transform below is exact on these integers, so the factor 1/8 moves into the token's scale
+                    const uint32_t lv = __byte_perm(0x120B0602u, 0xEEF5FAFEu, nib);
 #pragma unroll
-                    for (int x = 0; x < 4; ++x) y[4 * gi + x] = level[(nib >> (4 * x)) & 7u];
+                    for (int x = 0; x < 4; ++x) y[4 * gi + x] = (float)(int)(int8_t)(lv >> (8 * x));
                 }
             }
 #pragma unroll
@@ -938,7 +941,9 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
                     y[r] = __fmaf_rn(y[r], sgn[b], o);
                 }
             const float g = __half2float(reinterpret_cast<const __half*>(img + 12 * D)[tok]);
-            const float gr = __fmul_rn(g, rs);
+            // format 2: y holds 8 x the transform of the levels (all sums of the transform are exact integers below
+            // 2^13, so H(8 c) = 8 H(c) bit for bit) and gr y = (gr / 8)(8 y) is the same real product, rounded once
+            const float gr = FMT == 2 ? __fmul_rn(__fmul_rn(g, rs), 0.125f) : __fmul_rn(g, rs);
             uint32_t out[EPL / 4];
 #pragma unroll
             for (int r = 0; r < EPL / 4; ++r) out[r] = 0;
