@@ -52,8 +52,11 @@
  *     Block-table rows have one entry per page; slot_mapping = page * page_size + position.  With M > 1
  *     mkv_decode_attention() and mkv_decode_attention_scored() run the tensor-core kernel or, if
  *     selected, the CUDA-core kernel (MKV_DECODE_TMEM is refused with MKV_E_INVALID); the page mass is per page of 16 M
- *     tokens; mkv_demote() and mkv_promote() take three resp. two launches (page scale/zero, tiles,
- *     publication).
+ *     tokens; mkv_demote() takes two launches (page scale/zero, then the tiles) and mkv_promote() one when the call
+ *     converts at most 48 pages -- the table entries are then published from inside the tile kernel by the last
+ *     group of blocks to finish a page, counted in 48 ticket words of the pool's status tail -- and one more
+ *     launch (publication) for larger calls.  Two publishing calls on ONE pool must not overlap on the GPU
+ *     (issue them on one stream or order them with events): they would share the ticket words.
  */
 #ifndef MKV_H_
 #define MKV_H_

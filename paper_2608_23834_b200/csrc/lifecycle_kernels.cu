@@ -307,6 +307,21 @@ __device__ __forceinline__ uint32_t squeeze4(uint32_t x)
     return (x & 0xFu) | ((x >> 4) & 0xF0u) | ((x >> 8) & 0xF00u) | ((x >> 12) & 0xF000u);
 }
 
+// Pages of several tiles are converted by gridDim.y clusters per page (rows of tiles).  When the call publishes
+// from inside the kernel, every cluster draws a ticket of its page once all its tiles are written and fenced
+// (called by thread 0 of the cluster's first block after the cluster barrier); the cluster that draws the last
+// one publishes and leaves the counter at zero.  Nobody waits.  Without tickets (16-token pages: one cluster
+// per page) every caller is the last.
+__device__ __forceinline__ bool last_cluster_of_page(uint32_t* page_tickets, int page)
+{
+    if (page_tickets == nullptr) return true;
+    const uint32_t prev = atomicAdd(page_tickets + page, 1u);
+    if (prev != gridDim.y - 1) return false;
+    __threadfence();                    // the other clusters' tiles are ordered before what this thread writes next
+    page_tickets[page] = 0u;
+    return true;
+}
+
 // Constants of the key encoder that depend only on the lane (FMT: the record format's codebook).
 template <int D, int FMT>
 struct DemoteLane {
@@ -597,7 +612,7 @@ __global__ void __launch_bounds__(D) demote_kernel(const uint8_t* __restrict__ f
                                                       const int32_t* __restrict__ src_ids,
                                                       const int32_t* __restrict__ dst_ids, int32_t* block_table,
                                                       uint8_t* tier_tag, const int64_t* entry_index, int64_t n_entries,
-                                                      uint32_t* __restrict__ status)
+                                                      uint32_t* __restrict__ status, uint32_t* page_tickets)
 {
     constexpr int KROW = D + 8;          // padded row of the key-code tile
     constexpr int REC = 16 * D + 32;     // bytes of one TQ3 record
@@ -645,7 +660,7 @@ __global__ void __launch_bounds__(D) demote_kernel(const uint8_t* __restrict__ f
     // copy-before-publish: every head's record is complete and visible before the id and tag appear
     __threadfence();
     cluster_barrier();
-    if (valid && crank == 0 && tid == 0 && entry_index != nullptr) {
+    if (valid && crank == 0 && tid == 0 && entry_index != nullptr && last_cluster_of_page(page_tickets, page)) {
         const int64_t e = entry_index[page];
         if (e >= n_entries) atomicOr(status, kStBounds);      // an entry beyond the tables: flagged, nothing published
         else if (e >= 0) {
@@ -656,64 +671,93 @@ __global__ void __launch_bounds__(D) demote_kernel(const uint8_t* __restrict__ f
     }
 }
 
-// Pages of several tiles, first pass of Demote: thread c finds the minimum and maximum of value channel c
-// over all tokens of the page and writes the page's scale and zero (same arithmetic and order of the
-// halves as in the 16-token record).  One block per (page, KV head).
-template <int D>
-__global__ void __launch_bounds__(1024) demote_minmax_kernel(const uint8_t* __restrict__ fp8, uint8_t* __restrict__ tq3,
-                                                              int fp8_pages, int tq3_pages, int hkv, int tiles,
-                                                              float v_scale, const int32_t* __restrict__ src_ids,
-                                                              const int32_t* __restrict__ dst_ids)
+// Pages of several tiles, first pass of Demote: the minimum and maximum of every value channel over all tokens
+// of the page, then the page's scale and zero (same arithmetic and order of the halves as in the 16-token
+// record).  One cluster per (page, KV head); block r of the cluster scans tiles r, r + cluster size, ... with one
+// thread per channel, the partial extremes meet in the first block through distributed shared memory.
+// The extremes are defined by a scan in token order with strict comparisons; min/max instructions give the same
+// value except for the sign of a zero extreme and a leading NaN, and those channels (rare) are scanned again
+// literally, by the thread that writes the result.
+__device__ __forceinline__ float ld_cluster_f32(const float* local, uint32_t rank)
 {
-    constexpr int R = 1024 / D;                 // tile groups: thread (c, r) scans tiles r, r + R, ...
-    // The minimum and maximum are those a scan in token order with strict comparisons finds: of equal values
-    // (+0 and -0) the earliest token counts, so every candidate carries its token index.
-    __shared__ float mn_s[R][D], mx_s[R][D];
-    __shared__ int mni_s[R][D], mxi_s[R][D];
-    const int page = blockIdx.x / hkv, h = blockIdx.x % hkv, c = threadIdx.x % D, r = threadIdx.x / D;
+    uint32_t remote;
+    float v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"((uint32_t)__cvta_generic_to_shared(local)), "r"(rank));
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
+    return v;
+}
+
+template <int D>
+__global__ void __launch_bounds__(D) demote_minmax_kernel(const uint8_t* __restrict__ fp8, uint8_t* __restrict__ tq3,
+                                                           int fp8_pages, int tq3_pages, int hkv, int tiles,
+                                                           float v_scale, const int32_t* __restrict__ src_ids,
+                                                           const int32_t* __restrict__ dst_ids)
+{
+    __shared__ float part[2][D];
+    const int csize = (int)cluster_size(), crank = (int)cluster_rank();
+    const int unit = blockIdx.x / csize, page = unit / hkv, h = unit % hkv, c = threadIdx.x;
     const int src = src_ids[page], dst = dst_ids[page];
-    if (src < 0 || src >= fp8_pages || dst < 0 || dst >= tq3_pages) return;      // flagged by demote_kernel
-    const uint8_t* page8 = fp8 + ((size_t)src * hkv + h) * fp8_page_bytes(D, tiles);
-    // every group starts from the page's first token, so that an empty group (fewer tiles than groups) is neutral
-    float mn, mx;
-    int mni = 0, mxi = 0;
-    {
-        const uint32_t first = *reinterpret_cast<const uint32_t*>(page8 + 16 * D + c * kPage);
-        mn = mx = __fmul_rn(e4m3x2_to_f32(first & 0xFFFFu).x, v_scale);
-    }
-    for (int m = r; m < tiles; m += R) {
-        const uint4 raw = *reinterpret_cast<const uint4*>(page8 + (size_t)m * fp8_record_bytes(D) + 16 * D + c * kPage);
-        const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
+    const bool valid = src >= 0 && src < fp8_pages && dst >= 0 && dst < tq3_pages;      // flagged by demote_kernel
+    const uint8_t* page8 = fp8 + ((size_t)(valid ? src : 0) * hkv + h) * fp8_page_bytes(D, tiles);
+    auto value = [&](uint32_t two, int half) {
+        const float2 f = e4m3x2_to_f32(two & 0xFFFFu);
+        return __fmul_rn(half ? f.y : f.x, v_scale);
+    };
+    // every block starts from the page's first token, so that a block without tiles is neutral
+    const float first = valid ? value(*reinterpret_cast<const uint32_t*>(page8 + 16 * D + c * kPage), 0) : 0.f;
+    float mn = first, mx = first;
+    constexpr int AHEAD = 4;        // tiles whose loads are issued together (a thread's tiles are 4 KB apart)
+    for (int m0 = crank; valid && m0 < tiles; m0 += AHEAD * csize) {
+        uint4 raw[AHEAD];
 #pragma unroll
-        for (int t = 0; t < kPage; t += 2) {
-            const float2 f = e4m3x2_to_f32((rw[t >> 2] >> (8 * (t & 3))) & 0xFFFFu);
-            const float a = __fmul_rn(f.x, v_scale), b = __fmul_rn(f.y, v_scale);
-            const int ia = m * kPage + t;
-            if (a < mn) { mn = a; mni = ia; }
-            if (a > mx) { mx = a; mxi = ia; }
-            if (b < mn) { mn = b; mni = ia + 1; }
-            if (b > mx) { mx = b; mxi = ia + 1; }
+        for (int u = 0; u < AHEAD; ++u) {
+            const int m = m0 + u * csize;
+            raw[u] = m < tiles ? *reinterpret_cast<const uint4*>(page8 + (size_t)m * fp8_record_bytes(D) + 16 * D + c * kPage)
+                               : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int u = 0; u < AHEAD; ++u) {
+            if (m0 + u * csize >= tiles) break;
+            const uint32_t rw[4] = {raw[u].x, raw[u].y, raw[u].z, raw[u].w};
+#pragma unroll
+            for (int t = 0; t < kPage; t += 2) {
+                const uint32_t two = rw[t >> 2] >> (8 * (t & 3));
+                const float a = value(two, 0), b = value(two, 1);
+                mn = fminf(mn, fminf(a, b));
+                mx = fmaxf(mx, fmaxf(a, b));
+            }
         }
     }
-    mn_s[r][c] = mn;
-    mx_s[r][c] = mx;
-    mni_s[r][c] = mni;
-    mxi_s[r][c] = mxi;
-    __syncthreads();
-    if (r != 0) return;
+    part[0][c] = mn;
+    part[1][c] = mx;
+    cluster_barrier();
+    if (crank == 0 && valid) {
+        for (int k = 1; k < csize; ++k) {
+            mn = fminf(mn, ld_cluster_f32(&part[0][c], (uint32_t)k));
+            mx = fmaxf(mx, ld_cluster_f32(&part[1][c], (uint32_t)k));
+        }
+        if (!(mn != 0.0f && mx != 0.0f) || first != first) {
+            // the literal scan: of equal values (+0 and -0) the earliest token counts
+            mn = mx = first;
+            for (int m = 0; m < tiles; ++m) {
+                const uint4 raw = *reinterpret_cast<const uint4*>(page8 + (size_t)m * fp8_record_bytes(D) + 16 * D + c * kPage);
+                const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-    for (int k = 1; k < R; ++k) {
-        const float a = mn_s[k][c], b = mx_s[k][c];
-        const int ia = mni_s[k][c], ib = mxi_s[k][c];
-        if (a < mn || (a == mn && ia < mni)) { mn = a; mni = ia; }
-        if (b > mx || (b == mx && ib < mxi)) { mx = b; mxi = ib; }
+                for (int t = 0; t < kPage; ++t) {
+                    const float a = value(rw[t >> 2] >> (8 * (t & 2)), t & 1);
+                    if (a < mn) mn = a;
+                    if (a > mx) mx = a;
+                }
+            }
+        }
+        uint16_t* meta = reinterpret_cast<uint16_t*>(tq3 + ((size_t)dst * hkv + h) * tq3_page_bytes(D, tiles) +
+                                                     (size_t)tiles * (12 * D + 32));
+        const int cb = c >> 4, row = c & 15;
+        const int hi = (cb >> 1) * 64 + (row & 7) * 8 + 4 * (cb & 1) + (row >> 3);
+        meta[hi] = f32_to_f16_sat_bits(__fdiv_rn(__fsub_rn(mx, mn), 7.0f));
+        meta[hi + 2] = f32_to_f16_sat_bits(mn);
     }
-    uint16_t* meta = reinterpret_cast<uint16_t*>(tq3 + ((size_t)dst * hkv + h) * tq3_page_bytes(D, tiles) +
-                                                 (size_t)tiles * (12 * D + 32));
-    const int cb = c >> 4, row = c & 15;
-    const int hi = (cb >> 1) * 64 + (row & 7) * 8 + 4 * (cb & 1) + (row >> 3);
-    meta[hi] = f32_to_f16_sat_bits(__fdiv_rn(__fsub_rn(mx, mn), 7.0f));
-    meta[hi + 2] = f32_to_f16_sat_bits(mn);
+    cluster_barrier();              // the partial extremes stay readable until the first block has taken them
 }
 
 // Pages of several tiles, last pass of Demote / Promote: the kernels before it in the stream have written the
@@ -734,6 +778,12 @@ __global__ void publish_kernel(int n, const int32_t* __restrict__ src_ids, const
         tier_tag[e] = (uint8_t)tag;
     }
 }
+
+// Page tickets of the in-kernel publication: 48 counters in the pool's 256-byte status tail (word 0 is the status
+// word, words 16..63 the tickets; the tail is zeroed with the arenas and every use leaves its counter at zero).
+// Calls that convert more pages publish with a kernel of their own.
+constexpr int kPageTickets = 48;
+static uint32_t* page_tickets(mkv_pool* p) { return p->status_dev + 16; }
 
 // grid rows of the tile-parallel passes: at least 16, and enough to fill the GPU when few pages are converted
 static int tile_rows(int tiles, int n_pages, int hkv)
@@ -769,18 +819,25 @@ static int32_t launch_demote_d(mkv_pool* p, const int32_t* src, const int32_t* d
     if (p->tiles == 1) {
         MKV_CUDA(launch_clustered(demote_kernel<D, false, FMT>, n, c, D, s, (const uint8_t*)p->fp8, p->tq3, p->cfg.fp8_pages,
                                   p->cfg.tq3_pages, p->hkv, 1, p->cfg.k_scale, p->cfg.v_scale, p->sigma, src, dst, bt,
-                                  tags, entry, n_entries, p->status_dev));
+                                  tags, entry, n_entries, p->status_dev, (uint32_t*)nullptr));
         return MKV_OK;
     }
-    // pages of several tiles: scale/zero of the page, then the tiles in parallel, then the publication
-    demote_minmax_kernel<D><<<n * p->hkv, 1024, 0, s>>>(p->fp8, p->tq3, p->cfg.fp8_pages, p->cfg.tq3_pages, p->hkv, p->tiles,
-                                                     p->cfg.v_scale, src, dst);
-    MKV_CUDA(cudaGetLastError());
+    // pages of several tiles: scale/zero of the page, then the tiles in parallel, then the publication (from inside
+    // the tile kernel when the call is small enough for the pool's page tickets, else as a kernel of its own)
+    const bool fused = entry != nullptr && n <= kPageTickets;
+    {
+        // blocks per (page, head): up to a portable cluster of 8, fewer when the call fills the GPU anyway
+        int cs = 8;
+        while (cs > 1 && (cs > p->tiles || (long long)n * p->hkv * cs > 8LL * 148)) cs >>= 1;
+        MKV_CUDA(launch_clustered(demote_minmax_kernel<D>, n * p->hkv, cs, D, s, (const uint8_t*)p->fp8, p->tq3, p->cfg.fp8_pages,
+                                  p->cfg.tq3_pages, p->hkv, p->tiles, p->cfg.v_scale, src, dst));
+    }
     MKV_CUDA(launch_clustered_rows(demote_kernel<D, true, FMT>, n, heads_cluster(p->hkv, 0), tile_rows(p->tiles, n, p->hkv), D, s,
                                    (const uint8_t*)p->fp8, p->tq3, p->cfg.fp8_pages, p->cfg.tq3_pages, p->hkv, p->tiles,
-                                   p->cfg.k_scale, p->cfg.v_scale, p->sigma, src, dst, (int32_t*)nullptr,
-                                   (uint8_t*)nullptr, (const int64_t*)nullptr, (int64_t)0, p->status_dev));
-    if (entry) {
+                                   p->cfg.k_scale, p->cfg.v_scale, p->sigma, src, dst, fused ? bt : (int32_t*)nullptr,
+                                   fused ? tags : (uint8_t*)nullptr, fused ? entry : (const int64_t*)nullptr,
+                                   fused ? n_entries : (int64_t)0, p->status_dev, fused ? page_tickets(p) : (uint32_t*)nullptr));
+    if (entry && !fused) {
         publish_kernel<<<(n + 127) / 128, 128, 0, s>>>(n, src, dst, p->cfg.fp8_pages, p->cfg.tq3_pages, bt, tags, entry,
                                                        n_entries, MKV_TAG_STALE, p->status_dev);
         MKV_CUDA(cudaGetLastError());
@@ -817,7 +874,7 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
                                                      const int32_t* __restrict__ src_ids,
                                                      const int32_t* __restrict__ dst_ids, int32_t* block_table,
                                                      uint8_t* tier_tag, const int64_t* entry_index, int64_t n_entries,
-                                                     uint32_t* __restrict__ status)
+                                                     uint32_t* __restrict__ status, uint32_t* page_tickets)
 {
     constexpr int EPL = D / 32;
     constexpr int NT = D;
@@ -997,7 +1054,7 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
     // copy-before-publish
     __threadfence();
     cluster_barrier();
-    if (valid && crank == 0 && tid == 0 && entry_index != nullptr) {
+    if (valid && crank == 0 && tid == 0 && entry_index != nullptr && last_cluster_of_page(page_tickets, page)) {
         const int64_t e = entry_index[page];
         if (e >= n_entries) atomicOr(status, kStBounds);
         else if (e >= 0) {
@@ -1017,14 +1074,16 @@ static int32_t launch_promote_d(mkv_pool* p, const int32_t* src, const int32_t* 
     if (p->tiles == 1) {
         MKV_CUDA(launch_clustered(promote_kernel<D, false, FMT>, n, heads_cluster(p->hkv, n), D, s, (const uint8_t*)p->tq3, p->fp8,
                                   p->cfg.tq3_pages, p->cfg.fp8_pages, p->hkv, 1, ik, iv, rs, p->sigma, src, dst, bt, tags,
-                                  entry, n_entries, p->status_dev));
+                                  entry, n_entries, p->status_dev, (uint32_t*)nullptr));
         return MKV_OK;
     }
+    const bool fused = entry != nullptr && n <= kPageTickets;
     MKV_CUDA(launch_clustered_rows(promote_kernel<D, true, FMT>, n, heads_cluster(p->hkv, 0), tile_rows(p->tiles, n, p->hkv), D, s,
                                    (const uint8_t*)p->tq3, p->fp8, p->cfg.tq3_pages, p->cfg.fp8_pages, p->hkv, p->tiles, ik,
-                                   iv, rs, p->sigma, src, dst, (int32_t*)nullptr, (uint8_t*)nullptr,
-                                   (const int64_t*)nullptr, (int64_t)0, p->status_dev));
-    if (entry) {
+                                   iv, rs, p->sigma, src, dst, fused ? bt : (int32_t*)nullptr, fused ? tags : (uint8_t*)nullptr,
+                                   fused ? entry : (const int64_t*)nullptr, fused ? n_entries : (int64_t)0, p->status_dev,
+                                   fused ? page_tickets(p) : (uint32_t*)nullptr));
+    if (entry && !fused) {
         publish_kernel<<<(n + 127) / 128, 128, 0, s>>>(n, src, dst, p->cfg.tq3_pages, p->cfg.fp8_pages, bt, tags, entry,
                                                        n_entries, MKV_TAG_ANCHOR, p->status_dev);
         MKV_CUDA(cudaGetLastError());

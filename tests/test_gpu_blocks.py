@@ -178,3 +178,54 @@ def test_random_page_sizes_lengths_and_tier_mixes(seed):
                             case.tab.tier_tag, case.tab.seq_lens, spec.scale, page_tokens=page_tokens)
     got = mass.cpu().numpy().astype(np.float64)
     assert (np.abs(got - want) <= 1e-6 + 1e-4 * want).all(), np.abs(got - want).max()
+
+
+def test_publication_of_big_pages_in_small_and_large_calls():
+    """Pages of several tiles are written by many blocks; the table entry of a page may appear only after all of
+    them.  Small calls publish from inside the tile kernel (the cluster that draws the page's last ticket), large
+    calls with a kernel of their own.  Both must publish every page exactly as asked, the ticket counters must be
+    back at zero (a second small call works), and the records must be the oracle's."""
+    d, hkv, page_tokens = 128, 2, 48
+    Mt = page_tokens // 16
+    rng = np.random.default_rng(11)
+    n_big, n_small = 60, 5
+    n_pages = n_big + 2 * n_small
+    sigma = (rng.integers(0, 2, d) * 2 - 1).astype(np.int8)
+    pool = M.Pool(d, hkv, hkv, n_pages, n_pages, sigma, page_tokens=page_tokens)
+    k_bits, v_bits = _kv_bits(rng, n_pages * page_tokens, hkv, d)
+    slots = torch.arange(n_pages * page_tokens, dtype=torch.int32, device="cuda:0")
+    pool.append(bf16_tensor(k_bits), bf16_tensor(v_bits), slots)
+    kf, vf = oracle.bf16_bits_to_f32(k_bits), oracle.bf16_bits_to_f32(v_bits)
+    bt = torch.full((1, n_pages), -1, dtype=torch.int32, device="cuda:0")
+    tags = torch.zeros((1, n_pages), dtype=torch.uint8, device="cuda:0")
+    calls = [(0, n_big), (n_big, n_big + n_small), (n_big + n_small, n_pages)]      # large, small, small again
+    for lo, hi in calls:
+        ids = torch.arange(lo, hi, dtype=torch.int32, device="cuda:0")
+        dst = torch.arange(hi - 1, lo - 1, -1, dtype=torch.int32, device="cuda:0")     # reversed inside the call
+        entry = torch.arange(lo, hi, dtype=torch.int64, device="cuda:0")
+        if hi - lo == n_small:
+            entry[2] = -1                                                              # encoded, not published
+        pool.demote(ids, dst, bt, tags, entry)
+        torch.cuda.synchronize()
+        assert pool.status() == M.OK
+        btc, tc = bt.cpu().numpy()[0], tags.cpu().numpy()[0]
+        for i in range(lo, hi):
+            if hi - lo == n_small and i == lo + 2:
+                assert btc[i] == -1 and tc[i] == 0
+            else:
+                assert btc[i] == lo + hi - 1 - i and tc[i] == M.TAG_STALE, (lo, hi, i)
+    for page in (3, n_big + 1, n_pages - 1):
+        lo, hi = next(c for c in calls if c[0] <= page < c[1])
+        got = pool.page_read_raw(M.FMT_TQ3, lo + hi - 1 - page).reshape(hkv, -1)
+        for h in range(hkv):
+            fp8 = oracle.fp8_pack_block(kf[page * page_tokens:(page + 1) * page_tokens, h],
+                                        vf[page * page_tokens:(page + 1) * page_tokens, h])
+            assert np.array_equal(got[h], oracle.demote_block(fp8, d, Mt, sigma)), (page, h)
+    # and back: a large and a small Promote call
+    for lo, hi in ((0, n_big), (n_big, n_big + n_small)):
+        src = torch.arange(hi - 1, lo - 1, -1, dtype=torch.int32, device="cuda:0")
+        dst = torch.arange(lo, hi, dtype=torch.int32, device="cuda:0")
+        pool.promote(src, dst, bt, tags, torch.arange(lo, hi, dtype=torch.int64, device="cuda:0"))
+        torch.cuda.synchronize()
+        assert pool.status() == M.OK
+        assert (bt.cpu().numpy()[0, lo:hi] == np.arange(lo, hi)).all() and (tags.cpu().numpy()[0, lo:hi] == M.TAG_ANCHOR).all()
