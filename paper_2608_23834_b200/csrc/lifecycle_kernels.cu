@@ -291,6 +291,13 @@ static cudaError_t launch_clustered(Kernel kernel, int n_pages, int csize, int t
 // the packers, which read rows g and g + 8), value codes [channel][16 tokens], and two record images
 // (alternating per head, so that the copy-out of one head overlaps the encoding of the next).
 
+// 16 bytes global -> shared, asynchronously (both addresses 16-byte aligned); completion by cp.async.wait_all
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src)
+                 : "memory");
+}
+
 // two e4m3 bytes (low byte first) -> two fp32
 __device__ __forceinline__ float2 e4m3x2_to_f32(uint32_t two_bytes)
 {
@@ -867,6 +874,130 @@ int32_t launch_demote(mkv_pool* p, const int32_t* src, const int32_t* dst, int n
 // L = 4 (row % 8) + (slot % 8) / 2 holds, in nibble 2 rr + slot % 2 with rr = row / 8 + 2 (slot / 8),
 // the entry (row, slot) of every 16 x 16 block; for keys row = token and slot = channel % 16, for
 // values row = channel % 16 and slot = token.
+// D = A B + C with 8-bit integers: A 16 x 32 (row-major fragments), B 32 x 8 (column-major), C 16 x 8 in int32
+__device__ __forceinline__ void imma16832(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// Keys of one record of format 2 back to e4m3 rows (Promote), the inverse rotation as a matrix product.
+// The levels of format 2 are eighths of the integers +-2, +-6, +-11, +-18, so the transform H c of a token's d
+// levels consists of sums of integers below 2^13: every order of summation gives the same value, and the
+// butterflies can be replaced by the product C[16 tokens x d] H[d x d] in 8-bit integer tensor-core
+// instructions (exact int32 sums).  The record's key section already is the A operand: lane 4 (t % 8) + (k % 16) / 4
+// holds, per 32-dim step, the codes of tokens g, g + 8 at dims 4 tq .. + 3 and 16 + 4 tq .. + 3, and one
+// byte-table lookup turns four codes into four signed bytes.  H[k][n] = (-1)^popcount(k & n) needs no table: for
+// lane (g, tq), column n = 8 j + g and rows k = 32 s + 16 b + 4 tq + i its sign is the product of a per-lane
+// pattern over i, a per-warp part and a part that is known at compile time.
+// Warp w computes the column tiles j = w, w + D/32, ... (eight columns each); results go to `ktile`
+// [16 tokens][D] e4m3 in shared memory.  All D threads call it; the caller synchronises before reading ktile.
+// What promote_keys_v2 needs per lane and warp, computed once per block.
+template <int D>
+struct PromoteKeyLane {
+    uint32_t b0p, b1p, b0n, b1n;          // B fragments of H for this lane: both K halves, plain and negated
+    uint32_t odd_flip;                    // 0x44444444 in warps that see the odd steps negated (sign bit of every code), else 0
+    uint32_t flip[D / 8 / (D / 32)][2];   // rotation signs of the lane's two columns of every tile, as fp32 sign bits
+    __device__ __forceinline__ void init(const SigmaBits& sigma, int warp, int lane)
+    {
+        constexpr uint32_t NEG = 0xFEFEFEFEu;             // x ^ NEG negates bytes +-1
+        constexpr int NWARP = D / 32, NTILE = D / 8 / NWARP;
+        const int g = lane >> 2, tq = lane & 3;
+        // (-1)^popcount(k & n), k = 32 s + 16 b + 4 tq + i, n = 8 j + g, j = NWARP t + warp:
+        //   bits 0-1: i & g -> the byte pattern W over i;  bit 2: tq0 & g2;  bit 3: tq1 & j0 (j0 = warp & 1);
+        //   bit 4: b & j1 (j1 = (warp >> 1) & 1);  bits 5-7: s & (j >> 2), of which bit 0 of j >> 2 is warp >> 2 for
+        //   D = 256 (it negates the odd steps: done on the codes) and the rest is the tile index (compile time)
+        const uint32_t W = (g & 3) == 0 ? 0x01010101u : (g & 3) == 1 ? 0xFF01FF01u : (g & 3) == 2 ? 0xFFFF0101u : 0x01FFFF01u;
+        const bool lane_odd = (((tq & 1) & (g >> 2)) ^ ((tq >> 1) & (warp & 1))) != 0;
+        b0p = lane_odd ? (W ^ NEG) : W;
+        b1p = ((warp >> 1) & 1) ? (b0p ^ NEG) : b0p;
+        b0n = b0p ^ NEG;
+        b1n = b1p ^ NEG;
+        odd_flip = ((warp >> 2) & 1) ? 0x44444444u : 0u;
+#pragma unroll
+        for (int t = 0; t < NTILE; ++t) {
+            const int n0 = 8 * (NWARP * t + warp) + 2 * tq;
+            const uint32_t sg = (sigma.w[n0 >> 5] >> (n0 & 31)) & 3u;
+            flip[t][0] = (sg & 1u) << 31;
+            flip[t][1] = (sg & 2u) << 30;
+        }
+    }
+};
+
+// Keys of one record of format 2 back to e4m3 rows (Promote), the inverse rotation as a matrix product.
+// The levels of format 2 are eighths of the integers +-2, +-6, +-11, +-18, so the transform H c of a token's d
+// levels consists of sums of integers below 2^13: every order of summation gives the same value, and the
+// butterflies can be replaced by the product C[16 tokens x d] H[d x d] in 8-bit integer tensor-core
+// instructions (exact int32 sums).  The record's key section already is the A operand: lane 4 (t % 8) + (k % 16) / 4
+// holds, per 32-dim step, the codes of tokens g, g + 8 at dims 4 tq .. + 3 and 16 + 4 tq .. + 3, and one
+// byte-table lookup turns four codes into four signed bytes.  H[k][n] = (-1)^popcount(k & n) needs no table
+// (PromoteKeyLane).  Warp w computes the column tiles j = w, w + D/32, ... (eight columns each); results go to
+// `ktile` [16 tokens][D] e4m3 in shared memory.  All D threads call it; the caller synchronises before reading ktile.
+template <int D>
+__device__ __forceinline__ void promote_keys_v2(const uint8_t* img, uint8_t* ktile, const PromoteKeyLane<D>& L, float rs,
+                                                float inv_k_scale, bool unit_k)
+{
+    constexpr int NS = D / 32;            // 32-dim steps (K of the product)
+    constexpr int NWARP = D / 32;         // warps of the block
+    constexpr int NTILE = D / 8 / NWARP;  // column tiles per warp (4)
+    constexpr uint32_t T0 = 0x120B0602u, T1 = 0xEEF5FAFEu;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tq = lane & 3;
+    // ---- A: the record's codes as signed bytes, 4 registers per step
+    uint32_t a[NS][4];
+#pragma unroll
+    for (int j = 0; j < NS / 2; ++j) {
+        const uint32_t A = *reinterpret_cast<const uint32_t*>(img + lane_word_offset(D, lane, 3 * j));
+        const uint32_t Bw = *reinterpret_cast<const uint32_t*>(img + lane_word_offset(D, lane, 3 * j + 1));
+        const uint32_t Cw = *reinterpret_cast<const uint32_t*>(img + lane_word_offset(D, lane, 3 * j + 2));
+        const uint32_t s0 = A & 0x77777777u, s1 = Bw & 0x77777777u;
+        const uint32_t s2 = (((A >> 1) & 0x44444444u) | (Cw & 0x33333333u)) ^ L.odd_flip;
+        const uint32_t s3 = (((Bw >> 1) & 0x44444444u) | ((Cw >> 2) & 0x33333333u)) ^ L.odd_flip;
+        a[2 * j][0] = __byte_perm(T0, T1, s0);            // token g, dims 4 tq ..
+        a[2 * j][2] = __byte_perm(T0, T1, s0 >> 16);      // token g, dims 16 + 4 tq ..
+        a[2 * j][1] = __byte_perm(T0, T1, s1);            // token g + 8
+        a[2 * j][3] = __byte_perm(T0, T1, s1 >> 16);
+        a[2 * j + 1][0] = __byte_perm(T0, T1, s2);
+        a[2 * j + 1][2] = __byte_perm(T0, T1, s2 >> 16);
+        a[2 * j + 1][1] = __byte_perm(T0, T1, s3);
+        a[2 * j + 1][3] = __byte_perm(T0, T1, s3 >> 16);
+    }
+    // ---- per token scale g r / 8
+    const __half* gh = reinterpret_cast<const __half*>(img + 12 * D);
+    const float gr0 = __fmul_rn(__fmul_rn(__half2float(gh[g]), rs), 0.125f);
+    const float gr1 = __fmul_rn(__fmul_rn(__half2float(gh[g + 8]), rs), 0.125f);
+    float out[NTILE][4];
+#pragma unroll
+    for (int t = 0; t < NTILE; ++t) {
+        constexpr int JH = NWARP / 4;                     // j >> 2 = JH * t + (warp >> 2)
+        int c[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int s_ = 0; s_ < NS; ++s_) {
+            const bool neg = (__popc((unsigned)(s_ & (JH * t) & (NWARP == 8 ? 6 : 7))) & 1) != 0;     // compile-time part of bits 5-7
+            imma16832(c, a[s_][0], a[s_][1], a[s_][2], a[s_][3], neg ? L.b0n : L.b0p, neg ? L.b1n : L.b1p);
+        }
+        // columns n = 8 j + 2 tq, + 1 of tokens g (c0, c1) and g + 8 (c2, c3); j = NWARP t + warp
+        out[t][0] = __uint_as_float(__float_as_uint(__fmul_rn(gr0, (float)c[0])) ^ L.flip[t][0]);
+        out[t][1] = __uint_as_float(__float_as_uint(__fmul_rn(gr0, (float)c[1])) ^ L.flip[t][1]);
+        out[t][2] = __uint_as_float(__float_as_uint(__fmul_rn(gr1, (float)c[2])) ^ L.flip[t][0]);
+        out[t][3] = __uint_as_float(__float_as_uint(__fmul_rn(gr1, (float)c[3])) ^ L.flip[t][1]);
+    }
+    if (!unit_k) {                        // a product with 1 is skipped (a branch, not predicated multiplications)
+#pragma unroll
+        for (int t = 0; t < NTILE; ++t)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) out[t][e] = __fmul_rn(out[t][e], inv_k_scale);
+    }
+#pragma unroll
+    for (int t = 0; t < NTILE; ++t) {
+        const int n0 = 8 * (NWARP * t + warp) + 2 * tq;
+        *reinterpret_cast<uint16_t*>(ktile + g * D + n0) =
+            (uint16_t)__nv_cvt_float2_to_fp8x2(make_float2(out[t][0], out[t][1]), __NV_SATFINITE, __NV_E4M3);
+        *reinterpret_cast<uint16_t*>(ktile + (g + 8) * D + n0) =
+            (uint16_t)__nv_cvt_float2_to_fp8x2(make_float2(out[t][2], out[t][3]), __NV_SATFINITE, __NV_E4M3);
+    }
+}
+
 template <int D, bool BIG, int FMT>
 __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ tq3, uint8_t* __restrict__ fp8,
                                                      int tq3_pages, int fp8_pages, int hkv, int tiles, float inv_k_scale,
@@ -880,6 +1011,7 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
     constexpr int NT = D;
     constexpr int REC = 16 * D + 32;
     __shared__ __align__(16) uint8_t image[2][REC];
+    __shared__ __align__(16) uint8_t ktile[FMT == 2 ? kPage * D : 16];   // format 2: the rebuilt key rows of one record
     __shared__ float level[8];            // signed key levels by 3-bit code
 
     const int csize = (int)cluster_size(), crank = (int)cluster_rank();
@@ -912,6 +1044,8 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
 #pragma unroll
     for (int b = 0; b < 5; ++b) sgn[b] = ((lane >> b) & 1) ? -1.0f : 1.0f;
     const bool unit_k = inv_k_scale == 1.0f, unit_v = inv_v_scale == 1.0f;   // a product with 1 is skipped
+    PromoteKeyLane<D> key_lane;
+    if constexpr (FMT == 2) key_lane.init(sigma, warp, lane);
     // ---- per-thread constants of the value path: this thread rebuilds channel tid
     const int cb = tid >> 4, row = tid & 15;
     const int vj = cb >> 2, grp = (cb & 3) >> 1, k0 = 4 * (cb & 1) + (row >> 3);
@@ -926,26 +1060,39 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
     // y + gridDim.y, ...; a tile and the page's scale/zero behind it form the same image as a 16-token record.
     constexpr int TILE = 12 * D + 32;
     const int m_first = BIG ? (int)blockIdx.y : 0, m_step = BIG ? (int)gridDim.y : 1, m_end = BIG ? tiles : 1;
-    int it = 0;
-    for (int h = crank; valid && h < hkv; h += csize)
-    for (int m = m_first; m < m_end; m += m_step) {
-        const uint8_t* rec3 = tq3 + ((size_t)src * hkv + h) * tq3_page_bytes(D, tiles) + (size_t)m * TILE;
-        uint8_t* rec8 = fp8 + (((size_t)dst * hkv + h) * tiles + m) * fp8_record_bytes(D);
-        uint8_t* img = image[it++ & 1];
+    // The record of the next (head, tile) is copied into the other image asynchronously while this one is rebuilt.
+    auto fetch = [&](int h, int m, uint8_t* img) {
+        const uint8_t* page3 = tq3 + ((size_t)src * hkv + h) * tq3_page_bytes(D, tiles);
+        const uint8_t* rec3 = page3 + (size_t)m * TILE;
         if constexpr (!BIG) {
-            for (int i = tid; i < REC / 16; i += NT)
-                reinterpret_cast<uint4*>(img)[i] = reinterpret_cast<const uint4*>(rec3)[i];
+            for (int i = tid; i < REC / 16; i += NT) cp_async16(img + 16 * i, rec3 + 16 * i);
         } else {
-            const uint8_t* meta = tq3 + ((size_t)src * hkv + h) * tq3_page_bytes(D, tiles) + (size_t)tiles * TILE;
-            for (int i = tid; i < TILE / 16; i += NT)
-                reinterpret_cast<uint4*>(img)[i] = reinterpret_cast<const uint4*>(rec3)[i];
-            for (int i = tid; i < 4 * D / 16; i += NT)
-                reinterpret_cast<uint4*>(img + TILE)[i] = reinterpret_cast<const uint4*>(meta)[i];
+            const uint8_t* meta = page3 + (size_t)tiles * TILE;
+            for (int i = tid; i < TILE / 16; i += NT) cp_async16(img + 16 * i, rec3 + 16 * i);
+            for (int i = tid; i < 4 * D / 16; i += NT) cp_async16(img + TILE + 16 * i, meta + 16 * i);
         }
-        __syncthreads();
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    int h = crank, m = m_first;
+    bool more = valid && h < hkv && m < m_end;
+    if (more) fetch(h, m, image[0]);
+    for (int it = 0; more; ++it) {
+        int hn = h, mn = m + m_step;
+        if (mn >= m_end) {
+            mn = m_first;
+            hn = h + csize;
+        }
+        const bool more_next = hn < hkv;
+        uint8_t* rec8 = fp8 + (((size_t)dst * hkv + h) * tiles + m) * fp8_record_bytes(D);
+        uint8_t* img = image[it & 1];
+        asm volatile("cp.async.wait_all;" ::: "memory");
+        __syncthreads();            // this image has landed for every thread; the other image and ktile are no longer read
+        if (more_next) fetch(hn, mn, image[(it + 1) & 1]);
 
-        // ---- keys: warp w rebuilds tokens w, w + NT/32, ...
-        for (int tok = warp; tok < kPage; tok += NT / 32) {
+        // ---- keys.  Format 2: the inverse rotation as an integer matrix product (all warps, every token at once)
+        if constexpr (FMT == 2) promote_keys_v2<D>(img, ktile, key_lane, rs, inv_k_scale, unit_k);
+        // Format 1: warp w rebuilds tokens w, w + NT/32, ... with butterflies
+        for (int tok = warp; FMT != 2 && tok < kPage; tok += NT / 32) {
             float y[EPL];
             if constexpr (FMT == 2) {
                 // record format 2: four consecutive dims are the nibbles of one half-word of register
@@ -1037,19 +1184,25 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
                 code[2 * q + 9] = (st1 >> 6) & 7u;
             }
             uint32_t out[4] = {0u, 0u, 0u, 0u};
+            float vv[kPage];
 #pragma unroll
-            for (int t = 0; t < kPage; t += 2) {
-                float2 vv;
-                vv.x = __fadd_rn(__fmul_rn(sc, (float)code[t]), zp);
-                vv.y = __fadd_rn(__fmul_rn(sc, (float)code[t + 1]), zp);
-                if (!unit_v) {
-                    vv.x = __fmul_rn(vv.x, inv_v_scale);
-                    vv.y = __fmul_rn(vv.y, inv_v_scale);
-                }
-                out[t >> 2] |= (uint32_t)__nv_cvt_float2_to_fp8x2(vv, __NV_SATFINITE, __NV_E4M3) << (8 * (t & 3));
+            for (int t = 0; t < kPage; ++t) vv[t] = __fadd_rn(__fmul_rn(sc, (float)code[t]), zp);
+            if (!unit_v) {
+#pragma unroll
+                for (int t = 0; t < kPage; ++t) vv[t] = __fmul_rn(vv[t], inv_v_scale);
             }
+#pragma unroll
+            for (int t = 0; t < kPage; t += 2)
+                out[t >> 2] |= (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(vv[t], vv[t + 1]), __NV_SATFINITE, __NV_E4M3) << (8 * (t & 3));
             *reinterpret_cast<uint4*>(rec8 + 16 * D + tid * kPage) = make_uint4(out[0], out[1], out[2], out[3]);
         }
+        if constexpr (FMT == 2) {
+            __syncthreads();               // key rows complete; the next record's rows are written after the next barrier
+            reinterpret_cast<uint4*>(rec8)[tid] = reinterpret_cast<const uint4*>(ktile)[tid];      // 16 D bytes, D threads
+        }
+        h = hn;
+        m = mn;
+        more = more_next;
     }
     // copy-before-publish
     __threadfence();
