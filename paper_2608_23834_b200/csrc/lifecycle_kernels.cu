@@ -664,10 +664,12 @@ __global__ void __launch_bounds__(D) demote_kernel(const uint8_t* __restrict__ f
         }
     }
 
-    // copy-before-publish: every head's record is complete and visible before the id and tag appear
-    __threadfence();
+    // copy-before-publish: every head's record is complete and visible before the id and tag appear.  The cluster
+    // barrier (release / acquire) orders the record stores of every thread of the cluster before what the
+    // publishing thread does next, and that thread's fence is cumulative: it orders them, device-wide, before its
+    // own later stores.  (A fence in every thread would say the same and make each of them wait for its stores.)
     cluster_barrier();
-    if (valid && crank == 0 && tid == 0 && entry_index != nullptr && last_cluster_of_page(page_tickets, page)) {
+    if (valid && crank == 0 && tid == 0 && entry_index != nullptr && (__threadfence(), last_cluster_of_page(page_tickets, page))) {
         const int64_t e = entry_index[page];
         if (e >= n_entries) atomicOr(status, kStBounds);      // an entry beyond the tables: flagged, nothing published
         else if (e >= 0) {
@@ -897,7 +899,7 @@ __device__ __forceinline__ void imma16832(int (&c)[4], uint32_t a0, uint32_t a1,
 template <int D>
 struct PromoteKeyLane {
     uint32_t b0p, b1p, b0n, b1n;          // B fragments of H for this lane: both K halves, plain and negated
-    uint32_t odd_flip;                    // 0x44444444 in warps that see the odd steps negated (sign bit of every code), else 0
+    uint32_t o0p, o1p, o0n, o1n;          // the same for the odd steps (negated in warps whose columns have bit 5 of n set)
     uint32_t flip[D / 8 / (D / 32)][2];   // rotation signs of the lane's two columns of every tile, as fp32 sign bits
     __device__ __forceinline__ void init(const SigmaBits& sigma, int warp, int lane)
     {
@@ -907,14 +909,18 @@ struct PromoteKeyLane {
         // (-1)^popcount(k & n), k = 32 s + 16 b + 4 tq + i, n = 8 j + g, j = NWARP t + warp:
         //   bits 0-1: i & g -> the byte pattern W over i;  bit 2: tq0 & g2;  bit 3: tq1 & j0 (j0 = warp & 1);
         //   bit 4: b & j1 (j1 = (warp >> 1) & 1);  bits 5-7: s & (j >> 2), of which bit 0 of j >> 2 is warp >> 2 for
-        //   D = 256 (it negates the odd steps: done on the codes) and the rest is the tile index (compile time)
+        //   D = 256 (it negates the odd steps) and the rest is the tile index (compile time)
         const uint32_t W = (g & 3) == 0 ? 0x01010101u : (g & 3) == 1 ? 0xFF01FF01u : (g & 3) == 2 ? 0xFFFF0101u : 0x01FFFF01u;
         const bool lane_odd = (((tq & 1) & (g >> 2)) ^ ((tq >> 1) & (warp & 1))) != 0;
         b0p = lane_odd ? (W ^ NEG) : W;
         b1p = ((warp >> 1) & 1) ? (b0p ^ NEG) : b0p;
         b0n = b0p ^ NEG;
         b1n = b1p ^ NEG;
-        odd_flip = ((warp >> 2) & 1) ? 0x44444444u : 0u;
+        const bool w2 = ((warp >> 2) & 1) != 0;
+        o0p = w2 ? b0n : b0p;
+        o1p = w2 ? b1n : b1p;
+        o0n = w2 ? b0p : b0n;
+        o1n = w2 ? b1p : b1n;
 #pragma unroll
         for (int t = 0; t < NTILE; ++t) {
             const int n0 = 8 * (NWARP * t + warp) + 2 * tq;
@@ -935,32 +941,42 @@ struct PromoteKeyLane {
 // (PromoteKeyLane).  Warp w computes the column tiles j = w, w + D/32, ... (eight columns each); results go to
 // `ktile` [16 tokens][D] e4m3 in shared memory.  All D threads call it; the caller synchronises before reading ktile.
 template <int D>
-__device__ __forceinline__ void promote_keys_v2(const uint8_t* img, uint8_t* ktile, const PromoteKeyLane<D>& L, float rs,
-                                                float inv_k_scale, bool unit_k)
+__device__ __forceinline__ void promote_keys_v2(const uint8_t* img, uint8_t* ktile, uint4* afrag, const PromoteKeyLane<D>& L,
+                                                float rs, float inv_k_scale, bool unit_k)
 {
     constexpr int NS = D / 32;            // 32-dim steps (K of the product)
     constexpr int NWARP = D / 32;         // warps of the block
     constexpr int NTILE = D / 8 / NWARP;  // column tiles per warp (4)
     constexpr uint32_t T0 = 0x120B0602u, T1 = 0xEEF5FAFEu;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tq = lane & 3;
-    // ---- A: the record's codes as signed bytes, 4 registers per step
-    uint32_t a[NS][4];
-#pragma unroll
-    for (int j = 0; j < NS / 2; ++j) {
+    // ---- A: the record's codes as signed bytes, 4 registers per step.  Warp s unpacks step s for everybody
+    // (afrag [step][lane] in shared memory), then every warp fetches all steps.
+    {
+        const int j = warp >> 1;
         const uint32_t A = *reinterpret_cast<const uint32_t*>(img + lane_word_offset(D, lane, 3 * j));
         const uint32_t Bw = *reinterpret_cast<const uint32_t*>(img + lane_word_offset(D, lane, 3 * j + 1));
         const uint32_t Cw = *reinterpret_cast<const uint32_t*>(img + lane_word_offset(D, lane, 3 * j + 2));
-        const uint32_t s0 = A & 0x77777777u, s1 = Bw & 0x77777777u;
-        const uint32_t s2 = (((A >> 1) & 0x44444444u) | (Cw & 0x33333333u)) ^ L.odd_flip;
-        const uint32_t s3 = (((Bw >> 1) & 0x44444444u) | ((Cw >> 2) & 0x33333333u)) ^ L.odd_flip;
-        a[2 * j][0] = __byte_perm(T0, T1, s0);            // token g, dims 4 tq ..
-        a[2 * j][2] = __byte_perm(T0, T1, s0 >> 16);      // token g, dims 16 + 4 tq ..
-        a[2 * j][1] = __byte_perm(T0, T1, s1);            // token g + 8
-        a[2 * j][3] = __byte_perm(T0, T1, s1 >> 16);
-        a[2 * j + 1][0] = __byte_perm(T0, T1, s2);
-        a[2 * j + 1][2] = __byte_perm(T0, T1, s2 >> 16);
-        a[2 * j + 1][1] = __byte_perm(T0, T1, s3);
-        a[2 * j + 1][3] = __byte_perm(T0, T1, s3 >> 16);
+        uint32_t s0, s1;
+        if ((warp & 1) == 0) {
+            s0 = A & 0x77777777u;
+            s1 = Bw & 0x77777777u;
+        } else {
+            s0 = ((A >> 1) & 0x44444444u) | (Cw & 0x33333333u);
+            s1 = ((Bw >> 1) & 0x44444444u) | ((Cw >> 2) & 0x33333333u);
+        }
+        uint4 v;
+        v.x = __byte_perm(T0, T1, s0);            // token g, dims 4 tq ..
+        v.z = __byte_perm(T0, T1, s0 >> 16);      // token g, dims 16 + 4 tq ..
+        v.y = __byte_perm(T0, T1, s1);            // token g + 8
+        v.w = __byte_perm(T0, T1, s1 >> 16);
+        afrag[warp * 32 + lane] = v;
+    }
+    __syncthreads();
+    uint32_t a[NS][4];
+#pragma unroll
+    for (int s_ = 0; s_ < NS; ++s_) {
+        const uint4 v = afrag[s_ * 32 + lane];
+        a[s_][0] = v.x; a[s_][1] = v.y; a[s_][2] = v.z; a[s_][3] = v.w;
     }
     // ---- per token scale g r / 8
     const __half* gh = reinterpret_cast<const __half*>(img + 12 * D);
@@ -974,7 +990,8 @@ __device__ __forceinline__ void promote_keys_v2(const uint8_t* img, uint8_t* kti
 #pragma unroll
         for (int s_ = 0; s_ < NS; ++s_) {
             const bool neg = (__popc((unsigned)(s_ & (JH * t) & (NWARP == 8 ? 6 : 7))) & 1) != 0;     // compile-time part of bits 5-7
-            imma16832(c, a[s_][0], a[s_][1], a[s_][2], a[s_][3], neg ? L.b0n : L.b0p, neg ? L.b1n : L.b1p);
+            if (s_ & 1) imma16832(c, a[s_][0], a[s_][1], a[s_][2], a[s_][3], neg ? L.o0n : L.o0p, neg ? L.o1n : L.o1p);
+            else imma16832(c, a[s_][0], a[s_][1], a[s_][2], a[s_][3], neg ? L.b0n : L.b0p, neg ? L.b1n : L.b1p);
         }
         // columns n = 8 j + 2 tq, + 1 of tokens g (c0, c1) and g + 8 (c2, c3); j = NWARP t + warp
         out[t][0] = __uint_as_float(__float_as_uint(__fmul_rn(gr0, (float)c[0])) ^ L.flip[t][0]);
@@ -1012,6 +1029,7 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
     constexpr int REC = 16 * D + 32;
     __shared__ __align__(16) uint8_t image[2][REC];
     __shared__ __align__(16) uint8_t ktile[FMT == 2 ? kPage * D : 16];   // format 2: the rebuilt key rows of one record
+    __shared__ uint4 afrag[FMT == 2 ? D : 1];                            // format 2: [32-dim step][lane] A operands of the key product
     __shared__ float level[8];            // signed key levels by 3-bit code
 
     const int csize = (int)cluster_size(), crank = (int)cluster_rank();
@@ -1090,7 +1108,7 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
         if (more_next) fetch(hn, mn, image[(it + 1) & 1]);
 
         // ---- keys.  Format 2: the inverse rotation as an integer matrix product (all warps, every token at once)
-        if constexpr (FMT == 2) promote_keys_v2<D>(img, ktile, key_lane, rs, inv_k_scale, unit_k);
+        if constexpr (FMT == 2) promote_keys_v2<D>(img, ktile, afrag, key_lane, rs, inv_k_scale, unit_k);
         // Format 1: warp w rebuilds tokens w, w + NT/32, ... with butterflies
         for (int tok = warp; FMT != 2 && tok < kPage; tok += NT / 32) {
             float y[EPL];
@@ -1171,29 +1189,35 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
         {
             const __half* meta = reinterpret_cast<const __half*>(img + 12 * D + 32);
             const float sc = __half2float(meta[meta_i]), zp = __half2float(meta[meta_i + 2]);
-            uint32_t code[kPage];
+            // The channel's eight possible output bytes, e4m3((sc * code + zp) / v_scale) for code 0..7, computed
+            // once; a byte-table lookup then turns the codes of four tokens into four output bytes.
+            float lv[8];
+#pragma unroll
+            for (int cde = 0; cde < 8; ++cde) lv[cde] = __fadd_rn(__fmul_rn(sc, (float)cde), zp);
+            if (!unit_v) {
+#pragma unroll
+                for (int cde = 0; cde < 8; ++cde) lv[cde] = __fmul_rn(lv[cde], inv_v_scale);
+            }
+            uint32_t pr[4];
+#pragma unroll
+            for (int cde = 0; cde < 8; cde += 2)
+                pr[cde >> 1] = (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(lv[cde], lv[cde + 1]), __NV_SATFINITE, __NV_E4M3);
+            const uint32_t lut_lo = pr[0] | (pr[1] << 16), lut_hi = pr[2] | (pr[3] << 16);
+            uint32_t near[4], far[4];           // per q: codes of tokens (2q, 2q+1) and (2q+8, 2q+9) as two nibbles
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 const uint32_t lo = *reinterpret_cast<const uint32_t*>(img + off_v + q * str_v);
                 const uint32_t hi = *reinterpret_cast<const uint32_t*>(img + off_v1 + q * str_v1);
                 const uint32_t st0 = __byte_perm(lo, hi, sel0) >> (3 * k0);          // stream of the even tokens
                 const uint32_t st1 = __byte_perm(lo, hi, sel1) >> (3 * k0);          // stream of the odd tokens
-                code[2 * q] = st0 & 7u;
-                code[2 * q + 1] = st1 & 7u;
-                code[2 * q + 8] = (st0 >> 6) & 7u;
-                code[2 * q + 9] = (st1 >> 6) & 7u;
+                near[q] = (st0 & 7u) | ((st1 & 7u) << 4);
+                far[q] = ((st0 >> 6) & 7u) | (((st1 >> 6) & 7u) << 4);
             }
-            uint32_t out[4] = {0u, 0u, 0u, 0u};
-            float vv[kPage];
-#pragma unroll
-            for (int t = 0; t < kPage; ++t) vv[t] = __fadd_rn(__fmul_rn(sc, (float)code[t]), zp);
-            if (!unit_v) {
-#pragma unroll
-                for (int t = 0; t < kPage; ++t) vv[t] = __fmul_rn(vv[t], inv_v_scale);
-            }
-#pragma unroll
-            for (int t = 0; t < kPage; t += 2)
-                out[t >> 2] |= (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(vv[t], vv[t + 1]), __NV_SATFINITE, __NV_E4M3) << (8 * (t & 3));
+            uint32_t out[4];
+            out[0] = __byte_perm(lut_lo, lut_hi, near[0] | (near[1] << 8));           // tokens 0..3
+            out[1] = __byte_perm(lut_lo, lut_hi, near[2] | (near[3] << 8));           // tokens 4..7
+            out[2] = __byte_perm(lut_lo, lut_hi, far[0] | (far[1] << 8));             // tokens 8..11
+            out[3] = __byte_perm(lut_lo, lut_hi, far[2] | (far[3] << 8));             // tokens 12..15
             *reinterpret_cast<uint4*>(rec8 + 16 * D + tid * kPage) = make_uint4(out[0], out[1], out[2], out[3]);
         }
         if constexpr (FMT == 2) {
@@ -1204,10 +1228,9 @@ __global__ void __launch_bounds__(D) promote_kernel(const uint8_t* __restrict__ 
         m = mn;
         more = more_next;
     }
-    // copy-before-publish
-    __threadfence();
+    // copy-before-publish (as in demote_kernel: cluster barrier, then the publishing thread's cumulative fence)
     cluster_barrier();
-    if (valid && crank == 0 && tid == 0 && entry_index != nullptr && last_cluster_of_page(page_tickets, page)) {
+    if (valid && crank == 0 && tid == 0 && entry_index != nullptr && (__threadfence(), last_cluster_of_page(page_tickets, page))) {
         const int64_t e = entry_index[page];
         if (e >= n_entries) atomicOr(status, kStBounds);
         else if (e >= 0) {
