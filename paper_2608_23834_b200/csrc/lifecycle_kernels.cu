@@ -298,6 +298,38 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src)
                  : "memory");
 }
 
+// Two fp32 values in one 64-bit register and the packed operations on them (add, mul, fma, each half rounded to
+// nearest even exactly like the scalar instruction): half the instructions for element-wise arithmetic.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi)
+{
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b)
+{
+    f32x2 r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b)
+{
+    f32x2 r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c)
+{
+    f32x2 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+
 // two e4m3 bytes (low byte first) -> two fp32
 __device__ __forceinline__ float2 e4m3x2_to_f32(uint32_t two_bytes)
 {
@@ -390,28 +422,48 @@ __device__ __forceinline__ void demote_tile(const uint8_t* __restrict__ rec8, ui
 #pragma unroll
         for (int r = 0; r < EPL; ++r) a[r] = __uint_as_float(__float_as_uint(x[r]) ^ flip[r]);
         // Walsh-Hadamard butterflies, strides ascending: inside the lane, then across lanes
+        // (stride 1 pairs neighbours: scalar; from stride 2 on two butterflies share one packed instruction)
 #pragma unroll
-        for (int hh = 1; hh < EPL; hh <<= 1)
+        for (int r = 0; r < EPL; r += 2) {
+            const float u = a[r], w = a[r + 1];
+            a[r] = __fadd_rn(u, w);
+            a[r + 1] = __fsub_rn(u, w);
+        }
+        f32x2 ap[EPL / 2];
+        const f32x2 minus1 = pack2(-1.0f, -1.0f);
 #pragma unroll
-            for (int r = 0; r < EPL; ++r)
+        for (int r = 0; r < EPL / 2; ++r) ap[r] = pack2(a[2 * r], a[2 * r + 1]);
+#pragma unroll
+        for (int hh = 1; hh < EPL / 2; hh <<= 1)            // strides 2, 4 of the elements = 1, 2 of the pairs
+#pragma unroll
+            for (int r = 0; r < EPL / 2; ++r)
                 if ((r & hh) == 0) {
-                    const float u = a[r], w = a[r + hh];
-                    a[r] = __fadd_rn(u, w);
-                    a[r + hh] = __fsub_rn(u, w);
+                    const f32x2 u = ap[r], w = ap[r + hh];
+                    ap[r] = add2(u, w);
+                    ap[r + hh] = fma2(w, minus1, u);        // u - w: the product with -1 is exact, one rounding
                 }
 #pragma unroll
-        for (int b = 0; b < 5; ++b)
+        for (int b = 0; b < 5; ++b) {
+            const f32x2 s2 = pack2(sgn[b], sgn[b]);
 #pragma unroll
-            for (int r = 0; r < EPL; ++r) {
+            for (int r = 0; r < EPL / 2; ++r) {
                 // lower lane: o + a; upper lane: o - a.  The product with +-1 is exact, so the fused form rounds
                 // once, exactly like the single addition it stands for (zero signs included)
-                const float o = __shfl_xor_sync(0xffffffffu, a[r], 1 << b);
-                a[r] = __fmaf_rn(a[r], sgn[b], o);
+                float lo, hi;
+                unpack2(ap[r], lo, hi);
+                const float olo = __shfl_xor_sync(0xffffffffu, lo, 1 << b), ohi = __shfl_xor_sync(0xffffffffu, hi, 1 << b);
+                ap[r] = fma2(ap[r], s2, pack2(olo, ohi));
             }
+        }
+#pragma unroll
+        for (int r = 0; r < EPL / 2; ++r) unpack2(ap[r], a[2 * r], a[2 * r + 1]);
         // |x|^2: pairwise tree in index order (every element of the butterfly ends equal)
         float e[EPL];
 #pragma unroll
-        for (int r = 0; r < EPL; ++r) e[r] = __fmul_rn(x[r], x[r]);
+        for (int r = 0; r < EPL; r += 2) {
+            const f32x2 xx = pack2(x[r], x[r + 1]);
+            unpack2(mul2(xx, xx), e[r], e[r + 1]);
+        }
 #pragma unroll
         for (int hh = 1; hh < EPL; hh <<= 1)
 #pragma unroll
@@ -528,14 +580,19 @@ __device__ __forceinline__ void demote_tile(const uint8_t* __restrict__ rec8, ui
         uint32_t q4[4] = {0u, 0u, 0u, 0u};
         if (v_scale >= 9.5367431640625e-07f && v_scale <= 1048576.0f) {
             const float y = scf != 0.0f ? __frcp_rn(scf) : 0.0f;
+            // two tokens per instruction: the packed fp32 operations round each half like the scalar ones
+            const f32x2 y2 = pack2(y, y), nden2 = pack2(-den, -den), nzp2 = pack2(-zpf, -zpf);
 #pragma unroll
-            for (int t = 0; t < kPage; ++t) {
-                const float num = __fsub_rn(val[t], zpf);
-                const float q0 = __fmul_rn(num, y);
-                const float q1 = __fmaf_rn(__fmaf_rn(-den, q0, num), y, q0);
-                const float d = __fmaf_rn(__fmaf_rn(-den, q1, num), y, q1);
-                const float r = fminf(fmaxf(rintf(d), 0.0f), 7.0f);          // half to even; NaN -> 0
-                q4[t >> 2] |= (uint32_t)(int)r << (8 * (t & 3));
+            for (int t = 0; t < kPage; t += 2) {
+                const f32x2 num = add2(pack2(val[t], val[t + 1]), nzp2);           // val - zp (= val + (-zp), one rounding)
+                const f32x2 q0 = mul2(num, y2);
+                const f32x2 q1 = fma2(fma2(nden2, q0, num), y2, q0);
+                const f32x2 d2 = fma2(fma2(nden2, q1, num), y2, q1);
+                float d0, d1;
+                unpack2(d2, d0, d1);
+                const float r0 = fminf(fmaxf(rintf(d0), 0.0f), 7.0f);        // half to even; NaN -> 0
+                const float r1 = fminf(fmaxf(rintf(d1), 0.0f), 7.0f);
+                q4[t >> 2] |= ((uint32_t)(int)r0 << (8 * (t & 3))) | ((uint32_t)(int)r1 << (8 * ((t + 1) & 3)));
             }
         } else {
 #pragma unroll
