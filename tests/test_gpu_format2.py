@@ -173,3 +173,25 @@ def test_the_tensor_memory_variant_refuses_format2():
     assert e.value.code == M.E_INVALID and b"format 2" in M.lib().mkv_last_cuda_error()
     with pytest.raises(M.MkvError):
         M.Pool(128, 1, 1, 1, 1, np.ones(128, np.int8), tq3_format=3)
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_queries_with_outlier_dims_a_zero_head_and_mixed_scales(variant):
+    """The tensor-core scan carries the rotated query of format 2 as three base-128 digits per head, scaled to the
+    head's largest component.  Heads whose query is zero, has a few components 20 times the rest, or is small as a
+    whole must come out within the same tolerance."""
+    spec = W.config(2, seq_lens=(3008, 1000), recent_tokens=256, n_layers=1)
+    case = Case(spec, extra_fp8=2, extra_tq3=2)
+    q = oracle.bf16_bits_to_f32(case.L.q_bits).copy()                 # [B][Hq][d]
+    q[:, 0] = 0.0                                                      # a zero head: uniform attention
+    q[:, 1, 7] *= 20.0                                                 # outlier components
+    q[:, 1, 130] *= -20.0
+    q[:, 2] *= 1e-3                                                    # a small head
+    q[:, 3] *= 6.0                                                     # a large head (peaked attention)
+    q[1, 4, :] = q[1, 4, 0]                                            # constant over the dims
+    case.L.q_bits[:] = W.f32_to_bf16_bits(q)
+    from _gpu_util import bf16_tensor
+    case.q = bf16_tensor(case.L.q_bits)
+    out, lse = case.run(variant)
+    ref, ref_lse = case.reference()
+    check_case(case, out, lse, ref, ref_lse)
