@@ -195,3 +195,22 @@ def test_queries_with_outlier_dims_a_zero_head_and_mixed_scales(variant):
     out, lse = case.run(variant)
     ref, ref_lse = case.reference()
     check_case(case, out, lse, ref, ref_lse)
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("k_scale,v_scale", [(0.5, 2.0), (3.0, 0.37)])
+def test_decode_with_fp8_scales_other_than_one(k_scale, v_scale, variant):
+    """Pool-level FP8 scales: a Recent/Anchor byte means e4m3 x scale (the Stale records carry their own norms,
+    scales and zeros and are not rescaled).  The same pages read under other scales must match the oracle reading
+    them under the same scales."""
+    spec = W.config(1, seq_lens=(1500, 700, 16, 333), recent_tokens=400, anchor_span_tokens=64)
+    case = Case(spec, extra_fp8=2, extra_tq3=2, k_scale=k_scale, v_scale=v_scale)
+    out, lse = case.run(variant)
+    s = spec
+    ref, ref_lse = oracle.decode_attention(case.L.fp8_arena, case.L.tq3_arena, s.head_dim, s.n_kv_heads, s.group, case.L.sigma,
+                                           case.L.q_bits, case.tab.block_table, case.tab.tier_tag, case.tab.seq_lens, s.scale,
+                                           k_scale=k_scale, v_scale=v_scale)
+    check_case(case, out, lse, ref, ref_lse)
+    # and the scales matter: the result differs from the one under unit scales
+    ref1, _ = case.reference()
+    assert np.abs(ref - ref1).max() > 1e-2
