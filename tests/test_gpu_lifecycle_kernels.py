@@ -186,6 +186,34 @@ def test_demote_of_arbitrary_byte_patterns_is_bit_exact(d, hkv, k_scale, v_scale
                 assert np.array_equal(got[h], ref), (p, h, np.nonzero(got[h] != ref)[0][:8])
 
 
+@pytest.mark.parametrize("fmt", [1, 2])
+@pytest.mark.parametrize("d,hkv,k_scale,v_scale", [(256, 2, 1.0, 1.0), (128, 3, 1.0, 1.0), (256, 1, 0.5, 4.0), (128, 2, 3.0, 0.37)])
+def test_promote_of_arbitrary_records_is_bit_exact(d, hkv, k_scale, v_scale, fmt):
+    """TQ3 records filled with random bytes: every code pattern in every position, norm corrections, scales and
+    zeros anywhere in the finite fp16 range below 2.  The rebuilt FP8 pages must equal the oracle's byte for byte
+    (format 2 rebuilds the keys by an integer matrix product, format 1 by butterflies)."""
+    with oracle.record_format(fmt):
+        rng = np.random.default_rng(31 * d + hkv + fmt)
+        n = 10
+        sigma = (rng.integers(0, 2, d) * 2 - 1).astype(np.int8)
+        pool = M.Pool(d, hkv, hkv, n, n, sigma, k_scale, v_scale, tq3_format=fmt)
+        recs = rng.integers(0, 256, (n, hkv, 16 * d + 32), dtype=np.uint8)
+        meta = recs[:, :, 12 * d:].view(np.uint16)
+        meta &= 0xBFFF                                        # clear the top exponent bit: finite, |x| < 2
+        recs[0, :, 12 * d:12 * d + 32] = 0                    # a page whose norm corrections are all zero
+        for p in range(n):
+            pool.page_write_raw(M.FMT_TQ3, p, recs[p])
+        ids = torch.arange(n, dtype=torch.int32, device="cuda:0")
+        pool.promote(ids, ids)
+        torch.cuda.synchronize()
+        assert pool.status() == M.OK
+        for p in range(n):
+            got = pool.page_read_raw(M.FMT_FP8, p).reshape(hkv, 32 * d)
+            for h in range(hkv):
+                ref = oracle.promote_record(recs[p, h], d, sigma, k_scale, v_scale)
+                assert np.array_equal(got[h], ref), (p, h, np.nonzero(got[h] != ref)[0][:8])
+
+
 def test_out_of_range_ids_are_flagged_not_dereferenced():
     d, hkv = 128, 1
     pool = M.Pool(d, hkv, 4, 4, 4, np.ones(d, np.int8))
